@@ -1,0 +1,249 @@
+/*
+ * rtp.h - C ABI of the sparse-attention hot path (sm_100a).
+ *
+ * The library implements the inference-time attention mechanism of the paper's
+ * Section 3.2: a 16-dimensional token indexer (Eq. 4), a query-dependent top-p
+ * selection on the softmax mass of the indexer scores (Eq. 5, "Top-P"), exact
+ * attention restricted to the selected tokens on retrieval heads (Eq. 5), and
+ * attention-sink + sliding-window attention on local heads (Section 3.2,
+ * Table 2), plus dense causal attention as the in-library comparator.
+ *
+ * General contract
+ * ----------------
+ * - Every pointer marked DEVICE points to global memory of the current CUDA
+ *   device and must be 16-byte aligned; every pointer marked HOST is ordinary
+ *   host memory read during the call.  All tensors are dense, row-major.
+ * - The library allocates no device memory.  Caches, outputs, selection
+ *   buffers and scratch ("workspace", size from rtp_workspace_bytes) belong to
+ *   the caller.  Workspace contents are undefined after a call; two calls that
+ *   may overlap on the GPU must not share a workspace.
+ * - Calls are asynchronous on the CUDA stream passed as `stream` (a
+ *   cudaStream_t cast to void*, NULL = default stream).
+ * - Every call returns an rtp_status.  Errors detectable on the host (NULL or
+ *   misaligned pointers, unsupported sizes, p outside (0,1]) are returned before
+ *   anything is launched.  Conditions only visible on the device (a selection
+ *   list that overflows, a row position beyond its sequence) are reported by
+ *   writing the largest rtp_status code seen into the caller's DEVICE int32
+ *   `status` word (which the caller zeroes); kernels never trap.
+ * - bf16 = 16-bit brain float bit patterns.  Fixed sizes: head_dim 128,
+ *   index_dim 16, page_size 64.
+ *
+ * Head conventions: query head h reads KV head h / (n_q_heads / n_kv_heads).
+ * Retrieval query heads are listed in rtp_params.ret_q_heads; entry i has its
+ * own W_q[i] and its own selection, and scores against the index-key stream
+ * q_head_to_index_head[i].  Index head j projects the pre-RoPE keys of KV head
+ * index_head_kv[j] with W_k[j].
+ */
+#ifndef RTP_H_
+#define RTP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RTP_HEAD_DIM 128
+#define RTP_INDEX_DIM 16
+#define RTP_PAGE_SIZE 64
+#define RTP_MAX_Q_HEADS 128
+#define RTP_MAX_INDEX_HEADS 32
+#define RTP_MAX_HEADS_PER_INDEX_HEAD 16
+
+typedef enum rtp_status {
+  RTP_OK = 0,
+  RTP_ERR_INVALID = 1,     /* bad argument */
+  RTP_ERR_CAPACITY = 2,    /* a caller buffer is too small (lists, workspace) */
+  RTP_ERR_UNSUPPORTED = 3, /* valid request this build does not implement */
+  RTP_ERR_CUDA = 4,        /* a CUDA runtime call failed; see rtp_last_error */
+  RTP_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out */
+} rtp_status;
+
+/* Opaque host-side context: device properties and the last error string. */
+typedef struct rtp_ctx rtp_ctx;
+
+/* Method parameters (Table 2 gives the paper's values: index_dim 16, top_p 0.9,
+ * n_sink 4, window 8192).  The four head-map arrays are HOST pointers. */
+typedef struct rtp_params {
+  int32_t head_dim;      /* must be 128 */
+  int32_t index_dim;     /* must be 16 */
+  int32_t page_size;     /* must be 64 */
+  int32_t n_q_heads;     /* <= RTP_MAX_Q_HEADS, multiple of n_kv_heads */
+  int32_t n_kv_heads;
+  int32_t n_index_heads; /* <= RTP_MAX_INDEX_HEADS */
+  int32_t n_ret_q_heads; /* number of retrieval query heads */
+  int32_t n_local_kv_heads;
+  int32_t n_sink;        /* attention sinks of local heads (first n_sink tokens) */
+  int32_t window;        /* sliding window of local heads: positions (m-window, m] */
+  float top_p;           /* in (0, 1] */
+  float score_scale;     /* temperature on the indexer score; 1.0 in the paper */
+  float sm_scale;        /* softmax scale of the real attention, 1/sqrt(128) */
+  const int32_t* ret_q_heads;          /* HOST [n_ret_q_heads] query-head ids */
+  const int32_t* q_head_to_index_head; /* HOST [n_ret_q_heads] */
+  const int32_t* index_head_kv;        /* HOST [n_index_heads] KV head of each index head */
+  const int32_t* local_kv_heads;       /* HOST [n_local_kv_heads] */
+} rtp_params;
+
+/* Paged caches.  The index-key cache shares the KV block table. */
+typedef struct rtp_cache {
+  void* k_pages;              /* DEVICE bf16 [num_pages, n_kv_heads, 64, 128] */
+  void* v_pages;              /* DEVICE bf16 [num_pages, n_kv_heads, 64, 128] */
+  void* ikey_pages;           /* DEVICE bf16 [num_pages, n_index_heads, 64, 16] */
+  const int32_t* block_table; /* DEVICE int32 [batch, max_pages] physical page ids */
+  const int32_t* seq_lens;    /* DEVICE int32 [batch] tokens present per sequence */
+  int32_t num_pages;
+  int32_t batch;
+  int32_t max_pages;
+} rtp_cache;
+
+/* ---- utility ------------------------------------------------------------ */
+
+/* Library version, major*10000 + minor*100 + patch.  (No counterpart in the paper.) */
+int32_t rtp_version(void);
+
+/* Creates a context for the current CUDA device.  Returns RTP_ERR_CUDA when no
+ * usable sm_100 device is current.  (No counterpart in the paper.) */
+rtp_status rtp_create(rtp_ctx** out_ctx);
+void rtp_destroy(rtp_ctx* ctx);
+
+/* Text of the last error recorded on this context (never NULL). */
+const char* rtp_last_error(const rtp_ctx* ctx);
+
+/* Bytes of DEVICE workspace that any call below needs for `rows` query rows
+ * against sequences of at most `max_seq_len` tokens.  0 on invalid params. */
+size_t rtp_workspace_bytes(const rtp_params* params, int64_t rows, int64_t max_seq_len);
+
+/* Synchronises `stream`, reads the DEVICE status word and returns it as an
+ * rtp_status (RTP_ERR_CUDA if the stream reports an error). */
+rtp_status rtp_check_status(rtp_ctx* ctx, const int32_t* status, void* stream);
+
+/* ---- S0: index-key projection and cache append (Eq. 4, the W^K k_pre factor;
+ *      Section 3.4 calls the result the "compressed K sequence") -------------
+ * k_pre   DEVICE bf16 [T, n_index_heads, 128]  pre-RoPE keys of the index heads
+ * w_k     DEVICE bf16 [n_index_heads, 128, 16]
+ * tok_seq DEVICE int32 [T] sequence of each token; tok_pos DEVICE int32 [T] its position
+ * Writes ikey_pages[block_table[seq][pos/64], j, pos%64, :] for every token and
+ * index head j: fp32 accumulation, rounded to bf16.  Pages must already be
+ * mapped in block_table.  Nothing else is written. */
+rtp_status rtp_index_keys(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                          const void* k_pre, const void* w_k, const int32_t* tok_seq,
+                          const int32_t* tok_pos, int64_t T, void* stream);
+
+/* ---- S1: query projection (Eq. 4, the W^Q q_pre factor) --------------------
+ * q_pre  DEVICE bf16 [R, n_q_heads, 128] pre-RoPE queries (all heads; only the
+ *        retrieval heads are read)
+ * w_q    DEVICE bf16 [n_ret_q_heads, 128, 16]
+ * qt_out DEVICE bf16 [R, n_ret_q_heads, 16]
+ * Exposed so that tests can feed the oracle the projected queries the kernels use. */
+rtp_status rtp_index_queries(rtp_ctx* ctx, const rtp_params* params, const void* q_pre,
+                             const void* w_q, int64_t R, void* qt_out, void* stream);
+
+/* ---- S1-S3: indexer scores and softmax normaliser (Eq. 4; Section 3.3 for the
+ *      distribution softmax(s) that top-p cuts) ------------------------------
+ * Row i is the query at position row_pos[i] of sequence row_seq[i]; it scores
+ * keys 0..row_pos[i] (inclusive).  DEVICE int32 row_seq, row_pos [R].
+ * scores_out  DEVICE fp32 [R, n_ret_q_heads, score_stride] or NULL; entries past
+ *             the row's last key are left untouched
+ * row_max_out DEVICE fp32 [R, n_ret_q_heads] or NULL : M = max_n s
+ * row_sum_out DEVICE fp32 [R, n_ret_q_heads] or NULL : Z = sum_n exp(s - M)
+ * s = score_scale * sum_j qt_j kt_j with bf16 factors and fp32 accumulation. */
+rtp_status rtp_index_score(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                           const void* q_pre, const void* w_q, const int32_t* row_seq,
+                           const int32_t* row_pos, int64_t R, float* scores_out,
+                           int64_t score_stride, float* row_max_out, float* row_sum_out,
+                           void* workspace, size_t workspace_bytes, int32_t* status,
+                           void* stream);
+
+/* ---- S2-S4: fused indexer + top-p selection (Eq. 5, S = Top-P(s, p)) --------
+ * Selects, per row and retrieval query head, the shortest prefix of the keys in
+ * order of decreasing score (ties: smaller position first) whose softmax mass
+ * reaches top_p.  Mass sums are fp32; a token whose cumulative mass before its
+ * own inclusion is within 1e-5 of p may be included.  The set is never empty;
+ * top_p == 1 selects every causal key.
+ *
+ * Rows: either DEVICE row_seq/row_pos [R] (any rows; the decode path), or
+ * row_seq == row_pos == NULL and the rows are positions q_start..q_start+R-1 of
+ * sequence seq_id (a prefill chunk).
+ * sel_idx      DEVICE int32 [R, n_ret_q_heads, sel_stride] logical token
+ *              positions in unspecified order, or NULL (thresholds only)
+ * sel_count    DEVICE int32 [R, n_ret_q_heads] true size of the set, also when
+ *              it exceeds sel_stride (then only sel_stride ids are written and
+ *              RTP_ERR_CAPACITY is recorded in *status)
+ * sel_mass     DEVICE fp32  [R, n_ret_q_heads] softmax mass of the set (fp32 estimate)
+ * sel_thresh   DEVICE fp32  [R, n_ret_q_heads] smallest selected score
+ * sel_tie_last DEVICE int32 [R, n_ret_q_heads] largest selected position among
+ *              keys whose score equals sel_thresh; a key n belongs to the set
+ *              iff s > thresh or (s == thresh and n <= tie_last)
+ * status       DEVICE int32 [1] */
+rtp_status rtp_topp_select(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                           const void* q_pre, const void* w_q, const int32_t* row_seq,
+                           const int32_t* row_pos, int32_t seq_id, int32_t q_start, int64_t R,
+                           int32_t* sel_idx, int64_t sel_stride, int32_t* sel_count,
+                           float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
+                           int32_t* status, void* workspace, size_t workspace_bytes,
+                           void* stream);
+
+/* ---- S5 (+S8): sparse attention over selection lists (Eq. 5) ----------------
+ * For every row and retrieval query head: softmax(q.k * sm_scale) over the listed
+ * keys, times V; split over the list with a log-sum-exp merge when rows are few.
+ * q    DEVICE bf16 [R, n_q_heads, 128] post-RoPE queries
+ * out  DEVICE bf16 [R, n_q_heads, 128]; only retrieval heads' slots are written
+ * lse  DEVICE fp32 [R, n_q_heads] natural-log-sum-exp of the scaled logits, or NULL
+ * sel_idx / sel_count as written by rtp_topp_select (counts above sel_stride are
+ * clamped).  Ids must be < the row's key count; others are skipped and
+ * RTP_ERR_INVALID is recorded. */
+rtp_status rtp_sparse_attn_decode(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                                  const void* q, const int32_t* row_seq, const int32_t* row_pos,
+                                  int64_t R, const int32_t* sel_idx, int64_t sel_stride,
+                                  const int32_t* sel_count, void* out, float* lse,
+                                  void* workspace, size_t workspace_bytes, int32_t* status,
+                                  void* stream);
+
+/* ---- S6: sparse attention for a prefill chunk (Eq. 5 applied per query row; the
+ *      paper itself keeps retrieval heads dense in prefill) -------------------
+ * Rows are positions q_start..q_start+C-1 of sequence seq_id; causal.
+ * With sel_idx != NULL the lists are used as in rtp_sparse_attn_decode.  With
+ * sel_idx == NULL membership is re-evaluated inside the attention kernel from
+ * (sel_thresh, sel_tie_last) and the indexer score, which needs q_pre and w_q;
+ * key tiles in which no row selects anything are skipped.
+ * q, q_pre DEVICE bf16 [C, n_q_heads, 128]; out/lse as above. */
+rtp_status rtp_sparse_attn_prefill(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                                   const void* q, const void* q_pre, const void* w_q,
+                                   int32_t seq_id, int32_t q_start, int64_t C,
+                                   const int32_t* sel_idx, int64_t sel_stride,
+                                   const int32_t* sel_count, const float* sel_thresh,
+                                   const int32_t* sel_tie_last, void* out, float* lse,
+                                   void* workspace, size_t workspace_bytes, int32_t* status,
+                                   void* stream);
+
+/* ---- S7: local heads, attention sinks + sliding window (Section 3.2, Table 2) -
+ * Row at position m attends to {n <= m : n < n_sink or n > m - window}.
+ * Rows as in rtp_topp_select (row arrays = decode path with split-KV; NULL
+ * arrays = prefill chunk seq_id, q_start).  Only the query heads of
+ * params->local_kv_heads are computed and written. */
+rtp_status rtp_local_attn(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                          const void* q, const int32_t* row_seq, const int32_t* row_pos,
+                          int32_t seq_id, int32_t q_start, int64_t R, void* out, float* lse,
+                          void* workspace, size_t workspace_bytes, int32_t* status,
+                          void* stream);
+
+/* ---- S9: dense causal attention, the in-library comparator (what retrieval
+ *      heads run during the paper's prefill, Section 3.2) ---------------------
+ * kv_heads HOST int32 [n_heads] KV heads whose query heads are computed; NULL =
+ * all heads.  rtp_dense_attn_prefill: rows q_start.. of seq_id;
+ * rtp_dense_attn_decode: rows given by DEVICE row_seq/row_pos, split-KV. */
+rtp_status rtp_dense_attn_prefill(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                                  const void* q, int32_t seq_id, int32_t q_start, int64_t C,
+                                  const int32_t* kv_heads, int32_t n_heads, void* out, float* lse,
+                                  int32_t* status, void* stream);
+rtp_status rtp_dense_attn_decode(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                                 const void* q, const int32_t* row_seq, const int32_t* row_pos,
+                                 int64_t R, const int32_t* kv_heads, int32_t n_heads, void* out,
+                                 float* lse, void* workspace, size_t workspace_bytes,
+                                 int32_t* status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RTP_H_ */

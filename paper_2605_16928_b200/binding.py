@@ -1,0 +1,283 @@
+"""Thin ctypes binding of the C ABI in ``include/rtp.h``.
+
+Argument marshalling only: every step of the path runs inside ``librtp.so``.
+Tensors are torch CUDA tensors (torch is used for device memory and streams);
+bf16 tensors may be ``torch.bfloat16`` or raw ``int16``/``uint16`` views.  There
+is no CPU fallback: a missing library or a failing call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+_LIB: Optional[C.CDLL] = None
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "librtp.so")
+
+RTP_OK, RTP_ERR_INVALID, RTP_ERR_CAPACITY, RTP_ERR_UNSUPPORTED, RTP_ERR_CUDA, RTP_ERR_TIMEOUT = range(6)
+_STATUS_NAMES = ["RTP_OK", "RTP_ERR_INVALID", "RTP_ERR_CAPACITY", "RTP_ERR_UNSUPPORTED", "RTP_ERR_CUDA",
+                 "RTP_ERR_TIMEOUT"]
+
+EXPORTS = [
+    "rtp_version", "rtp_create", "rtp_destroy", "rtp_last_error", "rtp_workspace_bytes", "rtp_check_status",
+    "rtp_index_keys", "rtp_index_queries", "rtp_index_score", "rtp_topp_select", "rtp_sparse_attn_decode",
+    "rtp_sparse_attn_prefill", "rtp_local_attn", "rtp_dense_attn_prefill", "rtp_dense_attn_decode",
+]
+
+
+class RtpError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        name = _STATUS_NAMES[code] if 0 <= code < len(_STATUS_NAMES) else str(code)
+        super().__init__(f"{where}: {name}" + (f" ({detail})" if detail else ""))
+
+
+class RtpParams(C.Structure):
+    _fields_ = [
+        ("head_dim", C.c_int32), ("index_dim", C.c_int32), ("page_size", C.c_int32),
+        ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("n_index_heads", C.c_int32),
+        ("n_ret_q_heads", C.c_int32), ("n_local_kv_heads", C.c_int32),
+        ("n_sink", C.c_int32), ("window", C.c_int32),
+        ("top_p", C.c_float), ("score_scale", C.c_float), ("sm_scale", C.c_float),
+        ("ret_q_heads", C.POINTER(C.c_int32)), ("q_head_to_index_head", C.POINTER(C.c_int32)),
+        ("index_head_kv", C.POINTER(C.c_int32)), ("local_kv_heads", C.POINTER(C.c_int32)),
+    ]
+
+
+class RtpCache(C.Structure):
+    _fields_ = [
+        ("k_pages", C.c_void_p), ("v_pages", C.c_void_p), ("ikey_pages", C.c_void_p),
+        ("block_table", C.c_void_p), ("seq_lens", C.c_void_p),
+        ("num_pages", C.c_int32), ("batch", C.c_int32), ("max_pages", C.c_int32),
+    ]
+
+
+def load_library(path: Optional[str] = None) -> C.CDLL:
+    """Loads ``librtp.so`` (built in-tree by ``build.py``); raises if it is missing."""
+    global _LIB
+    if _LIB is not None and path is None:
+        return _LIB
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise RtpError(RTP_ERR_CUDA, "load_library",
+                       f"{p} not found: build it with `python -m paper_2605_16928_b200.build`")
+    lib = C.CDLL(p)
+    vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+    PP, PC = C.POINTER(RtpParams), C.POINTER(RtpCache)
+    lib.rtp_version.restype = i32
+    lib.rtp_version.argtypes = []
+    lib.rtp_create.restype = i32
+    lib.rtp_create.argtypes = [C.POINTER(vp)]
+    lib.rtp_destroy.restype = None
+    lib.rtp_destroy.argtypes = [vp]
+    lib.rtp_last_error.restype = C.c_char_p
+    lib.rtp_last_error.argtypes = [vp]
+    lib.rtp_workspace_bytes.restype = sz
+    lib.rtp_workspace_bytes.argtypes = [PP, i64, i64]
+    lib.rtp_check_status.restype = i32
+    lib.rtp_check_status.argtypes = [vp, vp, vp]
+    lib.rtp_index_keys.restype = i32
+    lib.rtp_index_keys.argtypes = [vp, PP, PC, vp, vp, vp, vp, i64, vp]
+    lib.rtp_index_queries.restype = i32
+    lib.rtp_index_queries.argtypes = [vp, PP, vp, vp, i64, vp, vp]
+    lib.rtp_index_score.restype = i32
+    lib.rtp_index_score.argtypes = [vp, PP, PC, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, sz, vp, vp]
+    lib.rtp_topp_select.restype = i32
+    lib.rtp_topp_select.argtypes = [vp, PP, PC, vp, vp, vp, vp, i32, i32, i64, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.rtp_sparse_attn_decode.restype = i32
+    lib.rtp_sparse_attn_decode.argtypes = [vp, PP, PC, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, sz, vp, vp]
+    lib.rtp_sparse_attn_prefill.restype = i32
+    lib.rtp_sparse_attn_prefill.argtypes = [vp, PP, PC, vp, vp, vp, i32, i32, i64, vp, i64, vp, vp, vp, vp, vp, vp,
+                                            sz, vp, vp]
+    lib.rtp_local_attn.restype = i32
+    lib.rtp_local_attn.argtypes = [vp, PP, PC, vp, vp, vp, i32, i32, i64, vp, vp, vp, sz, vp, vp]
+    lib.rtp_dense_attn_prefill.restype = i32
+    lib.rtp_dense_attn_prefill.argtypes = [vp, PP, PC, vp, i32, i32, i64, vp, i32, vp, vp, vp, vp]
+    lib.rtp_dense_attn_decode.restype = i32
+    lib.rtp_dense_attn_decode.argtypes = [vp, PP, PC, vp, vp, vp, i64, vp, i32, vp, vp, vp, sz, vp, vp]
+    if path is None:
+        _LIB = lib
+    return lib
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return int(t.data_ptr())
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream) or None
+    if isinstance(stream, int):
+        return stream or None
+    return int(stream.cuda_stream) or None
+
+
+def _i32_array(vals: Sequence[int]):
+    arr = (C.c_int32 * max(1, len(vals)))(*[int(v) for v in vals])
+    return arr
+
+
+class Params:
+    """Owns an ``rtp_params`` block and the host head-map arrays it points to."""
+
+    def __init__(self, n_q_heads: int, n_kv_heads: int, ret_q_heads: Sequence[int],
+                 q_head_to_index_head: Sequence[int], index_head_kv: Sequence[int],
+                 local_kv_heads: Sequence[int], n_sink: int = 4, window: int = 8192, top_p: float = 0.9,
+                 score_scale: float = 1.0, sm_scale: float = 128 ** -0.5):
+        self._a = _i32_array(ret_q_heads)
+        self._b = _i32_array(q_head_to_index_head)
+        self._c = _i32_array(index_head_kv)
+        self._d = _i32_array(local_kv_heads)
+        self.n_ret = len(ret_q_heads)
+        self.n_q_heads = n_q_heads
+        self.n_kv_heads = n_kv_heads
+        self.n_index_heads = len(index_head_kv)
+        self.ret_q_heads = list(ret_q_heads)
+        self.local_kv_heads = list(local_kv_heads)
+        self.c = RtpParams(128, 16, 64, n_q_heads, n_kv_heads, len(index_head_kv), len(ret_q_heads),
+                           len(local_kv_heads), n_sink, window, top_p, score_scale, sm_scale,
+                           C.cast(self._a, C.POINTER(C.c_int32)), C.cast(self._b, C.POINTER(C.c_int32)),
+                           C.cast(self._c, C.POINTER(C.c_int32)), C.cast(self._d, C.POINTER(C.c_int32)))
+
+    @classmethod
+    def from_workload(cls, wl, **over) -> "Params":
+        h = wl.heads
+        kw = dict(n_q_heads=h.n_q_heads, n_kv_heads=h.n_kv_heads, ret_q_heads=h.ret_q_heads,
+                  q_head_to_index_head=h.q_head_to_index_head, index_head_kv=h.index_head_kv,
+                  local_kv_heads=h.local_kv_heads, n_sink=h.n_sink, window=h.window, top_p=wl.top_p,
+                  score_scale=wl.score_scale, sm_scale=wl.sm_scale)
+        kw.update(over)
+        return cls(**kw)
+
+    def ref(self):
+        return C.byref(self.c)
+
+
+def make_cache(k_pages, v_pages, ikey_pages, block_table, seq_lens) -> RtpCache:
+    """Describes caller-owned paged caches (torch CUDA tensors) to the library."""
+    num_pages = int((k_pages if k_pages is not None else ikey_pages).shape[0])
+    return RtpCache(_ptr(k_pages), _ptr(v_pages), _ptr(ikey_pages), _ptr(block_table), _ptr(seq_lens),
+                    num_pages, int(block_table.shape[0]), int(block_table.shape[1]))
+
+
+class Context:
+    """``rtp_ctx`` for the current CUDA device."""
+
+    def __init__(self):
+        self.lib = load_library()
+        h = C.c_void_p()
+        rc = self.lib.rtp_create(C.byref(h))
+        if rc != RTP_OK:
+            raise RtpError(rc, "rtp_create", "needs a CUDA device of compute capability 10.x")
+        self.h = h
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.rtp_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int, where: str):
+        if rc != RTP_OK:
+            raise RtpError(rc, where, (self.lib.rtp_last_error(self.h) or b"").decode())
+
+
+def rtp_version() -> int:
+    return int(load_library().rtp_version())
+
+
+def rtp_workspace_bytes(params: Params, rows: int, max_seq_len: int) -> int:
+    return int(load_library().rtp_workspace_bytes(params.ref(), rows, max_seq_len))
+
+
+def rtp_check_status(ctx: Context, status, stream=None) -> int:
+    return int(ctx.lib.rtp_check_status(ctx.h, _ptr(status), _stream(stream)))
+
+
+def rtp_index_keys(ctx, params, cache, k_pre, w_k, tok_seq, tok_pos, stream=None):
+    ctx._check(ctx.lib.rtp_index_keys(ctx.h, params.ref(), C.byref(cache), _ptr(k_pre), _ptr(w_k), _ptr(tok_seq),
+                                      _ptr(tok_pos), int(tok_seq.shape[0]), _stream(stream)), "rtp_index_keys")
+
+
+def rtp_index_queries(ctx, params, q_pre, w_q, qt_out, stream=None):
+    ctx._check(ctx.lib.rtp_index_queries(ctx.h, params.ref(), _ptr(q_pre), _ptr(w_q), int(q_pre.shape[0]),
+                                         _ptr(qt_out), _stream(stream)), "rtp_index_queries")
+
+
+def rtp_index_score(ctx, params, cache, q_pre, w_q, row_seq, row_pos, scores_out, row_max_out, row_sum_out,
+                    workspace, status, stream=None):
+    stride = int(scores_out.shape[-1]) if scores_out is not None else 0
+    ctx._check(ctx.lib.rtp_index_score(ctx.h, params.ref(), C.byref(cache), _ptr(q_pre), _ptr(w_q), _ptr(row_seq),
+                                       _ptr(row_pos), int(row_seq.shape[0]), _ptr(scores_out), stride,
+                                       _ptr(row_max_out), _ptr(row_sum_out), _ptr(workspace),
+                                       int(workspace.numel() * workspace.element_size()), _ptr(status),
+                                       _stream(stream)), "rtp_index_score")
+
+
+def rtp_topp_select(ctx, params, cache, q_pre, w_q, row_seq, row_pos, seq_id, q_start, n_rows, sel_idx, sel_count,
+                    sel_mass, sel_thresh, sel_tie_last, status, workspace, stream=None):
+    stride = int(sel_idx.shape[-1]) if sel_idx is not None else 0
+    ctx._check(ctx.lib.rtp_topp_select(ctx.h, params.ref(), C.byref(cache), _ptr(q_pre), _ptr(w_q), _ptr(row_seq),
+                                       _ptr(row_pos), int(seq_id), int(q_start), int(n_rows), _ptr(sel_idx), stride,
+                                       _ptr(sel_count), _ptr(sel_mass), _ptr(sel_thresh), _ptr(sel_tie_last),
+                                       _ptr(status), _ptr(workspace),
+                                       int(workspace.numel() * workspace.element_size()), _stream(stream)),
+               "rtp_topp_select")
+
+
+def rtp_sparse_attn_decode(ctx, params, cache, q, row_seq, row_pos, sel_idx, sel_count, out, lse, workspace, status,
+                           stream=None):
+    ctx._check(ctx.lib.rtp_sparse_attn_decode(ctx.h, params.ref(), C.byref(cache), _ptr(q), _ptr(row_seq),
+                                              _ptr(row_pos), int(row_seq.shape[0]), _ptr(sel_idx),
+                                              int(sel_idx.shape[-1]), _ptr(sel_count), _ptr(out), _ptr(lse),
+                                              _ptr(workspace), int(workspace.numel() * workspace.element_size()),
+                                              _ptr(status), _stream(stream)), "rtp_sparse_attn_decode")
+
+
+def rtp_sparse_attn_prefill(ctx, params, cache, q, q_pre, w_q, seq_id, q_start, n_rows, sel_idx, sel_count,
+                            sel_thresh, sel_tie_last, out, lse, workspace, status, stream=None):
+    stride = int(sel_idx.shape[-1]) if sel_idx is not None else 0
+    ctx._check(ctx.lib.rtp_sparse_attn_prefill(ctx.h, params.ref(), C.byref(cache), _ptr(q), _ptr(q_pre), _ptr(w_q),
+                                               int(seq_id), int(q_start), int(n_rows), _ptr(sel_idx), stride,
+                                               _ptr(sel_count), _ptr(sel_thresh), _ptr(sel_tie_last), _ptr(out),
+                                               _ptr(lse), _ptr(workspace),
+                                               int(workspace.numel() * workspace.element_size()), _ptr(status),
+                                               _stream(stream)), "rtp_sparse_attn_prefill")
+
+
+def rtp_local_attn(ctx, params, cache, q, row_seq, row_pos, seq_id, q_start, n_rows, out, lse, workspace, status,
+                   stream=None):
+    ws_bytes = int(workspace.numel() * workspace.element_size()) if workspace is not None else 0
+    ctx._check(ctx.lib.rtp_local_attn(ctx.h, params.ref(), C.byref(cache), _ptr(q), _ptr(row_seq), _ptr(row_pos),
+                                      int(seq_id), int(q_start), int(n_rows), _ptr(out), _ptr(lse), _ptr(workspace),
+                                      ws_bytes, _ptr(status), _stream(stream)), "rtp_local_attn")
+
+
+def rtp_dense_attn_prefill(ctx, params, cache, q, seq_id, q_start, n_rows, kv_heads, out, lse, status, stream=None):
+    arr = _i32_array(kv_heads) if kv_heads is not None else None
+    ctx._check(ctx.lib.rtp_dense_attn_prefill(ctx.h, params.ref(), C.byref(cache), _ptr(q), int(seq_id), int(q_start),
+                                              int(n_rows), C.cast(arr, C.c_void_p) if arr is not None else None,
+                                              len(kv_heads) if kv_heads is not None else 0, _ptr(out), _ptr(lse),
+                                              _ptr(status), _stream(stream)), "rtp_dense_attn_prefill")
+
+
+def rtp_dense_attn_decode(ctx, params, cache, q, row_seq, row_pos, kv_heads, out, lse, workspace, status,
+                          stream=None):
+    arr = _i32_array(kv_heads) if kv_heads is not None else None
+    ctx._check(ctx.lib.rtp_dense_attn_decode(ctx.h, params.ref(), C.byref(cache), _ptr(q), _ptr(row_seq),
+                                             _ptr(row_pos), int(row_seq.shape[0]),
+                                             C.cast(arr, C.c_void_p) if arr is not None else None,
+                                             len(kv_heads) if kv_heads is not None else 0, _ptr(out), _ptr(lse),
+                                             _ptr(workspace), int(workspace.numel() * workspace.element_size()),
+                                             _ptr(status), _stream(stream)), "rtp_dense_attn_decode")

@@ -1,0 +1,233 @@
+// S0/S1: low-rank projections (Eq. 4 factors W^K k_pre and W^Q q_pre); S2/S3: materialised
+// indexer scores with the softmax normaliser.
+#include "rtp_device.cuh"
+
+namespace rtp {
+
+namespace {
+
+constexpr int kProjTokens = 16;   // tokens (rows) per CTA
+constexpr int kProjThreads = kProjTokens * kIndexDim;
+
+// One CTA projects 16 rows of one projection head: thread (t, j) owns output j of row t and
+// accumulates the 128 products in fp32 in channel order.
+template <bool kKeys>
+__global__ void __launch_bounds__(kProjThreads) project_kernel(
+    CacheView cv, Dims d, HeadMaps hm, const __nv_bfloat16* __restrict__ src,
+    const __nv_bfloat16* __restrict__ w, const int32_t* __restrict__ tok_seq,
+    const int32_t* __restrict__ tok_pos, int64_t T, __nv_bfloat16* __restrict__ qt) {
+  __shared__ float ws[kHeadDim * kIndexDim];                      // 8 KB
+  __shared__ __align__(16) __nv_bfloat16 xs[kProjTokens][kHeadDim];  // 4 KB
+  const int head = blockIdx.y;
+  const int tid = threadIdx.x;
+  const int64_t t0 = (int64_t)blockIdx.x * kProjTokens;
+
+  {  // weights: 2048 bf16, 8 per thread
+    const uint4 v = ld_nc_v4(w + (int64_t)head * kHeadDim * kIndexDim + tid * 8);
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __bfloat1622float2(p[i]);
+      ws[tid * 8 + 2 * i] = f.x;
+      ws[tid * 8 + 2 * i + 1] = f.y;
+    }
+  }
+  {  // rows: 16 x 256 B, one 16-byte load per thread
+    const int r = tid >> 4, c = tid & 15;
+    const int64_t t = t0 + r;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (t < T) {
+      const int64_t row = kKeys ? (t * d.n_ih + head) : (t * d.n_q + hm.ret_q_head[head]);
+      v = ld_stream_v4(src + row * kHeadDim + c * 8);
+    }
+    *reinterpret_cast<uint4*>(&xs[r][c * 8]) = v;
+  }
+  __syncthreads();
+
+  const int r = tid >> 4, j = tid & 15;
+  const int64_t t = t0 + r;
+  float acc = 0.f;
+#pragma unroll 16
+  for (int c = 0; c < kHeadDim; ++c) acc = fmaf(__bfloat162float(xs[r][c]), ws[c * kIndexDim + j], acc);
+  if (t >= T) return;
+  const __nv_bfloat16 o = __float2bfloat16_rn(acc);
+  if (kKeys) {
+    const int seq = tok_seq[t], pos = tok_pos[t];
+    if (seq < 0 || seq >= cv.batch || pos < 0 || (pos >> kPageShift) >= cv.max_pages) return;
+    const int phys = cv.block_table[(int64_t)seq * cv.max_pages + (pos >> kPageShift)];
+    if (phys < 0 || phys >= cv.num_pages) return;
+    cv.ikey[(((int64_t)phys * cv.n_ih + head) * kPage + (pos & (kPage - 1))) * kIndexDim + j] = o;
+  } else {
+    qt[(t * d.n_ret + head) * kIndexDim + j] = o;
+  }
+}
+
+// ---- materialised scores -----------------------------------------------------------------------
+constexpr int kScoreWarps = 4;
+
+// grid = (R * n_ih, splits).  Each CTA scans a contiguous range of pages of one (row, index head)
+// for all retrieval heads attached to that index head.
+__global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(
+    CacheView cv, Dims d, HeadMaps hm, Rows rows, const __nv_bfloat16* __restrict__ qt,
+    float* __restrict__ scores, int64_t score_stride, float2* __restrict__ partial, int n_splits,
+    int32_t* status) {
+  const int64_t r = blockIdx.x / d.n_ih;
+  const int ih = blockIdx.x % d.n_ih;
+  const int split = blockIdx.y;
+  const int nh = hm.ih_nheads[ih];
+  if (nh == 0) return;
+  const int seq = rows.row_seq(r);
+  int n_keys = rows.row_pos(r) + 1;
+  {
+    const int sl = (seq >= 0 && seq < cv.batch) ? cv.seq_lens[seq] : 0;
+    if (n_keys > sl) {
+      if (threadIdx.x == 0) set_status(status, RTP_ERR_INVALID);
+      n_keys = sl;
+    }
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, c = lane & 3;
+  const int n_pages = (n_keys + kPage - 1) >> kPageShift;
+  const int per = (n_pages + n_splits - 1) / n_splits;
+  const int p_lo = split * per;
+  const int p_hi = min(n_pages, p_lo + per);
+
+  const QFrag qf = load_qfrag(qt + r * d.n_ret * kIndexDim, hm.ih_heads[ih], nh, lane);
+  const int head_lo = g < nh ? hm.ih_heads[ih][g] : -1;
+  const int head_hi = g + 8 < nh ? hm.ih_heads[ih][g + 8] : -1;
+  float m_lo = -INFINITY, l_lo = 0.f, m_hi = -INFINITY, l_hi = 0.f;
+
+  for (int p = p_lo + warp; p < p_hi; p += kScoreWarps) {
+    const __nv_bfloat16* base = ikey_page_ptr(cv, seq, p, ih);
+    uint4 v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = ld_stream_v4(base + (i * 32 + lane) * 8);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float s_lo[4], s_hi[4];
+      score16(qf, v[i], lane, s_lo, s_hi);
+      const int n0 = p * kPage + i * 16 + 4 * c;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int n = n0 + e;
+        if (n >= n_keys) continue;
+        if (head_lo >= 0) {
+          const float s = finish_score(s_lo[e], d.score_scale);
+          if (scores) scores[(r * d.n_ret + head_lo) * score_stride + n] = s;
+          const float mn = fmaxf(m_lo, s);
+          l_lo = l_lo * __expf(m_lo - mn) + __expf(s - mn);
+          m_lo = mn;
+        }
+        if (head_hi >= 0) {
+          const float s = finish_score(s_hi[e], d.score_scale);
+          if (scores) scores[(r * d.n_ret + head_hi) * score_stride + n] = s;
+          const float mn = fmaxf(m_hi, s);
+          l_hi = l_hi * __expf(m_hi - mn) + __expf(s - mn);
+          m_hi = mn;
+        }
+      }
+    }
+  }
+  // combine the four lanes of a group, then the warps through shared memory
+  __shared__ float2 red[kScoreWarps][16];
+#pragma unroll
+  for (int o = 1; o <= 2; o <<= 1) {
+    float mo = __shfl_xor_sync(0xffffffffu, m_lo, o), lo = __shfl_xor_sync(0xffffffffu, l_lo, o);
+    float mn = fmaxf(m_lo, mo);
+    l_lo = (mn == -INFINITY) ? 0.f : l_lo * __expf(m_lo - mn) + lo * __expf(mo - mn);
+    m_lo = mn;
+    mo = __shfl_xor_sync(0xffffffffu, m_hi, o), lo = __shfl_xor_sync(0xffffffffu, l_hi, o);
+    mn = fmaxf(m_hi, mo);
+    l_hi = (mn == -INFINITY) ? 0.f : l_hi * __expf(m_hi - mn) + lo * __expf(mo - mn);
+    m_hi = mn;
+  }
+  if (c == 0) {
+    red[warp][g] = make_float2(m_lo, l_lo);
+    red[warp][g + 8] = make_float2(m_hi, l_hi);
+  }
+  __syncthreads();
+  if (threadIdx.x < nh) {
+    float m = -INFINITY, l = 0.f;
+    for (int w = 0; w < kScoreWarps; ++w) {
+      const float2 x = red[w][threadIdx.x];
+      const float mn = fmaxf(m, x.x);
+      if (mn != -INFINITY) l = l * __expf(m - mn) + x.y * __expf(x.x - mn);
+      m = mn;
+    }
+    const int head = hm.ih_heads[ih][threadIdx.x];
+    partial[(r * d.n_ret + head) * n_splits + split] = make_float2(m, l);
+  }
+}
+
+__global__ void score_merge_kernel(const float2* __restrict__ partial, int n_splits, int64_t n_rowheads,
+                                   float* __restrict__ row_max, float* __restrict__ row_sum) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_rowheads) return;
+  float m = -INFINITY, l = 0.f;
+  for (int s = 0; s < n_splits; ++s) {
+    const float2 x = partial[i * n_splits + s];
+    const float mn = fmaxf(m, x.x);
+    if (mn != -INFINITY) l = l * __expf(m - mn) + x.y * __expf(x.x - mn);
+    m = mn;
+  }
+  if (row_max) row_max[i] = m;
+  if (row_sum) row_sum[i] = l;
+}
+
+int score_splits(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
+  const int64_t pages = (max_len + kPage - 1) / kPage;
+  int64_t want = (4LL * sm_count + R * d.n_ih - 1) / (R * d.n_ih);
+  int64_t cap = (pages + 31) / 32;   // at least 32 pages (2048 keys) per CTA
+  int64_t s = want < cap ? want : cap;
+  if (s < 1) s = 1;
+  if (s > 1024) s = 1024;
+  return (int)s;
+}
+
+}  // namespace
+
+cudaError_t launch_index_keys(const CacheView& cv, const Dims& d, const __nv_bfloat16* k_pre,
+                              const __nv_bfloat16* w_k, const int32_t* tok_seq, const int32_t* tok_pos,
+                              int64_t T, cudaStream_t st) {
+  if (T == 0) return cudaSuccess;
+  HeadMaps hm = {};
+  dim3 grid((unsigned)((T + kProjTokens - 1) / kProjTokens), d.n_ih);
+  project_kernel<true><<<grid, kProjThreads, 0, st>>>(cv, d, hm, k_pre, w_k, tok_seq, tok_pos, T, nullptr);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_index_queries(const Dims& d, const HeadMaps& hm, const __nv_bfloat16* q_pre,
+                                 const __nv_bfloat16* w_q, int64_t R, __nv_bfloat16* qt, cudaStream_t st) {
+  if (R == 0 || d.n_ret == 0) return cudaSuccess;
+  CacheView cv = {};
+  dim3 grid((unsigned)((R + kProjTokens - 1) / kProjTokens), d.n_ret);
+  project_kernel<false><<<grid, kProjThreads, 0, st>>>(cv, d, hm, q_pre, w_q, nullptr, nullptr, R, qt);
+  return cudaGetLastError();
+}
+
+size_t score_workspace_bytes(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
+  if (R <= 0) return 0;
+  return (size_t)R * d.n_ret * score_splits(d, R, max_len, sm_count) * sizeof(float2);
+}
+
+cudaError_t launch_index_score(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                               const __nv_bfloat16* qt, int64_t max_len, float* scores, int64_t score_stride,
+                               float* row_max, float* row_sum, void* ws, int32_t* status, int sm_count,
+                               cudaStream_t st) {
+  if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
+  const int n_splits = score_splits(d, rows.R, max_len, sm_count);
+  dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
+  score_kernel<<<grid, kScoreWarps * 32, 0, st>>>(cv, d, hm, rows, qt, scores, score_stride,
+                                                  reinterpret_cast<float2*>(ws), n_splits, status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (row_max || row_sum) {
+    const int64_t n = rows.R * d.n_ret;
+    score_merge_kernel<<<(unsigned)((n + 127) / 128), 128, 0, st>>>(reinterpret_cast<const float2*>(ws),
+                                                                     n_splits, n, row_max, row_sum);
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+}  // namespace rtp

@@ -1,0 +1,128 @@
+// Device-side helpers: ordered float keys, bf16 MMA, streaming loads, the indexer score core.
+#pragma once
+
+#include "rtp_internal.cuh"
+
+namespace rtp {
+
+// ---- ordered keys: unsigned comparison of okey(a), okey(b) == float comparison of a, b ----------
+__device__ __forceinline__ uint32_t okey(float s) {
+  uint32_t b = __float_as_uint(s);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float okey_to_float(uint32_t k) {
+  uint32_t b = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+  return __uint_as_float(b);
+}
+
+__device__ __forceinline__ void set_status(int32_t* status, int code) {
+  if (status) atomicMax(status, code);
+}
+
+// ---- streaming 16-byte load (read-only data that is not reused by this SM) -----------------------
+__device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+// ---- warp MMA m16n8k16, bf16 inputs, fp32 accumulate ------------------------------------------------
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1, const float (&c)[4]) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%10,%11,%12,%13};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
+}
+
+// ---- indexer score core --------------------------------------------------------------------------
+// One warp scores 16 consecutive index keys (512 contiguous bytes, one 16-byte load per lane)
+// against up to 16 projected queries held as an MMA A fragment.  The 16 index dimensions are
+// fed to the MMA in a permuted order (the same permutation on both operands), chosen so that
+// each lane's 16-byte load plus one exchange with lane^2 yields its B fragments.
+//
+// Lane l = 4*g + c.  After score16(): lane (g, c) holds, for query slot g (s_lo) and g + 8
+// (s_hi), the UNSCALED scores of keys 4c .. 4c+3 of the group.
+struct QFrag {
+  uint32_t a0, a1, a2, a3;
+};
+
+// Offset (in elements) of the four physical index dimensions lane c feeds to the MMA.
+__device__ __forceinline__ int qfrag_dim_offset(int lane) {
+  const int c = lane & 3;
+  return 8 * (c & 1) + 4 * (c >> 1);
+}
+
+// qt_row: projected queries of one row, [n_ret][16] bf16.  heads: list of retrieval-head indices
+// that occupy MMA rows 0..n-1.
+__device__ __forceinline__ QFrag load_qfrag(const __nv_bfloat16* qt_row, const uint8_t* heads, int n,
+                                            int lane) {
+  QFrag f = {0u, 0u, 0u, 0u};
+  const int g = lane >> 2;
+  const int off = qfrag_dim_offset(lane);
+  if (g < n) {
+    const uint2 v = *reinterpret_cast<const uint2*>(qt_row + (int)heads[g] * kIndexDim + off);
+    f.a0 = v.x;
+    f.a2 = v.y;
+  }
+  if (g + 8 < n) {
+    const uint2 v = *reinterpret_cast<const uint2*>(qt_row + (int)heads[g + 8] * kIndexDim + off);
+    f.a1 = v.x;
+    f.a3 = v.y;
+  }
+  return f;
+}
+
+// v = this lane's 16 bytes of the 512-byte group (lane l holds bytes [16 l, 16 l + 16)).
+__device__ __forceinline__ void score16(const QFrag& q, const uint4& v, int lane, float (&s_lo)[4],
+                                        float (&s_hi)[4]) {
+  const bool u = (lane & 2) != 0;  // lanes with u == 0 loaded an even key, u == 1 an odd key
+  const uint32_t send0 = u ? v.x : v.z;
+  const uint32_t send1 = u ? v.y : v.w;
+  const uint32_t r0 = __shfl_xor_sync(0xffffffffu, send0, 2);
+  const uint32_t r1 = __shfl_xor_sync(0xffffffffu, send1, 2);
+  const uint32_t e0 = u ? r0 : v.x, e1 = u ? r1 : v.y;  // even keys (tile 0)
+  const uint32_t o0 = u ? v.z : r0, o1 = u ? v.w : r1;  // odd keys (tile 1)
+  const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+  float t0[4], t1[4];
+  mma_bf16_16816(t0, q.a0, q.a1, q.a2, q.a3, e0, e1, zero);
+  mma_bf16_16816(t1, q.a0, q.a1, q.a2, q.a3, o0, o1, zero);
+  s_lo[0] = t0[0]; s_lo[1] = t1[0]; s_lo[2] = t0[1]; s_lo[3] = t1[1];
+  s_hi[0] = t0[2]; s_hi[1] = t1[2]; s_hi[2] = t0[3]; s_hi[3] = t1[3];
+}
+
+// Final score value: temperature applied in fp32, -0 folded into +0 so that equal scores have
+// equal ordered keys.
+__device__ __forceinline__ float finish_score(float raw, float scale) {
+  return __fadd_rn(__fmul_rn(raw, scale), 0.0f);
+}
+
+// Address of the 2 KB index-key slice of (logical page, index head) of a sequence.
+__device__ __forceinline__ const __nv_bfloat16* ikey_page_ptr(const CacheView& cv, int seq, int page,
+                                                               int ih) {
+  const int phys = __ldg(cv.block_table + (int64_t)seq * cv.max_pages + page);
+  return cv.ikey + ((int64_t)phys * cv.n_ih + ih) * (kPage * kIndexDim);
+}
+
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+  return x;
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+}  // namespace rtp

@@ -1,0 +1,120 @@
+// Internal declarations shared by the kernels and the C-ABI layer (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rtp.h"
+
+namespace rtp {
+
+constexpr int kHeadDim = RTP_HEAD_DIM;     // 128
+constexpr int kIndexDim = RTP_INDEX_DIM;   // 16
+constexpr int kPage = RTP_PAGE_SIZE;       // 64
+constexpr int kPageShift = 6;
+
+// Selection (decode-style) constants.
+constexpr int kSelBins = 2048;             // bins per radix level (11 + 11 + 10 bits of the ordered key)
+constexpr int kCandCap = 4096;             // boundary candidates resolved exactly per (row, head)
+constexpr float kMassMargin = 1e-5f;       // relative slack added to p*Z against fp32 summation error
+
+// Head maps, passed to kernels by value.
+struct HeadMaps {
+  uint8_t ret_q_head[RTP_MAX_Q_HEADS];      // query-head id of retrieval head i
+  uint8_t q2ih[RTP_MAX_Q_HEADS];            // index head of retrieval head i
+  uint8_t slot_in_ih[RTP_MAX_Q_HEADS];      // position of retrieval head i inside its index head's list
+  uint8_t ih_kv[RTP_MAX_INDEX_HEADS];       // KV head of index head j
+  uint8_t ih_nheads[RTP_MAX_INDEX_HEADS];   // number of retrieval heads scoring against index head j
+  uint8_t ih_heads[RTP_MAX_INDEX_HEADS][RTP_MAX_HEADS_PER_INDEX_HEAD];
+  uint8_t kv_list[RTP_MAX_Q_HEADS];         // KV heads processed by a local / dense call
+  int32_t n_kv_list;
+};
+
+struct CacheView {
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  __nv_bfloat16* ikey;
+  const int32_t* block_table;
+  const int32_t* seq_lens;
+  int32_t num_pages, batch, max_pages;
+  int32_t n_kv, n_ih;
+};
+
+struct Dims {
+  int32_t n_q, n_kv, n_ih, n_ret, group;
+  int32_t n_sink, window;
+  float top_p, score_scale, sm_scale;
+};
+
+// Rows of a call: explicit arrays (decode) or a contiguous chunk of one sequence.
+struct Rows {
+  const int32_t* seq;   // may be NULL
+  const int32_t* pos;   // may be NULL
+  int32_t seq_id, q_start;
+  int64_t R;
+  __device__ __forceinline__ int row_seq(int64_t r) const { return seq ? seq[r] : seq_id; }
+  __device__ __forceinline__ int row_pos(int64_t r) const { return pos ? pos[r] : q_start + (int)r; }
+};
+
+// Per (row, retrieval head) selection state kept in the workspace between passes.
+struct SelState {
+  uint32_t max_key;      // ordered key of the row maximum (atomicMax during level 1)
+  uint32_t lo_key;       // current bucket [lo_key, hi_key] of ordered keys that holds the threshold
+  uint32_t hi_key;
+  int32_t level;         // radix levels completed
+  int32_t mode;          // 0 = refining, 1 = collect candidates, 2 = select all, 3 = exact ties (scan)
+  float M;               // row maximum
+  float Z;               // sum exp(s - M)
+  float target;          // mass to reach, relative to M (p * Z * (1 + margin))
+  float mass_above;      // mass of keys above the bucket
+  int32_t cnt_above;     // number of keys above the bucket
+  int32_t bucket_cnt;
+  float bucket_mass;
+  int32_t emit_cnt;      // ids written by the compaction pass
+  int32_t cand_cnt;      // candidates written by the compaction pass
+  int32_t n_keys;        // causal key count of the row
+  int32_t pad;
+};
+
+enum SelMode { kRefine = 0, kCollect = 1, kSelectAll = 2, kTieScan = 3 };
+
+// ---- host launchers (one per .cu file) ---------------------------------------
+cudaError_t launch_index_keys(const CacheView& cv, const Dims& d, const __nv_bfloat16* k_pre,
+                              const __nv_bfloat16* w_k, const int32_t* tok_seq, const int32_t* tok_pos,
+                              int64_t T, cudaStream_t st);
+cudaError_t launch_index_queries(const Dims& d, const HeadMaps& hm, const __nv_bfloat16* q_pre,
+                                 const __nv_bfloat16* w_q, int64_t R, __nv_bfloat16* qt, cudaStream_t st);
+
+size_t score_workspace_bytes(const Dims& d, int64_t R, int64_t max_len, int sm_count);
+cudaError_t launch_index_score(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                               const __nv_bfloat16* qt, int64_t max_len, float* scores, int64_t score_stride,
+                               float* row_max, float* row_sum, void* ws, int32_t* status, int sm_count,
+                               cudaStream_t st);
+
+size_t select_rows_workspace_bytes(const Dims& d, int64_t R);
+cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                               const __nv_bfloat16* qt, int64_t max_len, int32_t* sel_idx, int64_t sel_stride,
+                               int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
+                               int32_t* status, void* ws, int sm_count, cudaStream_t st);
+
+size_t select_chunk_workspace_bytes(const Dims& d, int64_t R);
+cudaError_t launch_select_chunk(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                                const __nv_bfloat16* qt, int32_t* sel_idx, int64_t sel_stride,
+                                int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
+                                int32_t* status, void* ws, int sm_count, cudaStream_t st);
+
+enum AttnSet { kSetList = 0, kSetLocal = 1, kSetDense = 2 };
+size_t attn_rows_workspace_bytes(const Dims& d, int64_t R, int n_units, int group, int sm_count, int64_t max_len);
+cudaError_t launch_attn_rows(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows, int set,
+                             const __nv_bfloat16* q, const int32_t* sel_idx, int64_t sel_stride,
+                             const int32_t* sel_count, __nv_bfloat16* out, float* lse, void* ws,
+                             size_t ws_bytes, int64_t max_len, int32_t* status, int sm_count, cudaStream_t st);
+
+enum PrefillMode { kPrefillDense = 0, kPrefillLocal = 1, kPrefillSparse = 2 };
+cudaError_t launch_attn_prefill(const CacheView& cv, const Dims& d, const HeadMaps& hm, int mode,
+                                const __nv_bfloat16* q, const __nv_bfloat16* qt, int32_t seq_id, int32_t q_start,
+                                int64_t C, const float* sel_thresh, const int32_t* sel_tie_last,
+                                __nv_bfloat16* out, float* lse, int32_t* status, int sm_count, cudaStream_t st);
+
+}  // namespace rtp

@@ -145,14 +145,19 @@ def build_paged_cache(k: list, v: list, seed: int, capacity: list | None = None,
     nxt = 0
     for b in range(B):
         L = int(k[b].shape[0])
-        for pi in range(n_pages_seq[b]):
-            phys = int(perm[nxt]); nxt += 1
-            block_table[b, pi] = phys
-            lo = pi * PAGE_SIZE
-            hi = min(L, lo + PAGE_SIZE)
-            if hi > lo:
-                k_pages[phys, :, : hi - lo, :] = np.transpose(k[b][lo:hi], (1, 0, 2))
-                v_pages[phys, :, : hi - lo, :] = np.transpose(v[b][lo:hi], (1, 0, 2))
+        phys = perm[nxt: nxt + n_pages_seq[b]]
+        nxt += n_pages_seq[b]
+        block_table[b, : n_pages_seq[b]] = phys
+        full = L // PAGE_SIZE
+        if full:
+            kk = k[b][: full * PAGE_SIZE].reshape(full, PAGE_SIZE, hkv, HEAD_DIM)
+            vv = v[b][: full * PAGE_SIZE].reshape(full, PAGE_SIZE, hkv, HEAD_DIM)
+            k_pages[phys[:full]] = np.transpose(kk, (0, 2, 1, 3))
+            v_pages[phys[:full]] = np.transpose(vv, (0, 2, 1, 3))
+        rem = L - full * PAGE_SIZE
+        if rem:
+            k_pages[phys[full], :, :rem, :] = np.transpose(k[b][full * PAGE_SIZE:], (1, 0, 2))
+            v_pages[phys[full], :, :rem, :] = np.transpose(v[b][full * PAGE_SIZE:], (1, 0, 2))
     seq_lens = np.array([int(k[b].shape[0]) for b in range(B)], dtype=np.int32)
     return PagedCache(k_pages, v_pages, block_table, seq_lens, num_pages)
 

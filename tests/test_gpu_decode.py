@@ -1,0 +1,165 @@
+"""GPU parity of the decode path (S0-S5, S7-S9) against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_16928_b200 import binding as rb
+from paper_2605_16928_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _harness():
+    from tests import gpu_harness as gh
+    return gh
+
+
+def _run_decode(wl, sel_stride=None, check_rows=None, dense_heads=(0,)):
+    gh = _harness()
+    dw = gh.DeviceWorkload(wl, sel_stride=sel_stride)
+    dw.index_all_keys()
+    gh.check_index_keys(dw)
+    qt = gh.check_queries(dw)
+    sc = gh.check_scores(dw, qt, rows=check_rows)
+    sel = dw.select()
+    stats = gh.check_selection(dw, sc, sel, rows=check_rows)
+    out, lse = dw.sparse_decode()
+    gh.check_sparse_attention(dw, sel, out, lse, rows=check_rows)
+    if wl.heads.local_kv_heads:
+        lo, ll = dw.local_decode()
+        gh.check_range_attention(dw, lo, ll, wl.heads.local_kv_heads[:2], "local", rows=check_rows)
+        # slots of retrieval heads are not touched by the local call
+        assert np.all(lo[:, wl.heads.ret_q_heads] == 0)
+    do, dl = dw.dense_decode(list(dense_heads))
+    gh.check_range_attention(dw, do, dl, list(dense_heads), "dense", rows=check_rows)
+    assert dw.status_code() == rb.RTP_OK
+    return dw, stats
+
+
+def test_config1_single_decode_with_needles():
+    wl = synth.config_1()
+    dw, stats = _run_decode(wl)
+    c, k_star, n = stats[0]
+    assert n == 4096 and 1 <= c <= 16
+    got = set(dw.sel["idx"][0, 0, :c].cpu().numpy().tolist())
+    assert got <= set(wl.notes["needles"].tolist())          # only planted keys are selected
+
+
+@pytest.mark.parametrize("L", [1, 2, 63, 64, 65, 130, 1000])
+def test_config1_ragged_lengths(L):
+    _run_decode(synth.config_1(L=L, n_needles=min(8, max(1, L // 4))))
+
+
+def test_config2_reduced_with_ragged_batch():
+    wl = synth.config_2(L=3000, batch=4, window=512)
+    # make the batch ragged: shorten every sequence differently
+    for b, cut in enumerate([0, 517, 1, 2049]):
+        L = 3000 - cut
+        wl.k[b], wl.v[b] = wl.k[b][:L], wl.v[b][:L]
+        wl.seq_lens[b] = L
+        wl.row_pos[b] = L - 1
+    _run_decode(wl, dense_heads=(0, 5))
+
+
+def test_config2_full_size():
+    wl = synth.config_2()
+    dw, stats = _run_decode(wl, dense_heads=(1,))
+    peaked = [c for (c, k, n) in stats[: 4 * 8]]
+    flat = [c / n for (c, k, n) in stats[4 * 8:]]
+    assert max(peaked) <= 80                                  # needles only
+    assert 0.05 <= np.mean(flat) <= 0.35                      # iid keys: a two-digit percentage
+
+
+def test_config5_point_128k():
+    wl = synth.config_5(L=131072, batch=1, top_p=0.9, frac=0.05)
+    dw, stats = _run_decode(wl, sel_stride=40000, dense_heads=(7,))
+    fr = [c / n for (c, k, n) in stats]
+    assert 0.01 <= np.mean(fr) <= 0.12
+
+
+def test_top_p_one_selects_everything_and_equals_dense():
+    gh = _harness()
+    wl = synth.config_2(L=700, batch=2, window=512)
+    wl.top_p = 1.0
+    dw = gh.DeviceWorkload(wl)
+    dw.index_all_keys()
+    sel = dw.select()
+    assert np.all(sel["cnt"].cpu().numpy() == 700)
+    out, lse = dw.sparse_decode()
+    do, dl = dw.dense_decode(wl.heads.ret_kv_heads)
+    h = wl.heads.ret_q_heads
+    assert np.abs(out[:, h] - do[:, h]).max() <= 2e-2
+    gh.check_range_attention(dw, out, lse, wl.heads.ret_kv_heads, "dense")
+
+
+@pytest.mark.parametrize("L", [100, 5000, 9000])
+def test_equal_scores_take_lowest_positions(L):
+    """All index keys equal -> all scores tie; the canonical set is the first ceil(p L) positions.
+    L > 4096 exercises the exact-tie path that cannot buffer all candidates."""
+    gh = _harness()
+    wl = synth.config_1(L=L)
+    wl.k[0][:, 0, :] = wl.k[0][0, 0, :]                        # identical keys
+    dw = gh.DeviceWorkload(wl)
+    dw.index_all_keys()
+    sc = dw.scores()[0]
+    assert np.all(sc[0, 0, :L] == sc[0, 0, 0])
+    sel = dw.select()
+    c = int(sel["cnt"][0, 0])
+    want = int(np.ceil(0.9 * L - 1e-9))
+    assert want <= c <= want + int(2e-4 * L) + 1
+    assert sorted(sel["idx"][0, 0, :c].cpu().numpy().tolist()) == list(range(c))
+    assert int(sel["tie"][0, 0]) == c - 1
+    gh.check_selection(dw, sc, sel)
+
+
+def test_window_larger_than_context_equals_dense():
+    gh = _harness()
+    wl = synth.config_2(L=900, batch=2, window=4096)
+    dw = gh.DeviceWorkload(wl)
+    lo, ll = dw.local_decode()
+    do, dl = dw.dense_decode(wl.heads.local_kv_heads)
+    h = [kv * 4 + j for kv in wl.heads.local_kv_heads for j in range(4)]
+    assert np.array_equal(lo[:, h], do[:, h])
+    np.testing.assert_allclose(ll[:, h], dl[:, h], rtol=1e-6)
+
+
+def test_list_overflow_reports_capacity_and_true_count():
+    gh = _harness()
+    wl = synth.config_5(L=8192, batch=1, frac=0.2)
+    dw = gh.DeviceWorkload(wl, sel_stride=64)
+    dw.index_all_keys()
+    sel = dw.select()
+    cnt = sel["cnt"].cpu().numpy()
+    assert cnt.max() > 64
+    assert dw.status_code() == rb.RTP_ERR_CAPACITY
+    idx = sel["idx"].cpu().numpy()
+    assert np.all(idx >= 0) and np.all(idx < 8192)             # the first 64 ids of every row are valid
+
+
+def test_row_beyond_sequence_is_reported_not_trapped():
+    gh = _harness()
+    wl = synth.config_1(L=256)
+    wl.row_pos[0] = 300
+    dw = gh.DeviceWorkload(wl)
+    dw.index_all_keys()
+    dw.select()
+    assert dw.status_code() == rb.RTP_ERR_INVALID
+    assert int(dw.sel["cnt"][0, 0]) <= 256
+
+
+def test_host_side_argument_errors():
+    gh = _harness()
+    wl = synth.config_1(L=256)
+    dw = gh.DeviceWorkload(wl)
+    with pytest.raises(rb.RtpError) as e:
+        rb.rtp_topp_select(dw.ctx, dw.params, dw.cache, dw.q, dw.w_q, dw.row_seq, None, 0, 0, 1, None,
+                           torch.zeros(1, dtype=torch.int32, device="cuda"), None, None, None, dw.status, dw.workspace)
+    assert e.value.code == rb.RTP_ERR_INVALID
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(rb.RtpError) as e:
+        rb.rtp_topp_select(dw.ctx, dw.params, dw.cache, dw.q, dw.w_q, dw.row_seq, dw.row_pos, 0, 0, 1, None,
+                           torch.zeros(1, dtype=torch.int32, device="cuda"), None, None, None, dw.status, small)
+    assert e.value.code == rb.RTP_ERR_CAPACITY
+    bad = rb.Params.from_workload(wl, top_p=0.0)
+    with pytest.raises(rb.RtpError):
+        rb.rtp_index_queries(dw.ctx, bad, dw.q, dw.w_q, torch.empty((1, 1, 16), dtype=torch.bfloat16, device="cuda"))
