@@ -18,10 +18,11 @@ namespace rtp {
 
 namespace {
 
-constexpr int kWarps = 4;
+constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kHeadsPerCta = 4;
-constexpr int kStage = 256;   // staged ids per (warp, head) before a flush
+constexpr int kStage = 128;      // staged ids per (warp, head) before a flush
+constexpr int kCandStage = 48;   // staged boundary candidates per (warp, head)
 
 struct Bin {
   float mass;
@@ -336,7 +337,9 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
     const __nv_bfloat16* __restrict__ qt, SelState* __restrict__ state, uint2* __restrict__ cand,
     int32_t* __restrict__ sel_idx, int64_t sel_stride, int n_splits, int32_t* status) {
   __shared__ int stage[kWarps][kHeadsPerCta][kStage];
+  __shared__ uint2 cstage[kWarps][kHeadsPerCta][kCandStage];
   __shared__ int stage_cnt[kWarps][kHeadsPerCta];
+  __shared__ int cstage_cnt[kWarps][kHeadsPerCta];
 
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
   const int z = blockIdx.z;
@@ -354,17 +357,22 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
     lo_key = st->lo_key;
     hi_key = st->hi_key;
   }
-  if (lane < kHeadsPerCta) stage_cnt[warp][lane] = 0;
+  if (lane < kHeadsPerCta) {
+    stage_cnt[warp][lane] = 0;
+    cstage_cnt[warp][lane] = 0;
+  }
   __syncwarp();
   const bool emit_ids = sel_idx != nullptr;
   const QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
 
-  auto flush = [&](int jj) {  // warp-uniform
+  auto row_head = [&](int jj) -> int64_t {
+    const int slot2 = (z >> 1) * 8 + (z & 1) * 4 + jj;
+    return x.r * d.n_ret + hm.ih_heads[x.ih][slot2];
+  };
+  auto flush_ids = [&](int jj) {  // warp-uniform
     const int n = stage_cnt[warp][jj];
     if (n == 0) return;
-    const int slot2 = (z >> 1) * 8 + (z & 1) * 4 + jj;
-    const int hd = hm.ih_heads[x.ih][slot2];
-    const int64_t rh = x.r * d.n_ret + hd;
+    const int64_t rh = row_head(jj);
     int gbase = 0;
     if (lane == 0) gbase = atomicAdd(&state[rh].emit_cnt, n);
     gbase = __shfl_sync(0xffffffffu, gbase, 0);
@@ -374,6 +382,27 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
     __syncwarp();
     if (lane == 0) stage_cnt[warp][jj] = 0;
     __syncwarp();
+  };
+  auto flush_cands = [&](int jj) {  // warp-uniform
+    const int n = cstage_cnt[warp][jj];
+    if (n == 0) return;
+    const int64_t rh = row_head(jj);
+    int gbase = 0;
+    if (lane == 0) gbase = atomicAdd(&state[rh].cand_cnt, n);
+    gbase = __shfl_sync(0xffffffffu, gbase, 0);
+    for (int i = lane; i < n; i += 32)
+      if (gbase + i < kCandCap) cand[rh * kCandCap + gbase + i] = cstage[warp][jj][i];
+    __syncwarp();
+    if (lane == 0) cstage_cnt[warp][jj] = 0;
+    __syncwarp();
+  };
+  // Appends the entries flagged in `flags` (bit e = key n0 + e) of every head to a per-warp stage.
+  auto group_offsets = [&](int k, int& incl) {
+    incl = k;
+    int t = __shfl_up_sync(0xffffffffu, incl, 1, 4);
+    if (c >= 1) incl += t;
+    t = __shfl_up_sync(0xffffffffu, incl, 2, 4);
+    if (c >= 2) incl += t;
   };
 
   for (int p = x.p_lo + warp; p < x.p_hi; p += kWarps) {
@@ -386,7 +415,10 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
       float s_lo[4], s_hi[4];
       score16(qf, v[i], lane, s_lo, s_hi);
       const int n0 = p * kPage + i * 16 + 4 * c;
-      int flags = 0;
+      int flags = 0, cflags = 0;
+      uint32_t keys4[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) keys4[e] = okey(finish_score(use_hi ? s_hi[e] : s_lo[e], d.score_scale));
       if (mode == kSelectAll) {
 #pragma unroll
         for (int e = 0; e < 4; ++e)
@@ -395,40 +427,54 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           if (n0 + e >= x.n_keys) continue;
-          const uint32_t key = okey(finish_score(use_hi ? s_hi[e] : s_lo[e], d.score_scale));
-          if (key > hi_key) {
+          if (keys4[e] > hi_key)
             flags |= 1 << e;
-          } else if (key >= lo_key && mode == kCollect) {
-            const int slot_c = atomicAdd(&st->cand_cnt, 1);
-            if (slot_c < kCandCap) cand[(x.r * d.n_ret + head) * kCandCap + slot_c] = make_uint2(key, n0 + e);
-          }
+          else if (keys4[e] >= lo_key && mode == kCollect)
+            cflags |= 1 << e;
         }
       }
-      if (!emit_ids) continue;
-      // append the flagged ids of each head to the warp's staging buffer
-      const int k = __popc(flags);
-      int incl = k;
-      int t = __shfl_up_sync(0xffffffffu, incl, 1, 4);
-      if (c >= 1) incl += t;
-      t = __shfl_up_sync(0xffffffffu, incl, 2, 4);
-      if (c >= 2) incl += t;
-      if (head >= 0 && k) {
-        int w = stage_cnt[warp][j] + incl - k;
+      // boundary candidates
+      {
+        const int k = __popc(cflags);
+        int incl;
+        group_offsets(k, incl);
+        if (head >= 0 && k) {
+          int w = cstage_cnt[warp][j] + incl - k;
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if (flags & (1 << e)) stage[warp][j][w++] = n0 + e;
+          for (int e = 0; e < 4; ++e)
+            if (cflags & (1 << e)) cstage[warp][j][w++] = make_uint2(keys4[e], (uint32_t)(n0 + e));
+        }
+        __syncwarp();
+        if (head >= 0 && c == 3 && incl) cstage_cnt[warp][j] += incl;
+        __syncwarp();
+#pragma unroll
+        for (int jj = 0; jj < kHeadsPerCta; ++jj)
+          if (cstage_cnt[warp][jj] > kCandStage - 16) flush_cands(jj);
       }
-      __syncwarp();
-      if (head >= 0 && c == 3 && incl) stage_cnt[warp][j] += incl;
-      __syncwarp();
+      if (!emit_ids) continue;
+      {
+        const int k = __popc(flags);
+        int incl;
+        group_offsets(k, incl);
+        if (head >= 0 && k) {
+          int w = stage_cnt[warp][j] + incl - k;
 #pragma unroll
-      for (int jj = 0; jj < kHeadsPerCta; ++jj)
-        if (stage_cnt[warp][jj] > kStage - 16) flush(jj);
+          for (int e = 0; e < 4; ++e)
+            if (flags & (1 << e)) stage[warp][j][w++] = n0 + e;
+        }
+        __syncwarp();
+        if (head >= 0 && c == 3 && incl) stage_cnt[warp][j] += incl;
+        __syncwarp();
+#pragma unroll
+        for (int jj = 0; jj < kHeadsPerCta; ++jj)
+          if (stage_cnt[warp][jj] > kStage - 16) flush_ids(jj);
+      }
     }
   }
-  if (emit_ids) {
 #pragma unroll
-    for (int jj = 0; jj < kHeadsPerCta; ++jj) flush(jj);
+  for (int jj = 0; jj < kHeadsPerCta; ++jj) {
+    flush_cands(jj);
+    if (emit_ids) flush_ids(jj);
   }
 }
 
@@ -657,7 +703,7 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
 int select_splits(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
   const int64_t pages = (max_len + kPage - 1) / kPage;
   int64_t want = (4LL * sm_count + R * d.n_ih - 1) / (R * d.n_ih);
-  int64_t cap = (pages + 63) / 64;  // at least 64 pages (4096 keys) per CTA
+  int64_t cap = (pages + 31) / 32;  // at least 32 pages (2048 keys) per CTA
   int64_t s = want < cap ? want : cap;
   if (s < 1) s = 1;
   if (s > 4096) s = 4096;

@@ -152,7 +152,11 @@ def check_index_keys(dw: DeviceWorkload):
         for j in range(wl.heads.n_index_heads):
             want = orc.index_project(kp[:, j], wl.w_k[j])
             d = bf16_ulp_diff(got[:, j], want)
-            assert d.max() <= 1, f"index key off by {d.max()} bf16 steps"
+            # one bf16 step, except where cancellation leaves a result so small that the fp32
+            # accumulation error (a few 2^-24 of the sum of magnitudes) spans several steps
+            floor = np.abs(orc.bf16_to_f64(kp[:, j])) @ np.abs(orc.bf16_to_f64(wl.w_k[j])) * 2.0 ** -21
+            bad = (d > 1) & (np.abs(orc.bf16_to_f64(got[:, j]) - orc.bf16_to_f64(want)) > floor)
+            assert not bad.any(), f"index key off by {d[bad].max()} bf16 steps"
             total += d.size
             equal += int((d == 0).sum())
     assert equal >= 0.999 * total, f"only {equal}/{total} index keys bit-equal"
@@ -164,7 +168,9 @@ def check_queries(dw: DeviceWorkload) -> np.ndarray:
     for i, h in enumerate(wl.heads.ret_q_heads):
         want = orc.index_project(wl.q[:, h], wl.w_q[i])
         d = bf16_ulp_diff(qt[:, i], want)
-        assert d.max() <= 1
+        floor = np.abs(orc.bf16_to_f64(wl.q[:, h])) @ np.abs(orc.bf16_to_f64(wl.w_q[i])) * 2.0 ** -21
+        bad = (d > 1) & (np.abs(orc.bf16_to_f64(qt[:, i]) - orc.bf16_to_f64(want)) > floor)
+        assert not bad.any()
     return qt
 
 
@@ -259,4 +265,130 @@ def check_range_attention(dw: DeviceWorkload, out, lse, kv_heads, kind: str, row
                     want, wlse = orc.dense_row(wl.q[r, h], wl.k[b][:, kv], wl.v[b][:, kv], m, wl.sm_scale)
                 err = np.abs(out[r, h] - want).max()
                 assert err <= tol, f"{kind} row {r} head {h}: max abs err {err}"
+                assert abs(lse[r, h] - wlse) <= 1e-3 * max(1.0, abs(wlse))
+
+
+# ------------------------------------------------------------------ prefill helpers
+class PrefillRun:
+    """Chunked prefill of a one-sequence workload whose query rows are positions 0..L-1."""
+
+    def __init__(self, dw: DeviceWorkload):
+        self.dw = dw
+        wl = dw.wl
+        self.L = int(wl.seq_lens[0])
+        self.Hq = wl.heads.n_q_heads
+        self.n_ret = dw.n_ret
+
+    def select_chunk(self, q_start: int, C: int, with_lists: bool = True, stride: int | None = None):
+        dw = self.dw
+        stride = stride or (q_start + C)
+        idx = torch.full((C, self.n_ret, stride), -1, dtype=torch.int32, device=DEV) if with_lists else None
+        cnt = torch.full((C, self.n_ret), -7, dtype=torch.int32, device=DEV)
+        mass = torch.zeros((C, self.n_ret), dtype=torch.float32, device=DEV)
+        thr = torch.zeros((C, self.n_ret), dtype=torch.float32, device=DEV)
+        tie = torch.zeros((C, self.n_ret), dtype=torch.int32, device=DEV)
+        q = dw.q[q_start:q_start + C]
+        rb.rtp_topp_select(dw.ctx, dw.params, dw.cache, q, dw.w_q, None, None, 0, q_start, C, idx, cnt, mass, thr,
+                           tie, dw.status, dw.workspace)
+        torch.cuda.synchronize()
+        return dict(idx=idx, cnt=cnt, mass=mass, thr=thr, tie=tie)
+
+    def sparse_prefill(self, q_start: int, C: int, sel: dict, use_lists: bool):
+        dw = self.dw
+        out = torch.zeros((C, self.Hq, 128), dtype=torch.bfloat16, device=DEV)
+        lse = torch.zeros((C, self.Hq), dtype=torch.float32, device=DEV)
+        q = dw.q[q_start:q_start + C]
+        rb.rtp_sparse_attn_prefill(dw.ctx, dw.params, dw.cache, q, q, dw.w_q, 0, q_start, C,
+                                   sel["idx"] if use_lists else None, sel["cnt"], sel["thr"], sel["tie"], out, lse,
+                                   dw.workspace, dw.status)
+        torch.cuda.synchronize()
+        return out.float().cpu().numpy(), lse.cpu().numpy()
+
+    def local_prefill(self, q_start: int, C: int):
+        dw = self.dw
+        out = torch.zeros((C, self.Hq, 128), dtype=torch.bfloat16, device=DEV)
+        lse = torch.zeros((C, self.Hq), dtype=torch.float32, device=DEV)
+        rb.rtp_local_attn(dw.ctx, dw.params, dw.cache, dw.q[q_start:q_start + C], None, None, 0, q_start, C, out, lse,
+                          dw.workspace, dw.status)
+        torch.cuda.synchronize()
+        return out.float().cpu().numpy(), lse.cpu().numpy()
+
+    def dense_prefill(self, q_start: int, C: int, kv_heads=None):
+        dw = self.dw
+        out = torch.zeros((C, self.Hq, 128), dtype=torch.bfloat16, device=DEV)
+        lse = torch.zeros((C, self.Hq), dtype=torch.float32, device=DEV)
+        rb.rtp_dense_attn_prefill(dw.ctx, dw.params, dw.cache, dw.q[q_start:q_start + C], 0, q_start, C, kv_heads, out,
+                                  lse, dw.status)
+        torch.cuda.synchronize()
+        return out.float().cpu().numpy(), lse.cpu().numpy()
+
+    def scores_for_rows(self, rows):
+        """Materialised GPU scores of the given positions (explicit-row entry point)."""
+        dw = self.dw
+        rows = np.asarray(rows, dtype=np.int32)
+        q = dw.q[torch.from_numpy(rows.astype(np.int64)).to(DEV)].contiguous()
+        sc = torch.full((len(rows), self.n_ret, self.L), float("nan"), dtype=torch.float32, device=DEV)
+        ws = torch.empty(max(1 << 20, rb.rtp_workspace_bytes(dw.params, len(rows), self.L)), dtype=torch.uint8, device=DEV)
+        rb.rtp_index_score(dw.ctx, dw.params, dw.cache, q, dw.w_q, dev_i32(np.zeros(len(rows))), dev_i32(rows), sc,
+                           None, None, ws, dw.status)
+        torch.cuda.synchronize()
+        return sc.cpu().numpy()
+
+
+def check_chunk_selection(pr: PrefillRun, q_start: int, sel: dict, rows, p=None):
+    """rows: absolute positions inside the chunk.  Uses the GPU's own scores."""
+    wl = pr.dw.wl
+    p = wl.top_p if p is None else p
+    sc = pr.scores_for_rows(rows)
+    idx = sel["idx"].cpu().numpy() if sel["idx"] is not None else None
+    cnt, mass = sel["cnt"].cpu().numpy(), sel["mass"].cpu().numpy()
+    thr, tie = sel["thr"].cpu().numpy(), sel["tie"].cpu().numpy()
+    fracs = []
+    for k, m in enumerate(rows):
+        r = m - q_start
+        for i in range(pr.n_ret):
+            s = sc[k, i, : m + 1]
+            c = int(cnt[r, i])
+            assert 1 <= c <= m + 1, f"row {m} head {i}: count {c}"
+            member = (s > thr[r, i]) | ((s == thr[r, i]) & (np.arange(m + 1) <= tie[r, i]))
+            assert int(member.sum()) == c, f"row {m} head {i}: rule gives {int(member.sum())}, count {c}"
+            got = set(np.nonzero(member)[0].tolist())
+            if idx is not None and c <= idx.shape[-1]:
+                lst = idx[r, i, :c]
+                assert set(lst.tolist()) == got and len(set(lst.tolist())) == c
+                assert np.all(idx[r, i, c:] == -1)
+            mand, forb = orc.classify_against_band(s, p)
+            assert mand <= got, f"row {m} head {i}: {len(mand - got)} mandatory tokens missing"
+            assert not (forb & got), f"row {m} head {i}: {len(forb & got)} forbidden tokens selected"
+            tm = orc.set_mass(s, got)
+            assert tm >= p or c == m + 1
+            assert abs(mass[r, i] - tm) <= 1e-4
+            fracs.append(c / (m + 1))
+    return sc, fracs
+
+
+def check_prefill_rows(pr: PrefillRun, q_start: int, out, lse, rows, kind: str, kv_heads, sets=None, tol=2e-2):
+    """kind: dense | local | sparse (sets[(m, i)] = ids for retrieval head i)."""
+    wl = pr.dw.wl
+    g = wl.heads.group
+    for m in rows:
+        r = m - q_start
+        if kind == "sparse":
+            for i, h in enumerate(wl.heads.ret_q_heads):
+                want, wlse = orc.attention_over_set(wl.q[m, h], wl.k[0][:, h // g], wl.v[0][:, h // g], sets[(m, i)],
+                                                    wl.sm_scale)
+                err = np.abs(out[r, h] - want).max()
+                assert err <= tol, f"sparse row {m} head {h}: {err}"
+                assert abs(lse[r, h] - wlse) <= 1e-3 * max(1.0, abs(wlse))
+            continue
+        for kv in kv_heads:
+            for j in range(g):
+                h = kv * g + j
+                if kind == "local":
+                    want, wlse = orc.local_row(wl.q[m, h], wl.k[0][:, kv], wl.v[0][:, kv], m, wl.heads.n_sink,
+                                               wl.heads.window, wl.sm_scale)
+                else:
+                    want, wlse = orc.dense_row(wl.q[m, h], wl.k[0][:, kv], wl.v[0][:, kv], m, wl.sm_scale)
+                err = np.abs(out[r, h] - want).max()
+                assert err <= tol, f"{kind} row {m} head {h}: {err}"
                 assert abs(lse[r, h] - wlse) <= 1e-3 * max(1.0, abs(wlse))
