@@ -12,8 +12,8 @@
 //   pass 2+  64-bin (mass, count) histograms of the ordered score key inside the bucket, 6 key bits
 //            per pass, until the bucket holds one key or all 32 key bits are fixed
 //   tie pass only when equal scores straddle the cut: position of the last tie taken
-//   emit     only when id lists are requested
-// Rows drop out as soon as they are resolved; the CTA stops when all its rows are.
+// Rows drop out as soon as they are resolved; the CTA stops when all its rows are.  When id lists
+// are requested, one more sweep appends every row's members in position order.
 #include "rtp_device.cuh"
 
 namespace rtp {
@@ -36,7 +36,7 @@ struct RowState {      // one per (row, head), in shared memory
   uint32_t base_key;   // level >= 2: bin = (key - base_key) >> shift, in [0, 64)
   int32_t shift;
   int32_t b1;          // level-1 bucket
-  int32_t phase;       // 0 max, 1 level-1, 2 key levels, 3 tie pass, 4 done
+  int32_t phase;       // 0 max, 1 level-1, 2 key levels, 3 tie pass, 4 resolved
   int32_t cnt_above;   // keys strictly above the current bucket
   int32_t tie_need;    // tie pass: number of ties to take
   uint32_t thr_key;    // result: selected <=> key > thr_key or (key == thr_key and n <= tie_last)
@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
     z.n_keys = ok ? min(m0 + po, seq_len - 1) + 1 : 0;
     z.phase = ok && z.n_keys > 0 ? 0 : 4;
     if (ok && z.n_keys > 0 && (d.top_p >= 1.0f || z.n_keys == 1)) {   // everything is selected
-      z.phase = sel_idx != nullptr ? 5 : 4;
+      z.phase = 4;
       z.thr_key = 0u;
       z.tie_last = z.n_keys - 1;
       z.count = z.n_keys;
@@ -155,7 +155,9 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
     // zero this warp's histograms
     for (int i = lane; i < 16 * kL1Bins; i += 32) hist[wrow * kL1Bins + i] = 0.f;
     __syncthreads();
-    const bool warp_active = __any_sync(0xffffffffu, (ph_a != 4 && ph_a != 6) || (ph_b != 4 && ph_b != 6));
+    const bool warp_active = __any_sync(0xffffffffu, ph_a != 4 || ph_b != 4);
+    // some row of the warp needs keys counted / written in position order this pass
+    const bool order_pass = __any_sync(0xffffffffu, ph_a == 3 || ph_b == 3);
 
     float mx_a = -INFINITY, mx_b = -INFINITY;   // phase 0
     int cnt_a = 0, cnt_b = 0;                   // phase 2: keys above the level-1 bucket (first key level only)
@@ -191,7 +193,7 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
               const int n = n_page + nt * 8 + 2 * c + (e & 1);
               const int pos = lo_row ? pos_a : pos_b;
               const int ph = lo_row ? ph_a : ph_b;
-              if (n > pos || ph == 4 || ph == 6) continue;
+              if (n > pos || ph == 4) continue;
               const float s = finish_score(s4[e], d.score_scale);
               const RowState& S = lo_row ? sa : sb;
               if (ph == 0) {
@@ -220,14 +222,10 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
                 if (okey(s) == S.thr_key) {
                   if (lo_row) tf_a |= 1 << (e & 1); else tf_b |= 1 << (e & 1);
                 }
-              } else if (ph == 5) {
-                const uint32_t key = okey(s);
-                if (key > S.thr_key || (key == S.thr_key && n <= S.tie_last)) {
-                  if (lo_row) tf_a |= 1 << (e & 1); else tf_b |= 1 << (e & 1);
-                }
               }
             }
-            if (__any_sync(0xffffffffu, ph_a == 3 || ph_b == 3 || ph_a == 5 || ph_b == 5)) {
+            __syncwarp();
+            if (order_pass) {
               // in-order prefix of the flagged keys inside the quad (lane c holds keys 2c, 2c+1 of the n8 tile)
               const int ka = __popc(tf_a), kb = __popc(tf_b);
               int ia = ka, ib = kb, t;
@@ -241,21 +239,11 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
                 int before = run_a + ia - ka;
                 for (int e = 0; e < 2; ++e)
                   if (tf_a & (1 << e)) { if (before < sa.tie_need) tl_a = max(tl_a, n_first + e); ++before; }
-              } else if (ph_a == 5 && ka) {
-                int w = run_a + ia - ka;
-                int32_t* dst = sel_idx + ((int64_t)(r0 + pofs + g) * d.n_ret + rh_head) * sel_stride;
-                for (int e = 0; e < 2; ++e)
-                  if (tf_a & (1 << e)) { if (w < sel_stride) dst[w] = n_first + e; ++w; }
               }
               if (ph_b == 3) {
                 int before = run_b + ib - kb;
                 for (int e = 0; e < 2; ++e)
                   if (tf_b & (1 << e)) { if (before < sb.tie_need) tl_b = max(tl_b, n_first + e); ++before; }
-              } else if (ph_b == 5 && kb) {
-                int w = run_b + ib - kb;
-                int32_t* dst = sel_idx + ((int64_t)(r0 + pofs + g + 8) * d.n_ret + rh_head) * sel_stride;
-                for (int e = 0; e < 2; ++e)
-                  if (tf_b & (1 << e)) { if (w < sel_stride) dst[w] = n_first + e; ++w; }
               }
               run_a += tot_a;
               run_b += tot_b;
@@ -293,7 +281,7 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
       const int ph = R.phase;
       const int src_lane = (rr & 7) * 4;          // a lane of the quad that owns row rr
       const bool is_b = rr >= 8;
-      if (ph == 4 || ph == 6 || R.n_keys == 0) continue;
+      if (ph == 4 || R.n_keys == 0) continue;
       if (ph == 0) {
         const float M = __shfl_sync(0xffffffffu, is_b ? mx_b : mx_a, src_lane);
         if (lane == 0) {
@@ -348,7 +336,7 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
             S->tie_last = R.n_keys - 1;
             S->count = R.n_keys;
             S->sel_mass = 1.0f;
-            S->phase = want_ids ? 5 : 4;
+            S->phase = 4;
           } else {
             // key range that certainly contains the bucket: scores in (M - (b+1)/4, M - b/4], widened
             const float hi_s = R.M - (float)best / kL1Scale, lo_s = R.M - (float)(best + 1) / kL1Scale;
@@ -402,7 +390,7 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
         if (best >= 64) {
           // empty bucket: cannot happen (the level-1 bucket holds at least one key)
           if (lane == 0) {
-            S->phase = want_ids ? 6 : 4;
+            S->phase = 4;
             set_status(status, RTP_ERR_UNSUPPORTED);
           }
         } else if (best == bhi || best == blo) {
@@ -434,7 +422,7 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
               S->phase = 3;
             } else {
               S->tie_last = R.n_keys - 1;
-              S->phase = want_ids ? 5 : 4;
+              S->phase = 4;
             }
           } else {
             S->shift = max(0, shift - 6);
@@ -444,25 +432,85 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
         const int tl = __shfl_sync(0xffffffffu, is_b ? tl_b : tl_a, src_lane);
         if (lane == 0) {
           S->tie_last = tl;
-          S->phase = want_ids ? 5 : 4;
-        }
-      } else if (ph == 5) {
-        if (lane == 0) {
-          if (R.count > sel_stride) set_status(status, RTP_ERR_CAPACITY);
-          S->phase = 6;
+          S->phase = 4;
         }
       }
     }
     __syncwarp();
     {
       int pend = 0;
-      if (a_ok && rs[la].phase != 4 && rs[la].phase != 6) pend = 1;
-      if (b_ok && rs[lb].phase != 4 && rs[lb].phase != 6) pend = 1;
+      if (a_ok && rs[la].phase != 4) pend = 1;
+      if (b_ok && rs[lb].phase != 4) pend = 1;
       if (pend) s_pending = 1;
     }
     __syncthreads();
     if (!s_pending) break;
     __syncthreads();
+  }
+
+  // ---- id lists: one more sweep over the keys, every resolved row appends its members in position order ----
+  if (want_ids) {
+    __syncthreads();
+    const RowState sa = rs[la], sb = rs[lb];
+    const bool em_a = a_ok && sa.phase == 4 && sa.n_keys > 0, em_b = b_ok && sb.phase == 4 && sb.n_keys > 0;
+    int32_t* dst_a = sel_idx + ((int64_t)(r0 + pofs + g) * d.n_ret + rh_head) * sel_stride;
+    int32_t* dst_b = sel_idx + ((int64_t)(r0 + pofs + g + 8) * d.n_ret + rh_head) * sel_stride;
+    int run_a = 0, run_b = 0;
+    load_stage(0, 0);
+    asm volatile("cp.async.commit_group;");
+    for (int sidx = 0; sidx < n_stages; ++sidx) {
+      const int buf = sidx & 1;
+      if (sidx + 1 < n_stages) load_stage(sidx + 1, buf ^ 1);
+      asm volatile("cp.async.commit_group;");
+      asm volatile("cp.async.wait_group 1;");
+      __syncthreads();
+      if (warp_ok) {
+        const unsigned char* st = stage_s + buf * kStageBytesC;
+        const int boff = 2 * qfrag_dim_offset(lane);
+#pragma unroll 1
+        for (int pg = 0; pg < kPagesPerStage; ++pg) {
+          const int n_page = (sidx * kPagesPerStage + pg) * kPage;
+          if (n_page > warp_m_hi) break;
+#pragma unroll 1
+          for (int nt = 0; nt < 8; ++nt) {
+            const uint2 b = *reinterpret_cast<const uint2*>(st + (pg * kPage + nt * 8 + g) * (kIndexDim * 2) + boff);
+            const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+            float s4[4];
+            mma_bf16_16816(s4, iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
+            const int n_first = n_page + nt * 8 + 2 * c;
+            int fa = 0, fb = 0;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int n = n_first + e;
+              const uint32_t ka_ = okey(finish_score(s4[e], d.score_scale));
+              const uint32_t kb_ = okey(finish_score(s4[2 + e], d.score_scale));
+              if (em_a && n <= pos_a && (ka_ > sa.thr_key || (ka_ == sa.thr_key && n <= sa.tie_last))) fa |= 1 << e;
+              if (em_b && n <= pos_b && (kb_ > sb.thr_key || (kb_ == sb.thr_key && n <= sb.tie_last))) fb |= 1 << e;
+            }
+            const int ka = __popc(fa), kb = __popc(fb);
+            int ia = ka, ib = kb, tt;
+            tt = __shfl_up_sync(0xffffffffu, ia, 1, 4); if (c >= 1) ia += tt;
+            tt = __shfl_up_sync(0xffffffffu, ia, 2, 4); if (c >= 2) ia += tt;
+            tt = __shfl_up_sync(0xffffffffu, ib, 1, 4); if (c >= 1) ib += tt;
+            tt = __shfl_up_sync(0xffffffffu, ib, 2, 4); if (c >= 2) ib += tt;
+            const int tot_a = __shfl_sync(0xffffffffu, ia, 3, 4), tot_b = __shfl_sync(0xffffffffu, ib, 3, 4);
+            int wa = run_a + ia - ka, wb = run_b + ib - kb;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              if (fa & (1 << e)) { if (wa < sel_stride) dst_a[wa] = n_first + e; ++wa; }
+              if (fb & (1 << e)) { if (wb < sel_stride) dst_b[wb] = n_first + e; ++wb; }
+            }
+            run_a += tot_a;
+            run_b += tot_b;
+          }
+        }
+      }
+      __syncthreads();
+    }
+    asm volatile("cp.async.wait_group 0;");
+    if (c == 0) {
+      if ((em_a && run_a > sel_stride) || (em_b && run_b > sel_stride)) set_status(status, RTP_ERR_CAPACITY);
+    }
   }
 
   // ---- results ----
@@ -471,7 +519,7 @@ __global__ void __launch_bounds__(kCThreads) select_chunk_kernel(
     if (hs < nh && po < rows_here) {
       const RowState& S = rs[tid];
       const int64_t o = (int64_t)(r0 + po) * d.n_ret + hm.ih_heads[ih][hs];
-      const bool done = S.phase == 4 || S.phase == 6;
+      const bool done = S.phase == 4;
       if (!done) set_status(status, RTP_ERR_TIMEOUT);
       sel_count[o] = S.n_keys == 0 ? 0 : S.count;
       if (sel_mass) sel_mass[o] = S.sel_mass;

