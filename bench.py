@@ -1,0 +1,436 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse-attention hot path on B200.
+
+Default workload ("c3"): chunked prefill of one 128K-token sequence (32 query / 8 KV heads, 2 retrieval
+KV heads with a 16-dim indexer and top-p 0.9, 6 local heads with 4 sinks + 8192 window, chunk 8192).
+One step = the whole hot path over the sequence: per chunk, index-key projection and append, fused
+indexer + top-p thresholds, threshold-masked sparse attention on retrieval heads and sink+window
+attention on local heads.  Metric: prefill tokens per second.
+
+The JSON line also carries the dense in-library baseline, decode-step latencies (sparse path vs dense
+split-KV decode), the roofline of the dominant kernel and the CPU oracle timed on the host cores.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c3|c2|c5]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(prefix="clocks_", suffix=".csv")
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1])); mx.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"],
+                                     parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out["sm_mhz"] = float(np.median(sm)); out["sm_max_mhz"] = float(max(mx)); out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def ev_time_ms(fn, stream):
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream); fn(); e1.record(stream); e1.synchronize()
+    return e0.elapsed_time(e1)
+
+
+# ------------------------------------------------------------------------------------------------ prefill
+def prefill_tile_flops(L: int, chunk: int, group: int, n_kv_heads: int, mode: str, n_sink: int, window: int) -> float:
+    """FLOPs of the key tiles a prefill kernel visits: 128 MMA rows x 64 keys x 128 dims x (QK^T + PV)."""
+    bmp = 128 // group
+    per_tile = 128 * 64 * 128 * 2 * 2
+    tiles = 0
+    for q_start in range(0, L, chunk):
+        C = min(chunk, L - q_start)
+        for r0 in range(0, C, bmp):
+            m0 = q_start + r0
+            m_last = m0 + min(bmp, C - r0) - 1
+            kt_last = m_last // 64
+            if mode == "local":
+                kt_first = max(0, m0 - window + 1) // 64
+                tiles += min((n_sink + 63) // 64, kt_first) + kt_last - kt_first + 1
+            else:
+                tiles += kt_last + 1
+    return float(tiles) * per_tile * n_kv_heads
+
+
+def bench_prefill(args, rank, world, device):
+    import torch
+    from paper_2605_16928_b200 import synth_device, pipeline
+    L, chunk = args.seq_len or 131072, args.chunk or 8192
+    data = synth_device.config_3_device(L=L, device=device)
+    path = pipeline.PrefillPath(data, chunk)
+    stream = torch.cuda.current_stream()
+    out = torch.empty((L, path.Hq, 128), dtype=torch.bfloat16, device=device)
+    k_pre = data.k_pre_rows(0, 0, L)
+    chunks = path.chunks()
+
+    def step():
+        for (s, C) in chunks:
+            path.run_chunk(s, C, data.q[s:s + C], k_pre[s:s + C], out[s:s + C])
+
+    def step_dense():
+        for (s, C) in chunks:
+            path.run_chunk_dense(s, C, data.q[s:s + C], out[s:s + C])
+
+    return data, path, step, step_dense, out, k_pre, chunks, L, chunk, stream
+
+
+def cpu_oracle_prefill(data, L, rows, budget_s=25.0):
+    """Times the CPU oracle on a bounded sample of query rows of the prefill workload (all 32 heads)."""
+    from oracle import rtp_oracle as orc
+    heads = data.heads
+    g = heads.group
+    to_np = lambda t: t.contiguous().view(__import__("torch").int16).cpu().numpy().view(np.uint16)
+    kv = {h: data.logical_kv(0, h, 0, L) for h in range(heads.n_kv_heads)}
+    q = to_np(data.q[[int(r) for r in rows]])
+    w_q, w_k = to_np(data.w_q), to_np(data.w_k)
+    t0 = time.perf_counter()
+    kt = [orc.index_project(kv[heads.index_head_kv[j]][0], w_k[j]) for j in range(heads.n_index_heads)]
+    t_proj = time.perf_counter() - t0
+    done, t_rows = 0, 0.0
+    for k, m in enumerate(rows):
+        t1 = time.perf_counter()
+        for i, h in enumerate(heads.ret_q_heads):
+            kh = h // g
+            orc.retrieval_row(q[k, h], q[k, h], w_q[i], kt[heads.q_head_to_index_head[i]], kv[kh][0], kv[kh][1],
+                              int(m), data.top_p, data.score_scale, data.sm_scale)
+        for kh in heads.local_kv_heads:
+            for j in range(g):
+                orc.local_row(q[k, kh * g + j], kv[kh][0], kv[kh][1], int(m), heads.n_sink, heads.window, data.sm_scale)
+        t_rows += time.perf_counter() - t1
+        done += 1
+        if t_rows + t_proj > budget_s:
+            break
+    per_tok = t_rows / done + t_proj / L
+    return 1.0 / per_tok, done, t_rows + t_proj
+
+
+# ------------------------------------------------------------------------------------------------ decode extras
+def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, iters=20):
+    import torch
+    from paper_2605_16928_b200 import synth_device, pipeline
+    data = synth_device.decode_device(L, B, top_p, frac, window, device=device, peaked_half=peaked_half, name=name)
+    stride = int(min(L, max(4096, 4 * frac * L)))
+    path = pipeline.DecodePath(data, stride)
+    path.build_index_cache()
+    k_pre_new = data.k_pre_rows(0, L - 1, L).repeat(B, 1, 1).contiguous()
+    for b in range(B):
+        k_pre_new[b] = data.k_pre_rows(b, L - 1, L)[0]
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(192 << 20, dtype=torch.uint8, device=device)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        ts = []
+        for _ in range(iters):
+            flush.zero_()
+            ts.append(ev_time_ms(fn, stream) * 1e3)
+        return float(np.median(ts))
+
+    t_sparse = timed(lambda: path.step(data.q, k_pre_new))
+    t_dense = timed(lambda: path.step_dense(data.q))
+    cnt = path.sel_cnt.float()
+    n_ih = data.heads.n_index_heads
+    sel_rows = float(cnt.sum().item())
+    alg_bytes = B * n_ih * 32.0 * L + 512.0 * sel_rows + 8.0 * sel_rows + \
+        B * len(data.heads.local_kv_heads) * 512.0 * min(L, 4 + window)
+    res = {"workload": name, "batch": B, "context": L, "top_p": top_p,
+           "selected_fraction_mean": float(cnt.mean().item()) / L,
+           "sparse_step_us": t_sparse, "dense_step_us": t_dense, "speedup_vs_dense": t_dense / t_sparse,
+           "algorithmic_bytes": alg_bytes, "sparse_path_gbs": alg_bytes / t_sparse / 1e3,
+           "dense_gbs": B * data.heads.n_kv_heads * 512.0 * L / t_dense / 1e3,
+           "status": path.status_code()}
+    del path, data
+    torch.cuda.empty_cache()
+    return res
+
+
+# ------------------------------------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--seq-len", type=int, default=0)
+    ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--no-extras", action="store_true", help="skip the dense baseline, decode points and CPU oracle")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    n_cores = len(os.sched_getaffinity(0))
+    L, chunk = args.seq_len or 131072, args.chunk or 8192
+    config = {"workload": "c3_chunked_prefill_128k" if L == 131072 else f"c3_chunked_prefill_{L}",
+              "seq_len": L, "chunk": chunk, "n_q_heads": 32, "n_kv_heads": 8, "retrieval_kv_heads": 2,
+              "index_dim": 16, "top_p": 0.9, "n_sink": 4, "window": 8192, "page_size": 64,
+              "l2": "inputs_larger_than_l2", "parallelism": "replicas" if world > 1 else "single_gpu"}
+
+    if args.impl == "reference":
+        # The reference arm is the CPU oracle, as it stands, on a bounded sample of the same workload.
+        if rank != 0:
+            return
+        import torch
+        from paper_2605_16928_b200 import synth_device
+        dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+        data = synth_device.config_3_device(L=L, device=dev)
+        rows = np.linspace(L // 16, L - 1, 6).astype(np.int64)
+        vals = []
+        t_all = time.perf_counter()
+        for s in range(args.warmup + args.steps):
+            v, done, _ = cpu_oracle_prefill(data, L, rows[(s % 3) * 2:(s % 3) * 2 + 2], budget_s=20.0)
+            if s >= args.warmup:
+                vals.append(v)
+        value = float(np.mean(vals))
+        line = {"impl": "reference", "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s",
+                "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": 1e3 * L / value, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f64", "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": n_cores, "kind": "oracle",
+                                 "sample": "2 query rows x 32 heads per step, extrapolated to the sequence"},
+                "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "wall_s": time.perf_counter() - t_all}
+        print(json.dumps(line))
+        return
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    from paper_2605_16928_b200 import build as rbuild
+    if rank == 0:
+        rbuild.build_library()
+    if world > 1:
+        dist.barrier()
+    peaks = load_peaks()
+
+    data, path, step, step_dense, out, k_pre, chunks, L, chunk, stream = bench_prefill(args, rank, world, device)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing ----
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    if world > 1:
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * L / (ms_per_step * 1e-3)
+    status = path.status_code()
+    sel_frac = float((path.sel_cnt.float() / (path.pos_all[L - len(path.sel_cnt):].float()[:, None] + 1)).mean().item())
+
+    # ---- end to end: pinned host buffers, H2D of the chunk's q / k / v / k_pre, D2H of its output ----
+    from paper_2605_16928_b200 import binding as rb
+    Hq, Hkv, nih = path.Hq, data.heads.n_kv_heads, data.heads.n_index_heads
+    h_q = torch.empty((L, Hq, 128), dtype=torch.bfloat16).pin_memory()
+    h_q.copy_(data.q)
+    h_kpre = torch.empty((L, nih, 128), dtype=torch.bfloat16).pin_memory()
+    h_kpre.copy_(k_pre)
+    h_k = torch.empty((L, Hkv, 128), dtype=torch.bfloat16).pin_memory()
+    h_v = torch.empty((L, Hkv, 128), dtype=torch.bfloat16).pin_memory()
+    for s in range(0, L, 16384):
+        e = min(L, s + 16384)
+        phys = data.block_table[0, s // 64:(e + 63) // 64].long()
+        h_k[s:e].copy_(data.k_pages[phys].permute(0, 2, 1, 3).reshape(-1, Hkv, 128)[: e - s])
+        h_v[s:e].copy_(data.v_pages[phys].permute(0, 2, 1, 3).reshape(-1, Hkv, 128)[: e - s])
+    h_out = torch.empty((L, Hq, 128), dtype=torch.bfloat16).pin_memory()
+    d_q = torch.empty((chunk, Hq, 128), dtype=torch.bfloat16, device=device)
+    d_kpre = torch.empty((chunk, nih, 128), dtype=torch.bfloat16, device=device)
+    d_k = torch.empty((chunk, Hkv, 128), dtype=torch.bfloat16, device=device)
+    d_v = torch.empty((chunk, Hkv, 128), dtype=torch.bfloat16, device=device)
+    d_out = torch.empty((chunk, Hq, 128), dtype=torch.bfloat16, device=device)
+
+    def step_e2e():
+        for (s, C) in chunks:
+            d_q[:C].copy_(h_q[s:s + C], non_blocking=True)
+            d_kpre[:C].copy_(h_kpre[s:s + C], non_blocking=True)
+            d_k[:C].copy_(h_k[s:s + C], non_blocking=True)
+            d_v[:C].copy_(h_v[s:s + C], non_blocking=True)
+            rb.rtp_kv_append(path.ctx, path.params, path.cache, d_k[:C], d_v[:C], path.tok_seq[:C],
+                             path.pos_all[s:s + C], path.status)
+            path.run_chunk(s, C, d_q[:C], d_kpre[:C], d_out[:C])
+            h_out[s:s + C].copy_(d_out[:C], non_blocking=True)
+
+    step_e2e()
+    barrier()
+    n_e2e = max(1, min(args.steps, 3))
+    e0.record(stream)
+    for _ in range(n_e2e):
+        step_e2e()
+    e1.record(stream)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1) / n_e2e
+    if world > 1:
+        t = torch.tensor([ms_e2e], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    h2d = int(L * (Hq + 2 * Hkv + nih) * 128 * 2)
+    d2h = int(L * Hq * 128 * 2)
+    del h_q, h_k, h_v, h_kpre, h_out
+
+    # ---- per-kernel timing of one instrumented step (not part of the timed region) ----
+    klass = {"index_keys": 0.0, "select": 0.0, "sparse_attn": 0.0, "local_attn": 0.0}
+    d, p = path.data, path.params
+    for (s, C) in chunks:
+        q, kp, o = data.q[s:s + C], k_pre[s:s + C], out[s:s + C]
+        klass["index_keys"] += ev_time_ms(lambda: rb.rtp_index_keys(path.ctx, p, path.cache, kp, d.w_k, path.tok_seq[:C], path.pos_all[s:s + C]), stream)
+        klass["select"] += ev_time_ms(lambda: rb.rtp_topp_select(path.ctx, p, path.cache, q, d.w_q, None, None, 0, s, C, None, path.sel_cnt, path.sel_mass, path.sel_thr, path.sel_tie, path.status, path.workspace), stream)
+        klass["sparse_attn"] += ev_time_ms(lambda: rb.rtp_sparse_attn_prefill(path.ctx, p, path.cache, q, q, d.w_q, 0, s, C, None, path.sel_cnt, path.sel_thr, path.sel_tie, o, None, path.workspace, path.status), stream)
+        klass["local_attn"] += ev_time_ms(lambda: rb.rtp_local_attn(path.ctx, p, path.cache, q, None, None, 0, s, C, o, None, path.workspace, path.status), stream)
+    g = data.heads.group
+    fl_sparse = prefill_tile_flops(L, chunk, g, len(data.heads.ret_kv_heads), "dense", 4, 8192)
+    fl_local = prefill_tile_flops(L, chunk, g, len(data.heads.local_kv_heads), "local", 4, 8192)
+    fl_dense = prefill_tile_flops(L, chunk, g, data.heads.n_kv_heads, "dense", 4, 8192)
+    pairs = sum((min(chunk, L - s)) * (2 * s + min(chunk, L - s) + 1) / 2 for s in range(0, L, chunk))
+    dom = max(klass, key=klass.get)
+    n_launch = len(chunks)
+    if dom in ("sparse_attn", "local_attn"):
+        fl = fl_sparse if dom == "sparse_attn" else fl_local
+        achieved = fl / (klass[dom] * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        roofline = {"kernel": "attn_prefill_kernel<%s>" % ("sparse" if dom == "sparse_attn" else "local"),
+                    "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)",
+                    "flops_per_launch": fl / n_launch, "launch_ms": klass[dom] / n_launch}
+    else:
+        # indexer + top-p: plain ALU / MUFU work; peak = 148 SMs x 128 lanes x clock, ~12 lane-ops per score and pass
+        scores = pairs * len(data.heads.ret_q_heads)
+        achieved = scores / (klass["select"] * 1e-3) / 1e12
+        peak = 148 * 128 * 1.9e9 / 12 / 1e12
+        roofline = {"kernel": "select_chunk_kernel", "bound": "alu", "achieved": achieved, "peak": peak,
+                    "unit": "Tscore/s", "frac": achieved / peak, "traffic": None,
+                    "peak_source": "derived: 148 SMs x 128 lanes x 1.9 GHz / 12 lane-ops per score"}
+
+    line = {"metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config, "clocks": clocks,
+            "e2e": {"value": world * L / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": args.steps * len(chunks) * path.launches_per_chunk,
+            "roofline": roofline, "device_status": status,
+            "selected_fraction_last_chunk": sel_frac,
+            "kernel_ms_per_step": klass,
+            "kernel_tflops": {"sparse_attn": fl_sparse / klass["sparse_attn"] / 1e9,
+                              "local_attn": fl_local / klass["local_attn"] / 1e9},
+            "indexer_scores_per_s": pairs * len(data.heads.ret_q_heads) / (klass["select"] * 1e-3)}
+
+    if rank == 0 and not args.no_extras:
+        # dense in-library baseline at the same shape
+        step_dense()
+        torch.cuda.synchronize()
+        t_dense = min(ev_time_ms(step_dense, stream) for _ in range(2))
+        line["dense_baseline"] = {"ms_per_step": t_dense, "tokens_per_s": L / (t_dense * 1e-3),
+                                  "tflops": fl_dense / t_dense / 1e9, "speedup_sparse_vs_dense": t_dense / ms_per_step}
+        # CPU oracle on a bounded sample of the same workload
+        rows = np.linspace(L // 8, L - 1, 8).astype(np.int64)
+        v, done, secs = cpu_oracle_prefill(data, L, rows, budget_s=25.0)
+        line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": n_cores, "kind": "oracle",
+                                "sample": f"{done} query rows x 32 heads spread over the sequence ({secs:.1f} s), "
+                                          f"extrapolated per token"}
+        del path, data, out, k_pre
+        torch.cuda.empty_cache()
+        dec = []
+        dec.append(bench_decode_point(device, "c2_decode_batched_gqa", 32768, 8, 0.95, 0.1, 2048, True))
+        dec.append(bench_decode_point(device, "c5_decode_b4_512k", 524288, 4, 0.9, 0.05, 4096, False))
+        line["decode"] = dec
+    elif "cpu_baseline" not in line:
+        line["cpu_baseline"] = None
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

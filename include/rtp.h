@@ -130,6 +130,17 @@ rtp_status rtp_index_keys(rtp_ctx* ctx, const rtp_params* params, const rtp_cach
                           const void* k_pre, const void* w_k, const int32_t* tok_seq,
                           const int32_t* tok_pos, int64_t T, void* stream);
 
+/* ---- cache append of new K/V rows (Section 3.2: the KV cache that prefill builds and decode
+ *      extends; retrieval heads keep it whole) ------------------------------------
+ * k_new, v_new DEVICE bf16 [T, n_kv_heads, 128] post-RoPE keys / values of T new tokens;
+ * tok_seq, tok_pos DEVICE int32 [T].  Copies every row to
+ * k_pages / v_pages[block_table[seq][pos/64], head, pos%64, :].  Tokens whose sequence or page
+ * is out of range are skipped and RTP_ERR_INVALID is recorded in *status.  seq_lens is not
+ * modified (it belongs to the caller). */
+rtp_status rtp_kv_append(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                         const void* k_new, const void* v_new, const int32_t* tok_seq,
+                         const int32_t* tok_pos, int64_t T, int32_t* status, void* stream);
+
 /* ---- S1: query projection (Eq. 4, the W^Q q_pre factor) --------------------
  * q_pre  DEVICE bf16 [R, n_q_heads, 128] pre-RoPE queries (all heads; only the
  *        retrieval heads are read)

@@ -21,7 +21,7 @@ _STATUS_NAMES = ["RTP_OK", "RTP_ERR_INVALID", "RTP_ERR_CAPACITY", "RTP_ERR_UNSUP
 
 EXPORTS = [
     "rtp_version", "rtp_create", "rtp_destroy", "rtp_last_error", "rtp_workspace_bytes", "rtp_check_status",
-    "rtp_index_keys", "rtp_index_queries", "rtp_index_score", "rtp_topp_select", "rtp_sparse_attn_decode",
+    "rtp_kv_append", "rtp_index_keys", "rtp_index_queries", "rtp_index_score", "rtp_topp_select", "rtp_sparse_attn_decode",
     "rtp_sparse_attn_prefill", "rtp_local_attn", "rtp_dense_attn_prefill", "rtp_dense_attn_decode",
 ]
 
@@ -79,6 +79,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.rtp_check_status.argtypes = [vp, vp, vp]
     lib.rtp_index_keys.restype = i32
     lib.rtp_index_keys.argtypes = [vp, PP, PC, vp, vp, vp, vp, i64, vp]
+    lib.rtp_kv_append.restype = i32
+    lib.rtp_kv_append.argtypes = [vp, PP, PC, vp, vp, vp, vp, i64, vp, vp]
     lib.rtp_index_queries.restype = i32
     lib.rtp_index_queries.argtypes = [vp, PP, vp, vp, i64, vp, vp]
     lib.rtp_index_score.restype = i32
@@ -208,6 +210,12 @@ def rtp_check_status(ctx: Context, status, stream=None) -> int:
 def rtp_index_keys(ctx, params, cache, k_pre, w_k, tok_seq, tok_pos, stream=None):
     ctx._check(ctx.lib.rtp_index_keys(ctx.h, params.ref(), C.byref(cache), _ptr(k_pre), _ptr(w_k), _ptr(tok_seq),
                                       _ptr(tok_pos), int(tok_seq.shape[0]), _stream(stream)), "rtp_index_keys")
+
+
+def rtp_kv_append(ctx, params, cache, k_new, v_new, tok_seq, tok_pos, status, stream=None):
+    ctx._check(ctx.lib.rtp_kv_append(ctx.h, params.ref(), C.byref(cache), _ptr(k_new), _ptr(v_new), _ptr(tok_seq),
+                                     _ptr(tok_pos), int(tok_seq.shape[0]), _ptr(status), _stream(stream)),
+               "rtp_kv_append")
 
 
 def rtp_index_queries(ctx, params, q_pre, w_q, qt_out, stream=None):

@@ -62,6 +62,35 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(
   }
 }
 
+// ---- K/V append: one 16-byte chunk per thread, K and V -----------------------------------------
+__global__ void kv_append_kernel(CacheView cv, const __nv_bfloat16* __restrict__ k_new,
+                                 const __nv_bfloat16* __restrict__ v_new, const int32_t* __restrict__ tok_seq,
+                                 const int32_t* __restrict__ tok_pos, int64_t T, int32_t* status) {
+  const int64_t chunks_per_tok = (int64_t)cv.n_kv * 16;
+  const int64_t total = T * chunks_per_tok;
+  __nv_bfloat16* kp = const_cast<__nv_bfloat16*>(cv.k);
+  __nv_bfloat16* vp = const_cast<__nv_bfloat16*>(cv.v);
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t t = i / chunks_per_tok;
+    const int rem = (int)(i % chunks_per_tok);
+    const int head = rem >> 4, ch = rem & 15;
+    const int seq = tok_seq[t], pos = tok_pos[t];
+    if (seq < 0 || seq >= cv.batch || pos < 0 || (pos >> kPageShift) >= cv.max_pages) {
+      set_status(status, RTP_ERR_INVALID);
+      continue;
+    }
+    const int phys = cv.block_table[(int64_t)seq * cv.max_pages + (pos >> kPageShift)];
+    if (phys < 0 || phys >= cv.num_pages) {
+      set_status(status, RTP_ERR_INVALID);
+      continue;
+    }
+    const int64_t src = (t * cv.n_kv + head) * kHeadDim + ch * 8;
+    const int64_t dst = (((int64_t)phys * cv.n_kv + head) * kPage + (pos & (kPage - 1))) * kHeadDim + ch * 8;
+    *reinterpret_cast<uint4*>(kp + dst) = ld_stream_v4(k_new + src);
+    *reinterpret_cast<uint4*>(vp + dst) = ld_stream_v4(v_new + src);
+  }
+}
+
 // ---- materialised scores -----------------------------------------------------------------------
 constexpr int kScoreWarps = 4;
 
@@ -185,6 +214,17 @@ int score_splits(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
 }
 
 }  // namespace
+
+cudaError_t launch_kv_append(const CacheView& cv, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new,
+                             const int32_t* tok_seq, const int32_t* tok_pos, int64_t T, int32_t* status,
+                             cudaStream_t st) {
+  if (T == 0) return cudaSuccess;
+  const int64_t total = T * cv.n_kv * 16;
+  int64_t blocks = (total + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  kv_append_kernel<<<(unsigned)blocks, 256, 0, st>>>(cv, k_new, v_new, tok_seq, tok_pos, T, status);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_index_keys(const CacheView& cv, const Dims& d, const __nv_bfloat16* k_pre,
                               const __nv_bfloat16* w_k, const int32_t* tok_seq, const int32_t* tok_pos,

@@ -221,6 +221,21 @@ rtp_status rtp_index_keys(rtp_ctx* ctx, const rtp_params* params, const rtp_cach
   return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_index_keys");
 }
 
+rtp_status rtp_kv_append(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* k_new,
+                         const void* v_new, const int32_t* tok_seq, const int32_t* tok_pos, int64_t T,
+                         int32_t* status, void* stream) {
+  RTP_COMMON_PROLOGUE(true, false)
+  if (T < 0) return fail(ctx, RTP_ERR_INVALID, "T is negative");
+  if (T == 0) return RTP_OK;
+  if (!k_new || !v_new || !tok_seq || !tok_pos) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
+  if (!aligned16(k_new) || !aligned16(v_new)) return fail(ctx, RTP_ERR_INVALID, "k_new / v_new must be 16-byte aligned");
+  (void)d;
+  (void)hm;
+  cudaError_t e = launch_kv_append(cv, reinterpret_cast<const __nv_bfloat16*>(k_new),
+                                   reinterpret_cast<const __nv_bfloat16*>(v_new), tok_seq, tok_pos, T, status, st);
+  return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_kv_append");
+}
+
 rtp_status rtp_index_queries(rtp_ctx* ctx, const rtp_params* params, const void* q_pre, const void* w_q, int64_t R,
                              void* qt_out, void* stream) {
   if (!ctx) return RTP_ERR_INVALID;

@@ -83,6 +83,9 @@ enum SelMode { kRefine = 0, kCollect = 1, kSelectAll = 2, kTieScan = 3 };
 cudaError_t launch_index_keys(const CacheView& cv, const Dims& d, const __nv_bfloat16* k_pre,
                               const __nv_bfloat16* w_k, const int32_t* tok_seq, const int32_t* tok_pos,
                               int64_t T, cudaStream_t st);
+cudaError_t launch_kv_append(const CacheView& cv, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new,
+                             const int32_t* tok_seq, const int32_t* tok_pos, int64_t T, int32_t* status,
+                             cudaStream_t st);
 cudaError_t launch_index_queries(const Dims& d, const HeadMaps& hm, const __nv_bfloat16* q_pre,
                                  const __nv_bfloat16* w_q, int64_t R, __nv_bfloat16* qt, cudaStream_t st);
 

@@ -163,3 +163,27 @@ def test_host_side_argument_errors():
     bad = rb.Params.from_workload(wl, top_p=0.0)
     with pytest.raises(rb.RtpError):
         rb.rtp_index_queries(dw.ctx, bad, dw.q, dw.w_q, torch.empty((1, 1, 16), dtype=torch.bfloat16, device="cuda"))
+
+
+def test_kv_append_writes_pages_bit_exactly():
+    gh = _harness()
+    wl = synth.config_2(L=333, batch=3, window=128)
+    dw = gh.DeviceWorkload(wl)
+    want_k, want_v = dw.k_pages.clone(), dw.v_pages.clone()
+    dw.k_pages.zero_()
+    dw.v_pages.zero_()
+    for b in range(3):
+        k = gh.dev_bf16(wl.k[b])
+        v = gh.dev_bf16(wl.v[b])
+        seq = torch.full((333,), b, dtype=torch.int32, device="cuda")
+        pos = torch.arange(333, dtype=torch.int32, device="cuda")
+        rb.rtp_kv_append(dw.ctx, dw.params, dw.cache, k, v, seq, pos, dw.status)
+    torch.cuda.synchronize()
+    assert torch.equal(dw.k_pages.view(torch.int16), want_k.view(torch.int16))
+    assert torch.equal(dw.v_pages.view(torch.int16), want_v.view(torch.int16))
+    assert dw.status_code() == rb.RTP_OK
+    # a token outside the block table is skipped and reported
+    rb.rtp_kv_append(dw.ctx, dw.params, dw.cache, gh.dev_bf16(wl.k[0][:1]), gh.dev_bf16(wl.v[0][:1]),
+                     torch.tensor([7], dtype=torch.int32, device="cuda"),
+                     torch.tensor([0], dtype=torch.int32, device="cuda"), dw.status)
+    assert dw.status_code() == rb.RTP_ERR_INVALID
