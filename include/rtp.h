@@ -211,6 +211,31 @@ rtp_status rtp_sparse_attn_decode(rtp_ctx* ctx, const rtp_params* params, const 
                                   void* workspace, size_t workspace_bytes, int32_t* status,
                                   void* stream);
 
+/* ---- rtp_sparse_attn_decode without a caller workspace (the paper has no counterpart; this is a
+ *      packaging variant) -----------------------------------------------------------------
+ * Same computation, arguments and results as rtp_sparse_attn_decode, for hosts that cannot provide
+ * scratch memory at call time: e.g. a serving process whose device heap was handed over entirely to a
+ * pool it does not own, a plugin that runs inside someone else's allocator-free region, or code that
+ * runs where cudaMalloc is forbidden.  The split partials live in a fixed 1 MiB array that is part of
+ * the library image (every GPU that loads the library holds it until the process exits); the call
+ * allocates nothing and calls no allocating routine.
+ *  - Limit: rows * n_ret_q_heads * n_splits * 520 bytes must fit in 1 MiB, where n_splits is the
+ *    split count the library plans for the call (about 8 * SM count / (rows * heads), at most one
+ *    split per 128 listed tokens; a decode batch of up to 64 sequences x 8 retrieval heads always
+ *    fits).  Larger calls return RTP_ERR_CAPACITY before anything is launched
+ *    and rtp_last_error says how many bytes were needed.
+ *  - The first call on each device looks up the array's device address (once per device, with that
+ *    device current); make that first call outside any CUDA stream capture.
+ *  - All calls share the one array.  Nothing in it has to start at zero (every slot that is read was
+ *    written earlier in the same call), and it keeps the last call's partials afterwards.  Two calls
+ *    that overlap on the GPU (different streams, or graphs replayed concurrently) race on it: issue
+ *    them in stream order, or use rtp_sparse_attn_decode with separate workspaces. */
+rtp_status rtp_sparse_attn_decode_static(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                                         const void* q, const int32_t* row_seq, const int32_t* row_pos,
+                                         int64_t R, const int32_t* sel_idx, int64_t sel_stride,
+                                         const int32_t* sel_count, void* out, float* lse, int32_t* status,
+                                         void* stream);
+
 /* ---- S6: sparse attention for a prefill chunk (Eq. 5 applied per query row; the
  *      paper itself keeps retrieval heads dense in prefill) -------------------
  * Rows are positions q_start..q_start+C-1 of sequence seq_id; causal.

@@ -21,7 +21,7 @@ _STATUS_NAMES = ["RTP_OK", "RTP_ERR_INVALID", "RTP_ERR_CAPACITY", "RTP_ERR_UNSUP
 
 EXPORTS = [
     "rtp_version", "rtp_create", "rtp_destroy", "rtp_last_error", "rtp_workspace_bytes", "rtp_check_status",
-    "rtp_kv_append", "rtp_index_keys", "rtp_index_queries", "rtp_index_score", "rtp_topp_select", "rtp_sparse_attn_decode",
+    "rtp_kv_append", "rtp_index_keys", "rtp_index_queries", "rtp_index_score", "rtp_topp_select", "rtp_sparse_attn_decode", "rtp_sparse_attn_decode_static",
     "rtp_sparse_attn_prefill", "rtp_local_attn", "rtp_dense_attn_prefill", "rtp_dense_attn_decode",
 ]
 
@@ -89,6 +89,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.rtp_topp_select.argtypes = [vp, PP, PC, vp, vp, vp, vp, i32, i32, i64, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.rtp_sparse_attn_decode.restype = i32
     lib.rtp_sparse_attn_decode.argtypes = [vp, PP, PC, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, sz, vp, vp]
+    lib.rtp_sparse_attn_decode_static.restype = i32
+    lib.rtp_sparse_attn_decode_static.argtypes = [vp, PP, PC, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, vp]
     lib.rtp_sparse_attn_prefill.restype = i32
     lib.rtp_sparse_attn_prefill.argtypes = [vp, PP, PC, vp, vp, vp, i32, i32, i64, vp, i64, vp, vp, vp, vp, vp, vp,
                                             sz, vp, vp]
@@ -251,6 +253,17 @@ def rtp_sparse_attn_decode(ctx, params, cache, q, row_seq, row_pos, sel_idx, sel
                                               int(sel_idx.shape[-1]), _ptr(sel_count), _ptr(out), _ptr(lse),
                                               _ptr(workspace), int(workspace.numel() * workspace.element_size()),
                                               _ptr(status), _stream(stream)), "rtp_sparse_attn_decode")
+
+
+def rtp_sparse_attn_decode_static(ctx, params, cache, q, row_seq, row_pos, sel_idx, sel_count, out, lse, status,
+                                  stream=None):
+    """rtp_sparse_attn_decode for callers that cannot hand over scratch memory: the split partials go to a
+    1 MiB array built into the library, so nothing is allocated.  Calls must not overlap on the GPU."""
+    ctx._check(ctx.lib.rtp_sparse_attn_decode_static(ctx.h, params.ref(), C.byref(cache), _ptr(q), _ptr(row_seq),
+                                                     _ptr(row_pos), int(row_seq.shape[0]), _ptr(sel_idx),
+                                                     int(sel_idx.shape[-1]), _ptr(sel_count), _ptr(out), _ptr(lse),
+                                                     _ptr(status), _stream(stream)),
+               "rtp_sparse_attn_decode_static")
 
 
 def rtp_sparse_attn_prefill(ctx, params, cache, q, q_pre, w_q, seq_id, q_start, n_rows, sel_idx, sel_count,

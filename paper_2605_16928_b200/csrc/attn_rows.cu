@@ -2,6 +2,8 @@
 // a selection list, the sink + window pattern, or the full causal prefix.  Bandwidth-bound: every
 // K and V row is read once with 16-byte loads (a half-warp per 256-byte row), all query heads of a
 // KV group share the loaded rows, the set is split over CTAs and merged by log-sum-exp.
+#include <mutex>
+
 #include "rtp_device.cuh"
 
 namespace rtp {
@@ -323,6 +325,49 @@ cudaError_t launch_attn_rows(const CacheView& cv, const Dims& d, const HeadMaps&
   }
 #undef RTP_LAUNCH
   return cudaErrorInvalidValue;
+}
+
+// ---- split partials in a static device array (entry point for callers that must not allocate) --------
+// kStaticScratchBytes of global memory are part of the library image on every GPU that loads it.
+constexpr size_t kStaticScratchBytes = 1u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device
+}  // namespace
+
+size_t attn_rows_static_scratch_bytes() { return kStaticScratchBytes; }
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel can use: the
+// device address is looked up once per device (with that device current) and cached.
+cudaError_t launch_attn_rows_static(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                                    const __nv_bfloat16* q, const int32_t* sel_idx, int64_t sel_stride,
+                                    const int32_t* sel_count, __nv_bfloat16* out, float* lse, int64_t max_len,
+                                    int32_t* status, int sm_count, size_t* needed_bytes, cudaStream_t st) {
+  *needed_bytes = 0;
+  if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
+  const int n_splits = plan_splits(rows.R * d.n_ret, max_set_len(d, kSetList, sel_stride, max_len), sm_count);
+  const size_t need = n_splits > 1 ? (size_t)rows.R * d.n_ret * n_splits * kPartial * sizeof(float) : 0;
+  *needed_bytes = need;
+  if (need > kStaticScratchBytes) return cudaErrorMemoryAllocation;   // reported as RTP_ERR_CAPACITY by the caller
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  void* ptr = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[dev]) {
+      e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+      if (e != cudaSuccess) return e;
+      g_scratch_ptr[dev] = ptr;
+    }
+    ptr = g_scratch_ptr[dev];
+  }
+  return launch_typed<1, kSetList>(cv, d, hm, rows, d.n_ret, q, sel_idx, sel_stride, sel_count, out, lse,
+                                   reinterpret_cast<float*>(ptr), n_splits, status, st);
 }
 
 }  // namespace rtp

@@ -329,6 +329,34 @@ rtp_status rtp_sparse_attn_decode(rtp_ctx* ctx, const rtp_params* params, const 
   return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_sparse_attn_decode");
 }
 
+rtp_status rtp_sparse_attn_decode_static(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
+                                         const void* q, const int32_t* row_seq, const int32_t* row_pos, int64_t R,
+                                         const int32_t* sel_idx, int64_t sel_stride, const int32_t* sel_count,
+                                         void* out, float* lse, int32_t* status, void* stream) {
+  RTP_COMMON_PROLOGUE(true, false)
+  Rows rows;
+  int64_t max_len = 0;
+  if (!row_seq || !row_pos) return fail(ctx, RTP_ERR_INVALID, "row_seq / row_pos is NULL");
+  if (const char* m = check_rows(row_seq, row_pos, 0, 0, R, cache, &rows, &max_len)) return fail(ctx, RTP_ERR_INVALID, m);
+  if (R == 0 || d.n_ret == 0) return RTP_OK;
+  if (!q || !sel_idx || !sel_count || !out) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
+  if (sel_stride <= 0) return fail(ctx, RTP_ERR_INVALID, "sel_stride must be positive");
+  if (!aligned16(q) || !aligned16(out)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
+  size_t need = 0;
+  cudaError_t e = launch_attn_rows_static(cv, d, hm, rows, reinterpret_cast<const __nv_bfloat16*>(q), sel_idx,
+                                          sel_stride, sel_count, reinterpret_cast<__nv_bfloat16*>(out), lse, max_len,
+                                          status, ctx->sm_count, &need, st);
+  if (e == cudaErrorMemoryAllocation && need > attn_rows_static_scratch_bytes()) {
+    char msg[192];
+    std::snprintf(msg, sizeof(msg),
+                  "rtp_sparse_attn_decode_static: this call needs %zu bytes of split scratch but the built-in "
+                  "array holds %zu; use rtp_sparse_attn_decode with a caller workspace or fewer rows",
+                  need, attn_rows_static_scratch_bytes());
+    return fail(ctx, RTP_ERR_CAPACITY, msg);
+  }
+  return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_sparse_attn_decode_static");
+}
+
 rtp_status rtp_sparse_attn_prefill(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q,
                                    const void* q_pre, const void* w_q, int32_t seq_id, int32_t q_start, int64_t C,
                                    const int32_t* sel_idx, int64_t sel_stride, const int32_t* sel_count,

@@ -114,6 +114,12 @@ cudaError_t launch_attn_rows(const CacheView& cv, const Dims& d, const HeadMaps&
                              const int32_t* sel_count, __nv_bfloat16* out, float* lse, void* ws,
                              size_t ws_bytes, int64_t max_len, int32_t* status, int sm_count, cudaStream_t st);
 
+size_t attn_rows_static_scratch_bytes();
+cudaError_t launch_attn_rows_static(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                                    const __nv_bfloat16* q, const int32_t* sel_idx, int64_t sel_stride,
+                                    const int32_t* sel_count, __nv_bfloat16* out, float* lse, int64_t max_len,
+                                    int32_t* status, int sm_count, size_t* needed_bytes, cudaStream_t st);
+
 enum PrefillMode { kPrefillDense = 0, kPrefillLocal = 1, kPrefillSparse = 2 };
 cudaError_t launch_attn_prefill(const CacheView& cv, const Dims& d, const HeadMaps& hm, int mode,
                                 const __nv_bfloat16* q, const __nv_bfloat16* qt, int32_t seq_id, int32_t q_start,
