@@ -146,7 +146,10 @@ __global__ void __launch_bounds__(kThreadsP, 2) attn_prefill_kernel(
 
   // sparse mode: projected query fragment and the rows' membership rule
   QFrag iq = {0u, 0u, 0u, 0u};
-  float thr_a = 0.f, thr_b = 0.f;
+  // Membership is tested on the unscaled MMA output: raw > up_x means "score above the threshold", raw >= lo_x
+  // means "score at or above it" (the two differ only for keys tied with the threshold score).
+  const float kInfP = __int_as_float(0x7f800000);
+  float lo_a = kInfP, up_a = kInfP, lo_b = kInfP, up_b = kInfP;
   int tie_a = -1, tie_b = -1;
   if (MODE == kPrefillSparse) {
     const int rh = hm.ih_heads[ih][hslot];   // retrieval-head index of this warp's head
@@ -156,7 +159,10 @@ __global__ void __launch_bounds__(kThreadsP, 2) attn_prefill_kernel(
       const uint2 v = *reinterpret_cast<const uint2*>(qt + rr * kIndexDim + off);
       iq.a0 = v.x;
       iq.a2 = v.y;
-      thr_a = sel_thresh[rr];
+      const uint32_t tk = okey(sel_thresh[rr]);
+      float dummy;
+      raw_preimage(d.score_scale, tk, tk, lo_a, dummy);
+      raw_preimage(d.score_scale, 0u, tk, dummy, up_a);
       tie_a = sel_tie_last[rr];
     }
     if (row_b_ok) {
@@ -164,7 +170,10 @@ __global__ void __launch_bounds__(kThreadsP, 2) attn_prefill_kernel(
       const uint2 v = *reinterpret_cast<const uint2*>(qt + rr * kIndexDim + off);
       iq.a1 = v.x;
       iq.a3 = v.y;
-      thr_b = sel_thresh[rr];
+      const uint32_t tk = okey(sel_thresh[rr]);
+      float dummy;
+      raw_preimage(d.score_scale, tk, tk, lo_b, dummy);
+      raw_preimage(d.score_scale, 0u, tk, dummy, up_b);
       tie_b = sel_tie_last[rr];
     }
   }
@@ -194,6 +203,8 @@ __global__ void __launch_bounds__(kThreadsP, 2) attn_prefill_kernel(
     uint32_t member = 0xffffffffu;
     if (MODE == kPrefillSparse && active) {
       member = 0;
+      const bool easy = (n_base + kBN - 1 <= warp_m_lo) &&
+                        __all_sync(0xffffffffu, (!row_a_ok || tie_a >= n_base + kBN - 1) && (!row_b_ok || tie_b >= n_base + kBN - 1));
       const unsigned char* ik = st + 2 * kTileBytes;
       const int boff = 2 * qfrag_dim_offset(lane);
 #pragma unroll
@@ -202,16 +213,20 @@ __global__ void __launch_bounds__(kThreadsP, 2) attn_prefill_kernel(
         const float zero[4] = {0.f, 0.f, 0.f, 0.f};
         float s4[4];
         mma_bf16_16816(s4, iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
+        if (easy) {
+          // every key of the tile is causal for every row of the warp and lies at or before the rows' tie positions
+          member |= (s4[0] >= lo_a ? 1u : 0u) << (nt * 4) | (s4[1] >= lo_a ? 1u : 0u) << (nt * 4 + 1) |
+                    (s4[2] >= lo_b ? 1u : 0u) << (nt * 4 + 2) | (s4[3] >= lo_b ? 1u : 0u) << (nt * 4 + 3);
+        } else {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int n = n_base + nt * 8 + 2 * c + (e & 1);
-          const float s = finish_score(s4[e], d.score_scale);
-          const bool lo_row = e < 2;
-          const float thr = lo_row ? thr_a : thr_b;
-          const int tie = lo_row ? tie_a : tie_b;
-          const int pos = lo_row ? pos_a : pos_b;
-          const bool in = (n <= pos) && (s > thr || (s == thr && n <= tie));
-          member |= (in ? 1u : 0u) << (nt * 4 + e);
+          for (int e = 0; e < 4; ++e) {
+            const int n = n_base + nt * 8 + 2 * c + (e & 1);
+            const bool lo_row = e < 2;
+            const float raw = s4[e];
+            const bool in = (n <= (lo_row ? pos_a : pos_b)) &&
+                            (raw > (lo_row ? up_a : up_b) || (raw >= (lo_row ? lo_a : lo_b) && n <= (lo_row ? tie_a : tie_b)));
+            member |= (in ? 1u : 0u) << (nt * 4 + e);
+          }
         }
       }
       active = __any_sync(0xffffffffu, member != 0);
@@ -266,8 +281,8 @@ __global__ void __launch_bounds__(kThreadsP, 2) attn_prefill_kernel(
       tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 1));
       tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 2));
       const float na = fmaxf(mx_a, ta * sc2), nb = fmaxf(mx_b, tb * sc2);
-      const float ca = (na == -INFINITY) ? 1.f : exp2f(mx_a - na);
-      const float cb = (nb == -INFINITY) ? 1.f : exp2f(mx_b - nb);
+      const float ca = (na == -INFINITY) ? 1.f : fast_ex2(mx_a - na);
+      const float cb = (nb == -INFINITY) ? 1.f : fast_ex2(mx_b - nb);
       const float ba = (na == -INFINITY) ? 0.f : na, bb = (nb == -INFINITY) ? 0.f : nb;
       mx_a = na;
       mx_b = nb;
@@ -275,8 +290,8 @@ __global__ void __launch_bounds__(kThreadsP, 2) attn_prefill_kernel(
       uint32_t pf[4][4];   // P as bf16 A fragments, one per 16 keys
 #pragma unroll
       for (int nt = 0; nt < 8; ++nt) {
-        const float p0 = exp2f(s[nt][0] * sc2 - ba), p1 = exp2f(s[nt][1] * sc2 - ba);
-        const float p2 = exp2f(s[nt][2] * sc2 - bb), p3 = exp2f(s[nt][3] * sc2 - bb);
+        const float p0 = fast_ex2(s[nt][0] * sc2 - ba), p1 = fast_ex2(s[nt][1] * sc2 - ba);
+        const float p2 = fast_ex2(s[nt][2] * sc2 - bb), p3 = fast_ex2(s[nt][3] * sc2 - bb);
         ra += p0 + p1;
         rb += p2 + p3;
         pf[nt >> 1][(nt & 1) * 2] = pack_bf16(p0, p1);

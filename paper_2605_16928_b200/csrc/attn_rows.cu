@@ -161,13 +161,13 @@ __global__ void __launch_bounds__(kThreads) attn_rows_kernel(
         for (int x = 0; x < kUnroll; ++x) pw[x][g] = 0.f;
         continue;
       }
-      const float corr = exp2f(m_run[g] - mx);
+      const float corr = fast_ex2(m_run[g] - mx);
       float ls = l_run[g] * corr;
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[g][i] *= corr;
 #pragma unroll
       for (int x = 0; x < kUnroll; ++x) {
-        pw[x][g] = exp2f(logit[x][g] - mx);
+        pw[x][g] = fast_ex2(logit[x][g] - mx);
         ls += pw[x][g];
       }
       l_run[g] = ls;
@@ -205,7 +205,7 @@ __global__ void __launch_bounds__(kThreads) attn_rows_kernel(
     if (mt != -INFINITY) {
 #pragma unroll
       for (int s = 0; s < kStreams; ++s) {
-        const float w = exp2f(red[s][g][kHeadDim] - mt);
+        const float w = fast_ex2(red[s][g][kHeadDim] - mt);
         lt += red[s][g][kHeadDim + 1] * w;
         a += red[s][g][dim] * w;
       }
@@ -243,7 +243,7 @@ __global__ void __launch_bounds__(kHeadDim) attn_merge_kernel(const Dims d, cons
   float lt = 0.f, a = 0.f;
   if (mt != -INFINITY) {
     for (int s = 0; s < n_splits; ++s) {
-      const float w = exp2f(p[(int64_t)s * kPartial + kHeadDim] - mt);
+      const float w = fast_ex2(p[(int64_t)s * kPartial + kHeadDim] - mt);
       lt += p[(int64_t)s * kPartial + kHeadDim + 1] * w;
       a += p[(int64_t)s * kPartial + dim] * w;
     }

@@ -107,11 +107,41 @@ __device__ __forceinline__ float finish_score(float raw, float scale) {
   return __fadd_rn(__fmul_rn(raw, scale), 0.0f);
 }
 
+// Closed interval [raw_lo, raw_hi] of unscaled MMA outputs whose finished score has an ordered key in
+// [key_lo, key_hi] (finish_score is monotone, so the preimage of a key interval is an interval; it is
+// empty, raw_lo > raw_hi, when no float maps into it).  64 bisection steps.
+__device__ __forceinline__ void raw_preimage(float scale, uint32_t key_lo, uint32_t key_hi, float& raw_lo, float& raw_hi) {
+  const uint32_t kmin = okey(-3.4028234e38f), kmax = okey(3.4028234e38f);
+  // smallest raw key with key(finish) >= key_lo
+  uint32_t a = kmin, b = kmax;   // answer in [a, b]; if even kmax fails the interval is empty
+  if (okey(finish_score(okey_to_float(a), scale)) >= key_lo) b = a;
+  while (a + 1 < b) {
+    const uint32_t mid = a + ((b - a) >> 1);
+    if (okey(finish_score(okey_to_float(mid), scale)) >= key_lo) b = mid; else a = mid;
+  }
+  raw_lo = okey_to_float(b);
+  // largest raw key with key(finish) <= key_hi
+  a = kmin; b = kmax;
+  if (okey(finish_score(okey_to_float(b), scale)) <= key_hi) a = b;
+  while (a + 1 < b) {
+    const uint32_t mid = a + ((b - a) >> 1);
+    if (okey(finish_score(okey_to_float(mid), scale)) <= key_hi) a = mid; else b = mid;
+  }
+  raw_hi = okey_to_float(a);
+}
+
 // Address of the 2 KB index-key slice of (logical page, index head) of a sequence.
 __device__ __forceinline__ const __nv_bfloat16* ikey_page_ptr(const CacheView& cv, int seq, int page,
                                                                int ih) {
   const int phys = __ldg(cv.block_table + (int64_t)seq * cv.max_pages + page);
   return cv.ikey + ((int64_t)phys * cv.n_ih + ih) * (kPage * kIndexDim);
+}
+
+// 2^x on the special-function unit (about 2 ulp; inputs of -inf give 0).
+__device__ __forceinline__ float fast_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
 __device__ __forceinline__ float warp_max(float x) {
