@@ -6,13 +6,16 @@
 // 0 .. last position (2 KB per page, cp.async double buffer) once per pass; a warp scores a 64-key
 // page against its 16 rows with eight m16n8k16 MMAs.  All selection state lives in shared memory, so
 // the whole selection of the chunk is one kernel without inter-CTA communication:
-//   pass 0   row maximum M                                            (1 op per score)
-//   pass 1   128-bin histogram of softmax mass over d = M - s in steps of 1/4 (d >= 31.75 pooled);
-//            gives Z and the bucket in which the cumulative mass reaches p * Z; the bucket is then
-//            turned into the exact interval of ordered score keys that fall into it (bisection)
-//   pass 2+  64-bin (mass, count) histograms of the ordered key inside the interval, 6 key bits per
-//            pass, until the interval holds one key or a single key value
-//   tie pass only when equal scores straddle the cut: position of the last tie taken
+//   max       row maximum M                                                   (1 op per score)
+//   level 1   64-bin histogram of softmax mass over d = M - s in steps of 1/2 (d >= 31.5 pooled), in
+//             fixed point with native 32-bit shared-memory adds; gives Z and the bucket in which the
+//             cumulative mass reaches p * Z; the bucket becomes an exact interval of ordered score keys
+//             (bisection) and of unscaled MMA outputs (so later passes compare raw values only)
+//   key level 64-bin mass histogram of the ordered key inside the interval, 6 key bits per pass, until the
+//             chosen bin provably holds at most 64 keys
+//   collect   the keys of the final bucket go to a 64-entry list, the keys above it are counted; the warp
+//             ranks the list exactly by (score descending, position ascending) and cuts it
+//   tie       only when more than 64 equal scores straddle the cut: position of the last tie taken
 // Rows drop out as soon as they are resolved; the CTA stops when all its rows are.  When id lists
 // are requested, one more sweep appends every row's members in position order.
 // Each pass has its own inner loop; pages that lie wholly below a warp's first row need no causal test.
@@ -29,34 +32,39 @@ constexpr int kCRows = 128;
 constexpr int kPagesPerStage = 4;
 constexpr int kStageKeys = kPagesPerStage * kPage;                  // 256 keys
 constexpr int kStageBytesC = kStageKeys * kIndexDim * 2;            // 8 KB
-constexpr int kL1Bins = 128;
-constexpr float kL1Scale = 4.0f;                                    // bins per unit of d
-constexpr int kSubBins = 64;
-constexpr int kMaxPasses = 12;
+constexpr int kBins = 64;                                           // bins per level
+constexpr float kL1Scale = 2.0f;                                    // level-1 bins per unit of d = M - s
+constexpr int kCandCapC = 64;                                       // candidates sorted exactly per row
+constexpr int kRowBytes = kBins * 8;                                // 512 B per row: 64 x {hi, lo} or 64 x {key, idx}
+constexpr int kMaxPasses = 14;
 constexpr float kLog2eC = 1.4426950408889634f;
+// A key adds floor(e_rel * 2^20) to its bin, split into two 32-bit words (hi = >> 10, lo = & 1023) so that native
+// 32-bit shared-memory adds never overflow for up to 2^20 keys.  e_rel = mass relative to the bin's (level 1) or
+// the bucket's (key levels) upper end, in (e^-0.5, 1]: every key adds at least kMinHi to the hi word.
+constexpr uint32_t kMinHi = 620;                                    // floor(e^-0.5 * 1024) - 1
 
-enum Phase { kPhMax = 0, kPhL1 = 1, kPhKey = 2, kPhTie = 3, kPhDone = 4 };
+enum Phase { kPhMax = 0, kPhL1 = 1, kPhKey = 2, kPhCollect = 3, kPhTie = 4, kPhDone = 5 };
 
 struct RowState {      // one per (row, head), in shared memory
   float M, Z, target, mass_above;
-  uint32_t base_key;   // key levels: bucket = keys in [base_key, base_key + span)
+  float ref_s;         // key levels: masses are accumulated relative to exp(ref_s - M) (upper end of the level-1 bucket)
+  float e_ref;         // exp(ref_s - M)
+  uint32_t base_key;   // bucket = keys in [base_key, base_key + span)
   uint32_t span;
-  int32_t shift;       // bin = (key - base_key) >> shift, in [0, 64)
-  uint32_t hi_count;   // first key level: keys > hi_count are counted as "above the bucket"; else 0xffffffff
+  int32_t shift;       // key levels: bin = (key - base_key) >> shift, in [0, 64)
+  float raw_lo, raw_hi;   // unscaled-score interval of the bucket
   int32_t phase;
-  int32_t cnt_above;   // keys strictly above the current bucket
+  int32_t cnt_above;   // keys strictly above the final bucket (counted in the collect pass)
+  int32_t cand_cnt;    // keys inside the final bucket (collect pass)
   int32_t tie_need;    // tie pass: number of ties to take
   uint32_t thr_key;    // result: selected <=> key > thr_key or (key == thr_key and n <= tie_last)
   int32_t tie_last;
   int32_t n_keys;
   float sel_mass;
   int32_t count;
-  float raw_lo, raw_hi;   // raw-value interval of the current key bucket
-  float raw_hic;          // first key level: raw values above this lie above the bucket; else +inf
-  float tie_lo, tie_hi;   // raw-value interval of thr_key (tie pass)
 };
 
-constexpr int kHistBytes = kCRows * kL1Bins * 4;                    // 64 KB (key levels reuse it as 64 x {mass,cnt})
+constexpr int kHistBytes = kCRows * kRowBytes;                      // 64 KB
 constexpr int kSmemC = kHistBytes + 2 * kStageBytesC + kCRows * (int)sizeof(RowState);
 
 __device__ __forceinline__ void cp_async16c(uint32_t dst, const void* src) {
@@ -68,20 +76,33 @@ __device__ __forceinline__ uint32_t smem_u32c(const void* p) {
 
 // Level-1 bin of a score: the same arithmetic in the histogram pass and in the bisection below.
 __device__ __forceinline__ int l1_bin(float M, float s) {
-  return min(kL1Bins - 1, (int)((M - s) * kL1Scale));
+  return max(0, min(kBins - 1, (int)((M - s) * kL1Scale)));
+}
+
+// Adds floor(2^x) (x <= 20) to a split accumulator.
+__device__ __forceinline__ void add_mass(uint32_t* acc, float x) {
+  const uint32_t q = min(__float2uint_rz(fast_ex2(x)), 1u << 20);
+  atomicAdd(acc, q >> 10);
+  atomicAdd(acc + 1, q & 1023u);
+}
+__device__ __forceinline__ float acc_mass(uint32_t hi, uint32_t lo) {   // in units of 2^-20
+  return (float)hi * 1024.0f + (float)lo;
 }
 
 // Per-lane view of its two rows for one pass (registers).
 struct LaneRows {
   float M_a, M_b;
-  uint32_t base_a, base_b;
-  int shift_a, shift_b;
   int pos_a, pos_b;
   // Unscaled MMA outputs are compared directly: the keys of a bucket are the images of one closed interval of
   // raw values (finish_score is monotone), found by bisection when the bucket is chosen.
-  float lo_a, hi_a, lo_b, hi_b;      // raw interval of the current key bucket (empty: lo = +inf, hi = -inf)
-  float hic_a, hic_b;                // raw values above this are counted as "above the bucket" (+inf: none)
-  float tlo_a, thi_a, tlo_b, thi_b;  // raw interval of the tied key value (tie pass)
+  float lo_a, hi_a, lo_b, hi_b;      // raw interval of the current bucket (empty: lo = +inf, hi = -inf)
+  float mid_a, hw_a, mid_b, hw_b;    // the same interval as centre and half width (slightly widened): 2-op reject
+  float cut_a, cut_b;                // collect pass: raw values above this are counted as above the bucket (+inf: none)
+  float tlo_a, thi_a, tlo_b, thi_b;  // tie pass: raw interval of the tied key value
+  float ref_a, ref_b;                // key levels: mass reference score
+  uint32_t base_a, base_b;
+  int shift_a, shift_b;
+  bool collect_a, collect_b;         // the bucket's keys are collected instead of histogrammed
 };
 
 // ---- one 64-key page, one warp ----------------------------------------------------------------------
@@ -110,7 +131,7 @@ __device__ __forceinline__ void page_max(const unsigned char* pg, const QFrag& i
 
 template <bool MASK>
 __device__ __forceinline__ void page_l1(const unsigned char* pg, const QFrag& iq, int lane, int n_page,
-                                        const LaneRows& L, float scale, float* hist_a, float* hist_b) {
+                                        const LaneRows& L, float scale, uint32_t* hist_a, uint32_t* hist_b) {
   const int g = lane >> 2, c = lane & 3;
   const int boff = 2 * qfrag_dim_offset(lane);
 #pragma unroll
@@ -126,18 +147,19 @@ __device__ __forceinline__ void page_l1(const unsigned char* pg, const QFrag& iq
       if (MASK && n0 + (e & 1) > (lo ? L.pos_a : L.pos_b)) continue;
       const float s = finish_score(s4[e], scale);
       const float dd = (lo ? L.M_a : L.M_b) - s;
-      const int bin = max(0, min(kL1Bins - 1, (int)(dd * kL1Scale)));   // (rows that are already done have no M)
-      atomicAdd((lo ? hist_a : hist_b) + bin, fast_ex2(-dd * kLog2eC));
+      const int bin = max(0, min(kBins - 1, (int)(dd * kL1Scale)));   // (rows that are already done have no M)
+      // mass relative to the bin's upper end: exp(-(dd - bin/2)), scaled by 2^20
+      add_mass((lo ? hist_a : hist_b) + 2 * bin, fmaf((float)bin, 0.5f * kLog2eC, fmaf(dd, -kLog2eC, 20.0f)));
     }
   }
 }
 
-// Key levels (and, when TIE, the in-order tie count).  Rows that are not in a key level carry span = 0 and
-// hic = 0xffffffff, rows that are not in the tie pass carry need = 0, so no per-row branching is needed.
-template <bool MASK, bool TIE>
+// Key levels, candidate collection and (when TIE) the in-order tie count.  Rows that take no part carry empty
+// intervals, so no per-row branching is needed on the common path.
+template <bool MASK, bool TIE, bool COUNT>
 __device__ __forceinline__ void page_late(const unsigned char* pg, const QFrag& iq, int lane, int n_page,
-                                          const LaneRows& L, float scale, float* hist_a, float* hist_b,
-                                          int& cnt_a, int& cnt_b, int need_a, int need_b,
+                                          const LaneRows& L, float scale, uint32_t* hist_a, uint32_t* hist_b,
+                                          int* ccnt_a, int* ccnt_b, int& cnt_a, int& cnt_b, int need_a, int need_b,
                                           int& run_a, int& run_b, int& tl_a, int& tl_b) {
   const int g = lane >> 2, c = lane & 3;
   const int boff = 2 * qfrag_dim_offset(lane);
@@ -148,24 +170,44 @@ __device__ __forceinline__ void page_late(const unsigned char* pg, const QFrag& 
     float s4[4];
     mma_bf16_16816(s4, iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
     const int n0 = n_page + nt * 8 + 2 * c;
+    if (MASK) {
+      const float nan = __int_as_float(0x7fc00000);   // fails every test below
+      if (n0 > L.pos_a) s4[0] = nan;
+      if (n0 + 1 > L.pos_a) s4[1] = nan;
+      if (n0 > L.pos_b) s4[2] = nan;
+      if (n0 + 1 > L.pos_b) s4[3] = nan;
+    }
+    if (COUNT) {   // keys above the bucket of a row that is collecting
+      cnt_a += (s4[0] > L.cut_a) + (s4[1] > L.cut_a);
+      cnt_b += (s4[2] > L.cut_b) + (s4[3] > L.cut_b);
+    }
+    // quick reject: |raw - mid| <= hw is implied by raw in [lo, hi]
+    const bool near = fabsf(s4[0] - L.mid_a) <= L.hw_a || fabsf(s4[1] - L.mid_a) <= L.hw_a ||
+                      fabsf(s4[2] - L.mid_b) <= L.hw_b || fabsf(s4[3] - L.mid_b) <= L.hw_b;
     int tf_a = 0, tf_b = 0;
+    if (near) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const bool lo = e < 2;
-      float raw = s4[e];
-      if (MASK && n0 + (e & 1) > (lo ? L.pos_a : L.pos_b)) raw = __int_as_float(0x7fc00000);   // NaN: fails every test
-      if (raw >= (lo ? L.lo_a : L.lo_b) && raw <= (lo ? L.hi_a : L.hi_b)) {
-        const float s = finish_score(raw, scale);
-        const uint32_t t = okey(s) - (lo ? L.base_a : L.base_b);
-        float* h = (lo ? hist_a : hist_b) + 2 * (t >> (lo ? L.shift_a : L.shift_b));
-        atomicAdd(h, fast_ex2((s - (lo ? L.M_a : L.M_b)) * kLog2eC));
-        atomicAdd(reinterpret_cast<int*>(h + 1), 1);
-      } else if (raw > (lo ? L.hic_a : L.hic_b)) {
-        if (lo) ++cnt_a; else ++cnt_b;
-      }
-      if (TIE) {
-        if (raw >= (lo ? L.tlo_a : L.tlo_b) && raw <= (lo ? L.thi_a : L.thi_b)) {
-          if (lo) tf_a |= 1 << (e & 1); else tf_b |= 1 << (e & 1);
+      for (int e = 0; e < 4; ++e) {
+        const bool lo = e < 2;
+        const float raw = s4[e];
+        if (raw >= (lo ? L.lo_a : L.lo_b) && raw <= (lo ? L.hi_a : L.hi_b)) {
+          if (TIE && (lo ? L.tlo_a : L.tlo_b) <= raw && raw <= (lo ? L.thi_a : L.thi_b)) {
+            if (lo) tf_a |= 1 << (e & 1); else tf_b |= 1 << (e & 1);
+            continue;
+          }
+          const float s = finish_score(raw, scale);
+          const uint32_t key = okey(s);
+          uint32_t* h = lo ? hist_a : hist_b;
+          if (lo ? L.collect_a : L.collect_b) {
+            const int slot = atomicAdd(lo ? ccnt_a : ccnt_b, 1);
+            if (slot < kCandCapC) {
+              h[2 * slot] = key;
+              h[2 * slot + 1] = (uint32_t)(n0 + (e & 1));
+            }
+          } else {
+            const uint32_t t = key - (lo ? L.base_a : L.base_b);
+            add_mass(h + 2 * (t >> (lo ? L.shift_a : L.shift_b)), fmaf(s - (lo ? L.ref_a : L.ref_b), kLog2eC, 20.0f));
+          }
         }
       }
     }
@@ -200,10 +242,11 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
     int32_t* __restrict__ sel_tie_last, int32_t* status, const int n_row_tiles, const int max_passes) {
   constexpr int BMP = kCRows / G;
   extern __shared__ __align__(128) unsigned char smem[];
-  float* hist = reinterpret_cast<float*>(smem);                            // [128][128] floats
+  uint32_t* hist = reinterpret_cast<uint32_t*>(smem);                      // [128 rows][128 words]
   unsigned char* stage_s = smem + kHistBytes;
   RowState* rs = reinterpret_cast<RowState*>(smem + kHistBytes + 2 * kStageBytesC);
   __shared__ int s_pending;
+  constexpr int kRowWords = kRowBytes / 4;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, c = lane & 3;
@@ -251,7 +294,6 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
     const bool ok = hs < nh && po < rows_here;
     z.n_keys = ok ? min(m0 + po, seq_len - 1) + 1 : 0;
     z.phase = ok && z.n_keys > 0 ? kPhMax : kPhDone;
-    z.hi_count = 0xffffffffu;
     if (ok && z.n_keys > 0 && (d.top_p >= 1.0f || z.n_keys == 1)) {   // everything is selected
       z.phase = kPhDone;
       z.thr_key = 0u;
@@ -281,37 +323,50 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
   };
 
   const bool want_ids = sel_idx != nullptr;
-  float* hist_a = hist + la * kL1Bins;
-  float* hist_b = hist + lb * kL1Bins;
+  uint32_t* hist_a = hist + la * kRowWords;
+  uint32_t* hist_b = hist + lb * kRowWords;
   const float scale = d.score_scale;
+  const float kInf = __int_as_float(0x7f800000);
 
   for (int pass = 0; pass < max_passes; ++pass) {
     // ---- what does this pass do for my two rows? ----
     const RowState sa = rs[la], sb = rs[lb];
     const int ph_a = a_ok ? sa.phase : kPhDone, ph_b = b_ok ? sb.phase : kPhDone;
     if (tid == 0) s_pending = 0;
-    for (int i = lane; i < 16 * kL1Bins; i += 32) hist[wrow * kL1Bins + i] = 0.f;   // this warp's histograms
+    for (int i = lane; i < 16 * kRowWords; i += 32) hist[wrow * kRowWords + i] = 0u;   // this warp's rows
     __syncthreads();
     const bool warp_active = __any_sync(0xffffffffu, ph_a != kPhDone || ph_b != kPhDone);
-    // All rows of a warp do the max pass and the level-1 pass together; later passes mix key levels and ties.
+    // All rows of a warp do the max pass and the level-1 pass together; later passes mix key levels,
+    // candidate collection and ties.
     const bool pass_max = __any_sync(0xffffffffu, ph_a == kPhMax || ph_b == kPhMax);
     const bool pass_l1 = __any_sync(0xffffffffu, ph_a == kPhL1 || ph_b == kPhL1);
     const bool pass_tie = __any_sync(0xffffffffu, ph_a == kPhTie || ph_b == kPhTie);
+    const bool pass_count = __any_sync(0xffffffffu, ph_a == kPhCollect || ph_b == kPhCollect);
 
     LaneRows LR;
-    const float kInf = __int_as_float(0x7f800000);
     LR.M_a = sa.M; LR.M_b = sb.M;
     LR.pos_a = pos_a; LR.pos_b = pos_b;
     LR.base_a = sa.base_key; LR.base_b = sb.base_key;
     LR.shift_a = sa.shift; LR.shift_b = sb.shift;
-    LR.lo_a = ph_a == kPhKey ? sa.raw_lo : kInf;  LR.hi_a = ph_a == kPhKey ? sa.raw_hi : -kInf;
-    LR.lo_b = ph_b == kPhKey ? sb.raw_lo : kInf;  LR.hi_b = ph_b == kPhKey ? sb.raw_hi : -kInf;
-    LR.hic_a = ph_a == kPhKey ? sa.raw_hic : kInf;
-    LR.hic_b = ph_b == kPhKey ? sb.raw_hic : kInf;
+    LR.ref_a = sa.ref_s; LR.ref_b = sb.ref_s;
+    const bool in_a = ph_a == kPhKey || ph_a == kPhCollect || ph_a == kPhTie;
+    const bool in_b = ph_b == kPhKey || ph_b == kPhCollect || ph_b == kPhTie;
+    LR.lo_a = in_a ? sa.raw_lo : kInf;  LR.hi_a = in_a ? sa.raw_hi : -kInf;
+    LR.lo_b = in_b ? sb.raw_lo : kInf;  LR.hi_b = in_b ? sb.raw_hi : -kInf;
+    // centre / half width of the interval; the half width is rounded up so that the quick test never rejects a member
+    LR.mid_a = in_a ? 0.5f * sa.raw_lo + 0.5f * sa.raw_hi : 0.f;
+    LR.mid_b = in_b ? 0.5f * sb.raw_lo + 0.5f * sb.raw_hi : 0.f;
+    LR.hw_a = in_a ? fmaxf(sa.raw_hi - LR.mid_a, LR.mid_a - sa.raw_lo) * 1.000001f + 1e-30f : -1.f;
+    LR.hw_b = in_b ? fmaxf(sb.raw_hi - LR.mid_b, LR.mid_b - sb.raw_lo) * 1.000001f + 1e-30f : -1.f;
+    LR.collect_a = ph_a == kPhCollect;  LR.collect_b = ph_b == kPhCollect;
+    LR.cut_a = LR.collect_a ? sa.raw_hi : kInf;
+    LR.cut_b = LR.collect_b ? sb.raw_hi : kInf;
     const bool tie_a = ph_a == kPhTie, tie_b = ph_b == kPhTie;
-    LR.tlo_a = tie_a ? sa.tie_lo : kInf;  LR.thi_a = tie_a ? sa.tie_hi : -kInf;
-    LR.tlo_b = tie_b ? sb.tie_lo : kInf;  LR.thi_b = tie_b ? sb.tie_hi : -kInf;
+    LR.tlo_a = tie_a ? sa.raw_lo : kInf;  LR.thi_a = tie_a ? sa.raw_hi : -kInf;
+    LR.tlo_b = tie_b ? sb.raw_lo : kInf;  LR.thi_b = tie_b ? sb.raw_hi : -kInf;
     const int need_a = tie_a ? sa.tie_need : 0, need_b = tie_b ? sb.tie_need : 0;
+    int* ccnt_a = &rs[la].cand_cnt;
+    int* ccnt_b = &rs[lb].cand_cnt;
 
     float mx_a = -INFINITY, mx_b = -INFINITY;
     int cnt_a = 0, cnt_b = 0;
@@ -340,12 +395,16 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
           } else if (pass_l1) {
             if (interior) page_l1<false>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b);
             else page_l1<true>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b);
-          } else if (pass_tie) {
-            if (interior) page_late<false, true>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b, cnt_a, cnt_b, need_a, need_b, run_a, run_b, tl_a, tl_b);
-            else page_late<true, true>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b, cnt_a, cnt_b, need_a, need_b, run_a, run_b, tl_a, tl_b);
           } else {
-            if (interior) page_late<false, false>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b, cnt_a, cnt_b, need_a, need_b, run_a, run_b, tl_a, tl_b);
-            else page_late<true, false>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b, cnt_a, cnt_b, need_a, need_b, run_a, run_b, tl_a, tl_b);
+#define RTP_LATE(M_, T_, C_) page_late<M_, T_, C_>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b, ccnt_a, ccnt_b, cnt_a, cnt_b, need_a, need_b, run_a, run_b, tl_a, tl_b)
+            if (pass_tie) {
+              if (interior) RTP_LATE(false, true, true); else RTP_LATE(true, true, true);
+            } else if (pass_count) {
+              if (interior) RTP_LATE(false, false, true); else RTP_LATE(true, false, true);
+            } else {
+              if (interior) RTP_LATE(false, false, false); else RTP_LATE(true, false, false);
+            }
+#undef RTP_LATE
           }
         }
       }
@@ -378,6 +437,7 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
       const int ph = R.phase;
       const int src_lane = (rr & 7) * 4;          // a lane of the quad that owns row rr
       const bool is_b = rr >= 8;
+      const uint32_t* h = hist + lr * kRowWords;
       if (ph == kPhDone || R.n_keys == 0) continue;
       if (ph == kPhMax) {
         // the maximum was taken on unscaled MMA outputs; scaling by a positive factor is monotone
@@ -386,178 +446,209 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
           S->M = M;
           S->phase = kPhL1;
         }
-      } else if (ph == kPhL1) {
-        // 128 bins, 4 per lane, bin 0 = highest scores
-        float m4[4], tot = 0.f;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          m4[k] = hist[lr * kL1Bins + lane * 4 + k];
-          tot += m4[k];
+      } else if (ph == kPhL1 || ph == kPhKey) {
+        // 64 bins of {hi, lo}; two bins per lane in order of decreasing score:
+        //   level 1: bin 0 is the top -> lane l takes bins 2l, 2l+1;  key levels: bin 63 is the top -> 63-2l, 62-2l
+        const bool l1 = ph == kPhL1;
+        const int b0 = l1 ? 2 * lane : 63 - 2 * lane, b1 = l1 ? 2 * lane + 1 : 62 - 2 * lane;
+        const uint32_t hi0 = h[2 * b0], lo0 = h[2 * b0 + 1], hi1 = h[2 * b1], lo1 = h[2 * b1 + 1];
+        // masses relative to M
+        float m0f, m1f;
+        if (l1) {
+          m0f = acc_mass(hi0, lo0) * fast_ex2(-0.5f * kLog2eC * (float)b0 - 20.0f);
+          m1f = acc_mass(hi1, lo1) * fast_ex2(-0.5f * kLog2eC * (float)b1 - 20.0f);
+        } else {
+          const float sc = R.e_ref * 9.5367431640625e-07f;   // 2^-20
+          m0f = acc_mass(hi0, lo0) * sc;
+          m1f = acc_mass(hi1, lo1) * sc;
         }
-        float inc = tot;
+        float incm = m0f + m1f;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-          const float tt = __shfl_up_sync(0xffffffffu, inc, o);
-          if (lane >= o) inc += tt;
+          const float tm = __shfl_up_sync(0xffffffffu, incm, o);
+          if (lane >= o) incm += tm;
         }
-        const float Z = __shfl_sync(0xffffffffu, inc, 31);
-        const float target = d.top_p * Z * (1.0f + kMassMargin);
-        int found = kL1Bins, lastb = -1;
-        {
-          float run = inc - tot;
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            if (m4[k] > 0.f) {
-              lastb = lane * 4 + k;
-              if (found == kL1Bins && run + m4[k] >= target) found = lane * 4 + k;
-            }
-            run += m4[k];
-          }
+        const float total = __shfl_sync(0xffffffffu, incm, 31);
+        const float Z = l1 ? total : R.Z;
+        const float target = l1 ? d.top_p * Z * (1.0f + kMassMargin) : R.target;
+        const float run = (l1 ? 0.f : R.mass_above) + incm - (m0f + m1f);
+        const bool pop0 = (hi0 | lo0) != 0u, pop1 = (hi1 | lo1) != 0u;
+        // order index of a bin = position from the top (0 .. 63)
+        int found = 64, last = -1;
+        if (pop0) {
+          last = 2 * lane;
+          if (run + m0f >= target) found = 2 * lane;
+        }
+        if (pop1) {
+          last = 2 * lane + 1;
+          if (found == 64 && run + m0f + m1f >= target) found = 2 * lane + 1;
         }
         int best = found;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, o));
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) lastb = max(lastb, __shfl_xor_sync(0xffffffffu, lastb, o));
-        // rounding may leave the target just out of reach: then the lowest populated bin is the bucket
-        if (best == kL1Bins) best = lastb;
-        if (best >= 0 && (best >> 2) == lane) {
-          float above = inc - tot;
-          for (int k = 0; k < (best & 3); ++k) above += m4[k];
-          S->Z = Z;
-          S->target = target;
-          S->mass_above = above;
-          if (best == kL1Bins - 1) {
-            // the cut falls into the pooled tail (mass below 2e-14 per key): take every key
-            S->thr_key = 0u;
-            S->tie_last = R.n_keys - 1;
-            S->count = R.n_keys;
-            S->sel_mass = 1.0f;
-            S->phase = kPhDone;
-          } else {
-            // Exact interval [klo, khi] of ordered keys whose level-1 bin is `best`: l1_bin is monotone in the
-            // key, so both ends are found by bisection between two keys that lie safely outside the bucket.
-            const float M = R.M;
-            const float hi_s = M - (float)best / kL1Scale, lo_s = M - (float)(best + 1) / kL1Scale;
-            const float pad = 1e-5f * fmaxf(1.0f, fmaxf(fabsf(hi_s), fabsf(lo_s))) + 1e-3f;
-            const uint32_t lo = okey(finish_score(lo_s - pad, 1.0f));
-            const uint32_t hi = okey(finish_score(fminf(hi_s + pad, M), 1.0f));
-            // klo = smallest key with bin <= best
-            uint32_t a = lo, b2 = hi;            // invariant: bin(b2) <= best; bin(a) > best unless a is the answer
-            if (l1_bin(M, okey_to_float(a)) <= best) b2 = a;
-            while (a + 1 < b2) {
-              const uint32_t mid = a + ((b2 - a) >> 1);
-              if (l1_bin(M, okey_to_float(mid)) <= best) b2 = mid; else a = mid;
-            }
-            const uint32_t klo = b2;
-            // khi = largest key with bin >= best
-            a = klo; b2 = hi;                    // invariant: bin(a) >= best; bin(b2) < best unless b2 is the answer
-            if (l1_bin(M, okey_to_float(b2)) >= best) a = b2;
-            while (a + 1 < b2) {
-              const uint32_t mid = a + ((b2 - a) >> 1);
-              if (l1_bin(M, okey_to_float(mid)) >= best) a = mid; else b2 = mid;
-            }
-            const uint32_t khi = a;
-            const uint32_t span = khi - klo + 1u;
-            const int bits = span > 1u ? 32 - __clz(span - 1u) : 0;
-            float rlo, rhi;
-            raw_preimage(scale, klo, khi, rlo, rhi);
-            S->base_key = klo;
-            S->span = span;
-            S->shift = max(0, bits - 6);
-            S->hi_count = khi;
-            S->raw_lo = rlo;
-            S->raw_hi = rhi;
-            S->raw_hic = rhi;
-            S->cnt_above = 0;
-            S->phase = kPhKey;
-          }
-        }
-      } else if (ph == kPhKey) {
-        // 64 bins of {mass, count}; bin 63 = highest keys.  Two bins per lane, lane 0 takes the top.
-        const float* h = hist + lr * kL1Bins;
-        const int bhi = 63 - 2 * lane, blo = bhi - 1;
-        const float mh = h[2 * bhi], ml = h[2 * blo];
-        const int ch = __float_as_int(h[2 * bhi + 1]), cl = __float_as_int(h[2 * blo + 1]);
-        float incm = mh + ml;
-        int incc = ch + cl;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const float tm = __shfl_up_sync(0xffffffffu, incm, o);
-          const int tc = __shfl_up_sync(0xffffffffu, incc, o);
-          if (lane >= o) {
-            incm += tm;
-            incc += tc;
-          }
-        }
-        const int extra_above = __shfl_sync(0xffffffffu, is_b ? cnt_b : cnt_a, src_lane);
-        const float target = R.target;
-        const float run = R.mass_above + incm - (mh + ml);
-        const int runc = incc - (ch + cl);
-        int found = -1, lowest = 64;
-        if (ch > 0) {
-          lowest = bhi;
-          if (run + mh >= target) found = bhi;
-        }
-        if (cl > 0) {
-          lowest = blo;
-          if (found < 0 && run + mh + ml >= target) found = blo;
-        }
-        int best = found;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) lowest = min(lowest, __shfl_xor_sync(0xffffffffu, lowest, o));
-        if (best < 0) best = lowest;   // target out of reach by rounding: lowest populated bin
-        if (best >= 64) {
-          // empty bucket: cannot happen (the level-1 bucket holds at least one key)
-          if (lane == 0) {
+        for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+        if (best == 64) best = last;   // rounding left the target just out of reach: lowest populated bin
+        if (best < 0) {
+          if (lane == 0) {             // empty histogram: cannot happen for a non-empty row
             S->phase = kPhDone;
             set_status(status, RTP_ERR_UNSUPPORTED);
           }
-        } else if (best == bhi || best == blo) {
-          const bool top = best == bhi;
-          const float f_above = top ? run : run + mh;
-          const int f_cnt_above = top ? runc : runc + ch;
-          const int f_cnt = top ? ch : cl;
-          const float f_mass = top ? mh : ml;
-          const int shift = R.shift;
-          const uint32_t ofs = (uint32_t)best << shift;
-          const uint32_t lo_key = R.base_key + ofs;
-          const uint32_t sub_span = min(1u << shift, R.span - ofs);
-          const int cnt_above = R.cnt_above + extra_above + f_cnt_above;
+        } else if ((best >> 1) == lane) {
+          const bool first = (best & 1) == 0;
+          const float f_above = first ? run : run + m0f;
+          const uint32_t f_hi = first ? hi0 : hi1;
+          const int bin = first ? b0 : b1;
+          const bool few = f_hi / kMinHi < (uint32_t)kCandCapC;   // at most (f_hi / kMinHi) keys in the bin
           S->mass_above = f_above;
-          S->cnt_above = cnt_above;
-          float rlo, rhi;
-          raw_preimage(scale, lo_key, lo_key + (sub_span - 1u), rlo, rhi);
-          S->base_key = lo_key;
-          S->span = sub_span;
-          S->hi_count = 0xffffffffu;
-          S->raw_lo = rlo;
-          S->raw_hi = rhi;
-          S->raw_hic = __int_as_float(0x7f800000);
-          if (f_cnt == 1 || shift == 0) {
-            // resolved: one key left, or a single key value (f_cnt equal scores)
-            int take = f_cnt;
-            if (f_cnt > 1) {
-              const float each = f_mass / (float)f_cnt;
-              take = (int)ceilf((target - f_above) / each);
-              take = max(1, min(take, f_cnt));
+          if (l1) {
+            S->Z = Z;
+            S->target = target;
+            if (bin == kBins - 1) {
+              // the cut falls into the pooled tail (mass below 2e-14 per key): take every key
+              S->thr_key = 0u;
+              S->tie_last = R.n_keys - 1;
+              S->count = R.n_keys;
+              S->sel_mass = 1.0f;
+              S->phase = kPhDone;
+            } else {
+              // Exact interval [klo, khi] of ordered keys whose level-1 bin is `bin`: l1_bin is monotone in the
+              // key, so both ends are found by bisection between two keys that lie safely outside the bucket.
+              const float M = R.M;
+              const float hi_s = M - (float)bin / kL1Scale, lo_s = M - (float)(bin + 1) / kL1Scale;
+              const float pad = 1e-5f * fmaxf(1.0f, fmaxf(fabsf(hi_s), fabsf(lo_s))) + 1e-3f;
+              const uint32_t lo = okey(finish_score(lo_s - pad, 1.0f));
+              const uint32_t hi = okey(finish_score(fminf(hi_s + pad, M), 1.0f));
+              uint32_t a = lo, b2 = hi;            // klo = smallest key with bin <= `bin`
+              if (l1_bin(M, okey_to_float(a)) <= bin) b2 = a;
+              while (a + 1 < b2) {
+                const uint32_t mid = a + ((b2 - a) >> 1);
+                if (l1_bin(M, okey_to_float(mid)) <= bin) b2 = mid; else a = mid;
+              }
+              const uint32_t klo = b2;
+              a = klo; b2 = hi;                    // khi = largest key with bin >= `bin`
+              if (l1_bin(M, okey_to_float(b2)) >= bin) a = b2;
+              while (a + 1 < b2) {
+                const uint32_t mid = a + ((b2 - a) >> 1);
+                if (l1_bin(M, okey_to_float(mid)) >= bin) a = mid; else b2 = mid;
+              }
+              const uint32_t khi = a;
+              const uint32_t span = khi - klo + 1u;
+              const int bits = span > 1u ? 32 - __clz(span - 1u) : 0;
+              float rlo, rhi;
+              raw_preimage(scale, klo, khi, rlo, rhi);
+              S->ref_s = hi_s;
+              S->e_ref = fast_ex2(-0.5f * kLog2eC * (float)bin);
+              S->base_key = klo;
+              S->span = span;
+              S->shift = max(0, bits - 6);
+              S->raw_lo = rlo;
+              S->raw_hi = rhi;
+              S->cand_cnt = 0;
+              S->phase = (few || span == 1u) ? kPhCollect : kPhKey;
             }
-            S->thr_key = lo_key;
-            S->count = cnt_above + take;
-            S->sel_mass = (f_above + f_mass * ((float)take / (float)f_cnt)) / R.Z;
-            if (take < f_cnt) {
+          } else {
+            const int shift = R.shift;
+            const uint32_t ofs = (uint32_t)bin << shift;
+            const uint32_t lo_key = R.base_key + ofs;
+            const uint32_t sub_span = min(1u << shift, R.span - ofs);
+            float rlo, rhi;
+            raw_preimage(scale, lo_key, lo_key + (sub_span - 1u), rlo, rhi);
+            S->base_key = lo_key;
+            S->span = sub_span;
+            S->shift = max(0, shift - 6);
+            S->raw_lo = rlo;
+            S->raw_hi = rhi;
+            S->cand_cnt = 0;
+            S->phase = (few || sub_span == 1u) ? kPhCollect : kPhKey;
+          }
+        }
+      } else if (ph == kPhCollect) {
+        const int n_c = R.cand_cnt;                  // keys inside the bucket
+        const int above = R.cnt_above + __shfl_sync(0xffffffffu, is_b ? cnt_b : cnt_a, src_lane);
+        if (n_c > kCandCapC) {
+          // only reachable when the bucket is a single key value: n_c equal scores straddle the cut
+          if (lane == 0) {
+            const float each = fast_ex2((okey_to_float(R.base_key) - R.M) * kLog2eC);
+            int take = (int)ceilf((R.target - R.mass_above) / each);
+            take = max(1, min(take, n_c));
+            S->cnt_above = above;
+            S->thr_key = R.base_key;
+            S->count = above + take;
+            S->sel_mass = (R.mass_above + (float)take * each) / R.Z;
+            if (R.span != 1u) set_status(status, RTP_ERR_UNSUPPORTED);
+            if (take < n_c) {
               S->tie_need = take;
-              S->tie_lo = rlo;   // shift == 0 here: the bucket is the single key value lo_key
-              S->tie_hi = rhi;
               S->phase = kPhTie;
             } else {
               S->tie_last = R.n_keys - 1;
               S->phase = kPhDone;
             }
-          } else {
-            S->shift = max(0, shift - 6);
+          }
+        } else {
+          // exact finish: rank the (at most 64) candidates by (score descending, position ascending)
+          unsigned long long ord[2];
+          float e[2];
+#pragma unroll
+          for (int x = 0; x < 2; ++x) {
+            const int i = 2 * lane + x;
+            ord[x] = ~0ull;
+            e[x] = 0.f;
+            if (i < n_c) {
+              const uint32_t key = h[2 * i], idx = h[2 * i + 1];
+              ord[x] = ((unsigned long long)(~key) << 32) | idx;
+              e[x] = fast_ex2((okey_to_float(key) - R.M) * kLog2eC);
+            }
+          }
+          int rank[2] = {0, 0};
+          float cum[2] = {R.mass_above, R.mass_above};
+          for (int j = 0; j < n_c; ++j) {
+            const int jl = j >> 1;
+            const unsigned long long oj = __shfl_sync(0xffffffffu, (j & 1) ? ord[1] : ord[0], jl);
+            const float ej = __shfl_sync(0xffffffffu, (j & 1) ? e[1] : e[0], jl);
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+              if (oj < ord[x]) ++rank[x];
+              if (oj <= ord[x]) cum[x] += ej;
+            }
+          }
+          // shortest prefix whose cumulative mass reaches the target (all candidates if none does)
+          int pick = 1 << 20;
+#pragma unroll
+          for (int x = 0; x < 2; ++x)
+            if (2 * lane + x < n_c && cum[x] >= R.target) pick = min(pick, rank[x]);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) pick = min(pick, __shfl_xor_sync(0xffffffffu, pick, o));
+          if (pick == (1 << 20)) pick = n_c - 1;
+          // the candidate of rank `pick` defines the threshold; ties with it that were taken have rank <= pick
+          uint32_t thr_key = 0;
+          float pick_cum = 0.f;
+#pragma unroll
+          for (int x = 0; x < 2; ++x)
+            if (2 * lane + x < n_c && rank[x] == pick) {
+              thr_key = ~(uint32_t)(ord[x] >> 32);
+              pick_cum = cum[x];
+            }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            thr_key = max(thr_key, __shfl_xor_sync(0xffffffffu, thr_key, o));
+            pick_cum = fmaxf(pick_cum, __shfl_xor_sync(0xffffffffu, pick_cum, o));
+          }
+          int tie_last = -1;
+#pragma unroll
+          for (int x = 0; x < 2; ++x)
+            if (2 * lane + x < n_c && rank[x] <= pick && ~(uint32_t)(ord[x] >> 32) == thr_key)
+              tie_last = max(tie_last, (int)(uint32_t)ord[x]);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) tie_last = max(tie_last, __shfl_xor_sync(0xffffffffu, tie_last, o));
+          if (lane == 0) {
+            S->cnt_above = above;
+            S->thr_key = thr_key;
+            S->tie_last = tie_last;
+            S->count = above + pick + 1;
+            S->sel_mass = pick_cum / R.Z;
+            S->phase = kPhDone;
+            if (n_c == 0) set_status(status, RTP_ERR_UNSUPPORTED);   // a chosen bucket always holds a key
           }
         }
       } else if (ph == kPhTie) {

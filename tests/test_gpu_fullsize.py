@@ -35,12 +35,20 @@ def test_prefill_128k_sampled_rows():
     assert path.status_code() == rb.RTP_OK
     rng = np.random.default_rng(1)
     rows = sorted({0, 1, 63, 64, chunk - 1, chunk, L - 1, L - chunk, *map(int, rng.integers(0, L, 6))})
-    # GPU-written index keys and projected queries feed the oracle's scoring (stage-wise parity)
+    # stage-wise parity on the sampled rows: GPU-written index keys and projected queries feed the oracle's
+    # scoring; the selection is judged on the GPU's own materialised scores; attention on the GPU's own set
     ik = _np16(path.ikey_pages[data.block_table[0].long()])               # [pages, nih, 64, 16]
     kt = np.transpose(ik, (0, 2, 1, 3)).reshape(-1, heads.n_index_heads, 16)[:L]
     qt = torch.empty((len(rows), path.n_ret, 16), dtype=torch.bfloat16, device="cuda")
     qrows = data.q[torch.tensor(rows, device="cuda")].contiguous()
     rb.rtp_index_queries(path.ctx, path.params, qrows, data.w_q, qt)
+    sc = torch.full((len(rows), path.n_ret, L), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(rb.rtp_workspace_bytes(path.params, len(rows), L), dtype=torch.uint8, device="cuda")
+    rb.rtp_index_score(path.ctx, path.params, path.cache, qrows, data.w_q,
+                       torch.zeros(len(rows), dtype=torch.int32, device="cuda"),
+                       torch.tensor(rows, dtype=torch.int32, device="cuda"), sc, None, None, ws, path.status)
+    torch.cuda.synchronize()
+    sc = sc.cpu().numpy()
     qt, qh = _np16(qt), _np16(qrows)
     thr_h, tie_h, cnt_h, mass_h = thr.cpu().numpy(), tie.cpu().numpy(), cnt.cpu().numpy(), mass.cpu().numpy()
     out_h, lse_h = out.float().cpu().numpy(), lse.cpu().numpy()
@@ -51,14 +59,19 @@ def test_prefill_128k_sampled_rows():
             kh = h // g
             if kh not in kv:
                 kv[kh] = data.logical_kv(0, kh)
-            s = orc.index_scores(qt[k, i], kt[: m + 1, heads.q_head_to_index_head[i]], data.score_scale)
+            s = sc[k, i, : m + 1]
+            want_s = orc.index_scores(qt[k, i], kt[: m + 1, heads.q_head_to_index_head[i]], data.score_scale)
+            qn = np.linalg.norm(orc.bf16_to_f64(qt[k, i]))
+            kn = np.linalg.norm(orc.bf16_to_f64(kt[: m + 1, heads.q_head_to_index_head[i]]), axis=-1)
+            assert np.all(np.abs(s - want_s) <= 1e-3 * np.abs(want_s) + 1e-5 * data.score_scale * qn * kn)
             member = (s > thr_h[m, i]) | ((s == thr_h[m, i]) & (np.arange(m + 1) <= tie_h[m, i]))
             got = set(np.nonzero(member)[0].tolist())
-            # the oracle's scores differ from the GPU's in the last bits, so compare through the band rule
-            mand, forb = orc.classify_against_band(s, data.top_p, band=2e-3)
+            assert len(got) == int(cnt_h[m, i]), f"row {m} head {i}"
+            mand, forb = orc.classify_against_band(s, data.top_p)
             assert mand <= got and not (forb & got), f"row {m} head {i}"
-            assert abs(len(got) - int(cnt_h[m, i])) <= max(2, int(0.002 * (m + 1)))
-            assert orc.set_mass(s, got) >= data.top_p - 1e-3
+            tm = orc.set_mass(s, got)
+            assert tm >= data.top_p or len(got) == m + 1
+            assert abs(tm - mass_h[m, i]) <= 1e-4
             want, wlse = orc.attention_over_set(qh[k, h], kv[kh][0], kv[kh][1], sorted(got), data.sm_scale)
             assert np.abs(out_h[m, h] - want).max() <= 2e-2, f"sparse row {m} head {h}"
             fr.append(len(got) / (m + 1))
