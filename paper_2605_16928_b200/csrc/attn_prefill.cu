@@ -10,6 +10,8 @@
 //   sparse  every tile up to the diagonal; membership of (row, key) in S_h(m) is re-evaluated from
 //           the 16-dim indexer score and the row's (threshold, tie position) pair, and a warp skips
 //           the two big MMAs of a tile in which none of its rows selects a key     (Eq. 5, S6)
+#include <cstdlib>
+
 #include "rtp_device.cuh"
 
 namespace rtp {
@@ -398,6 +400,11 @@ cudaError_t launch_attn_prefill(const CacheView& cv, const Dims& d, const HeadMa
                                        d.n_ih, st);
   }
   if (hm.n_kv_list == 0) return cudaSuccess;
+  {
+    // dense and sink+window modes run on tcgen05 / TMEM / TMA; RTP_PREFILL_TC=0 selects the warp-MMA kernel below
+    static const bool use_tc = [] { const char* e = getenv("RTP_PREFILL_TC"); return !(e && e[0] == '0'); }();
+    if (use_tc) return launch_attn_prefill_tc(cv, d, hm, mode, q, seq_id, q_start, C, out, lse, status, st);
+  }
   if (mode == kPrefillLocal)
     return launch_mode<kPrefillLocal>(cv, d, hm, q, qt, seq_id, q_start, C, sel_thresh, sel_tie_last, out, lse,
                                       hm.n_kv_list, st);

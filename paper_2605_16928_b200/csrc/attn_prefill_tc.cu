@@ -1,0 +1,526 @@
+// S7 / S9 for a prefill chunk on the 5th-generation tensor cores (tcgen05 + TMEM), dense and
+// sink+window modes.
+//
+// One CTA (320 threads, one per SM) owns 128 MMA rows = (128 / G) consecutive positions x the G query
+// heads of one KV head and walks the key tiles of 128 keys (two cache pages):
+//   warp 9    loader: K and V pages -> shared memory in the 128-byte-swizzled layout the MMA unit reads; TMA
+//             (cp.async.bulk.tensor, one lane) for whole tiles, zero-filling cp.async for the last tile; two stages
+//   warp 8    one elected lane issues tcgen05.mma: S = Q K^T (128 x 128 x 128) into one of two TMEM
+//             buffers, then O += P V (128 x 128 x 128) once the softmax warps have written P
+//   warps 0-7 two threads per row (TMEM lane = row, half of the columns each): reads S with tcgen05.ld, masks, online softmax,
+//             writes P (bf16) to shared memory; O accumulates in TMEM across tiles and is rescaled there
+//             only when the running reference maximum has to be raised
+// Hand-offs are mbarriers (tcgen05.commit on the MMA side).  Every wait is bounded: when a wait runs
+// out, the CTA records RTP_ERR_TIMEOUT, stops waiting (all later waits return at once), still walks its
+// loops to the end, frees its TMEM and exits.
+#include <cuda.h>
+
+#include "rtp_device.cuh"
+
+namespace rtp {
+
+namespace {
+
+constexpr int kBM = 128;
+constexpr int kBNt = 128;                 // keys per tile
+constexpr int kTcThreads = 320;           // warps 0-7 softmax, 8 MMA, 9 loader
+constexpr int kMmaWarp = 8, kLoadWarp0 = 9;
+constexpr int kBlk = 128 * 128;           // bytes of one [128 rows][64 elements] bf16 block (16 KB)
+constexpr int kQOff = 0;                  // Q: 2 blocks (dims 0-63, 64-127)
+constexpr int kKOff = 2 * kBlk;           // K: 2 stages x 2 blocks
+constexpr int kVOff = kKOff + 4 * kBlk;   // V: 2 stages x 2 blocks
+constexpr int kPOff = kVOff + 4 * kBlk;   // P: 2 blocks (keys 0-63, 64-127)
+constexpr int kBarOff = kPOff + 2 * kBlk; // mbarriers + TMEM base + abort flag
+constexpr int kXchOff = kBarOff + 256;     // float [2 tiles][2 halves][128 rows]: row-maximum exchange
+constexpr int kTcSmem = kXchOff + 2048 + 1024;   // + slack for 1024-byte alignment of the base
+constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr float kLog2eT = 1.4426950408889634f;
+constexpr float kLn2T = 0.6931471805599453f;
+
+enum Bar { kFullK0 = 0, kFullK1, kFullV0, kFullV1, kEmptyKV0, kEmptyKV1, kSFull0, kSFull1, kSEmpty0, kSEmpty1,
+           kPFull, kPEmpty, kNumBars };
+
+__device__ __forceinline__ uint32_t s_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  `abort_flag` (shared) is set by whoever runs out first; afterwards nobody waits any more.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (*abort_flag) return;
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try(bar, parity)) return;
+    if ((i & 1023u) == 1023u && *abort_flag) return;
+  }
+  *abort_flag = 1;
+  set_status(status, RTP_ERR_TIMEOUT);
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// 2-D tiled bulk tensor load (TMA): box -> shared memory, completion counted in bytes on an mbarrier.
+// x = innermost coordinate (elements; x * 2 bytes is a multiple of 16 here: 0 or 64), y = row.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+#define RTP_TMEM_LD32(r, addr)                                                                                     \
+  asm volatile(                                                                                                    \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                                    \
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28," \
+      "%29,%30,%31}, [%32];"                                                                                       \
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), \
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),      \
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),     \
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])                   \
+      : "r"(addr)                                                                                                  \
+      : "memory")
+#define RTP_TMEM_ST32(addr, r)                                                                                     \
+  asm volatile(                                                                                                    \
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "                                                              \
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29," \
+      "%30,%31,%32};" ::"r"(addr),                                                                                 \
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), \
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),   \
+      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),   \
+      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])                                                               \
+      : "memory")
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  sbo = byte distance between 8-row groups; lbo = byte
+// distance between 64-element atoms along the contiguous dimension (only used by MN-major operands).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3ffffu) >> 4);
+  d |= (uint64_t)((lbo >> 4) & 0x3fffu) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3fffu) << 32;
+  d |= (uint64_t)1 << 46;   // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;   // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; b_mn = B operand is MN-major (V as stored).
+__device__ __forceinline__ uint32_t instr_desc(bool b_mn) {
+  uint32_t d = 0;
+  d |= 1u << 4;                     // D format fp32
+  d |= 1u << 7;                     // A format bf16
+  d |= 1u << 10;                    // B format bf16
+  d |= (b_mn ? 1u : 0u) << 16;      // B major
+  d |= (uint32_t)(kBNt >> 3) << 17; // N / 8
+  d |= (uint32_t)(kBM >> 4) << 24;  // M / 16
+  return d;
+}
+__device__ __forceinline__ void cp16(uint32_t dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+// byte offset of 16-byte chunk c (0..7) of row r inside a [rows][64 elements] swizzled block
+__device__ __forceinline__ uint32_t sw128(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
+
+template <int G, int MODE>
+__global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
+    const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+    const CacheView cv, const Dims d, const HeadMaps hm, const __nv_bfloat16* __restrict__ q, const int seq_id,
+    const int q_start, const int C, __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int32_t* status,
+    const int n_row_tiles) {
+  constexpr int BMP = kBM / G;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = s_u32(smem);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kBarOff + kNumBars * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kBarOff + kNumBars * 8 + 8);
+  auto bar = [&](int i) { return sbase + kBarOff + i * 8; };
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tile = n_row_tiles - 1 - blockIdx.x;
+  const int kvh = hm.kv_list[blockIdx.y];
+  const int r0 = tile * BMP, m0 = q_start + r0;
+  const int rows_here = min(BMP, C - r0);
+  const int m_last = m0 + rows_here - 1;
+
+  // key tiles of 128 keys visited by this CTA
+  const int kt_last = m_last / kBNt;
+  int kt_first = 0, n_sink_tiles = 0;
+  if (MODE == kPrefillLocal) {
+    kt_first = max(0, m0 - d.window + 1) / kBNt;
+    n_sink_tiles = min((d.n_sink + kBNt - 1) / kBNt, kt_first);
+  }
+  const int n_tiles = n_sink_tiles + (kt_last - kt_first + 1);
+  auto tile_at = [&](int i) { return i < n_sink_tiles ? i : kt_first + (i - n_sink_tiles); };
+
+  if (tid == 0) {
+    mbar_init(bar(kFullK0), 1); mbar_init(bar(kFullK1), 1);
+    mbar_init(bar(kFullV0), 1); mbar_init(bar(kFullV1), 1);
+    mbar_init(bar(kEmptyKV0), 1); mbar_init(bar(kEmptyKV1), 1);
+    mbar_init(bar(kSFull0), 1); mbar_init(bar(kSFull1), 1);
+    mbar_init(bar(kSEmpty0), 256); mbar_init(bar(kSEmpty1), 256);
+    mbar_init(bar(kPFull), 256);
+    mbar_init(bar(kPEmpty), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kMmaWarp) {   // TMEM: 512 columns (S0, S1, O_tile; one CTA per SM)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(tmem_slot)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // Q tile -> shared (rows = [head][position]), by the softmax warps
+  if (warp < 8) {
+    for (int i = tid; i < kBM * 16; i += 256) {
+      const int row = i >> 4, ch = i & 15;
+      const int hs = row / BMP, po = row % BMP;
+      const bool ok = po < rows_here;
+      const __nv_bfloat16* src = q + ((int64_t)(r0 + (ok ? po : 0)) * d.n_q + kvh * d.group + hs) * kHeadDim + ch * 8;
+      cp16(sbase + kQOff + (ch >> 3) * kBlk + sw128(row, ch & 7), src, ok);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    fence_async_smem();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem_s[2] = {tmem, tmem + 128u};
+  const uint32_t tmem_o = tmem + 256u;
+
+  if (warp >= kLoadWarp0) {
+    // ================================ loader ================================
+    // Tiles whose 128 keys all exist are fetched by TMA (eight 8 KB boxes, completion in bytes on the stage's
+    // barriers; the warp does not wait for them).  The tile that holds the last position may reach into cache
+    // slots that were never written: it is copied with cp.async and zero-filled beyond the last position.
+    const int64_t bt_base = (int64_t)seq_id * cv.max_pages;
+    const int last_page = m_last >> kPageShift;
+    const int rsub = lane >> 3, ch = lane & 7;     // 4 rows x 8 chunks per warp instruction
+    for (int it = 0; it < n_tiles; ++it) {
+      const int stage = it & 1;
+      if (it >= 2) mbar_wait(bar(kEmptyKV0 + stage), ((it >> 1) - 1) & 1, abort_flag, status);
+      const int kt = tile_at(it);
+      const bool whole = kt * kBNt + kBNt - 1 <= m_last;
+      if (whole) {
+        if (lane == 0) {
+#pragma unroll
+          for (int which = 0; which < 2; ++which) {
+            const uint32_t dst0 = sbase + (which ? kVOff : kKOff) + stage * 2 * kBlk;
+            const uint32_t fb = bar(which ? kFullV0 + stage : kFullK0 + stage);
+            mbar_expect_tx(fb, 2 * kBlk);
+#pragma unroll
+            for (int pg = 0; pg < 2; ++pg) {
+              const int phys = __ldg(cv.block_table + bt_base + kt * 2 + pg);
+              const int y = (phys * cv.n_kv + kvh) * kPage;
+              tma_load_2d(dst0 + pg * (kPage * 128), which ? &map_v : &map_k, 0, y, fb);
+              tma_load_2d(dst0 + kBlk + pg * (kPage * 128), which ? &map_v : &map_k, 64, y, fb);
+            }
+          }
+        }
+        __syncwarp();
+        continue;
+      }
+#pragma unroll 1
+      for (int which = 0; which < 2; ++which) {     // 0: K, 1: V
+        const __nv_bfloat16* pages = which ? cv.v : cv.k;
+        const uint32_t dst0 = sbase + (which ? kVOff : kKOff) + stage * 2 * kBlk;
+#pragma unroll 1
+        for (int pg = 0; pg < 2; ++pg) {
+          const int page = kt * 2 + pg;
+          const bool page_ok = page <= last_page;
+          const int phys = page_ok ? __ldg(cv.block_table + bt_base + page) : 0;
+          const __nv_bfloat16* src0 = pages + ((int64_t)phys * cv.n_kv + kvh) * (kPage * kHeadDim);
+          const int n_ok = page_ok ? m_last - page * kPage + 1 : 0;   // keys of the page any row may attend
+#pragma unroll 4
+          for (int r4 = 0; r4 < 16; ++r4) {
+            const int row = r4 * 4 + rsub;            // key inside the page
+            const int trow = pg * kPage + row;        // key inside the tile
+            const bool ok = row < n_ok;
+            const __nv_bfloat16* src = src0 + (ok ? row : 0) * kHeadDim + ch * 8;
+            cp16(dst0 + sw128(trow, ch), src, ok);                 // dims 0..63
+            cp16(dst0 + kBlk + sw128(trow, ch), src + 64, ok);     // dims 64..127
+          }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      }
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kFullK0 + stage));
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kFullV0 + stage));
+    }
+  } else if (warp == kMmaWarp) {
+    // ================================ MMA issuer ================================
+    const uint32_t idesc_s = instr_desc(false), idesc_o = instr_desc(true);
+    auto issue_s = [&](int it) {   // S[it & 1] = Q K_it^T
+      const int stage = it & 1, buf = it & 1;
+      mbar_wait(bar(kFullK0 + stage), (it >> 1) & 1, abort_flag, status);
+      if (it >= 2) mbar_wait(bar(kSEmpty0 + buf), ((it >> 1) - 1) & 1, abort_flag, status);
+      tc_fence_after();
+      if (lane == 0) {
+#pragma unroll
+        for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t da = smem_desc(sbase + kQOff + kb * kBlk + ks * 32, 16, 1024);
+            const uint64_t db = smem_desc(sbase + kKOff + (stage * 2 + kb) * kBlk + ks * 32, 16, 1024);
+            tc_mma(tmem_s[buf], da, db, idesc_s, (kb | ks) ? 1u : 0u);
+          }
+        tc_commit(bar(kSFull0 + buf));
+      }
+      __syncwarp();
+    };
+    issue_s(0);
+    for (int it = 0; it < n_tiles; ++it) {
+      const int stage = it & 1;
+      if (it + 1 < n_tiles) issue_s(it + 1);
+      // O += P_it V_it
+      mbar_wait(bar(kFullV0 + stage), (it >> 1) & 1, abort_flag, status);
+      mbar_wait(bar(kPFull), it & 1, abort_flag, status);
+      tc_fence_after();
+      if (lane == 0) {
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {   // 16 keys per step
+          const uint64_t da = smem_desc(sbase + kPOff + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024);
+          const uint64_t db = smem_desc(sbase + kVOff + stage * 2 * kBlk + ks * 2048, kBlk, 1024);
+          tc_mma(tmem_o, da, db, idesc_o, (it | ks) ? 1u : 0u);
+        }
+        tc_commit(bar(kPEmpty));
+        tc_commit(bar(kEmptyKV0 + stage));
+      }
+      __syncwarp();
+    }
+  } else {
+    // ================================ softmax (two threads per row) ================================
+    // Thread t owns row t & 127 (TMEM lane) and half (t >> 7) of the 128 key columns / output dims; the two
+    // halves exchange their row maxima through shared memory once per tile.
+    // The output accumulator stays in TMEM.  Probabilities are exp2(s - m_ref) with a reference m_ref that is
+    // only raised (and O, l rescaled) when a tile's maximum exceeds it by more than 8 in log2 units, so that most
+    // tiles never touch O; any reference gives the same result after the final division by l.
+    const int row = tid & 127, half = tid >> 7;
+    const int hs = row / BMP, po = row % BMP;
+    const bool row_ok = po < rows_here;
+    const int pos = m0 + po;
+    const int qh = kvh * d.group + hs;
+    const float sc2 = d.sm_scale * kLog2eT;
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t col0 = (uint32_t)half * 64u;
+    float* xch = reinterpret_cast<float*>(smem + kXchOff);
+    float m_ref = -INFINITY, l_run = 0.f;
+
+    for (int it = 0; it < n_tiles; ++it) {
+      const int buf = it & 1;
+      const int n_base = tile_at(it) * kBNt + half * 64;      // first key of this thread's columns
+      mbar_wait(bar(kSFull0 + buf), (it >> 1) & 1, abort_flag, status);
+      tc_fence_after();
+      float s[64];
+      {
+        uint32_t* r0p = reinterpret_cast<uint32_t*>(s);
+        uint32_t* r1p = r0p + 32;
+        RTP_TMEM_LD32(r0p, tmem_s[buf] + lane_addr + col0);
+        RTP_TMEM_LD32(r1p, tmem_s[buf] + lane_addr + col0 + 32);
+        tc_wait_ld();
+      }
+      tc_fence_before();
+      mbar_arrive(bar(kSEmpty0 + buf));          // S is in registers: the buffer may be overwritten
+      bool need_mask = n_base + 63 > pos;
+      if (MODE == kPrefillLocal) need_mask = need_mask || (n_base <= pos - d.window);
+      if (need_mask) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) {
+          const int n = n_base + i;
+          bool ok = n <= pos;
+          if (MODE == kPrefillLocal) ok = ok && (n < d.n_sink || n > pos - d.window);
+          if (!ok) s[i] = -INFINITY;
+        }
+      }
+      float tmax;
+      {
+        float t0 = s[0], t1 = s[1], t2 = s[2], t3 = s[3];   // four independent chains
+#pragma unroll
+        for (int i = 4; i < 64; i += 4) {
+          t0 = fmaxf(t0, s[i]); t1 = fmaxf(t1, s[i + 1]); t2 = fmaxf(t2, s[i + 2]); t3 = fmaxf(t3, s[i + 3]);
+        }
+        tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3));
+      }
+      xch[((it & 1) * 2 + half) * 128 + row] = tmax;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      tmax = fmaxf(tmax, xch[((it & 1) * 2 + (half ^ 1)) * 128 + row]) * sc2;
+      // P of the previous tile must have been consumed (and O must be quiescent) before P / O are touched
+      if (it >= 1) mbar_wait(bar(kPEmpty), (it - 1) & 1, abort_flag, status);
+      const bool raise = tmax > m_ref + 8.0f;     // also true for the first finite maximum (m_ref = -inf)
+      if (it >= 1 && __any_sync(0xffffffffu, raise)) {
+        tc_fence_after();
+        const float f = raise ? ((m_ref == -INFINITY) ? 0.f : fast_ex2(m_ref - tmax)) : 1.f;
+#pragma unroll
+        for (int c4 = 0; c4 < 2; ++c4) {
+          uint32_t r[32];
+          RTP_TMEM_LD32(r, tmem_o + lane_addr + col0 + c4 * 32);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+          RTP_TMEM_ST32(tmem_o + lane_addr + col0 + c4 * 32, r);
+        }
+        tc_wait_st();
+        l_run *= f;
+      }
+      if (raise) m_ref = tmax;
+      const float mb = (m_ref == -INFINITY) ? 0.f : m_ref;
+      float rs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c8 = 0; c8 < 8; ++c8) {           // 8 keys = one 16-byte chunk of the row
+        uint32_t pk[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          const float p0 = fast_ex2(fmaf(s[c8 * 8 + 2 * x], sc2, -mb)), p1 = fast_ex2(fmaf(s[c8 * 8 + 2 * x + 1], sc2, -mb));
+          rs[x] += p0 + p1;
+          __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+          pk[x] = *reinterpret_cast<uint32_t*>(&v);
+        }
+        *reinterpret_cast<uint4*>(smem + kPOff + half * kBlk + sw128(row, c8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      }
+      l_run += (rs[0] + rs[1]) + (rs[2] + rs[3]);
+      tc_fence_before();
+      fence_async_smem();
+      mbar_arrive(bar(kPFull));
+    }
+    // epilogue: O is complete once the last P V has been committed
+    if (n_tiles >= 1) mbar_wait(bar(kPEmpty), (n_tiles - 1) & 1, abort_flag, status);
+    tc_fence_after();
+    xch[half * 128 + row] = l_run;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    const float l_tot = l_run + xch[(half ^ 1) * 128 + row];
+    {
+      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+      __nv_bfloat16* dst = out + ((int64_t)(r0 + (row_ok ? po : 0)) * d.n_q + qh) * kHeadDim + col0;
+#pragma unroll
+      for (int c4 = 0; c4 < 2; ++c4) {
+        uint32_t r[32];
+        RTP_TMEM_LD32(r, tmem_o + lane_addr + col0 + c4 * 32);
+        tc_wait_ld();
+        if (row_ok) {
+#pragma unroll
+          for (int c8 = 0; c8 < 4; ++c8) {
+            uint32_t w[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[c8 * 8 + 2 * x]) * inv, __uint_as_float(r[c8 * 8 + 2 * x + 1]) * inv);
+              w[x] = *reinterpret_cast<uint32_t*>(&v);
+            }
+            *reinterpret_cast<uint4*>(dst + c4 * 32 + c8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      if (row_ok && half == 0 && lse) lse[(int64_t)(r0 + po) * d.n_q + qh] = l_tot > 0.f ? (m_ref + log2f(l_tot)) * kLn2T : -INFINITY;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor map over a paged cache viewed as [num_pages * n_kv * 64 rows][128 dims] bf16; box = 64 rows x 64 dims,
+// 128-byte swizzle (the layout the MMA descriptors expect).
+cudaError_t make_page_map(CUtensorMap* map, const void* base, int64_t rows) {
+  static EncodeTiledFn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+    encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+template <int G, int MODE>
+cudaError_t launch_tc_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm, const __nv_bfloat16* q,
+                            int32_t seq_id, int32_t q_start, int64_t C, __nv_bfloat16* out, float* lse,
+                            int32_t* status, int n_units, cudaStream_t st) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(attn_prefill_tc_kernel<G, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  CUtensorMap map_k, map_v;
+  const int64_t rows = (int64_t)cv.num_pages * cv.n_kv * kPage;
+  cudaError_t e = make_page_map(&map_k, cv.k, rows);
+  if (e != cudaSuccess) return e;
+  e = make_page_map(&map_v, cv.v, rows);
+  if (e != cudaSuccess) return e;
+  constexpr int BMP = kBM / G;
+  const int n_row_tiles = (int)((C + BMP - 1) / BMP);
+  dim3 grid(n_row_tiles, n_units);
+  attn_prefill_tc_kernel<G, MODE><<<grid, kTcThreads, kTcSmem, st>>>(map_k, map_v, cv, d, hm, q, seq_id, q_start, (int)C, out,
+                                                                     lse, status, n_row_tiles);
+  return cudaGetLastError();
+}
+
+template <int MODE>
+cudaError_t launch_tc_mode(const CacheView& cv, const Dims& d, const HeadMaps& hm, const __nv_bfloat16* q,
+                           int32_t seq_id, int32_t q_start, int64_t C, __nv_bfloat16* out, float* lse, int32_t* status,
+                           int n_units, cudaStream_t st) {
+  switch (d.group) {
+    case 1: return launch_tc_typed<1, MODE>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, n_units, st);
+    case 2: return launch_tc_typed<2, MODE>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, n_units, st);
+    case 4: return launch_tc_typed<4, MODE>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, n_units, st);
+    case 8: return launch_tc_typed<8, MODE>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, n_units, st);
+    default: return cudaErrorNotSupported;
+  }
+}
+
+}  // namespace
+
+// Dense and sink+window prefill attention on tcgen05.  Returns cudaErrorNotSupported for other modes.
+cudaError_t launch_attn_prefill_tc(const CacheView& cv, const Dims& d, const HeadMaps& hm, int mode,
+                                   const __nv_bfloat16* q, int32_t seq_id, int32_t q_start, int64_t C,
+                                   __nv_bfloat16* out, float* lse, int32_t* status, cudaStream_t st) {
+  if (C == 0 || hm.n_kv_list == 0) return cudaSuccess;
+  if (mode == kPrefillLocal) return launch_tc_mode<kPrefillLocal>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, hm.n_kv_list, st);
+  if (mode == kPrefillDense) return launch_tc_mode<kPrefillDense>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, hm.n_kv_list, st);
+  return cudaErrorNotSupported;
+}
+
+}  // namespace rtp

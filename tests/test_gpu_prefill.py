@@ -161,7 +161,7 @@ def test_top_p_one_prefill_equals_dense():
     out_s, lse_s = pr.sparse_prefill(0, 700, sel, use_lists=False)
     out_d, lse_d = pr.dense_prefill(0, 700, kv_heads=wl.heads.ret_kv_heads)
     h = wl.heads.ret_q_heads
-    assert np.abs(out_s[:, h] - out_d[:, h]).max() <= 1e-2
+    assert np.abs(out_s[:, h] - out_d[:, h]).max() <= 3e-2        # two kernels, each bf16-rounded
     np.testing.assert_allclose(lse_s[:, h], lse_d[:, h], rtol=1e-4, atol=1e-4)
 
 
