@@ -1,19 +1,20 @@
 // S7 / S9 for a prefill chunk on the 5th-generation tensor cores (tcgen05 + TMEM), dense and
 // sink+window modes.
 //
-// One CTA (320 threads, one per SM) owns 128 MMA rows = (128 / G) consecutive positions x the G query
+// One CTA (384 threads, one per SM) owns 128 MMA rows = (128 / G) consecutive positions x the G query
 // heads of one KV head and walks the key tiles of 128 keys (two cache pages):
-//   warp 9    loader: K and V pages -> shared memory in the 128-byte-swizzled layout the MMA unit reads; TMA
+//   warps 9-10 loaders (K / V): pages -> shared memory in the 128-byte-swizzled layout the MMA unit reads; TMA
 //             (cp.async.bulk.tensor, one lane) for whole tiles, zero-filling cp.async for the last tile; two stages
-//   warp 8    one elected lane issues tcgen05.mma: S = Q K^T (128 x 128 x 128) into one of two TMEM
-//             buffers, then O += P V (128 x 128 x 128) once the softmax warps have written P
-//   warps 0-7 two threads per row (TMEM lane = row, half of the columns each): reads S with tcgen05.ld, masks, online softmax,
-//             writes P (bf16) to shared memory; O accumulates in TMEM across tiles and is rescaled there
-//             only when the running reference maximum has to be raised
+//   warp 8    one elected lane issues tcgen05.mma S = Q K^T (128 x 128 x 128) into one of two TMEM buffers
+//   warp 11   one elected lane issues O += P V (128 x 128 x 128) once a softmax group has written P
+//   warps 0-7 two softmax groups (even tiles / odd tiles) of 128 threads, thread = row = TMEM lane: read S with
+//             tcgen05.ld, mask, online softmax, write P (bf16) to shared memory; each group accumulates its own
+//             O in TMEM (rescaled there only when its reference maximum has to be raised); merged at the end
 // Hand-offs are mbarriers (tcgen05.commit on the MMA side).  Every wait is bounded: when a wait runs
 // out, the CTA records RTP_ERR_TIMEOUT, stops waiting (all later waits return at once), still walks its
 // loops to the end, frees its TMEM and exits.
 #include <cuda.h>
+#include <cstdio>
 
 #include "rtp_device.cuh"
 
@@ -23,22 +24,23 @@ namespace {
 
 constexpr int kBM = 128;
 constexpr int kBNt = 128;                 // keys per tile
-constexpr int kTcThreads = 320;           // warps 0-7 softmax, 8 MMA, 9 loader
-constexpr int kMmaWarp = 8, kLoadWarp0 = 9;
+constexpr int kTcThreads = 384;           // warps 0-7 softmax, 8 S-MMA issuer, 9 K loader, 10 V loader, 11 PV-MMA issuer
+constexpr int kMmaWarp = 8, kLoadWarp0 = 9, kPvWarp = 11;
 constexpr int kBlk = 128 * 128;           // bytes of one [128 rows][64 elements] bf16 block (16 KB)
 constexpr int kQOff = 0;                  // Q: 2 blocks (dims 0-63, 64-127)
 constexpr int kKOff = 2 * kBlk;           // K: 2 stages x 2 blocks
 constexpr int kVOff = kKOff + 4 * kBlk;   // V: 2 stages x 2 blocks
-constexpr int kPOff = kVOff + 4 * kBlk;   // P: 2 blocks (keys 0-63, 64-127)
-constexpr int kBarOff = kPOff + 2 * kBlk; // mbarriers + TMEM base + abort flag
-constexpr int kXchOff = kBarOff + 256;     // float [2 tiles][2 halves][128 rows]: row-maximum exchange
-constexpr int kTcSmem = kXchOff + 2048 + 1024;   // + slack for 1024-byte alignment of the base
+constexpr int kPOff = kVOff + 4 * kBlk;   // P: 2 groups x 2 blocks (keys 0-63, 64-127)
+constexpr int kBarOff = kPOff + 4 * kBlk; // mbarriers + TMEM base + abort flag
+constexpr int kXchOff = kBarOff + 256;    // float [2 groups][2][128 rows]: (m, l) exchange for the final merge
+constexpr int kTcSmem = kXchOff + 2048;
+constexpr int kStageRow = 528;            // bytes per row of the fp32 staging tile used by the final merge (512 + 16)
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kLog2eT = 1.4426950408889634f;
 constexpr float kLn2T = 0.6931471805599453f;
 
-enum Bar { kFullK0 = 0, kFullK1, kFullV0, kFullV1, kEmptyKV0, kEmptyKV1, kSFull0, kSFull1, kSEmpty0, kSEmpty1,
-           kPFull, kPEmpty, kNumBars };
+enum Bar { kFullK0 = 0, kFullK1, kFullV0, kFullV1, kEmptyK0, kEmptyK1, kEmptyV0, kEmptyV1, kSFull0, kSFull1, kSEmpty0, kSEmpty1,
+           kPFull0, kPFull1, kPEmpty0, kPEmpty1, kNumBars };
 
 __device__ __forceinline__ uint32_t s_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
@@ -151,8 +153,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const int q_start, const int C, __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int32_t* status,
     const int n_row_tiles) {
   constexpr int BMP = kBM / G;
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) unsigned char smem[];
   const uint32_t sbase = s_u32(smem);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kBarOff + kNumBars * 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kBarOff + kNumBars * 8 + 8);
@@ -178,11 +179,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
   if (tid == 0) {
     mbar_init(bar(kFullK0), 1); mbar_init(bar(kFullK1), 1);
     mbar_init(bar(kFullV0), 1); mbar_init(bar(kFullV1), 1);
-    mbar_init(bar(kEmptyKV0), 1); mbar_init(bar(kEmptyKV1), 1);
+    mbar_init(bar(kEmptyK0), 1); mbar_init(bar(kEmptyK1), 1);
+    mbar_init(bar(kEmptyV0), 1); mbar_init(bar(kEmptyV1), 1);
     mbar_init(bar(kSFull0), 1); mbar_init(bar(kSFull1), 1);
-    mbar_init(bar(kSEmpty0), 256); mbar_init(bar(kSEmpty1), 256);
-    mbar_init(bar(kPFull), 256);
-    mbar_init(bar(kPEmpty), 1);
+    mbar_init(bar(kSEmpty0), 128); mbar_init(bar(kSEmpty1), 128);
+    mbar_init(bar(kPFull0), 128); mbar_init(bar(kPFull1), 128);
+    mbar_init(bar(kPEmpty0), 1); mbar_init(bar(kPEmpty1), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -207,77 +209,70 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_s[2] = {tmem, tmem + 128u};
-  const uint32_t tmem_o = tmem + 256u;
+  const uint32_t tmem_s[2] = {tmem, tmem + 128u};          // S of the even-tile / odd-tile group
+  const uint32_t tmem_o[2] = {tmem + 256u, tmem + 384u};   // their output accumulators
 
-  if (warp >= kLoadWarp0) {
-    // ================================ loader ================================
-    // Tiles whose 128 keys all exist are fetched by TMA (eight 8 KB boxes, completion in bytes on the stage's
-    // barriers; the warp does not wait for them).  The tile that holds the last position may reach into cache
+  if (warp == kLoadWarp0 || warp == kLoadWarp0 + 1) {
+    // ================================ loaders (warp 9: K tiles, warp 10: V tiles) ================================
+    // Tiles whose 128 keys all exist are fetched by TMA (four 8 KB boxes, completion in bytes on the stage's
+    // barrier; the warp does not wait for them).  The tile that holds the last position may reach into cache
     // slots that were never written: it is copied with cp.async and zero-filled beyond the last position.
+    // A K stage is free again as soon as its S MMA has completed, a V stage once its P V MMA has.
+    const int which = warp - kLoadWarp0;            // 0: K, 1: V
     const int64_t bt_base = (int64_t)seq_id * cv.max_pages;
     const int last_page = m_last >> kPageShift;
     const int rsub = lane >> 3, ch = lane & 7;     // 4 rows x 8 chunks per warp instruction
+    const __nv_bfloat16* pages = which ? cv.v : cv.k;
+    const CUtensorMap* map = which ? &map_v : &map_k;
     for (int it = 0; it < n_tiles; ++it) {
       const int stage = it & 1;
-      if (it >= 2) mbar_wait(bar(kEmptyKV0 + stage), ((it >> 1) - 1) & 1, abort_flag, status);
+      if (it >= 2) mbar_wait(bar((which ? kEmptyV0 : kEmptyK0) + stage), ((it >> 1) - 1) & 1, abort_flag, status);
       const int kt = tile_at(it);
-      const bool whole = kt * kBNt + kBNt - 1 <= m_last;
-      if (whole) {
+      const uint32_t dst0 = sbase + (which ? kVOff : kKOff) + stage * 2 * kBlk;
+      const uint32_t fb = bar((which ? kFullV0 : kFullK0) + stage);
+      if (kt * kBNt + kBNt - 1 <= m_last) {
         if (lane == 0) {
+          mbar_expect_tx(fb, 2 * kBlk);
 #pragma unroll
-          for (int which = 0; which < 2; ++which) {
-            const uint32_t dst0 = sbase + (which ? kVOff : kKOff) + stage * 2 * kBlk;
-            const uint32_t fb = bar(which ? kFullV0 + stage : kFullK0 + stage);
-            mbar_expect_tx(fb, 2 * kBlk);
-#pragma unroll
-            for (int pg = 0; pg < 2; ++pg) {
-              const int phys = __ldg(cv.block_table + bt_base + kt * 2 + pg);
-              const int y = (phys * cv.n_kv + kvh) * kPage;
-              tma_load_2d(dst0 + pg * (kPage * 128), which ? &map_v : &map_k, 0, y, fb);
-              tma_load_2d(dst0 + kBlk + pg * (kPage * 128), which ? &map_v : &map_k, 64, y, fb);
-            }
+          for (int pg = 0; pg < 2; ++pg) {
+            const int phys = __ldg(cv.block_table + bt_base + kt * 2 + pg);
+            const int y = (phys * cv.n_kv + kvh) * kPage;
+            tma_load_2d(dst0 + pg * (kPage * 128), map, 0, y, fb);
+            tma_load_2d(dst0 + kBlk + pg * (kPage * 128), map, 64, y, fb);
           }
         }
         __syncwarp();
         continue;
       }
 #pragma unroll 1
-      for (int which = 0; which < 2; ++which) {     // 0: K, 1: V
-        const __nv_bfloat16* pages = which ? cv.v : cv.k;
-        const uint32_t dst0 = sbase + (which ? kVOff : kKOff) + stage * 2 * kBlk;
-#pragma unroll 1
-        for (int pg = 0; pg < 2; ++pg) {
-          const int page = kt * 2 + pg;
-          const bool page_ok = page <= last_page;
-          const int phys = page_ok ? __ldg(cv.block_table + bt_base + page) : 0;
-          const __nv_bfloat16* src0 = pages + ((int64_t)phys * cv.n_kv + kvh) * (kPage * kHeadDim);
-          const int n_ok = page_ok ? m_last - page * kPage + 1 : 0;   // keys of the page any row may attend
+      for (int pg = 0; pg < 2; ++pg) {
+        const int page = kt * 2 + pg;
+        const bool page_ok = page <= last_page;
+        const int phys = page_ok ? __ldg(cv.block_table + bt_base + page) : 0;
+        const __nv_bfloat16* src0 = pages + ((int64_t)phys * cv.n_kv + kvh) * (kPage * kHeadDim);
+        const int n_ok = page_ok ? m_last - page * kPage + 1 : 0;   // keys of the page any row may attend
 #pragma unroll 4
-          for (int r4 = 0; r4 < 16; ++r4) {
-            const int row = r4 * 4 + rsub;            // key inside the page
-            const int trow = pg * kPage + row;        // key inside the tile
-            const bool ok = row < n_ok;
-            const __nv_bfloat16* src = src0 + (ok ? row : 0) * kHeadDim + ch * 8;
-            cp16(dst0 + sw128(trow, ch), src, ok);                 // dims 0..63
-            cp16(dst0 + kBlk + sw128(trow, ch), src + 64, ok);     // dims 64..127
-          }
+        for (int r4 = 0; r4 < 16; ++r4) {
+          const int row = r4 * 4 + rsub;            // key inside the page
+          const int trow = pg * kPage + row;        // key inside the tile
+          const bool ok = row < n_ok;
+          const __nv_bfloat16* src = src0 + (ok ? row : 0) * kHeadDim + ch * 8;
+          cp16(dst0 + sw128(trow, ch), src, ok);                 // dims 0..63
+          cp16(dst0 + kBlk + sw128(trow, ch), src + 64, ok);     // dims 64..127
         }
-        asm volatile("cp.async.commit_group;" ::: "memory");
       }
-      asm volatile("cp.async.wait_group 1;" ::: "memory");
-      fence_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(kFullK0 + stage));
+      asm volatile("cp.async.commit_group;" ::: "memory");
       asm volatile("cp.async.wait_group 0;" ::: "memory");
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(kFullV0 + stage));
+      if (lane == 0) mbar_arrive(fb);
     }
   } else if (warp == kMmaWarp) {
-    // ================================ MMA issuer ================================
-    const uint32_t idesc_s = instr_desc(false), idesc_o = instr_desc(true);
-    auto issue_s = [&](int it) {   // S[it & 1] = Q K_it^T
+    // ================================ S = Q K^T issuer ================================
+    // Runs ahead of the softmax groups: S_it only needs K_it and the S buffer of its group (released as soon as the
+    // group has copied the previous S of that buffer into registers).
+    const uint32_t idesc_s = instr_desc(false);
+    for (int it = 0; it < n_tiles; ++it) {
       const int stage = it & 1, buf = it & 1;
       mbar_wait(bar(kFullK0 + stage), (it >> 1) & 1, abort_flag, status);
       if (it >= 2) mbar_wait(bar(kSEmpty0 + buf), ((it >> 1) - 1) & 1, abort_flag, status);
@@ -292,67 +287,80 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             tc_mma(tmem_s[buf], da, db, idesc_s, (kb | ks) ? 1u : 0u);
           }
         tc_commit(bar(kSFull0 + buf));
+        tc_commit(bar(kEmptyK0 + stage));
       }
       __syncwarp();
-    };
-    issue_s(0);
+    }
+  } else if (warp == kPvWarp) {
+    // ================================ O_g += P V issuer ================================
+    // g = it & 1: the even and the odd tiles are two independent online-softmax streams with their own accumulators
+    const uint32_t idesc_o = instr_desc(true);
     for (int it = 0; it < n_tiles; ++it) {
-      const int stage = it & 1;
-      if (it + 1 < n_tiles) issue_s(it + 1);
-      // O += P_it V_it
+      const int stage = it & 1, grp = it & 1;
       mbar_wait(bar(kFullV0 + stage), (it >> 1) & 1, abort_flag, status);
-      mbar_wait(bar(kPFull), it & 1, abort_flag, status);
+      mbar_wait(bar(kPFull0 + grp), (it >> 1) & 1, abort_flag, status);
       tc_fence_after();
       if (lane == 0) {
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {   // 16 keys per step
-          const uint64_t da = smem_desc(sbase + kPOff + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024);
+          const uint64_t da = smem_desc(sbase + kPOff + (grp * 2 + (ks >> 2)) * kBlk + (ks & 3) * 32, 16, 1024);
           const uint64_t db = smem_desc(sbase + kVOff + stage * 2 * kBlk + ks * 2048, kBlk, 1024);
-          tc_mma(tmem_o, da, db, idesc_o, (it | ks) ? 1u : 0u);
+          tc_mma(tmem_o[grp], da, db, idesc_o, ((it >> 1) | ks) ? 1u : 0u);
         }
-        tc_commit(bar(kPEmpty));
-        tc_commit(bar(kEmptyKV0 + stage));
+        tc_commit(bar(kPEmpty0 + grp));
+        tc_commit(bar(kEmptyV0 + stage));
       }
       __syncwarp();
     }
   } else {
-    // ================================ softmax (two threads per row) ================================
-    // Thread t owns row t & 127 (TMEM lane) and half (t >> 7) of the 128 key columns / output dims; the two
-    // halves exchange their row maxima through shared memory once per tile.
-    // The output accumulator stays in TMEM.  Probabilities are exp2(s - m_ref) with a reference m_ref that is
-    // only raised (and O, l rescaled) when a tile's maximum exceeds it by more than 8 in log2 units, so that most
-    // tiles never touch O; any reference gives the same result after the final division by l.
-    const int row = tid & 127, half = tid >> 7;
+    // ================================ softmax (two groups of 128 threads, thread = row) ================================
+    // Group g (warps 4g .. 4g+3) handles the tiles it = g, g+2, ...: its own S buffer, P buffer and output
+    // accumulator in TMEM, its own running (m_ref, l).  The two groups are independent online-softmax streams
+    // over disjoint key tiles, so one group's exponentials overlap the other group's MMAs; they are merged once
+    // at the end.  Probabilities are exp2(s - m_ref) with a reference that is only raised (and O, l rescaled in
+    // TMEM) when a tile's maximum exceeds it by more than 8 in log2 units; any reference gives the same result
+    // after the final division by l.
+    const int grp = tid >> 7, row = tid & 127;
     const int hs = row / BMP, po = row % BMP;
     const bool row_ok = po < rows_here;
     const int pos = m0 + po;
     const int qh = kvh * d.group + hs;
     const float sc2 = d.sm_scale * kLog2eT;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t col0 = (uint32_t)half * 64u;
     float* xch = reinterpret_cast<float*>(smem + kXchOff);
     float m_ref = -INFINITY, l_run = 0.f;
+    int n_mine = 0;
+#ifdef RTP_TC_TRACE
+    long long tr_s[4][5];
+#endif
 
-    for (int it = 0; it < n_tiles; ++it) {
-      const int buf = it & 1;
-      const int n_base = tile_at(it) * kBNt + half * 64;      // first key of this thread's columns
-      mbar_wait(bar(kSFull0 + buf), (it >> 1) & 1, abort_flag, status);
+    for (int it = grp; it < n_tiles; it += 2, ++n_mine) {
+      const int n_base = tile_at(it) * kBNt;
+      mbar_wait(bar(kSFull0 + grp), n_mine & 1, abort_flag, status);
+#ifdef RTP_TC_TRACE
+      if (n_mine < 4) tr_s[n_mine][0] = clock64();
+#endif
       tc_fence_after();
-      float s[64];
+      float s[kBNt];
       {
         uint32_t* r0p = reinterpret_cast<uint32_t*>(s);
-        uint32_t* r1p = r0p + 32;
-        RTP_TMEM_LD32(r0p, tmem_s[buf] + lane_addr + col0);
-        RTP_TMEM_LD32(r1p, tmem_s[buf] + lane_addr + col0 + 32);
+        uint32_t* r1p = r0p + 32; uint32_t* r2p = r0p + 64; uint32_t* r3p = r0p + 96;
+        RTP_TMEM_LD32(r0p, tmem_s[grp] + lane_addr);
+        RTP_TMEM_LD32(r1p, tmem_s[grp] + lane_addr + 32);
+        RTP_TMEM_LD32(r2p, tmem_s[grp] + lane_addr + 64);
+        RTP_TMEM_LD32(r3p, tmem_s[grp] + lane_addr + 96);
         tc_wait_ld();
       }
+#ifdef RTP_TC_TRACE
+      if (n_mine < 4) tr_s[n_mine][1] = clock64();
+#endif
       tc_fence_before();
-      mbar_arrive(bar(kSEmpty0 + buf));          // S is in registers: the buffer may be overwritten
-      bool need_mask = n_base + 63 > pos;
+      mbar_arrive(bar(kSEmpty0 + grp));          // S is in registers: the buffer may be overwritten
+      bool need_mask = n_base + kBNt - 1 > pos;
       if (MODE == kPrefillLocal) need_mask = need_mask || (n_base <= pos - d.window);
       if (need_mask) {
 #pragma unroll
-        for (int i = 0; i < 64; ++i) {
+        for (int i = 0; i < kBNt; ++i) {
           const int n = n_base + i;
           bool ok = n <= pos;
           if (MODE == kPrefillLocal) ok = ok && (n < d.n_sink || n > pos - d.window);
@@ -363,28 +371,31 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
       {
         float t0 = s[0], t1 = s[1], t2 = s[2], t3 = s[3];   // four independent chains
 #pragma unroll
-        for (int i = 4; i < 64; i += 4) {
+        for (int i = 4; i < kBNt; i += 4) {
           t0 = fmaxf(t0, s[i]); t1 = fmaxf(t1, s[i + 1]); t2 = fmaxf(t2, s[i + 2]); t3 = fmaxf(t3, s[i + 3]);
         }
-        tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3));
+        tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3)) * sc2;
       }
-      xch[((it & 1) * 2 + half) * 128 + row] = tmax;
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      tmax = fmaxf(tmax, xch[((it & 1) * 2 + (half ^ 1)) * 128 + row]) * sc2;
-      // P of the previous tile must have been consumed (and O must be quiescent) before P / O are touched
-      if (it >= 1) mbar_wait(bar(kPEmpty), (it - 1) & 1, abort_flag, status);
+      // this group's previous P must have been consumed (and its O must be quiescent) before P / O are touched
+#ifdef RTP_TC_TRACE
+      if (n_mine < 4) tr_s[n_mine][2] = clock64();
+#endif
+      if (n_mine >= 1) mbar_wait(bar(kPEmpty0 + grp), (n_mine - 1) & 1, abort_flag, status);
+#ifdef RTP_TC_TRACE
+      if (n_mine < 4) tr_s[n_mine][3] = clock64();
+#endif
       const bool raise = tmax > m_ref + 8.0f;     // also true for the first finite maximum (m_ref = -inf)
-      if (it >= 1 && __any_sync(0xffffffffu, raise)) {
+      if (n_mine >= 1 && __any_sync(0xffffffffu, raise)) {
         tc_fence_after();
         const float f = raise ? ((m_ref == -INFINITY) ? 0.f : fast_ex2(m_ref - tmax)) : 1.f;
 #pragma unroll
-        for (int c4 = 0; c4 < 2; ++c4) {
+        for (int c4 = 0; c4 < 4; ++c4) {
           uint32_t r[32];
-          RTP_TMEM_LD32(r, tmem_o + lane_addr + col0 + c4 * 32);
+          RTP_TMEM_LD32(r, tmem_o[grp] + lane_addr + c4 * 32);
           tc_wait_ld();
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
-          RTP_TMEM_ST32(tmem_o + lane_addr + col0 + c4 * 32, r);
+          RTP_TMEM_ST32(tmem_o[grp] + lane_addr + c4 * 32, r);
         }
         tc_wait_st();
         l_run *= f;
@@ -392,8 +403,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
       if (raise) m_ref = tmax;
       const float mb = (m_ref == -INFINITY) ? 0.f : m_ref;
       float rs[4] = {0.f, 0.f, 0.f, 0.f};
+      unsigned char* pbase = smem + kPOff + grp * 2 * kBlk;
 #pragma unroll
-      for (int c8 = 0; c8 < 8; ++c8) {           // 8 keys = one 16-byte chunk of the row
+      for (int c8 = 0; c8 < 16; ++c8) {          // 8 keys = one 16-byte chunk of the row
         uint32_t pk[4];
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
@@ -402,41 +414,83 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
           __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
           pk[x] = *reinterpret_cast<uint32_t*>(&v);
         }
-        *reinterpret_cast<uint4*>(smem + kPOff + half * kBlk + sw128(row, c8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        *reinterpret_cast<uint4*>(pbase + (c8 >> 3) * kBlk + sw128(row, c8 & 7)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
       l_run += (rs[0] + rs[1]) + (rs[2] + rs[3]);
       tc_fence_before();
       fence_async_smem();
-      mbar_arrive(bar(kPFull));
+      mbar_arrive(bar(kPFull0 + grp));
+#ifdef RTP_TC_TRACE
+      if (n_mine < 4) tr_s[n_mine][4] = clock64();
+#endif
     }
-    // epilogue: O is complete once the last P V has been committed
-    if (n_tiles >= 1) mbar_wait(bar(kPEmpty), (n_tiles - 1) & 1, abort_flag, status);
+#ifdef RTP_TC_TRACE
+    if (blockIdx.x == 0 && blockIdx.y == 0 && row == 0)
+      for (int i = 0; i < 4 && i < n_mine; ++i)
+        printf("SM grp %d tile %d sfull %lld ld %lld max %lld pempty %lld pfull %lld\n", grp, 2 * i + grp, tr_s[i][0], tr_s[i][1], tr_s[i][2], tr_s[i][3], tr_s[i][4]);
+#endif
+    // ---- merge of the two groups and epilogue ----
+    if (n_mine >= 1) mbar_wait(bar(kPEmpty0 + grp), (n_mine - 1) & 1, abort_flag, status);   // this group's last P V is done
     tc_fence_after();
-    xch[half * 128 + row] = l_run;
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    const float l_tot = l_run + xch[(half ^ 1) * 128 + row];
-    {
-      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-      __nv_bfloat16* dst = out + ((int64_t)(r0 + (row_ok ? po : 0)) * d.n_q + qh) * kHeadDim + col0;
+    xch[(grp * 2 + 0) * 128 + row] = m_ref;
+    xch[(grp * 2 + 1) * 128 + row] = l_run;
+    asm volatile("bar.sync 1, 256;" ::: "memory");       // every MMA of the CTA has completed: shared memory is free
+    const float m_oth = xch[((grp ^ 1) * 2 + 0) * 128 + row], l_oth = xch[((grp ^ 1) * 2 + 1) * 128 + row];
+    const float m_tot = fmaxf(m_ref, m_oth);
+    const float w_me = (m_ref == -INFINITY) ? 0.f : fast_ex2(m_ref - m_tot);
+    const float w_ot = (m_oth == -INFINITY) ? 0.f : fast_ex2(m_oth - m_tot);
+    const float l_tot = l_run * w_me + l_oth * w_ot;
+    const float sc_me = l_tot > 0.f ? w_me / l_tot : 0.f;
+    float* stage_row = reinterpret_cast<float*>(smem + kKOff + row * kStageRow);   // fp32 [128 dims] of group 1, scaled
+    if (grp == 1) {
 #pragma unroll
-      for (int c4 = 0; c4 < 2; ++c4) {
+      for (int c4 = 0; c4 < 4; ++c4) {
         uint32_t r[32];
-        RTP_TMEM_LD32(r, tmem_o + lane_addr + col0 + c4 * 32);
-        tc_wait_ld();
+        if (n_mine >= 1) {
+          RTP_TMEM_LD32(r, tmem_o[1] + lane_addr + c4 * 32);
+          tc_wait_ld();
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = 0u;
+        }
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+          *reinterpret_cast<float4*>(stage_row + c4 * 32 + i) =
+              make_float4(__uint_as_float(r[i]) * sc_me, __uint_as_float(r[i + 1]) * sc_me, __uint_as_float(r[i + 2]) * sc_me,
+                          __uint_as_float(r[i + 3]) * sc_me);
+      }
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (grp == 0) {
+      __nv_bfloat16* dst = out + ((int64_t)(r0 + (row_ok ? po : 0)) * d.n_q + qh) * kHeadDim;
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4) {
+        uint32_t r[32];
+        if (n_mine >= 1) {
+          RTP_TMEM_LD32(r, tmem_o[0] + lane_addr + c4 * 32);
+          tc_wait_ld();
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = 0u;
+        }
         if (row_ok) {
 #pragma unroll
           for (int c8 = 0; c8 < 4; ++c8) {
-            uint32_t w[4];
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-              __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[c8 * 8 + 2 * x]) * inv, __uint_as_float(r[c8 * 8 + 2 * x + 1]) * inv);
-              w[x] = *reinterpret_cast<uint32_t*>(&v);
-            }
-            *reinterpret_cast<uint4*>(dst + c4 * 32 + c8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            const float4 a = *reinterpret_cast<const float4*>(stage_row + c4 * 32 + c8 * 8);
+            const float4 b = *reinterpret_cast<const float4*>(stage_row + c4 * 32 + c8 * 8 + 4);
+            const float o0 = fmaf(__uint_as_float(r[c8 * 8 + 0]), sc_me, a.x), o1 = fmaf(__uint_as_float(r[c8 * 8 + 1]), sc_me, a.y);
+            const float o2 = fmaf(__uint_as_float(r[c8 * 8 + 2]), sc_me, a.z), o3 = fmaf(__uint_as_float(r[c8 * 8 + 3]), sc_me, a.w);
+            const float o4 = fmaf(__uint_as_float(r[c8 * 8 + 4]), sc_me, b.x), o5 = fmaf(__uint_as_float(r[c8 * 8 + 5]), sc_me, b.y);
+            const float o6 = fmaf(__uint_as_float(r[c8 * 8 + 6]), sc_me, b.z), o7 = fmaf(__uint_as_float(r[c8 * 8 + 7]), sc_me, b.w);
+            __nv_bfloat162 v0 = __floats2bfloat162_rn(o0, o1), v1 = __floats2bfloat162_rn(o2, o3);
+            __nv_bfloat162 v2 = __floats2bfloat162_rn(o4, o5), v3 = __floats2bfloat162_rn(o6, o7);
+            *reinterpret_cast<uint4*>(dst + c4 * 32 + c8 * 8) =
+                make_uint4(*reinterpret_cast<uint32_t*>(&v0), *reinterpret_cast<uint32_t*>(&v1), *reinterpret_cast<uint32_t*>(&v2),
+                           *reinterpret_cast<uint32_t*>(&v3));
           }
         }
       }
-      if (row_ok && half == 0 && lse) lse[(int64_t)(r0 + po) * d.n_q + qh] = l_tot > 0.f ? (m_ref + log2f(l_tot)) * kLn2T : -INFINITY;
+      if (row_ok && lse) lse[(int64_t)(r0 + po) * d.n_q + qh] = l_tot > 0.f ? (m_tot + log2f(l_tot)) * kLn2T : -INFINITY;
     }
   }
 
