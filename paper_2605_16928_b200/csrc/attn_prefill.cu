@@ -387,24 +387,24 @@ cudaError_t launch_attn_prefill(const CacheView& cv, const Dims& d, const HeadMa
                                 const __nv_bfloat16* q, const __nv_bfloat16* qt, int32_t seq_id, int32_t q_start,
                                 int64_t C, const float* sel_thresh, const int32_t* sel_tie_last,
                                 __nv_bfloat16* out, float* lse, int32_t* status, int sm_count, cudaStream_t st) {
-  (void)status;
   (void)sm_count;
   if (C == 0) return cudaSuccess;
+  // every mode runs on tcgen05 / TMEM / TMA; RTP_PREFILL_TC=0 selects the warp-MMA kernel of this file
+  static const bool use_tc = [] { const char* e = getenv("RTP_PREFILL_TC"); return !(e && e[0] == '0'); }();
   if (mode == kPrefillSparse) {
     // one CTA column per index head; every query head of its KV head must be a retrieval head on it
     for (int j = 0; j < d.n_ih; ++j)
       if (hm.ih_nheads[j] != d.group) return cudaErrorNotSupported;
     for (int i = 0; i < d.n_ret; ++i)
       if (hm.ret_q_head[i] != hm.ih_kv[hm.q2ih[i]] * d.group + hm.slot_in_ih[i]) return cudaErrorNotSupported;
+    if (use_tc)
+      return launch_attn_prefill_tc(cv, d, hm, mode, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, st);
     return launch_mode<kPrefillSparse>(cv, d, hm, q, qt, seq_id, q_start, C, sel_thresh, sel_tie_last, out, lse,
                                        d.n_ih, st);
   }
   if (hm.n_kv_list == 0) return cudaSuccess;
-  {
-    // dense and sink+window modes run on tcgen05 / TMEM / TMA; RTP_PREFILL_TC=0 selects the warp-MMA kernel below
-    static const bool use_tc = [] { const char* e = getenv("RTP_PREFILL_TC"); return !(e && e[0] == '0'); }();
-    if (use_tc) return launch_attn_prefill_tc(cv, d, hm, mode, q, seq_id, q_start, C, out, lse, status, st);
-  }
+  if (use_tc)
+    return launch_attn_prefill_tc(cv, d, hm, mode, q, nullptr, nullptr, nullptr, seq_id, q_start, C, out, lse, status, st);
   if (mode == kPrefillLocal)
     return launch_mode<kPrefillLocal>(cv, d, hm, q, qt, seq_id, q_start, C, sel_thresh, sel_tie_last, out, lse,
                                       hm.n_kv_list, st);

@@ -1,5 +1,5 @@
-// S7 / S9 for a prefill chunk on the 5th-generation tensor cores (tcgen05 + TMEM), dense and
-// sink+window modes.
+// S6 / S7 / S9 for a prefill chunk on the 5th-generation tensor cores (tcgen05 + TMEM): dense, sink+window
+// and sparse (Eq. 5) modes.
 //
 // One CTA (384 threads, one per SM) owns 128 MMA rows = (128 / G) consecutive positions x the G query
 // heads of one KV head and walks the key tiles of 128 keys (two cache pages):
@@ -9,7 +9,11 @@
 //   warp 11   one elected lane issues O += P V (128 x 128 x 128) once a softmax group has written P
 //   warps 0-7 two softmax groups (even tiles / odd tiles) of 128 threads, thread = row = TMEM lane: read S with
 //             tcgen05.ld, mask, online softmax, write P (bf16) to shared memory; each group accumulates its own
-//             O in TMEM (rescaled there only when its reference maximum has to be raised); merged at the end
+//             O in TMEM (rescaled there only when its reference maximum has to be raised); merged at the end.
+//             Sparse mode: while the S MMA of its tile is in flight, each softmax warp re-evaluates the membership
+//             of its 32 rows x 128 keys in S_h(m) from the 16-dim indexer scores (warp MMAs on index keys read
+//             straight from the cache, the same arithmetic as the selection kernels) against the rows'
+//             (threshold, tie position) pairs, and masks S with the resulting bits.
 // Hand-offs are mbarriers (tcgen05.commit on the MMA side).  Every wait is bounded: when a wait runs
 // out, the CTA records RTP_ERR_TIMEOUT, stops waiting (all later waits return at once), still walks its
 // loops to the end, frees its TMEM and exits.
@@ -25,7 +29,7 @@ namespace {
 constexpr int kBM = 128;
 constexpr int kBNt = 128;                 // keys per tile
 constexpr int kTcThreads = 384;           // warps 0-7 softmax, 8 S-MMA issuer, 9 K loader, 10 V loader, 11 PV-MMA issuer
-constexpr int kMmaWarp = 8, kLoadWarp0 = 9, kPvWarp = 11;
+constexpr int kMmaWarp = 8, kLoadWarp0 = 9;   // warp 11 issues the P V MMAs
 constexpr int kBlk = 128 * 128;           // bytes of one [128 rows][64 elements] bf16 block (16 KB)
 constexpr int kQOff = 0;                  // Q: 2 blocks (dims 0-63, 64-127)
 constexpr int kKOff = 2 * kBlk;           // K: 2 stages x 2 blocks
@@ -154,9 +158,10 @@ __device__ __forceinline__ uint32_t sw128(int r, int c) { return (uint32_t)(r * 
 template <int G, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-    const CacheView cv, const Dims d, const HeadMaps hm, const __nv_bfloat16* __restrict__ q, const int seq_id,
-    const int q_start, const int C, __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int32_t* status,
-    const int n_row_tiles) {
+    const CacheView cv, const Dims d, const HeadMaps hm, const __nv_bfloat16* __restrict__ q,
+    const __nv_bfloat16* __restrict__ qt, const float* __restrict__ sel_thresh, const int32_t* __restrict__ sel_tie_last,
+    const int seq_id, const int q_start, const int C, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
+    int32_t* status, const int n_row_tiles) {
   constexpr int BMP = kBM / G;
   extern __shared__ __align__(1024) unsigned char smem[];
   const uint32_t sbase = s_u32(smem);
@@ -166,7 +171,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile = n_row_tiles - 1 - blockIdx.x;
-  const int kvh = hm.kv_list[blockIdx.y];
+  const int kvh = (MODE == kPrefillSparse) ? hm.ih_kv[blockIdx.y] : hm.kv_list[blockIdx.y];
   const int r0 = tile * BMP, m0 = q_start + r0;
   const int rows_here = min(BMP, C - r0);
   const int m_last = m0 + rows_here - 1;
@@ -217,6 +222,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
   const uint32_t tmem_s[2] = {tmem, tmem + 128u};          // S of the even-tile / odd-tile group
   const uint32_t tmem_o[2] = {tmem + 256u, tmem + 384u};   // their output accumulators
 
+  // Register budget per role: the loader / issuer warpgroup hands registers back, the two softmax warpgroups (128
+  // scores per thread live at once) take them: 256 x 232 + 128 x 40 = 384 x 168.
+  if (warp >= 8) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
   if (warp == kLoadWarp0 || warp == kLoadWarp0 + 1) {
     // ================================ loaders (warp 9: K tiles, warp 10: V tiles) ================================
     // Tiles whose 128 keys all exist are fetched by TMA (four 8 KB boxes, completion in bytes on the stage's
@@ -296,7 +305,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
       }
       __syncwarp();
     }
-  } else if (warp == kPvWarp) {
+  } else {
     // ================================ O_g += P V issuer ================================
     // g = it & 1: the even and the odd tiles are two independent online-softmax streams with their own accumulators
     const uint32_t idesc_o = instr_desc(true);
@@ -317,7 +326,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
       }
       __syncwarp();
     }
+  }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
     // ================================ softmax (two groups of 128 threads, thread = row) ================================
     // Group g (warps 4g .. 4g+3) handles the tiles it = g, g+2, ...: its own S buffer, P buffer and output
     // accumulator in TMEM, its own running (m_ref, l).  The two groups are independent online-softmax streams
@@ -336,11 +347,159 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     float m_ref = -INFINITY, l_run = 0.f;
     int n_mine = 0;
 #ifdef RTP_TC_TRACE
-    long long tr_s[4][5];
+    long long tr_s[4][6];
 #endif
+    // ---- sparse mode: membership rule of the rows ----
+    // Membership is tested on the unscaled MMA output: raw > up means "score above the row's threshold",
+    // raw >= lo "at or above it" (they differ only for keys tied with the threshold score); upn is the next
+    // float above up, so that raw > up <=> raw >= upn.  The per-row values live in shared memory (the region the
+    // final merge reuses) and are re-read for every tile, like the projected-query fragments (from global
+    // memory): nothing of the rule stays in registers across the softmax of a tile.
+    const int ih = (MODE == kPrefillSparse) ? blockIdx.y : 0;
+    const int gq = lane >> 2, cq = lane & 3;
+    float* thr_lo = xch;                                      // [128 rows]
+    float* thr_upn = xch + 256;
+    int* thr_tie = reinterpret_cast<int*>(xch + 384);
+    int warp_pos_min = 0;
+    const __nv_bfloat16* qt_lane = qt;                        // projected query of row (warp's first row + g), this lane's dims
+    int qt_step[4] = {0, 0, 0, 0};                            // element offset of rows k*8 + g from it (-1: row absent)
+    if (MODE == kPrefillSparse) {
+      const float kInfT = __int_as_float(0x7f800000);
+      if (grp == 0) {
+        float lo_me = kInfT, up_me = kInfT;
+        int tie_me = -1;
+        if (row_ok) {
+          const int64_t rr = (int64_t)(r0 + po) * d.n_ret + hm.ih_heads[ih][hs];
+          const uint32_t tk = okey(sel_thresh[rr]);
+          float dummy;
+          raw_preimage(d.score_scale, tk, tk, lo_me, dummy);
+          raw_preimage(d.score_scale, 0u, tk, dummy, up_me);
+          tie_me = sel_tie_last[rr];
+        }
+        thr_lo[row] = lo_me;
+        thr_upn[row] = (up_me < kInfT) ? okey_to_float(okey(up_me) + 1u) : kInfT;
+        thr_tie[row] = tie_me;
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      warp_pos_min = 0x7fffffff;
+      const int row_w = (warp & 3) * 32;
+      const int64_t base_rr = (int64_t)(r0 + (row_w + gq) % BMP) * d.n_ret + hm.ih_heads[ih][(row_w + gq) / BMP];
+      qt_lane = qt + base_rr * kIndexDim + qfrag_dim_offset(lane);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int rowk = row_w + k * 8 + gq;
+        const int hsk = rowk / BMP, pok = rowk % BMP;
+        if (pok < rows_here) {
+          warp_pos_min = min(warp_pos_min, m0 + pok);
+          qt_step[k] = (int)(((int64_t)(r0 + pok) * d.n_ret + hm.ih_heads[ih][hsk] - base_rr) * kIndexDim);
+        } else {
+          qt_step[k] = -1;
+        }
+      }
+      warp_pos_min = -__reduce_max_sync(0xffffffffu, -warp_pos_min);
+    }
+    const int64_t bt_base_s = (int64_t)seq_id * cv.max_pages;
+    const int last_page_s = m_last >> kPageShift;
+    // Index keys of a tile: lane (g, c) reads its 8 bytes of key 8 nt + g for every 8-key group nt.
+    uint32_t iqa[2][4] = {{0u, 0u, 0u, 0u}, {0u, 0u, 0u, 0u}};   // A fragments of rows 0-15 / 16-31 of the warp
+    if (MODE == kPrefillSparse) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint2 v = make_uint2(0u, 0u);
+        if (qt_step[k] >= 0) v = __ldg(reinterpret_cast<const uint2*>(qt_lane + qt_step[k]));
+        iqa[k >> 1][k & 1] = v.x;        // a0 (row g) / a1 (row g + 8)
+        iqa[k >> 1][2 + (k & 1)] = v.y;  // a2 / a3
+      }
+    }
 
     for (int it = grp; it < n_tiles; it += 2, ++n_mine) {
       const int n_base = tile_at(it) * kBNt;
+#ifdef RTP_TC_TRACE
+      if (n_mine < 4) tr_s[n_mine][5] = clock64();
+#endif
+      uint32_t my[4] = {0u, 0u, 0u, 0u};   // this thread's row: bit 31 - (2 nt + e) of my[c] set <=> key 8 nt + 2 c + e is NOT a member
+      if (MODE == kPrefillSparse) {
+        // Tiles that are causal for every row of the warp and do not contain a row's tie position need one
+        // comparison per score: raw >= lo before the tie position, raw > up (= raw >= upn) after it.  The sign
+        // bits of (raw - threshold) are shifted into one word per row: the j-th appended element (j = 2 nt + e)
+        // ends at bit 31 - j, set = NOT a member.
+        uint32_t mw[4] = {0u, 0u, 0u, 0u};   // rows k*8 + g, columns 2 c, 2 c + 1 of every 8-key group
+        float thr[4];
+        bool fast = n_base + kBNt - 1 <= warp_pos_min;
+        const int row_w = (warp & 3) * 32;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int rowk = row_w + k * 8 + gq;
+          const int tie = thr_tie[rowk];
+          const bool before = n_base + kBNt - 1 <= tie, after = tie < n_base;
+          thr[k] = before ? thr_lo[rowk] : thr_upn[rowk];
+          fast = fast && (before || after);
+        }
+        fast = __all_sync(0xffffffffu, fast);
+        const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+        uint2 kb[16];
+#pragma unroll
+        for (int pg = 0; pg < 2; ++pg) {
+          const int phys = __ldg(cv.block_table + bt_base_s + min(n_base / kPage + pg, last_page_s));
+          const __nv_bfloat16* ik =
+              cv.ikey + ((int64_t)phys * cv.n_ih + ih) * (kPage * kIndexDim) + gq * kIndexDim + qfrag_dim_offset(lane);
+#pragma unroll
+          for (int n8 = 0; n8 < 8; ++n8) kb[pg * 8 + n8] = __ldg(reinterpret_cast<const uint2*>(ik + n8 * 8 * kIndexDim));
+        }
+        if (fast) {
+#pragma unroll
+          for (int nt = 0; nt < 16; ++nt) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+              float s4[4];
+              mma_bf16_16816(s4, iqa[t][0], iqa[t][1], iqa[t][2], iqa[t][3], kb[nt].x, kb[nt].y, zero);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int k = 2 * t + (e >> 1);
+                mw[k] = __funnelshift_l(__float_as_uint(s4[e] - thr[k]), mw[k], 1);
+              }
+            }
+          }
+        } else {
+          // general rule (diagonal tiles, tiles that hold a row's tie position): key n of the tile belongs to the
+          // row's set iff n <= position and raw >= (n <= tie position ? lo : upn)
+          float lo_k[4], upn_k[4];
+          int tie_rel[4], pos_rel[4];   // relative to the lane's first column of the tile
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int rowk = row_w + k * 8 + gq;
+            lo_k[k] = thr_lo[rowk];
+            upn_k[k] = thr_upn[rowk];
+            tie_rel[k] = thr_tie[rowk] - n_base - 2 * cq;
+            pos_rel[k] = m0 + rowk % BMP - n_base - 2 * cq;
+          }
+#pragma unroll
+          for (int nt = 0; nt < 16; ++nt) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+              float s4[4];
+              mma_bf16_16816(s4, iqa[t][0], iqa[t][1], iqa[t][2], iqa[t][3], kb[nt].x, kb[nt].y, zero);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int k = 2 * t + (e >> 1);
+                const int j = nt * 8 + (e & 1);
+                const float th = (j <= tie_rel[k]) ? lo_k[k] : upn_k[k];
+                const bool in = (j <= pos_rel[k]) && (s4[e] >= th);
+                mw[k] = (mw[k] << 1) | (in ? 0u : 1u);
+              }
+            }
+          }
+        }
+        // lane (g, c) -> thread = row: row k*8 + g collects its four words from the lanes of quad g
+        const int kk = lane >> 3;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int src = 4 * (lane & 7) + c;
+          const uint32_t v0 = __shfl_sync(0xffffffffu, mw[0], src), v1 = __shfl_sync(0xffffffffu, mw[1], src);
+          const uint32_t v2 = __shfl_sync(0xffffffffu, mw[2], src), v3 = __shfl_sync(0xffffffffu, mw[3], src);
+          my[c] = kk == 0 ? v0 : kk == 1 ? v1 : kk == 2 ? v2 : v3;
+        }
+      }
       mbar_wait(bar(kSFull0 + grp), n_mine & 1, abort_flag, status);
 #ifdef RTP_TC_TRACE
       if (n_mine < 4) tr_s[n_mine][0] = clock64();
@@ -359,8 +518,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 #endif
       tc_fence_before();
       mbar_arrive(bar(kSEmpty0 + grp));          // S is in registers: the buffer may be overwritten
+      if (MODE == kPrefillSparse) {
+#pragma unroll
+        for (int i = 0; i < kBNt; ++i)
+          if ((my[(i & 7) >> 1] >> (31 - (2 * (i >> 3) + (i & 1)))) & 1u) s[i] = -INFINITY;
+      }
       bool need_mask = n_base + kBNt - 1 > pos;
       if (MODE == kPrefillLocal) need_mask = need_mask || (n_base <= pos - d.window);
+      if (MODE == kPrefillSparse) need_mask = false;
       if (need_mask) {
 #pragma unroll
         for (int i = 0; i < kBNt; ++i) {
@@ -430,11 +595,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 #ifdef RTP_TC_TRACE
     if (blockIdx.x == 0 && blockIdx.y == 0 && row == 0)
       for (int i = 0; i < 4 && i < n_mine; ++i)
-        printf("SM grp %d tile %d sfull %lld ld %lld max %lld pempty %lld pfull %lld\n", grp, 2 * i + grp, tr_s[i][0], tr_s[i][1], tr_s[i][2], tr_s[i][3], tr_s[i][4]);
+        printf("SM grp %d tile %d top %lld sfull %lld ld %lld max %lld pempty %lld pfull %lld\n", grp, 2 * i + grp, tr_s[i][5] - tr_s[0][5], tr_s[i][0] - tr_s[0][5], tr_s[i][1] - tr_s[0][5], tr_s[i][2] - tr_s[0][5], tr_s[i][3] - tr_s[0][5], tr_s[i][4] - tr_s[0][5]);
 #endif
     // ---- merge of the two groups and epilogue ----
     if (n_mine >= 1) mbar_wait(bar(kPEmpty0 + grp), (n_mine - 1) & 1, abort_flag, status);   // this group's last P V is done
     tc_fence_after();
+    if (MODE == kPrefillSparse) asm volatile("bar.sync 1, 256;" ::: "memory");   // the rows' rule (same memory) is no longer read
     xch[(grp * 2 + 0) * 128 + row] = m_ref;
     xch[(grp * 2 + 1) * 128 + row] = l_run;
     asm volatile("bar.sync 1, 256;" ::: "memory");       // every MMA of the CTA has completed: shared memory is free
@@ -533,6 +699,7 @@ cudaError_t make_page_map(CUtensorMap* map, const void* base, int64_t rows) {
 
 template <int G, int MODE>
 cudaError_t launch_tc_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm, const __nv_bfloat16* q,
+                            const __nv_bfloat16* qt, const float* sel_thresh, const int32_t* sel_tie_last,
                             int32_t seq_id, int32_t q_start, int64_t C, __nv_bfloat16* out, float* lse,
                             int32_t* status, int n_units, cudaStream_t st) {
   static bool attr_done = false;
@@ -550,33 +717,45 @@ cudaError_t launch_tc_typed(const CacheView& cv, const Dims& d, const HeadMaps& 
   constexpr int BMP = kBM / G;
   const int n_row_tiles = (int)((C + BMP - 1) / BMP);
   dim3 grid(n_row_tiles, n_units);
-  attn_prefill_tc_kernel<G, MODE><<<grid, kTcThreads, kTcSmem, st>>>(map_k, map_v, cv, d, hm, q, seq_id, q_start, (int)C, out,
-                                                                     lse, status, n_row_tiles);
+  attn_prefill_tc_kernel<G, MODE><<<grid, kTcThreads, kTcSmem, st>>>(map_k, map_v, cv, d, hm, q, qt, sel_thresh, sel_tie_last,
+                                                                     seq_id, q_start, (int)C, out, lse, status, n_row_tiles);
   return cudaGetLastError();
 }
 
 template <int MODE>
 cudaError_t launch_tc_mode(const CacheView& cv, const Dims& d, const HeadMaps& hm, const __nv_bfloat16* q,
+                           const __nv_bfloat16* qt, const float* sel_thresh, const int32_t* sel_tie_last,
                            int32_t seq_id, int32_t q_start, int64_t C, __nv_bfloat16* out, float* lse, int32_t* status,
                            int n_units, cudaStream_t st) {
   switch (d.group) {
-    case 1: return launch_tc_typed<1, MODE>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, n_units, st);
-    case 2: return launch_tc_typed<2, MODE>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, n_units, st);
-    case 4: return launch_tc_typed<4, MODE>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, n_units, st);
-    case 8: return launch_tc_typed<8, MODE>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, n_units, st);
+    case 1: return launch_tc_typed<1, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st);
+    case 2: return launch_tc_typed<2, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st);
+    case 4: return launch_tc_typed<4, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st);
+    case 8: return launch_tc_typed<8, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st);
     default: return cudaErrorNotSupported;
   }
 }
 
 }  // namespace
 
-// Dense and sink+window prefill attention on tcgen05.  Returns cudaErrorNotSupported for other modes.
+// Prefill attention on tcgen05: dense and sink+window over the KV heads of hm.kv_list, sparse (one CTA column per
+// index head; the caller has checked that every index head serves the whole GQA group of its KV head).
 cudaError_t launch_attn_prefill_tc(const CacheView& cv, const Dims& d, const HeadMaps& hm, int mode,
-                                   const __nv_bfloat16* q, int32_t seq_id, int32_t q_start, int64_t C,
+                                   const __nv_bfloat16* q, const __nv_bfloat16* qt, const float* sel_thresh,
+                                   const int32_t* sel_tie_last, int32_t seq_id, int32_t q_start, int64_t C,
                                    __nv_bfloat16* out, float* lse, int32_t* status, cudaStream_t st) {
-  if (C == 0 || hm.n_kv_list == 0) return cudaSuccess;
-  if (mode == kPrefillLocal) return launch_tc_mode<kPrefillLocal>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, hm.n_kv_list, st);
-  if (mode == kPrefillDense) return launch_tc_mode<kPrefillDense>(cv, d, hm, q, seq_id, q_start, C, out, lse, status, hm.n_kv_list, st);
+  if (C == 0) return cudaSuccess;
+  if (mode == kPrefillSparse)
+    return d.n_ih == 0 ? cudaSuccess
+                       : launch_tc_mode<kPrefillSparse>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out,
+                                                        lse, status, d.n_ih, st);
+  if (hm.n_kv_list == 0) return cudaSuccess;
+  if (mode == kPrefillLocal)
+    return launch_tc_mode<kPrefillLocal>(cv, d, hm, q, nullptr, nullptr, nullptr, seq_id, q_start, C, out, lse, status,
+                                         hm.n_kv_list, st);
+  if (mode == kPrefillDense)
+    return launch_tc_mode<kPrefillDense>(cv, d, hm, q, nullptr, nullptr, nullptr, seq_id, q_start, C, out, lse, status,
+                                         hm.n_kv_list, st);
   return cudaErrorNotSupported;
 }
 

@@ -127,7 +127,8 @@ cudaError_t launch_attn_prefill(const CacheView& cv, const Dims& d, const HeadMa
                                 __nv_bfloat16* out, float* lse, int32_t* status, int sm_count, cudaStream_t st);
 
 cudaError_t launch_attn_prefill_tc(const CacheView& cv, const Dims& d, const HeadMaps& hm, int mode,
-                                   const __nv_bfloat16* q, int32_t seq_id, int32_t q_start, int64_t C,
+                                   const __nv_bfloat16* q, const __nv_bfloat16* qt, const float* sel_thresh,
+                                   const int32_t* sel_tie_last, int32_t seq_id, int32_t q_start, int64_t C,
                                    __nv_bfloat16* out, float* lse, int32_t* status, cudaStream_t st);
 
 }  // namespace rtp
