@@ -751,10 +751,6 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
   }
 }
 
-static int dbg_passes() {
-  const char* e = getenv("RTP_DEBUG_MAX_PASSES");
-  return e ? atoi(e) : kMaxPasses;
-}
 
 template <int G>
 cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
@@ -772,7 +768,7 @@ cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm,
   dim3 grid(n_row_tiles, d.n_ih);
   select_chunk_kernel<G><<<grid, kCThreads, kSmemC, st>>>(cv, d, hm, qt, rows.seq_id, rows.q_start, (int)rows.R,
                                                           sel_idx, sel_stride, sel_count, sel_mass, sel_thresh,
-                                                          sel_tie_last, status, n_row_tiles, dbg_passes());
+                                                          sel_tie_last, status, n_row_tiles, kMaxPasses);
   return cudaGetLastError();
 }
 
