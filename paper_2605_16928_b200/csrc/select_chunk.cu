@@ -7,12 +7,15 @@
 // page against its 16 rows with eight m16n8k16 MMAs.  All selection state lives in shared memory, so
 // the whole selection of the chunk is one kernel without inter-CTA communication:
 //   max       row maximum M                                                   (1 op per score)
-//   level 1   64-bin histogram of softmax mass over d = M - s in steps of 1/2 (d >= 31.5 pooled), in
+//   level 1   64-bin histogram of softmax mass over d = M - s in steps of 1/2 (d >= 31.25 pooled), in
 //             fixed point with native 32-bit shared-memory adds; gives Z and the bucket in which the
 //             cumulative mass reaches p * Z; the bucket becomes an exact interval of ordered score keys
 //             (bisection) and of unscaled MMA outputs (so later passes compare raw values only)
 //   key level 64-bin mass histogram of the ordered key inside the interval, 6 key bits per pass, until the
-//             chosen bin provably holds at most 64 keys
+//             chosen bin provably holds at most 64 keys.  From here on only a small share of the scores falls
+//             into a row's interval: a warp appends those hits (row, position, raw score) to a queue in shared
+//             memory and works them off 32 at a time, one hit per lane, so that the per-hit arithmetic and the
+//             shared-memory adds are issued once per 32 hits instead of once per MMA
 //   collect   the keys of the final bucket go to a 64-entry list, the keys above it are counted; the warp
 //             ranks the list exactly by (score descending, position ascending) and cuts it
 //   tie       only when more than 64 equal scores straddle the cut: position of the last tie taken
@@ -35,13 +38,15 @@ constexpr int kStageBytesC = kStageKeys * kIndexDim * 2;            // 8 KB
 constexpr int kBins = 64;                                           // bins per level
 constexpr float kL1Scale = 2.0f;                                    // level-1 bins per unit of d = M - s
 constexpr int kCandCapC = 64;                                       // candidates sorted exactly per row
-constexpr int kRowBytes = kBins * 8;                                // 512 B per row: 64 x {hi, lo} or 64 x {key, idx}
+constexpr int kRowBytes = kBins * 8 + 8;                            // per row: 64 x {sum, carries} or 64 x {key, idx}; +8 staggers the banks
 constexpr int kMaxPasses = 14;
 constexpr float kLog2eC = 1.4426950408889634f;
-// A key adds floor(e_rel * 2^20) to its bin, split into two 32-bit words (hi = >> 10, lo = & 1023) so that native
-// 32-bit shared-memory adds never overflow for up to 2^20 keys.  e_rel = mass relative to the bin's (level 1) or
-// the bucket's (key levels) upper end, in (e^-0.5, 1]: every key adds at least kMinHi to the hi word.
-constexpr uint32_t kMinHi = 620;                                    // floor(e^-0.5 * 1024) - 1
+// A key adds q = round(e_rel * 2^20) to its bin with one native 32-bit shared-memory add; the returned old value
+// tells whether the sum wrapped, and then (rarely) a second add counts the carry in the next word.  e_rel = mass
+// relative to the bin's (level 1) or the bucket's (key levels) upper end, in (e^-0.5, 1]: every key adds at
+// least kMinQ, which bounds the number of keys of a bin by its sum.
+constexpr float kMinQ = 634880.0f;                                  // (floor(e^-0.5 * 1024) - 1) * 1024
+constexpr int kQueueCap = 160;                                      // per-warp queue of bucket hits (entries of 8 bytes)
 
 enum Phase { kPhMax = 0, kPhL1 = 1, kPhKey = 2, kPhCollect = 3, kPhTie = 4, kPhDone = 5 };
 
@@ -65,7 +70,8 @@ struct RowState {      // one per (row, head), in shared memory
 };
 
 constexpr int kHistBytes = kCRows * kRowBytes;                      // 64 KB
-constexpr int kSmemC = kHistBytes + 2 * kStageBytesC + kCRows * (int)sizeof(RowState);
+constexpr int kQueueBytes = kCWarps * kQueueCap * 8;               // 10 KB
+constexpr int kSmemC = kHistBytes + 2 * kStageBytesC + kQueueBytes + kCRows * (int)sizeof(RowState);
 
 __device__ __forceinline__ void cp_async16c(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -74,19 +80,31 @@ __device__ __forceinline__ uint32_t smem_u32c(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
-// Level-1 bin of a score: the same arithmetic in the histogram pass and in the bisection below.
+// Level-1 bin of a score: the integer nearest to 2 (M - s), clamped to [0, 63]; bin b holds M - s in
+// [b/2 - 1/4, b/2 + 1/4] (the last bin pools everything below).  Adding 1.5 * 2^23 leaves that integer in the low
+// mantissa bits, so no float <-> int conversion instruction is needed; the same arithmetic serves the histogram
+// pass and the bisection that turns a bin into a key interval.
+constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
+__device__ __forceinline__ int l1_bin_f(float M, float s, float& bin_f) {
+  const float u = fminf(fmaxf((M - s) * kL1Scale, 0.0f), (float)(kBins - 1));
+  const float t = u + kMagic;
+  bin_f = t - kMagic;
+  return __float_as_int(t) & (kBins - 1);
+}
 __device__ __forceinline__ int l1_bin(float M, float s) {
-  return max(0, min(kBins - 1, (int)((M - s) * kL1Scale)));
+  float f;
+  return l1_bin_f(M, s, f);
 }
 
-// Adds floor(2^x) (x <= 20) to a split accumulator.
+// Adds round(2^x) (x <= 20) to an accumulator {sum mod 2^32, carries}.
 __device__ __forceinline__ void add_mass(uint32_t* acc, float x) {
-  const uint32_t q = min(__float2uint_rz(fast_ex2(x)), 1u << 20);
-  atomicAdd(acc, q >> 10);
-  atomicAdd(acc + 1, q & 1023u);
+  // nearest integer to 2^x through the mantissa of (2^x + 2^23): no conversion instruction
+  const uint32_t q = min(__float_as_uint(fast_ex2(x) + 8388608.0f) - 0x4b000000u, 1u << 20);
+  const uint32_t old = atomicAdd(acc, q);
+  if (old + q < old) atomicAdd(acc + 1, 1u);
 }
-__device__ __forceinline__ float acc_mass(uint32_t hi, uint32_t lo) {   // in units of 2^-20
-  return (float)hi * 1024.0f + (float)lo;
+__device__ __forceinline__ float acc_mass(uint32_t sum, uint32_t carries) {   // in units of 2^-20
+  return (float)carries * 4294967296.0f + (float)sum;
 }
 
 // Per-lane view of its two rows for one pass (registers).
@@ -146,10 +164,11 @@ __device__ __forceinline__ void page_l1(const unsigned char* pg, const QFrag& iq
       const bool lo = e < 2;
       if (MASK && n0 + (e & 1) > (lo ? L.pos_a : L.pos_b)) continue;
       const float s = finish_score(s4[e], scale);
-      const float dd = (lo ? L.M_a : L.M_b) - s;
-      const int bin = max(0, min(kBins - 1, (int)(dd * kL1Scale)));   // (rows that are already done have no M)
-      // mass relative to the bin's upper end: exp(-(dd - bin/2)), scaled by 2^20
-      add_mass((lo ? hist_a : hist_b) + 2 * bin, fmaf((float)bin, 0.5f * kLog2eC, fmaf(dd, -kLog2eC, 20.0f)));
+      const float M = lo ? L.M_a : L.M_b;
+      float bin_f;
+      const int bin = l1_bin_f(M, s, bin_f);   // (rows that are already done have no M: they land in bin 0)
+      // mass relative to the bin's upper end: exp(-((M - s) - (bin/2 - 1/4))), scaled by 2^20
+      add_mass((lo ? hist_a : hist_b) + 2 * bin, fmaf(bin_f, 0.5f * kLog2eC, fmaf(M - s, -kLog2eC, 20.0f - 0.25f * kLog2eC)));
     }
   }
 }
@@ -234,6 +253,84 @@ __device__ __forceinline__ void page_late(const unsigned char* pg, const QFrag& 
   }
 }
 
+// Works off the warp's queue of bucket hits: entry = {position | local row << 27, raw score bits}.
+__device__ __noinline__ void drain_hits(uint32_t* wq, int& qcnt, int lane, int wrow, RowState* rs, uint32_t* hist,
+                                           float scale) {
+  constexpr int kRowWords = kRowBytes / 4;
+  __syncwarp();
+  for (int base = 0; base < qcnt; base += 32) {
+    const int i = base + lane;
+    if (i < qcnt) {
+      const uint32_t w0 = wq[2 * i];
+      const float raw = __uint_as_float(wq[2 * i + 1]);
+      const int r = wrow + (int)(w0 >> 27);
+      RowState* S = rs + r;
+      const float s = finish_score(raw, scale);
+      const uint32_t key = okey(s);
+      uint32_t* h = hist + r * kRowWords;
+      if (S->phase == kPhCollect) {
+        const int slot = atomicAdd(&S->cand_cnt, 1);
+        if (slot < kCandCapC) {
+          h[2 * slot] = key;
+          h[2 * slot + 1] = w0 & 0x7ffffffu;
+        }
+      } else {
+        const uint32_t t = key - S->base_key;
+        add_mass(h + 2 * (t >> S->shift), fmaf(s - S->ref_s, kLog2eC, 20.0f));
+      }
+    }
+  }
+  __syncwarp();
+  qcnt = 0;
+}
+
+// Key levels and candidate collection without ties: hits go to the warp's queue.
+template <bool MASK, bool COUNT>
+__device__ __forceinline__ void page_hits(const unsigned char* pg, const QFrag& iq, int lane, int n_page,
+                                          const LaneRows& L, int& cnt_a, int& cnt_b, uint32_t* wq, int& qcnt,
+                                          int wrow, RowState* rs, uint32_t* hist, float scale) {
+  const int g = lane >> 2, c = lane & 3;
+  const int boff = 2 * qfrag_dim_offset(lane);
+  const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll
+  for (int nt = 0; nt < 8; ++nt) {
+    const uint2 b = *reinterpret_cast<const uint2*>(pg + (nt * 8 + g) * (kIndexDim * 2) + boff);
+    const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+    float s4[4];
+    mma_bf16_16816(s4, iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
+    const int n0 = n_page + nt * 8 + 2 * c;
+    if (MASK) {
+      const float nan = __int_as_float(0x7fc00000);   // fails every test below
+      if (n0 > L.pos_a) s4[0] = nan;
+      if (n0 + 1 > L.pos_a) s4[1] = nan;
+      if (n0 > L.pos_b) s4[2] = nan;
+      if (n0 + 1 > L.pos_b) s4[3] = nan;
+    }
+    if (COUNT) {   // keys above the bucket of a row that is collecting
+      cnt_a += (s4[0] > L.cut_a) + (s4[1] > L.cut_a);
+      cnt_b += (s4[2] > L.cut_b) + (s4[3] > L.cut_b);
+    }
+    const bool h0 = s4[0] >= L.lo_a && s4[0] <= L.hi_a, h1 = s4[1] >= L.lo_a && s4[1] <= L.hi_a;
+    const bool h2 = s4[2] >= L.lo_b && s4[2] <= L.hi_b, h3 = s4[3] >= L.lo_b && s4[3] <= L.hi_b;
+    if (__any_sync(0xffffffffu, h0 || h1 || h2 || h3)) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool hit = e == 0 ? h0 : e == 1 ? h1 : e == 2 ? h2 : h3;
+        const uint32_t m = __ballot_sync(0xffffffffu, hit);
+        if (m) {
+          if (hit) {
+            const int pos = qcnt + __popc(m & lt);
+            wq[2 * pos] = (uint32_t)(n0 + (e & 1)) | ((uint32_t)(g + (e >> 1) * 8) << 27);
+            wq[2 * pos + 1] = __float_as_uint(s4[e]);
+          }
+          qcnt += __popc(m);
+        }
+      }
+      if (qcnt >= 32) drain_hits(wq, qcnt, lane, wrow, rs, hist, scale);   // at most 31 + 128 entries queued
+    }
+  }
+}
+
 template <int G>
 __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
     const CacheView cv, const Dims d, const HeadMaps hm, const __nv_bfloat16* __restrict__ qt,
@@ -244,7 +341,8 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
   extern __shared__ __align__(128) unsigned char smem[];
   uint32_t* hist = reinterpret_cast<uint32_t*>(smem);                      // [128 rows][128 words]
   unsigned char* stage_s = smem + kHistBytes;
-  RowState* rs = reinterpret_cast<RowState*>(smem + kHistBytes + 2 * kStageBytesC);
+  uint32_t* queue = reinterpret_cast<uint32_t*>(smem + kHistBytes + 2 * kStageBytesC);
+  RowState* rs = reinterpret_cast<RowState*>(smem + kHistBytes + 2 * kStageBytesC + kQueueBytes);
   __shared__ int s_pending;
   constexpr int kRowWords = kRowBytes / 4;
 
@@ -372,6 +470,8 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
     int cnt_a = 0, cnt_b = 0;
     int run_a = 0, run_b = 0;
     int tl_a = -1, tl_b = -1;
+    uint32_t* wq = queue + warp * (kQueueCap * 2);
+    int qcnt = 0;
 
     load_stage(0, 0);
     asm volatile("cp.async.commit_group;" ::: "memory");
@@ -397,20 +497,23 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
             else page_l1<true>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b);
           } else {
 #define RTP_LATE(M_, T_, C_) page_late<M_, T_, C_>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b, ccnt_a, ccnt_b, cnt_a, cnt_b, need_a, need_b, run_a, run_b, tl_a, tl_b)
+#define RTP_HITS(M_, C_) page_hits<M_, C_>(pgp, iq, lane, n_page, LR, cnt_a, cnt_b, wq, qcnt, wrow, rs, hist, scale)
             if (pass_tie) {
               if (interior) RTP_LATE(false, true, true); else RTP_LATE(true, true, true);
             } else if (pass_count) {
-              if (interior) RTP_LATE(false, false, true); else RTP_LATE(true, false, true);
+              if (interior) RTP_HITS(false, true); else RTP_HITS(true, true);
             } else {
-              if (interior) RTP_LATE(false, false, false); else RTP_LATE(true, false, false);
+              if (interior) RTP_HITS(false, false); else RTP_HITS(true, false);
             }
 #undef RTP_LATE
+#undef RTP_HITS
           }
         }
       }
       __syncthreads();
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (qcnt > 0) drain_hits(wq, qcnt, lane, wrow, rs, hist, scale);
 
     // ---- end of pass: combine the quad's partial results ----
     mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
@@ -451,16 +554,17 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
         //   level 1: bin 0 is the top -> lane l takes bins 2l, 2l+1;  key levels: bin 63 is the top -> 63-2l, 62-2l
         const bool l1 = ph == kPhL1;
         const int b0 = l1 ? 2 * lane : 63 - 2 * lane, b1 = l1 ? 2 * lane + 1 : 62 - 2 * lane;
-        const uint32_t hi0 = h[2 * b0], lo0 = h[2 * b0 + 1], hi1 = h[2 * b1], lo1 = h[2 * b1 + 1];
+        const uint32_t sum0 = h[2 * b0], car0 = h[2 * b0 + 1], sum1 = h[2 * b1], car1 = h[2 * b1 + 1];
+        const float q0 = acc_mass(sum0, car0), q1 = acc_mass(sum1, car1);
         // masses relative to M
         float m0f, m1f;
         if (l1) {
-          m0f = acc_mass(hi0, lo0) * fast_ex2(-0.5f * kLog2eC * (float)b0 - 20.0f);
-          m1f = acc_mass(hi1, lo1) * fast_ex2(-0.5f * kLog2eC * (float)b1 - 20.0f);
+          m0f = q0 * fast_ex2(-kLog2eC * (0.5f * (float)b0 - 0.25f) - 20.0f);
+          m1f = q1 * fast_ex2(-kLog2eC * (0.5f * (float)b1 - 0.25f) - 20.0f);
         } else {
           const float sc = R.e_ref * 9.5367431640625e-07f;   // 2^-20
-          m0f = acc_mass(hi0, lo0) * sc;
-          m1f = acc_mass(hi1, lo1) * sc;
+          m0f = q0 * sc;
+          m1f = q1 * sc;
         }
         float incm = m0f + m1f;
 #pragma unroll
@@ -472,7 +576,7 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
         const float Z = l1 ? total : R.Z;
         const float target = l1 ? d.top_p * Z * (1.0f + kMassMargin) : R.target;
         const float run = (l1 ? 0.f : R.mass_above) + incm - (m0f + m1f);
-        const bool pop0 = (hi0 | lo0) != 0u, pop1 = (hi1 | lo1) != 0u;
+        const bool pop0 = (sum0 | car0) != 0u, pop1 = (sum1 | car1) != 0u;
         // order index of a bin = position from the top (0 .. 63)
         int found = 64, last = -1;
         if (pop0) {
@@ -497,9 +601,9 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
         } else if ((best >> 1) == lane) {
           const bool first = (best & 1) == 0;
           const float f_above = first ? run : run + m0f;
-          const uint32_t f_hi = first ? hi0 : hi1;
+          const float f_q = first ? q0 : q1;
           const int bin = first ? b0 : b1;
-          const bool few = f_hi / kMinHi < (uint32_t)kCandCapC;   // at most (f_hi / kMinHi) keys in the bin
+          const bool few = f_q < 0.999f * kMinQ * (float)kCandCapC;   // fewer than kCandCapC keys in the bin
           S->mass_above = f_above;
           if (l1) {
             S->Z = Z;
@@ -515,7 +619,7 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
               // Exact interval [klo, khi] of ordered keys whose level-1 bin is `bin`: l1_bin is monotone in the
               // key, so both ends are found by bisection between two keys that lie safely outside the bucket.
               const float M = R.M;
-              const float hi_s = M - (float)bin / kL1Scale, lo_s = M - (float)(bin + 1) / kL1Scale;
+              const float hi_s = M - ((float)bin - 0.5f) / kL1Scale, lo_s = M - ((float)bin + 0.5f) / kL1Scale;
               const float pad = 1e-5f * fmaxf(1.0f, fmaxf(fabsf(hi_s), fabsf(lo_s))) + 1e-3f;
               const uint32_t lo = okey(finish_score(lo_s - pad, 1.0f));
               const uint32_t hi = okey(finish_score(fminf(hi_s + pad, M), 1.0f));
@@ -538,7 +642,7 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
               float rlo, rhi;
               raw_preimage(scale, klo, khi, rlo, rhi);
               S->ref_s = hi_s;
-              S->e_ref = fast_ex2(-0.5f * kLog2eC * (float)bin);
+              S->e_ref = fast_ex2(-kLog2eC * (0.5f * (float)bin - 0.25f));
               S->base_key = klo;
               S->span = span;
               S->shift = max(0, bits - 6);
