@@ -130,6 +130,37 @@ __device__ __forceinline__ void raw_preimage(float scale, uint32_t key_lo, uint3
   raw_hi = okey_to_float(a);
 }
 
+// Warp-cooperative search on the ordered keys a <= k <= b for the smallest k with pred(k), pred monotone (false ..
+// true).  Returns b + 1 (as a 64-bit value) when pred(b) is false.  Every lane probes one point per step, so a 32-bit
+// range needs seven steps.  All 32 lanes must call it with the same arguments.
+template <class Pred>
+__device__ __forceinline__ unsigned long long warp_search_first(uint32_t a, uint32_t b, int lane, Pred pred) {
+  if (!pred(b)) return (unsigned long long)b + 1ull;
+  while (a < b) {   // the answer lies in [a, b]
+    const unsigned long long w = (unsigned long long)(b - a);
+    const uint32_t p = a + (uint32_t)((w * (unsigned long long)(lane + 1)) / 33ull);   // in [a, b)
+    const uint32_t m = __ballot_sync(0xffffffffu, pred(p));
+    const int f = m ? __ffs(m) - 1 : 32;                                                // first lane whose probe holds
+    const uint32_t p_f = __shfl_sync(0xffffffffu, p, f & 31), p_before = __shfl_sync(0xffffffffu, p, (f + 31) & 31);
+    if (f < 32) b = p_f;
+    if (f > 0) a = p_before + 1u;
+  }
+  return a;
+}
+
+// raw_preimage() with the work spread over a warp (same result).
+__device__ __forceinline__ void raw_preimage_warp(float scale, uint32_t key_lo, uint32_t key_hi, int lane, float& raw_lo,
+                                                  float& raw_hi) {
+  const uint32_t kmin = okey(-3.4028234e38f), kmax = okey(3.4028234e38f);
+  const unsigned long long lo =
+      warp_search_first(kmin, kmax, lane, [&](uint32_t k) { return okey(finish_score(okey_to_float(k), scale)) >= key_lo; });
+  const unsigned long long above =
+      warp_search_first(kmin, kmax, lane, [&](uint32_t k) { return okey(finish_score(okey_to_float(k), scale)) > key_hi; });
+  // lo > kmax: no float reaches key_lo; above == kmin: every float maps above key_hi: the interval is empty either way
+  raw_lo = lo > kmax ? __int_as_float(0x7f800000) : okey_to_float((uint32_t)lo);
+  raw_hi = above == kmin ? -__int_as_float(0x7f800000) : okey_to_float((uint32_t)(above - 1ull));
+}
+
 // Address of the 2 KB index-key slice of (logical page, index head) of a sequence.
 __device__ __forceinline__ const __nv_bfloat16* ikey_page_ptr(const CacheView& cv, int seq, int page,
                                                                int ih) {

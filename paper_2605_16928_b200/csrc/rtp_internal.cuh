@@ -15,7 +15,6 @@ constexpr int kPage = RTP_PAGE_SIZE;       // 64
 constexpr int kPageShift = 6;
 
 // Selection (decode-style) constants.
-constexpr int kSelBins = 2048;             // bins per radix level (11 + 11 + 10 bits of the ordered key)
 constexpr int kCandCap = 4096;             // boundary candidates resolved exactly per (row, head)
 constexpr float kMassMargin = 1e-5f;       // relative slack added to p*Z against fp32 summation error
 
@@ -59,18 +58,21 @@ struct Rows {
 
 // Per (row, retrieval head) selection state kept in the workspace between passes.
 struct SelState {
-  uint32_t max_key;      // ordered key of the row maximum (atomicMax during level 1)
+  uint32_t max_key;      // ordered key of the row maximum (atomicMax during the first pass)
   uint32_t lo_key;       // current bucket [lo_key, hi_key] of ordered keys that holds the threshold
   uint32_t hi_key;
-  int32_t level;         // radix levels completed
+  uint32_t span;         // hi_key - lo_key + 1
+  int32_t shift;         // key levels: bin = (key - lo_key) >> shift, in [0, 64)
   int32_t mode;          // 0 = refining, 1 = collect candidates, 2 = select all, 3 = exact ties (scan)
   float M;               // row maximum
   float Z;               // sum exp(s - M)
   float target;          // mass to reach, relative to M (p * Z * (1 + margin))
   float mass_above;      // mass of keys above the bucket
-  int32_t cnt_above;     // number of keys above the bucket
-  int32_t bucket_cnt;
-  float bucket_mass;
+  float raw_lo, raw_hi;  // the bucket as an interval of unscaled MMA outputs
+  float ref_s;           // key levels: masses are accumulated relative to exp(ref_s - M)
+  float e_ref;           // exp(ref_s - M)
+  int32_t cnt_above;     // number of keys above the bucket (counted by the compaction pass)
+  int32_t bucket_cnt;    // keys inside the bucket (exact after a key level)
   int32_t emit_cnt;      // ids written by the compaction pass
   int32_t cand_cnt;      // candidates written by the compaction pass
   int32_t n_keys;        // causal key count of the row

@@ -23,7 +23,7 @@
 // are requested, one more sweep appends every row's members in position order.
 // Each pass has its own inner loop; pages that lie wholly below a warp's first row need no causal test.
 #include <cstdlib>
-#include "rtp_device.cuh"
+#include "mass_hist.cuh"
 
 namespace rtp {
 
@@ -35,17 +35,10 @@ constexpr int kCRows = 128;
 constexpr int kPagesPerStage = 4;
 constexpr int kStageKeys = kPagesPerStage * kPage;                  // 256 keys
 constexpr int kStageBytesC = kStageKeys * kIndexDim * 2;            // 8 KB
-constexpr int kBins = 64;                                           // bins per level
-constexpr float kL1Scale = 2.0f;                                    // level-1 bins per unit of d = M - s
 constexpr int kCandCapC = 64;                                       // candidates sorted exactly per row
 constexpr int kRowBytes = kBins * 8 + 8;                            // per row: 64 x {sum, carries} or 64 x {key, idx}; +8 staggers the banks
 constexpr int kMaxPasses = 14;
-constexpr float kLog2eC = 1.4426950408889634f;
-// A key adds q = round(e_rel * 2^20) to its bin with one native 32-bit shared-memory add; the returned old value
-// tells whether the sum wrapped, and then (rarely) a second add counts the carry in the next word.  e_rel = mass
-// relative to the bin's (level 1) or the bucket's (key levels) upper end, in (e^-0.5, 1]: every key adds at
-// least kMinQ, which bounds the number of keys of a bin by its sum.
-constexpr float kMinQ = 634880.0f;                                  // (floor(e^-0.5 * 1024) - 1) * 1024
+constexpr float kLog2eC = kLog2eH;
 constexpr int kQueueCap = 160;                                      // per-warp queue of bucket hits (entries of 8 bytes)
 
 enum Phase { kPhMax = 0, kPhL1 = 1, kPhKey = 2, kPhCollect = 3, kPhTie = 4, kPhDone = 5 };
@@ -78,33 +71,6 @@ __device__ __forceinline__ void cp_async16c(uint32_t dst, const void* src) {
 }
 __device__ __forceinline__ uint32_t smem_u32c(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-// Level-1 bin of a score: the integer nearest to 2 (M - s), clamped to [0, 63]; bin b holds M - s in
-// [b/2 - 1/4, b/2 + 1/4] (the last bin pools everything below).  Adding 1.5 * 2^23 leaves that integer in the low
-// mantissa bits, so no float <-> int conversion instruction is needed; the same arithmetic serves the histogram
-// pass and the bisection that turns a bin into a key interval.
-constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
-__device__ __forceinline__ int l1_bin_f(float M, float s, float& bin_f) {
-  const float u = fminf(fmaxf((M - s) * kL1Scale, 0.0f), (float)(kBins - 1));
-  const float t = u + kMagic;
-  bin_f = t - kMagic;
-  return __float_as_int(t) & (kBins - 1);
-}
-__device__ __forceinline__ int l1_bin(float M, float s) {
-  float f;
-  return l1_bin_f(M, s, f);
-}
-
-// Adds round(2^x) (x <= 20) to an accumulator {sum mod 2^32, carries}.
-__device__ __forceinline__ void add_mass(uint32_t* acc, float x) {
-  // nearest integer to 2^x through the mantissa of (2^x + 2^23): no conversion instruction
-  const uint32_t q = min(__float_as_uint(fast_ex2(x) + 8388608.0f) - 0x4b000000u, 1u << 20);
-  const uint32_t old = atomicAdd(acc, q);
-  if (old + q < old) atomicAdd(acc + 1, 1u);
-}
-__device__ __forceinline__ float acc_mass(uint32_t sum, uint32_t carries) {   // in units of 2^-20
-  return (float)carries * 4294967296.0f + (float)sum;
 }
 
 // Per-lane view of its two rows for one pass (registers).
@@ -168,7 +134,7 @@ __device__ __forceinline__ void page_l1(const unsigned char* pg, const QFrag& iq
       float bin_f;
       const int bin = l1_bin_f(M, s, bin_f);   // (rows that are already done have no M: they land in bin 0)
       // mass relative to the bin's upper end: exp(-((M - s) - (bin/2 - 1/4))), scaled by 2^20
-      add_mass((lo ? hist_a : hist_b) + 2 * bin, fmaf(bin_f, 0.5f * kLog2eC, fmaf(M - s, -kLog2eC, 20.0f - 0.25f * kLog2eC)));
+      add_mass((lo ? hist_a : hist_b) + 2 * bin, l1_mass_arg(M, s, bin_f));
     }
   }
 }
@@ -559,8 +525,8 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
         // masses relative to M
         float m0f, m1f;
         if (l1) {
-          m0f = q0 * fast_ex2(-kLog2eC * (0.5f * (float)b0 - 0.25f) - 20.0f);
-          m1f = q1 * fast_ex2(-kLog2eC * (0.5f * (float)b1 - 0.25f) - 20.0f);
+          m0f = q0 * l1_bin_scale(b0);
+          m1f = q1 * l1_bin_scale(b1);
         } else {
           const float sc = R.e_ref * 9.5367431640625e-07f;   // 2^-20
           m0f = q0 * sc;
@@ -616,27 +582,10 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
               S->sel_mass = 1.0f;
               S->phase = kPhDone;
             } else {
-              // Exact interval [klo, khi] of ordered keys whose level-1 bin is `bin`: l1_bin is monotone in the
-              // key, so both ends are found by bisection between two keys that lie safely outside the bucket.
               const float M = R.M;
-              const float hi_s = M - ((float)bin - 0.5f) / kL1Scale, lo_s = M - ((float)bin + 0.5f) / kL1Scale;
-              const float pad = 1e-5f * fmaxf(1.0f, fmaxf(fabsf(hi_s), fabsf(lo_s))) + 1e-3f;
-              const uint32_t lo = okey(finish_score(lo_s - pad, 1.0f));
-              const uint32_t hi = okey(finish_score(fminf(hi_s + pad, M), 1.0f));
-              uint32_t a = lo, b2 = hi;            // klo = smallest key with bin <= `bin`
-              if (l1_bin(M, okey_to_float(a)) <= bin) b2 = a;
-              while (a + 1 < b2) {
-                const uint32_t mid = a + ((b2 - a) >> 1);
-                if (l1_bin(M, okey_to_float(mid)) <= bin) b2 = mid; else a = mid;
-              }
-              const uint32_t klo = b2;
-              a = klo; b2 = hi;                    // khi = largest key with bin >= `bin`
-              if (l1_bin(M, okey_to_float(b2)) >= bin) a = b2;
-              while (a + 1 < b2) {
-                const uint32_t mid = a + ((b2 - a) >> 1);
-                if (l1_bin(M, okey_to_float(mid)) >= bin) a = mid; else b2 = mid;
-              }
-              const uint32_t khi = a;
+              const float hi_s = l1_bin_hi(M, bin);
+              uint32_t klo, khi;
+              l1_bin_keys(M, bin, klo, khi);
               const uint32_t span = khi - klo + 1u;
               const int bits = span > 1u ? 32 - __clz(span - 1u) : 0;
               float rlo, rhi;

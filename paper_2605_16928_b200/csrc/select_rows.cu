@@ -1,18 +1,19 @@
 // S2-S4 for explicit rows (the decode path): fused indexer scan + top-p selection (Eq. 5).
 //
-// The context of one (row, index head) is split over many CTAs.  Selection is a radix descent on
-// the ordered 32-bit key of the fp32 score, with softmax mass as the weight:
-//   hist pass    every CTA scores its keys (MMA, see score16) and adds exp(s - ref) and a count to a
-//                2048-bin histogram of the next key bits (shared memory, then global atomics);
-//   resolve      one CTA per (row, head) walks the bins from the top and finds the bucket in which the
-//                cumulative mass reaches p * Z; as soon as that bucket holds <= kCandCap keys the row
-//                stops refining;
-//   compaction   every key above the bucket is emitted, keys inside it become candidates;
-//   finalize     one CTA per (row, head) sorts the candidates by (score desc, position asc) and takes
-//                the shortest prefix that reaches the target mass.
-// The first histogram needs no row maximum: bin b accumulates exp(s - ub(b)) with ub(b) the largest
-// value of the bin, and the resolve step rescales by exp(ub(b) - M) once M is known.
-#include "rtp_device.cuh"
+// The context of one (row, index head) unit is split over many CTAs; every pass scores its keys again (MMA, see
+// score16) from the index-key cache:
+//   max          row maximum M of every head (atomicMax on the ordered key);
+//   level 1      64-bin histogram of softmax mass over d = M - s in steps of 1/2, fixed point, one native
+//                shared-memory add per score, merged into global memory; the unit's last CTA to finish (ticket
+//                counter, nobody waits) finds Z and the bin in which the cumulative mass reaches p * Z and turns
+//                it into an exact interval of ordered keys and of unscaled MMA outputs;
+//   key levels   six more key bits per pass inside that interval, with exact counts, until the bucket holds at most
+//                kCandCap keys (or a single key value); hits are rare, so a warp queues them and works them off 32
+//                at a time;
+//   compaction   every key above the bucket is counted and emitted, keys inside it become candidates;
+//   finalize     one CTA per (row, head) sorts the candidates by (score desc, position asc) and takes the shortest
+//                prefix that reaches the target mass.
+#include "mass_hist.cuh"
 
 namespace rtp {
 
@@ -23,11 +24,6 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kHeadsPerCta = 4;
 constexpr int kStage = 128;      // staged ids per (warp, head) before a flush
 constexpr int kCandStage = 48;   // staged boundary candidates per (warp, head)
-
-struct Bin {
-  float mass;
-  uint32_t cnt;
-};
 
 struct RowCtx {
   int64_t r;
@@ -57,6 +53,13 @@ __device__ __forceinline__ RowCtx make_row_ctx(const CacheView& cv, const Dims& 
   return x;
 }
 
+// One 64-key page of index keys: 2 KB, four 16-byte loads per lane.
+__device__ __forceinline__ void load_page(const CacheView& cv, const RowCtx& x, int p, int lane, uint4 (&v)[4]) {
+  const __nv_bfloat16* base = ikey_page_ptr(cv, x.seq, p, x.ih);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) v[i] = ld_stream_v4(base + (i * 32 + lane) * 8);
+}
+
 // Which retrieval head (index into ret_q_heads) this lane post-processes in head group z, or -1.
 // MMA row g holds head slot g, row g + 8 holds slot g + 8; group z covers slots 4z .. 4z+3.
 __device__ __forceinline__ int lane_head_slot(int lane, int z) {
@@ -81,253 +84,471 @@ __global__ void sel_init_kernel(const CacheView cv, const Dims d, const Rows row
   state[i] = s;
 }
 
-// ---- histogram pass -----------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) sel_hist_kernel(
-    const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows,
-    const __nv_bfloat16* __restrict__ qt, SelState* __restrict__ state, Bin* __restrict__ hist,
-    int n_splits, int32_t* status) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* h_mass = reinterpret_cast<float*>(smem_raw);                              // [4][2048]
-  uint32_t* h_cnt = reinterpret_cast<uint32_t*>(smem_raw + kHeadsPerCta * kSelBins * 4);  // [4][2048]
-  __shared__ int any_active;
-
-  const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, status);
-  const int z = blockIdx.z;
-  if (z * kHeadsPerCta >= x.nh || x.p_lo >= x.p_hi) return;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, c = lane & 3;
-
-  const int slot = lane_head_slot(lane, z);
-  const bool use_hi = (z >> 1) != 0;
-  const int j = (lane >> 2) & 3;
-  int head = (slot >= 0 && slot < x.nh) ? hm.ih_heads[x.ih][slot] : -1;
-  SelState* st = head >= 0 ? state + (x.r * d.n_ret + head) : nullptr;
-  int level = 0, have_M = 0;
-  uint32_t lo_key = 0;
-  float M = 0.f;
-  if (st) {
-    if (st->mode != kRefine) {
-      head = -1;
-    } else {
-      level = st->level;
-      have_M = st->pad;
-      lo_key = st->lo_key;
-      M = st->M;
+// ---- which scores a lane post-processes ------------------------------------------------------------
+// After score16() lane (g, c) holds keys 4c .. 4c+3 of the 16-key group for head slots g (s_lo) and g + 8 (s_hi).
+// With at most four heads on the index head (NH4) the lanes g >= 4 would idle: they take over keys 4c+2, 4c+3 of
+// the lane that holds the same slot (g - 4), so that every lane handles two scores of slot g & 3.  Otherwise a lane
+// handles four scores of slot g (set A) and four of slot g + 8 (set B).
+template <bool NH4>
+struct LaneElems {
+  static constexpr int kN = NH4 ? 2 : 8;
+  float raw[kN];
+  int koff[kN];   // key offset inside the 16-key group
+};
+template <bool NH4>
+__device__ __forceinline__ LaneElems<NH4> lane_elems(const float (&s_lo)[4], const float (&s_hi)[4], int lane) {
+  LaneElems<NH4> r;
+  const int c = lane & 3;
+  if (NH4) {
+    const float t2 = __shfl_sync(0xffffffffu, s_lo[2], lane & 15), t3 = __shfl_sync(0xffffffffu, s_lo[3], lane & 15);
+    const bool up = lane >= 16;
+    r.raw[0] = up ? t2 : s_lo[0];
+    r.raw[1] = up ? t3 : s_lo[1];
+    r.koff[0] = 4 * c + (up ? 2 : 0);
+    r.koff[1] = r.koff[0] + 1;
+  } else {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      r.raw[e] = s_lo[e];
+      r.raw[4 + e] = s_hi[e];
+      r.koff[e] = r.koff[4 + e] = 4 * c + e;
     }
   }
-  if (threadIdx.x == 0) any_active = 0;
+  return r;
+}
+// head slot of element e of this lane
+template <bool NH4>
+__device__ __forceinline__ int elem_slot(int lane, int e) {
+  const int g = lane >> 2;
+  return NH4 ? (g & 3) : (e < 4 ? g : g + 8);
+}
+
+// The last CTA of a (row, index head) unit to finish a pass resolves it: every CTA publishes its partial results,
+// fences, and takes a ticket; the one that draws the last ticket sees all of them.  Nobody waits.
+__device__ __forceinline__ bool take_last_ticket(uint32_t* ticket, uint32_t n_ctas) {
+  __shared__ int s_is_last;
+  __threadfence();
   __syncthreads();
-  if (head >= 0) any_active = 1;
-  __syncthreads();
-  if (!any_active) return;
-  for (int i = threadIdx.x; i < kHeadsPerCta * kSelBins; i += kThreads) {
-    h_mass[i] = 0.f;
-    h_cnt[i] = 0u;
+  if (threadIdx.x == 0) {
+    const uint32_t t = atomicAdd(ticket, 1u);
+    s_is_last = (t == n_ctas - 1u) ? 1 : 0;
+    if (s_is_last) *ticket = 0u;   // ready for the next pass
   }
   __syncthreads();
+  if (s_is_last) __threadfence();
+  return s_is_last != 0;
+}
 
+// ---- pass 1: row maximum ----------------------------------------------------------------------------
+template <bool NH4>
+__global__ void __launch_bounds__(kThreads) sel_max_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
+                                                           const Rows rows, const __nv_bfloat16* __restrict__ qt,
+                                                           SelState* __restrict__ state, int n_splits, int32_t* status) {
+  __shared__ float s_max[kWarps][16];
+  const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, status);
+  if (x.p_lo >= x.p_hi) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
-  uint32_t max_key = 0;
+  float mx_a = -INFINITY, mx_b = -INFINITY;
+  uint4 v[4], vn[4];
+  if (x.p_lo + warp < x.p_hi) load_page(cv, x, x.p_lo + warp, lane, vn);
   for (int p = x.p_lo + warp; p < x.p_hi; p += kWarps) {
-    const __nv_bfloat16* base = ikey_page_ptr(cv, x.seq, p, x.ih);
-    uint4 v[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) v[i] = ld_stream_v4(base + (i * 32 + lane) * 8);
+    for (int i = 0; i < 4; ++i) v[i] = vn[i];
+    if (p + kWarps < x.p_hi) load_page(cv, x, p + kWarps, lane, vn);   // in flight while this page is worked on
+    const bool tail = (p + 1) * kPage > x.n_keys;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       float s_lo[4], s_hi[4];
       score16(qf, v[i], lane, s_lo, s_hi);
-      if (head < 0) continue;
-      const int n0 = p * kPage + i * 16 + 4 * c;
+      const LaneElems<NH4> el = lane_elems<NH4>(s_lo, s_hi, lane);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (n0 + e >= x.n_keys) continue;
-        const float s = finish_score(use_hi ? s_hi[e] : s_lo[e], d.score_scale);
-        const uint32_t key = okey(s);
-        int bin;
-        float ref = M;
-        if (level == 0) {
-          bin = key >> 21;
-          max_key = max(max_key, key);
-          if (!have_M) ref = okey_to_float((key | 0x1fffffu));
-        } else if (level == 11) {
-          if ((key ^ lo_key) >> 21) continue;
-          bin = (key >> 10) & 0x7ff;
-        } else {
-          if ((key ^ lo_key) >> 10) continue;
-          bin = key & 0x3ff;
-        }
-        atomicAdd(&h_mass[j * kSelBins + bin], __expf(s - ref));
-        atomicAdd(&h_cnt[j * kSelBins + bin], 1u);
+      for (int e = 0; e < LaneElems<NH4>::kN; ++e) {
+        if (tail && p * kPage + i * 16 + el.koff[e] >= x.n_keys) continue;
+        if (NH4 || e < 4) mx_a = fmaxf(mx_a, el.raw[e]); else mx_b = fmaxf(mx_b, el.raw[e]);
       }
     }
   }
-  max_key = max(max_key, __shfl_xor_sync(0xffffffffu, max_key, 1));
-  max_key = max(max_key, __shfl_xor_sync(0xffffffffu, max_key, 2));
-  if (level == 0 && head >= 0 && c == 0 && max_key) atomicMax(&st->max_key, max_key);
+  mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
+  mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+  if (NH4) mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 16));
+  mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
+  mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+  if ((lane & 3) == 0) {
+    const int g = lane >> 2;
+    if (NH4) {
+      if (g < 4) s_max[warp][g] = mx_a;
+    } else {
+      s_max[warp][g] = mx_a;
+      s_max[warp][g + 8] = mx_b;
+    }
+  }
   __syncthreads();
-  for (int i = threadIdx.x; i < kHeadsPerCta * kSelBins; i += kThreads) {
-    const uint32_t n = h_cnt[i];
-    if (n == 0) continue;
-    const int jj = i / kSelBins, bin = i % kSelBins;
-    const int slot2 = (z >> 1) * 8 + (z & 1) * 4 + jj;  // head slot of entry jj in group z
-    if (slot2 >= x.nh) continue;
-    const int hd = hm.ih_heads[x.ih][slot2];
-    Bin* b = hist + (x.r * d.n_ret + hd) * kSelBins + bin;
-    atomicAdd(&b->mass, h_mass[i]);
-    atomicAdd(&b->cnt, n);
+  if (threadIdx.x < x.nh) {
+    float m = -INFINITY;
+    for (int w = 0; w < kWarps; ++w) m = fmaxf(m, s_max[w][threadIdx.x]);
+    // the maximum was taken on unscaled MMA outputs; scaling by a positive factor is monotone
+    if (m > -INFINITY) atomicMax(&state[x.r * d.n_ret + hm.ih_heads[x.ih][threadIdx.x]].max_key, okey(finish_score(m, d.score_scale)));
   }
 }
 
-// ---- resolve --------------------------------------------------------------------------------------
-constexpr int kResThreads = 256;
-
-__global__ void __launch_bounds__(kResThreads) sel_resolve_kernel(const Dims d, SelState* __restrict__ state,
-                                                                  Bin* __restrict__ hist) {
-  SelState* st = state + blockIdx.x;
-  if (st->mode != kRefine) return;
-  Bin* bins = hist + (int64_t)blockIdx.x * kSelBins;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int level = st->level;
-  const int have_M = st->pad;
-  const int nb = (level == 22) ? 1024 : kSelBins;
-  const float M = (level == 0 && !have_M) ? okey_to_float(st->max_key) : st->M;
-  __shared__ float w_mass[kResThreads / 32];
-  __shared__ uint32_t w_cnt[kResThreads / 32];
-  __shared__ int s_wide, s_found, s_last;
-  if (tid == 0) {
-    s_wide = 0;
-    s_found = 0x7fffffff;
-    s_last = -1;
+// ---- pass 2: level-1 mass histogram over M - s, resolved by the unit's last CTA ----------------------------------
+template <bool NH4>
+__global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
+                                                          const Rows rows, const __nv_bfloat16* __restrict__ qt,
+                                                          SelState* __restrict__ state, unsigned long long* __restrict__ g_mass,
+                                                          uint32_t* __restrict__ tickets, int n_splits, int32_t* status) {
+  __shared__ uint32_t hist[16][kBins][2];
+  __shared__ float s_M[16];
+  __shared__ int s_on[16];
+  const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x < 16) {
+    int on = 0;
+    float M = 0.f;
+    if (threadIdx.x < x.nh) {
+      const SelState* st = state + (x.r * d.n_ret + hm.ih_heads[x.ih][threadIdx.x]);
+      on = st->mode == kRefine && st->n_keys > 0;
+      M = okey_to_float(st->max_key);
+    }
+    s_on[threadIdx.x] = on;
+    s_M[threadIdx.x] = M;
   }
+  for (int i = threadIdx.x; i < 16 * kBins * 2; i += kThreads) (&hist[0][0][0])[i] = 0u;
   __syncthreads();
+  int any = 0;
+  for (int j = 0; j < x.nh; ++j) any |= s_on[j];
+  if (!any) return;   // the same decision in every CTA of the unit
 
-  float mass[8];
-  uint32_t cnt[8];
-  float tm = 0.f;
-  uint32_t tc = 0;
+  const int slot_a = elem_slot<NH4>(lane, 0), slot_b = NH4 ? slot_a : elem_slot<NH4>(lane, 4);
+  const bool on_a = slot_a < x.nh && s_on[slot_a], on_b = !NH4 && slot_b < x.nh && s_on[slot_b];
+  const float M_a = s_M[slot_a], M_b = s_M[slot_b];
+  const QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
+  uint4 v[4], vn[4];
+  if (x.p_lo + warp < x.p_hi) load_page(cv, x, x.p_lo + warp, lane, vn);
+  for (int p = x.p_lo + warp; p < x.p_hi; p += kWarps) {
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const int o = tid * 8 + k;  // order index: 0 = top bin
-    mass[k] = 0.f;
-    cnt[k] = 0;
-    if (o < nb) {
-      const int bin = nb - 1 - o;
-      const Bin b = bins[bin];
-      bins[bin] = Bin{0.f, 0u};
-      cnt[k] = b.cnt;
-      float m = b.mass;
-      if (level == 0 && !have_M && b.cnt) {
-        const uint32_t ubk = ((uint32_t)bin << 21) | 0x1fffffu;
-        const uint32_t ex = (ubk & 0x80000000u) ? ((ubk >> 23) & 0xff) : ((~ubk >> 23) & 0xff);
-        if (ex >= 127 + 8) s_wide = 1;
-        m *= __expf(okey_to_float(ubk) - M);
+    for (int i = 0; i < 4; ++i) v[i] = vn[i];
+    if (p + kWarps < x.p_hi) load_page(cv, x, p + kWarps, lane, vn);   // in flight while this page is worked on
+    const bool tail = (p + 1) * kPage > x.n_keys;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float s_lo[4], s_hi[4];
+      score16(qf, v[i], lane, s_lo, s_hi);
+      const LaneElems<NH4> el = lane_elems<NH4>(s_lo, s_hi, lane);
+#pragma unroll
+      for (int e = 0; e < LaneElems<NH4>::kN; ++e) {
+        const bool set_a = NH4 || e < 4;
+        if (!(set_a ? on_a : on_b)) continue;
+        if (tail && p * kPage + i * 16 + el.koff[e] >= x.n_keys) continue;
+        const float s = finish_score(el.raw[e], d.score_scale);
+        const float M = set_a ? M_a : M_b;
+        float bin_f;
+        const int bin = l1_bin_f(M, s, bin_f);
+        add_mass(&hist[set_a ? slot_a : slot_b][bin][0], l1_mass_arg(M, s, bin_f));
       }
-      mass[k] = m;
-      tm += m;
-      tc += b.cnt;
     }
   }
   __syncthreads();
-  if (s_wide) {  // very large scores: the bin-relative masses may have underflowed; redo relative to M
-    if (tid == 0) {
-      st->M = M;
-      st->pad = 1;
-    }
-    return;
+  for (int i = threadIdx.x; i < x.nh * kBins; i += kThreads) {
+    const int j = i / kBins, bin = i % kBins;
+    const uint32_t sum = hist[j][bin][0], car = hist[j][bin][1];
+    if (sum | car)
+      atomicAdd(g_mass + (x.r * d.n_ret + hm.ih_heads[x.ih][j]) * kBins + bin, ((unsigned long long)car << 32) | sum);
   }
-  // block exclusive scan of (tm, tc) in order of tid
-  float im = tm;
-  uint32_t ic = tc;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const float a = __shfl_up_sync(0xffffffffu, im, o);
-    const uint32_t b = __shfl_up_sync(0xffffffffu, ic, o);
-    if (lane >= o) {
-      im += a;
-      ic += b;
-    }
-  }
-  if (lane == 31) {
-    w_mass[warp] = im;
-    w_cnt[warp] = ic;
-  }
-  __syncthreads();
-  float base_m = 0.f, total_m = 0.f;
-  uint32_t base_c = 0;
-  for (int w = 0; w < kResThreads / 32; ++w) {
-    if (w < warp) {
-      base_m += w_mass[w];
-      base_c += w_cnt[w];
-    }
-    total_m += w_mass[w];
-  }
-  float ex_m = base_m + im - tm;  // mass of bins before this thread's first bin
-  uint32_t ex_c = base_c + ic - tc;
+  if (!take_last_ticket(tickets + blockIdx.x, gridDim.y)) return;
 
-  float Z = st->Z, target = st->target;
-  if (level == 0) {
-    Z = total_m;
-    target = d.top_p * Z * (1.0f + kMassMargin);
-  }
-  const float above0 = st->mass_above;
-  // first bin (from the top) at which the cumulative mass reaches the target
-  {
-    float run = ex_m;
-    int found = -1, last = -1;
+  // ---- resolve: one warp per head; lane l looks at bins 2l, 2l+1 (bin 0 is the top) ----
+  for (int j = warp; j < x.nh; j += kWarps) {
+    if (!s_on[j]) continue;
+    const int64_t rh = x.r * d.n_ret + hm.ih_heads[x.ih][j];
+    SelState* st = state + rh;
+    unsigned long long* gm = g_mass + rh * kBins;
+    const int b0 = 2 * lane, b1 = 2 * lane + 1;
+    const unsigned long long u0 = __ldcg(gm + b0), u1 = __ldcg(gm + b1);
+    gm[b0] = 0ull;
+    gm[b1] = 0ull;
+    const float q0 = __ull2float_rn(u0), q1 = __ull2float_rn(u1);
+    const float m0 = q0 * l1_bin_scale(b0), m1 = q1 * l1_bin_scale(b1);
+    float inc = m0 + m1;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      if (cnt[k]) {
-        last = tid * 8 + k;
-        if (found < 0 && above0 + run + mass[k] >= target) found = tid * 8 + k;
+    for (int o = 1; o < 32; o <<= 1) {
+      const float t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    const float Z = __shfl_sync(0xffffffffu, inc, 31);
+    const float target = d.top_p * Z * (1.0f + kMassMargin);
+    const float run = inc - (m0 + m1);
+    int found = 64, last = -1;
+    if (u0) {
+      last = b0;
+      if (run + m0 >= target) found = b0;
+    }
+    if (u1) {
+      last = b1;
+      if (found == 64 && run + m0 + m1 >= target) found = b1;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      found = min(found, __shfl_xor_sync(0xffffffffu, found, o));
+      last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+    }
+    if (found == 64) found = last;   // rounding left the target just out of reach: lowest populated bin
+    if (found < 0) {
+      if (lane == 0) {               // empty histogram: cannot happen for a non-empty row
+        st->mode = kSelectAll;
+        set_status(status, RTP_ERR_UNSUPPORTED);
       }
-      run += mass[k];
+      continue;
     }
-    if (found >= 0) atomicMin(&s_found, found);
-    if (last >= 0) atomicMax(&s_last, last);
+    {
+      // the lane that owns the bin hands its figures to the warp; the interval searches are warp-wide
+      const int owner = found >> 1;
+      const bool first = (found & 1) == 0;
+      const float M = s_M[j];
+      const float above = __shfl_sync(0xffffffffu, first ? run : run + m0, owner);
+      const float q = __shfl_sync(0xffffffffu, first ? q0 : q1, owner);
+      uint32_t klo = 0u, khi = 0u;
+      float rlo = 0.f, rhi = 0.f;
+      if (found != kBins - 1) {
+        l1_bin_keys_warp(M, found, lane, klo, khi);
+        raw_preimage_warp(d.score_scale, klo, khi, lane, rlo, rhi);
+      }
+      if (lane == 0) {
+        st->M = M;
+        st->Z = Z;
+        st->target = target;
+        st->mass_above = above;
+        if (found == kBins - 1) {
+          st->mode = kSelectAll;       // the cut falls into the pooled tail (mass below 1e-13 per key): take every key
+        } else {
+          const uint32_t span = khi - klo + 1u;
+          const int bits = span > 1u ? 32 - __clz(span - 1u) : 0;
+          st->lo_key = klo;
+          st->hi_key = khi;
+          st->span = span;
+          st->shift = max(0, bits - 6);
+          st->raw_lo = rlo;
+          st->raw_hi = rhi;
+          st->ref_s = l1_bin_hi(M, found);
+          st->e_ref = fast_ex2(-kLog2eH * (0.5f * (float)found - 0.25f));
+          if (q < 0.999f * kMinQ * (float)kCandCap) st->mode = kCollect;   // fewer than kCandCap keys in the bin
+        }
+      }
+    }
   }
+}
+
+// ---- pass 3 (repeated): 64-bin mass histogram of the next six key bits inside the bucket --------------------------
+// Only a small share of the scores falls into a head's bucket: a warp appends those hits to a queue in shared
+// memory and works them off 32 at a time, one hit per lane.
+constexpr int kQueueCapR = 160;   // >= 31 + 4 x 32 entries
+
+struct KeyParams {   // per head slot, shared memory
+  uint32_t base_key;
+  int32_t shift;
+  float ref_s;
+};
+
+__device__ __noinline__ void drain_row_hits(uint32_t* wq, int& qcnt, int lane, const KeyParams* kp,
+                                            uint32_t (*hist)[kBins][3], float scale) {
+  __syncwarp();
+  for (int base = 0; base < qcnt; base += 32) {
+    const int i = base + lane;
+    if (i < qcnt) {
+      const int slot = (int)wq[2 * i];
+      const float s = finish_score(__uint_as_float(wq[2 * i + 1]), scale);
+      const uint32_t t = okey(s) - kp[slot].base_key;
+      uint32_t* acc = &hist[slot][t >> kp[slot].shift][0];
+      add_mass(acc, fmaf(s - kp[slot].ref_s, kLog2eH, 20.0f));
+      atomicAdd(acc + 2, 1u);
+    }
+  }
+  __syncwarp();
+  qcnt = 0;
+}
+
+template <bool NH4>
+__global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
+                                                           const Rows rows, const __nv_bfloat16* __restrict__ qt,
+                                                           SelState* __restrict__ state, unsigned long long* __restrict__ g_mass,
+                                                           uint32_t* __restrict__ g_cnt, uint32_t* __restrict__ tickets,
+                                                           int n_splits, int max_levels, int32_t* status) {
+  __shared__ uint32_t hist[16][kBins][3];   // {sum, carries, count}
+  __shared__ uint32_t queue[kWarps][kQueueCapR * 2];
+  __shared__ KeyParams kp[16];
+  __shared__ float s_lo_raw[16], s_hi_raw[16];
+  __shared__ int s_on[16];
+  const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float kInf = __int_as_float(0x7f800000);
+  // With one CTA per unit (n_splits == 1) the CTA is always the one that resolves, and it goes on with the next
+  // level by itself: max_levels > 1 takes whatever the split passes left unresolved to the end.
+#pragma unroll 1
+  for (int level = 0; level < max_levels; ++level) {
+  if (threadIdx.x < 16) {
+    int on = 0;
+    float lo = kInf, hi = -kInf;
+    KeyParams k = {0u, 0, 0.f};
+    if (threadIdx.x < x.nh) {
+      const volatile SelState* st = state + (x.r * d.n_ret + hm.ih_heads[x.ih][threadIdx.x]);
+      on = st->mode == kRefine && st->n_keys > 0;
+      if (on) {
+        lo = st->raw_lo;
+        hi = st->raw_hi;
+        k.base_key = st->lo_key;
+        k.shift = st->shift;
+        k.ref_s = st->ref_s;
+      }
+    }
+    s_on[threadIdx.x] = on;
+    s_lo_raw[threadIdx.x] = lo;
+    s_hi_raw[threadIdx.x] = hi;
+    kp[threadIdx.x] = k;
+  }
+  for (int i = threadIdx.x; i < 16 * kBins * 3; i += kThreads) (&hist[0][0][0])[i] = 0u;
   __syncthreads();
-  int pick = s_found;
-  if (pick == 0x7fffffff) pick = s_last;  // rounding left the target just out of reach: take everything
-  if (pick < 0) return;                   // empty histogram (cannot happen for a non-empty row)
-  if (pick / 8 == tid) {
-    float run = ex_m;
-    uint32_t runc = ex_c;
-    for (int k = 0; k < (pick & 7); ++k) {
-      run += mass[k];
-      runc += cnt[k];
+  int any = 0;
+  for (int j = 0; j < x.nh; ++j) any |= s_on[j];
+  if (!any) return;   // the same decision in every CTA of the unit
+
+  const int slot_a = elem_slot<NH4>(lane, 0), slot_b = NH4 ? slot_a : elem_slot<NH4>(lane, 4);
+  const float lo_a = s_lo_raw[slot_a], hi_a = s_hi_raw[slot_a];
+  const float lo_b = NH4 ? kInf : s_lo_raw[slot_b], hi_b = NH4 ? -kInf : s_hi_raw[slot_b];
+  const QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
+  uint32_t* wq = queue[warp];
+  int qcnt = 0;
+  const uint32_t lt = (1u << lane) - 1u;
+  uint4 v[4], vn[4];
+  if (x.p_lo + warp < x.p_hi) load_page(cv, x, x.p_lo + warp, lane, vn);
+  for (int p = x.p_lo + warp; p < x.p_hi; p += kWarps) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = vn[i];
+    if (p + kWarps < x.p_hi) load_page(cv, x, p + kWarps, lane, vn);   // in flight while this page is worked on
+    const bool tail = (p + 1) * kPage > x.n_keys;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float s_lo[4], s_hi[4];
+      score16(qf, v[i], lane, s_lo, s_hi);
+      const LaneElems<NH4> el = lane_elems<NH4>(s_lo, s_hi, lane);
+      bool hit[LaneElems<NH4>::kN];
+      bool any_hit = false;
+#pragma unroll
+      for (int e = 0; e < LaneElems<NH4>::kN; ++e) {
+        const bool set_a = NH4 || e < 4;
+        hit[e] = el.raw[e] >= (set_a ? lo_a : lo_b) && el.raw[e] <= (set_a ? hi_a : hi_b);
+        if (tail && p * kPage + i * 16 + el.koff[e] >= x.n_keys) hit[e] = false;
+        any_hit = any_hit || hit[e];
+      }
+      if (!__any_sync(0xffffffffu, any_hit)) continue;
+#pragma unroll
+      for (int e = 0; e < LaneElems<NH4>::kN; ++e) {
+        const uint32_t m = __ballot_sync(0xffffffffu, hit[e]);
+        if (m) {
+          if (hit[e]) {
+            const int pos = qcnt + __popc(m & lt);
+            wq[2 * pos] = (uint32_t)((NH4 || e < 4) ? slot_a : slot_b);
+            wq[2 * pos + 1] = __float_as_uint(el.raw[e]);
+          }
+          qcnt += __popc(m);
+        }
+        if ((e & 3) == 3 || e == LaneElems<NH4>::kN - 1)
+          if (qcnt >= 32) drain_row_hits(wq, qcnt, lane, kp, hist, d.score_scale);
+      }
     }
-    const int k = pick & 7;
-    const uint32_t bin = (uint32_t)(nb - 1 - pick);
-    uint32_t lo, hi;
-    int new_level;
-    if (level == 0) {
-      lo = bin << 21;
-      hi = lo | 0x1fffffu;
-      new_level = 11;
-    } else if (level == 11) {
-      lo = (st->lo_key & 0xffe00000u) | (bin << 10);
-      hi = lo | 0x3ffu;
-      new_level = 22;
-    } else {
-      lo = (st->lo_key & 0xfffffc00u) | bin;
-      hi = lo;
-      new_level = 32;
+  }
+  if (qcnt > 0) drain_row_hits(wq, qcnt, lane, kp, hist, d.score_scale);
+  __syncthreads();
+  for (int i = threadIdx.x; i < x.nh * kBins; i += kThreads) {
+    const int j = i / kBins, bin = i % kBins;
+    const uint32_t n = hist[j][bin][2];
+    if (n) {
+      const int64_t o = (x.r * d.n_ret + hm.ih_heads[x.ih][j]) * kBins + bin;
+      atomicAdd(g_mass + o, ((unsigned long long)hist[j][bin][1] << 32) | hist[j][bin][0]);
+      atomicAdd(g_cnt + o, n);
     }
-    st->lo_key = lo;
-    st->hi_key = hi;
-    st->level = new_level;
-    st->M = M;
-    st->Z = Z;
-    st->target = target;
-    st->mass_above = above0 + run;
-    st->cnt_above = st->cnt_above + (int)runc;
-    st->bucket_cnt = (int)cnt[k];
-    st->bucket_mass = mass[k];
-    st->pad = 1;
-    if ((int)cnt[k] <= kCandCap)
-      st->mode = kCollect;
-    else if (new_level == 32)
-      st->mode = kTieScan;
+  }
+  if (!take_last_ticket(tickets + blockIdx.x, gridDim.y)) return;
+
+  // ---- resolve: one warp per head; lane l looks at bins 63 - 2l, 62 - 2l (bin 63 is the top) ----
+  for (int j = warp; j < x.nh; j += kWarps) {
+    if (!s_on[j]) continue;
+    const int64_t rh = x.r * d.n_ret + hm.ih_heads[x.ih][j];
+    SelState* st = state + rh;
+    unsigned long long* gm = g_mass + rh * kBins;
+    uint32_t* gc = g_cnt + rh * kBins;
+    const int b0 = 63 - 2 * lane, b1 = 62 - 2 * lane;
+    const unsigned long long u0 = __ldcg(gm + b0), u1 = __ldcg(gm + b1);
+    const uint32_t c0 = __ldcg(gc + b0), c1 = __ldcg(gc + b1);
+    gm[b0] = 0ull;
+    gm[b1] = 0ull;
+    gc[b0] = 0u;
+    gc[b1] = 0u;
+    const float sc = st->e_ref * 9.5367431640625e-07f;   // 2^-20
+    const float m0 = __ull2float_rn(u0) * sc, m1 = __ull2float_rn(u1) * sc;
+    float inc = m0 + m1;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const float t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    const float above0 = st->mass_above, target = st->target;
+    const float run = above0 + inc - (m0 + m1);
+    int found = 64, last = -1;   // order index from the top
+    if (c0) {
+      last = 2 * lane;
+      if (run + m0 >= target) found = 2 * lane;
+    }
+    if (c1) {
+      last = 2 * lane + 1;
+      if (found == 64 && run + m0 + m1 >= target) found = 2 * lane + 1;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      found = min(found, __shfl_xor_sync(0xffffffffu, found, o));
+      last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+    }
+    if (found == 64) found = last;
+    __syncwarp();
+    if (found < 0) {
+      if (lane == 0) {               // a chosen bucket always holds a key
+        st->mode = kSelectAll;
+        set_status(status, RTP_ERR_UNSUPPORTED);
+      }
+      continue;
+    }
+    {
+      const int owner = found >> 1;
+      const bool first = (found & 1) == 0;
+      const int bin = 63 - found;
+      const uint32_t cnt = __shfl_sync(0xffffffffu, first ? c0 : c1, owner);
+      const float above = __shfl_sync(0xffffffffu, first ? run : run + m0, owner);
+      const int shift = st->shift;
+      const uint32_t ofs = (uint32_t)bin << shift;
+      const uint32_t lo_key = st->lo_key + ofs;
+      const uint32_t sub_span = min(1u << shift, st->span - ofs);
+      float rlo, rhi;
+      raw_preimage_warp(d.score_scale, lo_key, lo_key + (sub_span - 1u), lane, rlo, rhi);
+      __syncwarp();
+      if (lane == 0) {
+        st->mass_above = above;
+        st->lo_key = lo_key;
+        st->hi_key = lo_key + (sub_span - 1u);
+        st->span = sub_span;
+        st->bucket_cnt = (int)cnt;
+        st->raw_lo = rlo;
+        st->raw_hi = rhi;
+        st->shift = max(0, shift - 6);
+        if (cnt <= (uint32_t)kCandCap)
+          st->mode = kCollect;
+        else if (sub_span == 1u)
+          st->mode = kTieScan;         // more than kCandCap equal scores straddle the cut
+      }
+      __syncwarp();
+    }
+  }
+  __threadfence();
+  __syncthreads();
   }
 }
 
@@ -364,6 +585,7 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
   __syncwarp();
   const bool emit_ids = sel_idx != nullptr;
   const QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
+  int n_above = 0;   // keys above the bucket seen by this lane
 
   auto row_head = [&](int jj) -> int64_t {
     const int slot2 = (z >> 1) * 8 + (z & 1) * 4 + jj;
@@ -451,6 +673,7 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
         for (int jj = 0; jj < kHeadsPerCta; ++jj)
           if (cstage_cnt[warp][jj] > kCandStage - 16) flush_cands(jj);
       }
+      n_above += __popc(flags);
       if (!emit_ids) continue;
       {
         const int k = __popc(flags);
@@ -476,6 +699,162 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
     flush_cands(jj);
     if (emit_ids) flush_ids(jj);
   }
+  n_above += __shfl_xor_sync(0xffffffffu, n_above, 1);
+  n_above += __shfl_xor_sync(0xffffffffu, n_above, 2);
+  if (st && c == 0 && n_above && mode != kSelectAll) atomicAdd(&st->cnt_above, n_above);
+}
+
+// ---- compaction, at most four heads per index head ----------------------------------------------------------------
+// Every lane handles two scores of head slot (lane >> 2) & 3 (see lane_elems).  Keys above the bucket are counted and,
+// when id lists are requested, emitted; keys inside it become candidates for the exact finish.  Both kinds are rare
+// (a few per cent of the keys): a warp ballots them into per-head stages in shared memory.  The eight lanes of a
+// head keep the fill of its two stages in a register each (equal across those lanes).  The kernel runs for a few
+// microseconds per CTA, so its code is kept small: one 16-key group per loop iteration, flushes out of line.
+struct CompactStages {
+  int ids[kWarps][4][kStage];
+  uint2 cands[kWarps][4][kCandStage];
+};
+
+// Flushes the stages of all four heads of a warp (ids: which = 0, candidates: which = 1); cnt = this lane's head's fill.
+__device__ __noinline__ void flush_stage(CompactStages* sm, int which, int& cnt, int warp, int lane, int64_t row_base,
+                                         const uint8_t* heads, SelState* state, uint2* cand, int32_t* sel_idx,
+                                         int64_t sel_stride, int32_t* status) {
+  __syncwarp();
+#pragma unroll 1
+  for (int j = 0; j < 4; ++j) {
+    const int n = __shfl_sync(0xffffffffu, cnt, 4 * j);
+    if (n == 0) continue;
+    const int64_t rh = row_base + heads[j];
+    int gbase = 0;
+    if (lane == 0) gbase = atomicAdd(which == 0 ? &state[rh].emit_cnt : &state[rh].cand_cnt, n);
+    gbase = __shfl_sync(0xffffffffu, gbase, 0);
+    for (int i = lane; i < n; i += 32) {
+      if (which == 0) {
+        if (gbase + i < sel_stride) sel_idx[rh * sel_stride + gbase + i] = sm->ids[warp][j][i];
+      } else {
+        if (gbase + i < kCandCap) cand[rh * kCandCap + gbase + i] = sm->cands[warp][j][i];
+      }
+    }
+    if (which == 0 && gbase + n > sel_stride && lane == 0) set_status(status, RTP_ERR_CAPACITY);
+  }
+  __syncwarp();
+  cnt = 0;
+}
+
+__global__ void __launch_bounds__(kThreads) sel_compact4_kernel(
+    const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows,
+    const __nv_bfloat16* __restrict__ qt, SelState* __restrict__ state, uint2* __restrict__ cand,
+    int32_t* __restrict__ sel_idx, int64_t sel_stride, int n_splits, int32_t* status) {
+  __shared__ CompactStages sm;
+  __shared__ int s_left[2][kWarps][4];   // [ids / candidates][warp][head]
+  __shared__ int s_base[2][4];
+  const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
+  if (x.p_lo >= x.p_hi) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int slot = (lane >> 2) & 3;
+  const float kInf = __int_as_float(0x7f800000);
+  const int64_t row_base = x.r * d.n_ret;
+  const uint8_t* heads = hm.ih_heads[x.ih];
+  SelState* st = slot < x.nh ? state + (row_base + heads[slot]) : nullptr;
+  const int mode = st ? st->mode : -1;
+  float above = kInf, c_lo = kInf, c_hi = -kInf;   // emit raw > above; candidate raw in [c_lo, c_hi]
+  if (mode == kSelectAll) above = -kInf;
+  if (mode == kCollect || mode == kTieScan) above = st->raw_hi;
+  if (mode == kCollect) {
+    c_lo = st->raw_lo;
+    c_hi = st->raw_hi;
+  }
+  const bool emit_ids = sel_idx != nullptr;
+  const uint32_t lt = (1u << lane) - 1u;
+  const uint32_t mine = 0x000f000fu << (4 * slot);   // the lanes of this lane's head
+  int cnt_i = 0, cnt_c = 0;                          // fill of this head's stages (equal across its lanes)
+  int n_above = 0;
+  const QFrag qf = load_qfrag(qt + row_base * kIndexDim, heads, x.nh, lane);
+
+  // flat loop over the 16-key groups of the warp's pages, the next two groups' keys in flight
+  const int n_it = x.p_lo + warp < x.p_hi ? ((x.p_hi - 1 - (x.p_lo + warp)) / kWarps + 1) * 4 : 0;
+  auto group_ptr = [&](int it) {
+    return ikey_page_ptr(cv, x.seq, x.p_lo + warp + (it >> 2) * kWarps, x.ih) + ((it & 3) * 32 + lane) * 8;
+  };
+  uint4 v1 = make_uint4(0u, 0u, 0u, 0u), v2 = v1;
+  if (n_it > 0) v1 = ld_stream_v4(group_ptr(0));
+  if (n_it > 1) v2 = ld_stream_v4(group_ptr(1));
+#pragma unroll 1
+  for (int it = 0; it < n_it; ++it) {
+    const uint4 v = v1;
+    v1 = v2;
+    if (it + 2 < n_it) v2 = ld_stream_v4(group_ptr(it + 2));
+    const int n_grp = (x.p_lo + warp + (it >> 2) * kWarps) * kPage + (it & 3) * 16;
+    float s_lo[4], s_hi[4];
+    score16(qf, v, lane, s_lo, s_hi);
+    const LaneElems<true> el = lane_elems<true>(s_lo, s_hi, lane);
+    bool fa[2], fc[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const bool ok = n_grp + el.koff[e] < x.n_keys;
+      fa[e] = ok && el.raw[e] > above;
+      fc[e] = ok && el.raw[e] >= c_lo && el.raw[e] <= c_hi;
+    }
+    n_above += (int)fa[0] + (int)fa[1];
+    if (!__any_sync(0xffffffffu, fc[0] || fc[1] || (emit_ids && (fa[0] || fa[1])))) continue;
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int n = n_grp + el.koff[e];
+      const uint32_t mc = __ballot_sync(0xffffffffu, fc[e]) & mine;
+      if (fc[e]) sm.cands[warp][slot][cnt_c + __popc(mc & lt)] = make_uint2(okey(finish_score(el.raw[e], d.score_scale)), (uint32_t)n);
+      cnt_c += __popc(mc);
+      if (emit_ids) {
+        const uint32_t ma = __ballot_sync(0xffffffffu, fa[e]) & mine;
+        if (fa[e]) sm.ids[warp][slot][cnt_i + __popc(ma & lt)] = n;
+        cnt_i += __popc(ma);
+      }
+    }
+    // one group of 16 keys adds at most 16 entries per head
+    if (__any_sync(0xffffffffu, cnt_c > kCandStage - 16))
+      flush_stage(&sm, 1, cnt_c, warp, lane, row_base, heads, state, cand, sel_idx, sel_stride, status);
+    if (__any_sync(0xffffffffu, cnt_i > kStage - 16))
+      flush_stage(&sm, 0, cnt_i, warp, lane, row_base, heads, state, cand, sel_idx, sel_stride, status);
+  }
+
+  // What is left in the stages is written with one counter update per CTA and head (thousands of warps updating the
+  // same few counters one by one would serialise in L2).
+  if ((lane & 19) == 0) {   // lanes 0, 4, 8, 12: one per head
+    s_left[0][warp][slot] = cnt_i;
+    s_left[1][warp][slot] = cnt_c;
+  }
+  __syncthreads();
+  if (threadIdx.x < 8) {
+    const int kind = threadIdx.x >> 2, j = threadIdx.x & 3;
+    int tot = 0;
+    for (int w = 0; w < kWarps; ++w) tot += s_left[kind][w][j];
+    int gbase = 0;
+    if (tot > 0) {
+      SelState* sj = state + (row_base + heads[j]);
+      gbase = atomicAdd(kind == 0 ? &sj->emit_cnt : &sj->cand_cnt, tot);
+      if (kind == 0 && gbase + tot > sel_stride) set_status(status, RTP_ERR_CAPACITY);
+    }
+    s_base[kind][j] = gbase;
+  }
+  __syncthreads();
+#pragma unroll 1
+  for (int j = 0; j < 4; ++j) {
+    const int ni = s_left[0][warp][j], nc = s_left[1][warp][j];
+    if (ni == 0 && nc == 0) continue;
+    const int64_t rh = row_base + heads[j];
+    int off_i = s_base[0][j], off_c = s_base[1][j];
+    for (int w = 0; w < warp; ++w) {
+      off_i += s_left[0][w][j];
+      off_c += s_left[1][w][j];
+    }
+    for (int i = lane; i < ni; i += 32)
+      if (off_i + i < sel_stride) sel_idx[rh * sel_stride + off_i + i] = sm.ids[warp][j][i];
+    for (int i = lane; i < nc; i += 32)
+      if (off_c + i < kCandCap) cand[rh * kCandCap + off_c + i] = sm.cands[warp][j][i];
+  }
+  n_above += __shfl_xor_sync(0xffffffffu, n_above, 1);
+  n_above += __shfl_xor_sync(0xffffffffu, n_above, 2);
+  n_above += __shfl_xor_sync(0xffffffffu, n_above, 16);
+  if (st && lane < 16 && (lane & 3) == 0 && n_above && mode != kSelectAll) atomicAdd(&st->cnt_above, n_above);
 }
 
 // ---- finalize ---------------------------------------------------------------------------------------
@@ -489,11 +868,14 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
     int32_t* __restrict__ sel_idx, int64_t sel_stride, int32_t* __restrict__ sel_count,
     float* __restrict__ sel_mass, float* __restrict__ sel_thresh, int32_t* __restrict__ sel_tie_last,
     int32_t* status) {
-  __shared__ unsigned long long keys[kCandCap];  // 32 KB
+  extern __shared__ __align__(16) unsigned char fin_smem[];
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(fin_smem);       // [kCandCap] candidates
+  unsigned long long* keys2 = keys + kCandCap;                                       // [kCandCap] the other buffer
+  __shared__ uint32_t fh[kBins][3];   // narrowing: {sum, carries, count} per bin
   __shared__ float w_sum[kFinWarps];
   __shared__ int w_cnt[kFinWarps];
-  __shared__ int s_pick, s_emitted, s_last;
-  __shared__ float s_run, s_pick_mass;
+  __shared__ int s_pick, s_emitted, s_last, s_bin, s_n2, s_sel;
+  __shared__ float s_run, s_pick_mass, s_above;
   const int64_t rh = blockIdx.x;
   SelState* st = state + rh;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -520,22 +902,100 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
     }
     return;
   }
-  const float M = st->M, Z = st->Z, target = st->target, above = st->mass_above;
-  const int base = st->cnt_above;
-  const int emit_base = ids ? st->emit_cnt : base;
+  const float M = st->M, Z = st->Z, target = st->target;
+  float above = st->mass_above;
+  int base = st->cnt_above;
+  int emit_base = ids ? st->emit_cnt : base;
 
   if (mode == kCollect) {
-    const int n = min(st->cand_cnt, kCandCap);
+    int n = min(st->cand_cnt, kCandCap);
+    for (int i = tid; i < n; i += kFinThreads) {
+      const uint2 cnd = cand[rh * kCandCap + i];
+      keys[i] = ((unsigned long long)(~cnd.x) << 32) | (unsigned long long)cnd.y;
+    }
+    __syncthreads();
+    // Narrowing: while many candidates are left, one more 64-bin mass histogram over the next six key bits of the
+    // bucket, now on the candidate list in shared memory: candidates above the chosen bin are selected (and their
+    // ids emitted), those below are dropped, those inside go on.  The exact sort below then sees a short list.
+    {
+      uint32_t lo_key = st->lo_key, span = st->span;
+      const float ref_s = st->ref_s, sc = st->e_ref * 9.5367431640625e-07f;   // 2^-20
+      while (n > 256 && span > 1u) {
+        const int bits = 32 - __clz(span - 1u);
+        const int shift = max(0, bits - 6);
+        for (int i = tid; i < kBins * 3; i += kFinThreads) (&fh[0][0])[i] = 0u;
+        if (tid == 0) {
+          s_n2 = 0;
+          s_sel = 0;
+        }
+        __syncthreads();
+        for (int i = tid; i < n; i += kFinThreads) {
+          const uint32_t key = ~(uint32_t)(keys[i] >> 32);
+          uint32_t* acc = &fh[(key - lo_key) >> shift][0];
+          add_mass(acc, fmaf(okey_to_float(key) - ref_s, kLog2eH, 20.0f));
+          atomicAdd(acc + 2, 1u);
+        }
+        __syncthreads();
+        if (warp == 0) {   // lane l looks at bins 63 - 2l, 62 - 2l (bin 63 is the top)
+          const int b0 = 63 - 2 * lane, b1 = 62 - 2 * lane;
+          const float m0 = acc_mass(fh[b0][0], fh[b0][1]) * sc, m1 = acc_mass(fh[b1][0], fh[b1][1]) * sc;
+          const uint32_t c0 = fh[b0][2], c1 = fh[b1][2];
+          float inc = m0 + m1;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const float t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += t;
+          }
+          const float run = above + inc - (m0 + m1);
+          int found = 64, last = -1;
+          if (c0) {
+            last = 2 * lane;
+            if (run + m0 >= target) found = 2 * lane;
+          }
+          if (c1) {
+            last = 2 * lane + 1;
+            if (found == 64 && run + m0 + m1 >= target) found = 2 * lane + 1;
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            found = min(found, __shfl_xor_sync(0xffffffffu, found, o));
+            last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+          }
+          if (found == 64) found = last;
+          if ((found >> 1) == lane) {
+            s_bin = 63 - found;
+            s_above = (found & 1) ? run + m0 : run;
+          }
+        }
+        __syncthreads();
+        const int bin = s_bin;
+        for (int i = tid; i < n; i += kFinThreads) {
+          const unsigned long long k = keys[i];
+          const int b = (int)((~(uint32_t)(k >> 32) - lo_key) >> shift);
+          if (b > bin) {
+            const int pos = atomicAdd(&s_sel, 1);
+            if (ids && emit_base + pos < sel_stride) ids[emit_base + pos] = (int)(uint32_t)k;
+          } else if (b == bin) {
+            keys2[atomicAdd(&s_n2, 1)] = k;
+          }
+        }
+        __syncthreads();
+        above = s_above;
+        base += s_sel;
+        emit_base += s_sel;
+        n = s_n2;
+        const uint32_t ofs = (uint32_t)bin << shift;
+        lo_key += ofs;
+        span = min(1u << shift, span - ofs);
+        unsigned long long* t = keys;
+        keys = keys2;
+        keys2 = t;
+        __syncthreads();
+      }
+    }
     int np = 1;
     while (np < n) np <<= 1;
-    for (int i = tid; i < np; i += kFinThreads) {
-      unsigned long long k = ~0ull;
-      if (i < n) {
-        const uint2 cnd = cand[rh * kCandCap + i];
-        k = ((unsigned long long)(~cnd.x) << 32) | (unsigned long long)cnd.y;
-      }
-      keys[i] = k;
-    }
+    for (int i = n + tid; i < np; i += kFinThreads) keys[i] = ~0ull;
     if (tid == 0) {
       s_pick = kNoPick;
       s_run = 0.f;
@@ -712,12 +1172,15 @@ int select_splits(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
 
 struct SelWorkspace {
   SelState* state;
-  Bin* hist;
+  unsigned long long* g_mass;   // [row heads][64] merged bin sums
+  uint32_t* g_cnt;              // [row heads][64] merged bin counts
+  uint32_t* tickets;            // [rows * index heads]
   uint2* cand;
+  size_t zero_off, zero_bytes;  // the part that must be zero before the first pass
   size_t bytes;
 };
 
-SelWorkspace carve(void* ws, int64_t n_rowheads) {
+SelWorkspace carve(void* ws, int64_t n_rowheads, int64_t n_units) {
   SelWorkspace w;
   size_t off = 0;
   auto take = [&](size_t n) {
@@ -726,21 +1189,44 @@ SelWorkspace carve(void* ws, int64_t n_rowheads) {
     return o;
   };
   const size_t o_state = take(sizeof(SelState) * n_rowheads);
-  const size_t o_hist = take(sizeof(Bin) * kSelBins * n_rowheads);
+  const size_t o_mass = take(sizeof(unsigned long long) * kBins * n_rowheads);
+  const size_t o_cnt = take(sizeof(uint32_t) * kBins * n_rowheads);
+  const size_t o_tick = take(sizeof(uint32_t) * n_units);
   const size_t o_cand = take(sizeof(uint2) * kCandCap * n_rowheads);
   char* b = reinterpret_cast<char*>(ws);
   w.state = reinterpret_cast<SelState*>(b + o_state);
-  w.hist = reinterpret_cast<Bin*>(b + o_hist);
+  w.g_mass = reinterpret_cast<unsigned long long*>(b + o_mass);
+  w.g_cnt = reinterpret_cast<uint32_t*>(b + o_cnt);
+  w.tickets = reinterpret_cast<uint32_t*>(b + o_tick);
   w.cand = reinterpret_cast<uint2*>(b + o_cand);
+  w.zero_off = o_mass;
+  w.zero_bytes = o_cand - o_mass;
   w.bytes = off;
   return w;
+}
+
+constexpr int kKeyLevels = 6;   // 6 bits each: a level-1 bucket spans fewer than 2^32 key values
+
+template <bool NH4>
+cudaError_t launch_passes(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                          const __nv_bfloat16* qt, const SelWorkspace& w, int n_splits, int32_t* status,
+                          cudaStream_t st) {
+  dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
+  sel_max_kernel<NH4><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, n_splits, status);
+  sel_l1_kernel<NH4><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.g_mass, w.tickets, n_splits, status);
+  sel_key_kernel<NH4><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.g_mass, w.g_cnt, w.tickets, n_splits, 1,
+                                                 status);
+  // whatever is still unresolved (rare: dense clusters of nearly equal scores) is finished by one CTA per unit
+  sel_key_kernel<NH4><<<dim3(grid.x, 1), kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.g_mass, w.g_cnt, w.tickets, 1,
+                                                            kKeyLevels, status);
+  return cudaGetLastError();
 }
 
 }  // namespace
 
 size_t select_rows_workspace_bytes(const Dims& d, int64_t R) {
   if (R <= 0 || d.n_ret <= 0) return 0;
-  return carve(nullptr, R * d.n_ret).bytes;
+  return carve(nullptr, R * d.n_ret, R * d.n_ih).bytes;
 }
 
 cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
@@ -749,28 +1235,33 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
                                int32_t* status, void* ws, int sm_count, cudaStream_t st) {
   if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
   const int64_t nrh = rows.R * d.n_ret;
-  const SelWorkspace w = carve(ws, nrh);
-  cudaError_t e = cudaMemsetAsync(w.hist, 0, sizeof(Bin) * kSelBins * nrh, st);
+  const SelWorkspace w = carve(ws, nrh, rows.R * d.n_ih);
+  cudaError_t e = cudaMemsetAsync(reinterpret_cast<char*>(ws) + w.zero_off, 0, w.zero_bytes, st);
   if (e != cudaSuccess) return e;
   sel_init_kernel<<<(unsigned)((nrh + 127) / 128), 128, 0, st>>>(cv, d, rows, w.state, nrh);
   int max_nh = 0;
   for (int i = 0; i < d.n_ih; ++i) max_nh = hm.ih_nheads[i] > max_nh ? hm.ih_nheads[i] : max_nh;
   const int n_splits = select_splits(d, rows.R, max_len, sm_count);
-  dim3 grid((unsigned)(rows.R * d.n_ih), n_splits, (max_nh + kHeadsPerCta - 1) / kHeadsPerCta);
-  const size_t hist_smem = (size_t)kHeadsPerCta * kSelBins * 8;
-  static bool attr_done = false;
-  if (!attr_done) {
-    e = cudaFuncSetAttribute(sel_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hist_smem);
+  e = max_nh <= 4 ? launch_passes<true>(cv, d, hm, rows, qt, w, n_splits, status, st)
+                  : launch_passes<false>(cv, d, hm, rows, qt, w, n_splits, status, st);
+  if (e != cudaSuccess) return e;
+  if (max_nh <= 4) {
+    dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
+    sel_compact4_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.cand, sel_idx, sel_stride, n_splits,
+                                                   status);
+  } else {
+    dim3 grid((unsigned)(rows.R * d.n_ih), n_splits, (max_nh + kHeadsPerCta - 1) / kHeadsPerCta);
+    sel_compact_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.cand, sel_idx, sel_stride, n_splits,
+                                                  status);
+  }
+  constexpr int kFinSmem = 2 * kCandCap * 8;
+  static bool fin_attr_done = false;
+  if (!fin_attr_done) {
+    e = cudaFuncSetAttribute(sel_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinSmem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    fin_attr_done = true;
   }
-  for (int it = 0; it < 4; ++it) {
-    sel_hist_kernel<<<grid, kThreads, hist_smem, st>>>(cv, d, hm, rows, qt, w.state, w.hist, n_splits, status);
-    sel_resolve_kernel<<<(unsigned)nrh, kResThreads, 0, st>>>(d, w.state, w.hist);
-  }
-  sel_compact_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.cand, sel_idx, sel_stride,
-                                                n_splits, status);
-  sel_finalize_kernel<<<(unsigned)nrh, kFinThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.cand, sel_idx,
+  sel_finalize_kernel<<<(unsigned)nrh, kFinThreads, kFinSmem, st>>>(cv, d, hm, rows, qt, w.state, w.cand, sel_idx,
                                                              sel_stride, sel_count, sel_mass, sel_thresh,
                                                              sel_tie_last, status);
   return cudaGetLastError();
