@@ -61,6 +61,12 @@ def test_config2_reduced_with_ragged_batch():
     _run_decode(wl, dense_heads=(0, 5))
 
 
+def test_group_of_eight_query_heads_per_kv_head():
+    """G = 8: eight retrieval heads share one index head (the selection kernels' path for more than four heads)."""
+    wl = synth.config_2(L=2600, batch=2, n_q_heads=16, n_kv_heads=2, ret_kv_heads=(0,), window=300)
+    _run_decode(wl, dense_heads=(0,))
+
+
 def test_config2_full_size():
     wl = synth.config_2()
     dw, stats = _run_decode(wl, dense_heads=(1,))
