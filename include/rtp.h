@@ -183,9 +183,12 @@ rtp_status rtp_index_score(rtp_ctx* ctx, const rtp_params* params, const rtp_cac
  *              RTP_ERR_CAPACITY is recorded in *status)
  * sel_mass     DEVICE fp32  [R, n_ret_q_heads] softmax mass of the set (fp32 estimate)
  * sel_thresh   DEVICE fp32  [R, n_ret_q_heads] smallest selected score
- * sel_tie_last DEVICE int32 [R, n_ret_q_heads] largest selected position among
- *              keys whose score equals sel_thresh; a key n belongs to the set
- *              iff s > thresh or (s == thresh and n <= tie_last)
+ * sel_tie_last DEVICE int32 [R, n_ret_q_heads] position bound for keys whose score
+ *              equals sel_thresh: a key n belongs to the set iff s > thresh or
+ *              (s == thresh and n <= tie_last).  Any value from the largest selected
+ *              tied position up to (excluding) the smallest tied position left out
+ *              describes the same set; the row's last position is returned when no
+ *              tied key is left out.
  * status       DEVICE int32 [1] */
 rtp_status rtp_topp_select(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
                            const void* q_pre, const void* w_q, const int32_t* row_seq,

@@ -461,8 +461,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             }
           }
         } else {
-          // general rule (diagonal tiles, tiles that hold a row's tie position): key n of the tile belongs to the
-          // row's set iff n <= position and raw >= (n <= tie position ? lo : upn)
+          // general rule (diagonal tiles; tiles that hold the tie position of a row with tied keys left out): key n of
+          // the tile belongs to the row's set iff n <= position and raw >= (n <= tie position ? lo : upn).  Rare, so
+          // the loop stays rolled (small code): the 8-key group's fragment is picked from the registers by a switch-free
+          // select chain.
           float lo_k[4], upn_k[4];
           int tie_rel[4], pos_rel[4];   // relative to the lane's first column of the tile
 #pragma unroll
@@ -473,12 +475,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
             tie_rel[k] = thr_tie[rowk] - n_base - 2 * cq;
             pos_rel[k] = m0 + rowk % BMP - n_base - 2 * cq;
           }
-#pragma unroll
+#pragma unroll 1
           for (int nt = 0; nt < 16; ++nt) {
+            uint2 b = kb[0];
+#pragma unroll
+            for (int x = 1; x < 16; ++x)
+              if (nt == x) b = kb[x];
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
               float s4[4];
-              mma_bf16_16816(s4, iqa[t][0], iqa[t][1], iqa[t][2], iqa[t][3], kb[nt].x, kb[nt].y, zero);
+              mma_bf16_16816(s4, iqa[t][0], iqa[t][1], iqa[t][2], iqa[t][3], b.x, b.y, zero);
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
                 const int k = 2 * t + (e >> 1);

@@ -687,13 +687,17 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
             thr_key = max(thr_key, __shfl_xor_sync(0xffffffffu, thr_key, o));
             pick_cum = fmaxf(pick_cum, __shfl_xor_sync(0xffffffffu, pick_cum, o));
           }
-          int tie_last = -1;
+          // Position bound for keys that tie with the threshold score: the last one taken, or the row's last key
+          // when none is left out (the usual case: then the attention kernel never has to look at positions).
+          int tie_last = -1, left_out = 0;
 #pragma unroll
           for (int x = 0; x < 2; ++x)
-            if (2 * lane + x < n_c && rank[x] <= pick && ~(uint32_t)(ord[x] >> 32) == thr_key)
-              tie_last = max(tie_last, (int)(uint32_t)ord[x]);
+            if (2 * lane + x < n_c && ~(uint32_t)(ord[x] >> 32) == thr_key) {
+              if (rank[x] <= pick) tie_last = max(tie_last, (int)(uint32_t)ord[x]); else left_out = 1;
+            }
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) tie_last = max(tie_last, __shfl_xor_sync(0xffffffffu, tie_last, o));
+          if (!__any_sync(0xffffffffu, left_out)) tie_last = R.n_keys - 1;
           if (lane == 0) {
             S->cnt_above = above;
             S->thr_key = thr_key;
