@@ -220,8 +220,9 @@ __device__ __forceinline__ void page_late(const unsigned char* pg, const QFrag& 
 }
 
 // Works off the warp's queue of bucket hits: entry = {position | local row << 27, raw score bits}.
-__device__ __noinline__ void drain_hits(uint32_t* wq, int& qcnt, int lane, int wrow, RowState* rs, uint32_t* hist,
-                                           float scale) {
+// (The count is passed by value: a reference would pin the caller's counter to local memory.)
+__device__ __noinline__ void drain_hits(uint32_t* wq, int qcnt, int lane, int wrow, RowState* rs, uint32_t* hist,
+                                        float scale) {
   constexpr int kRowWords = kRowBytes / 4;
   __syncwarp();
   for (int base = 0; base < qcnt; base += 32) {
@@ -247,7 +248,6 @@ __device__ __noinline__ void drain_hits(uint32_t* wq, int& qcnt, int lane, int w
     }
   }
   __syncwarp();
-  qcnt = 0;
 }
 
 // Key levels and candidate collection without ties: hits go to the warp's queue.
@@ -292,7 +292,10 @@ __device__ __forceinline__ void page_hits(const unsigned char* pg, const QFrag& 
           qcnt += __popc(m);
         }
       }
-      if (qcnt >= 32) drain_hits(wq, qcnt, lane, wrow, rs, hist, scale);   // at most 31 + 128 entries queued
+      if (qcnt >= 32) {   // at most 31 + 128 entries queued
+        drain_hits(wq, qcnt, lane, wrow, rs, hist, scale);
+        qcnt = 0;
+      }
     }
   }
 }
@@ -480,6 +483,7 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     if (qcnt > 0) drain_hits(wq, qcnt, lane, wrow, rs, hist, scale);
+    qcnt = 0;
 
     // ---- end of pass: combine the quad's partial results ----
     mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));

@@ -350,7 +350,8 @@ struct KeyParams {   // per head slot, shared memory
   float ref_s;
 };
 
-__device__ __noinline__ void drain_row_hits(uint32_t* wq, int& qcnt, int lane, const KeyParams* kp,
+// (the count is passed by value: a reference would pin the caller's counter to local memory)
+__device__ __noinline__ void drain_row_hits(uint32_t* wq, int qcnt, int lane, const KeyParams* kp,
                                             uint32_t (*hist)[kBins][3], float scale) {
   __syncwarp();
   for (int base = 0; base < qcnt; base += 32) {
@@ -365,7 +366,6 @@ __device__ __noinline__ void drain_row_hits(uint32_t* wq, int& qcnt, int lane, c
     }
   }
   __syncwarp();
-  qcnt = 0;
 }
 
 template <bool NH4>
@@ -453,11 +453,15 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
           qcnt += __popc(m);
         }
         if ((e & 3) == 3 || e == LaneElems<NH4>::kN - 1)
-          if (qcnt >= 32) drain_row_hits(wq, qcnt, lane, kp, hist, d.score_scale);
+          if (qcnt >= 32) {
+            drain_row_hits(wq, qcnt, lane, kp, hist, d.score_scale);
+            qcnt = 0;
+          }
       }
     }
   }
   if (qcnt > 0) drain_row_hits(wq, qcnt, lane, kp, hist, d.score_scale);
+  qcnt = 0;
   __syncthreads();
   for (int i = threadIdx.x; i < x.nh * kBins; i += kThreads) {
     const int j = i / kBins, bin = i % kBins;
@@ -716,15 +720,17 @@ struct CompactStages {
 };
 
 // Flushes the stages of all four heads of a warp (ids: which = 0, candidates: which = 1); cnt = this lane's head's fill.
-__device__ __noinline__ void flush_stage(CompactStages* sm, int which, int& cnt, int warp, int lane, int64_t row_base,
-                                         const uint8_t* heads, SelState* state, uint2* cand, int32_t* sel_idx,
+// (cnt is passed by value: a reference would pin the caller's counter to local memory)
+// heads4 = the retrieval-head indices of the four slots, one byte each.
+__device__ __noinline__ void flush_stage(CompactStages* sm, int which, int cnt, int warp, int lane, int64_t row_base,
+                                         uint32_t heads4, SelState* state, uint2* cand, int32_t* sel_idx,
                                          int64_t sel_stride, int32_t* status) {
   __syncwarp();
 #pragma unroll 1
   for (int j = 0; j < 4; ++j) {
     const int n = __shfl_sync(0xffffffffu, cnt, 4 * j);
     if (n == 0) continue;
-    const int64_t rh = row_base + heads[j];
+    const int64_t rh = row_base + ((heads4 >> (8 * j)) & 0xffu);
     int gbase = 0;
     if (lane == 0) gbase = atomicAdd(which == 0 ? &state[rh].emit_cnt : &state[rh].cand_cnt, n);
     gbase = __shfl_sync(0xffffffffu, gbase, 0);
@@ -738,7 +744,6 @@ __device__ __noinline__ void flush_stage(CompactStages* sm, int which, int& cnt,
     if (which == 0 && gbase + n > sel_stride && lane == 0) set_status(status, RTP_ERR_CAPACITY);
   }
   __syncwarp();
-  cnt = 0;
 }
 
 __global__ void __launch_bounds__(kThreads) sel_compact4_kernel(
@@ -754,8 +759,10 @@ __global__ void __launch_bounds__(kThreads) sel_compact4_kernel(
   const int slot = (lane >> 2) & 3;
   const float kInf = __int_as_float(0x7f800000);
   const int64_t row_base = x.r * d.n_ret;
-  const uint8_t* heads = hm.ih_heads[x.ih];
-  SelState* st = slot < x.nh ? state + (row_base + heads[slot]) : nullptr;
+  // (kernel parameters are only ever read by value: a pointer into them would force a copy of the struct to local memory)
+  const uint32_t heads4 = (uint32_t)hm.ih_heads[x.ih][0] | ((uint32_t)hm.ih_heads[x.ih][1] << 8) |
+                          ((uint32_t)hm.ih_heads[x.ih][2] << 16) | ((uint32_t)hm.ih_heads[x.ih][3] << 24);
+  SelState* st = slot < x.nh ? state + (row_base + ((heads4 >> (8 * slot)) & 0xffu)) : nullptr;
   const int mode = st ? st->mode : -1;
   float above = kInf, c_lo = kInf, c_hi = -kInf;   // emit raw > above; candidate raw in [c_lo, c_hi]
   if (mode == kSelectAll) above = -kInf;
@@ -769,7 +776,7 @@ __global__ void __launch_bounds__(kThreads) sel_compact4_kernel(
   const uint32_t mine = 0x000f000fu << (4 * slot);   // the lanes of this lane's head
   int cnt_i = 0, cnt_c = 0;                          // fill of this head's stages (equal across its lanes)
   int n_above = 0;
-  const QFrag qf = load_qfrag(qt + row_base * kIndexDim, heads, x.nh, lane);
+  const QFrag qf = load_qfrag(qt + row_base * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
 
   // flat loop over the 16-key groups of the warp's pages, the next two groups' keys in flight
   const int n_it = x.p_lo + warp < x.p_hi ? ((x.p_hi - 1 - (x.p_lo + warp)) / kWarps + 1) * 4 : 0;
@@ -810,10 +817,14 @@ __global__ void __launch_bounds__(kThreads) sel_compact4_kernel(
       }
     }
     // one group of 16 keys adds at most 16 entries per head
-    if (__any_sync(0xffffffffu, cnt_c > kCandStage - 16))
-      flush_stage(&sm, 1, cnt_c, warp, lane, row_base, heads, state, cand, sel_idx, sel_stride, status);
-    if (__any_sync(0xffffffffu, cnt_i > kStage - 16))
-      flush_stage(&sm, 0, cnt_i, warp, lane, row_base, heads, state, cand, sel_idx, sel_stride, status);
+    if (__any_sync(0xffffffffu, cnt_c > kCandStage - 16)) {
+      flush_stage(&sm, 1, cnt_c, warp, lane, row_base, heads4, state, cand, sel_idx, sel_stride, status);
+      cnt_c = 0;
+    }
+    if (__any_sync(0xffffffffu, cnt_i > kStage - 16)) {
+      flush_stage(&sm, 0, cnt_i, warp, lane, row_base, heads4, state, cand, sel_idx, sel_stride, status);
+      cnt_i = 0;
+    }
   }
 
   // What is left in the stages is written with one counter update per CTA and head (thousands of warps updating the
@@ -829,7 +840,7 @@ __global__ void __launch_bounds__(kThreads) sel_compact4_kernel(
     for (int w = 0; w < kWarps; ++w) tot += s_left[kind][w][j];
     int gbase = 0;
     if (tot > 0) {
-      SelState* sj = state + (row_base + heads[j]);
+      SelState* sj = state + (row_base + ((heads4 >> (8 * j)) & 0xffu));
       gbase = atomicAdd(kind == 0 ? &sj->emit_cnt : &sj->cand_cnt, tot);
       if (kind == 0 && gbase + tot > sel_stride) set_status(status, RTP_ERR_CAPACITY);
     }
@@ -840,7 +851,7 @@ __global__ void __launch_bounds__(kThreads) sel_compact4_kernel(
   for (int j = 0; j < 4; ++j) {
     const int ni = s_left[0][warp][j], nc = s_left[1][warp][j];
     if (ni == 0 && nc == 0) continue;
-    const int64_t rh = row_base + heads[j];
+    const int64_t rh = row_base + ((heads4 >> (8 * j)) & 0xffu);
     int off_i = s_base[0][j], off_c = s_base[1][j];
     for (int w = 0; w < warp; ++w) {
       off_i += s_left[0][w][j];
