@@ -336,22 +336,51 @@ def main():
         h_k[s:e].copy_(data.k_pages[phys].permute(0, 2, 1, 3).reshape(-1, Hkv, 128)[: e - s])
         h_v[s:e].copy_(data.v_pages[phys].permute(0, 2, 1, 3).reshape(-1, Hkv, 128)[: e - s])
     h_out = torch.empty((L, Hq, 128), dtype=torch.bfloat16).pin_memory()
-    d_q = torch.empty((chunk, Hq, 128), dtype=torch.bfloat16, device=device)
-    d_kpre = torch.empty((chunk, nih, 128), dtype=torch.bfloat16, device=device)
-    d_k = torch.empty((chunk, Hkv, 128), dtype=torch.bfloat16, device=device)
-    d_v = torch.empty((chunk, Hkv, 128), dtype=torch.bfloat16, device=device)
-    d_out = torch.empty((chunk, Hq, 128), dtype=torch.bfloat16, device=device)
+
+    # Two sets of device staging buffers and a copy stream: the H2D copies of chunk i+1 and the D2H copy of chunk
+    # i-1 overlap the kernels of chunk i (events order the hand-offs; everything ends on the compute stream).
+    copy_stream = torch.cuda.Stream(device=device)
+    stage = [dict(q=torch.empty((chunk, Hq, 128), dtype=torch.bfloat16, device=device),
+                  kpre=torch.empty((chunk, nih, 128), dtype=torch.bfloat16, device=device),
+                  k=torch.empty((chunk, Hkv, 128), dtype=torch.bfloat16, device=device),
+                  v=torch.empty((chunk, Hkv, 128), dtype=torch.bfloat16, device=device),
+                  out=torch.empty((chunk, Hq, 128), dtype=torch.bfloat16, device=device),
+                  loaded=torch.cuda.Event(), computed=torch.cuda.Event(), drained=torch.cuda.Event()) for _ in range(2)]
 
     def step_e2e():
-        for (s, C) in chunks:
-            d_q[:C].copy_(h_q[s:s + C], non_blocking=True)
-            d_kpre[:C].copy_(h_kpre[s:s + C], non_blocking=True)
-            d_k[:C].copy_(h_k[s:s + C], non_blocking=True)
-            d_v[:C].copy_(h_v[s:s + C], non_blocking=True)
-            rb.rtp_kv_append(path.ctx, path.params, path.cache, d_k[:C], d_v[:C], path.tok_seq[:C],
+        copy_stream.wait_stream(stream)
+        for b in stage:
+            b["drained"].record(copy_stream)
+
+        def load(i):
+            s, C = chunks[i]
+            b = stage[i & 1]
+            with torch.cuda.stream(copy_stream):
+                copy_stream.wait_event(b["computed"])     # the previous user of this buffer set has finished computing
+                b["q"][:C].copy_(h_q[s:s + C], non_blocking=True)
+                b["kpre"][:C].copy_(h_kpre[s:s + C], non_blocking=True)
+                b["k"][:C].copy_(h_k[s:s + C], non_blocking=True)
+                b["v"][:C].copy_(h_v[s:s + C], non_blocking=True)
+                b["loaded"].record(copy_stream)
+
+        for b in stage:
+            b["computed"].record(stream)
+        load(0)
+        for i, (s, C) in enumerate(chunks):
+            b = stage[i & 1]
+            if i + 1 < len(chunks):
+                load(i + 1)
+            stream.wait_event(b["loaded"])
+            stream.wait_event(b["drained"])               # the output buffer of this set has been copied out
+            rb.rtp_kv_append(path.ctx, path.params, path.cache, b["k"][:C], b["v"][:C], path.tok_seq[:C],
                              path.pos_all[s:s + C], path.status)
-            path.run_chunk(s, C, d_q[:C], d_kpre[:C], d_out[:C])
-            h_out[s:s + C].copy_(d_out[:C], non_blocking=True)
+            path.run_chunk(s, C, b["q"][:C], b["kpre"][:C], b["out"][:C])
+            b["computed"].record(stream)
+            with torch.cuda.stream(copy_stream):
+                copy_stream.wait_event(b["computed"])
+                h_out[s:s + C].copy_(b["out"][:C], non_blocking=True)
+                b["drained"].record(copy_stream)
+        stream.wait_stream(copy_stream)
 
     step_e2e()
     barrier()
@@ -368,6 +397,11 @@ def main():
         ms_e2e = float(t.item())
     h2d = int(L * (Hq + 2 * Hkv + nih) * 128 * 2)
     d2h = int(L * Hq * 128 * 2)
+    torch.cuda.synchronize()
+    s_chk, C_chk = chunks[-1]
+    step()                                                  # resident outputs for the comparison below
+    torch.cuda.synchronize()
+    e2e_ok = bool(torch.equal(h_out[s_chk:s_chk + C_chk].to(device), out[s_chk:s_chk + C_chk]))
     del h_q, h_k, h_v, h_kpre, h_out
 
     # ---- per-kernel timing of one instrumented step (not part of the timed region) ----
@@ -418,7 +452,9 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config, "clocks": clocks,
             "e2e": {"value": world * L / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e,
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "overlap": "two staging buffer sets, copies on a second stream",
+                    "last_chunk_equals_resident_run": e2e_ok},
             "gpu_launches": args.steps * len(chunks) * path.launches_per_chunk,
             "roofline": roofline, "device_status": status,
             "selected_fraction_last_chunk": sel_frac,
