@@ -103,36 +103,53 @@ __global__ void __launch_bounds__(kThreads) attn_rows_kernel(
   }
   const int64_t bt_base = (int64_t)seq * cv.max_pages;
 
-  for (int tb = t_lo + warp * 2; tb < t_hi; tb += kStreams * kUnroll) {
-    uint4 kr[kUnroll], vr[kUnroll];
-    bool ok[kUnroll];
+  // Where the rows of a batch of tokens live (list entry -> block table -> offset) is resolved one batch ahead, so
+  // that these two dependent loads are in flight together with the K / V rows of the current batch.
+  int64_t off_n[kUnroll];
+  bool ok_n[kUnroll];
+  auto resolve = [&](int tb) {
 #pragma unroll
     for (int x = 0; x < kUnroll; ++x) {
       const int t = tb + hw + x * kStreams;
-      ok[x] = t < t_hi;
-      kr[x] = make_uint4(0, 0, 0, 0);
-      vr[x] = make_uint4(0, 0, 0, 0);
-      if (ok[x]) {
+      ok_n[x] = t < t_hi;
+      off_n[x] = 0;
+      if (ok_n[x]) {
         int tok;
         if (SET == kSetList) {
           tok = __ldg(ids + t);
           if (tok < 0 || tok >= n_keys) {
             set_status(status, RTP_ERR_INVALID);
-            ok[x] = false;
+            ok_n[x] = false;
           }
         } else if (SET == kSetLocal) {
           tok = t < ns ? t : wlo + (t - ns);
         } else {
           tok = t;
         }
-        if (ok[x]) {
+        if (ok_n[x]) {
           const int phys = __ldg(cv.block_table + bt_base + (tok >> kPageShift));
-          const int64_t off = (((int64_t)phys * cv.n_kv + kvh) * kPage + (tok & (kPage - 1))) * kHeadDim + l16 * 8;
-          kr[x] = ld_stream_v4(cv.k + off);
-          vr[x] = ld_stream_v4(cv.v + off);
+          off_n[x] = (((int64_t)phys * cv.n_kv + kvh) * kPage + (tok & (kPage - 1))) * kHeadDim + l16 * 8;
         }
       }
     }
+  };
+  // (only lists have the extra dependent load; the other sets resolve in place and keep their register count)
+  if (SET == kSetList) resolve(t_lo + warp * 2);
+  for (int tb = t_lo + warp * 2; tb < t_hi; tb += kStreams * kUnroll) {
+    if (SET != kSetList) resolve(tb);
+    uint4 kr[kUnroll], vr[kUnroll];
+    bool ok[kUnroll];
+#pragma unroll
+    for (int x = 0; x < kUnroll; ++x) {
+      ok[x] = ok_n[x];
+      kr[x] = make_uint4(0, 0, 0, 0);
+      vr[x] = make_uint4(0, 0, 0, 0);
+      if (ok[x]) {
+        kr[x] = ld_stream_v4(cv.k + off_n[x]);
+        vr[x] = ld_stream_v4(cv.v + off_n[x]);
+      }
+    }
+    if (SET == kSetList) resolve(tb + kStreams * kUnroll);
     float logit[kUnroll][G];
 #pragma unroll
     for (int x = 0; x < kUnroll; ++x) {
