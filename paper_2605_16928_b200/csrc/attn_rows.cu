@@ -29,7 +29,7 @@ __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
 }
 
 template <int G, int SET>
-__global__ void __launch_bounds__(kThreads) attn_rows_kernel(
+__global__ void __launch_bounds__(kThreads, (G == 1) ? 6 : 1) attn_rows_kernel(
     const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows, const int n_units,
     const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ sel_idx, const int64_t sel_stride,
     const int32_t* __restrict__ sel_count, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
