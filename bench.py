@@ -124,8 +124,9 @@ def prefill_tile_flops(L: int, chunk: int, group: int, n_kv_heads: int, mode: st
 def bench_prefill(args, rank, world, device):
     import torch
     from paper_2605_16928_b200 import synth_device, pipeline
-    L, chunk = args.seq_len or 131072, args.chunk or 8192
-    data = synth_device.config_3_device(L=L, device=device)
+    c4 = args.workload == "c4"
+    L, chunk = args.seq_len or (1048576 if c4 else 131072), args.chunk or (16384 if c4 else 8192)
+    data = synth_device.config_3_device(L=L, device=device, ret_kv_heads=(0,) if c4 else (0, 1))
     path = pipeline.PrefillPath(data, chunk)
     stream = torch.cuda.current_stream()
     out = torch.empty((L, path.Hq, 128), dtype=torch.bfloat16, device=device)
@@ -221,6 +222,9 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=["c3", "c4"],
+                    help="c3: 128K chunked prefill, 2 retrieval KV heads (default, the bench line); "
+                         "c4: 1M prefill, chunk 16K, 1 retrieval KV head (long run, no end-to-end leg)")
     ap.add_argument("--seq-len", type=int, default=0)
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the dense baseline, decode points and CPU oracle")
@@ -234,9 +238,11 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     n_cores = len(os.sched_getaffinity(0))
-    L, chunk = args.seq_len or 131072, args.chunk or 8192
-    config = {"workload": "c3_chunked_prefill_128k" if L == 131072 else f"c3_chunked_prefill_{L}",
-              "seq_len": L, "chunk": chunk, "n_q_heads": 32, "n_kv_heads": 8, "retrieval_kv_heads": 2,
+    c4 = args.workload == "c4"
+    L, chunk = args.seq_len or (1048576 if c4 else 131072), args.chunk or (16384 if c4 else 8192)
+    config = {"workload": (f"c4_long_prefill_{L}" if c4 else
+                           "c3_chunked_prefill_128k" if L == 131072 else f"c3_chunked_prefill_{L}"),
+              "seq_len": L, "chunk": chunk, "n_q_heads": 32, "n_kv_heads": 8, "retrieval_kv_heads": 1 if c4 else 2,
               "index_dim": 16, "top_p": 0.9, "n_sink": 4, "window": 8192, "page_size": 64,
               "l2": "inputs_larger_than_l2", "parallelism": "replicas" if world > 1 else "single_gpu"}
 
@@ -321,88 +327,96 @@ def main():
     status = path.status_code()
     sel_frac = float((path.sel_cnt.float() / (path.pos_all[L - len(path.sel_cnt):].float()[:, None] + 1)).mean().item())
 
-    # ---- end to end: pinned host buffers, H2D of the chunk's q / k / v / k_pre, D2H of its output ----
     from paper_2605_16928_b200 import binding as rb
     Hq, Hkv, nih = path.Hq, data.heads.n_kv_heads, data.heads.n_index_heads
-    h_q = torch.empty((L, Hq, 128), dtype=torch.bfloat16).pin_memory()
-    h_q.copy_(data.q)
-    h_kpre = torch.empty((L, nih, 128), dtype=torch.bfloat16).pin_memory()
-    h_kpre.copy_(k_pre)
-    h_k = torch.empty((L, Hkv, 128), dtype=torch.bfloat16).pin_memory()
-    h_v = torch.empty((L, Hkv, 128), dtype=torch.bfloat16).pin_memory()
-    for s in range(0, L, 16384):
-        e = min(L, s + 16384)
-        phys = data.block_table[0, s // 64:(e + 63) // 64].long()
-        h_k[s:e].copy_(data.k_pages[phys].permute(0, 2, 1, 3).reshape(-1, Hkv, 128)[: e - s])
-        h_v[s:e].copy_(data.v_pages[phys].permute(0, 2, 1, 3).reshape(-1, Hkv, 128)[: e - s])
-    h_out = torch.empty((L, Hq, 128), dtype=torch.bfloat16).pin_memory()
 
-    # Two sets of device staging buffers and a copy stream: the H2D copies of chunk i+1 and the D2H copy of chunk
-    # i-1 overlap the kernels of chunk i (events order the hand-offs; everything ends on the compute stream).
-    copy_stream = torch.cuda.Stream(device=device)
-    stage = [dict(q=torch.empty((chunk, Hq, 128), dtype=torch.bfloat16, device=device),
-                  kpre=torch.empty((chunk, nih, 128), dtype=torch.bfloat16, device=device),
-                  k=torch.empty((chunk, Hkv, 128), dtype=torch.bfloat16, device=device),
-                  v=torch.empty((chunk, Hkv, 128), dtype=torch.bfloat16, device=device),
-                  out=torch.empty((chunk, Hq, 128), dtype=torch.bfloat16, device=device),
-                  loaded=torch.cuda.Event(), computed=torch.cuda.Event(), drained=torch.cuda.Event()) for _ in range(2)]
+    def run_e2e():
+        # ---- end to end: pinned host buffers, H2D of the chunk's q / k / v / k_pre, D2H of its output ----
+        h_q = torch.empty((L, Hq, 128), dtype=torch.bfloat16).pin_memory()
+        h_q.copy_(data.q)
+        h_kpre = torch.empty((L, nih, 128), dtype=torch.bfloat16).pin_memory()
+        h_kpre.copy_(k_pre)
+        h_k = torch.empty((L, Hkv, 128), dtype=torch.bfloat16).pin_memory()
+        h_v = torch.empty((L, Hkv, 128), dtype=torch.bfloat16).pin_memory()
+        for s in range(0, L, 16384):
+            e = min(L, s + 16384)
+            phys = data.block_table[0, s // 64:(e + 63) // 64].long()
+            h_k[s:e].copy_(data.k_pages[phys].permute(0, 2, 1, 3).reshape(-1, Hkv, 128)[: e - s])
+            h_v[s:e].copy_(data.v_pages[phys].permute(0, 2, 1, 3).reshape(-1, Hkv, 128)[: e - s])
+        h_out = torch.empty((L, Hq, 128), dtype=torch.bfloat16).pin_memory()
 
-    def step_e2e():
-        copy_stream.wait_stream(stream)
-        for b in stage:
-            b["drained"].record(copy_stream)
+        # Two sets of device staging buffers and a copy stream: the H2D copies of chunk i+1 and the D2H copy of chunk
+        # i-1 overlap the kernels of chunk i (events order the hand-offs; everything ends on the compute stream).
+        copy_stream = torch.cuda.Stream(device=device)
+        stage = [dict(q=torch.empty((chunk, Hq, 128), dtype=torch.bfloat16, device=device),
+                      kpre=torch.empty((chunk, nih, 128), dtype=torch.bfloat16, device=device),
+                      k=torch.empty((chunk, Hkv, 128), dtype=torch.bfloat16, device=device),
+                      v=torch.empty((chunk, Hkv, 128), dtype=torch.bfloat16, device=device),
+                      out=torch.empty((chunk, Hq, 128), dtype=torch.bfloat16, device=device),
+                      loaded=torch.cuda.Event(), computed=torch.cuda.Event(), drained=torch.cuda.Event()) for _ in range(2)]
 
-        def load(i):
-            s, C = chunks[i]
-            b = stage[i & 1]
-            with torch.cuda.stream(copy_stream):
-                copy_stream.wait_event(b["computed"])     # the previous user of this buffer set has finished computing
-                b["q"][:C].copy_(h_q[s:s + C], non_blocking=True)
-                b["kpre"][:C].copy_(h_kpre[s:s + C], non_blocking=True)
-                b["k"][:C].copy_(h_k[s:s + C], non_blocking=True)
-                b["v"][:C].copy_(h_v[s:s + C], non_blocking=True)
-                b["loaded"].record(copy_stream)
-
-        for b in stage:
-            b["computed"].record(stream)
-        load(0)
-        for i, (s, C) in enumerate(chunks):
-            b = stage[i & 1]
-            if i + 1 < len(chunks):
-                load(i + 1)
-            stream.wait_event(b["loaded"])
-            stream.wait_event(b["drained"])               # the output buffer of this set has been copied out
-            rb.rtp_kv_append(path.ctx, path.params, path.cache, b["k"][:C], b["v"][:C], path.tok_seq[:C],
-                             path.pos_all[s:s + C], path.status)
-            path.run_chunk(s, C, b["q"][:C], b["kpre"][:C], b["out"][:C])
-            b["computed"].record(stream)
-            with torch.cuda.stream(copy_stream):
-                copy_stream.wait_event(b["computed"])
-                h_out[s:s + C].copy_(b["out"][:C], non_blocking=True)
+        def step_e2e():
+            copy_stream.wait_stream(stream)
+            for b in stage:
                 b["drained"].record(copy_stream)
-        stream.wait_stream(copy_stream)
 
-    step_e2e()
-    barrier()
-    n_e2e = max(1, min(args.steps, 3))
-    e0.record(stream)
-    for _ in range(n_e2e):
+            def load(i):
+                s, C = chunks[i]
+                b = stage[i & 1]
+                with torch.cuda.stream(copy_stream):
+                    copy_stream.wait_event(b["computed"])     # the previous user of this buffer set has finished computing
+                    b["q"][:C].copy_(h_q[s:s + C], non_blocking=True)
+                    b["kpre"][:C].copy_(h_kpre[s:s + C], non_blocking=True)
+                    b["k"][:C].copy_(h_k[s:s + C], non_blocking=True)
+                    b["v"][:C].copy_(h_v[s:s + C], non_blocking=True)
+                    b["loaded"].record(copy_stream)
+
+            for b in stage:
+                b["computed"].record(stream)
+            load(0)
+            for i, (s, C) in enumerate(chunks):
+                b = stage[i & 1]
+                if i + 1 < len(chunks):
+                    load(i + 1)
+                stream.wait_event(b["loaded"])
+                stream.wait_event(b["drained"])               # the output buffer of this set has been copied out
+                rb.rtp_kv_append(path.ctx, path.params, path.cache, b["k"][:C], b["v"][:C], path.tok_seq[:C],
+                                 path.pos_all[s:s + C], path.status)
+                path.run_chunk(s, C, b["q"][:C], b["kpre"][:C], b["out"][:C])
+                b["computed"].record(stream)
+                with torch.cuda.stream(copy_stream):
+                    copy_stream.wait_event(b["computed"])
+                    h_out[s:s + C].copy_(b["out"][:C], non_blocking=True)
+                    b["drained"].record(copy_stream)
+            stream.wait_stream(copy_stream)
+
         step_e2e()
-    e1.record(stream)
-    barrier()
-    ms_e2e = e0.elapsed_time(e1) / n_e2e
-    if world > 1:
-        t = torch.tensor([ms_e2e], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    h2d = int(L * (Hq + 2 * Hkv + nih) * 128 * 2)
-    d2h = int(L * Hq * 128 * 2)
-    torch.cuda.synchronize()
-    s_chk, C_chk = chunks[-1]
-    step()                                                  # resident outputs for the comparison below
-    torch.cuda.synchronize()
-    e2e_ok = bool(torch.equal(h_out[s_chk:s_chk + C_chk].to(device), out[s_chk:s_chk + C_chk]))
-    del h_q, h_k, h_v, h_kpre, h_out
+        barrier()
+        n_e2e = max(1, min(args.steps, 3))
+        e0.record(stream)
+        for _ in range(n_e2e):
+            step_e2e()
+        e1.record(stream)
+        barrier()
+        ms_e2e = e0.elapsed_time(e1) / n_e2e
+        if world > 1:
+            t = torch.tensor([ms_e2e], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        h2d = int(L * (Hq + 2 * Hkv + nih) * 128 * 2)
+        d2h = int(L * Hq * 128 * 2)
+        torch.cuda.synchronize()
+        s_chk, C_chk = chunks[-1]
+        step()                                                  # resident outputs for the comparison below
+        torch.cuda.synchronize()
+        e2e_ok = bool(torch.equal(h_out[s_chk:s_chk + C_chk].to(device), out[s_chk:s_chk + C_chk]))
+        return ms_e2e, h2d, d2h, e2e_ok
+
+    if args.workload == "c4":
+        # 1M tokens: the pinned host copies of q and out alone are 17 GB; the end-to-end leg is run on c3 only
+        ms_e2e, h2d, d2h, e2e_ok = None, 0, 0, None
+    else:
+        ms_e2e, h2d, d2h, e2e_ok = run_e2e()
 
     # ---- per-kernel timing of one instrumented step (not part of the timed region) ----
     klass = {"index_keys": 0.0, "select": 0.0, "sparse_attn": 0.0, "local_attn": 0.0}
@@ -451,7 +465,7 @@ def main():
     line = {"metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config, "clocks": clocks,
-            "e2e": {"value": world * L / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e,
+            "e2e": {"value": world * L / (ms_e2e * 1e-3) if ms_e2e else None, "unit": "tokens/s", "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "overlap": "two staging buffer sets, copies on a second stream",
                     "last_chunk_equals_resident_run": e2e_ok},
@@ -492,6 +506,9 @@ def main():
         line["paper_prefill_mode"] = {"what": "retrieval heads dense + local heads sink/window + index-key append",
                                       "ms_per_step": t_paper, "tokens_per_s": L / (t_paper * 1e-3),
                                       "speedup_vs_dense": t_dense / t_paper}
+        if c4:
+            print(json.dumps(line))
+            return
         # CPU oracle on a bounded sample of the same workload
         rows = np.linspace(L // 8, L - 1, 160).astype(np.int64)
         v, done, secs = cpu_oracle_prefill(data, L, rows, budget_s=20.0)
