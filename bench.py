@@ -199,6 +199,21 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
 
     t_sparse = timed(lambda: path.step(data.q, k_pre_new))
     t_dense = timed(lambda: path.step_dense(data.q))
+    # the same sparse step replayed from a CUDA graph (the four library calls captured once): no host launch cost
+    t_graph = None
+    try:
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream(device=device)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            path.step(data.q, k_pre_new)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph):
+            path.step(data.q, k_pre_new)
+        t_graph = timed(graph.replay)
+    except Exception as exc:   # capture is an extra; the plain numbers above stand on their own
+        t_graph = f"not captured: {type(exc).__name__}"
     cnt = path.sel_cnt.float()
     n_ih = data.heads.n_index_heads
     sel_rows = float(cnt.sum().item())
@@ -206,7 +221,8 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
         B * len(data.heads.local_kv_heads) * 512.0 * min(L, 4 + window)
     res = {"workload": name, "batch": B, "context": L, "top_p": top_p,
            "selected_fraction_mean": float(cnt.mean().item()) / L,
-           "sparse_step_us": t_sparse, "dense_step_us": t_dense, "speedup_vs_dense": t_dense / t_sparse,
+           "sparse_step_us": t_sparse, "sparse_step_us_cuda_graph": t_graph, "dense_step_us": t_dense,
+           "speedup_vs_dense": t_dense / t_sparse,
            "algorithmic_bytes": alg_bytes, "sparse_path_gbs": alg_bytes / t_sparse / 1e3,
            "dense_gbs": B * data.heads.n_kv_heads * 512.0 * L / t_dense / 1e3,
            "status": path.status_code()}
