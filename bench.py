@@ -250,9 +250,8 @@ def main():
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2605_16928_b200 import replicas
+    rank, world, local_rank = replicas.env_rank_world()
     n_cores = len(os.sched_getaffinity(0))
     c4 = args.workload == "c4"
     L, chunk = args.seq_len or (1048576 if c4 else 131072), args.chunk or (16384 if c4 else 8192)
@@ -295,14 +294,11 @@ def main():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local_rank)
     device = f"cuda:{local_rank}"
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl")
+    dist = replicas.init("nccl", world)
     from paper_2605_16928_b200 import build as rbuild
     if rank == 0:
         rbuild.build_library()
-    if world > 1:
-        dist.barrier()
+    replicas.barrier(dist, device)
     peaks = load_peaks()
 
     if args.decode_only:
@@ -315,10 +311,7 @@ def main():
     data, path, step, step_dense, out, k_pre, chunks, L, chunk, stream = bench_prefill(args, rank, world, device)
 
     def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
+        replicas.barrier(dist, device)
 
     # ---- device-resident timing ----
     for _ in range(args.warmup):
@@ -334,12 +327,9 @@ def main():
     barrier()
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop()
-    if world > 1:
-        t = torch.tensor([ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = replicas.max_over_ranks(dist, ms, device)
     ms_per_step = ms / args.steps
-    value = world * L / (ms_per_step * 1e-3)
+    value = replicas.whole_job_rate(world, L, ms_per_step)
     status = path.status_code()
     sel_frac = float((path.sel_cnt.float() / (path.pos_all[L - len(path.sel_cnt):].float()[:, None] + 1)).mean().item())
 
@@ -415,10 +405,7 @@ def main():
         e1.record(stream)
         barrier()
         ms_e2e = e0.elapsed_time(e1) / n_e2e
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = replicas.max_over_ranks(dist, ms_e2e, device)
         h2d = int(L * (Hq + 2 * Hkv + nih) * 128 * 2)
         d2h = int(L * Hq * 128 * 2)
         torch.cuda.synchronize()
@@ -481,7 +468,7 @@ def main():
     line = {"metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config, "clocks": clocks,
-            "e2e": {"value": world * L / (ms_e2e * 1e-3) if ms_e2e else None, "unit": "tokens/s", "ms_per_step": ms_e2e,
+            "e2e": {"value": replicas.whole_job_rate(world, L, ms_e2e) if ms_e2e else None, "unit": "tokens/s", "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "overlap": "two staging buffer sets, copies on a second stream",
                     "last_chunk_equals_resident_run": e2e_ok},
@@ -522,26 +509,24 @@ def main():
         line["paper_prefill_mode"] = {"what": "retrieval heads dense + local heads sink/window + index-key append",
                                       "ms_per_step": t_paper, "tokens_per_s": L / (t_paper * 1e-3),
                                       "speedup_vs_dense": t_dense / t_paper}
-        if c4:
-            print(json.dumps(line))
-            return
-        # CPU oracle on a bounded sample of the same workload
-        rows = np.linspace(L // 8, L - 1, 160).astype(np.int64)
-        v, done, secs = cpu_oracle_prefill(data, L, rows, budget_s=20.0)
-        line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": n_cores, "kind": "oracle",
-                                "sample": f"{done} query rows x 32 heads spread over the sequence ({secs:.1f} s), "
-                                          f"extrapolated per token"}
-        del path, data, out, k_pre
-        torch.cuda.empty_cache()
-        dec = []
-        dec.append(bench_decode_point(device, "c2_decode_batched_gqa", 32768, 8, 0.95, 0.1, 2048, True))
-        dec.append(bench_decode_point(device, "c5_decode_b4_512k", 524288, 4, 0.9, 0.05, 4096, False))
-        line["decode"] = dec
+        if not c4:   # the 1M run stops at the comparators: no CPU sample, no decode points
+            # CPU oracle on a bounded sample of the same workload
+            rows = np.linspace(L // 8, L - 1, 160).astype(np.int64)
+            v, done, secs = cpu_oracle_prefill(data, L, rows, budget_s=20.0)
+            line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": n_cores, "kind": "oracle",
+                                    "sample": f"{done} query rows x 32 heads spread over the sequence ({secs:.1f} s), "
+                                              f"extrapolated per token"}
+            del path, data, out, k_pre
+            torch.cuda.empty_cache()
+            dec = []
+            dec.append(bench_decode_point(device, "c2_decode_batched_gqa", 32768, 8, 0.95, 0.1, 2048, True))
+            dec.append(bench_decode_point(device, "c5_decode_b4_512k", 524288, 4, 0.9, 0.05, 4096, False))
+            line["decode"] = dec
     elif "cpu_baseline" not in line:
         line["cpu_baseline"] = None
     if rank == 0:
         print(json.dumps(line))
-    if world > 1:
+    if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
 
