@@ -83,6 +83,17 @@ def test_config5_point_128k():
     assert 0.01 <= np.mean(fr) <= 0.12
 
 
+@pytest.mark.parametrize("top_p,frac,batch,L", [(0.8, 0.2, 2, 20000), (0.99, 0.01, 3, 30000), (0.9, 0.001, 16, 9000),
+                                                 (0.99, 0.2, 1, 70000)])
+def test_config5_sweep_corners(top_p, frac, batch, L):
+    """Corners of the long-context sweep at sizes the oracle finishes quickly: top-p 0.8 .. 0.99, selected fractions
+    0.1 % .. 20 %, batch 1 .. 16 (the 20 % / 70K point needs a key level and more than 4096 candidates per level-1 bin)."""
+    wl = synth.config_5(L=L, batch=batch, top_p=top_p, frac=frac)
+    dw, stats = _run_decode(wl, sel_stride=int(min(L, max(4096, 4 * frac * L))), dense_heads=(3,))
+    fr = np.array([c / n for (c, k, n) in stats])
+    assert 0.2 * frac <= fr.mean() <= 4.0 * frac
+
+
 def test_top_p_one_selects_everything_and_equals_dense():
     gh = _harness()
     wl = synth.config_2(L=700, batch=2, window=512)
