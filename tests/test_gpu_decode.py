@@ -129,6 +129,24 @@ def test_equal_scores_take_lowest_positions(L):
     gh.check_selection(dw, sc, sel)
 
 
+def test_dense_cluster_of_near_equal_scores():
+    """12000 keys that differ from one needle key by single bf16 mantissa bits: their scores crowd into one level-1
+    bin (far more than the 4096 candidates the exact finish takes), many tie exactly, and the cut falls among them:
+    several key levels, the one-CTA tail pass and the tie rule all have to agree with the oracle."""
+    wl = synth.config_1(L=20000, n_needles=4)
+    K = wl.k[0]                                                 # bf16 bit patterns, [L, 1, 128]
+    rng = np.random.default_rng(7)
+    base = K[int(wl.notes["needles"][0]), 0].copy()
+    for n in range(3000, 15000):
+        k = base.copy()
+        dims = rng.integers(0, 128, size=3)
+        k[dims] ^= np.uint16(1)                                # one mantissa ulp in three dimensions
+        K[n, 0] = k
+    dw, stats = _run_decode(wl, sel_stride=20000)
+    c, k_star, n = stats[0]
+    assert 8000 <= c <= 12100                                   # about 90 % of the cluster carries 90 % of the mass
+
+
 def test_window_larger_than_context_equals_dense():
     gh = _harness()
     wl = synth.config_2(L=900, batch=2, window=4096)
