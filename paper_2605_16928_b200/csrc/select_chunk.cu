@@ -258,36 +258,51 @@ __device__ __forceinline__ void page_hits(const unsigned char* pg, const QFrag& 
   const int g = lane >> 2, c = lane & 3;
   const int boff = 2 * qfrag_dim_offset(lane);
   const uint32_t lt = (1u << lane) - 1u;
+  // Four 8-key groups at a time: their MMAs and interval tests are issued back to back, and one vote decides whether
+  // any of the 512 scores is a hit (the usual answer in the later passes is no).
 #pragma unroll
-  for (int nt = 0; nt < 8; ++nt) {
-    const uint2 b = *reinterpret_cast<const uint2*>(pg + (nt * 8 + g) * (kIndexDim * 2) + boff);
-    const float zero[4] = {0.f, 0.f, 0.f, 0.f};
-    float s4[4];
-    mma_bf16_16816(s4, iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
-    const int n0 = n_page + nt * 8 + 2 * c;
-    if (MASK) {
-      const float nan = __int_as_float(0x7fc00000);   // fails every test below
-      if (n0 > L.pos_a) s4[0] = nan;
-      if (n0 + 1 > L.pos_a) s4[1] = nan;
-      if (n0 > L.pos_b) s4[2] = nan;
-      if (n0 + 1 > L.pos_b) s4[3] = nan;
+  for (int half = 0; half < 2; ++half) {
+    float s[4][4];
+    uint32_t hits = 0;   // bit 4 q + e: score e of group q is inside its row's bucket
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int nt = half * 4 + q;
+      const uint2 b = *reinterpret_cast<const uint2*>(pg + (nt * 8 + g) * (kIndexDim * 2) + boff);
+      const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+      mma_bf16_16816(s[q], iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
     }
-    if (COUNT) {   // keys above the bucket of a row that is collecting
-      cnt_a += (s4[0] > L.cut_a) + (s4[1] > L.cut_a);
-      cnt_b += (s4[2] > L.cut_b) + (s4[3] > L.cut_b);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int n0 = n_page + (half * 4 + q) * 8 + 2 * c;
+      if (MASK) {
+        const float nan = __int_as_float(0x7fc00000);   // fails every test below
+        if (n0 > L.pos_a) s[q][0] = nan;
+        if (n0 + 1 > L.pos_a) s[q][1] = nan;
+        if (n0 > L.pos_b) s[q][2] = nan;
+        if (n0 + 1 > L.pos_b) s[q][3] = nan;
+      }
+      if (COUNT) {   // keys above the bucket of a row that is collecting
+        cnt_a += (s[q][0] > L.cut_a) + (s[q][1] > L.cut_a);
+        cnt_b += (s[q][2] > L.cut_b) + (s[q][3] > L.cut_b);
+      }
+      if (s[q][0] >= L.lo_a && s[q][0] <= L.hi_a) hits |= 1u << (4 * q);
+      if (s[q][1] >= L.lo_a && s[q][1] <= L.hi_a) hits |= 2u << (4 * q);
+      if (s[q][2] >= L.lo_b && s[q][2] <= L.hi_b) hits |= 4u << (4 * q);
+      if (s[q][3] >= L.lo_b && s[q][3] <= L.hi_b) hits |= 8u << (4 * q);
     }
-    const bool h0 = s4[0] >= L.lo_a && s4[0] <= L.hi_a, h1 = s4[1] >= L.lo_a && s4[1] <= L.hi_a;
-    const bool h2 = s4[2] >= L.lo_b && s4[2] <= L.hi_b, h3 = s4[3] >= L.lo_b && s4[3] <= L.hi_b;
-    if (__any_sync(0xffffffffu, h0 || h1 || h2 || h3)) {
+    if (!__any_sync(0xffffffffu, hits != 0u)) continue;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int n0 = n_page + (half * 4 + q) * 8 + 2 * c;
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const bool hit = e == 0 ? h0 : e == 1 ? h1 : e == 2 ? h2 : h3;
+        const bool hit = (hits >> (4 * q + e)) & 1u;
         const uint32_t m = __ballot_sync(0xffffffffu, hit);
         if (m) {
           if (hit) {
             const int pos = qcnt + __popc(m & lt);
             wq[2 * pos] = (uint32_t)(n0 + (e & 1)) | ((uint32_t)(g + (e >> 1) * 8) << 27);
-            wq[2 * pos + 1] = __float_as_uint(s4[e]);
+            wq[2 * pos + 1] = __float_as_uint(s[q][e]);
           }
           qcnt += __popc(m);
         }
