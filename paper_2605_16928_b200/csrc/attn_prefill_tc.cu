@@ -18,7 +18,6 @@
 // out, the CTA records RTP_ERR_TIMEOUT, stops waiting (all later waits return at once), still walks its
 // loops to the end, frees its TMEM and exits.
 #include <cuda.h>
-#include <cstdio>
 
 #include "rtp_device.cuh"
 
@@ -346,9 +345,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     float* xch = reinterpret_cast<float*>(smem + kXchOff);
     float m_ref = -INFINITY, l_run = 0.f;
     int n_mine = 0;
-#ifdef RTP_TC_TRACE
-    long long tr_s[4][6];
-#endif
     // ---- sparse mode: membership rule of the rows ----
     // Membership is tested on the unscaled MMA output: raw > up means "score above the row's threshold",
     // raw >= lo "at or above it" (they differ only for keys tied with the threshold score); upn is the next
@@ -414,9 +410,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 
     for (int it = grp; it < n_tiles; it += 2, ++n_mine) {
       const int n_base = tile_at(it) * kBNt;
-#ifdef RTP_TC_TRACE
-      if (n_mine < 4) tr_s[n_mine][5] = clock64();
-#endif
       uint32_t my[4] = {0u, 0u, 0u, 0u};   // this thread's row: bit 31 - (2 nt + e) of my[c] set <=> key 8 nt + 2 c + e is NOT a member
       if (MODE == kPrefillSparse) {
         // Tiles that are causal for every row of the warp and do not contain a row's tie position need one
@@ -507,9 +500,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         }
       }
       mbar_wait(bar(kSFull0 + grp), n_mine & 1, abort_flag, status);
-#ifdef RTP_TC_TRACE
-      if (n_mine < 4) tr_s[n_mine][0] = clock64();
-#endif
       tc_fence_after();
       float s[kBNt];
       {
@@ -519,9 +509,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         RTP_TMEM_LD64(r1p, tmem_s[grp] + lane_addr + 64);
         tc_wait_ld();
       }
-#ifdef RTP_TC_TRACE
-      if (n_mine < 4) tr_s[n_mine][1] = clock64();
-#endif
       tc_fence_before();
       mbar_arrive(bar(kSEmpty0 + grp));          // S is in registers: the buffer may be overwritten
       if (MODE == kPrefillSparse) {
@@ -551,13 +538,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3)) * sc2;
       }
       // this group's previous P must have been consumed (and its O must be quiescent) before P / O are touched
-#ifdef RTP_TC_TRACE
-      if (n_mine < 4) tr_s[n_mine][2] = clock64();
-#endif
       if (n_mine >= 1) mbar_wait(bar(kPEmpty0 + grp), (n_mine - 1) & 1, abort_flag, status);
-#ifdef RTP_TC_TRACE
-      if (n_mine < 4) tr_s[n_mine][3] = clock64();
-#endif
       const bool raise = tmax > m_ref + 8.0f;     // also true for the first finite maximum (m_ref = -inf)
       if (n_mine >= 1 && __any_sync(0xffffffffu, raise)) {
         tc_fence_after();
@@ -594,15 +575,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
       tc_fence_before();
       fence_async_smem();
       mbar_arrive(bar(kPFull0 + grp));
-#ifdef RTP_TC_TRACE
-      if (n_mine < 4) tr_s[n_mine][4] = clock64();
-#endif
     }
-#ifdef RTP_TC_TRACE
-    if (blockIdx.x == 0 && blockIdx.y == 0 && row == 0)
-      for (int i = 0; i < 4 && i < n_mine; ++i)
-        printf("SM grp %d tile %d top %lld sfull %lld ld %lld max %lld pempty %lld pfull %lld\n", grp, 2 * i + grp, tr_s[i][5] - tr_s[0][5], tr_s[i][0] - tr_s[0][5], tr_s[i][1] - tr_s[0][5], tr_s[i][2] - tr_s[0][5], tr_s[i][3] - tr_s[0][5], tr_s[i][4] - tr_s[0][5]);
-#endif
     // ---- merge of the two groups and epilogue ----
     if (n_mine >= 1) mbar_wait(bar(kPEmpty0 + grp), (n_mine - 1) & 1, abort_flag, status);   // this group's last P V is done
     tc_fence_after();
