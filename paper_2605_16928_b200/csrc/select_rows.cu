@@ -379,11 +379,12 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
   __shared__ KeyParams kp[16];
   __shared__ float s_lo_raw[16], s_hi_raw[16];
   __shared__ int s_on[16];
-  const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
+  RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float kInf = __int_as_float(0x7f800000);
-  // With one CTA per unit (n_splits == 1) the CTA is always the one that resolves, and it goes on with the next
-  // level by itself: max_levels > 1 takes whatever the split passes left unresolved to the end.
+  uint32_t n_ctas = gridDim.y;
+  // The first level is split over the unit's CTAs.  The CTA that resolves it goes on alone with whatever is still
+  // unresolved (rare: dense clusters of nearly equal scores), scanning the whole unit, up to max_levels in all.
 #pragma unroll 1
   for (int level = 0; level < max_levels; ++level) {
   if (threadIdx.x < 16) {
@@ -472,7 +473,7 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
       atomicAdd(g_cnt + o, n);
     }
   }
-  if (!take_last_ticket(tickets + blockIdx.x, gridDim.y)) return;
+  if (!take_last_ticket(tickets + blockIdx.x, n_ctas)) return;
 
   // ---- resolve: one warp per head; lane l looks at bins 63 - 2l, 62 - 2l (bin 63 is the top) ----
   for (int j = warp; j < x.nh; j += kWarps) {
@@ -553,6 +554,9 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
   }
   __threadfence();
   __syncthreads();
+  x.p_lo = 0;                                   // from here on this CTA owns the whole unit
+  x.p_hi = (x.n_keys + kPage - 1) >> kPageShift;
+  n_ctas = 1;
   }
 }
 
@@ -1225,11 +1229,8 @@ cudaError_t launch_passes(const CacheView& cv, const Dims& d, const HeadMaps& hm
   dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
   sel_max_kernel<NH4><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, n_splits, status);
   sel_l1_kernel<NH4><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.g_mass, w.tickets, n_splits, status);
-  sel_key_kernel<NH4><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.g_mass, w.g_cnt, w.tickets, n_splits, 1,
-                                                 status);
-  // whatever is still unresolved (rare: dense clusters of nearly equal scores) is finished by one CTA per unit
-  sel_key_kernel<NH4><<<dim3(grid.x, 1), kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.g_mass, w.g_cnt, w.tickets, 1,
-                                                            kKeyLevels, status);
+  sel_key_kernel<NH4><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.g_mass, w.g_cnt, w.tickets, n_splits,
+                                                 1 + kKeyLevels, status);
   return cudaGetLastError();
 }
 
