@@ -69,19 +69,23 @@ __device__ __forceinline__ int lane_head_slot(int lane, int z) {
 }
 
 __global__ void sel_init_kernel(const CacheView cv, const Dims d, const Rows rows, SelState* state,
-                                int64_t n_rowheads) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n_rowheads) return;
-  const int64_t r = i / d.n_ret;
-  const int seq = rows.row_seq(r);
-  int n_keys = rows.row_pos(r) + 1;
-  const int sl = (seq >= 0 && seq < cv.batch) ? cv.seq_lens[seq] : 0;
-  n_keys = max(0, min(n_keys, sl));
-  SelState s = {};
-  s.n_keys = n_keys;
-  s.mode = (d.top_p >= 1.0f || n_keys <= 1) ? kSelectAll : kRefine;
-  s.hi_key = 0xffffffffu;
-  state[i] = s;
+                                int64_t n_rowheads, uint32_t* zero_words, int64_t n_zero_words) {
+  const int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  // merged histograms, counts and tickets start at zero (this replaces a separate memset)
+  for (int64_t i = i0; i < n_zero_words; i += stride) zero_words[i] = 0u;
+  for (int64_t i = i0; i < n_rowheads; i += stride) {
+    const int64_t r = i / d.n_ret;
+    const int seq = rows.row_seq(r);
+    int n_keys = rows.row_pos(r) + 1;
+    const int sl = (seq >= 0 && seq < cv.batch) ? cv.seq_lens[seq] : 0;
+    n_keys = max(0, min(n_keys, sl));
+    SelState s = {};
+    s.n_keys = n_keys;
+    s.mode = (d.top_p >= 1.0f || n_keys <= 1) ? kSelectAll : kRefine;
+    s.hi_key = 0xffffffffu;
+    state[i] = s;
+  }
 }
 
 // ---- which scores a lane post-processes ------------------------------------------------------------
@@ -1248,9 +1252,14 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
   if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
   const int64_t nrh = rows.R * d.n_ret;
   const SelWorkspace w = carve(ws, nrh, rows.R * d.n_ih);
-  cudaError_t e = cudaMemsetAsync(reinterpret_cast<char*>(ws) + w.zero_off, 0, w.zero_bytes, st);
-  if (e != cudaSuccess) return e;
-  sel_init_kernel<<<(unsigned)((nrh + 127) / 128), 128, 0, st>>>(cv, d, rows, w.state, nrh);
+  cudaError_t e = cudaSuccess;
+  {
+    const int64_t n_zero = (int64_t)(w.zero_bytes / 4);
+    const int64_t work = n_zero > nrh ? n_zero : nrh;
+    const unsigned blocks = (unsigned)((work + 255) / 256 < 1184 ? (work + 255) / 256 : 1184);
+    sel_init_kernel<<<blocks, 256, 0, st>>>(cv, d, rows, w.state, nrh,
+                                            reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + w.zero_off), n_zero);
+  }
   int max_nh = 0;
   for (int i = 0; i < d.n_ih; ++i) max_nh = hm.ih_nheads[i] > max_nh ? hm.ih_nheads[i] : max_nh;
   const int n_splits = select_splits(d, rows.R, max_len, sm_count);
