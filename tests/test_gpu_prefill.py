@@ -71,6 +71,27 @@ def test_config3_reduced_select_and_sparse_prefill():
     assert 0.005 <= np.mean(all_fracs) <= 0.6
 
 
+@pytest.mark.parametrize("n_q,n_kv", [(16, 2), (4, 2), (2, 2)])
+def test_other_group_sizes(n_q, n_kv):
+    """G = 8, 2 and 1 query heads per KV head: 16, 64 and 128 positions per CTA tile in the chunk kernels."""
+    wl = synth.config_3(L=1400, n_q_heads=n_q, n_kv_heads=n_kv, ret_kv_heads=(0,), window=300)
+    gh, dw, pr = _prep(wl)
+    rng = np.random.default_rng(n_q)
+    for q_start, C in [(0, 700), (700, 700)]:
+        rows = _sample_rows(q_start, C, rng, extra=(15, 16, 17, 63, 64, 127, 128, 129))
+        sel = pr.select_chunk(q_start, C, with_lists=True)
+        gh.check_chunk_selection(pr, q_start, sel, rows)
+        idx, cnt = sel["idx"].cpu().numpy(), sel["cnt"].cpu().numpy()
+        sets = {(m, i): idx[m - q_start, i, : cnt[m - q_start, i]] for m in rows for i in range(dw.n_ret)}
+        out, lse = pr.sparse_prefill(q_start, C, sel, use_lists=False)
+        gh.check_prefill_rows(pr, q_start, out, lse, rows, "sparse", None, sets)
+        out, lse = pr.local_prefill(q_start, C)
+        gh.check_prefill_rows(pr, q_start, out, lse, rows, "local", wl.heads.local_kv_heads[:1])
+        out, lse = pr.dense_prefill(q_start, C, kv_heads=[1])
+        gh.check_prefill_rows(pr, q_start, out, lse, rows, "dense", [1])
+    assert dw.status_code() == rb.RTP_OK
+
+
 def test_config4_reduced_needle_rows():
     wl = synth.config_4(L=4096, n_needles=32)
     gh, dw, pr = _prep(wl)
