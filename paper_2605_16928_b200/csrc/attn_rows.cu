@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(kHeadDim) attn_merge_kernel(const Dims d, cons
 int plan_splits(int64_t units, int64_t max_set, int sm_count) {
   if (units <= 0) return 1;
   int64_t want = (8LL * sm_count + units - 1) / units;
-  int64_t cap = (max_set + 127) / 128;  // at least 128 tokens per CTA
+  int64_t cap = (max_set + 255) / 256;  // at least 256 tokens per CTA
   int64_t s = want < cap ? want : cap;
   if (s < 1) s = 1;
   if (s > 512) s = 512;
