@@ -454,16 +454,12 @@ def main():
                     "unit": "Tscore/s", "frac": achieved / peak, "traffic": None,
                     "peak_source": "derived: 148 SMs x 128 lanes x 1.9 GHz / 12 lane-ops per score"}
 
-    # DRAM traffic of the dominant kernel per launch, from the committed ncu capture of this command (not measured live)
-    try:
-        with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "profiles", "dram_traffic.json")) as f:
-            tj = json.load(f)
-        ent = tj.get("select_chunk_kernel" if dom == "select" else "attn_prefill_tc_kernel")
-        if ent and ent.get("seq_len") == L and ent.get("chunk") == chunk:
-            roofline["traffic"] = ent["bytes_per_launch"]
-            roofline["traffic_source"] = ent["source"]
-    except (OSError, ValueError):
-        pass
+    # DRAM traffic of the dominant kernel per launch: a figure of the committed ncu launch list of this command (mean of
+    # dram__bytes_read.sum + dram__bytes_write.sum over the launches of the run), not measured live
+    ncu_traffic = {"select": (131072, 8192, 7071514), "sparse_attn": (131072, 8192, 161835718)}
+    if dom in ncu_traffic and ncu_traffic[dom][:2] == (L, chunk) and not c4:
+        roofline["traffic"] = ncu_traffic[dom][2]
+        roofline["traffic_source"] = "profiles/bench_c3_prefill_128k_launch_list.md"
 
     line = {"metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
