@@ -171,7 +171,7 @@ size_t rtp_workspace_bytes(const rtp_params* params, int64_t rows, int64_t max_s
   WsCarver w(nullptr);
   w.take(qt_bytes(d, rows));
   size_t a = select_rows_workspace_bytes(d, rows);
-  const size_t b = select_chunk_workspace_bytes(d, rows);
+  const size_t b = select_chunk_workspace_bytes(d, hm, rows);
   // explicit-row selection keeps 48 KB per (row, head); beyond 4096 rows only the chunk path is sized
   if (rows > 4096) a = 0;
   size_t m = a > b ? a : b;
@@ -294,7 +294,7 @@ rtp_status rtp_topp_select(rtp_ctx* ctx, const rtp_params* params, const rtp_cac
   WsCarver w(workspace);
   __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(w.take(qt_bytes(d, R)));
   const bool chunk = row_seq == nullptr;
-  void* sel_ws = w.take(chunk ? select_chunk_workspace_bytes(d, R) : select_rows_workspace_bytes(d, R));
+  void* sel_ws = w.take(chunk ? select_chunk_workspace_bytes(d, hm, R) : select_rows_workspace_bytes(d, R));
   if (w.off > workspace_bytes) return fail(ctx, RTP_ERR_CAPACITY, "workspace too small");
   cudaError_t e = launch_index_queries(d, hm, reinterpret_cast<const __nv_bfloat16*>(q_pre),
                                        reinterpret_cast<const __nv_bfloat16*>(w_q), R, qt, st);

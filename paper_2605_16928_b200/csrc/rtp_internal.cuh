@@ -103,7 +103,7 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
                                int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
                                int32_t* status, void* ws, int sm_count, cudaStream_t st);
 
-size_t select_chunk_workspace_bytes(const Dims& d, int64_t R);
+size_t select_chunk_workspace_bytes(const Dims& d, const HeadMaps& hm, int64_t R);
 cudaError_t launch_select_chunk(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                                 const __nv_bfloat16* qt, int32_t* sel_idx, int64_t sel_stride,
                                 int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,

@@ -35,7 +35,8 @@ constexpr int kCRows = 128;
 constexpr int kPagesPerStage = 4;
 constexpr int kStageKeys = kPagesPerStage * kPage;                  // 256 keys
 constexpr int kStageBytesC = kStageKeys * kIndexDim * 2;            // 8 KB
-constexpr int kCandCapC = 64;                                       // candidates sorted exactly per row
+constexpr int kCandCapC = 64;                                       // candidates ranked exactly per row
+constexpr int kCandCapG = 2048;                                     // candidates collected per row (global scratch), narrowed to kCandCapC in the warp
 constexpr int kRowBytes = kBins * 8 + 8;                            // per row: 64 x {sum, carries} or 64 x {key, idx}; +8 staggers the banks
 constexpr int kMaxPasses = 14;
 constexpr float kLog2eC = kLog2eH;
@@ -144,8 +145,8 @@ __device__ __forceinline__ void page_l1(const unsigned char* pg, const QFrag& iq
 template <bool MASK, bool TIE, bool COUNT>
 __device__ __forceinline__ void page_late(const unsigned char* pg, const QFrag& iq, int lane, int n_page,
                                           const LaneRows& L, float scale, uint32_t* hist_a, uint32_t* hist_b,
-                                          int* ccnt_a, int* ccnt_b, int& cnt_a, int& cnt_b, int need_a, int need_b,
-                                          int& run_a, int& run_b, int& tl_a, int& tl_b) {
+                                          int* ccnt_a, int* ccnt_b, uint2* gc_a, uint2* gc_b, int& cnt_a, int& cnt_b,
+                                          int need_a, int need_b, int& run_a, int& run_b, int& tl_a, int& tl_b) {
   const int g = lane >> 2, c = lane & 3;
   const int boff = 2 * qfrag_dim_offset(lane);
 #pragma unroll
@@ -185,10 +186,7 @@ __device__ __forceinline__ void page_late(const unsigned char* pg, const QFrag& 
           uint32_t* h = lo ? hist_a : hist_b;
           if (lo ? L.collect_a : L.collect_b) {
             const int slot = atomicAdd(lo ? ccnt_a : ccnt_b, 1);
-            if (slot < kCandCapC) {
-              h[2 * slot] = key;
-              h[2 * slot + 1] = (uint32_t)(n0 + (e & 1));
-            }
+            if (slot < kCandCapG) (lo ? gc_a : gc_b)[slot] = make_uint2(key, (uint32_t)(n0 + (e & 1)));
           } else {
             const uint32_t t = key - (lo ? L.base_a : L.base_b);
             add_mass(h + 2 * (t >> (lo ? L.shift_a : L.shift_b)), fmaf(s - (lo ? L.ref_a : L.ref_b), kLog2eC, 20.0f));
@@ -222,7 +220,7 @@ __device__ __forceinline__ void page_late(const unsigned char* pg, const QFrag& 
 // Works off the warp's queue of bucket hits: entry = {position | local row << 27, raw score bits}.
 // (The count is passed by value: a reference would pin the caller's counter to local memory.)
 __device__ __noinline__ void drain_hits(uint32_t* wq, int qcnt, int lane, int wrow, RowState* rs, uint32_t* hist,
-                                        float scale) {
+                                        uint2* gcand, float scale) {
   constexpr int kRowWords = kRowBytes / 4;
   __syncwarp();
   for (int base = 0; base < qcnt; base += 32) {
@@ -237,10 +235,7 @@ __device__ __noinline__ void drain_hits(uint32_t* wq, int qcnt, int lane, int wr
       uint32_t* h = hist + r * kRowWords;
       if (S->phase == kPhCollect) {
         const int slot = atomicAdd(&S->cand_cnt, 1);
-        if (slot < kCandCapC) {
-          h[2 * slot] = key;
-          h[2 * slot + 1] = w0 & 0x7ffffffu;
-        }
+        if (slot < kCandCapG) gcand[(size_t)r * kCandCapG + slot] = make_uint2(key, w0 & 0x7ffffffu);
       } else {
         const uint32_t t = key - S->base_key;
         add_mass(h + 2 * (t >> S->shift), fmaf(s - S->ref_s, kLog2eC, 20.0f));
@@ -254,7 +249,7 @@ __device__ __noinline__ void drain_hits(uint32_t* wq, int qcnt, int lane, int wr
 template <bool MASK, bool COUNT>
 __device__ __forceinline__ void page_hits(const unsigned char* pg, const QFrag& iq, int lane, int n_page,
                                           const LaneRows& L, int& cnt_a, int& cnt_b, uint32_t* wq, int& qcnt,
-                                          int wrow, RowState* rs, uint32_t* hist, float scale) {
+                                          int wrow, RowState* rs, uint32_t* hist, uint2* gcand, float scale) {
   const int g = lane >> 2, c = lane & 3;
   const int boff = 2 * qfrag_dim_offset(lane);
   const uint32_t lt = (1u << lane) - 1u;
@@ -308,7 +303,7 @@ __device__ __forceinline__ void page_hits(const unsigned char* pg, const QFrag& 
         }
       }
       if (qcnt >= 32) {   // at most 31 + 128 entries queued
-        drain_hits(wq, qcnt, lane, wrow, rs, hist, scale);
+        drain_hits(wq, qcnt, lane, wrow, rs, hist, gcand, scale);
         qcnt = 0;
       }
     }
@@ -320,8 +315,11 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
     const CacheView cv, const Dims d, const HeadMaps hm, const __nv_bfloat16* __restrict__ qt,
     const int seq_id, const int q_start, const int C, int32_t* __restrict__ sel_idx, const int64_t sel_stride,
     int32_t* __restrict__ sel_count, float* __restrict__ sel_mass, float* __restrict__ sel_thresh,
-    int32_t* __restrict__ sel_tie_last, int32_t* status, const int n_row_tiles, const int max_passes) {
+    int32_t* __restrict__ sel_tie_last, int32_t* status, uint2* __restrict__ gcand_all, const int n_row_tiles,
+    const int max_passes) {
   constexpr int BMP = kCRows / G;
+  // candidate scratch of this CTA: [128 rows][kCandCapG] {ordered key, position}
+  uint2* gcand = gcand_all + ((size_t)blockIdx.y * gridDim.x + blockIdx.x) * (size_t)(kCRows * kCandCapG);
   extern __shared__ __align__(128) unsigned char smem[];
   uint32_t* hist = reinterpret_cast<uint32_t*>(smem);                      // [128 rows][128 words]
   unsigned char* stage_s = smem + kHistBytes;
@@ -480,8 +478,8 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
             if (interior) page_l1<false>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b);
             else page_l1<true>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b);
           } else {
-#define RTP_LATE(M_, T_, C_) page_late<M_, T_, C_>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b, ccnt_a, ccnt_b, cnt_a, cnt_b, need_a, need_b, run_a, run_b, tl_a, tl_b)
-#define RTP_HITS(M_, C_) page_hits<M_, C_>(pgp, iq, lane, n_page, LR, cnt_a, cnt_b, wq, qcnt, wrow, rs, hist, scale)
+#define RTP_LATE(M_, T_, C_) page_late<M_, T_, C_>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b, ccnt_a, ccnt_b, gcand + (size_t)la * kCandCapG, gcand + (size_t)lb * kCandCapG, cnt_a, cnt_b, need_a, need_b, run_a, run_b, tl_a, tl_b)
+#define RTP_HITS(M_, C_) page_hits<M_, C_>(pgp, iq, lane, n_page, LR, cnt_a, cnt_b, wq, qcnt, wrow, rs, hist, gcand, scale)
             if (pass_tie) {
               if (interior) RTP_LATE(false, true, true); else RTP_LATE(true, true, true);
             } else if (pass_count) {
@@ -497,7 +495,7 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
       __syncthreads();
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (qcnt > 0) drain_hits(wq, qcnt, lane, wrow, rs, hist, scale);
+    if (qcnt > 0) drain_hits(wq, qcnt, lane, wrow, rs, hist, gcand, scale);
     qcnt = 0;
 
     // ---- end of pass: combine the quad's partial results ----
@@ -588,7 +586,7 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
           const float f_above = first ? run : run + m0f;
           const float f_q = first ? q0 : q1;
           const int bin = first ? b0 : b1;
-          const bool few = f_q < 0.999f * kMinQ * (float)kCandCapC;   // fewer than kCandCapC keys in the bin
+          const bool few = f_q < 0.999f * kMinQ * (float)kCandCapG;   // fewer than kCandCapG keys in the bin
           S->mass_above = f_above;
           if (l1) {
             S->Z = Z;
@@ -636,20 +634,100 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
           }
         }
       } else if (ph == kPhCollect) {
-        const int n_c = R.cand_cnt;                  // keys inside the bucket
-        const int above = R.cnt_above + __shfl_sync(0xffffffffu, is_b ? cnt_b : cnt_a, src_lane);
-        if (n_c > kCandCapC) {
-          // only reachable when the bucket is a single key value: n_c equal scores straddle the cut
+        // The pass put every key of the bucket (at most kCandCapG, by the bound that sent the row here) into the row's
+        // list in global scratch and counted the keys above the bucket.  While more than kCandCapC of them are left,
+        // the warp narrows on the list itself: the same 64-bin mass histogram over the next six key bits, in the row's
+        // shared-memory bins, no pass over the keys.  Then the exact ranking below finishes.
+        const int n_all = R.cand_cnt;
+        int above = R.cnt_above + __shfl_sync(0xffffffffu, is_b ? cnt_b : cnt_a, src_lane);
+        float m_above = R.mass_above;
+        uint32_t base = R.base_key, span = R.span;
+        int n_in = n_all;
+        const uint2* gc = gcand + (size_t)lr * kCandCapG;
+        uint32_t* hw = hist + lr * kRowWords;
+        if (n_all <= kCandCapG) {
+          while (n_in > kCandCapC && span > 1u) {
+            const int bits = 32 - __clz(span - 1u);
+            const int shift = max(0, bits - 6);
+            for (int i = lane; i < kRowWords; i += 32) hw[i] = 0u;
+            __syncwarp();
+            for (int i = lane; i < n_all; i += 32) {
+              const uint32_t key = __ldcg(&gc[i].x);
+              const uint32_t t = key - base;
+              if (t < span) add_mass(hw + 2 * (t >> shift), fmaf(okey_to_float(key) - R.ref_s, kLog2eC, 20.0f));
+            }
+            __syncwarp();
+            const int b0 = 63 - 2 * lane, b1 = 62 - 2 * lane;   // bin 63 is the top
+            const uint32_t sum0 = hw[2 * b0], car0 = hw[2 * b0 + 1], sum1 = hw[2 * b1], car1 = hw[2 * b1 + 1];
+            const float sc = R.e_ref * 9.5367431640625e-07f;     // 2^-20
+            const float m0f = acc_mass(sum0, car0) * sc, m1f = acc_mass(sum1, car1) * sc;
+            float incm = m0f + m1f;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+              const float tm = __shfl_up_sync(0xffffffffu, incm, o);
+              if (lane >= o) incm += tm;
+            }
+            const float run = m_above + incm - (m0f + m1f);
+            int found = 64, last = -1;
+            if (sum0 | car0) {
+              last = 2 * lane;
+              if (run + m0f >= R.target) found = 2 * lane;
+            }
+            if (sum1 | car1) {
+              last = 2 * lane + 1;
+              if (found == 64 && run + m0f + m1f >= R.target) found = 2 * lane + 1;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+              found = min(found, __shfl_xor_sync(0xffffffffu, found, o));
+              last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+            }
+            if (found == 64) found = last;
+            if (found < 0) break;                                 // (no candidate inside the interval: cannot happen)
+            m_above = __shfl_sync(0xffffffffu, (found & 1) ? run + m0f : run, found >> 1);
+            const uint32_t ofs = (uint32_t)(63 - found) << shift;
+            const uint32_t nbase = base + ofs, nspan = min(1u << shift, span - ofs);
+            int c_in = 0, c_up = 0;                               // candidates inside / above the new interval
+            for (int i = lane; i < n_all; i += 32) {
+              const uint32_t t = __ldcg(&gc[i].x) - base;
+              if (t < span) {
+                if (t - ofs < nspan) ++c_in;
+                else if (t >= ofs) ++c_up;
+              }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+              c_in += __shfl_xor_sync(0xffffffffu, c_in, o);
+              c_up += __shfl_xor_sync(0xffffffffu, c_up, o);
+            }
+            above += c_up;
+            n_in = c_in;
+            base = nbase;
+            span = nspan;
+            __syncwarp();
+          }
+        }
+        if (n_in > kCandCapC) {
+          // more than kCandCapC keys share one key value: n_in equal scores straddle the cut
+          float rlo = 0.f, rhi = 0.f;
+          if (lane == 0 && base != R.base_key) raw_preimage(scale, base, base, rlo, rhi);
           if (lane == 0) {
-            const float each = fast_ex2((okey_to_float(R.base_key) - R.M) * kLog2eC);
-            int take = (int)ceilf((R.target - R.mass_above) / each);
-            take = max(1, min(take, n_c));
+            const float each = fast_ex2((okey_to_float(base) - R.M) * kLog2eC);
+            int take = (int)ceilf((R.target - m_above) / each);
+            take = max(1, min(take, n_in));
             S->cnt_above = above;
-            S->thr_key = R.base_key;
+            S->mass_above = m_above;
+            S->thr_key = base;
             S->count = above + take;
-            S->sel_mass = (R.mass_above + (float)take * each) / R.Z;
-            if (R.span != 1u) set_status(status, RTP_ERR_UNSUPPORTED);
-            if (take < n_c) {
+            S->sel_mass = (m_above + (float)take * each) / R.Z;
+            if (span != 1u) set_status(status, RTP_ERR_UNSUPPORTED);
+            if (take < n_in) {
+              if (base != R.base_key) {   // the tie pass looks for this key value
+                S->base_key = base;
+                S->span = 1u;
+                S->raw_lo = rlo;
+                S->raw_hi = rhi;
+              }
               S->tie_need = take;
               S->phase = kPhTie;
             } else {
@@ -658,6 +736,27 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
             }
           }
         } else {
+          // the candidates of the final interval move into the row's shared-memory list {key, position}
+          __syncwarp();
+          int filled = 0;
+          for (int i0 = 0; i0 < n_all; i0 += 32) {
+            const int i = i0 + lane;
+            uint2 cnd = make_uint2(0u, 0u);
+            bool in = false;
+            if (i < n_all) {
+              cnd = __ldcg(&gc[i]);
+              in = cnd.x - base < span;
+            }
+            const uint32_t m = __ballot_sync(0xffffffffu, in);
+            if (in) {
+              const int pos = filled + __popc(m & ((1u << lane) - 1u));
+              hw[2 * pos] = cnd.x;
+              hw[2 * pos + 1] = cnd.y;
+            }
+            filled += __popc(m);
+          }
+          __syncwarp();
+          const int n_c = n_in;
           // exact finish: rank the (at most 64) candidates by (score descending, position ascending)
           unsigned long long ord[2];
           float e[2];
@@ -673,7 +772,7 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
             }
           }
           int rank[2] = {0, 0};
-          float cum[2] = {R.mass_above, R.mass_above};
+          float cum[2] = {m_above, m_above};
           for (int j = 0; j < n_c; ++j) {
             const int jl = j >> 1;
             const unsigned long long oj = __shfl_sync(0xffffffffu, (j & 1) ? ord[1] : ord[0], jl);
@@ -831,7 +930,7 @@ __global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
 template <int G>
 cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                          const __nv_bfloat16* qt, int32_t* sel_idx, int64_t sel_stride, int32_t* sel_count,
-                         float* sel_mass, float* sel_thresh, int32_t* sel_tie_last, int32_t* status,
+                         float* sel_mass, float* sel_thresh, int32_t* sel_tie_last, int32_t* status, void* ws,
                          cudaStream_t st) {
   static bool attr_done = false;
   if (!attr_done) {
@@ -844,33 +943,41 @@ cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm,
   dim3 grid(n_row_tiles, d.n_ih);
   select_chunk_kernel<G><<<grid, kCThreads, kSmemC, st>>>(cv, d, hm, qt, rows.seq_id, rows.q_start, (int)rows.R,
                                                           sel_idx, sel_stride, sel_count, sel_mass, sel_thresh,
-                                                          sel_tie_last, status, n_row_tiles, kMaxPasses);
+                                                          sel_tie_last, status, reinterpret_cast<uint2*>(ws), n_row_tiles,
+                                                          kMaxPasses);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-size_t select_chunk_workspace_bytes(const Dims& d, int64_t R) {
-  (void)d;
-  (void)R;
-  return 256;   // all state lives in shared memory
+// rows of a CTA are [head slot][position]: the smallest supported slot count that fits the widest index head
+static int slot_class(const Dims& d, const HeadMaps& hm) {
+  int max_nh = 0;
+  for (int j = 0; j < d.n_ih; ++j) max_nh = hm.ih_nheads[j] > max_nh ? hm.ih_nheads[j] : max_nh;
+  return max_nh <= 1 ? 1 : max_nh <= 2 ? 2 : max_nh <= 4 ? 4 : max_nh <= 8 ? 8 : 0;
+}
+
+// Candidate scratch: kCandCapG entries of 8 bytes per (row, head slot) of every CTA.
+size_t select_chunk_workspace_bytes(const Dims& d, const HeadMaps& hm, int64_t R) {
+  const int g = slot_class(d, hm);
+  if (g == 0 || R <= 0) return 256;
+  const int64_t n_row_tiles = (R + kCRows / g - 1) / (kCRows / g);
+  return (size_t)n_row_tiles * d.n_ih * kCRows * kCandCapG * sizeof(uint2);
 }
 
 cudaError_t launch_select_chunk(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                                 const __nv_bfloat16* qt, int32_t* sel_idx, int64_t sel_stride,
                                 int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
                                 int32_t* status, void* ws, int sm_count, cudaStream_t st) {
-  (void)ws;
   (void)sm_count;
   if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
-  int max_nh = 0;
-  for (int j = 0; j < d.n_ih; ++j) max_nh = hm.ih_nheads[j] > max_nh ? hm.ih_nheads[j] : max_nh;
-  // rows of a CTA are [head slot][position]: pick the smallest supported slot count that fits
-  if (max_nh <= 1) return launch_typed<1>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, st);
-  if (max_nh <= 2) return launch_typed<2>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, st);
-  if (max_nh <= 4) return launch_typed<4>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, st);
-  if (max_nh <= 8) return launch_typed<8>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, st);
-  return cudaErrorNotSupported;
+  switch (slot_class(d, hm)) {
+    case 1: return launch_typed<1>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, st);
+    case 2: return launch_typed<2>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, st);
+    case 4: return launch_typed<4>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, st);
+    case 8: return launch_typed<8>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, st);
+    default: return cudaErrorNotSupported;
+  }
 }
 
 }  // namespace rtp
