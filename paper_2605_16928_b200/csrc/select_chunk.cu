@@ -36,7 +36,7 @@ constexpr int kPagesPerStage = 4;
 constexpr int kStageKeys = kPagesPerStage * kPage;                  // 256 keys
 constexpr int kStageBytesC = kStageKeys * kIndexDim * 2;            // 8 KB
 constexpr int kCandCapC = 64;                                       // candidates ranked exactly per row
-constexpr int kCandCapG = 2048;                                     // candidates collected per row (global scratch), narrowed to kCandCapC in the warp
+constexpr int kCandCapG = 4096;                                     // candidates collected per row (global scratch), narrowed to kCandCapC in the warp
 constexpr int kRowBytes = kBins * 8 + 8;                            // per row: 64 x {sum, carries} or 64 x {key, idx}; +8 staggers the banks
 constexpr int kMaxPasses = 14;
 constexpr float kLog2eC = kLog2eH;
