@@ -111,7 +111,10 @@ void rtp_destroy(rtp_ctx* ctx);
 const char* rtp_last_error(const rtp_ctx* ctx);
 
 /* Bytes of DEVICE workspace that any call below needs for `rows` query rows
- * against sequences of at most `max_seq_len` tokens.  0 on invalid params. */
+ * against sequences of at most `max_seq_len` tokens.  0 on invalid params.
+ * The largest consumer is rtp_topp_select in chunk mode: 32 KB per (row,
+ * retrieval head) for the candidate lists of the exact finish, rounded up to
+ * whole tiles of 128 (row, head) pairs (2 GB for 8192 rows x 8 heads). */
 size_t rtp_workspace_bytes(const rtp_params* params, int64_t rows, int64_t max_seq_len);
 
 /* Synchronises `stream`, reads the DEVICE status word and returns it as an
