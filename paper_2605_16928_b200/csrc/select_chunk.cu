@@ -40,7 +40,7 @@ constexpr int kCandCapG = 4096;                                     // candidate
 constexpr int kRowBytes = kBins * 8 + 8;                            // per row: 64 x {sum, carries} or 64 x {key, idx}; +8 staggers the banks
 constexpr int kMaxPasses = 14;
 constexpr float kLog2eC = kLog2eH;
-constexpr int kQueueCap = 160;                                      // per-warp queue of bucket hits (entries of 8 bytes)
+constexpr int kQueueCap = 288;                                      // per-warp queue of bucket hits (entries of 8 bytes)
 
 enum Phase { kPhMax = 0, kPhL1 = 1, kPhKey = 2, kPhCollect = 3, kPhTie = 4, kPhDone = 5 };
 
@@ -64,7 +64,7 @@ struct RowState {      // one per (row, head), in shared memory
 };
 
 constexpr int kHistBytes = kCRows * kRowBytes;                      // 64 KB
-constexpr int kQueueBytes = kCWarps * kQueueCap * 8;               // 10 KB
+constexpr int kQueueBytes = kCWarps * kQueueCap * 8;               // 18 KB
 constexpr int kSmemC = kHistBytes + 2 * kStageBytesC + kQueueBytes + kCRows * (int)sizeof(RowState);
 
 __device__ __forceinline__ void cp_async16c(uint32_t dst, const void* src) {
@@ -252,7 +252,6 @@ __device__ __forceinline__ void page_hits(const unsigned char* pg, const QFrag& 
                                           int wrow, RowState* rs, uint32_t* hist, uint2* gcand, float scale) {
   const int g = lane >> 2, c = lane & 3;
   const int boff = 2 * qfrag_dim_offset(lane);
-  const uint32_t lt = (1u << lane) - 1u;
   // Four 8-key groups at a time: their MMAs and interval tests are issued back to back, and one vote decides whether
   // any of the 512 scores is a hit (the usual answer in the later passes is no).
 #pragma unroll
@@ -286,23 +285,34 @@ __device__ __forceinline__ void page_hits(const unsigned char* pg, const QFrag& 
       if (s[q][3] >= L.lo_b && s[q][3] <= L.hi_b) hits |= 8u << (4 * q);
     }
     if (!__any_sync(0xffffffffu, hits != 0u)) continue;
+    // every lane appends its hits behind those of the lower lanes: a prefix sum over the lanes' hit counts, then
+    // predicated stores (no vote per score); two 8-key groups at a time bound the queue growth by 256 entries
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int n0 = n_page + (half * 4 + q) * 8 + 2 * c;
+    for (int pr = 0; pr < 2; ++pr) {
+      const uint32_t hb = (hits >> (8 * pr)) & 0xffu;
+      const int mine = __popc(hb);
+      int incl = mine;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const bool hit = (hits >> (4 * q + e)) & 1u;
-        const uint32_t m = __ballot_sync(0xffffffffu, hit);
-        if (m) {
-          if (hit) {
-            const int pos = qcnt + __popc(m & lt);
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      int pos = qcnt + incl - mine;
+      qcnt += __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll
+      for (int qq = 0; qq < 2; ++qq) {
+        const int q = 2 * pr + qq;
+        const int n0 = n_page + (half * 4 + q) * 8 + 2 * c;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if ((hb >> (4 * qq + e)) & 1u) {
             wq[2 * pos] = (uint32_t)(n0 + (e & 1)) | ((uint32_t)(g + (e >> 1) * 8) << 27);
             wq[2 * pos + 1] = __float_as_uint(s[q][e]);
+            ++pos;
           }
-          qcnt += __popc(m);
         }
       }
-      if (qcnt >= 32) {   // at most 31 + 128 entries queued
+      if (qcnt >= 32) {   // at most 31 + 256 entries queued
         drain_hits(wq, qcnt, lane, wrow, rs, hist, gcand, scale);
         qcnt = 0;
       }
