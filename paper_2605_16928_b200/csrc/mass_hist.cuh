@@ -21,8 +21,10 @@ constexpr float kMinQ = 634880.0f;        // (floor(e^-0.5 * 1024) - 1) * 1024
 // mantissa bits, so no float <-> int conversion instruction is needed; the same arithmetic serves the histogram
 // pass and the bisection that turns a bin into a key interval.
 constexpr float kMagic = 12582912.0f;     // 1.5 * 2^23
+// (s <= M for every score of the row, so only the upper clamp is needed; the mask keeps the index in range whatever
+// the inputs.)
 __device__ __forceinline__ int l1_bin_f(float M, float s, float& bin_f) {
-  const float u = fminf(fmaxf((M - s) * kL1Scale, 0.0f), (float)(kBins - 1));
+  const float u = fminf(fmaf(s, -kL1Scale, kL1Scale * M), (float)(kBins - 1));
   const float t = u + kMagic;
   bin_f = t - kMagic;
   return __float_as_int(t) & (kBins - 1);
@@ -46,7 +48,8 @@ __device__ __forceinline__ float l1_bin_lo(float M, int b) { return M - ((float)
 // Adds round(2^x) (x <= 20) to an accumulator {sum mod 2^32, carries} in shared memory.
 __device__ __forceinline__ void add_mass(uint32_t* acc, float x) {
   // nearest integer to 2^x through the mantissa of (2^x + 2^23): no conversion instruction
-  const uint32_t q = min(__float_as_uint(fast_ex2(x) + 8388608.0f) - 0x4b000000u, 1u << 20);
+  // (x can exceed 20 by a rounding error: a contribution a few units above 2^20 is as good as any)
+  const uint32_t q = __float_as_uint(fast_ex2(x) + 8388608.0f) - 0x4b000000u;
   const uint32_t old = atomicAdd(acc, q);
   if (old + q < old) atomicAdd(acc + 1, 1u);
 }

@@ -130,7 +130,7 @@ __device__ __forceinline__ void page_l1(const unsigned char* pg, const QFrag& iq
     for (int e = 0; e < 4; ++e) {
       const bool lo = e < 2;
       if (MASK && n0 + (e & 1) > (lo ? L.pos_a : L.pos_b)) continue;
-      const float s = finish_score(s4[e], scale);
+      const float s = s4[e] * scale;   // (the sign of a zero score does not matter here)
       const float M = lo ? L.M_a : L.M_b;
       float bin_f;
       const int bin = l1_bin_f(M, s, bin_f);   // (rows that are already done have no M: they land in bin 0)
