@@ -456,7 +456,7 @@ def main():
 
     # DRAM traffic of the dominant kernel per launch: a figure of the committed ncu launch list of this command (mean of
     # dram__bytes_read.sum + dram__bytes_write.sum over the launches of the run), not measured live
-    ncu_traffic = {"select": (131072, 8192, 757835200), "sparse_attn": (131072, 8192, 161724942)}
+    ncu_traffic = {"select": (131072, 8192, 755511344), "sparse_attn": (131072, 8192, 161831196)}
     if dom in ncu_traffic and ncu_traffic[dom][:2] == (L, chunk) and not c4:
         roofline["traffic"] = ncu_traffic[dom][2]
         roofline["traffic_source"] = "profiles/bench_c3_prefill_128k_launch_list.md"
