@@ -88,6 +88,11 @@ class DecodePath(_Base):
         self.sel_tie = torch.empty((B, self.n_ret), dtype=torch.int32, device=self.dev)
         self.out = torch.empty((B, self.Hq, 128), dtype=torch.bfloat16, device=self.dev)
         self.lse = torch.empty((B, self.Hq), dtype=torch.float32, device=self.dev)
+        # local heads do not depend on the retrieval heads: their attention runs on a second stream with a workspace
+        # of its own and joins before the step returns
+        self.side = torch.cuda.Stream(device=self.dev)
+        self.workspace_local = torch.empty_like(self.workspace)
+        self.has_local = len(data.heads.local_kv_heads) > 0
 
     def build_index_cache(self, step: int = 1 << 17):
         for b in range(self.B):
@@ -97,13 +102,18 @@ class DecodePath(_Base):
     def step(self, q, k_pre_new):
         """q: bf16 [B, Hq, 128]; k_pre_new: bf16 [B, n_index_heads, 128] pre-RoPE keys of the newest tokens."""
         d, p = self.data, self.params
+        main = torch.cuda.current_stream()
+        if self.has_local:
+            self.side.wait_stream(main)
+            rb.rtp_local_attn(self.ctx, p, self.cache, q, d.row_seq, d.row_pos, 0, 0, self.B, self.out, self.lse,
+                              self.workspace_local, self.status, stream=self.side)
         rb.rtp_index_keys(self.ctx, p, self.cache, k_pre_new, d.w_k, d.row_seq, d.row_pos)
         rb.rtp_topp_select(self.ctx, p, self.cache, q, d.w_q, d.row_seq, d.row_pos, 0, 0, self.B, self.sel_idx,
                            self.sel_cnt, self.sel_mass, self.sel_thr, self.sel_tie, self.status, self.workspace)
         rb.rtp_sparse_attn_decode(self.ctx, p, self.cache, q, d.row_seq, d.row_pos, self.sel_idx, self.sel_cnt,
                                   self.out, self.lse, self.workspace, self.status)
-        rb.rtp_local_attn(self.ctx, p, self.cache, q, d.row_seq, d.row_pos, 0, 0, self.B, self.out, self.lse,
-                          self.workspace, self.status)
+        if self.has_local:
+            main.wait_stream(self.side)
 
     def step_dense(self, q):
         d = self.data
