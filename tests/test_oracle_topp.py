@@ -143,6 +143,63 @@ def test_band_classification_consistent():
     assert orc.set_mass(s, ids) >= 0.9
 
 
+def _geometric(n=60):
+    # s_i = -i ln 2: softmax masses 2^-(i+1) / (1 - 2^-n); cumulative mass before token k is 1 - 2^-k
+    return -np.arange(n, dtype=np.float64) * np.log(2.0)
+
+
+def test_set_mass_closed_form_geometric():
+    s = _geometric()
+    for k in (1, 2, 4, 7, 20):
+        assert orc.set_mass(s, range(k)) == pytest.approx(1.0 - 2.0 ** -k, abs=1e-12)
+    # an arbitrary subset, given in any order and as any iterable
+    assert orc.set_mass(s, [3, 1]) == pytest.approx(2.0 ** -2 + 2.0 ** -4, abs=1e-12)
+    assert orc.set_mass(s, {0}) == pytest.approx(0.5, abs=1e-12)
+    # normalised over the WHOLE row, whatever constant is added to the scores
+    assert orc.set_mass(s + 37.5, range(4)) == pytest.approx(0.9375, abs=1e-12)
+    assert orc.set_mass(s, range(len(s))) == pytest.approx(1.0, abs=1e-12)
+
+
+def test_band_classification_closed_form_geometric():
+    s = _geometric().astype(np.float32)
+    n = len(s)
+    # p = 0.9: cumulative mass before tokens 0..3 is 0, .5, .75, .875 (mandatory); before token 4 it is .9375
+    mand, forb = orc.classify_against_band(s, 0.9)
+    assert mand == {0, 1, 2, 3}
+    assert forb == set(range(4, n))
+    # the mass before token 4 is 0.9375: it is mandatory / optional / forbidden according to where p lies
+    # relative to 0.9375 -+ 1e-4; token 3 (before: .875) and token 5 (before: .96875) never change class
+    cases = [(+2e-4, "mandatory"), (+5e-5, "optional"), (-5e-5, "optional"), (-2e-4, "forbidden")]
+    for delta, want in cases:
+        mand, forb = orc.classify_against_band(s, 0.9375 + delta)
+        got = "mandatory" if 4 in mand else "forbidden" if 4 in forb else "optional"
+        assert got == want, (delta, got)
+        assert {0, 1, 2, 3} <= mand and 5 in forb and 5 not in mand
+        assert not (mand & forb)
+    # the band argument is honoured: ten times wider makes token 4 optional in both outer cases,
+    # a hundred times narrower leaves no optional token at +-5e-5
+    for delta in (+2e-4, -2e-4):
+        mand, forb = orc.classify_against_band(s, 0.9375 + delta, band=1e-3)
+        assert 4 not in mand and 4 not in forb
+    mand, forb = orc.classify_against_band(s, 0.9375 + 5e-5, band=1e-6)
+    assert 4 in mand
+    mand, forb = orc.classify_against_band(s, 0.9375 - 5e-5, band=1e-6)
+    assert 4 in forb
+    # every token is classified at most once and p = 1 makes every token mandatory
+    mand, forb = orc.classify_against_band(s, 1.0)
+    assert mand == set(range(n)) and forb == set()
+
+
+def test_band_classification_uses_mass_before_inclusion():
+    # two tokens of mass 0.6 / 0.4 (scores ln 0.6, ln 0.4): for p = 0.6 the first token alone reaches p; the
+    # second has 0.6 before it, which is inside the band around p, so it may go either way; for p = 0.5 it is
+    # forbidden, for p = 0.7 mandatory
+    s = np.log(np.array([0.6, 0.4])).astype(np.float32)
+    assert orc.classify_against_band(s, 0.6) == ({0}, set())
+    assert orc.classify_against_band(s, 0.5) == ({0}, {1})
+    assert orc.classify_against_band(s, 0.7) == ({0, 1}, set())
+
+
 def test_rejects_bad_p():
     with pytest.raises(ValueError):
         orc.topp_select(np.zeros(4, np.float32), 0.0)
