@@ -1,960 +1,1024 @@
-// S2-S4 for a prefill chunk: fused indexer + top-p selection (Eq. 5) for rows q_start .. q_start+C-1
-// of one sequence.
+// S2-S4 for a prefill chunk: fused indexer + top-p selection (Eq. 5) for rows q_start .. q_start+C-1 of one
+// sequence, on the 5th-generation tensor cores.
 //
-// A CTA owns 128 (row, head) pairs: (128 / G) consecutive positions x the G retrieval heads of one
-// index head; each warp owns 16 of them (one head, 16 positions).  The CTA streams the index keys
-// 0 .. last position (2 KB per page, cp.async double buffer) once per pass; a warp scores a 64-key
-// page against its 16 rows with eight m16n8k16 MMAs.  All selection state lives in shared memory, so
-// the whole selection of the chunk is one kernel without inter-CTA communication:
-//   max       row maximum M                                                   (1 op per score)
-//   level 1   64-bin histogram of softmax mass over d = M - s in steps of 1/2 (d >= 31.25 pooled), in
-//             fixed point with native 32-bit shared-memory adds; gives Z and the bucket in which the
-//             cumulative mass reaches p * Z; the bucket becomes an exact interval of ordered score keys
-//             (bisection) and of unscaled MMA outputs (so later passes compare raw values only)
-//   key level 64-bin mass histogram of the ordered key inside the interval, 6 key bits per pass, until the
-//             chosen bin provably holds at most 64 keys.  From here on only a small share of the scores falls
-//             into a row's interval: a warp appends those hits (row, position, raw score) to a queue in shared
-//             memory and works them off 32 at a time, one hit per lane, so that the per-hit arithmetic and the
-//             shared-memory adds are issued once per 32 hits instead of once per MMA
-//   collect   the keys of the final bucket go to a 64-entry list, the keys above it are counted; the warp
-//             ranks the list exactly by (score descending, position ascending) and cuts it
-//   tie       only when more than 64 equal scores straddle the cut: position of the last tie taken
-// Rows drop out as soon as they are resolved; the CTA stops when all its rows are.  When id lists
-// are requested, one more sweep appends every row's members in position order.
-// Each pass has its own inner loop; pages that lie wholly below a warp's first row need no causal test.
+// A CTA owns 128 (row, head) pairs: (128 / G) consecutive positions x the G retrieval heads of one index head.
+// The 16-dimensional scores q~ . k~ (Eq. 4) are one tcgen05.mma per 64-key cache page (M = 128 rows, N = 64 keys,
+// K = 16) into tensor memory; thread t of the four score warps owns row t = TMEM lane t and reads its 64 scores of a
+// page with tcgen05.ld, so a row's keys arrive at one thread in position order and all per-row state is private to it:
+//   warp 4    TMA: index-key pages -> shared memory (SWIZZLE_32B rows of 32 bytes), four stages
+//   warp 5    one lane issues the MMAs into two 64-column TMEM buffers
+//   warps 0-3 passes over the keys 0 .. last position, each row on its own:
+//     max      row maximum
+//     level 1  mass histogram over a fixed grid of score bins of width 1/4 (bin = round(-4 s) relative to the bin of
+//              the maximum; 64 bins, the last one pools everything below): the thread's private column of a
+//              [64 bins][128 rows] array in shared memory, fixed point (2^18 = the bin's upper end), plain
+//              load-add-store without atomics or bank conflicts; gives Z and the bin in which the cumulative mass
+//              reaches p * Z.  A crossing inside the pooled bin repeats the level with the window moved down.
+//     late     the keys of the chosen bin ("bucket") are appended to the row's list in global scratch, the keys
+//              above it are counted.  A bucket that may hold more keys than the list (long rows) is first narrowed
+//              by key levels: the list is used as a queue and drained into a 64-bin histogram of the next six key bits.
+//     finish   the warp narrows the list with the same 64-bin mass histogram until at most 64 keys are left and ranks
+//              those exactly by (score descending, position ascending); more than 64 equal scores at the cut take
+//              one more pass that finds the position of the last tie taken.
+//   When id lists are requested, one more sweep appends every row's members in position order.
+// Hand-offs are mbarriers with bounded waits (a wait that runs out records RTP_ERR_TIMEOUT and lets every later wait
+// fall through); the CTA always frees its tensor memory.
+#include <algorithm>
+#include <atomic>
+#include <cstdio>
 #include <cstdlib>
+
 #include "mass_hist.cuh"
+#include "tc_common.cuh"
 
 namespace rtp {
 
 namespace {
 
-constexpr int kCWarps = 8;
-constexpr int kCThreads = kCWarps * 32;
-constexpr int kCRows = 128;
-constexpr int kPagesPerStage = 4;
-constexpr int kStageKeys = kPagesPerStage * kPage;                  // 256 keys
-constexpr int kStageBytesC = kStageKeys * kIndexDim * 2;            // 8 KB
-constexpr int kCandCapC = 64;                                       // candidates ranked exactly per row
-constexpr int kCandCapG = 4096;                                     // candidates collected per row (global scratch), narrowed to kCandCapC in the warp
-constexpr int kRowBytes = kBins * 8 + 8;                            // per row: 64 x {sum, carries} or 64 x {key, idx}; +8 staggers the banks
-constexpr int kMaxPasses = 14;
+constexpr int kSRows = 128;
+constexpr int kSTile = kPage;                 // keys per MMA = one cache page
+constexpr int kSStages = 4;
+constexpr int kSThreads = 128;                // threads of one pipeline: thread = row
+constexpr int kTmemColsS = 128;               // two score buffers of 64 columns
+constexpr int kStageBytesS = kSTile * kIndexDim * 2;   // 2 KB
+constexpr int kCandCapC = 64;                 // candidates ranked exactly per row
+constexpr int kCandCapG = 8192;               // entries (unscaled score bits) of a row's list in global scratch
+constexpr int kMaxPasses = 24;
+constexpr int kMaxShift = 63 * 6;             // level-1 windows below this depth hold no representable mass
 constexpr float kLog2eC = kLog2eH;
-constexpr int kQueueCap = 288;                                      // per-warp queue of bucket hits (entries of 8 bytes)
+constexpr float kMagicC = 12582912.0f;        // 1.5 * 2^23: adding it leaves the nearest integer in the low mantissa bits
+constexpr uint32_t kMagicBits = 0x4B400000u;
+constexpr int kFixBits = 17;                  // fixed point of the private histograms: 2^17 = upper end of the bin
+// every key adds at least this to its bin (floor(e^-1/4 * 2^17) - 2), which bounds the number of keys by the sum
+constexpr float kMinQ18 = 102077.0f;
+constexpr float kMinQ11 = 1593.0f;            // the same for the 2^11 fixed point of the key-level histograms
+// A bin's 32-bit sum grows by at most 2^23 per page (64 keys x 2^17); every kNormEvery pages the sums above 2^30 hand
+// their upper bits to the bin's 8-bit counter (units of 2^30), so no add in between can wrap: 2^30 + 16 x 2^23 < 2^32.
+// 255 x 2^30 / 2^17 bounds a row at two million keys per bin.
+constexpr int kNormEvery = 16;
 
+constexpr int kHistOff = 0;                                  // u32 [64 bins][128 rows]
+constexpr int kCarryOff = kBins * kSRows * 4;                // u32 [16][128 rows]: four 8-bit wrap counters per word
+constexpr int kStageOffS = kCarryOff + 16 * kSRows * 4;      // kSStages x 2 KB
+constexpr int kAOff = kStageOffS + kSStages * kStageBytesS;  // projected queries [128 rows][16] bf16
+constexpr int kBarOffS = kAOff + kSRows * kIndexDim * 2;
+constexpr int kSubs = 4;                                     // independent pipelines per CTA
+constexpr int kSmemSub = (kBarOffS + 256 + 1023) & ~1023;    // shared memory of one sub
+constexpr int kSmemS = kSubs * kSmemSub;
+
+enum BarS { kFullK = 0, kSFull = kSStages, kNumBarsS = kSStages + 2 };
 enum Phase { kPhMax = 0, kPhL1 = 1, kPhKey = 2, kPhCollect = 3, kPhTie = 4, kPhDone = 5 };
+enum PassKind { kPassNone = 0, kPassMax = 1, kPassL1 = 2, kPassLate = 3, kPassEmit = 4 };
 
-struct RowState {      // one per (row, head), in shared memory
-  float M, Z, target, mass_above;
-  float ref_s;         // key levels: masses are accumulated relative to exp(ref_s - M) (upper end of the level-1 bucket)
-  float e_ref;         // exp(ref_s - M)
-  uint32_t base_key;   // bucket = keys in [base_key, base_key + span)
-  uint32_t span;
-  int32_t shift;       // key levels: bin = (key - base_key) >> shift, in [0, 64)
-  float raw_lo, raw_hi;   // unscaled-score interval of the bucket
-  int32_t phase;
-  int32_t cnt_above;   // keys strictly above the final bucket (counted in the collect pass)
-  int32_t cand_cnt;    // keys inside the final bucket (collect pass)
-  int32_t tie_need;    // tie pass: number of ties to take
-  uint32_t thr_key;    // result: selected <=> key > thr_key or (key == thr_key and n <= tie_last)
-  int32_t tie_last;
-  int32_t n_keys;
-  float sel_mass;
-  int32_t count;
-};
-
-constexpr int kHistBytes = kCRows * kRowBytes;                      // 64 KB
-constexpr int kQueueBytes = kCWarps * kQueueCap * 8;               // 18 KB
-constexpr int kSmemC = kHistBytes + 2 * kStageBytesC + kQueueBytes + kCRows * (int)sizeof(RowState);
-
-__device__ __forceinline__ void cp_async16c(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+  return v;
 }
-__device__ __forceinline__ uint32_t smem_u32c(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+
+// Private histogram column of a thread: bin b of the sums at col + 512 b, the 8-bit overflow counters (units of 2^30)
+// of bins 4w .. 4w+3 at ccol + 512 w.
+__device__ __forceinline__ void hist_add(uint32_t col, int bin, uint32_t q) {
+  const uint32_t a = col + (uint32_t)bin * (kSRows * 4);
+  sts32(a, lds32(a) + q);
 }
-
-// Per-lane view of its two rows for one pass (registers).
-struct LaneRows {
-  float M_a, M_b;
-  int pos_a, pos_b;
-  // Unscaled MMA outputs are compared directly: the keys of a bucket are the images of one closed interval of
-  // raw values (finish_score is monotone), found by bisection when the bucket is chosen.
-  float lo_a, hi_a, lo_b, hi_b;      // raw interval of the current bucket (empty: lo = +inf, hi = -inf)
-  float mid_a, hw_a, mid_b, hw_b;    // the same interval as centre and half width (slightly widened): 2-op reject
-  float cut_a, cut_b;                // collect pass: raw values above this are counted as above the bucket (+inf: none)
-  float tlo_a, thi_a, tlo_b, thi_b;  // tie pass: raw interval of the tied key value
-  float ref_a, ref_b;                // key levels: mass reference score
-  uint32_t base_a, base_b;
-  int shift_a, shift_b;
-  bool collect_a, collect_b;         // the bucket's keys are collected instead of histogrammed
-};
-
-// ---- one 64-key page, one warp ----------------------------------------------------------------------
-template <bool MASK>
-__device__ __forceinline__ void page_max(const unsigned char* pg, const QFrag& iq, int lane, int n_page,
-                                         const LaneRows& L, float& mx_a, float& mx_b) {
-  const int g = lane >> 2, c = lane & 3;
-  const int boff = 2 * qfrag_dim_offset(lane);
+// Moves the bits above 2^30 of every sum into the bin's counter.
+__device__ __noinline__ void hist_normalize(uint32_t col, uint32_t ccol) {
+  for (int w = 0; w < kBins / 4; ++w) {
+    uint32_t add = 0u;
 #pragma unroll
-  for (int nt = 0; nt < 8; ++nt) {
-    const uint2 b = *reinterpret_cast<const uint2*>(pg + (nt * 8 + g) * (kIndexDim * 2) + boff);
-    const float zero[4] = {0.f, 0.f, 0.f, 0.f};
-    float s4[4];
-    mma_bf16_16816(s4, iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
-    if (MASK) {
-      const int n0 = n_page + nt * 8 + 2 * c;
-      if (n0 > L.pos_a) s4[0] = -INFINITY;
-      if (n0 + 1 > L.pos_a) s4[1] = -INFINITY;
-      if (n0 > L.pos_b) s4[2] = -INFINITY;
-      if (n0 + 1 > L.pos_b) s4[3] = -INFINITY;
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t a = col + (uint32_t)(4 * w + k) * (kSRows * 4);
+      const uint32_t v = lds32(a);
+      if (v >> 30) {
+        add += (v >> 30) << (8 * k);
+        sts32(a, v & 0x3fffffffu);
+      }
     }
-    mx_a = fmaxf(mx_a, fmaxf(s4[0], s4[1]));
-    mx_b = fmaxf(mx_b, fmaxf(s4[2], s4[3]));
-  }
-}
-
-template <bool MASK>
-__device__ __forceinline__ void page_l1(const unsigned char* pg, const QFrag& iq, int lane, int n_page,
-                                        const LaneRows& L, float scale, uint32_t* hist_a, uint32_t* hist_b) {
-  const int g = lane >> 2, c = lane & 3;
-  const int boff = 2 * qfrag_dim_offset(lane);
-#pragma unroll
-  for (int nt = 0; nt < 8; ++nt) {
-    const uint2 b = *reinterpret_cast<const uint2*>(pg + (nt * 8 + g) * (kIndexDim * 2) + boff);
-    const float zero[4] = {0.f, 0.f, 0.f, 0.f};
-    float s4[4];
-    mma_bf16_16816(s4, iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
-    const int n0 = n_page + nt * 8 + 2 * c;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const bool lo = e < 2;
-      if (MASK && n0 + (e & 1) > (lo ? L.pos_a : L.pos_b)) continue;
-      const float s = s4[e] * scale;   // (the sign of a zero score does not matter here)
-      const float M = lo ? L.M_a : L.M_b;
-      float bin_f;
-      const int bin = l1_bin_f(M, s, bin_f);   // (rows that are already done have no M: they land in bin 0)
-      // mass relative to the bin's upper end: exp(-((M - s) - (bin/2 - 1/4))), scaled by 2^20
-      add_mass((lo ? hist_a : hist_b) + 2 * bin, l1_mass_arg(M, s, bin_f));
+    if (add) {
+      const uint32_t ca = ccol + (uint32_t)w * (kSRows * 4);
+      sts32(ca, lds32(ca) + add);
     }
   }
 }
+__device__ __forceinline__ float hist_read(uint32_t col, uint32_t ccol, int bin, bool& populated) {   // in units of 2^-17
+  const uint32_t sum = lds32(col + (uint32_t)bin * (kSRows * 4));
+  const uint32_t car = (lds32(ccol + (uint32_t)(bin >> 2) * (kSRows * 4)) >> ((bin & 3) * 8)) & 255u;
+  populated = (sum | car) != 0u;
+  return (float)car * 1073741824.0f + (float)sum;
+}
+// round(2^x) for x <= 17 (+ a rounding error) through the mantissa of 2^x + 2^23
+__device__ __forceinline__ uint32_t fix_q(float x) { return __float_as_uint(fast_ex2(x) + 8388608.0f) - 0x4b000000u; }
 
-// Key levels, candidate collection and (when TIE) the in-order tie count.  Rows that take no part carry empty
-// intervals, so no per-row branching is needed on the common path.
-template <bool MASK, bool TIE, bool COUNT>
-__device__ __forceinline__ void page_late(const unsigned char* pg, const QFrag& iq, int lane, int n_page,
-                                          const LaneRows& L, float scale, uint32_t* hist_a, uint32_t* hist_b,
-                                          int* ccnt_a, int* ccnt_b, uint2* gc_a, uint2* gc_b, int& cnt_a, int& cnt_b,
-                                          int need_a, int need_b, int& run_a, int& run_b, int& tl_a, int& tl_b) {
-  const int g = lane >> 2, c = lane & 3;
-  const int boff = 2 * qfrag_dim_offset(lane);
-#pragma unroll
-  for (int nt = 0; nt < 8; ++nt) {
-    const uint2 b = *reinterpret_cast<const uint2*>(pg + (nt * 8 + g) * (kIndexDim * 2) + boff);
-    const float zero[4] = {0.f, 0.f, 0.f, 0.f};
-    float s4[4];
-    mma_bf16_16816(s4, iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
-    const int n0 = n_page + nt * 8 + 2 * c;
-    if (MASK) {
-      const float nan = __int_as_float(0x7fc00000);   // fails every test below
-      if (n0 > L.pos_a) s4[0] = nan;
-      if (n0 + 1 > L.pos_a) s4[1] = nan;
-      if (n0 > L.pos_b) s4[2] = nan;
-      if (n0 + 1 > L.pos_b) s4[3] = nan;
+// Level-1 update of a thread's private histogram for two unscaled scores r0, r1 (bit patterns):
+//   s = r * scale;  t = min(fma(s, -4, dd), magic + 63)  (bin = low mantissa bits of t);
+//   q = round(2^(fma(t - magic, log2e / 4, fma(s, log2e, cx))))  through the mantissa of (2^x + 2^23);
+//   word at hb + 512 * bits(t) += q.
+__device__ __forceinline__ void l1_pair(uint32_t r0, uint32_t r1, float scale, float dd, float cx, uint32_t hb) {
+  asm volatile(
+      "{\n"
+      ".reg .f32 s0, s1, t0, t1, x0, x1, e0, e1;\n"
+      ".reg .u32 q0, q1, a0, a1, o0, o1, n0, n1;\n"
+      ".reg .pred pe;\n"
+      "mul.f32 s0, %0, %2;\n"
+      "mul.f32 s1, %1, %2;\n"
+      "fma.rn.f32 t0, s0, 0fC0800000, %3;\n"
+      "fma.rn.f32 t1, s1, 0fC0800000, %3;\n"
+      "min.f32 t0, t0, 0f4B40003F;\n"
+      "min.f32 t1, t1, 0f4B40003F;\n"
+      "fma.rn.f32 x0, s0, 0f3FB8AA3B, %4;\n"
+      "fma.rn.f32 x1, s1, 0f3FB8AA3B, %4;\n"
+      "sub.f32 e0, t0, 0f4B400000;\n"
+      "sub.f32 e1, t1, 0f4B400000;\n"
+      "fma.rn.f32 x0, e0, 0f3EB8AA3B, x0;\n"
+      "fma.rn.f32 x1, e1, 0f3EB8AA3B, x1;\n"
+      "ex2.approx.ftz.f32 e0, x0;\n"
+      "ex2.approx.ftz.f32 e1, x1;\n"
+      "add.f32 e0, e0, 0f4B000000;\n"
+      "add.f32 e1, e1, 0f4B000000;\n"
+      "mov.b32 q0, e0;\n"
+      "mov.b32 q1, e1;\n"
+      "mov.b32 a0, t0;\n"
+      "mov.b32 a1, t1;\n"
+      "mad.lo.u32 a0, a0, 512, %5;\n"
+      "mad.lo.u32 a1, a1, 512, %5;\n"
+      "ld.shared.u32 o0, [a0];\n"
+      "ld.shared.u32 o1, [a1];\n"
+      "add.u32 n0, o0, q0;\n"
+      "add.u32 n0, n0, 0xB5000000;\n"
+      "setp.eq.u32 pe, a0, a1;\n"
+      "selp.u32 o1, n0, o1, pe;\n"
+      "add.u32 n1, o1, q1;\n"
+      "add.u32 n1, n1, 0xB5000000;\n"
+      "st.shared.u32 [a0], n0;\n"
+      "st.shared.u32 [a1], n1;\n"
+      "}\n" ::"f"(__uint_as_float(r0)),
+      "f"(__uint_as_float(r1)), "f"(scale), "f"(dd), "f"(cx), "r"(hb)
+      : "memory");
+}
+
+// Late pass, collecting rows: counts a score above `cut` and queues a score inside [lo, hi] at shared address qa.
+__device__ __forceinline__ void late_one(uint32_t r, float cut, float lo, float hi, int& above, uint32_t& qa) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p0, p1;\n"
+      "setp.gt.f32 p0, %2, %3;\n"
+      "@p0 add.s32 %0, %0, 1;\n"
+      "setp.ge.f32 p1, %2, %4;\n"
+      "setp.le.and.f32 p1, %2, %5, p1;\n"
+      "@p1 st.shared.u32 [%1], %6;\n"
+      "@p1 add.u32 %1, %1, 512;\n"
+      "}\n"
+      : "+r"(above), "+r"(qa)
+      : "f"(__uint_as_float(r)), "f"(cut), "f"(lo), "f"(hi), "r"(r)
+      : "memory");
+}
+
+// Waits for the thread's tcgen05.ld results; the registers are operands so that no use of them moves above the wait.
+__device__ __forceinline__ void tmem_wait16(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :
+               : "memory");
+}
+__device__ __forceinline__ void red_add_shared(uint32_t a, uint32_t v) {
+  asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+
+// Grid bin of a score: round(-4 s) as an integer (monotone non-increasing in s; |s| < 2^18).
+__device__ __forceinline__ int grid_bin(float s) { return (int)(__float_as_uint(fmaf(s, -4.0f, kMagicC)) - kMagicBits); }
+
+// Exact interval [klo, khi] of ordered keys whose grid bin is `a`.
+__device__ void grid_bin_keys(int a, uint32_t& klo, uint32_t& khi) {
+  const float mid = -0.25f * (float)a;
+  const uint32_t lo = okey(mid - 0.5f), hi = okey(mid + 0.5f);   // safely outside the bin on both sides
+  uint32_t x = lo, y = hi;                 // klo = smallest key with grid_bin <= a
+  if (grid_bin(okey_to_float(x)) <= a) y = x;
+  while (x + 1 < y) {
+    const uint32_t m = x + ((y - x) >> 1);
+    if (grid_bin(okey_to_float(m)) <= a) y = m; else x = m;
+  }
+  klo = y;
+  x = klo; y = hi;                         // khi = largest key with grid_bin >= a
+  if (grid_bin(okey_to_float(y)) >= a) x = y;
+  while (x + 1 < y) {
+    const uint32_t m = x + ((y - x) >> 1);
+    if (grid_bin(okey_to_float(m)) >= a) x = m; else y = m;
+  }
+  khi = x;
+}
+
+// ---- exact finish of one row by a warp ---------------------------------------------------------------------------
+struct FinIn {
+  int n_all, above, n_keys;
+  float m_above, target, ref_s, e_ref, ref0, Z, scale;
+  uint32_t base, span;
+};
+struct FinOut {
+  int phase, cnt_above, count, tie_last, tie_need, bad;
+  float mass_above, sel_mass;
+  uint32_t thr_key;
+};
+
+// gc: the row's list of unscaled score bits (n_all entries, all inside the bucket [base, base + span) of ordered
+// keys); hw: 256 words of shared scratch of this warp.  Masses are relative to exp(ref0); target and m_above too.
+// The cut inside the bucket is found on score values alone: when it falls between keys of equal score, the first
+// `tie_need` of them in position order belong to the set and one more pass over the keys finds where that is.
+__device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* gc, uint32_t* hw, const int lane) {
+  FinOut o;
+  o.bad = 0;
+  o.tie_need = 0;
+  const int n_all = in.n_all;
+  int above = in.above;
+  float m_above = in.m_above;
+  uint32_t base = in.base, span = in.span;
+  int n_in = n_all;
+  auto key_of = [&](uint32_t raw_bits) { return okey(finish_score(__uint_as_float(raw_bits), in.scale)); };
+  // narrow on the list while more than kCandCapC candidates are left: 64-bin mass histogram over the next six key bits
+  while (n_in > kCandCapC && span > 1u) {
+    const int bits = 32 - __clz(span - 1u);
+    const int shift = max(0, bits - 6);
+    for (int i = lane; i < 2 * kBins; i += 32) hw[i] = 0u;
+    __syncwarp();
+    for (int i = lane; i < n_all; i += 32) {
+      const uint32_t key = key_of(__ldcg(gc + i));
+      const uint32_t t = key - base;
+      if (t < span) add_mass(hw + 2 * (t >> shift), fmaf(okey_to_float(key) - in.ref_s, kLog2eC, 20.0f));
     }
-    if (COUNT) {   // keys above the bucket of a row that is collecting
-      cnt_a += (s4[0] > L.cut_a) + (s4[1] > L.cut_a);
-      cnt_b += (s4[2] > L.cut_b) + (s4[3] > L.cut_b);
-    }
-    // quick reject: |raw - mid| <= hw is implied by raw in [lo, hi]
-    const bool near = fabsf(s4[0] - L.mid_a) <= L.hw_a || fabsf(s4[1] - L.mid_a) <= L.hw_a ||
-                      fabsf(s4[2] - L.mid_b) <= L.hw_b || fabsf(s4[3] - L.mid_b) <= L.hw_b;
-    int tf_a = 0, tf_b = 0;
-    if (near) {
+    __syncwarp();
+    const int b0 = 63 - 2 * lane, b1 = 62 - 2 * lane;   // bin 63 is the top
+    const uint32_t sum0 = hw[2 * b0], car0 = hw[2 * b0 + 1], sum1 = hw[2 * b1], car1 = hw[2 * b1 + 1];
+    const float sc = in.e_ref * 9.5367431640625e-07f;     // 2^-20
+    const float m0f = acc_mass(sum0, car0) * sc, m1f = acc_mass(sum1, car1) * sc;
+    float incm = m0f + m1f;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const bool lo = e < 2;
-        const float raw = s4[e];
-        if (raw >= (lo ? L.lo_a : L.lo_b) && raw <= (lo ? L.hi_a : L.hi_b)) {
-          if (TIE && (lo ? L.tlo_a : L.tlo_b) <= raw && raw <= (lo ? L.thi_a : L.thi_b)) {
-            if (lo) tf_a |= 1 << (e & 1); else tf_b |= 1 << (e & 1);
-            continue;
-          }
-          const float s = finish_score(raw, scale);
-          const uint32_t key = okey(s);
-          uint32_t* h = lo ? hist_a : hist_b;
-          if (lo ? L.collect_a : L.collect_b) {
-            const int slot = atomicAdd(lo ? ccnt_a : ccnt_b, 1);
-            if (slot < kCandCapG) (lo ? gc_a : gc_b)[slot] = make_uint2(key, (uint32_t)(n0 + (e & 1)));
-          } else {
-            const uint32_t t = key - (lo ? L.base_a : L.base_b);
-            add_mass(h + 2 * (t >> (lo ? L.shift_a : L.shift_b)), fmaf(s - (lo ? L.ref_a : L.ref_b), kLog2eC, 20.0f));
-          }
+    for (int ofs = 1; ofs < 32; ofs <<= 1) {
+      const float tm = __shfl_up_sync(0xffffffffu, incm, ofs);
+      if (lane >= ofs) incm += tm;
+    }
+    const float run = m_above + incm - (m0f + m1f);
+    int found = 64, last = -1;
+    if (sum0 | car0) {
+      last = 2 * lane;
+      if (run + m0f >= in.target) found = 2 * lane;
+    }
+    if (sum1 | car1) {
+      last = 2 * lane + 1;
+      if (found == 64 && run + m0f + m1f >= in.target) found = 2 * lane + 1;
+    }
+#pragma unroll
+    for (int ofs = 16; ofs > 0; ofs >>= 1) {
+      found = min(found, __shfl_xor_sync(0xffffffffu, found, ofs));
+      last = max(last, __shfl_xor_sync(0xffffffffu, last, ofs));
+    }
+    if (found == 64) found = last;
+    if (found < 0) break;                                 // (no candidate inside the interval: cannot happen)
+    m_above = __shfl_sync(0xffffffffu, (found & 1) ? run + m0f : run, found >> 1);
+    const uint32_t ofs_k = (uint32_t)(63 - found) << shift;
+    const uint32_t nbase = base + ofs_k, nspan = min(1u << shift, span - ofs_k);
+    int c_in = 0, c_up = 0;                               // candidates inside / above the new interval
+    for (int i = lane; i < n_all; i += 32) {
+      const uint32_t t = key_of(__ldcg(gc + i)) - base;
+      if (t < span) {
+        if (t - ofs_k < nspan) ++c_in;
+        else if (t >= ofs_k) ++c_up;
+      }
+    }
+#pragma unroll
+    for (int ofs = 16; ofs > 0; ofs >>= 1) {
+      c_in += __shfl_xor_sync(0xffffffffu, c_in, ofs);
+      c_up += __shfl_xor_sync(0xffffffffu, c_up, ofs);
+    }
+    above += c_up;
+    n_in = c_in;
+    base = nbase;
+    span = nspan;
+    __syncwarp();
+  }
+  // (thr_key, g = keys of the interval above it, eq = keys equal to it, m_gt = mass of the g keys, each = mass of one)
+  uint32_t thr_key = base;
+  int g = 0, eq = n_in;
+  float m_gt = 0.f, each = 0.f;
+  if (n_in > kCandCapC) {
+    // more than kCandCapC keys share one key value
+    each = fast_ex2((okey_to_float(base) - in.ref0) * kLog2eC);
+    if (span != 1u) o.bad = 1;
+  } else {
+    // the candidates of the final interval move into shared memory; each is compared with all the others
+    __syncwarp();
+    int filled = 0;
+    for (int i0 = 0; i0 < n_all; i0 += 32) {
+      const int i = i0 + lane;
+      uint32_t key = 0u;
+      bool inside = false;
+      if (i < n_all) {
+        key = key_of(__ldcg(gc + i));
+        inside = key - base < span;
+      }
+      const uint32_t m = __ballot_sync(0xffffffffu, inside);
+      if (inside) {
+        const int p = filled + __popc(m & ((1u << lane) - 1u));
+        if (p < kCandCapC) hw[p] = key;
+      }
+      filled += __popc(m);
+    }
+    __syncwarp();
+    const int n_c = min(n_in, kCandCapC);
+    if (n_c <= 0) o.bad = 1;   // a chosen bucket always holds a key
+    uint32_t key[2];
+    float e[2], mg[2] = {0.f, 0.f};
+    int gg[2] = {0, 0}, ee[2] = {0, 0};
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+      const int i = 2 * lane + x;
+      key[x] = i < n_c ? hw[i] : 0u;
+      e[x] = i < n_c ? fast_ex2((okey_to_float(key[x]) - in.ref0) * kLog2eC) : 0.f;
+    }
+    for (int j = 0; j < n_c; ++j) {
+      const uint32_t kj = __shfl_sync(0xffffffffu, (j & 1) ? key[1] : key[0], j >> 1);
+      const float ej = __shfl_sync(0xffffffffu, (j & 1) ? e[1] : e[0], j >> 1);
+#pragma unroll
+      for (int x = 0; x < 2; ++x) {
+        if (kj > key[x]) {
+          ++gg[x];
+          mg[x] += ej;
+        } else if (kj == key[x]) {
+          ++ee[x];
         }
       }
     }
-    if (TIE) {
-      // in-order prefix of the tied keys inside the quad (lane c holds keys 2c, 2c+1 of the n8 tile)
-      const int ka = __popc(tf_a), kb = __popc(tf_b);
-      int ia = ka, ib = kb, t;
-      t = __shfl_up_sync(0xffffffffu, ia, 1, 4); if (c >= 1) ia += t;
-      t = __shfl_up_sync(0xffffffffu, ia, 2, 4); if (c >= 2) ia += t;
-      t = __shfl_up_sync(0xffffffffu, ib, 1, 4); if (c >= 1) ib += t;
-      t = __shfl_up_sync(0xffffffffu, ib, 2, 4); if (c >= 2) ib += t;
-      const int tot_a = __shfl_sync(0xffffffffu, ia, 3, 4), tot_b = __shfl_sync(0xffffffffu, ib, 3, 4);
-      int before = run_a + ia - ka;
+    // the largest key whose group completes the target (the smallest key if rounding leaves the target out of reach)
+    unsigned long long best = 0ull, lowest = ~0ull;
 #pragma unroll
-      for (int e = 0; e < 2; ++e)
-        if (tf_a & (1 << e)) { if (before < need_a) tl_a = max(tl_a, n0 + e); ++before; }
-      before = run_b + ib - kb;
+    for (int x = 0; x < 2; ++x)
+      if (2 * lane + x < n_c) {
+        const unsigned long long id = ((unsigned long long)key[x] << 8) | (unsigned long long)(2 * lane + x);
+        if (m_above + mg[x] + (float)ee[x] * e[x] >= in.target) best = max(best, id);
+        lowest = min(lowest, id);
+      }
 #pragma unroll
-      for (int e = 0; e < 2; ++e)
-        if (tf_b & (1 << e)) { if (before < need_b) tl_b = max(tl_b, n0 + e); ++before; }
-      run_a += tot_a;
-      run_b += tot_b;
+    for (int ofs = 16; ofs > 0; ofs >>= 1) {
+      best = max(best, __shfl_xor_sync(0xffffffffu, best, ofs));
+      lowest = min(lowest, __shfl_xor_sync(0xffffffffu, lowest, ofs));
     }
+    if (best == 0ull) best = lowest;
+    const int src = (int)(best & 255ull);
+    const int sl = (src >> 1) & 31, sx = src & 1;
+    thr_key = __shfl_sync(0xffffffffu, sx ? key[1] : key[0], sl);
+    g = __shfl_sync(0xffffffffu, sx ? gg[1] : gg[0], sl);
+    eq = __shfl_sync(0xffffffffu, sx ? ee[1] : ee[0], sl);
+    m_gt = __shfl_sync(0xffffffffu, sx ? mg[1] : mg[0], sl);
+    each = __shfl_sync(0xffffffffu, sx ? e[1] : e[0], sl);
+    __syncwarp();
   }
+  const float cum = m_above + m_gt;
+  int take = eq;   // (a key too light to register in fp32 cannot split its group)
+  if (each > 0.f) take = (int)fminf(ceilf((in.target - cum) / each), (float)eq);
+  take = max(1, min(take, eq));
+  o.cnt_above = above;
+  o.mass_above = cum;
+  o.thr_key = thr_key;
+  o.count = above + g + take;
+  o.sel_mass = (cum + (float)take * each) / in.Z;
+  if (take < eq) {
+    o.tie_need = take;
+    o.tie_last = -1;
+    o.phase = kPhTie;
+  } else {
+    o.tie_last = in.n_keys - 1;
+    o.phase = kPhDone;
+  }
+  return o;
 }
 
-// Works off the warp's queue of bucket hits: entry = {position | local row << 27, raw score bits}.
-// (The count is passed by value: a reference would pin the caller's counter to local memory.)
-__device__ __noinline__ void drain_hits(uint32_t* wq, int qcnt, int lane, int wrow, RowState* rs, uint32_t* hist,
-                                        uint2* gcand, float scale) {
-  constexpr int kRowWords = kRowBytes / 4;
-  __syncwarp();
-  for (int base = 0; base < qcnt; base += 32) {
-    const int i = base + lane;
-    if (i < qcnt) {
-      const uint32_t w0 = wq[2 * i];
-      const float raw = __uint_as_float(wq[2 * i + 1]);
-      const int r = wrow + (int)(w0 >> 27);
-      RowState* S = rs + r;
-      const float s = finish_score(raw, scale);
-      const uint32_t key = okey(s);
-      uint32_t* h = hist + r * kRowWords;
-      if (S->phase == kPhCollect) {
-        const int slot = atomicAdd(&S->cand_cnt, 1);
-        if (slot < kCandCapG) gcand[(size_t)r * kCandCapG + slot] = make_uint2(key, w0 & 0x7ffffffu);
-      } else {
-        const uint32_t t = key - S->base_key;
-        add_mass(h + 2 * (t >> S->shift), fmaf(s - S->ref_s, kLog2eC, 20.0f));
-      }
-    }
-  }
-  __syncwarp();
-}
-
-// Key levels and candidate collection without ties: hits go to the warp's queue.
-template <bool MASK, bool COUNT>
-__device__ __forceinline__ void page_hits(const unsigned char* pg, const QFrag& iq, int lane, int n_page,
-                                          const LaneRows& L, int& cnt_a, int& cnt_b, uint32_t* wq, int& qcnt,
-                                          int wrow, RowState* rs, uint32_t* hist, uint2* gcand, float scale) {
-  const int g = lane >> 2, c = lane & 3;
-  const int boff = 2 * qfrag_dim_offset(lane);
-  // Four 8-key groups at a time: their MMAs and interval tests are issued back to back, and one vote decides whether
-  // any of the 512 scores is a hit (the usual answer in the later passes is no).
-#pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    float s[4][4];
-    uint32_t hits = 0;   // bit 4 q + e: score e of group q is inside its row's bucket
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int nt = half * 4 + q;
-      const uint2 b = *reinterpret_cast<const uint2*>(pg + (nt * 8 + g) * (kIndexDim * 2) + boff);
-      const float zero[4] = {0.f, 0.f, 0.f, 0.f};
-      mma_bf16_16816(s[q], iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
-    }
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int n0 = n_page + (half * 4 + q) * 8 + 2 * c;
-      if (MASK) {
-        const float nan = __int_as_float(0x7fc00000);   // fails every test below
-        if (n0 > L.pos_a) s[q][0] = nan;
-        if (n0 + 1 > L.pos_a) s[q][1] = nan;
-        if (n0 > L.pos_b) s[q][2] = nan;
-        if (n0 + 1 > L.pos_b) s[q][3] = nan;
-      }
-      if (COUNT) {   // keys above the bucket of a row that is collecting
-        cnt_a += (s[q][0] > L.cut_a) + (s[q][1] > L.cut_a);
-        cnt_b += (s[q][2] > L.cut_b) + (s[q][3] > L.cut_b);
-      }
-      if (s[q][0] >= L.lo_a && s[q][0] <= L.hi_a) hits |= 1u << (4 * q);
-      if (s[q][1] >= L.lo_a && s[q][1] <= L.hi_a) hits |= 2u << (4 * q);
-      if (s[q][2] >= L.lo_b && s[q][2] <= L.hi_b) hits |= 4u << (4 * q);
-      if (s[q][3] >= L.lo_b && s[q][3] <= L.hi_b) hits |= 8u << (4 * q);
-    }
-    if (!__any_sync(0xffffffffu, hits != 0u)) continue;
-    // every lane appends its hits behind those of the lower lanes: a prefix sum over the lanes' hit counts, then
-    // predicated stores (no vote per score); two 8-key groups at a time bound the queue growth by 256 entries
-#pragma unroll
-    for (int pr = 0; pr < 2; ++pr) {
-      const uint32_t hb = (hits >> (8 * pr)) & 0xffu;
-      const int mine = __popc(hb);
-      int incl = mine;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-      }
-      int pos = qcnt + incl - mine;
-      qcnt += __shfl_sync(0xffffffffu, incl, 31);
-#pragma unroll
-      for (int qq = 0; qq < 2; ++qq) {
-        const int q = 2 * pr + qq;
-        const int n0 = n_page + (half * 4 + q) * 8 + 2 * c;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if ((hb >> (4 * qq + e)) & 1u) {
-            wq[2 * pos] = (uint32_t)(n0 + (e & 1)) | ((uint32_t)(g + (e >> 1) * 8) << 27);
-            wq[2 * pos + 1] = __float_as_uint(s[q][e]);
-            ++pos;
-          }
-        }
-      }
-      if (qcnt >= 32) {   // at most 31 + 256 entries queued
-        drain_hits(wq, qcnt, lane, wrow, rs, hist, gcand, scale);
-        qcnt = 0;
-      }
-    }
-  }
-}
+// One page of the pass: wait for its scores in tensor memory ... release the buffer.  The last of the four warps to
+// release it (ticket counter in shared memory; nobody waits for anybody) hands the buffer to the page two ahead: it
+// issues that page's MMA (its keys were requested kSStages pages earlier) and requests the keys of the page kSStages
+// ahead, whose stage the completed MMA of this page has freed.
+#define RTP_SEL_TILE_BEGIN                                                              \
+  const int buf = (int)(gt & 1u);                                                       \
+  mbar_wait(bar(kSFull + buf), (gt >> 1) & 1u, abort_flag, status);                     \
+  tc_fence_after();                                                                     \
+  const int n_base = it * kSTile;                                                       \
+  const bool interior = n_base + kSTile - 1 <= min_pos;                                 \
+  const uint32_t taddr = tmem + lane_addr + (uint32_t)(buf * kSTile);
+#define RTP_SEL_TILE_END                                                                \
+  tc_fence_before();                                                                    \
+  __syncwarp();                                                                         \
+  if (lane == 0) {                                                                      \
+    __threadfence_block();                                                              \
+    if (atomicAdd(&rel[buf], 1u) == 3u) {                                               \
+      rel[buf] = 0u;                                                                    \
+      tc_fence_after();                                                                 \
+      if (it + 2 < n_tiles) issue_mma(gt + 2u);                                         \
+      if (it + kSStages < n_tiles) issue_tma(gt + (uint32_t)kSStages, it + kSStages);   \
+    }                                                                                   \
+  }                                                                                     \
+  __syncwarp();                                                                         \
+  ++gt;
 
 template <int G>
-__global__ void __launch_bounds__(kCThreads, 2) select_chunk_kernel(
-    const CacheView cv, const Dims d, const HeadMaps hm, const __nv_bfloat16* __restrict__ qt,
-    const int seq_id, const int q_start, const int C, int32_t* __restrict__ sel_idx, const int64_t sel_stride,
-    int32_t* __restrict__ sel_count, float* __restrict__ sel_mass, float* __restrict__ sel_thresh,
-    int32_t* __restrict__ sel_tie_last, int32_t* status, uint2* __restrict__ gcand_all, const int n_row_tiles,
-    const int max_passes) {
-  constexpr int BMP = kCRows / G;
-  // candidate scratch of this CTA: [128 rows][kCandCapG] {ordered key, position}
-  uint2* gcand = gcand_all + ((size_t)blockIdx.y * gridDim.x + blockIdx.x) * (size_t)(kCRows * kCandCapG);
-  extern __shared__ __align__(128) unsigned char smem[];
-  uint32_t* hist = reinterpret_cast<uint32_t*>(smem);                      // [128 rows][128 words]
-  unsigned char* stage_s = smem + kHistBytes;
-  uint32_t* queue = reinterpret_cast<uint32_t*>(smem + kHistBytes + 2 * kStageBytesC);
-  RowState* rs = reinterpret_cast<RowState*>(smem + kHistBytes + 2 * kStageBytesC + kQueueBytes);
-  __shared__ int s_pending;
-  constexpr int kRowWords = kRowBytes / 4;
+__global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
+    const __grid_constant__ CUtensorMap map_ik, const CacheView cv, const Dims d, const HeadMaps hm,
+    const __nv_bfloat16* __restrict__ qt, const int seq_id, const int q_start, const int C,
+    int32_t* __restrict__ sel_idx, const int64_t sel_stride, int32_t* __restrict__ sel_count,
+    float* __restrict__ sel_mass, float* __restrict__ sel_thresh, int32_t* __restrict__ sel_tie_last, int32_t* status,
+    uint32_t* __restrict__ gcand_all, const int n_row_tiles, const int max_passes) {
+  constexpr int BMP = kSRows / G;
+  extern __shared__ __align__(1024) unsigned char smem_all[];
+  // A kernel that uses tensor memory runs one CTA per SM, so the CTA holds kSubs independent pipelines ("subs") of
+  // kSThreads threads, each with its own slice of shared memory, its own 128 TMEM columns and its own named barrier.
+  const int sub = threadIdx.x / kSThreads;
+  const int tid = threadIdx.x - sub * kSThreads, lane = tid & 31, warp = tid >> 5;
+  unsigned char* smem = smem_all + sub * kSmemSub;
+  const uint32_t sbase = s_u32(smem);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_all + kBarOffS + kNumBarsS * 8);   // (sub 0's slot serves the CTA)
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kBarOffS + kNumBarsS * 8 + 4);
+  volatile int* pass_flags = reinterpret_cast<volatile int*>(smem + kBarOffS + kNumBarsS * 8 + 8);   // [2]
+  unsigned int* rel = reinterpret_cast<unsigned int*>(smem + kBarOffS + kNumBarsS * 8 + 16);         // [2] release tickets
+  auto bar = [&](int i) { return sbase + kBarOffS + i * 8; };
+  auto sub_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(1 + sub), "r"(kSThreads) : "memory"); };
+  const int seq_len = cv.seq_lens[seq_id];
+  const bool want_ids = sel_idx != nullptr;
+  const float scale = d.score_scale;
+  const int n_units = n_row_tiles * d.n_ih;
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int g = lane >> 2, c = lane & 3;
-  const int tile = n_row_tiles - 1 - blockIdx.x;
-  const int ih = blockIdx.y;
+  if (tid == 0) {
+    for (int i = 0; i < kSStages; ++i) mbar_init(bar(kFullK + i), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(kSFull + i), 1);
+      rel[i] = 0u;
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (threadIdx.x < 32) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(tmem_slot)), "r"(kSubs * kTmemColsS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_cta = *tmem_slot;
+  const uint32_t tmem = tmem_cta + (uint32_t)(sub * kTmemColsS);
+  // a warp reaches the 32 TMEM lanes of its quarter (warp index within the CTA modulo 4): the four score warps of a
+  // sub are consecutive warps of the CTA, so they cover the four quarters in some rotation
+  const int quarter = (int)(threadIdx.x >> 5) & 3;
+  const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+  const int row = quarter * 32 + lane;
+  const uint32_t hist_col = sbase + kHistOff + (uint32_t)row * 4u;
+  const uint32_t carry_col = sbase + kCarryOff + (uint32_t)row * 4u;
+
+  uint32_t gt = 0;               // key tiles consumed so far by this role (all roles of a sub walk the same sequence)
+  // units (row tile, index head) in order of decreasing length, dealt round-robin to the SMs and then to their subs
+  for (int unit = blockIdx.x + (int)gridDim.x * sub; unit < n_units; unit += (int)gridDim.x * kSubs) {
+  const int tile = n_row_tiles - 1 - unit / d.n_ih;
+  const int ih = unit % d.n_ih;
   const int nh = hm.ih_nheads[ih];
   const int r0 = tile * BMP;
   const int rows_here = min(BMP, C - r0);
   const int m0 = q_start + r0;
-  const int seq_len = cv.seq_lens[seq_id];
   const int m_last = min(m0 + rows_here - 1, seq_len - 1);
+  const int n_tiles = m_last >= 0 ? (m_last >> kPageShift) + 1 : 0;
+  const int min_pos = min(m0, seq_len - 1);
+  sub_sync();                    // the previous unit is finished by every thread of the sub
+  if (tid == 0) {
+    pass_flags[0] = 0;
+    pass_flags[1] = 0;
+    if (m0 + rows_here - 1 >= seq_len) set_status(status, RTP_ERR_INVALID);
+  }
+  sub_sync();
 
-  const int wrow = warp * 16;
-  const int hslot = wrow / BMP, pofs = wrow % BMP;
-  const bool warp_has_head = hslot < nh;
-  const int rh_head = warp_has_head ? hm.ih_heads[ih][hslot] : 0;
-  // the two rows of this lane: local ids la, lb in [0,128)
-  const int la = wrow + g, lb = la + 8;
-  const bool a_ok = warp_has_head && pofs + g < rows_here;
-  const bool b_ok = warp_has_head && pofs + g + 8 < rows_here;
-  const int pos_a = min(m0 + pofs + g, seq_len - 1), pos_b = min(m0 + pofs + g + 8, seq_len - 1);
-  if (tid == 0 && m0 + rows_here - 1 >= seq_len) set_status(status, RTP_ERR_INVALID);
-  const int warp_m_lo = min(m0 + pofs, seq_len - 1);
-  const int warp_m_hi = min(m0 + pofs + 15, m_last);
-  const bool warp_ok = warp_has_head && pofs < rows_here;
-
-  // projected queries of the warp's rows
-  QFrag iq = {0u, 0u, 0u, 0u};
+  // ---- per-row state of the score threads (registers) ----
+  const int hs = row / BMP, po = row % BMP;
+  const bool row_ok = hs < nh && po < rows_here;
+  const int rh_head = hs < nh ? hm.ih_heads[ih][hs] : 0;
+  const int pos = min(m0 + po, seq_len - 1);
+  const int n_keys = row_ok ? pos + 1 : 0;
+  int phase = kPhDone;
+  uint32_t thr_key = 0u;
+  int tie_last = -1, count = 0;
+  float sel_m = 0.f;
+  if (row_ok && n_keys > 0) {
+    phase = kPhMax;
+    if (d.top_p >= 1.0f || n_keys == 1) {   // everything is selected
+      phase = kPhDone;
+      tie_last = n_keys - 1;
+      count = n_keys;
+      sel_m = 1.0f;
+    }
+  }
   {
-    const int off = qfrag_dim_offset(lane);
-    if (a_ok) {
-      const uint2 v = *reinterpret_cast<const uint2*>(qt + ((int64_t)(r0 + pofs + g) * d.n_ret + rh_head) * kIndexDim + off);
-      iq.a0 = v.x;
-      iq.a2 = v.y;
+    // projected queries of the unit's rows -> the A operand (rows of 32 bytes, SWIZZLE_32B: the two 16-byte halves of
+    // rows 4-7 of every 8-row group are exchanged)
+    uint4 v0 = make_uint4(0u, 0u, 0u, 0u), v1 = v0;
+    if (row_ok) {
+      const uint4* src = reinterpret_cast<const uint4*>(qt + ((int64_t)(r0 + po) * d.n_ret + rh_head) * kIndexDim);
+      v0 = __ldg(src);
+      v1 = __ldg(src + 1);
     }
-    if (b_ok) {
-      const uint2 v = *reinterpret_cast<const uint2*>(qt + ((int64_t)(r0 + pofs + g + 8) * d.n_ret + rh_head) * kIndexDim + off);
-      iq.a1 = v.x;
-      iq.a3 = v.y;
-    }
+    const int sw = (row >> 2) & 1;
+    *reinterpret_cast<uint4*>(smem + kAOff + row * 32 + ((0 ^ sw) << 4)) = v0;
+    *reinterpret_cast<uint4*>(smem + kAOff + row * 32 + ((1 ^ sw) << 4)) = v1;
+    fence_async_smem();
+    if (phase != kPhDone) atomicOr(const_cast<int*>(&pass_flags[0]), 1 << kPhMax);
   }
-  if (tid < kCRows) {
-    RowState z = {};
-    const int hs = tid / BMP, po = tid % BMP;
-    const bool ok = hs < nh && po < rows_here;
-    z.n_keys = ok ? min(m0 + po, seq_len - 1) + 1 : 0;
-    z.phase = ok && z.n_keys > 0 ? kPhMax : kPhDone;
-    if (ok && z.n_keys > 0 && (d.top_p >= 1.0f || z.n_keys == 1)) {   // everything is selected
-      z.phase = kPhDone;
-      z.thr_key = 0u;
-      z.tie_last = z.n_keys - 1;
-      z.count = z.n_keys;
-      z.sel_mass = 1.0f;
-    }
-    rs[tid] = z;
-  }
-  __syncthreads();
+  sub_sync();
+  uint32_t* gc = gcand_all + (size_t)unit * (size_t)(kSRows * kCandCapG) + (size_t)row * kCandCapG;
 
-  const int n_pages = (m_last >> kPageShift) + 1;
-  const int n_stages = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
+  // level 1
+  int aI = 0, w0 = 0;            // grid bin of the maximum; offset of the current 64-bin window below it
+  float ref0 = 0.f;              // score of the upper end of the maximum's bin: every mass is relative to exp(ref0)
+  float Z = 0.f, target = 0.f, mass_above = 0.f;
+  bool have_z = false;
+  // bucket
+  uint32_t base_key = 0u, span = 0u;
+  int shift = 0;
+  float raw_lo = __int_as_float(0x7f800000), raw_hi = -__int_as_float(0x7f800000);
+  float ref_s = 0.f, e_ref = 0.f;
+  int cnt_above = 0, cand_cnt = 0, tie_need = 0, tie_run = 0;
+
+  // page `page` of the current pass, the g-th page this pipeline has walked since the kernel started: stage g % kSStages
   const int64_t bt_base = (int64_t)seq_id * cv.max_pages;
-  auto load_stage = [&](int sidx, int buf) {
-    // 512 chunks of 16 bytes: page = chunk / 128
-#pragma unroll
-    for (int x = 0; x < 2; ++x) {
-      const int ch = tid + x * kCThreads;
-      const int pg = sidx * kPagesPerStage + (ch >> 7);
-      if (pg < n_pages) {
-        const int phys = __ldg(cv.block_table + bt_base + pg);
-        const __nv_bfloat16* src = cv.ikey + ((int64_t)phys * cv.n_ih + ih) * (kPage * kIndexDim) + (ch & 127) * 8;
-        cp_async16c(smem_u32c(stage_s + buf * kStageBytesC + ch * 16), src);
-      }
-    }
+  auto issue_tma = [&](uint32_t g, int page) {
+    const int stage = (int)(g % kSStages);
+    const int phys = __ldg(cv.block_table + bt_base + page);
+    mbar_expect_tx(bar(kFullK + stage), kStageBytesS);
+    tma_load_2d(sbase + kStageOffS + stage * kStageBytesS, &map_ik, 0, (phys * cv.n_ih + ih) * kPage, bar(kFullK + stage));
   };
-
-  const bool want_ids = sel_idx != nullptr;
-  uint32_t* hist_a = hist + la * kRowWords;
-  uint32_t* hist_b = hist + lb * kRowWords;
-  const float scale = d.score_scale;
-  const float kInf = __int_as_float(0x7f800000);
-
+  auto issue_mma = [&](uint32_t g) {
+    const int stage = (int)(g % kSStages), b2 = (int)(g & 1u);
+    mbar_wait(bar(kFullK + stage), (g / kSStages) & 1u, abort_flag, status);
+    tc_fence_after();
+    tc_mma(tmem + (uint32_t)(b2 * kSTile), smem_desc_sw(sbase + kAOff, 16, 256, 6),
+           smem_desc_sw(sbase + kStageOffS + stage * kStageBytesS, 16, 256, 6), instr_desc_mn(kSRows, kSTile, false), 0u);
+    tc_commit(bar(kSFull + b2));
+  };
+  int done_emit = 0;
   for (int pass = 0; pass < max_passes; ++pass) {
-    // ---- what does this pass do for my two rows? ----
-    const RowState sa = rs[la], sb = rs[lb];
-    const int ph_a = a_ok ? sa.phase : kPhDone, ph_b = b_ok ? sb.phase : kPhDone;
-    if (tid == 0) s_pending = 0;
-    for (int i = lane; i < 16 * kRowWords; i += 32) hist[wrow * kRowWords + i] = 0u;   // this warp's rows
-    __syncthreads();
-    const bool warp_active = __any_sync(0xffffffffu, ph_a != kPhDone || ph_b != kPhDone);
-    // All rows of a warp do the max pass and the level-1 pass together; later passes mix key levels,
-    // candidate collection and ties.
-    const bool pass_max = __any_sync(0xffffffffu, ph_a == kPhMax || ph_b == kPhMax);
-    const bool pass_l1 = __any_sync(0xffffffffu, ph_a == kPhL1 || ph_b == kPhL1);
-    const bool pass_tie = __any_sync(0xffffffffu, ph_a == kPhTie || ph_b == kPhTie);
-    const bool pass_count = __any_sync(0xffffffffu, ph_a == kPhCollect || ph_b == kPhCollect);
-
-    LaneRows LR;
-    LR.M_a = sa.M; LR.M_b = sb.M;
-    LR.pos_a = pos_a; LR.pos_b = pos_b;
-    LR.base_a = sa.base_key; LR.base_b = sb.base_key;
-    LR.shift_a = sa.shift; LR.shift_b = sb.shift;
-    LR.ref_a = sa.ref_s; LR.ref_b = sb.ref_s;
-    const bool in_a = ph_a == kPhKey || ph_a == kPhCollect || ph_a == kPhTie;
-    const bool in_b = ph_b == kPhKey || ph_b == kPhCollect || ph_b == kPhTie;
-    LR.lo_a = in_a ? sa.raw_lo : kInf;  LR.hi_a = in_a ? sa.raw_hi : -kInf;
-    LR.lo_b = in_b ? sb.raw_lo : kInf;  LR.hi_b = in_b ? sb.raw_hi : -kInf;
-    // centre / half width of the interval; the half width is rounded up so that the quick test never rejects a member
-    LR.mid_a = in_a ? 0.5f * sa.raw_lo + 0.5f * sa.raw_hi : 0.f;
-    LR.mid_b = in_b ? 0.5f * sb.raw_lo + 0.5f * sb.raw_hi : 0.f;
-    LR.hw_a = in_a ? fmaxf(sa.raw_hi - LR.mid_a, LR.mid_a - sa.raw_lo) * 1.000001f + 1e-30f : -1.f;
-    LR.hw_b = in_b ? fmaxf(sb.raw_hi - LR.mid_b, LR.mid_b - sb.raw_lo) * 1.000001f + 1e-30f : -1.f;
-    LR.collect_a = ph_a == kPhCollect;  LR.collect_b = ph_b == kPhCollect;
-    LR.cut_a = LR.collect_a ? sa.raw_hi : kInf;
-    LR.cut_b = LR.collect_b ? sb.raw_hi : kInf;
-    const bool tie_a = ph_a == kPhTie, tie_b = ph_b == kPhTie;
-    LR.tlo_a = tie_a ? sa.raw_lo : kInf;  LR.thi_a = tie_a ? sa.raw_hi : -kInf;
-    LR.tlo_b = tie_b ? sb.raw_lo : kInf;  LR.thi_b = tie_b ? sb.raw_hi : -kInf;
-    const int need_a = tie_a ? sa.tie_need : 0, need_b = tie_b ? sb.tie_need : 0;
-    int* ccnt_a = &rs[la].cand_cnt;
-    int* ccnt_b = &rs[lb].cand_cnt;
-
-    float mx_a = -INFINITY, mx_b = -INFINITY;
-    int cnt_a = 0, cnt_b = 0;
-    int run_a = 0, run_b = 0;
-    int tl_a = -1, tl_b = -1;
-    uint32_t* wq = queue + warp * (kQueueCap * 2);
-    int qcnt = 0;
-
-    load_stage(0, 0);
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    for (int sidx = 0; sidx < n_stages; ++sidx) {
-      const int buf = sidx & 1;
-      if (sidx + 1 < n_stages) load_stage(sidx + 1, buf ^ 1);
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      asm volatile("cp.async.wait_group 1;" ::: "memory");
-      __syncthreads();
-      if (warp_active && warp_ok) {
-        const unsigned char* st = stage_s + buf * kStageBytesC;
-#pragma unroll 1
-        for (int pg = 0; pg < kPagesPerStage; ++pg) {
-          const int n_page = (sidx * kPagesPerStage + pg) * kPage;
-          if (n_page > warp_m_hi) break;
-          const unsigned char* pgp = st + pg * (kPage * kIndexDim * 2);
-          const bool interior = n_page + kPage - 1 <= warp_m_lo;   // every key visible to every row of the warp
-          if (pass_max) {
-            if (interior) page_max<false>(pgp, iq, lane, n_page, LR, mx_a, mx_b);
-            else page_max<true>(pgp, iq, lane, n_page, LR, mx_a, mx_b);
-          } else if (pass_l1) {
-            if (interior) page_l1<false>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b);
-            else page_l1<true>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b);
-          } else {
-#define RTP_LATE(M_, T_, C_) page_late<M_, T_, C_>(pgp, iq, lane, n_page, LR, scale, hist_a, hist_b, ccnt_a, ccnt_b, gcand + (size_t)la * kCandCapG, gcand + (size_t)lb * kCandCapG, cnt_a, cnt_b, need_a, need_b, run_a, run_b, tl_a, tl_b)
-#define RTP_HITS(M_, C_) page_hits<M_, C_>(pgp, iq, lane, n_page, LR, cnt_a, cnt_b, wq, qcnt, wrow, rs, hist, gcand, scale)
-            if (pass_tie) {
-              if (interior) RTP_LATE(false, true, true); else RTP_LATE(true, true, true);
-            } else if (pass_count) {
-              if (interior) RTP_HITS(false, true); else RTP_HITS(true, true);
-            } else {
-              if (interior) RTP_HITS(false, false); else RTP_HITS(true, false);
-            }
-#undef RTP_LATE
-#undef RTP_HITS
-          }
-        }
-      }
-      __syncthreads();
+    const int flags = pass_flags[pass & 1];
+    int kind = (flags & (1 << kPhMax)) ? kPassMax : (flags & (1 << kPhL1)) ? kPassL1 : (flags & ~(1 << kPhDone)) ? kPassLate : kPassNone;
+    if (kind == kPassNone && want_ids && !done_emit) {
+      kind = kPassEmit;
+      done_emit = 1;
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (qcnt > 0) drain_hits(wq, qcnt, lane, wrow, rs, hist, gcand, scale);
-    qcnt = 0;
+    if (kind == kPassNone || n_tiles == 0) break;
 
-    // ---- end of pass: combine the quad's partial results ----
-    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
-    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
-    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
-    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
-    cnt_a += __shfl_xor_sync(0xffffffffu, cnt_a, 1);
-    cnt_a += __shfl_xor_sync(0xffffffffu, cnt_a, 2);
-    cnt_b += __shfl_xor_sync(0xffffffffu, cnt_b, 1);
-    cnt_b += __shfl_xor_sync(0xffffffffu, cnt_b, 2);
-    tl_a = max(tl_a, __shfl_xor_sync(0xffffffffu, tl_a, 1));
-    tl_a = max(tl_a, __shfl_xor_sync(0xffffffffu, tl_a, 2));
-    tl_b = max(tl_b, __shfl_xor_sync(0xffffffffu, tl_b, 1));
-    tl_b = max(tl_b, __shfl_xor_sync(0xffffffffu, tl_b, 2));
-    __syncwarp();
-
-    // Each of the warp's 16 rows is resolved by the whole warp in turn (bins spread over the lanes).
-    // Every lane first copies the row state, then the warp synchronises, then one lane writes.
-    for (int rr = 0; rr < 16; ++rr) {
-      const int lr = wrow + rr;
-      RowState* S = rs + lr;
-      const RowState R = *S;
-      __syncwarp();
-      const int ph = R.phase;
-      const int src_lane = (rr & 7) * 4;          // a lane of the quad that owns row rr
-      const bool is_b = rr >= 8;
-      const uint32_t* h = hist + lr * kRowWords;
-      if (ph == kPhDone || R.n_keys == 0) continue;
-      if (ph == kPhMax) {
-        // the maximum was taken on unscaled MMA outputs; scaling by a positive factor is monotone
-        const float M = finish_score(__shfl_sync(0xffffffffu, is_b ? mx_b : mx_a, src_lane), scale);
-        if (lane == 0) {
-          S->M = M;
-          S->phase = kPhL1;
-        }
-      } else if (ph == kPhL1 || ph == kPhKey) {
-        // 64 bins of {hi, lo}; two bins per lane in order of decreasing score:
-        //   level 1: bin 0 is the top -> lane l takes bins 2l, 2l+1;  key levels: bin 63 is the top -> 63-2l, 62-2l
-        const bool l1 = ph == kPhL1;
-        const int b0 = l1 ? 2 * lane : 63 - 2 * lane, b1 = l1 ? 2 * lane + 1 : 62 - 2 * lane;
-        const uint32_t sum0 = h[2 * b0], car0 = h[2 * b0 + 1], sum1 = h[2 * b1], car1 = h[2 * b1 + 1];
-        const float q0 = acc_mass(sum0, car0), q1 = acc_mass(sum1, car1);
-        // masses relative to M
-        float m0f, m1f;
-        if (l1) {
-          m0f = q0 * l1_bin_scale(b0);
-          m1f = q1 * l1_bin_scale(b1);
-        } else {
-          const float sc = R.e_ref * 9.5367431640625e-07f;   // 2^-20
-          m0f = q0 * sc;
-          m1f = q1 * sc;
-        }
-        float incm = m0f + m1f;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const float tm = __shfl_up_sync(0xffffffffu, incm, o);
-          if (lane >= o) incm += tm;
-        }
-        const float total = __shfl_sync(0xffffffffu, incm, 31);
-        const float Z = l1 ? total : R.Z;
-        const float target = l1 ? d.top_p * Z * (1.0f + kMassMargin) : R.target;
-        const float run = (l1 ? 0.f : R.mass_above) + incm - (m0f + m1f);
-        const bool pop0 = (sum0 | car0) != 0u, pop1 = (sum1 | car1) != 0u;
-        // order index of a bin = position from the top (0 .. 63)
-        int found = 64, last = -1;
-        if (pop0) {
-          last = 2 * lane;
-          if (run + m0f >= target) found = 2 * lane;
-        }
-        if (pop1) {
-          last = 2 * lane + 1;
-          if (found == 64 && run + m0f + m1f >= target) found = 2 * lane + 1;
-        }
-        int best = found;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, o));
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
-        if (best == 64) best = last;   // rounding left the target just out of reach: lowest populated bin
-        if (best < 0) {
-          if (lane == 0) {             // empty histogram: cannot happen for a non-empty row
-            S->phase = kPhDone;
-            set_status(status, RTP_ERR_UNSUPPORTED);
-          }
-        } else if ((best >> 1) == lane) {
-          const bool first = (best & 1) == 0;
-          const float f_above = first ? run : run + m0f;
-          const float f_q = first ? q0 : q1;
-          const int bin = first ? b0 : b1;
-          const bool few = f_q < 0.999f * kMinQ * (float)kCandCapG;   // fewer than kCandCapG keys in the bin
-          S->mass_above = f_above;
-          if (l1) {
-            S->Z = Z;
-            S->target = target;
-            if (bin == kBins - 1) {
-              // the cut falls into the pooled tail (mass below 2e-14 per key): take every key
-              S->thr_key = 0u;
-              S->tie_last = R.n_keys - 1;
-              S->count = R.n_keys;
-              S->sel_mass = 1.0f;
-              S->phase = kPhDone;
-            } else {
-              const float M = R.M;
-              const float hi_s = l1_bin_hi(M, bin);
-              uint32_t klo, khi;
-              l1_bin_keys(M, bin, klo, khi);
-              const uint32_t span = khi - klo + 1u;
-              const int bits = span > 1u ? 32 - __clz(span - 1u) : 0;
-              float rlo, rhi;
-              raw_preimage(scale, klo, khi, rlo, rhi);
-              S->ref_s = hi_s;
-              S->e_ref = fast_ex2(-kLog2eC * (0.5f * (float)bin - 0.25f));
-              S->base_key = klo;
-              S->span = span;
-              S->shift = max(0, bits - 6);
-              S->raw_lo = rlo;
-              S->raw_hi = rhi;
-              S->cand_cnt = 0;
-              S->phase = (few || span == 1u) ? kPhCollect : kPhKey;
-            }
-          } else {
-            const int shift = R.shift;
-            const uint32_t ofs = (uint32_t)bin << shift;
-            const uint32_t lo_key = R.base_key + ofs;
-            const uint32_t sub_span = min(1u << shift, R.span - ofs);
-            float rlo, rhi;
-            raw_preimage(scale, lo_key, lo_key + (sub_span - 1u), rlo, rhi);
-            S->base_key = lo_key;
-            S->span = sub_span;
-            S->shift = max(0, shift - 6);
-            S->raw_lo = rlo;
-            S->raw_hi = rhi;
-            S->cand_cnt = 0;
-            S->phase = (few || sub_span == 1u) ? kPhCollect : kPhKey;
-          }
-        }
-      } else if (ph == kPhCollect) {
-        // The pass put every key of the bucket (at most kCandCapG, by the bound that sent the row here) into the row's
-        // list in global scratch and counted the keys above the bucket.  While more than kCandCapC of them are left,
-        // the warp narrows on the list itself: the same 64-bin mass histogram over the next six key bits, in the row's
-        // shared-memory bins, no pass over the keys.  Then the exact ranking below finishes.
-        const int n_all = R.cand_cnt;
-        int above = R.cnt_above + __shfl_sync(0xffffffffu, is_b ? cnt_b : cnt_a, src_lane);
-        float m_above = R.mass_above;
-        uint32_t base = R.base_key, span = R.span;
-        int n_in = n_all;
-        const uint2* gc = gcand + (size_t)lr * kCandCapG;
-        uint32_t* hw = hist + lr * kRowWords;
-        if (n_all <= kCandCapG) {
-          while (n_in > kCandCapC && span > 1u) {
-            const int bits = 32 - __clz(span - 1u);
-            const int shift = max(0, bits - 6);
-            for (int i = lane; i < kRowWords; i += 32) hw[i] = 0u;
-            __syncwarp();
-            for (int i = lane; i < n_all; i += 32) {
-              const uint32_t key = __ldcg(&gc[i].x);
-              const uint32_t t = key - base;
-              if (t < span) add_mass(hw + 2 * (t >> shift), fmaf(okey_to_float(key) - R.ref_s, kLog2eC, 20.0f));
-            }
-            __syncwarp();
-            const int b0 = 63 - 2 * lane, b1 = 62 - 2 * lane;   // bin 63 is the top
-            const uint32_t sum0 = hw[2 * b0], car0 = hw[2 * b0 + 1], sum1 = hw[2 * b1], car1 = hw[2 * b1 + 1];
-            const float sc = R.e_ref * 9.5367431640625e-07f;     // 2^-20
-            const float m0f = acc_mass(sum0, car0) * sc, m1f = acc_mass(sum1, car1) * sc;
-            float incm = m0f + m1f;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-              const float tm = __shfl_up_sync(0xffffffffu, incm, o);
-              if (lane >= o) incm += tm;
-            }
-            const float run = m_above + incm - (m0f + m1f);
-            int found = 64, last = -1;
-            if (sum0 | car0) {
-              last = 2 * lane;
-              if (run + m0f >= R.target) found = 2 * lane;
-            }
-            if (sum1 | car1) {
-              last = 2 * lane + 1;
-              if (found == 64 && run + m0f + m1f >= R.target) found = 2 * lane + 1;
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-              found = min(found, __shfl_xor_sync(0xffffffffu, found, o));
-              last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
-            }
-            if (found == 64) found = last;
-            if (found < 0) break;                                 // (no candidate inside the interval: cannot happen)
-            m_above = __shfl_sync(0xffffffffu, (found & 1) ? run + m0f : run, found >> 1);
-            const uint32_t ofs = (uint32_t)(63 - found) << shift;
-            const uint32_t nbase = base + ofs, nspan = min(1u << shift, span - ofs);
-            int c_in = 0, c_up = 0;                               // candidates inside / above the new interval
-            for (int i = lane; i < n_all; i += 32) {
-              const uint32_t t = __ldcg(&gc[i].x) - base;
-              if (t < span) {
-                if (t - ofs < nspan) ++c_in;
-                else if (t >= ofs) ++c_up;
-              }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-              c_in += __shfl_xor_sync(0xffffffffu, c_in, o);
-              c_up += __shfl_xor_sync(0xffffffffu, c_up, o);
-            }
-            above += c_up;
-            n_in = c_in;
-            base = nbase;
-            span = nspan;
-            __syncwarp();
-          }
-        }
-        if (n_in > kCandCapC) {
-          // more than kCandCapC keys share one key value: n_in equal scores straddle the cut
-          float rlo = 0.f, rhi = 0.f;
-          if (lane == 0 && base != R.base_key) raw_preimage(scale, base, base, rlo, rhi);
-          if (lane == 0) {
-            const float each = fast_ex2((okey_to_float(base) - R.M) * kLog2eC);
-            int take = (int)ceilf((R.target - m_above) / each);
-            take = max(1, min(take, n_in));
-            S->cnt_above = above;
-            S->mass_above = m_above;
-            S->thr_key = base;
-            S->count = above + take;
-            S->sel_mass = (m_above + (float)take * each) / R.Z;
-            if (span != 1u) set_status(status, RTP_ERR_UNSUPPORTED);
-            if (take < n_in) {
-              if (base != R.base_key) {   // the tie pass looks for this key value
-                S->base_key = base;
-                S->span = 1u;
-                S->raw_lo = rlo;
-                S->raw_hi = rhi;
-              }
-              S->tie_need = take;
-              S->phase = kPhTie;
-            } else {
-              S->tie_last = R.n_keys - 1;
-              S->phase = kPhDone;
-            }
-          }
-        } else {
-          // the candidates of the final interval move into the row's shared-memory list {key, position}
-          __syncwarp();
-          int filled = 0;
-          for (int i0 = 0; i0 < n_all; i0 += 32) {
-            const int i = i0 + lane;
-            uint2 cnd = make_uint2(0u, 0u);
-            bool in = false;
-            if (i < n_all) {
-              cnd = __ldcg(&gc[i]);
-              in = cnd.x - base < span;
-            }
-            const uint32_t m = __ballot_sync(0xffffffffu, in);
-            if (in) {
-              const int pos = filled + __popc(m & ((1u << lane) - 1u));
-              hw[2 * pos] = cnd.x;
-              hw[2 * pos + 1] = cnd.y;
-            }
-            filled += __popc(m);
-          }
-          __syncwarp();
-          const int n_c = n_in;
-          // exact finish: rank the (at most 64) candidates by (score descending, position ascending)
-          unsigned long long ord[2];
-          float e[2];
-#pragma unroll
-          for (int x = 0; x < 2; ++x) {
-            const int i = 2 * lane + x;
-            ord[x] = ~0ull;
-            e[x] = 0.f;
-            if (i < n_c) {
-              const uint32_t key = h[2 * i], idx = h[2 * i + 1];
-              ord[x] = ((unsigned long long)(~key) << 32) | idx;
-              e[x] = fast_ex2((okey_to_float(key) - R.M) * kLog2eC);
-            }
-          }
-          int rank[2] = {0, 0};
-          float cum[2] = {m_above, m_above};
-          for (int j = 0; j < n_c; ++j) {
-            const int jl = j >> 1;
-            const unsigned long long oj = __shfl_sync(0xffffffffu, (j & 1) ? ord[1] : ord[0], jl);
-            const float ej = __shfl_sync(0xffffffffu, (j & 1) ? e[1] : e[0], jl);
-#pragma unroll
-            for (int x = 0; x < 2; ++x) {
-              if (oj < ord[x]) ++rank[x];
-              if (oj <= ord[x]) cum[x] += ej;
-            }
-          }
-          // shortest prefix whose cumulative mass reaches the target (all candidates if none does)
-          int pick = 1 << 20;
-#pragma unroll
-          for (int x = 0; x < 2; ++x)
-            if (2 * lane + x < n_c && cum[x] >= R.target) pick = min(pick, rank[x]);
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) pick = min(pick, __shfl_xor_sync(0xffffffffu, pick, o));
-          if (pick == (1 << 20)) pick = n_c - 1;
-          // the candidate of rank `pick` defines the threshold; ties with it that were taken have rank <= pick
-          uint32_t thr_key = 0;
-          float pick_cum = 0.f;
-#pragma unroll
-          for (int x = 0; x < 2; ++x)
-            if (2 * lane + x < n_c && rank[x] == pick) {
-              thr_key = ~(uint32_t)(ord[x] >> 32);
-              pick_cum = cum[x];
-            }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            thr_key = max(thr_key, __shfl_xor_sync(0xffffffffu, thr_key, o));
-            pick_cum = fmaxf(pick_cum, __shfl_xor_sync(0xffffffffu, pick_cum, o));
-          }
-          // Position bound for keys that tie with the threshold score: the last one taken, or the row's last key
-          // when none is left out (the usual case: then the attention kernel never has to look at positions).
-          int tie_last = -1, left_out = 0;
-#pragma unroll
-          for (int x = 0; x < 2; ++x)
-            if (2 * lane + x < n_c && ~(uint32_t)(ord[x] >> 32) == thr_key) {
-              if (rank[x] <= pick) tie_last = max(tie_last, (int)(uint32_t)ord[x]); else left_out = 1;
-            }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) tie_last = max(tie_last, __shfl_xor_sync(0xffffffffu, tie_last, o));
-          if (!__any_sync(0xffffffffu, left_out)) tie_last = R.n_keys - 1;
-          if (lane == 0) {
-            S->cnt_above = above;
-            S->thr_key = thr_key;
-            S->tie_last = tie_last;
-            S->count = above + pick + 1;
-            S->sel_mass = pick_cum / R.Z;
-            S->phase = kPhDone;
-            if (n_c == 0) set_status(status, RTP_ERR_UNSUPPORTED);   // a chosen bucket always holds a key
-          }
-        }
-      } else if (ph == kPhTie) {
-        const int tl = __shfl_sync(0xffffffffu, is_b ? tl_b : tl_a, src_lane);
-        if (lane == 0) {
-          S->tie_last = tl;
-          S->phase = kPhDone;
-        }
-      }
-    }
-    __syncwarp();
     {
-      int pend = 0;
-      if (a_ok && rs[la].phase != kPhDone) pend = 1;
-      if (b_ok && rs[lb].phase != kPhDone) pend = 1;
-      if (pend) s_pending = 1;
-    }
-    __syncthreads();
-    if (!s_pending) break;
-    __syncthreads();
+      // prologue of the pass by one thread: request the keys of the first kSStages pages, multiply the first two
+      if (warp == 0 && lane == 0) {
+        for (int j = 0; j < kSStages && j < n_tiles; ++j) issue_tma(gt + (uint32_t)j, j);
+        for (int j = 0; j < 2 && j < n_tiles; ++j) issue_mma(gt + (uint32_t)j);
+      }
+      __syncwarp();
+      // ================================ score threads (thread = row) ================================
+      for (int b = 0; b < kBins; ++b) sts32(hist_col + (uint32_t)b * (kSRows * 4), 0u);
+      for (int b = 0; b < 16; ++b) sts32(carry_col + (uint32_t)b * (kSRows * 4), 0u);
+      // A page's 64 scores are read from tensor memory sixteen at a time; the next sixteen are in flight while the
+      // current ones are processed (small code: the instruction cache is shared by four pipelines).
+#define RTP_SEL_GROUPS(PROCESS)                                                          \
+  {                                                                                      \
+    uint32_t ra[16], rb[16];                                                             \
+    RTP_TMEM_LD16(ra, taddr);                                                            \
+    tmem_wait16(ra);                                                                     \
+    _Pragma("unroll 1") for (int g = 0; g < 4; g += 2) {                                 \
+      RTP_TMEM_LD16(rb, taddr + (uint32_t)(16 * g + 16));                                \
+      PROCESS(ra, n_base + 16 * g);                                                      \
+      tmem_wait16(rb);                                                                   \
+      if (g + 2 < 4) RTP_TMEM_LD16(ra, taddr + (uint32_t)(16 * g + 32));                 \
+      PROCESS(rb, n_base + 16 * g + 16);                                                 \
+      tmem_wait16(ra);                                                                   \
+    }                                                                                    \
   }
-
-  // ---- id lists: one more sweep over the keys, every resolved row appends its members in position order ----
-  if (want_ids) {
-    __syncthreads();
-    const RowState sa = rs[la], sb = rs[lb];
-    const bool em_a = a_ok && sa.phase == kPhDone && sa.n_keys > 0, em_b = b_ok && sb.phase == kPhDone && sb.n_keys > 0;
-    int32_t* dst_a = sel_idx + ((int64_t)(r0 + pofs + g) * d.n_ret + rh_head) * sel_stride;
-    int32_t* dst_b = sel_idx + ((int64_t)(r0 + pofs + g + 8) * d.n_ret + rh_head) * sel_stride;
-    int run_a = 0, run_b = 0;
-    load_stage(0, 0);
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    for (int sidx = 0; sidx < n_stages; ++sidx) {
-      const int buf = sidx & 1;
-      if (sidx + 1 < n_stages) load_stage(sidx + 1, buf ^ 1);
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      asm volatile("cp.async.wait_group 1;" ::: "memory");
-      __syncthreads();
-      if (warp_ok) {
-        const unsigned char* st = stage_s + buf * kStageBytesC;
-        const int boff = 2 * qfrag_dim_offset(lane);
-#pragma unroll 1
-        for (int pg = 0; pg < kPagesPerStage; ++pg) {
-          const int n_page = (sidx * kPagesPerStage + pg) * kPage;
-          if (n_page > warp_m_hi) break;
-#pragma unroll 1
-          for (int nt = 0; nt < 8; ++nt) {
-            const uint2 b = *reinterpret_cast<const uint2*>(st + (pg * kPage + nt * 8 + g) * (kIndexDim * 2) + boff);
-            const float zero[4] = {0.f, 0.f, 0.f, 0.f};
-            float s4[4];
-            mma_bf16_16816(s4, iq.a0, iq.a1, iq.a2, iq.a3, b.x, b.y, zero);
-            const int n_first = n_page + nt * 8 + 2 * c;
-            int fa = 0, fb = 0;
+      if (kind == kPassMax) {
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+        auto proc_max = [&](const uint32_t(&r)[16], const int n0, const bool interior) {
+          if (interior) {
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const int n = n_first + e;
-              const uint32_t ka_ = okey(finish_score(s4[e], scale));
-              const uint32_t kb_ = okey(finish_score(s4[2 + e], scale));
-              if (em_a && n <= pos_a && (ka_ > sa.thr_key || (ka_ == sa.thr_key && n <= sa.tie_last))) fa |= 1 << e;
-              if (em_b && n <= pos_b && (kb_ > sb.thr_key || (kb_ == sb.thr_key && n <= sb.tie_last))) fb |= 1 << e;
+            for (int j = 0; j < 16; j += 4) {
+              mx0 = fmaxf(mx0, __uint_as_float(r[j]));
+              mx1 = fmaxf(mx1, __uint_as_float(r[j + 1]));
+              mx2 = fmaxf(mx2, __uint_as_float(r[j + 2]));
+              mx3 = fmaxf(mx3, __uint_as_float(r[j + 3]));
             }
-            const int ka = __popc(fa), kb = __popc(fb);
-            int ia = ka, ib = kb, tt;
-            tt = __shfl_up_sync(0xffffffffu, ia, 1, 4); if (c >= 1) ia += tt;
-            tt = __shfl_up_sync(0xffffffffu, ia, 2, 4); if (c >= 2) ia += tt;
-            tt = __shfl_up_sync(0xffffffffu, ib, 1, 4); if (c >= 1) ib += tt;
-            tt = __shfl_up_sync(0xffffffffu, ib, 2, 4); if (c >= 2) ib += tt;
-            const int tot_a = __shfl_sync(0xffffffffu, ia, 3, 4), tot_b = __shfl_sync(0xffffffffu, ib, 3, 4);
-            int wa = run_a + ia - ka, wb = run_b + ib - kb;
+          } else {
+            const int valid = pos - n0 + 1;
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              if (fa & (1 << e)) { if (wa < sel_stride) dst_a[wa] = n_first + e; ++wa; }
-              if (fb & (1 << e)) { if (wb < sel_stride) dst_b[wb] = n_first + e; ++wb; }
-            }
-            run_a += tot_a;
-            run_b += tot_b;
+            for (int j = 0; j < 16; ++j)
+              if (j < valid) mx0 = fmaxf(mx0, __uint_as_float(r[j]));
+          }
+        };
+#pragma unroll 1
+        for (int it = 0; it < n_tiles; ++it) {
+          RTP_SEL_TILE_BEGIN
+#define RTP_P(r_, n0_) proc_max(r_, n0_, interior)
+          RTP_SEL_GROUPS(RTP_P)
+#undef RTP_P
+          RTP_SEL_TILE_END
+        }
+        if (phase == kPhMax) {
+          const float s_max = finish_score(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)), scale);
+          if (!(fabsf(s_max) < 262144.0f)) {
+            // no finite score, or scores beyond the range of the fixed grid: every key is kept and the call reports it
+            set_status(status, RTP_ERR_UNSUPPORTED);
+            phase = kPhDone;
+            tie_last = n_keys - 1;
+            count = n_keys;
+            sel_m = 1.0f;
+          } else {
+            aI = grid_bin(s_max);
+            w0 = 0;
+            ref0 = -0.25f * ((float)aI - 0.5f);
+            mass_above = 0.f;
+            phase = kPhL1;
           }
         }
+      } else if (kind == kPassL1) {
+        // bin = round(-4 s) - aI - w0, clamped to 63; mass relative to the bin's upper end, 2^18 fixed point
+        const bool shifted = w0 > 0;
+        const bool active = phase == kPhL1;
+        // rows that take no part land in bin 63 of their own column whatever their scores are
+        const float dd = active ? kMagicC - (float)(aI + w0) : __int_as_float(0x7f800000);
+        const float cx = (float)kFixBits + (kLog2eC * 0.25f) * ((float)(aI + w0) - 0.5f);
+        const uint32_t hb = hist_col - kMagicBits * (uint32_t)(kSRows * 4);
+        auto proc_l1 = [&](const uint32_t(&r)[16], const int n0, const bool fast) {
+          if (fast) {
+            // two scores at a time, written out instruction by instruction: both bins are loaded before either is
+            // stored (the second takes the first's new value when they are the same bin)
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) l1_pair(r[j], r[j + 1], scale, dd, cx, hb);
+          } else if (active) {
+            const int valid = pos - n0 + 1;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float s = __uint_as_float(r[j]) * scale;
+              float t = fmaf(s, -4.0f, dd);
+              // (t < magic: above the window, accounted for by an earlier level)
+              if (j < valid && !(t < kMagicC)) {
+                t = fminf(t, kMagicC + 63.0f);
+                const float x = fmaf(t - kMagicC, kLog2eC * 0.25f, fmaf(s, kLog2eC, cx));
+                hist_add(hist_col, (int)(__float_as_uint(t) & 63u), fix_q(x));
+              }
+            }
+          }
+        };
+#pragma unroll 1
+        for (int it = 0; it < n_tiles; ++it) {
+          RTP_SEL_TILE_BEGIN
+          const bool fast = interior && !shifted;
+#define RTP_P(r_, n0_) proc_l1(r_, n0_, fast)
+          RTP_SEL_GROUPS(RTP_P)
+#undef RTP_P
+          RTP_SEL_TILE_END
+          if ((it & (kNormEvery - 1)) == kNormEvery - 1) hist_normalize(hist_col, carry_col);
+        }
+        hist_normalize(hist_col, carry_col);
+        if (active) {
+          if (!have_z) {
+            float tot = 0.f;
+            for (int b = 0; b < kBins; ++b) {
+              bool pop;
+              const float qf = hist_read(hist_col, carry_col, b, pop);
+              tot += qf * fast_ex2(-(float)kFixBits - (float)b * (kLog2eC * 0.25f));
+            }
+            Z = tot;
+            target = d.top_p * Z * (1.0f + kMassMargin);
+            have_z = true;
+          }
+          float run = mass_above;
+          int found = -1, last = -1;
+          float above_found = 0.f, above_last = 0.f, q_found = 0.f, q_last = 0.f;
+          for (int b = 0; b < kBins; ++b) {
+            bool pop;
+            const float qf = hist_read(hist_col, carry_col, b, pop);
+            const float m = qf * fast_ex2(-(float)kFixBits - (float)(w0 + b) * (kLog2eC * 0.25f));
+            if (pop) {
+              last = b;
+              above_last = run;
+              q_last = qf;
+              if (found < 0 && run + m >= target) {
+                found = b;
+                above_found = run;
+                q_found = qf;
+              }
+            }
+            run += m;
+          }
+          if (found < 0) {   // rounding left the target just out of reach: lowest populated bin
+            found = last;
+            above_found = above_last;
+            q_found = q_last;
+          }
+          if (found < 0) {
+            // an empty window below the mass already counted: nothing is left to add
+            set_status(status, RTP_ERR_UNSUPPORTED);
+            phase = kPhDone;
+            tie_last = n_keys - 1;
+            count = n_keys;
+            sel_m = 1.0f;
+          } else if (found == kBins - 1) {
+            // the pooled bin: look at it with a window of its own, unless it lies so deep that it holds no mass
+            mass_above = above_found;
+            w0 += kBins - 1;
+            if (w0 > kMaxShift) {
+              phase = kPhDone;
+              tie_last = n_keys - 1;
+              count = n_keys;
+              sel_m = 1.0f;
+            }
+          } else {
+            mass_above = above_found;
+            const int a_abs = aI + w0 + found;
+            uint32_t klo, khi;
+            grid_bin_keys(a_abs, klo, khi);
+            base_key = klo;
+            span = khi - klo + 1u;
+            const int bits = span > 1u ? 32 - __clz(span - 1u) : 0;
+            shift = max(0, bits - 6);
+            raw_preimage(scale, klo, khi, raw_lo, raw_hi);
+            ref_s = -0.25f * ((float)a_abs - 0.5f);
+            e_ref = fast_ex2(-(float)(w0 + found) * (kLog2eC * 0.25f));
+            cand_cnt = 0;
+            cnt_above = 0;
+            const bool few = q_found < 0.999f * kMinQ18 * (float)kCandCapG;
+            phase = (few || span == 1u) ? kPhCollect : kPhKey;
+          }
+        }
+      } else if (kind == kPassLate) {
+        // The unscaled scores inside a row's interval are queued in shared memory and moved on by the whole warp:
+        //   collecting rows   queue = the row's own (idle) histogram column, 64 words; destination = the row's list in
+        //                     global scratch (raw bits, position order); the keys above the interval are counted
+        //   key-level rows    queue = the 16 words of the row's counter column; destination = the 64-bin mass histogram
+        //                     of the next six key bits in the row's histogram column (2^11 fixed point: a bucket that
+        //                     needs a key level holds thousands of keys of nearly equal mass, so coarse rounding of each
+        //                     is harmless and the sums cannot overflow)
+        //   tie rows          no queue: the position of the tie_need-th key with the threshold score is noted in passing
+        const bool collecting = phase == kPhCollect, keying = phase == kPhKey, tying = phase == kPhTie;
+        const bool listing = collecting || keying;
+        const float kInfL = __int_as_float(0x7f800000);
+        const float lo = listing ? raw_lo : kInfL, hi = listing ? raw_hi : -kInfL;
+        const float cut = collecting ? raw_hi : kInfL;
+        const float tlo = tying ? raw_lo : kInfL, thi = tying ? raw_hi : -kInfL;
+        const bool any_tie = (flags & (1 << kPhTie)) != 0;
+        const uint32_t qbase = keying ? carry_col : hist_col;
+        const uint32_t qfull = qbase + (uint32_t)((keying ? 8 : 56) * kSRows * 4);   // more entries than this: flush
+        const uint32_t qhalf = qbase + (uint32_t)((keying ? 4 : 28) * kSRows * 4);
+        uint32_t qa = qbase;                               // address of the next free queue word (512 bytes apart)
+        int cnt = 0, above = 0;
+        auto warp_flush = [&](const bool everything) {
+          const uint32_t m = __ballot_sync(0xffffffffu, everything ? qa > qbase : qa > qhalf);
+          for (uint32_t rest = m; rest; rest &= rest - 1u) {
+            const int l = __ffs(rest) - 1;
+            const uint32_t qb_l = __shfl_sync(0xffffffffu, qbase, l);
+            const int qn_l = (int)((__shfl_sync(0xffffffffu, qa, l) - qb_l) / (uint32_t)(kSRows * 4));
+            if (!__shfl_sync(0xffffffffu, (int)keying, l)) {
+              const int cnt_l = __shfl_sync(0xffffffffu, cnt, l);
+              uint32_t* g_l = gc + (ptrdiff_t)(l - lane) * kCandCapG;
+              for (int i = lane; i < qn_l; i += 32)
+                if (cnt_l + i < kCandCapG) g_l[cnt_l + i] = lds32(qb_l + (uint32_t)i * (kSRows * 4));
+            } else {
+              const uint32_t base_l = __shfl_sync(0xffffffffu, base_key, l), span_l = __shfl_sync(0xffffffffu, span, l);
+              const int shift_l = __shfl_sync(0xffffffffu, shift, l);
+              const float ref_l = __shfl_sync(0xffffffffu, ref_s, l);
+              const uint32_t hcol_l = __shfl_sync(0xffffffffu, hist_col, l);
+              for (int i = lane; i < qn_l; i += 32) {
+                const float s = finish_score(__uint_as_float(lds32(qb_l + (uint32_t)i * (kSRows * 4))), scale);
+                const uint32_t t = okey(s) - base_l;
+                if (t < span_l) red_add_shared(hcol_l + (uint32_t)(t >> shift_l) * (kSRows * 4), fix_q(fmaf(s - ref_l, kLog2eC, 11.0f)));
+              }
+            }
+            if (lane == l) {
+              cnt += qn_l;
+              qa = qbase;
+            }
+          }
+          __syncwarp();
+        };
+        // eight scores; `valid` = how many of them the row may see (8 on interior pages)
+        auto proc8 = [&](const uint32_t* r, const int n0, const bool interior) {
+          if (interior && !any_tie) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) late_one(r[j], cut, lo, hi, above, qa);
+          } else {
+            const int valid = interior ? 8 : pos - n0 + 1;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float raw = __uint_as_float(r[j]);
+              if (j < valid && raw > cut) ++above;
+              if (j < valid && raw >= lo && raw <= hi) {
+                sts32(qa, r[j]);
+                qa += (uint32_t)(kSRows * 4);
+              }
+              if (j < valid && raw >= tlo && raw <= thi) {
+                if (++tie_run == tie_need) tie_last = n0 + j;
+              }
+            }
+          }
+          if (__any_sync(0xffffffffu, qa > qfull)) warp_flush(false);
+        };
+        auto proc_late = [&](const uint32_t(&r)[16], const int n0, const bool interior) {
+          proc8(&r[0], n0, interior);
+          proc8(&r[8], n0 + 8, interior);
+        };
+#pragma unroll 1
+        for (int it = 0; it < n_tiles; ++it) {
+          RTP_SEL_TILE_BEGIN
+#define RTP_P(r_, n0_) proc_late(r_, n0_, interior)
+          RTP_SEL_GROUPS(RTP_P)
+#undef RTP_P
+          RTP_SEL_TILE_END
+        }
+        warp_flush(true);
+        if (collecting && cnt > kCandCapG) {   // the bucket's mass bounds its size below the list's capacity: cannot happen
+          set_status(status, RTP_ERR_CAPACITY);
+          cnt = kCandCapG;
+        }
+        if (keying) {
+          // bins in order of decreasing score: 63 is the top
+          float run = mass_above;
+          int found = -1, last = -1;
+          float above_found = 0.f, above_last = 0.f, q_found = 0.f, q_last = 0.f;
+          for (int b = kBins - 1; b >= 0; --b) {
+            const uint32_t sum = lds32(hist_col + (uint32_t)b * (kSRows * 4));
+            const float qf = (float)sum;
+            const float m = qf * e_ref * 4.8828125e-04f;   // 2^-11
+            if (sum != 0u) {
+              last = b;
+              above_last = run;
+              q_last = qf;
+              if (found < 0 && run + m >= target) {
+                found = b;
+                above_found = run;
+                q_found = qf;
+              }
+            }
+            run += m;
+          }
+          if (found < 0) {
+            found = last;
+            above_found = above_last;
+            q_found = q_last;
+          }
+          if (found < 0) {
+            set_status(status, RTP_ERR_UNSUPPORTED);   // a chosen bucket always holds a key
+            phase = kPhDone;
+            tie_last = n_keys - 1;
+            count = n_keys;
+            sel_m = 1.0f;
+          } else {
+            mass_above = above_found;
+            const uint32_t ofs = (uint32_t)found << shift;
+            const uint32_t lo_key = base_key + ofs;
+            const uint32_t sub_span = min(1u << shift, span - ofs);
+            raw_preimage(scale, lo_key, lo_key + (sub_span - 1u), raw_lo, raw_hi);
+            base_key = lo_key;
+            span = sub_span;
+            shift = max(0, shift - 6);
+            cand_cnt = 0;
+            cnt_above = 0;
+            const bool few = q_found < 0.999f * kMinQ11 * (float)kCandCapG;
+            phase = (few || sub_span == 1u) ? kPhCollect : kPhKey;
+          }
+        } else if (collecting) {
+          cand_cnt = cnt;
+          cnt_above = above;
+        } else if (tying) {
+          if (tie_last < 0) {           // fewer ties than counted before: cannot happen
+            set_status(status, RTP_ERR_UNSUPPORTED);
+            tie_last = n_keys - 1;
+          }
+          phase = kPhDone;
+        }
+        // ---- exact finish of the rows that collected, one row at a time by the whole warp ----
+        sub_sync();   // every row has read its histogram: the carry words become scratch
+        uint32_t* hw = reinterpret_cast<uint32_t*>(smem + kCarryOff) + warp * 512;
+        const uint32_t need = __ballot_sync(0xffffffffu, collecting);
+        for (uint32_t rest = need; rest; rest &= rest - 1u) {
+          const int rr = __ffs(rest) - 1;
+          FinIn fi;
+          fi.n_all = __shfl_sync(0xffffffffu, cand_cnt, rr);
+          fi.above = __shfl_sync(0xffffffffu, cnt_above, rr);
+          fi.n_keys = __shfl_sync(0xffffffffu, n_keys, rr);
+          fi.m_above = __shfl_sync(0xffffffffu, mass_above, rr);
+          fi.target = __shfl_sync(0xffffffffu, target, rr);
+          fi.ref_s = __shfl_sync(0xffffffffu, ref_s, rr);
+          fi.e_ref = __shfl_sync(0xffffffffu, e_ref, rr);
+          fi.ref0 = __shfl_sync(0xffffffffu, ref0, rr);
+          fi.Z = __shfl_sync(0xffffffffu, Z, rr);
+          fi.scale = scale;
+          fi.base = __shfl_sync(0xffffffffu, base_key, rr);
+          fi.span = __shfl_sync(0xffffffffu, span, rr);
+          const uint32_t* gcr = gc + (ptrdiff_t)(rr - lane) * kCandCapG;
+          const FinOut fo = finish_row(fi, gcr, hw, lane);
+          if (lane == rr) {
+            phase = fo.phase;
+            cnt_above = fo.cnt_above;
+            mass_above = fo.mass_above;
+            thr_key = fo.thr_key;
+            count = fo.count;
+            sel_m = fo.sel_mass;
+            tie_last = fo.tie_last;
+            if (fo.bad) set_status(status, RTP_ERR_UNSUPPORTED);
+            if (fo.phase == kPhTie) {   // the next pass finds the position of the tie_need-th key with this score
+              tie_need = fo.tie_need;
+              tie_run = 0;
+              raw_preimage(scale, thr_key, thr_key, raw_lo, raw_hi);
+            }
+          }
+        }
+      } else {   // kPassEmit: every resolved row appends its members in position order
+        const bool em = row_ok && phase == kPhDone && n_keys > 0;
+        int32_t* dst = sel_idx + ((int64_t)(r0 + (row_ok ? po : 0)) * d.n_ret + rh_head) * sel_stride;
+        int run = 0;
+        auto proc_e = [&](const uint32_t(&r)[16], const int n0) {
+          const int valid = em ? pos - n0 + 1 : 0;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const uint32_t k = okey(finish_score(__uint_as_float(r[j]), scale));
+            if (j < valid && (k > thr_key || (k == thr_key && n0 + j <= tie_last))) {
+              if (run < sel_stride) dst[run] = n0 + j;
+              ++run;
+            }
+          }
+        };
+#pragma unroll 1
+        for (int it = 0; it < n_tiles; ++it) {
+          RTP_SEL_TILE_BEGIN
+          (void)interior;
+#define RTP_P(r_, n0_) proc_e(r_, n0_)
+          RTP_SEL_GROUPS(RTP_P)
+#undef RTP_P
+          RTP_SEL_TILE_END
+        }
+        if (em && run > sel_stride) set_status(status, RTP_ERR_CAPACITY);
       }
-      __syncthreads();
+#undef RTP_SEL_GROUPS
+      if (kind != kPassEmit && phase != kPhDone) atomicOr(const_cast<int*>(&pass_flags[(pass + 1) & 1]), 1 << phase);
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (c == 0) {
-      if ((em_a && run_a > sel_stride) || (em_b && run_b > sel_stride)) set_status(status, RTP_ERR_CAPACITY);
-    }
+    sub_sync();
+    if (tid == 0) pass_flags[pass & 1] = 0;
+    sub_sync();
   }
 
   // ---- results ----
-  if (tid < kCRows) {
-    const int hs = tid / BMP, po = tid % BMP;
-    if (hs < nh && po < rows_here) {
-      const RowState& S = rs[tid];
-      const int64_t o = (int64_t)(r0 + po) * d.n_ret + hm.ih_heads[ih][hs];
-      if (S.phase != kPhDone) set_status(status, RTP_ERR_TIMEOUT);
-      sel_count[o] = S.n_keys == 0 ? 0 : S.count;
-      if (sel_mass) sel_mass[o] = S.sel_mass;
-      if (sel_thresh) sel_thresh[o] = S.thr_key == 0u ? -INFINITY : okey_to_float(S.thr_key);
-      if (sel_tie_last) sel_tie_last[o] = S.n_keys == 0 ? -1 : S.tie_last;
-    }
+  if (row_ok) {
+    const int64_t o = (int64_t)(r0 + po) * d.n_ret + rh_head;
+    if (phase != kPhDone) set_status(status, RTP_ERR_TIMEOUT);
+    sel_count[o] = n_keys == 0 ? 0 : count;
+    if (sel_mass) sel_mass[o] = sel_m;
+    if (sel_thresh) sel_thresh[o] = thr_key == 0u ? -INFINITY : okey_to_float(thr_key);
+    if (sel_tie_last) sel_tie_last[o] = n_keys == 0 ? -1 : tie_last;
+  }
+  }   // units
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_cta), "r"(kSubs * kTmemColsS) : "memory");
   }
 }
 
+// The kernel's dynamic shared memory attribute is a per-device setting: applied once per device and instantiation.
+template <int G>
+cudaError_t set_smem_attr() {
+  static std::atomic<uint64_t> done[2] = {};   // bit per device ordinal (up to 128 devices)
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 128) return cudaErrorInvalidDevice;
+  const uint64_t bit = 1ull << (dev & 63);
+  if (done[dev >> 6].load(std::memory_order_acquire) & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(select_chunk_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemS);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(select_chunk_kernel<G>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+  if (e != cudaSuccess) return e;
+  done[dev >> 6].fetch_or(bit, std::memory_order_release);
+  return cudaSuccess;
+}
 
 template <int G>
 cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                          const __nv_bfloat16* qt, int32_t* sel_idx, int64_t sel_stride, int32_t* sel_count,
                          float* sel_mass, float* sel_thresh, int32_t* sel_tie_last, int32_t* status, void* ws,
-                         cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(select_chunk_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemC);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
-  constexpr int BMP = kCRows / G;
+                         int sm_count, cudaStream_t st) {
+  cudaError_t e = set_smem_attr<G>();
+  if (e != cudaSuccess) return e;
+  CUtensorMap map_ik;
+  e = make_rows_map(&map_ik, cv.ikey, (int64_t)cv.num_pages * cv.n_ih * kPage, kIndexDim, kIndexDim, kPage,
+                    (int)CU_TENSOR_MAP_SWIZZLE_32B);
+  if (e != cudaSuccess) return e;
+  constexpr int BMP = kSRows / G;
   const int n_row_tiles = (int)((rows.R + BMP - 1) / BMP);
-  dim3 grid(n_row_tiles, d.n_ih);
-  select_chunk_kernel<G><<<grid, kCThreads, kSmemC, st>>>(cv, d, hm, qt, rows.seq_id, rows.q_start, (int)rows.R,
+  const int n_units = n_row_tiles * d.n_ih;
+  dim3 grid(std::max(1, std::min(sm_count, (n_units + kSubs - 1) / kSubs)));
+  int mp = kMaxPasses;
+  if (const char* e_ = getenv("RTP_SEL_MAX_PASSES")) mp = atoi(e_);   // TEMPORARY (timing probe)
+  select_chunk_kernel<G><<<grid, kSubs * kSThreads, kSmemS, st>>>(map_ik, cv, d, hm, qt, rows.seq_id, rows.q_start, (int)rows.R,
                                                           sel_idx, sel_stride, sel_count, sel_mass, sel_thresh,
-                                                          sel_tie_last, status, reinterpret_cast<uint2*>(ws), n_row_tiles,
-                                                          kMaxPasses);
+                                                          sel_tie_last, status, reinterpret_cast<uint32_t*>(ws), n_row_tiles,
+                                                          mp);
   return cudaGetLastError();
 }
 
@@ -967,25 +1031,25 @@ static int slot_class(const Dims& d, const HeadMaps& hm) {
   return max_nh <= 1 ? 1 : max_nh <= 2 ? 2 : max_nh <= 4 ? 4 : max_nh <= 8 ? 8 : 0;
 }
 
-// Candidate scratch: kCandCapG entries of 8 bytes per (row, head slot) of every CTA.
+// Candidate scratch: kCandCapG entries of 4 bytes per (row, head slot) of every unit.
 size_t select_chunk_workspace_bytes(const Dims& d, const HeadMaps& hm, int64_t R) {
   const int g = slot_class(d, hm);
   if (g == 0 || R <= 0) return 256;
-  const int64_t n_row_tiles = (R + kCRows / g - 1) / (kCRows / g);
-  return (size_t)n_row_tiles * d.n_ih * kCRows * kCandCapG * sizeof(uint2);
+  const int64_t n_row_tiles = (R + kSRows / g - 1) / (kSRows / g);
+  return (size_t)n_row_tiles * d.n_ih * kSRows * kCandCapG * sizeof(uint32_t);
 }
 
 cudaError_t launch_select_chunk(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                                 const __nv_bfloat16* qt, int32_t* sel_idx, int64_t sel_stride,
                                 int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
                                 int32_t* status, void* ws, int sm_count, cudaStream_t st) {
-  (void)sm_count;
   if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
+  if ((int64_t)rows.q_start + rows.R > (int64_t)1 << 21) return cudaErrorNotSupported;   // 8-bit overflow counters of the bins
   switch (slot_class(d, hm)) {
-    case 1: return launch_typed<1>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, st);
-    case 2: return launch_typed<2>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, st);
-    case 4: return launch_typed<4>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, st);
-    case 8: return launch_typed<8>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, st);
+    case 1: return launch_typed<1>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, sm_count, st);
+    case 2: return launch_typed<2>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, sm_count, st);
+    case 4: return launch_typed<4>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, sm_count, st);
+    case 8: return launch_typed<8>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, sm_count, st);
     default: return cudaErrorNotSupported;
   }
 }

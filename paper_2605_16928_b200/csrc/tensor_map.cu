@@ -1,0 +1,46 @@
+// Host side of the TMA descriptors: cuTensorMapEncodeTiled through the runtime's driver entry point.
+#include <mutex>
+
+#include "tc_common.cuh"
+
+namespace rtp {
+
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The entry point is a property of the driver, not of a device: looked up once per process, under a lock.
+EncodeTiledFn encode_fn(cudaError_t* err) {
+  static std::mutex mu;
+  static EncodeTiledFn fn = nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  *err = cudaSuccess;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) { *err = e; return nullptr; }
+    if (qres != cudaDriverEntryPointSuccess || !p) { *err = cudaErrorNotSupported; return nullptr; }
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+}  // namespace
+
+cudaError_t make_rows_map(CUtensorMap* map, const void* base, int64_t rows, int row_elems, int box_cols, int box_rows,
+                          int swizzle) {
+  cudaError_t e;
+  EncodeTiledFn encode = encode_fn(&e);
+  if (!encode) return e;
+  const cuuint64_t dims[2] = {(cuuint64_t)row_elems, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)row_elems * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, (CUtensorMapSwizzle)swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+}  // namespace rtp
