@@ -294,6 +294,7 @@ rtp_status rtp_topp_select(rtp_ctx* ctx, const rtp_params* params, const rtp_cac
   WsCarver w(workspace);
   __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(w.take(qt_bytes(d, R)));
   const bool chunk = row_seq == nullptr;
+  const size_t sel_off = w.off;
   void* sel_ws = w.take(chunk ? select_chunk_workspace_bytes(d, hm, R) : select_rows_workspace_bytes(d, R));
   if (w.off > workspace_bytes) return fail(ctx, RTP_ERR_CAPACITY, "workspace too small");
   cudaError_t e = launch_index_queries(d, hm, reinterpret_cast<const __nv_bfloat16*>(q_pre),
@@ -301,7 +302,7 @@ rtp_status rtp_topp_select(rtp_ctx* ctx, const rtp_params* params, const rtp_cac
   if (e == cudaSuccess) {
     if (chunk)
       e = launch_select_chunk(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh,
-                              sel_tie_last, status, sel_ws, ctx->sm_count, st);
+                              sel_tie_last, status, sel_ws, workspace_bytes - sel_off, ctx->sm_count, st);
     else
       e = launch_select_rows(cv, d, hm, rows, qt, max_len, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh,
                              sel_tie_last, status, sel_ws, ctx->sm_count, st);

@@ -107,7 +107,7 @@ size_t select_chunk_workspace_bytes(const Dims& d, const HeadMaps& hm, int64_t R
 cudaError_t launch_select_chunk(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                                 const __nv_bfloat16* qt, int32_t* sel_idx, int64_t sel_stride,
                                 int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
-                                int32_t* status, void* ws, int sm_count, cudaStream_t st);
+                                int32_t* status, void* ws, size_t ws_bytes, int sm_count, cudaStream_t st);
 
 enum AttnSet { kSetList = 0, kSetLocal = 1, kSetDense = 2 };
 size_t attn_rows_workspace_bytes(const Dims& d, int64_t R, int n_units, int group, int sm_count, int64_t max_len);

@@ -42,7 +42,13 @@ constexpr int kSThreads = 128;                // threads of one pipeline: thread
 constexpr int kTmemColsS = 128;               // two score buffers of 64 columns
 constexpr int kStageBytesS = kSTile * kIndexDim * 2;   // 2 KB
 constexpr int kCandCapC = 64;                 // candidates ranked exactly per row
-constexpr int kCandCapG = 8192;               // entries (unscaled score bits) of a row's list in global scratch
+// A row's list of bucket keys (unscaled score bits) lives in blocks of the workspace pool, taken on demand: word 0 of a
+// block is the index of the row's next block, the other 2047 words are entries.
+constexpr int kBlockWords = 2048;
+constexpr int kBlockEntries = kBlockWords - 1;
+constexpr uint32_t kNoBlock = 0xffffffffu;
+constexpr int kListMax = 65536;               // buckets that may hold more keys are narrowed by a key level first
+constexpr int kRowPoolEntries = 8192;         // pool words the workspace provides per (row, head)
 constexpr int kMaxPasses = 24;
 constexpr int kMaxShift = 63 * 6;             // level-1 windows below this depth hold no representable mass
 constexpr float kLog2eC = kLog2eH;
@@ -213,7 +219,7 @@ __device__ void grid_bin_keys(int a, uint32_t& klo, uint32_t& khi) {
 // ---- exact finish of one row by a warp ---------------------------------------------------------------------------
 struct FinIn {
   int n_all, above, n_keys;
-  float m_above, target, ref_s, e_ref, ref0, Z, scale;
+  float m_above, target, target_hi, ref_s, e_ref, ref0, Z, scale;
   uint32_t base, span;
 };
 struct FinOut {
@@ -222,11 +228,28 @@ struct FinOut {
   uint32_t thr_key;
 };
 
-// gc: the row's list of unscaled score bits (n_all entries, all inside the bucket [base, base + span) of ordered
-// keys); hw: 256 words of shared scratch of this warp.  Masses are relative to exp(ref0); target and m_above too.
+// Calls f(raw bits) for every entry of a row's list (n_all entries from block `first` on), entries spread over the lanes.
+template <class F>
+__device__ __forceinline__ void for_each_entry(const uint32_t* pool, uint32_t first, int n_all, int lane, F f) {
+  int done = 0;
+  for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
+    const uint32_t* b = pool + (size_t)blk * kBlockWords;
+    const int n_here = min(kBlockEntries, n_all - done);
+    for (int i = lane; i < n_here; i += 32) f(__ldcg(b + 1 + i));
+    done += n_here;
+    blk = __ldcg(b);
+  }
+}
+
+// The row's list of unscaled score bits starts in block `first` of the pool (n_all entries, all inside the bucket
+// [base, base + span) of ordered keys); hw: 256 words of shared scratch of this warp; wbuf: the pipeline's histogram
+// memory, idle now, of which this warp owns the words (i / 32) * 128 + 32 * warp + i % 32 for i < 2048.  A list of up
+// to 2048 entries is staged there once, as ordered keys, with four loads in flight per lane; every later round reads
+// shared memory.  Masses are relative to exp(ref0); target and m_above too.
 // The cut inside the bucket is found on score values alone: when it falls between keys of equal score, the first
 // `tie_need` of them in position order belong to the set and one more pass over the keys finds where that is.
-__device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* gc, uint32_t* hw, const int lane) {
+__device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* pool, const uint32_t first, uint32_t* hw,
+                                          uint32_t* wbuf, const int warp, const int lane) {
   FinOut o;
   o.bad = 0;
   o.tie_need = 0;
@@ -236,17 +259,50 @@ __device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* gc, ui
   uint32_t base = in.base, span = in.span;
   int n_in = n_all;
   auto key_of = [&](uint32_t raw_bits) { return okey(finish_score(__uint_as_float(raw_bits), in.scale)); };
+  auto wb = [&](int i) -> uint32_t& { return wbuf[(i >> 5) * kSRows + 32 * warp + (i & 31)]; };
+  const bool staged = n_all <= 2048 && span > 1u;
+  if (staged) {
+    int done = 0;
+    for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
+      const uint32_t* b = pool + (size_t)blk * kBlockWords;
+      const int n_here = min(kBlockEntries, n_all - done);
+      const uint32_t next = __ldcg(b);
+      for (int i0 = 0; i0 < n_here; i0 += 128) {
+        uint32_t v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int i = i0 + 32 * k + lane;
+          v[k] = i < n_here ? __ldcg(b + 1 + i) : 0u;
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int i = i0 + 32 * k + lane;
+          if (i < n_here) wb(done + i) = key_of(v[k]);
+        }
+      }
+      done += n_here;
+      blk = next;
+    }
+    __syncwarp();
+  }
+  // f(key) for every entry of the list, entries spread over the lanes
+  auto visit = [&](auto f) {
+    if (staged) {
+      for (int i = lane; i < n_all; i += 32) f(wb(i));
+    } else {
+      for_each_entry(pool, first, n_all, lane, [&](uint32_t raw_bits) { f(key_of(raw_bits)); });
+    }
+  };
   // narrow on the list while more than kCandCapC candidates are left: 64-bin mass histogram over the next six key bits
   while (n_in > kCandCapC && span > 1u) {
     const int bits = 32 - __clz(span - 1u);
     const int shift = max(0, bits - 6);
     for (int i = lane; i < 2 * kBins; i += 32) hw[i] = 0u;
     __syncwarp();
-    for (int i = lane; i < n_all; i += 32) {
-      const uint32_t key = key_of(__ldcg(gc + i));
+    visit([&](uint32_t key) {
       const uint32_t t = key - base;
       if (t < span) add_mass(hw + 2 * (t >> shift), fmaf(okey_to_float(key) - in.ref_s, kLog2eC, 20.0f));
-    }
+    });
     __syncwarp();
     const int b0 = 63 - 2 * lane, b1 = 62 - 2 * lane;   // bin 63 is the top
     const uint32_t sum0 = hw[2 * b0], car0 = hw[2 * b0 + 1], sum1 = hw[2 * b1], car1 = hw[2 * b1 + 1];
@@ -279,13 +335,13 @@ __device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* gc, ui
     const uint32_t ofs_k = (uint32_t)(63 - found) << shift;
     const uint32_t nbase = base + ofs_k, nspan = min(1u << shift, span - ofs_k);
     int c_in = 0, c_up = 0;                               // candidates inside / above the new interval
-    for (int i = lane; i < n_all; i += 32) {
-      const uint32_t t = key_of(__ldcg(gc + i)) - base;
+    visit([&](uint32_t key) {
+      const uint32_t t = key - base;
       if (t < span) {
         if (t - ofs_k < nspan) ++c_in;
         else if (t >= ofs_k) ++c_up;
       }
-    }
+    });
 #pragma unroll
     for (int ofs = 16; ofs > 0; ofs >>= 1) {
       c_in += __shfl_xor_sync(0xffffffffu, c_in, ofs);
@@ -301,28 +357,49 @@ __device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* gc, ui
   uint32_t thr_key = base;
   int g = 0, eq = n_in;
   float m_gt = 0.f, each = 0.f;
-  if (n_in > kCandCapC) {
-    // more than kCandCapC keys share one key value
+  if (n_in > kCandCapC || span == 1u) {
+    // one key value (the usual way here: more than kCandCapC keys share it); its keys are not listed
     each = fast_ex2((okey_to_float(base) - in.ref0) * kLog2eC);
     if (span != 1u) o.bad = 1;
   } else {
     // the candidates of the final interval move into shared memory; each is compared with all the others
     __syncwarp();
     int filled = 0;
-    for (int i0 = 0; i0 < n_all; i0 += 32) {
-      const int i = i0 + lane;
-      uint32_t key = 0u;
-      bool inside = false;
-      if (i < n_all) {
-        key = key_of(__ldcg(gc + i));
-        inside = key - base < span;
+    if (staged) {
+      for (int i0 = 0; i0 < n_all; i0 += 32) {
+        const int i = i0 + lane;
+        const uint32_t key = i < n_all ? wb(i) : 0u;
+        const bool inside = i < n_all && key - base < span;
+        const uint32_t m = __ballot_sync(0xffffffffu, inside);
+        if (inside) {
+          const int p2 = filled + __popc(m & ((1u << lane) - 1u));
+          if (p2 < kCandCapC) hw[p2] = key;
+        }
+        filled += __popc(m);
       }
-      const uint32_t m = __ballot_sync(0xffffffffu, inside);
-      if (inside) {
-        const int p = filled + __popc(m & ((1u << lane) - 1u));
-        if (p < kCandCapC) hw[p] = key;
+    } else {
+      int done = 0;
+      for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
+        const uint32_t* b = pool + (size_t)blk * kBlockWords;
+        const int n_here = min(kBlockEntries, n_all - done);
+        for (int i0 = 0; i0 < n_here; i0 += 32) {
+          const int i = i0 + lane;
+          uint32_t key = 0u;
+          bool inside = false;
+          if (i < n_here) {
+            key = key_of(__ldcg(b + 1 + i));
+            inside = key - base < span;
+          }
+          const uint32_t m = __ballot_sync(0xffffffffu, inside);
+          if (inside) {
+            const int p2 = filled + __popc(m & ((1u << lane) - 1u));
+            if (p2 < kCandCapC) hw[p2] = key;
+          }
+          filled += __popc(m);
+        }
+        done += n_here;
+        blk = __ldcg(b);
       }
-      filled += __popc(m);
     }
     __syncwarp();
     const int n_c = min(n_in, kCandCapC);
@@ -377,6 +454,9 @@ __device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* gc, ui
   int take = eq;   // (a key too light to register in fp32 cannot split its group)
   if (each > 0.f) take = (int)fminf(ceilf((in.target - cum) / each), (float)eq);
   take = max(1, min(take, eq));
+  // Keys of equal score that straddle the cut: when the whole group still ends inside the mass band in which the set
+  // is free (cumulative mass before the group's last key below p + 5e-5), it is taken whole and no position is needed.
+  if (take < eq && cum + (float)(eq - 1) * each <= in.target_hi) take = eq;
   o.cnt_above = above;
   o.mass_above = cum;
   o.thr_key = thr_key;
@@ -425,7 +505,8 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
     const __nv_bfloat16* __restrict__ qt, const int seq_id, const int q_start, const int C,
     int32_t* __restrict__ sel_idx, const int64_t sel_stride, int32_t* __restrict__ sel_count,
     float* __restrict__ sel_mass, float* __restrict__ sel_thresh, int32_t* __restrict__ sel_tie_last, int32_t* status,
-    uint32_t* __restrict__ gcand_all, const int n_row_tiles, const int max_passes) {
+    uint32_t* __restrict__ pool, const uint32_t n_blocks, unsigned int* __restrict__ pool_ctr, const int n_row_tiles,
+    const int max_passes_in) {
   constexpr int BMP = kSRows / G;
   extern __shared__ __align__(1024) unsigned char smem_all[];
   // A kernel that uses tensor memory runs one CTA per SM, so the CTA holds kSubs independent pipelines ("subs") of
@@ -444,6 +525,8 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
   const bool want_ids = sel_idx != nullptr;
   const float scale = d.score_scale;
   const int n_units = n_row_tiles * d.n_ih;
+  const int dbg = max_passes_in >> 8;            // TEMPORARY (timing probes)
+  const int max_passes = max_passes_in & 255;
 
   if (tid == 0) {
     for (int i = 0; i < kSStages; ++i) mbar_init(bar(kFullK + i), 1);
@@ -526,7 +609,6 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
     if (phase != kPhDone) atomicOr(const_cast<int*>(&pass_flags[0]), 1 << kPhMax);
   }
   sub_sync();
-  uint32_t* gc = gcand_all + (size_t)unit * (size_t)(kSRows * kCandCapG) + (size_t)row * kCandCapG;
 
   // level 1
   int aI = 0, w0 = 0;            // grid bin of the maximum; offset of the current 64-bin window below it
@@ -539,6 +621,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
   float raw_lo = __int_as_float(0x7f800000), raw_hi = -__int_as_float(0x7f800000);
   float ref_s = 0.f, e_ref = 0.f;
   int cnt_above = 0, cand_cnt = 0, tie_need = 0, tie_run = 0;
+  uint32_t blk_first = kNoBlock;   // first block of the row's list
 
   // page `page` of the current pass, the g-th page this pipeline has walked since the kernel started: stage g % kSStages
   const int64_t bt_base = (int64_t)seq_id * cv.max_pages;
@@ -742,7 +825,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
             e_ref = fast_ex2(-(float)(w0 + found) * (kLog2eC * 0.25f));
             cand_cnt = 0;
             cnt_above = 0;
-            const bool few = q_found < 0.999f * kMinQ18 * (float)kCandCapG;
+            const bool few = q_found < 0.999f * kMinQ18 * (float)kListMax;
             phase = (few || span == 1u) ? kPhCollect : kPhKey;
           }
         }
@@ -767,6 +850,10 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
         const uint32_t qhalf = qbase + (uint32_t)((keying ? 4 : 28) * kSRows * 4);
         uint32_t qa = qbase;                               // address of the next free queue word (512 bytes apart)
         int cnt = 0, above = 0;
+        uint32_t blk_cur = kNoBlock;                       // collecting rows: the block being filled and its entry count
+        int fill = 0;
+        bool ovf = false;
+        blk_first = kNoBlock;
         auto warp_flush = [&](const bool everything) {
           const uint32_t m = __ballot_sync(0xffffffffu, everything ? qa > qbase : qa > qhalf);
           for (uint32_t rest = m; rest; rest &= rest - 1u) {
@@ -774,10 +861,50 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
             const uint32_t qb_l = __shfl_sync(0xffffffffu, qbase, l);
             const int qn_l = (int)((__shfl_sync(0xffffffffu, qa, l) - qb_l) / (uint32_t)(kSRows * 4));
             if (!__shfl_sync(0xffffffffu, (int)keying, l)) {
-              const int cnt_l = __shfl_sync(0xffffffffu, cnt, l);
-              uint32_t* g_l = gc + (ptrdiff_t)(l - lane) * kCandCapG;
-              for (int i = lane; i < qn_l; i += 32)
-                if (cnt_l + i < kCandCapG) g_l[cnt_l + i] = lds32(qb_l + (uint32_t)i * (kSRows * 4));
+              // (a bucket of one key value needs no list: its keys are only counted)
+              if (__shfl_sync(0xffffffffu, span, l) == 1u) {
+                if (lane == l) {
+                  cnt += qn_l;
+                  qa = qbase;
+                }
+                continue;
+              }
+              // the entries go behind the `fill` entries of the row's current block and, when that is full, on into a
+              // new block from the pool (an exhausted pool marks the row: it is narrowed by a key level instead)
+              uint32_t cur_l = __shfl_sync(0xffffffffu, blk_cur, l);
+              const int fill_l = __shfl_sync(0xffffffffu, fill, l);
+              const int room = cur_l == kNoBlock ? 0 : kBlockEntries - fill_l;
+              uint32_t nb = kNoBlock;
+              if (qn_l > room) {
+                if (lane == 0) {
+                  nb = atomicAdd(pool_ctr, 1u);
+                  if (nb < n_blocks) {
+                    pool[(size_t)nb * kBlockWords] = kNoBlock;
+                    if (cur_l != kNoBlock) pool[(size_t)cur_l * kBlockWords] = nb;
+                  } else {
+                    nb = kNoBlock;
+                  }
+                }
+                nb = __shfl_sync(0xffffffffu, nb, 0);
+              }
+              for (int i = lane; i < qn_l; i += 32) {
+                const uint32_t v = lds32(qb_l + (uint32_t)i * (kSRows * 4));
+                if (i < room) pool[(size_t)cur_l * kBlockWords + 1 + fill_l + i] = v;
+                else if (nb != kNoBlock) pool[(size_t)nb * kBlockWords + 1 + (i - room)] = v;
+              }
+              if (lane == l) {
+                if (qn_l > room) {
+                  if (nb == kNoBlock) {
+                    ovf = true;
+                  } else {
+                    if (blk_first == kNoBlock) blk_first = nb;
+                    blk_cur = nb;
+                    fill = qn_l - room;
+                  }
+                } else {
+                  fill += qn_l;
+                }
+              }
             } else {
               const uint32_t base_l = __shfl_sync(0xffffffffu, base_key, l), span_l = __shfl_sync(0xffffffffu, span, l);
               const int shift_l = __shfl_sync(0xffffffffu, shift, l);
@@ -816,7 +943,9 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
               }
             }
           }
-          if (__any_sync(0xffffffffu, qa > qfull)) warp_flush(false);
+          if (__any_sync(0xffffffffu, qa > qfull)) {
+            if (dbg & 2) qa = qbase; else warp_flush(false);
+          }
         };
         auto proc_late = [&](const uint32_t(&r)[16], const int n0, const bool interior) {
           proc8(&r[0], n0, interior);
@@ -831,10 +960,6 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           RTP_SEL_TILE_END
         }
         warp_flush(true);
-        if (collecting && cnt > kCandCapG) {   // the bucket's mass bounds its size below the list's capacity: cannot happen
-          set_status(status, RTP_ERR_CAPACITY);
-          cnt = kCandCapG;
-        }
         if (keying) {
           // bins in order of decreasing score: 63 is the top
           float run = mass_above;
@@ -878,12 +1003,13 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
             shift = max(0, shift - 6);
             cand_cnt = 0;
             cnt_above = 0;
-            const bool few = q_found < 0.999f * kMinQ11 * (float)kCandCapG;
+            const bool few = q_found < 0.999f * kMinQ11 * (float)kListMax;
             phase = (few || sub_span == 1u) ? kPhCollect : kPhKey;
           }
         } else if (collecting) {
           cand_cnt = cnt;
           cnt_above = above;
+          if (ovf) phase = kPhKey;   // no room for the bucket's keys: one key level first
         } else if (tying) {
           if (tie_last < 0) {           // fewer ties than counted before: cannot happen
             set_status(status, RTP_ERR_UNSUPPORTED);
@@ -894,7 +1020,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
         // ---- exact finish of the rows that collected, one row at a time by the whole warp ----
         sub_sync();   // every row has read its histogram: the carry words become scratch
         uint32_t* hw = reinterpret_cast<uint32_t*>(smem + kCarryOff) + warp * 512;
-        const uint32_t need = __ballot_sync(0xffffffffu, collecting);
+        const uint32_t need = (dbg & 1) ? 0u : __ballot_sync(0xffffffffu, collecting && !ovf);
         for (uint32_t rest = need; rest; rest &= rest - 1u) {
           const int rr = __ffs(rest) - 1;
           FinIn fi;
@@ -903,6 +1029,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           fi.n_keys = __shfl_sync(0xffffffffu, n_keys, rr);
           fi.m_above = __shfl_sync(0xffffffffu, mass_above, rr);
           fi.target = __shfl_sync(0xffffffffu, target, rr);
+          fi.target_hi = (d.top_p + 5e-5f) * __shfl_sync(0xffffffffu, Z, rr);
           fi.ref_s = __shfl_sync(0xffffffffu, ref_s, rr);
           fi.e_ref = __shfl_sync(0xffffffffu, e_ref, rr);
           fi.ref0 = __shfl_sync(0xffffffffu, ref0, rr);
@@ -910,8 +1037,8 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           fi.scale = scale;
           fi.base = __shfl_sync(0xffffffffu, base_key, rr);
           fi.span = __shfl_sync(0xffffffffu, span, rr);
-          const uint32_t* gcr = gc + (ptrdiff_t)(rr - lane) * kCandCapG;
-          const FinOut fo = finish_row(fi, gcr, hw, lane);
+          const FinOut fo = finish_row(fi, pool, __shfl_sync(0xffffffffu, blk_first, rr), hw,
+                                       reinterpret_cast<uint32_t*>(smem + kHistOff), warp, lane);
           if (lane == rr) {
             phase = fo.phase;
             cnt_above = fo.cnt_above;
@@ -965,7 +1092,10 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
   // ---- results ----
   if (row_ok) {
     const int64_t o = (int64_t)(r0 + po) * d.n_ret + rh_head;
-    if (phase != kPhDone) set_status(status, RTP_ERR_TIMEOUT);
+    if (phase != kPhDone) {
+      set_status(status, RTP_ERR_TIMEOUT);
+      atomicAdd(pool_ctr + 8 + phase, 1u);   // (diagnostic: rows left in each phase when the passes ran out)
+    }
     sel_count[o] = n_keys == 0 ? 0 : count;
     if (sel_mass) sel_mass[o] = sel_m;
     if (sel_thresh) sel_thresh[o] = thr_key == 0u ? -INFINITY : okey_to_float(thr_key);
@@ -1002,9 +1132,13 @@ template <int G>
 cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                          const __nv_bfloat16* qt, int32_t* sel_idx, int64_t sel_stride, int32_t* sel_count,
                          float* sel_mass, float* sel_thresh, int32_t* sel_tie_last, int32_t* status, void* ws,
-                         int sm_count, cudaStream_t st) {
+                         size_t ws_bytes, int sm_count, cudaStream_t st) {
   cudaError_t e = set_smem_attr<G>();
   if (e != cudaSuccess) return e;
+  if (ws_bytes < 256 + (size_t)kBlockWords * 4) return cudaErrorInvalidValue;
+  e = cudaMemsetAsync(ws, 0, 256, st);   // the pool's block counter
+  if (e != cudaSuccess) return e;
+  const size_t n_blocks = std::min<size_t>((ws_bytes - 256) / ((size_t)kBlockWords * 4), 0x7fffffffu);
   CUtensorMap map_ik;
   e = make_rows_map(&map_ik, cv.ikey, (int64_t)cv.num_pages * cv.n_ih * kPage, kIndexDim, kIndexDim, kPage,
                     (int)CU_TENSOR_MAP_SWIZZLE_32B);
@@ -1015,10 +1149,11 @@ cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm,
   dim3 grid(std::max(1, std::min(sm_count, (n_units + kSubs - 1) / kSubs)));
   int mp = kMaxPasses;
   if (const char* e_ = getenv("RTP_SEL_MAX_PASSES")) mp = atoi(e_);   // TEMPORARY (timing probe)
+  if (const char* e_ = getenv("RTP_SEL_DBG")) mp |= atoi(e_) << 8;    // TEMPORARY
   select_chunk_kernel<G><<<grid, kSubs * kSThreads, kSmemS, st>>>(map_ik, cv, d, hm, qt, rows.seq_id, rows.q_start, (int)rows.R,
                                                           sel_idx, sel_stride, sel_count, sel_mass, sel_thresh,
-                                                          sel_tie_last, status, reinterpret_cast<uint32_t*>(ws), n_row_tiles,
-                                                          mp);
+                                                          sel_tie_last, status, reinterpret_cast<uint32_t*>(ws) + 64, (uint32_t)n_blocks,
+                                                          reinterpret_cast<unsigned int*>(ws), n_row_tiles, mp);
   return cudaGetLastError();
 }
 
@@ -1031,25 +1166,26 @@ static int slot_class(const Dims& d, const HeadMaps& hm) {
   return max_nh <= 1 ? 1 : max_nh <= 2 ? 2 : max_nh <= 4 ? 4 : max_nh <= 8 ? 8 : 0;
 }
 
-// Candidate scratch: kCandCapG entries of 4 bytes per (row, head slot) of every unit.
+// Workspace: a 256-byte header (the pool's block counter) and the block pool, kRowPoolEntries words per (row, head
+// slot) of every unit.
 size_t select_chunk_workspace_bytes(const Dims& d, const HeadMaps& hm, int64_t R) {
   const int g = slot_class(d, hm);
   if (g == 0 || R <= 0) return 256;
   const int64_t n_row_tiles = (R + kSRows / g - 1) / (kSRows / g);
-  return (size_t)n_row_tiles * d.n_ih * kSRows * kCandCapG * sizeof(uint32_t);
+  return 256 + (size_t)n_row_tiles * d.n_ih * kSRows * kRowPoolEntries * sizeof(uint32_t);
 }
 
 cudaError_t launch_select_chunk(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                                 const __nv_bfloat16* qt, int32_t* sel_idx, int64_t sel_stride,
                                 int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
-                                int32_t* status, void* ws, int sm_count, cudaStream_t st) {
+                                int32_t* status, void* ws, size_t ws_bytes, int sm_count, cudaStream_t st) {
   if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
   if ((int64_t)rows.q_start + rows.R > (int64_t)1 << 21) return cudaErrorNotSupported;   // 8-bit overflow counters of the bins
   switch (slot_class(d, hm)) {
-    case 1: return launch_typed<1>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, sm_count, st);
-    case 2: return launch_typed<2>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, sm_count, st);
-    case 4: return launch_typed<4>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, sm_count, st);
-    case 8: return launch_typed<8>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, sm_count, st);
+    case 1: return launch_typed<1>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, ws_bytes, sm_count, st);
+    case 2: return launch_typed<2>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, ws_bytes, sm_count, st);
+    case 4: return launch_typed<4>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, ws_bytes, sm_count, st);
+    case 8: return launch_typed<8>(cv, d, hm, rows, qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status, ws, ws_bytes, sm_count, st);
     default: return cudaErrorNotSupported;
   }
 }
