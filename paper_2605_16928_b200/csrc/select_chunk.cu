@@ -47,6 +47,7 @@ constexpr int kCandCapC = 64;                 // candidates ranked exactly per r
 constexpr int kBlockWords = 2048;
 constexpr int kBlockEntries = kBlockWords - 1;
 constexpr uint32_t kNoBlock = 0xffffffffu;
+constexpr uint32_t kMarker = 0xffc00000u, kMarkerMask = 0x003fffffu;   // list words that are position markers
 constexpr int kListMax = 65536;               // buckets that may hold more keys are narrowed by a key level first
 constexpr int kRowPoolEntries = 8192;         // pool words the workspace provides per (row, head)
 constexpr int kMaxPasses = 24;
@@ -57,7 +58,7 @@ constexpr uint32_t kMagicBits = 0x4B400000u;
 constexpr int kFixBits = 17;                  // fixed point of the private histograms: 2^17 = upper end of the bin
 // every key adds at least this to its bin (floor(e^-1/4 * 2^17) - 2), which bounds the number of keys by the sum
 constexpr float kMinQ18 = 102077.0f;
-constexpr float kMinQ11 = 1593.0f;            // the same for the 2^11 fixed point of the key-level histograms
+constexpr float kMinQ14 = 12757.0f;           // the same for the 2^14 fixed point of the key-level histograms
 // A bin's 32-bit sum grows by at most 2^23 per page (64 keys x 2^17); every kNormEvery pages the sums above 2^30 hand
 // their upper bits to the bin's 8-bit counter (units of 2^30), so no add in between can wrap: 2^30 + 16 x 2^23 < 2^32.
 // 255 x 2^30 / 2^17 bounds a row at two million keys per bin.
@@ -189,10 +190,6 @@ __device__ __forceinline__ void tmem_wait16(uint32_t (&r)[16]) {
                :
                : "memory");
 }
-__device__ __forceinline__ void red_add_shared(uint32_t a, uint32_t v) {
-  asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
-}
-
 // Grid bin of a score: round(-4 s) as an integer (monotone non-increasing in s; |s| < 2^18).
 __device__ __forceinline__ int grid_bin(float s) { return (int)(__float_as_uint(fmaf(s, -4.0f, kMagicC)) - kMagicBits); }
 
@@ -235,7 +232,10 @@ __device__ __forceinline__ void for_each_entry(const uint32_t* pool, uint32_t fi
   for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
     const uint32_t* b = pool + (size_t)blk * kBlockWords;
     const int n_here = min(kBlockEntries, n_all - done);
-    for (int i = lane; i < n_here; i += 32) f(__ldcg(b + 1 + i));
+    for (int i = lane; i < n_here; i += 32) {
+      const uint32_t w = __ldcg(b + 1 + i);
+      if ((w & kMarker) != kMarker) f(w);   // (position markers are not keys)
+    }
     done += n_here;
     blk = __ldcg(b);
   }
@@ -243,9 +243,9 @@ __device__ __forceinline__ void for_each_entry(const uint32_t* pool, uint32_t fi
 
 // The row's list of unscaled score bits starts in block `first` of the pool (n_all entries, all inside the bucket
 // [base, base + span) of ordered keys); hw: 256 words of shared scratch of this warp; wbuf: the pipeline's histogram
-// memory, idle now, of which this warp owns the words (i / 32) * 128 + 32 * warp + i % 32 for i < 2048.  A list of up
-// to 2048 entries is staged there once, as ordered keys, with four loads in flight per lane; every later round reads
-// shared memory.  Masses are relative to exp(ref0); target and m_above too.
+// memory (or NULL), of which this warp owns the words (i / 32) * 128 + 32 * warp + i % 32 for i < 2048: a list of up
+// to 2048 entries is staged there once, as ordered keys, with four loads in flight per lane, and every later round
+// reads shared memory.  Masses are relative to exp(ref0); target and m_above too.
 // The cut inside the bucket is found on score values alone: when it falls between keys of equal score, the first
 // `tie_need` of them in position order belong to the set and one more pass over the keys finds where that is.
 __device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* pool, const uint32_t first, uint32_t* hw,
@@ -260,7 +260,7 @@ __device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* pool, 
   int n_in = n_all;
   auto key_of = [&](uint32_t raw_bits) { return okey(finish_score(__uint_as_float(raw_bits), in.scale)); };
   auto wb = [&](int i) -> uint32_t& { return wbuf[(i >> 5) * kSRows + 32 * warp + (i & 31)]; };
-  const bool staged = n_all <= 2048 && span > 1u;
+  const bool staged = wbuf != nullptr && n_all <= 2048 && span > 1u;
   if (staged) {
     int done = 0;
     for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
@@ -277,7 +277,7 @@ __device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* pool, 
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int i = i0 + 32 * k + lane;
-          if (i < n_here) wb(done + i) = key_of(v[k]);
+          if (i < n_here) wb(done + i) = (v[k] & kMarker) != kMarker ? key_of(v[k]) : in.base - 1u;   // (markers: outside)
         }
       }
       done += n_here;
@@ -387,8 +387,9 @@ __device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* pool, 
           uint32_t key = 0u;
           bool inside = false;
           if (i < n_here) {
-            key = key_of(__ldcg(b + 1 + i));
-            inside = key - base < span;
+            const uint32_t w = __ldcg(b + 1 + i);
+            key = key_of(w);
+            inside = (w & kMarker) != kMarker && key - base < span;
           }
           const uint32_t m = __ballot_sync(0xffffffffu, inside);
           if (inside) {
@@ -492,8 +493,8 @@ __device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* pool, 
     if (atomicAdd(&rel[buf], 1u) == 3u) {                                               \
       rel[buf] = 0u;                                                                    \
       tc_fence_after();                                                                 \
-      if (it + 2 < n_tiles) issue_mma(gt + 2u);                                         \
-      if (it + kSStages < n_tiles) issue_tma(gt + (uint32_t)kSStages, it + kSStages);   \
+      if (it + 2 < t_hi) issue_mma(gt + 2u);                                            \
+      if (it + kSStages < t_hi) issue_tma(gt + (uint32_t)kSStages, it + kSStages);      \
     }                                                                                   \
   }                                                                                     \
   __syncwarp();                                                                         \
@@ -519,6 +520,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kBarOffS + kNumBarsS * 8 + 4);
   volatile int* pass_flags = reinterpret_cast<volatile int*>(smem + kBarOffS + kNumBarsS * 8 + 8);   // [2]
   unsigned int* rel = reinterpret_cast<unsigned int*>(smem + kBarOffS + kNumBarsS * 8 + 16);         // [2] release tickets
+  int* pass_rng = reinterpret_cast<int*>(smem + kBarOffS + kNumBarsS * 8 + 32);   // [2][2] page range of a pass of tie rows
   auto bar = [&](int i) { return sbase + kBarOffS + i * 8; };
   auto sub_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(1 + sub), "r"(kSThreads) : "memory"); };
   const int seq_len = cv.seq_lens[seq_id];
@@ -570,6 +572,8 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
   if (tid == 0) {
     pass_flags[0] = 0;
     pass_flags[1] = 0;
+    pass_rng[0] = pass_rng[2] = 0x7fffffff;
+    pass_rng[1] = pass_rng[3] = 0;
     if (m0 + rows_here - 1 >= seq_len) set_status(status, RTP_ERR_INVALID);
   }
   sub_sync();
@@ -622,6 +626,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
   float ref_s = 0.f, e_ref = 0.f;
   int cnt_above = 0, cand_cnt = 0, tie_need = 0, tie_run = 0;
   uint32_t blk_first = kNoBlock;   // first block of the row's list
+  int tie_pos_lo = 0, tie_pos_hi = 0x7fffffff;   // tie rows: the positions among which the tie_need-th tie lies
 
   // page `page` of the current pass, the g-th page this pipeline has walked since the kernel started: stage g % kSStages
   const int64_t bt_base = (int64_t)seq_id * cv.max_pages;
@@ -648,12 +653,18 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
       done_emit = 1;
     }
     if (kind == kPassNone || n_tiles == 0) break;
+    // pages walked by the pass: all of them, except when only tie rows are left, which know where to look
+    int t_lo = 0, t_hi = n_tiles;
+    if (kind == kPassLate && flags == (1 << kPhTie) && !(dbg & 8)) {
+      t_lo = max(0, min(pass_rng[2 * (pass & 1)], n_tiles - 1));
+      t_hi = max(t_lo + 1, min(pass_rng[2 * (pass & 1) + 1], n_tiles));
+    }
 
     {
       // prologue of the pass by one thread: request the keys of the first kSStages pages, multiply the first two
       if (warp == 0 && lane == 0) {
-        for (int j = 0; j < kSStages && j < n_tiles; ++j) issue_tma(gt + (uint32_t)j, j);
-        for (int j = 0; j < 2 && j < n_tiles; ++j) issue_mma(gt + (uint32_t)j);
+        for (int j = 0; j < kSStages && t_lo + j < t_hi; ++j) issue_tma(gt + (uint32_t)j, t_lo + j);
+        for (int j = 0; j < 2 && t_lo + j < t_hi; ++j) issue_mma(gt + (uint32_t)j);
       }
       __syncwarp();
       // ================================ score threads (thread = row) ================================
@@ -694,7 +705,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           }
         };
 #pragma unroll 1
-        for (int it = 0; it < n_tiles; ++it) {
+        for (int it = t_lo; it < t_hi; ++it) {
           RTP_SEL_TILE_BEGIN
 #define RTP_P(r_, n0_) proc_max(r_, n0_, interior)
           RTP_SEL_GROUPS(RTP_P)
@@ -705,7 +716,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           const float s_max = finish_score(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)), scale);
           if (!(fabsf(s_max) < 262144.0f)) {
             // no finite score, or scores beyond the range of the fixed grid: every key is kept and the call reports it
-            set_status(status, RTP_ERR_UNSUPPORTED);
+            { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 1); }
             phase = kPhDone;
             tie_last = n_keys - 1;
             count = n_keys;
@@ -748,7 +759,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           }
         };
 #pragma unroll 1
-        for (int it = 0; it < n_tiles; ++it) {
+        for (int it = t_lo; it < t_hi; ++it) {
           RTP_SEL_TILE_BEGIN
           const bool fast = interior && !shifted;
 #define RTP_P(r_, n0_) proc_l1(r_, n0_, fast)
@@ -796,7 +807,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           }
           if (found < 0) {
             // an empty window below the mass already counted: nothing is left to add
-            set_status(status, RTP_ERR_UNSUPPORTED);
+            { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 2); }
             phase = kPhDone;
             tie_last = n_keys - 1;
             count = n_keys;
@@ -830,100 +841,66 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           }
         }
       } else if (kind == kPassLate) {
-        // The unscaled scores inside a row's interval are queued in shared memory and moved on by the whole warp:
-        //   collecting rows   queue = the row's own (idle) histogram column, 64 words; destination = the row's list in
-        //                     global scratch (raw bits, position order); the keys above the interval are counted
-        //   key-level rows    queue = the 16 words of the row's counter column; destination = the 64-bin mass histogram
-        //                     of the next six key bits in the row's histogram column (2^11 fixed point: a bucket that
-        //                     needs a key level holds thousands of keys of nearly equal mass, so coarse rounding of each
-        //                     is harmless and the sums cannot overflow)
-        //   tie rows          no queue: the position of the tie_need-th key with the threshold score is noted in passing
+        // The keys of a row's bucket (unscaled scores inside its interval) are queued in the 16 words of the row's
+        // counter column and, whenever some row of the warp has more than eight queued, every thread works off its own
+        // queue: each key goes into the 64-bin mass histogram of the next six key bits in the row's private histogram
+        // column (2^14 fixed point; a bucket holds at most kListMax keys) and, for collecting rows, onto the row's list
+        // in the pool.  After the pass a row knows the sixty-fourth of its bucket in which the mass reaches the target;
+        // one coalesced sweep over its list moves the keys of that sub-interval (normally a few dozen) into its column,
+        // and the thread walks them in order of decreasing score.  Key-level rows (buckets too large to list) just
+        // adopt the sub-interval as their new bucket.  Tie rows note the position of the tie_need-th key with the
+        // threshold score in passing.
         const bool collecting = phase == kPhCollect, keying = phase == kPhKey, tying = phase == kPhTie;
         const bool listing = collecting || keying;
+        const bool append = collecting && span > 1u;   // (a bucket of one key value needs no list: its keys are counted)
         const float kInfL = __int_as_float(0x7f800000);
         const float lo = listing ? raw_lo : kInfL, hi = listing ? raw_hi : -kInfL;
         const float cut = collecting ? raw_hi : kInfL;
         const float tlo = tying ? raw_lo : kInfL, thi = tying ? raw_hi : -kInfL;
         const bool any_tie = (flags & (1 << kPhTie)) != 0;
-        const uint32_t qbase = keying ? carry_col : hist_col;
-        const uint32_t qfull = qbase + (uint32_t)((keying ? 8 : 56) * kSRows * 4);   // more entries than this: flush
-        const uint32_t qhalf = qbase + (uint32_t)((keying ? 4 : 28) * kSRows * 4);
+        constexpr uint32_t kStep = kSRows * 4;
+        const uint32_t qbase = carry_col, qfull = carry_col + 8u * kStep;
         uint32_t qa = qbase;                               // address of the next free queue word (512 bytes apart)
         int cnt = 0, above = 0;
         uint32_t blk_cur = kNoBlock;                       // collecting rows: the block being filled and its entry count
         int fill = 0;
         bool ovf = false;
         blk_first = kNoBlock;
-        auto warp_flush = [&](const bool everything) {
-          const uint32_t m = __ballot_sync(0xffffffffu, everything ? qa > qbase : qa > qhalf);
-          for (uint32_t rest = m; rest; rest &= rest - 1u) {
-            const int l = __ffs(rest) - 1;
-            const uint32_t qb_l = __shfl_sync(0xffffffffu, qbase, l);
-            const int qn_l = (int)((__shfl_sync(0xffffffffu, qa, l) - qb_l) / (uint32_t)(kSRows * 4));
-            if (!__shfl_sync(0xffffffffu, (int)keying, l)) {
-              // (a bucket of one key value needs no list: its keys are only counted)
-              if (__shfl_sync(0xffffffffu, span, l) == 1u) {
-                if (lane == l) {
-                  cnt += qn_l;
-                  qa = qbase;
-                }
-                continue;
-              }
-              // the entries go behind the `fill` entries of the row's current block and, when that is full, on into a
-              // new block from the pool (an exhausted pool marks the row: it is narrowed by a key level instead)
-              uint32_t cur_l = __shfl_sync(0xffffffffu, blk_cur, l);
-              const int fill_l = __shfl_sync(0xffffffffu, fill, l);
-              const int room = cur_l == kNoBlock ? 0 : kBlockEntries - fill_l;
-              uint32_t nb = kNoBlock;
-              if (qn_l > room) {
-                if (lane == 0) {
-                  nb = atomicAdd(pool_ctr, 1u);
-                  if (nb < n_blocks) {
-                    pool[(size_t)nb * kBlockWords] = kNoBlock;
-                    if (cur_l != kNoBlock) pool[(size_t)cur_l * kBlockWords] = nb;
-                  } else {
-                    nb = kNoBlock;
-                  }
-                }
-                nb = __shfl_sync(0xffffffffu, nb, 0);
-              }
-              for (int i = lane; i < qn_l; i += 32) {
-                const uint32_t v = lds32(qb_l + (uint32_t)i * (kSRows * 4));
-                if (i < room) pool[(size_t)cur_l * kBlockWords + 1 + fill_l + i] = v;
-                else if (nb != kNoBlock) pool[(size_t)nb * kBlockWords + 1 + (i - room)] = v;
-              }
-              if (lane == l) {
-                if (qn_l > room) {
-                  if (nb == kNoBlock) {
-                    ovf = true;
-                  } else {
-                    if (blk_first == kNoBlock) blk_first = nb;
-                    blk_cur = nb;
-                    fill = qn_l - room;
-                  }
-                } else {
-                  fill += qn_l;
-                }
-              }
+        // words of the row's list so far: the bucket's keys and, behind every batch, a marker (a NaN pattern, which no
+        // score has; every reader of a list tells markers from keys by it) with the index of the next group of eight
+        // positions: the keys of a batch lie between the positions of two markers
+        int n_words = 0;
+        auto push = [&](const uint32_t w) {
+          if (blk_cur == kNoBlock || fill == kBlockEntries) {
+            const uint32_t nb = atomicAdd(pool_ctr, 1u);
+            if (nb < n_blocks) {
+              pool[(size_t)nb * kBlockWords] = kNoBlock;
+              if (blk_cur != kNoBlock) pool[(size_t)blk_cur * kBlockWords] = nb; else blk_first = nb;
+              blk_cur = nb;
+              fill = 0;
             } else {
-              const uint32_t base_l = __shfl_sync(0xffffffffu, base_key, l), span_l = __shfl_sync(0xffffffffu, span, l);
-              const int shift_l = __shfl_sync(0xffffffffu, shift, l);
-              const float ref_l = __shfl_sync(0xffffffffu, ref_s, l);
-              const uint32_t hcol_l = __shfl_sync(0xffffffffu, hist_col, l);
-              for (int i = lane; i < qn_l; i += 32) {
-                const float s = finish_score(__uint_as_float(lds32(qb_l + (uint32_t)i * (kSRows * 4))), scale);
-                const uint32_t t = okey(s) - base_l;
-                if (t < span_l) red_add_shared(hcol_l + (uint32_t)(t >> shift_l) * (kSRows * 4), fix_q(fmaf(s - ref_l, kLog2eC, 11.0f)));
-              }
-            }
-            if (lane == l) {
-              cnt += qn_l;
-              qa = qbase;
+              ovf = true;   // the pool is exhausted: the row is narrowed by a key level instead
             }
           }
-          __syncwarp();
+          if (!ovf) {
+            pool[(size_t)blk_cur * kBlockWords + 1 + fill++] = w;
+            ++n_words;
+          }
         };
-        // eight scores; `valid` = how many of them the row may see (8 on interior pages)
+        auto flush_own = [&](const int next_group) {
+          const int qn = (int)((qa - qbase) / kStep);
+          for (int i = 0; i < qn; ++i) {
+            const uint32_t rb = lds32(qbase + (uint32_t)i * kStep);
+            const float s = finish_score(__uint_as_float(rb), scale);
+            const uint32_t t = okey(s) - base_key;
+            if (t < span) hist_add(hist_col, (int)(t >> shift), fix_q(fmaf(s - ref_s, kLog2eC, 14.0f)));
+            if (append && !ovf) push(rb);
+          }
+          if (append && !ovf && qn > 0) push(kMarker | ((uint32_t)next_group & kMarkerMask));
+          cnt += qn;
+          qa = qbase;
+        };
+        // eight scores of the row
         auto proc8 = [&](const uint32_t* r, const int n0, const bool interior) {
           if (interior && !any_tie) {
 #pragma unroll
@@ -936,15 +913,15 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
               if (j < valid && raw > cut) ++above;
               if (j < valid && raw >= lo && raw <= hi) {
                 sts32(qa, r[j]);
-                qa += (uint32_t)(kSRows * 4);
+                qa += kStep;
               }
-              if (j < valid && raw >= tlo && raw <= thi) {
+              if (j < valid && raw >= tlo && raw <= thi && n0 + j >= tie_pos_lo && n0 + j < tie_pos_hi) {
                 if (++tie_run == tie_need) tie_last = n0 + j;
               }
             }
           }
           if (__any_sync(0xffffffffu, qa > qfull)) {
-            if (dbg & 2) qa = qbase; else warp_flush(false);
+            if (!(dbg & 2)) flush_own((n0 + 8) >> 3); else qa = qbase;
           }
         };
         auto proc_late = [&](const uint32_t(&r)[16], const int n0, const bool interior) {
@@ -952,23 +929,26 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           proc8(&r[8], n0 + 8, interior);
         };
 #pragma unroll 1
-        for (int it = 0; it < n_tiles; ++it) {
+        for (int it = t_lo; it < t_hi; ++it) {
           RTP_SEL_TILE_BEGIN
 #define RTP_P(r_, n0_) proc_late(r_, n0_, interior)
           RTP_SEL_GROUPS(RTP_P)
 #undef RTP_P
           RTP_SEL_TILE_END
         }
-        warp_flush(true);
-        if (keying) {
-          // bins in order of decreasing score: 63 is the top
+        flush_own((int)kMarkerMask);
+        // ---- the sub-interval in which the mass reaches the target (bins in order of decreasing score: 63 is the top) ----
+        uint32_t sub_base = base_key, sub_span = span;
+        float sub_above = mass_above;
+        bool sub_ok = true;
+        if (listing && span > 1u && (keying || cnt > kCandCapC)) {
           float run = mass_above;
           int found = -1, last = -1;
           float above_found = 0.f, above_last = 0.f, q_found = 0.f, q_last = 0.f;
           for (int b = kBins - 1; b >= 0; --b) {
-            const uint32_t sum = lds32(hist_col + (uint32_t)b * (kSRows * 4));
+            const uint32_t sum = lds32(hist_col + (uint32_t)b * kStep);
             const float qf = (float)sum;
-            const float m = qf * e_ref * 4.8828125e-04f;   // 2^-11
+            const float m = qf * e_ref * 6.103515625e-05f;   // 2^-14
             if (sum != 0u) {
               last = b;
               above_last = run;
@@ -987,73 +967,255 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
             q_found = q_last;
           }
           if (found < 0) {
-            set_status(status, RTP_ERR_UNSUPPORTED);   // a chosen bucket always holds a key
-            phase = kPhDone;
-            tie_last = n_keys - 1;
-            count = n_keys;
-            sel_m = 1.0f;
+            sub_ok = false;   // a chosen bucket always holds a key
           } else {
-            mass_above = above_found;
             const uint32_t ofs = (uint32_t)found << shift;
-            const uint32_t lo_key = base_key + ofs;
-            const uint32_t sub_span = min(1u << shift, span - ofs);
-            raw_preimage(scale, lo_key, lo_key + (sub_span - 1u), raw_lo, raw_hi);
-            base_key = lo_key;
+            sub_base = base_key + ofs;
+            sub_span = min(1u << shift, span - ofs);
+            sub_above = above_found;
+          }
+          if (keying && sub_ok) {
+            mass_above = sub_above;
+            raw_preimage(scale, sub_base, sub_base + (sub_span - 1u), raw_lo, raw_hi);
+            base_key = sub_base;
             span = sub_span;
             shift = max(0, shift - 6);
             cand_cnt = 0;
             cnt_above = 0;
-            const bool few = q_found < 0.999f * kMinQ11 * (float)kListMax;
+            const bool few = q_found < 0.999f * kMinQ14 * (float)kListMax;
             phase = (few || sub_span == 1u) ? kPhCollect : kPhKey;
           }
-        } else if (collecting) {
-          cand_cnt = cnt;
-          cnt_above = above;
-          if (ovf) phase = kPhKey;   // no room for the bucket's keys: one key level first
-        } else if (tying) {
+        }
+        if (listing && !sub_ok) {
+          { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 3); }
+          phase = kPhDone;
+          tie_last = n_keys - 1;
+          count = n_keys;
+          sel_m = 1.0f;
+        }
+        if (tying) {
           if (tie_last < 0) {           // fewer ties than counted before: cannot happen
-            set_status(status, RTP_ERR_UNSUPPORTED);
+            { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 4); }
             tie_last = n_keys - 1;
           }
           phase = kPhDone;
         }
-        // ---- exact finish of the rows that collected, one row at a time by the whole warp ----
-        sub_sync();   // every row has read its histogram: the carry words become scratch
-        uint32_t* hw = reinterpret_cast<uint32_t*>(smem + kCarryOff) + warp * 512;
-        const uint32_t need = (dbg & 1) ? 0u : __ballot_sync(0xffffffffu, collecting && !ovf);
-        for (uint32_t rest = need; rest; rest &= rest - 1u) {
-          const int rr = __ffs(rest) - 1;
-          FinIn fi;
-          fi.n_all = __shfl_sync(0xffffffffu, cand_cnt, rr);
-          fi.above = __shfl_sync(0xffffffffu, cnt_above, rr);
-          fi.n_keys = __shfl_sync(0xffffffffu, n_keys, rr);
-          fi.m_above = __shfl_sync(0xffffffffu, mass_above, rr);
-          fi.target = __shfl_sync(0xffffffffu, target, rr);
-          fi.target_hi = (d.top_p + 5e-5f) * __shfl_sync(0xffffffffu, Z, rr);
-          fi.ref_s = __shfl_sync(0xffffffffu, ref_s, rr);
-          fi.e_ref = __shfl_sync(0xffffffffu, e_ref, rr);
-          fi.ref0 = __shfl_sync(0xffffffffu, ref0, rr);
-          fi.Z = __shfl_sync(0xffffffffu, Z, rr);
-          fi.scale = scale;
-          fi.base = __shfl_sync(0xffffffffu, base_key, rr);
-          fi.span = __shfl_sync(0xffffffffu, span, rr);
-          const FinOut fo = finish_row(fi, pool, __shfl_sync(0xffffffffu, blk_first, rr), hw,
-                                       reinterpret_cast<uint32_t*>(smem + kHistOff), warp, lane);
-          if (lane == rr) {
-            phase = fo.phase;
-            cnt_above = fo.cnt_above;
-            mass_above = fo.mass_above;
-            thr_key = fo.thr_key;
-            count = fo.count;
-            sel_m = fo.sel_mass;
-            tie_last = fo.tie_last;
-            if (fo.bad) set_status(status, RTP_ERR_UNSUPPORTED);
-            if (fo.phase == kPhTie) {   // the next pass finds the position of the tie_need-th key with this score
-              tie_need = fo.tie_need;
-              tie_run = 0;
-              raw_preimage(scale, thr_key, thr_key, raw_lo, raw_hi);
+        if (collecting && ovf) {        // no room for the bucket's keys: the sub-interval becomes the bucket, listed next pass
+          if (sub_ok && span > 1u) {
+            mass_above = sub_above;
+            raw_preimage(scale, sub_base, sub_base + (sub_span - 1u), raw_lo, raw_hi);
+            base_key = sub_base;
+            span = sub_span;
+            shift = max(0, shift - 6);
+          }
+          cand_cnt = 0;
+          cnt_above = 0;
+        }
+        __syncwarp();   // every thread has read its histogram column: it now receives the row's final candidates
+        // ---- exact finish of the rows that collected ----
+        const bool fin = collecting && !ovf && sub_ok && !(dbg & 1);
+        bool new_tie = false;
+        int c_in = fin ? cnt : 0, c_up = 0;   // keys inside / above the sub-interval (inside the bucket)
+        {
+          // one coalesced sweep over the list of every row whose sub-interval is a part of its bucket
+          const uint32_t sweep = __ballot_sync(0xffffffffu, fin && span > 1u);
+          for (uint32_t rest = sweep; rest; rest &= rest - 1u) {
+            const int rr = __ffs(rest) - 1;
+            const uint32_t first = __shfl_sync(0xffffffffu, blk_first, rr);
+            const int n_all = __shfl_sync(0xffffffffu, n_words, rr);
+            const uint32_t b0 = __shfl_sync(0xffffffffu, base_key, rr), s0 = __shfl_sync(0xffffffffu, span, rr);
+            const uint32_t b1 = __shfl_sync(0xffffffffu, sub_base, rr), s1 = __shfl_sync(0xffffffffu, sub_span, rr);
+            const uint32_t col_rr = __shfl_sync(0xffffffffu, hist_col, rr);
+            int filled = 0, ups = 0, done = 0;
+            for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
+              const uint32_t* b = pool + (size_t)blk * kBlockWords;
+              const int n_here = min(kBlockEntries, n_all - done);
+              const uint32_t next = __ldcg(b);
+              for (int i0 = 0; i0 < n_here; i0 += 128) {
+                uint32_t v[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const int i = i0 + 32 * k + lane;
+                  v[k] = i < n_here ? __ldcg(b + 1 + i) : 0u;
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const int i = i0 + 32 * k + lane;
+                  const uint32_t key = okey(finish_score(__uint_as_float(v[k]), scale));
+                  const bool in_b = i < n_here && (v[k] & kMarker) != kMarker && key - b0 < s0;
+                  const bool inside = in_b && key - b1 < s1;
+                  const uint32_t m = __ballot_sync(0xffffffffu, inside);
+                  ups += __popc(__ballot_sync(0xffffffffu, in_b && !inside && key >= b1));
+                  if (inside) {
+                    const int p2 = filled + __popc(m & ((1u << lane) - 1u));
+                    if (p2 < kCandCapC) sts32(col_rr + (uint32_t)p2 * kStep, key);
+                  }
+                  filled += __popc(m);
+                }
+              }
+              done += n_here;
+              blk = next;
+            }
+            if (lane == rr) {
+              c_in = filled;
+              c_up = ups;
             }
           }
+          __syncwarp();
+        }
+        // rows whose sub-interval still holds more than kCandCapC keys: the warp narrows on the list (rare)
+        {
+          const uint32_t slow = __ballot_sync(0xffffffffu, fin && span > 1u && c_in > kCandCapC);
+          uint32_t* hw = reinterpret_cast<uint32_t*>(smem + kStageOffS) + warp * 256;   // (the key stages are idle between passes)
+          for (uint32_t rest = slow; rest; rest &= rest - 1u) {
+            const int rr = __ffs(rest) - 1;
+            FinIn fi;
+            fi.n_all = __shfl_sync(0xffffffffu, n_words, rr);
+            fi.above = __shfl_sync(0xffffffffu, above + c_up, rr);
+            fi.n_keys = __shfl_sync(0xffffffffu, n_keys, rr);
+            fi.m_above = __shfl_sync(0xffffffffu, sub_above, rr);
+            fi.target = __shfl_sync(0xffffffffu, target, rr);
+            fi.target_hi = (d.top_p + 5e-5f) * __shfl_sync(0xffffffffu, Z, rr);
+            fi.ref_s = __shfl_sync(0xffffffffu, ref_s, rr);
+            fi.e_ref = __shfl_sync(0xffffffffu, e_ref, rr);
+            fi.ref0 = __shfl_sync(0xffffffffu, ref0, rr);
+            fi.Z = __shfl_sync(0xffffffffu, Z, rr);
+            fi.scale = scale;
+            fi.base = __shfl_sync(0xffffffffu, sub_base, rr);
+            fi.span = __shfl_sync(0xffffffffu, sub_span, rr);
+            const FinOut fo = finish_row(fi, pool, __shfl_sync(0xffffffffu, blk_first, rr), hw, nullptr, warp, lane);
+            if (lane == rr) {
+              phase = fo.phase;
+              cnt_above = fo.cnt_above;
+              mass_above = fo.mass_above;
+              thr_key = fo.thr_key;
+              count = fo.count;
+              sel_m = fo.sel_mass;
+              tie_last = fo.tie_last;
+              if (fo.bad) { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 5); }
+              if (fo.phase == kPhTie) {
+                tie_need = fo.tie_need;
+                tie_run = 0;
+                raw_preimage(scale, thr_key, thr_key, raw_lo, raw_hi);
+                new_tie = true;
+              }
+            }
+          }
+          __syncwarp();
+        }
+        // every other collecting row: the thread walks the key values of its column in decreasing order until the mass
+        // reaches the target
+        if (fin && (span == 1u || c_in <= kCandCapC)) {
+          // (thr, g = keys of the sub-interval above it, eq = keys equal to it, m_gt = mass of the g keys, each = mass of one)
+          uint32_t thr = sub_base;
+          int g = 0, eq = c_in;
+          float m_gt = 0.f, each = 0.f;
+          if (span == 1u) {
+            each = fast_ex2((okey_to_float(base_key) - ref0) * kLog2eC);
+          } else {
+            if (c_in <= 0) { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 6); }   // a chosen bucket always holds a key
+            uint32_t bound = 0u;
+            bool first_step = true;
+            for (int step = 0; step < kCandCapC; ++step) {
+              uint32_t mx = 0u;
+              int c = 0;
+              for (int i = 0; i < c_in; ++i) {
+                const uint32_t k = lds32(hist_col + (uint32_t)i * kStep);
+                if (first_step || k < bound) {
+                  if (k > mx) {
+                    mx = k;
+                    c = 1;
+                  } else if (k == mx) {
+                    ++c;
+                  }
+                }
+              }
+              if (c == 0) break;   // every key walked without reaching the target (rounding): the last group stands
+              if (!first_step) {
+                m_gt += (float)eq * each;
+                g += eq;
+              }
+              thr = mx;
+              eq = c;
+              each = fast_ex2((okey_to_float(mx) - ref0) * kLog2eC);
+              first_step = false;
+              bound = mx;
+              if (sub_above + m_gt + (float)eq * each >= target) break;
+            }
+          }
+          const float cum = sub_above + m_gt;
+          int take = eq;   // (a key too light to register in fp32 cannot split its group)
+          if (each > 0.f) take = (int)fminf(ceilf((target - cum) / each), (float)eq);
+          take = max(1, min(take, eq));
+          // Keys of equal score that straddle the cut: when the whole group still ends inside the mass band in which
+          // the set is free (cumulative mass before the group's last key below p + 5e-5), it is taken whole and no
+          // position is needed.
+          if (take < eq && cum + (float)(eq - 1) * each <= (d.top_p + 5e-5f) * Z) take = eq;
+          cnt_above = above + c_up;
+          mass_above = cum;
+          thr_key = thr;
+          count = above + c_up + g + take;
+          sel_m = (cum + (float)take * each) / Z;
+          if (take < eq) {   // the next pass finds the position of the tie_need-th key with this score
+            tie_need = take;
+            tie_run = 0;
+            tie_last = -1;
+            raw_preimage(scale, thr_key, thr_key, raw_lo, raw_hi);
+            phase = kPhTie;
+            new_tie = true;
+          } else {
+            tie_last = n_keys - 1;
+            phase = kPhDone;
+          }
+        }
+        // ---- rows whose cut falls between keys of equal score: where in the list is the tie_need-th of them? ----
+        if (new_tie) {
+          tie_pos_lo = 0;
+          tie_pos_hi = 0x7fffffff;
+        }
+        {
+          const uint32_t loc = __ballot_sync(0xffffffffu, new_tie && span > 1u);
+          for (uint32_t rest = loc; rest; rest &= rest - 1u) {
+            const int rr = __ffs(rest) - 1;
+            const uint32_t first = __shfl_sync(0xffffffffu, blk_first, rr);
+            const int n_all = __shfl_sync(0xffffffffu, n_words, rr);
+            const uint32_t tk = __shfl_sync(0xffffffffu, thr_key, rr);
+            const int need_t = __shfl_sync(0xffffffffu, tie_need, rr);
+            int ties = 0, ties_at_mark = 0, g_lo = 0, g_hi = -1, done = 0;   // g_hi >= 0: found
+            for (uint32_t blk = first; blk != kNoBlock && done < n_all && g_hi < 0;) {
+              const uint32_t* b = pool + (size_t)blk * kBlockWords;
+              const int n_here = min(kBlockEntries, n_all - done);
+              for (int i0 = 0; i0 < n_here && g_hi < 0; i0 += 32) {
+                const int i = i0 + lane;
+                const uint32_t w = i < n_here ? __ldcg(b + 1 + i) : 0u;
+                const bool is_mark = i < n_here && (w & kMarker) == kMarker;
+                const bool is_tie = i < n_here && !is_mark && okey(finish_score(__uint_as_float(w), scale)) == tk;
+                const uint32_t mm = __ballot_sync(0xffffffffu, is_mark), tm = __ballot_sync(0xffffffffu, is_tie);
+                for (uint32_t ev = mm | tm; ev && g_hi < 0; ev &= ev - 1u) {
+                  const int e = __ffs(ev) - 1;
+                  if ((tm >> e) & 1u) {
+                    ++ties;
+                  } else {
+                    const int gmark = (int)(__shfl_sync(0xffffffffu, w, e) & kMarkerMask);
+                    if (ties >= need_t) {
+                      g_hi = gmark;          // the batch that ends here holds the tie_need-th tie
+                    } else {
+                      g_lo = gmark;
+                      ties_at_mark = ties;
+                    }
+                  }
+                }
+              }
+              done += n_here;
+              blk = __ldcg(b);
+            }
+            if (lane == rr && g_hi >= 0 && !(dbg & 16)) {
+              tie_pos_lo = g_lo << 3;
+              tie_pos_hi = g_hi >= (int)kMarkerMask ? 0x7fffffff : g_hi << 3;
+              tie_run = ties_at_mark;
+            }
+          }
+          __syncwarp();
         }
       } else {   // kPassEmit: every resolved row appends its members in position order
         const bool em = row_ok && phase == kPhDone && n_keys > 0;
@@ -1071,7 +1233,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           }
         };
 #pragma unroll 1
-        for (int it = 0; it < n_tiles; ++it) {
+        for (int it = t_lo; it < t_hi; ++it) {
           RTP_SEL_TILE_BEGIN
           (void)interior;
 #define RTP_P(r_, n0_) proc_e(r_, n0_)
@@ -1083,9 +1245,17 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
       }
 #undef RTP_SEL_GROUPS
       if (kind != kPassEmit && phase != kPhDone) atomicOr(const_cast<int*>(&pass_flags[(pass + 1) & 1]), 1 << phase);
+      if (kind != kPassEmit && phase == kPhTie) {
+        atomicMin(&pass_rng[2 * ((pass + 1) & 1)], tie_pos_lo >> kPageShift);
+        atomicMax(&pass_rng[2 * ((pass + 1) & 1) + 1], (int)min((unsigned)n_tiles, (((unsigned)tie_pos_hi - 1u) >> kPageShift) + 1u));
+      }
     }
     sub_sync();
-    if (tid == 0) pass_flags[pass & 1] = 0;
+    if (tid == 0) {
+      pass_flags[pass & 1] = 0;
+      pass_rng[2 * (pass & 1)] = 0x7fffffff;
+      pass_rng[2 * (pass & 1) + 1] = 0;
+    }
     sub_sync();
   }
 
