@@ -49,6 +49,7 @@ constexpr int kBlockEntries = kBlockWords - 1;
 constexpr uint32_t kNoBlock = 0xffffffffu;
 constexpr uint32_t kMarker = 0xffc00000u, kMarkerMask = 0x003fffffu;   // list words that are position markers
 constexpr int kListMax = 65536;               // buckets that may hold more keys are narrowed by a key level first
+constexpr int kSweepLoads = 16;               // list words a lane has in flight during the sweeps after a pass
 constexpr int kRowPoolEntries = 8192;         // pool words the workspace provides per (row, head)
 constexpr int kMaxPasses = 24;
 constexpr int kMaxShift = 63 * 6;             // level-1 windows below this depth hold no representable mass
@@ -190,6 +191,10 @@ __device__ __forceinline__ void tmem_wait16(uint32_t (&r)[16]) {
                :
                : "memory");
 }
+__device__ __forceinline__ void red_add_shared(uint32_t a, uint32_t v) {
+  asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+
 // Grid bin of a score: round(-4 s) as an integer (monotone non-increasing in s; |s| < 2^18).
 __device__ __forceinline__ int grid_bin(float s) { return (int)(__float_as_uint(fmaf(s, -4.0f, kMagicC)) - kMagicBits); }
 
@@ -211,267 +216,6 @@ __device__ void grid_bin_keys(int a, uint32_t& klo, uint32_t& khi) {
     if (grid_bin(okey_to_float(m)) >= a) x = m; else y = m;
   }
   khi = x;
-}
-
-// ---- exact finish of one row by a warp ---------------------------------------------------------------------------
-struct FinIn {
-  int n_all, above, n_keys;
-  float m_above, target, target_hi, ref_s, e_ref, ref0, Z, scale;
-  uint32_t base, span;
-};
-struct FinOut {
-  int phase, cnt_above, count, tie_last, tie_need, bad;
-  float mass_above, sel_mass;
-  uint32_t thr_key;
-};
-
-// Calls f(raw bits) for every entry of a row's list (n_all entries from block `first` on), entries spread over the lanes.
-template <class F>
-__device__ __forceinline__ void for_each_entry(const uint32_t* pool, uint32_t first, int n_all, int lane, F f) {
-  int done = 0;
-  for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
-    const uint32_t* b = pool + (size_t)blk * kBlockWords;
-    const int n_here = min(kBlockEntries, n_all - done);
-    for (int i = lane; i < n_here; i += 32) {
-      const uint32_t w = __ldcg(b + 1 + i);
-      if ((w & kMarker) != kMarker) f(w);   // (position markers are not keys)
-    }
-    done += n_here;
-    blk = __ldcg(b);
-  }
-}
-
-// The row's list of unscaled score bits starts in block `first` of the pool (n_all entries, all inside the bucket
-// [base, base + span) of ordered keys); hw: 256 words of shared scratch of this warp; wbuf: the pipeline's histogram
-// memory (or NULL), of which this warp owns the words (i / 32) * 128 + 32 * warp + i % 32 for i < 2048: a list of up
-// to 2048 entries is staged there once, as ordered keys, with four loads in flight per lane, and every later round
-// reads shared memory.  Masses are relative to exp(ref0); target and m_above too.
-// The cut inside the bucket is found on score values alone: when it falls between keys of equal score, the first
-// `tie_need` of them in position order belong to the set and one more pass over the keys finds where that is.
-__device__ __noinline__ FinOut finish_row(const FinIn in, const uint32_t* pool, const uint32_t first, uint32_t* hw,
-                                          uint32_t* wbuf, const int warp, const int lane) {
-  FinOut o;
-  o.bad = 0;
-  o.tie_need = 0;
-  const int n_all = in.n_all;
-  int above = in.above;
-  float m_above = in.m_above;
-  uint32_t base = in.base, span = in.span;
-  int n_in = n_all;
-  auto key_of = [&](uint32_t raw_bits) { return okey(finish_score(__uint_as_float(raw_bits), in.scale)); };
-  auto wb = [&](int i) -> uint32_t& { return wbuf[(i >> 5) * kSRows + 32 * warp + (i & 31)]; };
-  const bool staged = wbuf != nullptr && n_all <= 2048 && span > 1u;
-  if (staged) {
-    int done = 0;
-    for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
-      const uint32_t* b = pool + (size_t)blk * kBlockWords;
-      const int n_here = min(kBlockEntries, n_all - done);
-      const uint32_t next = __ldcg(b);
-      for (int i0 = 0; i0 < n_here; i0 += 128) {
-        uint32_t v[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const int i = i0 + 32 * k + lane;
-          v[k] = i < n_here ? __ldcg(b + 1 + i) : 0u;
-        }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const int i = i0 + 32 * k + lane;
-          if (i < n_here) wb(done + i) = (v[k] & kMarker) != kMarker ? key_of(v[k]) : in.base - 1u;   // (markers: outside)
-        }
-      }
-      done += n_here;
-      blk = next;
-    }
-    __syncwarp();
-  }
-  // f(key) for every entry of the list, entries spread over the lanes
-  auto visit = [&](auto f) {
-    if (staged) {
-      for (int i = lane; i < n_all; i += 32) f(wb(i));
-    } else {
-      for_each_entry(pool, first, n_all, lane, [&](uint32_t raw_bits) { f(key_of(raw_bits)); });
-    }
-  };
-  // narrow on the list while more than kCandCapC candidates are left: 64-bin mass histogram over the next six key bits
-  while (n_in > kCandCapC && span > 1u) {
-    const int bits = 32 - __clz(span - 1u);
-    const int shift = max(0, bits - 6);
-    for (int i = lane; i < 2 * kBins; i += 32) hw[i] = 0u;
-    __syncwarp();
-    visit([&](uint32_t key) {
-      const uint32_t t = key - base;
-      if (t < span) add_mass(hw + 2 * (t >> shift), fmaf(okey_to_float(key) - in.ref_s, kLog2eC, 20.0f));
-    });
-    __syncwarp();
-    const int b0 = 63 - 2 * lane, b1 = 62 - 2 * lane;   // bin 63 is the top
-    const uint32_t sum0 = hw[2 * b0], car0 = hw[2 * b0 + 1], sum1 = hw[2 * b1], car1 = hw[2 * b1 + 1];
-    const float sc = in.e_ref * 9.5367431640625e-07f;     // 2^-20
-    const float m0f = acc_mass(sum0, car0) * sc, m1f = acc_mass(sum1, car1) * sc;
-    float incm = m0f + m1f;
-#pragma unroll
-    for (int ofs = 1; ofs < 32; ofs <<= 1) {
-      const float tm = __shfl_up_sync(0xffffffffu, incm, ofs);
-      if (lane >= ofs) incm += tm;
-    }
-    const float run = m_above + incm - (m0f + m1f);
-    int found = 64, last = -1;
-    if (sum0 | car0) {
-      last = 2 * lane;
-      if (run + m0f >= in.target) found = 2 * lane;
-    }
-    if (sum1 | car1) {
-      last = 2 * lane + 1;
-      if (found == 64 && run + m0f + m1f >= in.target) found = 2 * lane + 1;
-    }
-#pragma unroll
-    for (int ofs = 16; ofs > 0; ofs >>= 1) {
-      found = min(found, __shfl_xor_sync(0xffffffffu, found, ofs));
-      last = max(last, __shfl_xor_sync(0xffffffffu, last, ofs));
-    }
-    if (found == 64) found = last;
-    if (found < 0) break;                                 // (no candidate inside the interval: cannot happen)
-    m_above = __shfl_sync(0xffffffffu, (found & 1) ? run + m0f : run, found >> 1);
-    const uint32_t ofs_k = (uint32_t)(63 - found) << shift;
-    const uint32_t nbase = base + ofs_k, nspan = min(1u << shift, span - ofs_k);
-    int c_in = 0, c_up = 0;                               // candidates inside / above the new interval
-    visit([&](uint32_t key) {
-      const uint32_t t = key - base;
-      if (t < span) {
-        if (t - ofs_k < nspan) ++c_in;
-        else if (t >= ofs_k) ++c_up;
-      }
-    });
-#pragma unroll
-    for (int ofs = 16; ofs > 0; ofs >>= 1) {
-      c_in += __shfl_xor_sync(0xffffffffu, c_in, ofs);
-      c_up += __shfl_xor_sync(0xffffffffu, c_up, ofs);
-    }
-    above += c_up;
-    n_in = c_in;
-    base = nbase;
-    span = nspan;
-    __syncwarp();
-  }
-  // (thr_key, g = keys of the interval above it, eq = keys equal to it, m_gt = mass of the g keys, each = mass of one)
-  uint32_t thr_key = base;
-  int g = 0, eq = n_in;
-  float m_gt = 0.f, each = 0.f;
-  if (n_in > kCandCapC || span == 1u) {
-    // one key value (the usual way here: more than kCandCapC keys share it); its keys are not listed
-    each = fast_ex2((okey_to_float(base) - in.ref0) * kLog2eC);
-    if (span != 1u) o.bad = 1;
-  } else {
-    // the candidates of the final interval move into shared memory; each is compared with all the others
-    __syncwarp();
-    int filled = 0;
-    if (staged) {
-      for (int i0 = 0; i0 < n_all; i0 += 32) {
-        const int i = i0 + lane;
-        const uint32_t key = i < n_all ? wb(i) : 0u;
-        const bool inside = i < n_all && key - base < span;
-        const uint32_t m = __ballot_sync(0xffffffffu, inside);
-        if (inside) {
-          const int p2 = filled + __popc(m & ((1u << lane) - 1u));
-          if (p2 < kCandCapC) hw[p2] = key;
-        }
-        filled += __popc(m);
-      }
-    } else {
-      int done = 0;
-      for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
-        const uint32_t* b = pool + (size_t)blk * kBlockWords;
-        const int n_here = min(kBlockEntries, n_all - done);
-        for (int i0 = 0; i0 < n_here; i0 += 32) {
-          const int i = i0 + lane;
-          uint32_t key = 0u;
-          bool inside = false;
-          if (i < n_here) {
-            const uint32_t w = __ldcg(b + 1 + i);
-            key = key_of(w);
-            inside = (w & kMarker) != kMarker && key - base < span;
-          }
-          const uint32_t m = __ballot_sync(0xffffffffu, inside);
-          if (inside) {
-            const int p2 = filled + __popc(m & ((1u << lane) - 1u));
-            if (p2 < kCandCapC) hw[p2] = key;
-          }
-          filled += __popc(m);
-        }
-        done += n_here;
-        blk = __ldcg(b);
-      }
-    }
-    __syncwarp();
-    const int n_c = min(n_in, kCandCapC);
-    if (n_c <= 0) o.bad = 1;   // a chosen bucket always holds a key
-    uint32_t key[2];
-    float e[2], mg[2] = {0.f, 0.f};
-    int gg[2] = {0, 0}, ee[2] = {0, 0};
-#pragma unroll
-    for (int x = 0; x < 2; ++x) {
-      const int i = 2 * lane + x;
-      key[x] = i < n_c ? hw[i] : 0u;
-      e[x] = i < n_c ? fast_ex2((okey_to_float(key[x]) - in.ref0) * kLog2eC) : 0.f;
-    }
-    for (int j = 0; j < n_c; ++j) {
-      const uint32_t kj = __shfl_sync(0xffffffffu, (j & 1) ? key[1] : key[0], j >> 1);
-      const float ej = __shfl_sync(0xffffffffu, (j & 1) ? e[1] : e[0], j >> 1);
-#pragma unroll
-      for (int x = 0; x < 2; ++x) {
-        if (kj > key[x]) {
-          ++gg[x];
-          mg[x] += ej;
-        } else if (kj == key[x]) {
-          ++ee[x];
-        }
-      }
-    }
-    // the largest key whose group completes the target (the smallest key if rounding leaves the target out of reach)
-    unsigned long long best = 0ull, lowest = ~0ull;
-#pragma unroll
-    for (int x = 0; x < 2; ++x)
-      if (2 * lane + x < n_c) {
-        const unsigned long long id = ((unsigned long long)key[x] << 8) | (unsigned long long)(2 * lane + x);
-        if (m_above + mg[x] + (float)ee[x] * e[x] >= in.target) best = max(best, id);
-        lowest = min(lowest, id);
-      }
-#pragma unroll
-    for (int ofs = 16; ofs > 0; ofs >>= 1) {
-      best = max(best, __shfl_xor_sync(0xffffffffu, best, ofs));
-      lowest = min(lowest, __shfl_xor_sync(0xffffffffu, lowest, ofs));
-    }
-    if (best == 0ull) best = lowest;
-    const int src = (int)(best & 255ull);
-    const int sl = (src >> 1) & 31, sx = src & 1;
-    thr_key = __shfl_sync(0xffffffffu, sx ? key[1] : key[0], sl);
-    g = __shfl_sync(0xffffffffu, sx ? gg[1] : gg[0], sl);
-    eq = __shfl_sync(0xffffffffu, sx ? ee[1] : ee[0], sl);
-    m_gt = __shfl_sync(0xffffffffu, sx ? mg[1] : mg[0], sl);
-    each = __shfl_sync(0xffffffffu, sx ? e[1] : e[0], sl);
-    __syncwarp();
-  }
-  const float cum = m_above + m_gt;
-  int take = eq;   // (a key too light to register in fp32 cannot split its group)
-  if (each > 0.f) take = (int)fminf(ceilf((in.target - cum) / each), (float)eq);
-  take = max(1, min(take, eq));
-  // Keys of equal score that straddle the cut: when the whole group still ends inside the mass band in which the set
-  // is free (cumulative mass before the group's last key below p + 5e-5), it is taken whole and no position is needed.
-  if (take < eq && cum + (float)(eq - 1) * each <= in.target_hi) take = eq;
-  o.cnt_above = above;
-  o.mass_above = cum;
-  o.thr_key = thr_key;
-  o.count = above + g + take;
-  o.sel_mass = (cum + (float)take * each) / in.Z;
-  if (take < eq) {
-    o.tie_need = take;
-    o.tie_last = -1;
-    o.phase = kPhTie;
-  } else {
-    o.tie_last = in.n_keys - 1;
-    o.phase = kPhDone;
-  }
-  return o;
 }
 
 // One page of the pass: wait for its scores in tensor memory ... release the buffer.  The last of the four warps to
@@ -841,64 +585,108 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           }
         }
       } else if (kind == kPassLate) {
-        // The keys of a row's bucket (unscaled scores inside its interval) are queued in the 16 words of the row's
-        // counter column and, whenever some row of the warp has more than eight queued, every thread works off its own
-        // queue: each key goes into the 64-bin mass histogram of the next six key bits in the row's private histogram
-        // column (2^14 fixed point; a bucket holds at most kListMax keys) and, for collecting rows, onto the row's list
-        // in the pool.  After the pass a row knows the sixty-fourth of its bucket in which the mass reaches the target;
-        // one coalesced sweep over its list moves the keys of that sub-interval (normally a few dozen) into its column,
-        // and the thread walks them in order of decreasing score.  Key-level rows (buckets too large to list) just
-        // adopt the sub-interval as their new bucket.  Tie rows note the position of the tie_need-th key with the
-        // threshold score in passing.
+        // The unscaled scores inside a row's interval are queued in shared memory and moved on by the whole warp:
+        //   collecting rows   queue = the row's own (idle) histogram column, 64 words; destination = the row's list in
+        //                     the pool (raw bits in position order; behind every batch a marker word with the index of
+        //                     the next group of eight positions, so that the keys of a batch are known to lie between
+        //                     the positions of two markers); the keys above the interval are counted
+        //   key-level rows    (buckets too large to list) queue = the 16 words of the row's counter column;
+        //                     destination = the 64-bin mass histogram of the next six key bits in the row's histogram
+        //                     column (2^14 fixed point)
+        //   tie rows          no queue: the position of the tie_need-th key with the threshold score is noted in passing
+        // After the pass the warp takes its collecting rows one by one: a sweep over the list builds the same 64-bin
+        // histogram (only when the bucket holds more than kCandCapC keys), the sixty-fourth of the bucket in which the
+        // mass reaches the target is found, and a second sweep moves the keys of that sub-interval (normally a few dozen)
+        // into the row's column; then every thread walks its own row's candidates in order of decreasing score.
         const bool collecting = phase == kPhCollect, keying = phase == kPhKey, tying = phase == kPhTie;
         const bool listing = collecting || keying;
-        const bool append = collecting && span > 1u;   // (a bucket of one key value needs no list: its keys are counted)
         const float kInfL = __int_as_float(0x7f800000);
         const float lo = listing ? raw_lo : kInfL, hi = listing ? raw_hi : -kInfL;
         const float cut = collecting ? raw_hi : kInfL;
         const float tlo = tying ? raw_lo : kInfL, thi = tying ? raw_hi : -kInfL;
         const bool any_tie = (flags & (1 << kPhTie)) != 0;
         constexpr uint32_t kStep = kSRows * 4;
-        const uint32_t qbase = carry_col, qfull = carry_col + 8u * kStep;
+        const uint32_t qbase = keying ? carry_col : hist_col;
+        const uint32_t qfull = qbase + (uint32_t)(keying ? 8 : 56) * kStep;   // more entries than this: flush
+        const uint32_t qhalf = qbase + (uint32_t)(keying ? 4 : 28) * kStep;
         uint32_t qa = qbase;                               // address of the next free queue word (512 bytes apart)
-        int cnt = 0, above = 0;
-        uint32_t blk_cur = kNoBlock;                       // collecting rows: the block being filled and its entry count
+        int cnt = 0, above = 0, n_words = 0;               // keys seen / keys above the interval / words of the list
+        uint32_t blk_cur = kNoBlock;                       // collecting rows: the block being filled and its word count
         int fill = 0;
         bool ovf = false;
         blk_first = kNoBlock;
-        // words of the row's list so far: the bucket's keys and, behind every batch, a marker (a NaN pattern, which no
-        // score has; every reader of a list tells markers from keys by it) with the index of the next group of eight
-        // positions: the keys of a batch lie between the positions of two markers
-        int n_words = 0;
-        auto push = [&](const uint32_t w) {
-          if (blk_cur == kNoBlock || fill == kBlockEntries) {
-            const uint32_t nb = atomicAdd(pool_ctr, 1u);
-            if (nb < n_blocks) {
-              pool[(size_t)nb * kBlockWords] = kNoBlock;
-              if (blk_cur != kNoBlock) pool[(size_t)blk_cur * kBlockWords] = nb; else blk_first = nb;
-              blk_cur = nb;
-              fill = 0;
+        auto warp_flush = [&](const bool everything, const int next_group) {
+          const uint32_t m = __ballot_sync(0xffffffffu, everything ? qa > qbase : qa > qhalf);
+          for (uint32_t rest = m; rest; rest &= rest - 1u) {
+            const int l = __ffs(rest) - 1;
+            const uint32_t qb_l = __shfl_sync(0xffffffffu, qbase, l);
+            const int qn_l = (int)((__shfl_sync(0xffffffffu, qa, l) - qb_l) / kStep);
+            if (!__shfl_sync(0xffffffffu, (int)keying, l)) {
+              // (a bucket of one key value needs no list: its keys are only counted)
+              if (__shfl_sync(0xffffffffu, span, l) == 1u || __shfl_sync(0xffffffffu, (int)ovf, l)) {
+                if (lane == l) {
+                  cnt += qn_l;
+                  qa = qbase;
+                }
+                continue;
+              }
+              // the words (qn_l keys and the marker) go behind the `fill` words of the row's current block and, when that
+              // is full, on into a new block from the pool (an exhausted pool marks the row: its bucket is narrowed by
+              // a key level instead)
+              const int nw = qn_l + 1;
+              uint32_t cur_l = __shfl_sync(0xffffffffu, blk_cur, l);
+              const int fill_l = __shfl_sync(0xffffffffu, fill, l);
+              const int room = cur_l == kNoBlock ? 0 : kBlockEntries - fill_l;
+              uint32_t nb = kNoBlock;
+              if (nw > room) {
+                if (lane == 0) {
+                  nb = atomicAdd(pool_ctr, 1u);
+                  if (nb < n_blocks) {
+                    pool[(size_t)nb * kBlockWords] = kNoBlock;
+                    if (cur_l != kNoBlock) pool[(size_t)cur_l * kBlockWords] = nb;
+                  } else {
+                    nb = kNoBlock;
+                  }
+                }
+                nb = __shfl_sync(0xffffffffu, nb, 0);
+              }
+              for (int i = lane; i < nw; i += 32) {
+                const uint32_t v = i < qn_l ? lds32(qb_l + (uint32_t)i * kStep) : (kMarker | ((uint32_t)next_group & kMarkerMask));
+                if (i < room) pool[(size_t)cur_l * kBlockWords + 1 + fill_l + i] = v;
+                else if (nb != kNoBlock) pool[(size_t)nb * kBlockWords + 1 + (i - room)] = v;
+              }
+              if (lane == l) {
+                if (nw > room) {
+                  if (nb == kNoBlock) {
+                    ovf = true;
+                  } else {
+                    if (blk_first == kNoBlock) blk_first = nb;
+                    blk_cur = nb;
+                    fill = nw - room;
+                    n_words += nw;
+                  }
+                } else {
+                  fill += nw;
+                  n_words += nw;
+                }
+              }
             } else {
-              ovf = true;   // the pool is exhausted: the row is narrowed by a key level instead
+              const uint32_t base_l = __shfl_sync(0xffffffffu, base_key, l), span_l = __shfl_sync(0xffffffffu, span, l);
+              const int shift_l = __shfl_sync(0xffffffffu, shift, l);
+              const float ref_l = __shfl_sync(0xffffffffu, ref_s, l);
+              const uint32_t hcol_l = __shfl_sync(0xffffffffu, hist_col, l);
+              for (int i = lane; i < qn_l; i += 32) {
+                const float s = finish_score(__uint_as_float(lds32(qb_l + (uint32_t)i * kStep)), scale);
+                const uint32_t t = okey(s) - base_l;
+                if (t < span_l) red_add_shared(hcol_l + (uint32_t)(t >> shift_l) * kStep, fix_q(fmaf(s - ref_l, kLog2eC, 14.0f)));
+              }
+            }
+            if (lane == l) {
+              cnt += qn_l;
+              qa = qbase;
             }
           }
-          if (!ovf) {
-            pool[(size_t)blk_cur * kBlockWords + 1 + fill++] = w;
-            ++n_words;
-          }
-        };
-        auto flush_own = [&](const int next_group) {
-          const int qn = (int)((qa - qbase) / kStep);
-          for (int i = 0; i < qn; ++i) {
-            const uint32_t rb = lds32(qbase + (uint32_t)i * kStep);
-            const float s = finish_score(__uint_as_float(rb), scale);
-            const uint32_t t = okey(s) - base_key;
-            if (t < span) hist_add(hist_col, (int)(t >> shift), fix_q(fmaf(s - ref_s, kLog2eC, 14.0f)));
-            if (append && !ovf) push(rb);
-          }
-          if (append && !ovf && qn > 0) push(kMarker | ((uint32_t)next_group & kMarkerMask));
-          cnt += qn;
-          qa = qbase;
+          __syncwarp();
         };
         // eight scores of the row
         auto proc8 = [&](const uint32_t* r, const int n0, const bool interior) {
@@ -921,7 +709,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
             }
           }
           if (__any_sync(0xffffffffu, qa > qfull)) {
-            if (!(dbg & 2)) flush_own((n0 + 8) >> 3); else qa = qbase;
+            if (dbg & 2) qa = qbase; else warp_flush(false, (n0 + 8) >> 3);
           }
         };
         auto proc_late = [&](const uint32_t(&r)[16], const int n0, const bool interior) {
@@ -936,13 +724,11 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
 #undef RTP_P
           RTP_SEL_TILE_END
         }
-        flush_own((int)kMarkerMask);
-        // ---- the sub-interval in which the mass reaches the target (bins in order of decreasing score: 63 is the top) ----
-        uint32_t sub_base = base_key, sub_span = span;
-        float sub_above = mass_above;
+        warp_flush(true, (int)kMarkerMask);
+        // ---- key-level rows: the sub-interval in which the mass reaches the target becomes the bucket ----
         bool sub_ok = true;
-        if (listing && span > 1u && (keying || cnt > kCandCapC)) {
-          float run = mass_above;
+        if (keying) {
+          float run = mass_above;   // bins in order of decreasing score: 63 is the top
           int found = -1, last = -1;
           float above_found = 0.f, above_last = 0.f, q_found = 0.f, q_last = 0.f;
           for (int b = kBins - 1; b >= 0; --b) {
@@ -969,149 +755,186 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           if (found < 0) {
             sub_ok = false;   // a chosen bucket always holds a key
           } else {
+            mass_above = above_found;
             const uint32_t ofs = (uint32_t)found << shift;
-            sub_base = base_key + ofs;
-            sub_span = min(1u << shift, span - ofs);
-            sub_above = above_found;
-          }
-          if (keying && sub_ok) {
-            mass_above = sub_above;
-            raw_preimage(scale, sub_base, sub_base + (sub_span - 1u), raw_lo, raw_hi);
-            base_key = sub_base;
-            span = sub_span;
+            const uint32_t lo_key = base_key + ofs;
+            const uint32_t s_span = min(1u << shift, span - ofs);
+            raw_preimage(scale, lo_key, lo_key + (s_span - 1u), raw_lo, raw_hi);
+            base_key = lo_key;
+            span = s_span;
             shift = max(0, shift - 6);
             cand_cnt = 0;
             cnt_above = 0;
             const bool few = q_found < 0.999f * kMinQ14 * (float)kListMax;
-            phase = (few || sub_span == 1u) ? kPhCollect : kPhKey;
+            phase = (few || s_span == 1u) ? kPhCollect : kPhKey;
           }
-        }
-        if (listing && !sub_ok) {
-          { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 3); }
-          phase = kPhDone;
-          tie_last = n_keys - 1;
-          count = n_keys;
-          sel_m = 1.0f;
         }
         if (tying) {
           if (tie_last < 0) {           // fewer ties than counted before: cannot happen
-            { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 4); }
+            set_status(status, RTP_ERR_UNSUPPORTED);
             tie_last = n_keys - 1;
           }
           phase = kPhDone;
         }
-        if (collecting && ovf) {        // no room for the bucket's keys: the sub-interval becomes the bucket, listed next pass
-          if (sub_ok && span > 1u) {
-            mass_above = sub_above;
-            raw_preimage(scale, sub_base, sub_base + (sub_span - 1u), raw_lo, raw_hi);
-            base_key = sub_base;
-            span = sub_span;
-            shift = max(0, shift - 6);
-          }
-          cand_cnt = 0;
-          cnt_above = 0;
-        }
+        if (collecting && ovf) phase = kPhKey;   // no room for the bucket's keys: one key level first
         __syncwarp();   // every thread has read its histogram column: it now receives the row's final candidates
         // ---- exact finish of the rows that collected ----
-        const bool fin = collecting && !ovf && sub_ok && !(dbg & 1);
+        const bool fin = collecting && !ovf && !(dbg & 1);
         bool new_tie = false;
+        uint32_t sub_base = base_key, sub_span = span;
+        float sub_above = mass_above;
         int c_in = fin ? cnt : 0, c_up = 0;   // keys inside / above the sub-interval (inside the bucket)
         {
-          // one coalesced sweep over the list of every row whose sub-interval is a part of its bucket
+          uint32_t* hw2 = reinterpret_cast<uint32_t*>(smem + kStageOffS) + warp * 256;   // (the key stages are idle between passes)
+          const uint32_t hw2_a = s_u32(hw2);
           const uint32_t sweep = __ballot_sync(0xffffffffu, fin && span > 1u);
           for (uint32_t rest = sweep; rest; rest &= rest - 1u) {
             const int rr = __ffs(rest) - 1;
             const uint32_t first = __shfl_sync(0xffffffffu, blk_first, rr);
             const int n_all = __shfl_sync(0xffffffffu, n_words, rr);
+            const int n_k = __shfl_sync(0xffffffffu, cnt, rr);
             const uint32_t b0 = __shfl_sync(0xffffffffu, base_key, rr), s0 = __shfl_sync(0xffffffffu, span, rr);
-            const uint32_t b1 = __shfl_sync(0xffffffffu, sub_base, rr), s1 = __shfl_sync(0xffffffffu, sub_span, rr);
+            const float ref_l = __shfl_sync(0xffffffffu, ref_s, rr);
+            const float sc14 = __shfl_sync(0xffffffffu, e_ref, rr) * 6.103515625e-05f;   // 2^-14
+            const float tg = __shfl_sync(0xffffffffu, target, rr);
             const uint32_t col_rr = __shfl_sync(0xffffffffu, hist_col, rr);
-            int filled = 0, ups = 0, done = 0;
-            for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
-              const uint32_t* b = pool + (size_t)blk * kBlockWords;
-              const int n_here = min(kBlockEntries, n_all - done);
-              const uint32_t next = __ldcg(b);
-              for (int i0 = 0; i0 < n_here; i0 += 128) {
-                uint32_t v[4];
+            uint32_t b1 = b0, s1 = s0;      // the interval that holds the cut, narrowed level by level
+            float ab1 = __shfl_sync(0xffffffffu, mass_above, rr);
+            int nk = n_k, filled = 0, ups = 0;
+            bool ok1 = true;
+            for (int level = 0; level < 8 && ok1; ++level) {
+              uint32_t nb = b1, ns = s1;
+              if (nk > kCandCapC && s1 > 1u) {
+                // first sweep: mass histogram of the interval's next six key bits
+                const int shift_l = max(0, 32 - __clz(s1 - 1u) - 6);
+                hw2[lane] = 0u;
+                hw2[lane + 32] = 0u;
+                __syncwarp();
+                int done = 0;
+                for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
+                  const uint32_t* b = pool + (size_t)blk * kBlockWords;
+                  const int n_here = min(kBlockEntries, n_all - done);
+                  const uint32_t next = __ldcg(b);
+                  for (int i0 = 0; i0 < n_here; i0 += 32 * kSweepLoads) {
+                    uint32_t v[kSweepLoads];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  const int i = i0 + 32 * k + lane;
-                  v[k] = i < n_here ? __ldcg(b + 1 + i) : 0u;
-                }
+                    for (int k = 0; k < kSweepLoads; ++k) {
+                      const int i = i0 + 32 * k + lane;
+                      v[k] = i < n_here ? __ldcg(b + 1 + i) : kMarker;
+                    }
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  const int i = i0 + 32 * k + lane;
-                  const uint32_t key = okey(finish_score(__uint_as_float(v[k]), scale));
-                  const bool in_b = i < n_here && (v[k] & kMarker) != kMarker && key - b0 < s0;
-                  const bool inside = in_b && key - b1 < s1;
-                  const uint32_t m = __ballot_sync(0xffffffffu, inside);
-                  ups += __popc(__ballot_sync(0xffffffffu, in_b && !inside && key >= b1));
-                  if (inside) {
-                    const int p2 = filled + __popc(m & ((1u << lane) - 1u));
-                    if (p2 < kCandCapC) sts32(col_rr + (uint32_t)p2 * kStep, key);
+                    for (int k = 0; k < kSweepLoads; ++k) {
+                      const float sc_ = finish_score(__uint_as_float(v[k]), scale);
+                      const uint32_t t = okey(sc_) - b1;
+                      if ((v[k] & kMarker) != kMarker && t < s1)
+                        red_add_shared(hw2_a + 4u * (t >> shift_l), fix_q(fmaf(sc_ - ref_l, kLog2eC, 14.0f)));
+                    }
                   }
-                  filled += __popc(m);
+                  done += n_here;
+                  blk = next;
                 }
+                __syncwarp();
+                // two bins per lane in order of decreasing score: lane l takes bins 63 - 2 l and 62 - 2 l
+                const uint32_t sum0 = hw2[63 - 2 * lane], sum1 = hw2[62 - 2 * lane];
+                const float m0f = (float)sum0 * sc14, m1f = (float)sum1 * sc14;
+                float incm = m0f + m1f;
+#pragma unroll
+                for (int ofs = 1; ofs < 32; ofs <<= 1) {
+                  const float tm = __shfl_up_sync(0xffffffffu, incm, ofs);
+                  if (lane >= ofs) incm += tm;
+                }
+                const float run = ab1 + incm - (m0f + m1f);
+                int found = 64, last = -1;
+                if (sum0) {
+                  last = 2 * lane;
+                  if (run + m0f >= tg) found = 2 * lane;
+                }
+                if (sum1) {
+                  last = 2 * lane + 1;
+                  if (found == 64 && run + m0f + m1f >= tg) found = 2 * lane + 1;
+                }
+#pragma unroll
+                for (int ofs = 16; ofs > 0; ofs >>= 1) {
+                  found = min(found, __shfl_xor_sync(0xffffffffu, found, ofs));
+                  last = max(last, __shfl_xor_sync(0xffffffffu, last, ofs));
+                }
+                if (found == 64) found = last;
+                if (found < 0) {
+                  ok1 = false;   // a chosen interval always holds a key
+                  break;
+                }
+                ab1 = __shfl_sync(0xffffffffu, (found & 1) ? run + m0f : run, found >> 1);
+                const uint32_t ofs_k = (uint32_t)(63 - found) << shift_l;
+                nb = b1 + ofs_k;
+                ns = min(1u << shift_l, s1 - ofs_k);
+                __syncwarp();
               }
-              done += n_here;
-              blk = next;
+              // second sweep: the keys of the sub-interval move into the row's column (as many as fit); the keys of the
+              // interval above it are counted
+              int fl = 0, up = 0, done = 0;
+              for (uint32_t blk = first; blk != kNoBlock && done < n_all;) {
+                const uint32_t* b = pool + (size_t)blk * kBlockWords;
+                const int n_here = min(kBlockEntries, n_all - done);
+                const uint32_t next = __ldcg(b);
+                for (int i0 = 0; i0 < n_here; i0 += 32 * kSweepLoads) {
+                  uint32_t v[kSweepLoads];
+#pragma unroll
+                  for (int k = 0; k < kSweepLoads; ++k) {
+                    const int i = i0 + 32 * k + lane;
+                    v[k] = i < n_here ? __ldcg(b + 1 + i) : kMarker;
+                  }
+#pragma unroll
+                  for (int k = 0; k < kSweepLoads; ++k) {
+                    const uint32_t key = okey(finish_score(__uint_as_float(v[k]), scale));
+                    const bool in_b = (v[k] & kMarker) != kMarker && key - b1 < s1;
+                    const bool inside = in_b && key - nb < ns;
+                    const uint32_t m = __ballot_sync(0xffffffffu, inside);
+                    up += __popc(__ballot_sync(0xffffffffu, in_b && !inside && key >= nb));
+                    if (inside) {
+                      const int p2 = fl + __popc(m & ((1u << lane) - 1u));
+                      if (p2 < kCandCapC) sts32(col_rr + (uint32_t)p2 * kStep, key);
+                    }
+                    fl += __popc(m);
+                  }
+                }
+                done += n_here;
+                blk = next;
+              }
+              ups += up;
+              filled = fl;
+              b1 = nb;
+              s1 = ns;
+              nk = fl;
+              if (nk <= kCandCapC || s1 == 1u) break;
             }
             if (lane == rr) {
               c_in = filled;
               c_up = ups;
+              sub_base = b1;
+              sub_span = s1;
+              sub_above = ab1;
+              if (!ok1) sub_ok = false;
             }
           }
           __syncwarp();
         }
-        // rows whose sub-interval still holds more than kCandCapC keys: the warp narrows on the list (rare)
-        {
-          const uint32_t slow = __ballot_sync(0xffffffffu, fin && span > 1u && c_in > kCandCapC);
-          uint32_t* hw = reinterpret_cast<uint32_t*>(smem + kStageOffS) + warp * 256;   // (the key stages are idle between passes)
-          for (uint32_t rest = slow; rest; rest &= rest - 1u) {
-            const int rr = __ffs(rest) - 1;
-            FinIn fi;
-            fi.n_all = __shfl_sync(0xffffffffu, n_words, rr);
-            fi.above = __shfl_sync(0xffffffffu, above + c_up, rr);
-            fi.n_keys = __shfl_sync(0xffffffffu, n_keys, rr);
-            fi.m_above = __shfl_sync(0xffffffffu, sub_above, rr);
-            fi.target = __shfl_sync(0xffffffffu, target, rr);
-            fi.target_hi = (d.top_p + 5e-5f) * __shfl_sync(0xffffffffu, Z, rr);
-            fi.ref_s = __shfl_sync(0xffffffffu, ref_s, rr);
-            fi.e_ref = __shfl_sync(0xffffffffu, e_ref, rr);
-            fi.ref0 = __shfl_sync(0xffffffffu, ref0, rr);
-            fi.Z = __shfl_sync(0xffffffffu, Z, rr);
-            fi.scale = scale;
-            fi.base = __shfl_sync(0xffffffffu, sub_base, rr);
-            fi.span = __shfl_sync(0xffffffffu, sub_span, rr);
-            const FinOut fo = finish_row(fi, pool, __shfl_sync(0xffffffffu, blk_first, rr), hw, nullptr, warp, lane);
-            if (lane == rr) {
-              phase = fo.phase;
-              cnt_above = fo.cnt_above;
-              mass_above = fo.mass_above;
-              thr_key = fo.thr_key;
-              count = fo.count;
-              sel_m = fo.sel_mass;
-              tie_last = fo.tie_last;
-              if (fo.bad) { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 5); }
-              if (fo.phase == kPhTie) {
-                tie_need = fo.tie_need;
-                tie_run = 0;
-                raw_preimage(scale, thr_key, thr_key, raw_lo, raw_hi);
-                new_tie = true;
-              }
-            }
-          }
-          __syncwarp();
+        if ((keying || fin) && !sub_ok) {
+          set_status(status, RTP_ERR_UNSUPPORTED);
+          phase = kPhDone;
+          tie_last = n_keys - 1;
+          count = n_keys;
+          sel_m = 1.0f;
         }
-        // every other collecting row: the thread walks the key values of its column in decreasing order until the mass
-        // reaches the target
-        if (fin && (span == 1u || c_in <= kCandCapC)) {
+        // every collecting row: the thread walks the key values of its column in decreasing order until the mass reaches
+        // the target (an interval of one key value, which may hold any number of keys, has nothing to walk)
+        if (fin && sub_ok) {
           // (thr, g = keys of the sub-interval above it, eq = keys equal to it, m_gt = mass of the g keys, each = mass of one)
           uint32_t thr = sub_base;
           int g = 0, eq = c_in;
           float m_gt = 0.f, each = 0.f;
-          if (span == 1u) {
-            each = fast_ex2((okey_to_float(base_key) - ref0) * kLog2eC);
+          if (sub_span == 1u || c_in > kCandCapC) {
+            each = fast_ex2((okey_to_float(sub_base) - ref0) * kLog2eC);
+            if (sub_span != 1u) set_status(status, RTP_ERR_UNSUPPORTED);   // (more levels than any key has bits)
           } else {
             if (c_in <= 0) { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 6); }   // a chosen bucket always holds a key
             uint32_t bound = 0u;
