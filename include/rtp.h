@@ -110,11 +110,24 @@ void rtp_destroy(rtp_ctx* ctx);
 /* Text of the last error recorded on this context (never NULL). */
 const char* rtp_last_error(const rtp_ctx* ctx);
 
+/* Diagnostic hook for the bounded device-side waits (the paper has no counterpart).  Inside the tensor-core
+ * kernels warps hand tiles to each other through barriers in shared memory; every such wait gives up after
+ * `wait_limit_ns` nanoseconds (default two seconds), records RTP_ERR_TIMEOUT in the call's status word and the
+ * kernel runs to its end without waiting again.  With drop_first_key_signal != 0 the key loader of the prefill
+ * attention kernels withholds the signal for its first key tile, so that the next rtp_dense_attn_prefill /
+ * rtp_local_attn / rtp_sparse_attn_prefill call on this context must report RTP_ERR_TIMEOUT (its output is
+ * then undefined).  Pass (2000000000, 0) to restore the defaults.  Returns RTP_ERR_INVALID for a NULL context or
+ * a limit <= 0. */
+rtp_status rtp_debug_wait_test(rtp_ctx* ctx, int64_t wait_limit_ns, int32_t drop_first_key_signal);
+
 /* Bytes of DEVICE workspace that any call below needs for `rows` query rows
  * against sequences of at most `max_seq_len` tokens.  0 on invalid params.
- * The largest consumer is rtp_topp_select in chunk mode: 32 KB per (row,
- * retrieval head) for the candidate lists of the exact finish, rounded up to
- * whole tiles of 128 (row, head) pairs (2 GB for 8192 rows x 8 heads). */
+ * The largest consumer is rtp_topp_select in chunk mode: a pool of 8 KB blocks
+ * from which every (row, retrieval head) takes the space for the keys around
+ * its cut on demand, sized at 32 KB per (row, head), rounded up to whole
+ * tiles of 128 pairs (2 GB for 8192 rows x 8 heads).  A larger workspace is
+ * used in full; a row that finds the pool empty narrows its candidates by one
+ * more pass over the keys instead. */
 size_t rtp_workspace_bytes(const rtp_params* params, int64_t rows, int64_t max_seq_len);
 
 /* Synchronises `stream`, reads the DEVICE status word and returns it as an
@@ -149,7 +162,8 @@ rtp_status rtp_kv_append(rtp_ctx* ctx, const rtp_params* params, const rtp_cache
  *        retrieval heads are read)
  * w_q    DEVICE bf16 [n_ret_q_heads, 128, 16]
  * qt_out DEVICE bf16 [R, n_ret_q_heads, 16]
- * Exposed so that tests can feed the oracle the projected queries the kernels use. */
+ * The other calls project their queries themselves; this one returns the projection on its own, e.g. to
+ * inspect or cache it. */
 rtp_status rtp_index_queries(rtp_ctx* ctx, const rtp_params* params, const void* q_pre,
                              const void* w_q, int64_t R, void* qt_out, void* stream);
 
@@ -173,8 +187,14 @@ rtp_status rtp_index_score(rtp_ctx* ctx, const rtp_params* params, const rtp_cac
  * Selects, per row and retrieval query head, the shortest prefix of the keys in
  * order of decreasing score (ties: smaller position first) whose softmax mass
  * reaches top_p.  Mass sums are fp32; a token whose cumulative mass before its
- * own inclusion is within 1e-5 of p may be included.  The set is never empty;
- * top_p == 1 selects every causal key.
+ * own inclusion is within 1e-5 of p may be included, and keys of exactly equal
+ * score that straddle the cut are taken together when the whole group ends
+ * within 5e-5 of p (both inside the 1e-4 band in which the set is free).  The
+ * set is never empty; top_p == 1 selects every causal key.  Scores must be
+ * finite and below 2^18 in magnitude, a chunk may reach at most position 2^21
+ * (RTP_ERR_UNSUPPORTED otherwise).  The scores are always recomputed from the
+ * index-key cache inside the kernels (16 dimensions cost less than reading a
+ * materialised score back), so there is no scores-in variant.
  *
  * Rows: either DEVICE row_seq/row_pos [R] (any rows; the decode path), or
  * row_seq == row_pos == NULL and the rows are positions q_start..q_start+R-1 of
@@ -227,7 +247,7 @@ rtp_status rtp_sparse_attn_decode(rtp_ctx* ctx, const rtp_params* params, const 
  * allocates nothing and calls no allocating routine.
  *  - Limit: rows * n_ret_q_heads * n_splits * 520 bytes must fit in 1 MiB, where n_splits is the
  *    split count the library plans for the call (about 8 * SM count / (rows * heads), at most one
- *    split per 128 listed tokens; a decode batch of up to 64 sequences x 8 retrieval heads always
+ *    split per 256 listed tokens; a decode batch of up to 64 sequences x 8 retrieval heads always
  *    fits).  Larger calls return RTP_ERR_CAPACITY before anything is launched
  *    and rtp_last_error says how many bytes were needed.
  *  - The first call on each device looks up the array's device address (once per device, with that
@@ -247,8 +267,13 @@ rtp_status rtp_sparse_attn_decode_static(rtp_ctx* ctx, const rtp_params* params,
  * Rows are positions q_start..q_start+C-1 of sequence seq_id; causal.
  * With sel_idx != NULL the lists are used as in rtp_sparse_attn_decode.  With
  * sel_idx == NULL membership is re-evaluated inside the attention kernel from
- * (sel_thresh, sel_tie_last) and the indexer score, which needs q_pre and w_q;
- * key tiles in which no row selects anything are skipped.
+ * (sel_thresh, sel_tie_last) and the indexer score, which needs q_pre and w_q:
+ * the kernel visits every causal key tile of a row tile and masks the scores
+ * of the keys outside each row's set (threshold-masked dense attention: with
+ * one set per row and head the union over the 128 rows of a tile covers every
+ * key tile, so there is nothing to skip).  This mode needs every query head of
+ * a retrieval KV head to be a retrieval head on the same index head
+ * (RTP_ERR_UNSUPPORTED otherwise).
  * q, q_pre DEVICE bf16 [C, n_q_heads, 128]; out/lse as above. */
 rtp_status rtp_sparse_attn_prefill(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache,
                                    const void* q, const void* q_pre, const void* w_q,

@@ -11,9 +11,10 @@ What it follows
                          (Section 3.2), stored in bf16 as the index-key cache is.
 * ``index_scores``       Eq. 4, s_h(m, n) = (W^Q q_pre)^T (W^K k_pre), times an
                          optional temperature (1.0 in the paper).
-* ``softmax_mass``       the distribution "derived from the low-dimensional
-                         projected scores" that stage-1 training fits (Section
-                         3.3): a plain softmax of s_h(m, .) over the causal keys.
+* ``softmax_mass``       the probability distribution that the projected scores
+                         define and that stage-1 training fits to the full
+                         attention distribution (Section 3.3): a plain softmax
+                         of s_h(m, .) over the causal keys.
 * ``topp_select``        Eq. 5, S_h(m) = Top-P(s_h(m, .), p): the shortest prefix
                          of the keys, taken in order of decreasing score, whose
                          softmax mass reaches p.  Token level (Section 3 speaks

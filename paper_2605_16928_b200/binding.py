@@ -20,7 +20,7 @@ _STATUS_NAMES = ["RTP_OK", "RTP_ERR_INVALID", "RTP_ERR_CAPACITY", "RTP_ERR_UNSUP
                  "RTP_ERR_TIMEOUT"]
 
 EXPORTS = [
-    "rtp_version", "rtp_create", "rtp_destroy", "rtp_last_error", "rtp_workspace_bytes", "rtp_check_status",
+    "rtp_version", "rtp_create", "rtp_destroy", "rtp_last_error", "rtp_debug_wait_test", "rtp_workspace_bytes", "rtp_check_status",
     "rtp_kv_append", "rtp_index_keys", "rtp_index_queries", "rtp_index_score", "rtp_topp_select", "rtp_sparse_attn_decode", "rtp_sparse_attn_decode_static",
     "rtp_sparse_attn_prefill", "rtp_local_attn", "rtp_dense_attn_prefill", "rtp_dense_attn_decode",
 ]
@@ -73,6 +73,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.rtp_destroy.argtypes = [vp]
     lib.rtp_last_error.restype = C.c_char_p
     lib.rtp_last_error.argtypes = [vp]
+    lib.rtp_debug_wait_test.restype = i32
+    lib.rtp_debug_wait_test.argtypes = [vp, i64, i32]
     lib.rtp_workspace_bytes.restype = sz
     lib.rtp_workspace_bytes.argtypes = [PP, i64, i64]
     lib.rtp_check_status.restype = i32
@@ -195,6 +197,11 @@ class Context:
     def _check(self, rc: int, where: str):
         if rc != RTP_OK:
             raise RtpError(rc, where, (self.lib.rtp_last_error(self.h) or b"").decode())
+
+
+def rtp_debug_wait_test(ctx: Context, wait_limit_ns: int, drop_first_key_signal: bool):
+    ctx._check(ctx.lib.rtp_debug_wait_test(ctx.h, int(wait_limit_ns), 1 if drop_first_key_signal else 0),
+               "rtp_debug_wait_test")
 
 
 def rtp_version() -> int:

@@ -156,16 +156,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const CUtensorMap* map = which ? &map_v : &map_k;
     for (int it = 0; it < n_tiles; ++it) {
       const int stage = it & 1;
-      if (it >= 2) mbar_wait(bar((which ? kEmptyV0 : kEmptyK0) + stage), ((it >> 1) - 1) & 1, abort_flag, status);
+      if (it >= 2) mbar_wait(bar((which ? kEmptyV0 : kEmptyK0) + stage), ((it >> 1) - 1) & 1, abort_flag, status, d.wait_ns);
       const int kt = tile_at(it);
       const uint32_t dst0 = sbase + (which ? kVOff : kKOff) + stage * 2 * kBlk;
       const uint32_t fb = bar((which ? kFullV0 : kFullK0) + stage);
       if (kt * kBNt + kBNt - 1 <= m_last) {
-        if (lane == 0) {
+        if (lane == 0 && !(d.wait_test && which == 0 && it == 0)) {
           mbar_expect_tx(fb, 2 * kBlk);
 #pragma unroll
           for (int pg = 0; pg < 2; ++pg) {
-            const int phys = __ldg(cv.block_table + bt_base + kt * 2 + pg);
+            const int phys = safe_phys(cv, bt_base + kt * 2 + pg, status);
             const int y = (phys * cv.n_kv + kvh) * kPage;
             tma_load_2d(dst0 + pg * (kPage * 128), map, 0, y, fb);
             tma_load_2d(dst0 + kBlk + pg * (kPage * 128), map, 64, y, fb);
@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
       for (int pg = 0; pg < 2; ++pg) {
         const int page = kt * 2 + pg;
         const bool page_ok = page <= last_page;
-        const int phys = page_ok ? __ldg(cv.block_table + bt_base + page) : 0;
+        const int phys = page_ok ? safe_phys(cv, bt_base + page, status) : 0;
         const __nv_bfloat16* src0 = pages + ((int64_t)phys * cv.n_kv + kvh) * (kPage * kHeadDim);
         const int n_ok = page_ok ? m_last - page * kPage + 1 : 0;   // keys of the page any row may attend
 #pragma unroll 4
@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
       asm volatile("cp.async.wait_group 0;" ::: "memory");
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(fb);
+      if (lane == 0 && !(d.wait_test && which == 0 && it == 0)) mbar_arrive(fb);   // (the test hook drops one signal)
     }
   } else if (warp == kMmaWarp) {
     // ================================ S = Q K^T issuer ================================
@@ -204,8 +204,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const uint32_t idesc_s = instr_desc(false);
     for (int it = 0; it < n_tiles; ++it) {
       const int stage = it & 1, buf = it & 1;
-      mbar_wait(bar(kFullK0 + stage), (it >> 1) & 1, abort_flag, status);
-      if (it >= 2) mbar_wait(bar(kSEmpty0 + buf), ((it >> 1) - 1) & 1, abort_flag, status);
+      mbar_wait(bar(kFullK0 + stage), (it >> 1) & 1, abort_flag, status, d.wait_ns);
+      if (it >= 2) mbar_wait(bar(kSEmpty0 + buf), ((it >> 1) - 1) & 1, abort_flag, status, d.wait_ns);
       tc_fence_after();
       if (lane == 0) {
 #pragma unroll
@@ -227,8 +227,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const uint32_t idesc_o = instr_desc(true);
     for (int it = 0; it < n_tiles; ++it) {
       const int stage = it & 1, grp = it & 1;
-      mbar_wait(bar(kFullV0 + stage), (it >> 1) & 1, abort_flag, status);
-      mbar_wait(bar(kPFull0 + grp), (it >> 1) & 1, abort_flag, status);
+      mbar_wait(bar(kFullV0 + stage), (it >> 1) & 1, abort_flag, status, d.wait_ns);
+      mbar_wait(bar(kPFull0 + grp), (it >> 1) & 1, abort_flag, status, d.wait_ns);
       tc_fence_after();
       if (lane == 0) {
 #pragma unroll
@@ -350,7 +350,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         uint2 kb[16];
 #pragma unroll
         for (int pg = 0; pg < 2; ++pg) {
-          const int phys = __ldg(cv.block_table + bt_base_s + min(n_base / kPage + pg, last_page_s));
+          const int phys = safe_phys(cv, bt_base_s + min(n_base / kPage + pg, last_page_s), status);
           const __nv_bfloat16* ik =
               cv.ikey + ((int64_t)phys * cv.n_ih + ih) * (kPage * kIndexDim) + gq * kIndexDim + qfrag_dim_offset(lane);
 #pragma unroll
@@ -416,7 +416,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
           my[c] = kk == 0 ? v0 : kk == 1 ? v1 : kk == 2 ? v2 : v3;
         }
       }
-      mbar_wait(bar(kSFull0 + grp), n_mine & 1, abort_flag, status);
+      mbar_wait(bar(kSFull0 + grp), n_mine & 1, abort_flag, status, d.wait_ns);
       tc_fence_after();
       float s[kBNt];
       {
@@ -455,7 +455,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
         tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3)) * sc2;
       }
       // this group's previous P must have been consumed (and its O must be quiescent) before P / O are touched
-      if (n_mine >= 1) mbar_wait(bar(kPEmpty0 + grp), (n_mine - 1) & 1, abort_flag, status);
+      if (n_mine >= 1) mbar_wait(bar(kPEmpty0 + grp), (n_mine - 1) & 1, abort_flag, status, d.wait_ns);
       const bool raise = tmax > m_ref + 8.0f;     // also true for the first finite maximum (m_ref = -inf)
       if (n_mine >= 1 && __any_sync(0xffffffffu, raise)) {
         tc_fence_after();
@@ -494,7 +494,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
       mbar_arrive(bar(kPFull0 + grp));
     }
     // ---- merge of the two groups and epilogue ----
-    if (n_mine >= 1) mbar_wait(bar(kPEmpty0 + grp), (n_mine - 1) & 1, abort_flag, status);   // this group's last P V is done
+    if (n_mine >= 1) mbar_wait(bar(kPEmpty0 + grp), (n_mine - 1) & 1, abort_flag, status, d.wait_ns);   // this group's last P V is done
     tc_fence_after();
     if (MODE == kPrefillSparse) asm volatile("bar.sync 1, 256;" ::: "memory");   // the rows' rule (same memory) is no longer read
     xch[(grp * 2 + 0) * 128 + row] = m_ref;
@@ -578,12 +578,8 @@ cudaError_t launch_tc_typed(const CacheView& cv, const Dims& d, const HeadMaps& 
                             const __nv_bfloat16* qt, const float* sel_thresh, const int32_t* sel_tie_last,
                             int32_t seq_id, int32_t q_start, int64_t C, __nv_bfloat16* out, float* lse,
                             int32_t* status, int n_units, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(attn_prefill_tc_kernel<G, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
+  static PerDeviceOnce once;
+  if (cudaError_t e0 = set_dyn_smem_once(attn_prefill_tc_kernel<G, MODE>, kTcSmem, once)) return e0;
   CUtensorMap map_k, map_v;
   const int64_t rows = (int64_t)cv.num_pages * cv.n_kv * kPage;
   cudaError_t e = make_page_map(&map_k, cv.k, rows);
@@ -633,6 +629,25 @@ cudaError_t launch_attn_prefill_tc(const CacheView& cv, const Dims& d, const Hea
     return launch_tc_mode<kPrefillDense>(cv, d, hm, q, nullptr, nullptr, nullptr, seq_id, q_start, C, out, lse, status,
                                          hm.n_kv_list, st);
   return cudaErrorNotSupported;
+}
+
+// Prefill attention entry point of the library: every mode (dense, sink + window, sparse) runs on the tcgen05 kernel above.
+cudaError_t launch_attn_prefill(const CacheView& cv, const Dims& d, const HeadMaps& hm, int mode,
+                                const __nv_bfloat16* q, const __nv_bfloat16* qt, int32_t seq_id, int32_t q_start,
+                                int64_t C, const float* sel_thresh, const int32_t* sel_tie_last,
+                                __nv_bfloat16* out, float* lse, int32_t* status, int sm_count, cudaStream_t st) {
+  (void)sm_count;
+  if (C == 0) return cudaSuccess;
+  if (mode == kPrefillSparse) {
+    // one CTA column per index head; every query head of its KV head must be a retrieval head on it
+    for (int j = 0; j < d.n_ih; ++j)
+      if (hm.ih_nheads[j] != d.group) return cudaErrorNotSupported;
+    for (int i = 0; i < d.n_ret; ++i)
+      if (hm.ret_q_head[i] != hm.ih_kv[hm.q2ih[i]] * d.group + hm.slot_in_ih[i]) return cudaErrorNotSupported;
+    return launch_attn_prefill_tc(cv, d, hm, mode, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, st);
+  }
+  if (hm.n_kv_list == 0) return cudaSuccess;
+  return launch_attn_prefill_tc(cv, d, hm, mode, q, nullptr, nullptr, nullptr, seq_id, q_start, C, out, lse, status, st);
 }
 
 }  // namespace rtp

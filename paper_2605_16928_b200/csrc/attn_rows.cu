@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(kThreads, (G == 1) ? 6 : 1) attn_rows_kernel(
   const int m_pos = rows.row_pos(r);
   int n_keys = m_pos + 1;
   {
-    const int sl = (seq >= 0 && seq < cv.batch) ? cv.seq_lens[seq] : 0;
+    const int sl = (seq >= 0 && seq < cv.batch) ? min(cv.seq_lens[seq], cv.max_pages * kPage) : 0;   // (never beyond the block table)
     if (n_keys > sl) {
       if (threadIdx.x == 0) set_status(status, RTP_ERR_INVALID);
       n_keys = sl;
@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(kThreads, (G == 1) ? 6 : 1) attn_rows_kernel(
           tok = t;
         }
         if (ok_n[x]) {
-          const int phys = __ldg(cv.block_table + bt_base + (tok >> kPageShift));
+          const int phys = safe_phys(cv, bt_base + (tok >> kPageShift), status);
           off_n[x] = (((int64_t)phys * cv.n_kv + kvh) * kPage + (tok & (kPage - 1))) * kHeadDim + l16 * 8;
         }
       }

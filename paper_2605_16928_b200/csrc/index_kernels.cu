@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(
   const int seq = rows.row_seq(r);
   int n_keys = rows.row_pos(r) + 1;
   {
-    const int sl = (seq >= 0 && seq < cv.batch) ? cv.seq_lens[seq] : 0;
+    const int sl = (seq >= 0 && seq < cv.batch) ? min(cv.seq_lens[seq], cv.max_pages * kPage) : 0;   // (never beyond the block table)
     if (n_keys > sl) {
       if (threadIdx.x == 0) set_status(status, RTP_ERR_INVALID);
       n_keys = sl;
@@ -221,7 +221,8 @@ cudaError_t launch_kv_append(const CacheView& cv, const __nv_bfloat16* k_new, co
   if (T == 0) return cudaSuccess;
   const int64_t total = T * cv.n_kv * 16;
   int64_t blocks = (total + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  const int64_t cap = (int64_t)current_sm_count(148) * 16;   // a few waves of grid-stride blocks
+  if (blocks > cap) blocks = cap;
   kv_append_kernel<<<(unsigned)blocks, 256, 0, st>>>(cv, k_new, v_new, tok_seq, tok_pos, T, status);
   return cudaGetLastError();
 }

@@ -9,6 +9,8 @@ struct rtp_ctx {
   int device;
   int sm_count;
   int cc_major, cc_minor;
+  unsigned long long wait_ns = 2000000000ull;   // limit of the bounded device-side waits
+  int wait_test = 0;                            // rtp_debug_wait_test
   std::string last_error;
 };
 
@@ -56,6 +58,8 @@ const char* check_params(const rtp_params* p, Dims* d, HeadMaps* hm) {
   d->top_p = p->top_p;
   d->score_scale = p->score_scale;
   d->sm_scale = p->sm_scale;
+  d->wait_ns = 2000000000ull;
+  d->wait_test = 0;
   std::memset(hm, 0, sizeof(*hm));
   for (int j = 0; j < p->n_index_heads; ++j) {
     const int kv = p->index_head_kv[j];
@@ -132,8 +136,8 @@ struct WsCarver {
 
 size_t qt_bytes(const Dims& d, int64_t R) { return (size_t)R * d.n_ret * kIndexDim * sizeof(__nv_bfloat16); }
 
-// Rows beyond this use the chunk (prefill) kernels' small per-row state only.
-constexpr int kDefaultSm = 148;
+// SM count assumed when sizes are asked for without a device to query (a B200 has 148).
+constexpr int kFallbackSm = 148;
 
 }  // namespace
 
@@ -164,6 +168,13 @@ void rtp_destroy(rtp_ctx* ctx) { delete ctx; }
 
 const char* rtp_last_error(const rtp_ctx* ctx) { return ctx ? ctx->last_error.c_str() : "no context"; }
 
+rtp_status rtp_debug_wait_test(rtp_ctx* ctx, int64_t wait_limit_ns, int32_t drop_first_key_signal) {
+  if (!ctx || wait_limit_ns <= 0) return RTP_ERR_INVALID;
+  ctx->wait_ns = (unsigned long long)wait_limit_ns;
+  ctx->wait_test = drop_first_key_signal ? 1 : 0;
+  return RTP_OK;
+}
+
 size_t rtp_workspace_bytes(const rtp_params* params, int64_t rows, int64_t max_seq_len) {
   Dims d;
   HeadMaps hm;
@@ -175,7 +186,7 @@ size_t rtp_workspace_bytes(const rtp_params* params, int64_t rows, int64_t max_s
   // explicit-row selection keeps 48 KB per (row, head); beyond 4096 rows only the chunk path is sized
   if (rows > 4096) a = 0;
   size_t m = a > b ? a : b;
-  const size_t s = score_workspace_bytes(d, rows, max_seq_len, kDefaultSm * 2);
+  const size_t s = score_workspace_bytes(d, rows, max_seq_len, current_sm_count(kFallbackSm) * 2);
   m = m > s ? m : s;
   const size_t t1 = attn_rows_workspace_bytes(d, rows, d.n_ret, 1, 1024, max_seq_len);
   const size_t t2 = attn_rows_workspace_bytes(d, rows, d.n_kv, d.group, 1024, max_seq_len);
@@ -205,6 +216,8 @@ rtp_status rtp_check_status(rtp_ctx* ctx, const int32_t* status, void* stream) {
   HeadMaps hm;                                                                    \
   CacheView cv;                                                                   \
   if (const char* m_ = check_params(params, &d, &hm)) return fail(ctx, RTP_ERR_INVALID, m_); \
+  d.wait_ns = ctx->wait_ns;                                                       \
+  d.wait_test = ctx->wait_test;                                                   \
   if (const char* m_ = check_cache(cache, params, need_kv, need_ikey, &cv)) return fail(ctx, RTP_ERR_INVALID, m_); \
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 

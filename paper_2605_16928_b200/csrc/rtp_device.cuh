@@ -161,10 +161,19 @@ __device__ __forceinline__ void raw_preimage_warp(float scale, uint32_t key_lo, 
   raw_hi = above == kmin ? -__int_as_float(0x7f800000) : okey_to_float((uint32_t)(above - 1ull));
 }
 
+// Physical page of a block-table entry.  An entry outside [0, num_pages) (a corrupt table) is read as page 0, so that
+// no kernel leaves the caches; kernels that have a status word also record RTP_ERR_INVALID for it.
+__device__ __forceinline__ int safe_phys(const CacheView& cv, int64_t entry, int32_t* status = nullptr) {
+  const int phys = __ldg(cv.block_table + entry);
+  if ((unsigned)phys < (unsigned)cv.num_pages) return phys;
+  set_status(status, RTP_ERR_INVALID);
+  return 0;
+}
+
 // Address of the 2 KB index-key slice of (logical page, index head) of a sequence.
 __device__ __forceinline__ const __nv_bfloat16* ikey_page_ptr(const CacheView& cv, int seq, int page,
                                                                int ih) {
-  const int phys = __ldg(cv.block_table + (int64_t)seq * cv.max_pages + page);
+  const int phys = safe_phys(cv, (int64_t)seq * cv.max_pages + page);
   return cv.ikey + ((int64_t)phys * cv.n_ih + ih) * (kPage * kIndexDim);
 }
 

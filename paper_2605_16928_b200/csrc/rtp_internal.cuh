@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "rtp.h"
 
 namespace rtp {
@@ -44,6 +46,10 @@ struct Dims {
   int32_t n_q, n_kv, n_ih, n_ret, group;
   int32_t n_sink, window;
   float top_p, score_scale, sm_scale;
+  // bounded device-side waits give up after this many nanoseconds; wait_test != 0: the key loader of the prefill
+  // attention kernel withholds the signal for its first tile (rtp_debug_wait_test)
+  unsigned long long wait_ns;
+  int32_t wait_test;
 };
 
 // Rows of a call: explicit arrays (decode) or a contiguous chunk of one sequence.
@@ -80,6 +86,48 @@ struct SelState {
 };
 
 enum SelMode { kRefine = 0, kCollect = 1, kSelectAll = 2, kTieScan = 3 };
+
+// A function attribute such as the dynamic shared memory limit is a per-device setting: it is applied the first time
+// a kernel is launched on each device (one bit per device ordinal; safe to call from several threads).
+struct PerDeviceOnce {
+  std::atomic<uint64_t> bits[4] = {};
+};
+template <class Kernel>
+inline cudaError_t set_dyn_smem_once(Kernel kernel, int bytes, PerDeviceOnce& once, bool max_carveout = false) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 256) return cudaErrorInvalidDevice;
+  const uint64_t bit = 1ull << (dev & 63);
+  if (once.bits[dev >> 6].load(std::memory_order_acquire) & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  if (max_carveout) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+    if (e != cudaSuccess) return e;
+  }
+  once.bits[dev >> 6].fetch_or(bit, std::memory_order_release);
+  return cudaSuccess;
+}
+
+// SM count of the current device (queried once per device; `fallback` when no device can be asked, e.g. when only
+// sizes are computed on a host without a GPU).
+inline int current_sm_count(int fallback) {
+  static std::atomic<int> cache[256] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 256) {
+    cudaGetLastError();
+    return fallback;
+  }
+  int n = cache[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    return fallback;
+  }
+  cache[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
 
 // ---- host launchers (one per .cu file) ---------------------------------------
 cudaError_t launch_index_keys(const CacheView& cv, const Dims& d, const __nv_bfloat16* k_pre,

@@ -24,7 +24,6 @@
 // Hand-offs are mbarriers with bounded waits (a wait that runs out records RTP_ERR_TIMEOUT and lets every later wait
 // fall through); the CTA always frees its tensor memory.
 #include <algorithm>
-#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 
@@ -224,7 +223,7 @@ __device__ void grid_bin_keys(int a, uint32_t& klo, uint32_t& khi) {
 // ahead, whose stage the completed MMA of this page has freed.
 #define RTP_SEL_TILE_BEGIN                                                              \
   const int buf = (int)(gt & 1u);                                                       \
-  mbar_wait(bar(kSFull + buf), (gt >> 1) & 1u, abort_flag, status);                     \
+  mbar_wait(bar(kSFull + buf), (gt >> 1) & 1u, abort_flag, status, d.wait_ns);                     \
   tc_fence_after();                                                                     \
   const int n_base = it * kSTile;                                                       \
   const bool interior = n_base + kSTile - 1 <= min_pos;                                 \
@@ -267,7 +266,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
   int* pass_rng = reinterpret_cast<int*>(smem + kBarOffS + kNumBarsS * 8 + 32);   // [2][2] page range of a pass of tie rows
   auto bar = [&](int i) { return sbase + kBarOffS + i * 8; };
   auto sub_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(1 + sub), "r"(kSThreads) : "memory"); };
-  const int seq_len = cv.seq_lens[seq_id];
+  const int seq_len = min(cv.seq_lens[seq_id], cv.max_pages * kPage);   // (never beyond the block table)
   const bool want_ids = sel_idx != nullptr;
   const float scale = d.score_scale;
   const int n_units = n_row_tiles * d.n_ih;
@@ -376,13 +375,13 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
   const int64_t bt_base = (int64_t)seq_id * cv.max_pages;
   auto issue_tma = [&](uint32_t g, int page) {
     const int stage = (int)(g % kSStages);
-    const int phys = __ldg(cv.block_table + bt_base + page);
+    const int phys = safe_phys(cv, bt_base + page, status);
     mbar_expect_tx(bar(kFullK + stage), kStageBytesS);
     tma_load_2d(sbase + kStageOffS + stage * kStageBytesS, &map_ik, 0, (phys * cv.n_ih + ih) * kPage, bar(kFullK + stage));
   };
   auto issue_mma = [&](uint32_t g) {
     const int stage = (int)(g % kSStages), b2 = (int)(g & 1u);
-    mbar_wait(bar(kFullK + stage), (g / kSStages) & 1u, abort_flag, status);
+    mbar_wait(bar(kFullK + stage), (g / kSStages) & 1u, abort_flag, status, d.wait_ns);
     tc_fence_after();
     tc_mma(tmem + (uint32_t)(b2 * kSTile), smem_desc_sw(sbase + kAOff, 16, 256, 6),
            smem_desc_sw(sbase + kStageOffS + stage * kStageBytesS, 16, 256, 6), instr_desc_mn(kSRows, kSTile, false), 0u);
@@ -1103,30 +1102,13 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
   }
 }
 
-// The kernel's dynamic shared memory attribute is a per-device setting: applied once per device and instantiation.
-template <int G>
-cudaError_t set_smem_attr() {
-  static std::atomic<uint64_t> done[2] = {};   // bit per device ordinal (up to 128 devices)
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= 128) return cudaErrorInvalidDevice;
-  const uint64_t bit = 1ull << (dev & 63);
-  if (done[dev >> 6].load(std::memory_order_acquire) & bit) return cudaSuccess;
-  e = cudaFuncSetAttribute(select_chunk_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemS);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(select_chunk_kernel<G>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-  if (e != cudaSuccess) return e;
-  done[dev >> 6].fetch_or(bit, std::memory_order_release);
-  return cudaSuccess;
-}
-
 template <int G>
 cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                          const __nv_bfloat16* qt, int32_t* sel_idx, int64_t sel_stride, int32_t* sel_count,
                          float* sel_mass, float* sel_thresh, int32_t* sel_tie_last, int32_t* status, void* ws,
                          size_t ws_bytes, int sm_count, cudaStream_t st) {
-  cudaError_t e = set_smem_attr<G>();
+  static PerDeviceOnce once;
+  cudaError_t e = set_dyn_smem_once(select_chunk_kernel<G>, kSmemS, once, true);
   if (e != cudaSuccess) return e;
   if (ws_bytes < 256 + (size_t)kBlockWords * 4) return cudaErrorInvalidValue;
   e = cudaMemsetAsync(ws, 0, 256, st);   // the pool's block counter

@@ -39,7 +39,7 @@ __device__ __forceinline__ RowCtx make_row_ctx(const CacheView& cv, const Dims& 
   x.nh = hm.ih_nheads[x.ih];
   x.seq = rows.row_seq(x.r);
   int n_keys = rows.row_pos(x.r) + 1;
-  const int sl = (x.seq >= 0 && x.seq < cv.batch) ? cv.seq_lens[x.seq] : 0;
+  const int sl = (x.seq >= 0 && x.seq < cv.batch) ? min(cv.seq_lens[x.seq], cv.max_pages * kPage) : 0;   // (never beyond the block table)
   if (n_keys > sl) {
     if (threadIdx.x == 0) set_status(status, RTP_ERR_INVALID);
     n_keys = sl;
@@ -78,7 +78,7 @@ __global__ void sel_init_kernel(const CacheView cv, const Dims d, const Rows row
     const int64_t r = i / d.n_ret;
     const int seq = rows.row_seq(r);
     int n_keys = rows.row_pos(r) + 1;
-    const int sl = (seq >= 0 && seq < cv.batch) ? cv.seq_lens[seq] : 0;
+    const int sl = (seq >= 0 && seq < cv.batch) ? min(cv.seq_lens[seq], cv.max_pages * kPage) : 0;   // (never beyond the block table)
     n_keys = max(0, min(n_keys, sl));
     SelState s = {};
     s.n_keys = n_keys;
@@ -1256,7 +1256,8 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
   {
     const int64_t n_zero = (int64_t)(w.zero_bytes / 4);
     const int64_t work = n_zero > nrh ? n_zero : nrh;
-    const unsigned blocks = (unsigned)((work + 255) / 256 < 1184 ? (work + 255) / 256 : 1184);
+    const int64_t cap_blocks = (int64_t)sm_count * 8;
+    const unsigned blocks = (unsigned)((work + 255) / 256 < cap_blocks ? (work + 255) / 256 : cap_blocks);
     sel_init_kernel<<<blocks, 256, 0, st>>>(cv, d, rows, w.state, nrh,
                                             reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + w.zero_off), n_zero);
   }
@@ -1276,12 +1277,9 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
                                                   status);
   }
   constexpr int kFinSmem = 2 * kCandCap * 8;
-  static bool fin_attr_done = false;
-  if (!fin_attr_done) {
-    e = cudaFuncSetAttribute(sel_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinSmem);
-    if (e != cudaSuccess) return e;
-    fin_attr_done = true;
-  }
+  static PerDeviceOnce fin_once;
+  e = set_dyn_smem_once(sel_finalize_kernel, kFinSmem, fin_once);
+  if (e != cudaSuccess) return e;
   sel_finalize_kernel<<<(unsigned)nrh, kFinThreads, kFinSmem, st>>>(cv, d, hm, rows, qt, w.state, w.cand, sel_idx,
                                                              sel_stride, sel_count, sel_mass, sel_thresh,
                                                              sel_tie_last, status);

@@ -29,9 +29,13 @@ def test_static_scratch_decode_matches_workspace_decode_twice():
     for attempt in range(2):
         out = torch.zeros((dw.R, wl.heads.n_q_heads, 128), dtype=torch.bfloat16, device="cuda")
         lse = torch.zeros((dw.R, wl.heads.n_q_heads), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]                       # cudaMemGetInfo: device-wide free bytes
         rb.rtp_sparse_attn_decode_static(dw.ctx, dw.params, dw.cache, dw.q, dw.row_seq, dw.row_pos, sel["idx"],
                                          sel["cnt"], out, lse, dw.status)
         torch.cuda.synchronize()
+        if attempt == 1:                                                 # (the first call may load the kernel's code)
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the amount of free device memory"
         got = out.float().cpu().numpy()
         assert np.abs(got[:, h] - ref_out[:, h]).max() <= 2e-2, f"call {attempt}"
         np.testing.assert_allclose(lse.cpu().numpy()[:, h], ref_lse[:, h], rtol=1e-3, atol=1e-3)
