@@ -10,7 +10,10 @@ attention on local heads.  Metric: prefill tokens per second.
 The JSON line also carries the dense in-library baseline, decode-step latencies (sparse path vs dense
 split-KV decode), the roofline of the dominant kernel and the CPU oracle timed on the host cores.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c3|c2|c5]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c3|c4|c5]
+
+--workload c4 is the one-million-token prefill with planted needles (chunk 16K, one retrieval KV head);
+--workload c5 is the long-context decode sweep (batch x context x top-p x score temperature) printed as one table.
 """
 from __future__ import annotations
 
@@ -126,7 +129,10 @@ def bench_prefill(args, rank, world, device):
     from paper_2605_16928_b200 import synth_device, pipeline
     c4 = args.workload == "c4"
     L, chunk = args.seq_len or (1048576 if c4 else 131072), args.chunk or (16384 if c4 else 8192)
-    data = synth_device.config_3_device(L=L, device=device, ret_kv_heads=(0,) if c4 else (0, 1))
+    if c4:
+        data = synth_device.config_4_device(L=L, device=device)
+    else:
+        data = synth_device.config_3_device(L=L, device=device)
     path = pipeline.PrefillPath(data, chunk)
     stream = torch.cuda.current_stream()
     out = torch.empty((L, path.Hq, 128), dtype=torch.bfloat16, device=device)
@@ -144,6 +150,44 @@ def bench_prefill(args, rank, world, device):
     return data, path, step, step_dense, out, k_pre, chunks, L, chunk, stream
 
 
+def prefill_sparsity(path, data, chunks, L, rows_per_chunk=16, n_chunks=4):
+    """Compute sparsity (per query head) and memory sparsity (union over the query heads of a KV head) of the retrieval
+    heads (Section 3.2), counted on sampled rows of a few chunks from the selection the library wrote and the scores it
+    materialises for those rows.  Counting only: no part of the timed path."""
+    import torch
+    from paper_2605_16928_b200 import binding as rb
+    g, n_ret = data.heads.group, path.n_ret
+    pick = sorted({int(round(x)) for x in np.linspace(0, len(chunks) - 1, min(n_chunks, len(chunks)))})
+    rng = np.random.default_rng(7)
+    comp, mem, ratio = [], [], []
+    R = rows_per_chunk
+    sc = torch.empty((R, n_ret, L), dtype=torch.float32, device=path.dev)
+    ws = torch.empty(rb.rtp_workspace_bytes(path.params, R, L), dtype=torch.uint8, device=path.dev)
+    pos = torch.arange(L, device=path.dev)
+    for ci in pick:
+        s0, C = chunks[ci]
+        q = data.q[s0:s0 + C]
+        rb.rtp_topp_select(path.ctx, path.params, path.cache, q, data.w_q, None, None, 0, s0, C, None, path.sel_cnt,
+                           path.sel_mass, path.sel_thr, path.sel_tie, path.status, path.workspace)
+        r = torch.from_numpy(np.sort(rng.choice(C, size=min(R, C), replace=False))).to(path.dev)
+        rows = (r + s0).to(torch.int32)
+        sc.fill_(float("nan"))
+        rb.rtp_index_score(path.ctx, path.params, path.cache, q[r].contiguous(), data.w_q,
+                           torch.zeros(len(r), dtype=torch.int32, device=path.dev), rows, sc[:len(r)], None, None, ws,
+                           path.status)
+        thr, tie = path.sel_thr[r][:, :, None], path.sel_tie[r][:, :, None]
+        member = (sc[:len(r)] > thr) | ((sc[:len(r)] == thr) & (pos[None, None, :] <= tie))
+        per_head = member.sum(-1).double()                                          # [R, n_ret]
+        union = member.view(len(r), n_ret // g, g, L).any(2).sum(-1).double()        # [R, n_ret / g]
+        ctx_len = (rows.double() + 1.0)[:, None]
+        comp.append((per_head / ctx_len).mean().item())
+        mem.append((union / ctx_len).mean().item())
+        ratio.append((union / per_head.view(len(r), n_ret // g, g).mean(-1)).mean().item())
+    return {"compute_sparsity": 1.0 - float(np.mean(comp)), "memory_sparsity": 1.0 - float(np.mean(mem)),
+            "union_over_mean_head_set": float(np.mean(ratio)),
+            "sample": f"{R} rows in each of chunks {pick}; union over the {g} query heads of a retrieval KV head"}
+
+
 def cpu_oracle_prefill(data, L, rows, budget_s=25.0):
     """Times the CPU oracle on a bounded sample of query rows of the prefill workload (all 32 heads)."""
     from oracle import rtp_oracle as orc
@@ -153,6 +197,7 @@ def cpu_oracle_prefill(data, L, rows, budget_s=25.0):
     kv = {h: data.logical_kv(0, h, 0, L) for h in range(heads.n_kv_heads)}
     q = to_np(data.q[[int(r) for r in rows]])
     w_q, w_k = to_np(data.w_q), to_np(data.w_k)
+    c0 = time.process_time()
     t0 = time.perf_counter()
     kt = [orc.index_project(kv[heads.index_head_kv[j]][0], w_k[j]) for j in range(heads.n_index_heads)]
     t_proj = time.perf_counter() - t0
@@ -171,7 +216,10 @@ def cpu_oracle_prefill(data, L, rows, budget_s=25.0):
         if t_rows + t_proj > budget_s:
             break
     per_tok = t_rows / done + t_proj / L
-    return 1.0 / per_tok, done, t_rows + t_proj
+    # threads the oracle really kept busy: process CPU time over wall time (numpy's BLAS calls may use several, the
+    # sorts and elementwise steps use one)
+    busy = (time.process_time() - c0) / max(1e-9, t_rows + t_proj)
+    return 1.0 / per_tok, done, t_rows + t_proj, max(1, int(round(busy)))
 
 
 # ------------------------------------------------------------------------------------------------ decode extras
@@ -231,6 +279,61 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
     return res
 
 
+def bench_c5_sweep(device, iters=10, batches=(1, 4, 16), contexts=(131072, 524288, 1048576), tops=(0.8, 0.9, 0.99),
+                   fracs=(0.001, 0.02, 0.2)):
+    """The long-context decode sweep: one cache per (batch, context); top-p and the score temperature (set from the
+    Gaussian closed form for a target selected fraction) change the queries only.  One row per point."""
+    import torch
+    from paper_2605_16928_b200 import synth_device, pipeline, binding as rb
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(192 << 20, dtype=torch.uint8, device=device)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        ts = []
+        for _ in range(iters):
+            flush.zero_()
+            ts.append(ev_time_ms(fn, stream) * 1e3)
+        return float(np.median(ts))
+
+    table = []
+    for B in batches:
+        for L in contexts:
+            base = synth_device.decode_device(L, B, 0.9, 0.05, 4096, device=device)
+            path = pipeline.DecodePath(base, L)
+            path.build_index_cache()
+            k_new = torch.stack([base.k_pre_rows(b, L - 1, L)[0] for b in range(B)]).contiguous()
+            heads = base.heads
+            g, n_ih, n_ret = heads.group, heads.n_index_heads, len(heads.ret_q_heads)
+            t_dense = timed(lambda: path.step_dense(base.q))
+            dense_bytes = B * heads.n_kv_heads * 512.0 * L
+            for p in tops:
+                for frac in fracs:
+                    data = synth_device.decode_retarget(base, p, frac)
+                    path.data, path.params = data, rb.Params.from_workload(data)
+                    t = timed(lambda: path.step(data.q, k_new))
+                    cnt = path.sel_cnt.long()
+                    # memory sparsity: union of the lists of the query heads that share a KV head
+                    valid = torch.arange(L, device=device)[None, None, :] < cnt[:, :, None]
+                    bi, hi, ji = torch.nonzero(valid, as_tuple=True)
+                    mask = torch.zeros((B, n_ret // g, L), dtype=torch.bool, device=device)
+                    mask[bi, hi // g, path.sel_idx[bi, hi, ji].long()] = True
+                    union = mask.sum(-1).double()
+                    del valid, bi, hi, ji, mask
+                    sel_rows = float(cnt.sum().item())
+                    alg = B * n_ih * 32.0 * L + 520.0 * sel_rows + B * len(heads.local_kv_heads) * 512.0 * min(L, 4 + 4096)
+                    table.append({"batch": B, "context": L, "top_p": p, "target_fraction": frac,
+                                  "selected_fraction": sel_rows / (B * n_ret * L),
+                                  "union_fraction_per_kv_head": float(union.mean().item()) / L,
+                                  "sparse_step_us": t, "dense_step_us": t_dense, "speedup_vs_dense": t_dense / t,
+                                  "algorithmic_bytes": alg, "sparse_path_gbs": alg / t / 1e3,
+                                  "dense_gbs": dense_bytes / t_dense / 1e3, "status": path.status_code()})
+            del path, base
+            torch.cuda.empty_cache()
+    return table
+
+
 # ------------------------------------------------------------------------------------------------ main
 def main():
     ap = argparse.ArgumentParser()
@@ -238,9 +341,10 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c3", "c4"],
+    ap.add_argument("--workload", default="c3", choices=["c3", "c4", "c5"],
                     help="c3: 128K chunked prefill, 2 retrieval KV heads (default, the bench line); "
-                         "c4: 1M prefill, chunk 16K, 1 retrieval KV head (long run, no end-to-end leg)")
+                         "c4: 1M prefill with planted needles, chunk 16K, 1 retrieval KV head (long run, no end-to-end "
+                         "leg); c5: the long-context decode sweep as one table")
     ap.add_argument("--seq-len", type=int, default=0)
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the dense baseline, decode points and CPU oracle")
@@ -268,13 +372,13 @@ def main():
         import torch
         from paper_2605_16928_b200 import synth_device
         dev = "cuda:0" if torch.cuda.is_available() else "cpu"
-        data = synth_device.config_3_device(L=L, device=dev)
+        data = synth_device.config_4_device(L=L, device=dev) if c4 else synth_device.config_3_device(L=L, device=dev)
         per_step = 24
         rows = np.linspace(L // 16, L - 1, 3 * per_step).astype(np.int64)
         vals = []
         t_all = time.perf_counter()
         for s in range(args.warmup + args.steps):
-            v, done, _ = cpu_oracle_prefill(data, L, rows[(s % 3)::3], budget_s=6.0)
+            v, done, _, used = cpu_oracle_prefill(data, L, rows[(s % 3)::3], budget_s=6.0)
             if s >= args.warmup:
                 vals.append(v)
         value = float(np.mean(vals))
@@ -282,7 +386,8 @@ def main():
                 "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": 1e3 * L / value, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f64", "data": "synthetic", "config": config,
-                "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": n_cores, "kind": "oracle",
+                "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": used, "cores_available": n_cores,
+                                 "kind": "oracle (numpy, fp64)",
                                  "sample": "up to 24 query rows x 32 heads per step (6 s budget), extrapolated to the sequence"},
                 "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
                 "wall_s": time.perf_counter() - t_all}
@@ -300,6 +405,34 @@ def main():
         rbuild.build_library()
     replicas.barrier(dist, device)
     peaks = load_peaks()
+
+    if args.workload == "c5":
+        if rank == 0:
+            sampler = ClockSampler(local_rank)
+            sampler.start()
+            table = bench_c5_sweep(device, iters=max(3, args.steps))
+            clocks = sampler.stop()
+            ref = next(r for r in table if (r["batch"], r["context"], r["top_p"], r["target_fraction"]) == (4, 524288, 0.9, 0.02))
+            hdr = f"{'B':>3} {'context':>8} {'p':>5} {'target':>7} {'selected':>9} {'union':>7} {'sparse us':>10} {'dense us':>10} {'x':>6} {'GB/s':>7}"
+            print(hdr, file=sys.stderr)
+            for r in table:
+                print(f"{r['batch']:>3} {r['context']:>8} {r['top_p']:>5} {r['target_fraction']:>7.3f} {r['selected_fraction']:>9.4f} "
+                      f"{r['union_fraction_per_kv_head']:>7.4f} {r['sparse_step_us']:>10.1f} {r['dense_step_us']:>10.1f} "
+                      f"{r['speedup_vs_dense']:>6.2f} {r['sparse_path_gbs']:>7.0f}", file=sys.stderr)
+            print(json.dumps({"metric": "decode_step_us", "value": ref["sparse_step_us"], "unit": "us", "n_gpus": 1,
+                              "steps": max(3, args.steps), "warmup": 3, "ms_per_step": ref["sparse_step_us"] / 1e3,
+                              "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+                              "data": "synthetic", "clocks": clocks,
+                              "config": {"workload": "c5_decode_sweep", "value_point": "batch 4, context 512K, top-p 0.9, target fraction 2 %",
+                                         "l2": "flushed between timed iterations"},
+                              "roofline": {"bound": "hbm", "achieved": ref["sparse_path_gbs"], "peak": peaks["hbm_gbs"],
+                                           "unit": "GB/s", "frac": ref["sparse_path_gbs"] / peaks["hbm_gbs"], "traffic": None,
+                                           "peak_source": peaks["source"]},
+                              "table": table}))
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
 
     if args.decode_only:
         if rank == 0:
@@ -424,10 +557,12 @@ def main():
     # ---- per-kernel timing of one instrumented step (not part of the timed region) ----
     klass = {"index_keys": 0.0, "select": 0.0, "sparse_attn": 0.0, "local_attn": 0.0}
     d, p = path.data, path.params
+    n_selected = torch.zeros((), dtype=torch.float64, device=device)
     for (s, C) in chunks:
         q, kp, o = data.q[s:s + C], k_pre[s:s + C], out[s:s + C]
         klass["index_keys"] += ev_time_ms(lambda: rb.rtp_index_keys(path.ctx, p, path.cache, kp, d.w_k, path.tok_seq[:C], path.pos_all[s:s + C]), stream)
         klass["select"] += ev_time_ms(lambda: rb.rtp_topp_select(path.ctx, p, path.cache, q, d.w_q, None, None, 0, s, C, None, path.sel_cnt, path.sel_mass, path.sel_thr, path.sel_tie, path.status, path.workspace), stream)
+        n_selected += path.sel_cnt[:C].sum(dtype=torch.float64)
         klass["sparse_attn"] += ev_time_ms(lambda: rb.rtp_sparse_attn_prefill(path.ctx, p, path.cache, q, q, d.w_q, 0, s, C, None, path.sel_cnt, path.sel_thr, path.sel_tie, o, None, path.workspace, path.status), stream)
         klass["local_attn"] += ev_time_ms(lambda: rb.rtp_local_attn(path.ctx, p, path.cache, q, None, None, 0, s, C, o, None, path.workspace, path.status), stream)
     g = data.heads.group
@@ -446,20 +581,26 @@ def main():
                     "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)",
                     "flops_per_launch": fl / n_launch, "launch_ms": klass[dom] / n_launch}
     else:
-        # indexer + top-p: plain ALU / MUFU work; peak = 148 SMs x 128 lanes x clock, ~12 lane-ops per score and pass
+        # indexer + top-p: one exponential per score and pass on the special-function unit, the rest plain ALU work
         scores = pairs * len(data.heads.ret_q_heads)
         achieved = scores / (klass["select"] * 1e-3) / 1e12
-        peak = 148 * 128 * 1.9e9 / 12 / 1e12
+        props = torch.cuda.get_device_properties(device)
+        n_sm = props.multi_processor_count
+        clk_mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
+        peak = 16.0 * n_sm * clk_mhz * 1e6 / 1e12
+        alu_ops = 12.0
+        peak_alu = n_sm * 128 * clk_mhz * 1e6 / alu_ops / 1e12
         roofline = {"kernel": "select_chunk_kernel", "bound": "alu", "achieved": achieved, "peak": peak,
                     "unit": "Tscore/s", "frac": achieved / peak, "traffic": None,
-                    "peak_source": "derived: 148 SMs x 128 lanes x 1.9 GHz / 12 lane-ops per score"}
-
-    # DRAM traffic of the dominant kernel per launch: a figure of the committed ncu launch list of this command (mean of
-    # dram__bytes_read.sum + dram__bytes_write.sum over the launches of the run), not measured live
-    ncu_traffic = {"select": (131072, 8192, 755511344), "sparse_attn": (131072, 8192, 161831196)}
-    if dom in ncu_traffic and ncu_traffic[dom][:2] == (L, chunk) and not c4:
-        roofline["traffic"] = ncu_traffic[dom][2]
-        roofline["traffic_source"] = "profiles/bench_c3_prefill_128k_launch_list.md"
+                    "peak_source": f"16 ex2 per clock per SM x {n_sm} SMs x {clk_mhz:.0f} MHz (median SM clock sampled in the timed region)",
+                    "alu_derived": {"peak": peak_alu, "frac": achieved / peak_alu,
+                                    "source": f"{n_sm} SMs x 128 lanes x {clk_mhz:.0f} MHz / {alu_ops:.0f} lane-ops per score and pass"},
+                    "scores_per_launch": scores / n_launch, "launch_ms": klass["select"] / n_launch}
+    useful_flops = float(n_selected.item()) * 128 * 2 * 2
+    s6 = {"useful_flops": useful_flops, "executed_flops": fl_sparse, "union_factor": fl_sparse / max(1.0, useful_flops),
+          "note": "executed = every causal 128-key tile of the retrieval heads (threshold-masked, no tile skipping); "
+                  "useful = 512 flops per selected (row, head, key)"}
+    sparsity = prefill_sparsity(path, data, chunks, L)
 
     line = {"metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -470,7 +611,7 @@ def main():
                     "last_chunk_equals_resident_run": e2e_ok},
             "gpu_launches": args.steps * len(chunks) * path.launches_per_chunk,
             "roofline": roofline, "device_status": status,
-            "selected_fraction_last_chunk": sel_frac,
+            "selected_fraction_last_chunk": sel_frac, "sparse_prefill_flops": s6, "sparsity": sparsity,
             "kernel_ms_per_step": klass,
             "kernel_tflops": {"sparse_attn": fl_sparse / klass["sparse_attn"] / 1e9,
                               "local_attn": fl_local / klass["local_attn"] / 1e9},
@@ -508,8 +649,9 @@ def main():
         if not c4:   # the 1M run stops at the comparators: no CPU sample, no decode points
             # CPU oracle on a bounded sample of the same workload
             rows = np.linspace(L // 8, L - 1, 160).astype(np.int64)
-            v, done, secs = cpu_oracle_prefill(data, L, rows, budget_s=20.0)
-            line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": n_cores, "kind": "oracle",
+            v, done, secs, used = cpu_oracle_prefill(data, L, rows, budget_s=20.0)
+            line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": used, "cores_available": n_cores,
+                                    "kind": "oracle (numpy, fp64)",
                                     "sample": f"{done} query rows x 32 heads spread over the sequence ({secs:.1f} s), "
                                               f"extrapolated per token"}
             del path, data, out, k_pre

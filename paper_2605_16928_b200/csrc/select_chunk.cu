@@ -51,7 +51,8 @@ constexpr int kListMax = 65536;               // buckets that may hold more keys
 constexpr int kSweepLoads = 16;               // list words a lane has in flight during the sweeps after a pass
 constexpr int kRowPoolEntries = 8192;         // pool words the workspace provides per (row, head)
 constexpr int kMaxPasses = 24;
-constexpr int kMaxShift = 63 * 6;             // level-1 windows below this depth hold no representable mass
+constexpr int kPoolBin = 62;                  // level-1 bin that pools everything below the window (an even shift, see aI)
+constexpr int kMaxShift = kPoolBin * 6;             // level-1 windows below this depth hold no representable mass
 constexpr float kLog2eC = kLog2eH;
 constexpr float kMagicC = 12582912.0f;        // 1.5 * 2^23: adding it leaves the nearest integer in the low mantissa bits
 constexpr uint32_t kMagicBits = 0x4B400000u;
@@ -119,7 +120,7 @@ __device__ __forceinline__ float hist_read(uint32_t col, uint32_t ccol, int bin,
 __device__ __forceinline__ uint32_t fix_q(float x) { return __float_as_uint(fast_ex2(x) + 8388608.0f) - 0x4b000000u; }
 
 // Level-1 update of a thread's private histogram for two unscaled scores r0, r1 (bit patterns):
-//   s = r * scale;  t = min(fma(s, -4, dd), magic + 63)  (bin = low mantissa bits of t);
+//   s = r * scale;  t = min(fma(s, -4, dd), magic + 62)  (bin = low mantissa bits of t);
 //   q = round(2^(fma(t - magic, log2e / 4, fma(s, log2e, cx))))  through the mantissa of (2^x + 2^23);
 //   word at hb + 512 * bits(t) += q.
 __device__ __forceinline__ void l1_pair(uint32_t r0, uint32_t r1, float scale, float dd, float cx, uint32_t hb) {
@@ -132,8 +133,8 @@ __device__ __forceinline__ void l1_pair(uint32_t r0, uint32_t r1, float scale, f
       "mul.f32 s1, %1, %2;\n"
       "fma.rn.f32 t0, s0, 0fC0800000, %3;\n"
       "fma.rn.f32 t1, s1, 0fC0800000, %3;\n"
-      "min.f32 t0, t0, 0f4B40003F;\n"
-      "min.f32 t1, t1, 0f4B40003F;\n"
+      "min.f32 t0, t0, 0f4B40003E;\n"
+      "min.f32 t1, t1, 0f4B40003E;\n"
       "fma.rn.f32 x0, s0, 0f3FB8AA3B, %4;\n"
       "fma.rn.f32 x1, s1, 0f3FB8AA3B, %4;\n"
       "sub.f32 e0, t0, 0f4B400000;\n"
@@ -465,7 +466,10 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
             count = n_keys;
             sel_m = 1.0f;
           } else {
-            aI = grid_bin(s_max);
+            // The window is anchored on an even grid bin and moves by an even number of bins: the binning of the level-1
+            // pass rounds -4 s - (aI + w0) to the nearest even on a tie, which then agrees with grid_bin's round(-4 s) for
+            // a score that lies exactly between two bins.
+            aI = grid_bin(s_max) & ~1;
             w0 = 0;
             ref0 = -0.25f * ((float)aI - 0.5f);
             mass_above = 0.f;
@@ -473,10 +477,10 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           }
         }
       } else if (kind == kPassL1) {
-        // bin = round(-4 s) - aI - w0, clamped to 63; mass relative to the bin's upper end, 2^18 fixed point
+        // bin = round(-4 s) - aI - w0, clamped to kPoolBin; mass relative to the bin's upper end, 2^18 fixed point
         const bool shifted = w0 > 0;
         const bool active = phase == kPhL1;
-        // rows that take no part land in bin 63 of their own column whatever their scores are
+        // rows that take no part land in the pooling bin of their own column whatever their scores are
         const float dd = active ? kMagicC - (float)(aI + w0) : __int_as_float(0x7f800000);
         const float cx = (float)kFixBits + (kLog2eC * 0.25f) * ((float)(aI + w0) - 0.5f);
         const uint32_t hb = hist_col - kMagicBits * (uint32_t)(kSRows * 4);
@@ -494,7 +498,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
               float t = fmaf(s, -4.0f, dd);
               // (t < magic: above the window, accounted for by an earlier level)
               if (j < valid && !(t < kMagicC)) {
-                t = fminf(t, kMagicC + 63.0f);
+                t = fminf(t, kMagicC + (float)kPoolBin);
                 const float x = fmaf(t - kMagicC, kLog2eC * 0.25f, fmaf(s, kLog2eC, cx));
                 hist_add(hist_col, (int)(__float_as_uint(t) & 63u), fix_q(x));
               }
@@ -555,10 +559,10 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
             tie_last = n_keys - 1;
             count = n_keys;
             sel_m = 1.0f;
-          } else if (found == kBins - 1) {
+          } else if (found == kPoolBin) {
             // the pooled bin: look at it with a window of its own, unless it lies so deep that it holds no mass
             mass_above = above_found;
-            w0 += kBins - 1;
+            w0 += kPoolBin;
             if (w0 > kMaxShift) {
               phase = kPhDone;
               tie_last = n_keys - 1;
@@ -935,7 +939,14 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
             each = fast_ex2((okey_to_float(sub_base) - ref0) * kLog2eC);
             if (sub_span != 1u) set_status(status, RTP_ERR_UNSUPPORTED);   // (more levels than any key has bits)
           } else {
-            if (c_in <= 0) { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 6); }   // a chosen bucket always holds a key
+            if (c_in <= 0) { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 6);
+              if (atomicCAS(pool_ctr + 32, 0u, 1u) == 0u) {   // TEMPORARY
+                pool_ctr[33] = (uint32_t)pos; pool_ctr[34] = (uint32_t)cnt; pool_ctr[35] = (uint32_t)n_words; pool_ctr[36] = base_key;
+                pool_ctr[37] = span; pool_ctr[38] = sub_base; pool_ctr[39] = sub_span; pool_ctr[40] = blk_first; pool_ctr[41] = (uint32_t)c_up;
+                pool_ctr[42] = (uint32_t)pass; pool_ctr[43] = __float_as_uint(raw_lo); pool_ctr[44] = __float_as_uint(raw_hi);
+                pool_ctr[45] = __float_as_uint(mass_above); pool_ctr[46] = __float_as_uint(target); pool_ctr[47] = (uint32_t)above;
+                pool_ctr[48] = __float_as_uint(sub_above); pool_ctr[49] = __float_as_uint(ref_s); pool_ctr[50] = __float_as_uint(scale);
+              } }
             uint32_t bound = 0u;
             bool first_step = true;
             for (int step = 0; step < kCandCapC; ++step) {

@@ -308,6 +308,32 @@ def config_3(L: int = 131072, n_q_heads: int = 32, n_kv_heads: int = 8, ret_kv_h
         row_seq=np.zeros(L, np.int32), row_pos=np.arange(L, dtype=np.int32), seed=seed)
 
 
+def config_grid_ties(L: int = 3000, n_q_heads: int = 32, n_kv_heads: int = 8, ret_kv_heads=(0, 1), window: int = 512,
+                     top_p: float = 0.9, amp: int = 3, seed: int = BASE_SEED + 33) -> Workload:
+    """A stress input for equal and grid-aligned scores (not one of the paper's workloads): the indexer's matrices pick
+    the first 16 coordinates, and those coordinates of the retrieval heads' keys and queries are small integers, so with
+    the temperature 1/8 every score is a multiple of 1/8, half of them lie exactly between two quarter-wide score bins,
+    and every value is shared by many keys.  The other coordinates, the values and the local heads are N(0,1)."""
+    rng = _rng(seed)
+    heads = HeadMap(n_q_heads, n_kv_heads, list(ret_kv_heads), n_sink=4, window=window)
+    g = heads.group
+    K = _normal(rng, (L, n_kv_heads, HEAD_DIM))
+    V = _normal(rng, (L, n_kv_heads, HEAD_DIM))
+    Q = _normal(rng, (L, n_q_heads, HEAD_DIM))
+    for kv in heads.ret_kv_heads:
+        K[:, kv, :INDEX_DIM] = rng.integers(-amp, amp + 1, size=(L, INDEX_DIM)).astype(np.float32)
+        for j in range(g):
+            Q[:, kv * g + j, :INDEX_DIM] = rng.integers(-amp, amp + 1, size=(L, INDEX_DIM)).astype(np.float32)
+    sel = np.zeros((HEAD_DIM, INDEX_DIM), np.float32)
+    sel[np.arange(INDEX_DIM), np.arange(INDEX_DIM)] = 1.0
+    w_k = to_bf16(np.stack([sel for _ in heads.ret_kv_heads]))
+    w_q = to_bf16(np.stack([sel for _ in heads.q_head_to_index_head]))
+    return Workload(
+        name="grid_ties", heads=heads, top_p=top_p, score_scale=0.125, sm_scale=1.0 / np.sqrt(HEAD_DIM),
+        seq_lens=np.array([L], np.int32), k=[to_bf16(K)], v=[to_bf16(V)], w_q=w_q, w_k=w_k, q=to_bf16(Q),
+        row_seq=np.zeros(L, np.int32), row_pos=np.arange(L, dtype=np.int32), seed=seed)
+
+
 # --------------------------------------------------------------------------
 # configuration 4: long prefill with planted needles matched to query rows
 # --------------------------------------------------------------------------

@@ -123,6 +123,75 @@ def config_3_device(L: int = 131072, device="cuda:0", seed: int = synth.BASE_SEE
                       torch.arange(L, dtype=torch.int32, device=device), seed)
 
 
+def config_4_device(L: int = 1048576, device="cuda:0", seed: int = synth.BASE_SEED + 4, top_p: float = 0.9,
+                    flat_sigma: float = 3.0, n_needles: int = 1024, window: int = 8192, n_q_heads: int = 32,
+                    n_kv_heads: int = 8, ret_kv_heads=(0,), needle_gain: float = 2.0) -> DeviceData:
+    """Long-prefill workload: N(0,1) keys, values and queries; on the retrieval KV heads every query head's rows are
+    "flat" (a direction inside the indexer's subspace scaled so that the projected scores have standard deviation
+    ``flat_sigma``), except for ``n_needles`` rows: a needle key (cosine 0.8 with a direction of the subspace) is
+    planted at a uniformly drawn position and matched to a distinct later query row, whose four query heads of the
+    group all point in the needle's direction (the same recipe as ``synth.config_4``, drawn on the device).  The matched
+    rows' queries are ``needle_gain`` times as long as in the host recipe: with a million keys behind it a needle has to
+    score about ln(1e6) higher than at a few thousand to carry most of its row's mass."""
+    g = _gen(device, seed)
+    heads = synth.HeadMap(n_q_heads, n_kv_heads, list(ret_kv_heads), 4, window)
+    grp = heads.group
+    scale = 0.125
+    W = torch.randn((len(ret_kv_heads), 128, 16), device=device, generator=g) / math.sqrt(128)
+    num_pages, bt = _paged(1, L, n_kv_heads, device, g)
+    k_pages = torch.empty((num_pages, n_kv_heads, PAGE, 128), device=device, dtype=torch.bfloat16)
+    v_pages = torch.empty_like(k_pages)
+    _fill_pages(k_pages, bt, g)
+    _fill_pages(v_pages, bt, g)
+    q = torch.empty((L, n_q_heads, 128), device=device, dtype=torch.bfloat16)
+    ret_q = set(heads.ret_q_heads)
+    for lo in range(0, L, 16384):
+        hi = min(L, lo + 16384)
+        x = torch.randn((hi - lo, n_q_heads, 128), device=device, generator=g)
+        for ih, kv in enumerate(heads.ret_kv_heads):
+            for j in range(grp):
+                a = torch.randn((hi - lo, 16), device=device, generator=g)
+                dvec = a @ W[ih].T
+                dvec = dvec / dvec.norm(dim=-1, keepdim=True)
+                qt = (dvec @ W[ih]).norm(dim=-1, keepdim=True)
+                x[:, kv * grp + j] = flat_sigma / (scale * qt) * dvec
+        q[lo:hi] = x.to(torch.bfloat16)
+    # needles: key positions uniform without replacement, each matched to a distinct later query row
+    cpu = np.random.Generator(np.random.PCG64(seed))
+    n_needles = min(n_needles, max(1, L // 8))
+    kpos = np.sort(cpu.choice(L - 1, size=n_needles, replace=False))
+    qrow = np.empty(n_needles, dtype=np.int64)
+    taken = set()
+    for i, n in enumerate(kpos):
+        while True:
+            r = int(cpu.integers(n + 1, L))
+            if r not in taken:
+                taken.add(r)
+                break
+        qrow[i] = r
+    kpos_t = torch.from_numpy(kpos).to(device)
+    qrow_t = torch.from_numpy(qrow).to(device)
+    for ih, kv in enumerate(heads.ret_kv_heads):
+        a = torch.randn((n_needles, 16), device=device, generator=g)
+        q_dir = a @ W[ih].T
+        q_dir = q_dir / q_dir.norm(dim=-1, keepdim=True)
+        gg = torch.randn((n_needles, 128), device=device, generator=g)
+        gg = gg - (gg * q_dir).sum(-1, keepdim=True) * q_dir
+        gg = gg / gg.norm(dim=-1, keepdim=True)
+        needle = math.sqrt(128.0) * (0.8 * q_dir + 0.6 * gg)
+        phys = bt[0, (kpos_t // PAGE)].long()
+        k_pages[phys, kv, (kpos_t % PAGE)] = needle.to(torch.bfloat16)
+        for j in range(grp):
+            q[qrow_t, kv * grp + j] = (needle_gain * math.sqrt(128.0) * q_dir).to(torch.bfloat16)
+    w_k = W.to(torch.bfloat16).contiguous()
+    w_q = W[[heads.q_head_to_index_head[i] for i in range(len(heads.ret_q_heads))]].to(torch.bfloat16).contiguous()
+    return DeviceData("c4_prefill_long", heads, top_p, scale, 1.0 / math.sqrt(128),
+                      torch.tensor([L], dtype=torch.int32, device=device), bt, k_pages, v_pages, w_q, w_k, q,
+                      torch.zeros(L, dtype=torch.int32, device=device),
+                      torch.arange(L, dtype=torch.int32, device=device), seed,
+                      {"needle_key_pos": kpos, "needle_query_row": qrow, "flat_sigma": flat_sigma, "needle_gain": needle_gain})
+
+
 def decode_device(L: int, batch: int, top_p: float, frac: float, window: int, device="cuda:0",
                   seed: int = synth.BASE_SEED + 5, n_q_heads: int = 32, n_kv_heads: int = 8,
                   ret_kv_heads=(0, 1), peaked_half: bool = False, name: str = "c5_decode_sweep") -> DeviceData:
@@ -142,6 +211,7 @@ def decode_device(L: int, batch: int, top_p: float, frac: float, window: int, de
     _fill_pages(v_pages, bt, g)
     q = torch.randn((batch, n_q_heads, 128), device=device, generator=g)
     cpu = np.random.Generator(np.random.PCG64(seed))
+    dirs, qt_norms = [], []
     for i, h in enumerate(heads.ret_q_heads):
         ih = i // grp
         a = torch.randn((batch, 16), device=device, generator=g)
@@ -149,6 +219,8 @@ def decode_device(L: int, batch: int, top_p: float, frac: float, window: int, de
         dvec = dvec / dvec.norm(dim=-1, keepdim=True)
         qt = (dvec @ W[ih]).norm(dim=-1, keepdim=True)
         q[:, h] = sigma / (scale * qt) * dvec
+        dirs.append(dvec)
+        qt_norms.append(qt)
         if peaked_half:
             for b in range(batch // 2):
                 q[b, h] = math.sqrt(128.0) * dvec[b]
@@ -166,4 +238,16 @@ def decode_device(L: int, batch: int, top_p: float, frac: float, window: int, de
                       torch.full((batch,), L, dtype=torch.int32, device=device), bt, k_pages, v_pages, w_q, w_k,
                       q.to(torch.bfloat16), torch.arange(batch, dtype=torch.int32, device=device),
                       torch.full((batch,), L - 1, dtype=torch.int32, device=device), seed,
-                      {"sigma": sigma, "target_fraction": frac})
+                      {"sigma": sigma, "target_fraction": frac, "ret_dirs": dirs, "ret_qt_norms": qt_norms})
+
+
+def decode_retarget(data: DeviceData, top_p: float, frac: float) -> DeviceData:
+    """The same cache and query directions as ``data`` (a ``decode_device`` workload without planted keys) at another
+    top-p and another score temperature: only the lengths of the retrieval heads' queries change."""
+    import dataclasses
+    sigma = synth.sigma_for_fraction(top_p, frac)
+    q = data.q.clone()
+    for i, h in enumerate(data.heads.ret_q_heads):
+        q[:, h] = (sigma / (data.score_scale * data.notes["ret_qt_norms"][i]) * data.notes["ret_dirs"][i]).to(q.dtype)
+    notes = dict(data.notes, sigma=sigma, target_fraction=frac)
+    return dataclasses.replace(data, top_p=top_p, q=q, notes=notes)

@@ -71,6 +71,28 @@ def test_config3_reduced_select_and_sparse_prefill():
     assert 0.005 <= np.mean(all_fracs) <= 0.6
 
 
+@pytest.mark.parametrize("amp,top_p", [(3, 0.9), (1, 0.5), (6, 0.99)])
+def test_select_scores_on_bin_boundaries_and_heavy_ties(amp, top_p):
+    """Integer-valued index features with temperature 1/8: scores are multiples of 1/8, so half of them sit exactly between
+    two of the selection kernel's quarter-wide bins, and every score value is shared by many keys."""
+    wl = synth.config_grid_ties(L=3000, amp=amp, top_p=top_p)
+    gh, dw, pr = _prep(wl)
+    rng = np.random.default_rng(amp)
+    for q_start, C in [(0, 1024), (1024, 1024), (2048, 952)]:
+        rows = _sample_rows(q_start, C, rng, extra=(1, 2, 5, 63, 64, 65))
+        sel = pr.select_chunk(q_start, C, with_lists=True)
+        sc, _ = gh.check_chunk_selection(pr, q_start, sel, rows)
+        assert np.all(sc[np.isfinite(sc)] * 8 == np.round(sc[np.isfinite(sc)] * 8))      # the input does what it says
+        sel2 = pr.select_chunk(q_start, C, with_lists=False)
+        assert torch.equal(sel2["cnt"], sel["cnt"]) and torch.equal(sel2["tie"], sel["tie"])
+        assert torch.equal(sel2["thr"], sel["thr"])
+        idx, cnt = sel["idx"].cpu().numpy(), sel["cnt"].cpu().numpy()
+        sets = {(m, i): idx[m - q_start, i, : cnt[m - q_start, i]] for m in rows for i in range(dw.n_ret)}
+        out_t, lse_t = pr.sparse_prefill(q_start, C, sel, use_lists=False)
+        gh.check_prefill_rows(pr, q_start, out_t, lse_t, rows, "sparse", None, sets)
+    assert dw.status_code() == rb.RTP_OK
+
+
 @pytest.mark.parametrize("n_q,n_kv", [(16, 2), (4, 2), (2, 2)])
 def test_other_group_sizes(n_q, n_kv):
     """G = 8, 2 and 1 query heads per KV head: 16, 64 and 128 positions per CTA tile in the chunk kernels."""
