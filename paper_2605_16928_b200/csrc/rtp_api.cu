@@ -181,9 +181,10 @@ size_t rtp_workspace_bytes(const rtp_params* params, int64_t rows, int64_t max_s
   if (check_params(params, &d, &hm) || rows <= 0 || max_seq_len <= 0) return 0;
   WsCarver w(nullptr);
   w.take(qt_bytes(d, rows));
-  size_t a = select_rows_workspace_bytes(d, rows);
+  size_t a = select_rows_workspace_bytes(d, rows, max_seq_len);
   const size_t b = select_chunk_workspace_bytes(d, hm, rows);
-  // explicit-row selection keeps 48 KB per (row, head); beyond 4096 rows only the chunk path is sized
+  // explicit-row selection keeps 48 KB and one fp32 score per key for every (row, head); beyond 4096 rows only the
+  // chunk path is sized
   if (rows > 4096) a = 0;
   size_t m = a > b ? a : b;
   const size_t s = score_workspace_bytes(d, rows, max_seq_len, current_sm_count(kFallbackSm) * 2);
@@ -308,7 +309,7 @@ rtp_status rtp_topp_select(rtp_ctx* ctx, const rtp_params* params, const rtp_cac
   __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(w.take(qt_bytes(d, R)));
   const bool chunk = row_seq == nullptr;
   const size_t sel_off = w.off;
-  void* sel_ws = w.take(chunk ? select_chunk_workspace_bytes(d, hm, R) : select_rows_workspace_bytes(d, R));
+  void* sel_ws = w.take(chunk ? select_chunk_workspace_bytes(d, hm, R) : select_rows_workspace_bytes(d, R, max_len));
   if (w.off > workspace_bytes) return fail(ctx, RTP_ERR_CAPACITY, "workspace too small");
   cudaError_t e = launch_index_queries(d, hm, reinterpret_cast<const __nv_bfloat16*>(q_pre),
                                        reinterpret_cast<const __nv_bfloat16*>(w_q), R, qt, st);

@@ -145,7 +145,7 @@ cudaError_t launch_index_score(const CacheView& cv, const Dims& d, const HeadMap
                                float* row_max, float* row_sum, void* ws, int32_t* status, int sm_count,
                                cudaStream_t st);
 
-size_t select_rows_workspace_bytes(const Dims& d, int64_t R);
+size_t select_rows_workspace_bytes(const Dims& d, int64_t R, int64_t max_len);
 cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                                const __nv_bfloat16* qt, int64_t max_len, int32_t* sel_idx, int64_t sel_stride,
                                int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,

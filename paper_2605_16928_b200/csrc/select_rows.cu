@@ -1,15 +1,16 @@
 // S2-S4 for explicit rows (the decode path): fused indexer scan + top-p selection (Eq. 5).
 //
-// The context of one (row, index head) unit is split over many CTAs; every pass scores its keys again (MMA, see
-// score16) from the index-key cache:
-//   max          row maximum M of every head (atomicMax on the ordered key);
+// The context of one (row, index head) unit is split over many CTAs.  The index keys are read once:
+//   scores       every key is scored (MMA, see score16) for the unit's heads; the fp32 scores are stored, 4 bytes per
+//                (head, key), and the row maxima M are taken (atomicMax on the ordered key).
+// The other passes read the stored scores (half the bytes of the keys for four heads, no MMA, and at the usual sizes
+// still in the L2 cache):
 //   level 1      64-bin histogram of softmax mass over d = M - s in steps of 1/2, fixed point, one native
 //                shared-memory add per score, merged into global memory; the unit's last CTA to finish (ticket
 //                counter, nobody waits) finds Z and the bin in which the cumulative mass reaches p * Z and turns
-//                it into an exact interval of ordered keys and of unscaled MMA outputs;
+//                it into an exact interval of ordered keys;
 //   key levels   six more key bits per pass inside that interval, with exact counts, until the bucket holds at most
-//                kCandCap keys (or a single key value); hits are rare, so a warp queues them and works them off 32
-//                at a time;
+//                kCandCap keys (or a single key value);
 //   compaction   every key above the bucket is counted and emitted, keys inside it become candidates;
 //   finalize     one CTA per (row, head) sorts the candidates by (score desc, position asc) and takes the shortest
 //                prefix that reaches the target mass.
@@ -22,8 +23,6 @@ namespace {
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kHeadsPerCta = 4;
-constexpr int kStage = 128;      // staged ids per (warp, head) before a flush
-constexpr int kCandStage = 48;   // staged boundary candidates per (warp, head)
 
 struct RowCtx {
   int64_t r;
@@ -58,14 +57,6 @@ __device__ __forceinline__ void load_page(const CacheView& cv, const RowCtx& x, 
   const __nv_bfloat16* base = ikey_page_ptr(cv, x.seq, p, x.ih);
 #pragma unroll
   for (int i = 0; i < 4; ++i) v[i] = ld_stream_v4(base + (i * 32 + lane) * 8);
-}
-
-// Which retrieval head (index into ret_q_heads) this lane post-processes in head group z, or -1.
-// MMA row g holds head slot g, row g + 8 holds slot g + 8; group z covers slots 4z .. 4z+3.
-__device__ __forceinline__ int lane_head_slot(int lane, int z) {
-  const int g = lane >> 2;
-  if ((g >> 2) != (z & 1)) return -1;
-  return (z >> 1) * 8 + g;
 }
 
 __global__ void sel_init_kernel(const CacheView cv, const Dims d, const Rows rows, SelState* state,
@@ -143,16 +134,21 @@ __device__ __forceinline__ bool take_last_ticket(uint32_t* ticket, uint32_t n_ct
   return s_is_last != 0;
 }
 
-// ---- pass 1: row maximum ----------------------------------------------------------------------------
+// ---- pass 1: scores of the unit's keys, written once for the later passes, and the row maximum -----------------------
+// scores: float [rows * retrieval heads][l_pad]; entry n of a row holds finish_score(q~ . k~_n) for n < n_keys.
 template <bool NH4>
-__global__ void __launch_bounds__(kThreads) sel_max_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
-                                                           const Rows rows, const __nv_bfloat16* __restrict__ qt,
-                                                           SelState* __restrict__ state, int n_splits, int32_t* status) {
+__global__ void __launch_bounds__(kThreads) sel_score_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
+                                                             const Rows rows, const __nv_bfloat16* __restrict__ qt,
+                                                             SelState* __restrict__ state, float* __restrict__ scores,
+                                                             const int64_t l_pad, int n_splits, int32_t* status) {
   __shared__ float s_max[kWarps][16];
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, status);
   if (x.p_lo >= x.p_hi) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
+  const int slot_a = elem_slot<NH4>(lane, 0), slot_b = NH4 ? slot_a : elem_slot<NH4>(lane, 4);
+  float* row_a = slot_a < x.nh ? scores + (x.r * d.n_ret + hm.ih_heads[x.ih][slot_a]) * l_pad : nullptr;
+  float* row_b = (!NH4 && slot_b < x.nh) ? scores + (x.r * d.n_ret + hm.ih_heads[x.ih][slot_b]) * l_pad : nullptr;
   float mx_a = -INFINITY, mx_b = -INFINITY;
   uint4 v[4], vn[4];
   if (x.p_lo + warp < x.p_hi) load_page(cv, x, x.p_lo + warp, lane, vn);
@@ -166,6 +162,22 @@ __global__ void __launch_bounds__(kThreads) sel_max_kernel(const CacheView cv, c
       float s_lo[4], s_hi[4];
       score16(qf, v[i], lane, s_lo, s_hi);
       const LaneElems<NH4> el = lane_elems<NH4>(s_lo, s_hi, lane);
+      const int n0 = p * kPage + i * 16 + el.koff[0];
+      // (a page lies inside l_pad whatever n_keys is: entries beyond the row's keys are written and never read)
+      if (NH4) {
+        if (row_a)
+          *reinterpret_cast<float2*>(row_a + n0) =
+              make_float2(finish_score(el.raw[0], d.score_scale), finish_score(el.raw[1], d.score_scale));
+      } else {
+        if (row_a)
+          *reinterpret_cast<float4*>(row_a + n0) =
+              make_float4(finish_score(el.raw[0], d.score_scale), finish_score(el.raw[1], d.score_scale),
+                          finish_score(el.raw[2], d.score_scale), finish_score(el.raw[3], d.score_scale));
+        if (row_b)
+          *reinterpret_cast<float4*>(row_b + n0) =
+              make_float4(finish_score(el.raw[4], d.score_scale), finish_score(el.raw[5], d.score_scale),
+                          finish_score(el.raw[6], d.score_scale), finish_score(el.raw[7], d.score_scale));
+      }
 #pragma unroll
       for (int e = 0; e < LaneElems<NH4>::kN; ++e) {
         if (tail && p * kPage + i * 16 + el.koff[e] >= x.n_keys) continue;
@@ -196,13 +208,30 @@ __global__ void __launch_bounds__(kThreads) sel_max_kernel(const CacheView cv, c
   }
 }
 
+// The later passes read the stored scores: the CTA's share of a row is keys [k_lo, k_hi), four consecutive keys per
+// thread and step (one 16-byte load).
+struct KeySpan {
+  int k_lo, k_hi;
+};
+__device__ __forceinline__ KeySpan key_span(const RowCtx& x) {
+  KeySpan s;
+  s.k_lo = x.p_lo * kPage;
+  s.k_hi = min(x.p_hi * kPage, x.n_keys);
+  return s;
+}
+__device__ __forceinline__ float4 ld_scores4(const float* p) {
+  float4 v;
+  asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+
 // ---- pass 2: level-1 mass histogram over M - s, resolved by the unit's last CTA ----------------------------------
-template <bool NH4>
 __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
-                                                          const Rows rows, const __nv_bfloat16* __restrict__ qt,
-                                                          SelState* __restrict__ state, unsigned long long* __restrict__ g_mass,
+                                                          const Rows rows, const float* __restrict__ scores,
+                                                          const int64_t l_pad, SelState* __restrict__ state,
+                                                          unsigned long long* __restrict__ g_mass,
                                                           uint32_t* __restrict__ tickets, int n_splits, int32_t* status) {
-  __shared__ uint32_t hist[16][kBins][2];
+  __shared__ uint32_t hist[kWarps][kBins][2];   // one private histogram per warp, for the head being scanned
   __shared__ float s_M[16];
   __shared__ int s_on[16];
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
@@ -218,47 +247,40 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
     s_on[threadIdx.x] = on;
     s_M[threadIdx.x] = M;
   }
-  for (int i = threadIdx.x; i < 16 * kBins * 2; i += kThreads) (&hist[0][0][0])[i] = 0u;
+  for (int i = threadIdx.x; i < kWarps * kBins * 2; i += kThreads) (&hist[0][0][0])[i] = 0u;
   __syncthreads();
   int any = 0;
   for (int j = 0; j < x.nh; ++j) any |= s_on[j];
   if (!any) return;   // the same decision in every CTA of the unit
 
-  const int slot_a = elem_slot<NH4>(lane, 0), slot_b = NH4 ? slot_a : elem_slot<NH4>(lane, 4);
-  const bool on_a = slot_a < x.nh && s_on[slot_a], on_b = !NH4 && slot_b < x.nh && s_on[slot_b];
-  const float M_a = s_M[slot_a], M_b = s_M[slot_b];
-  const QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
-  uint4 v[4], vn[4];
-  if (x.p_lo + warp < x.p_hi) load_page(cv, x, x.p_lo + warp, lane, vn);
-  for (int p = x.p_lo + warp; p < x.p_hi; p += kWarps) {
+  const KeySpan ks = key_span(x);
+  for (int j = 0; j < x.nh; ++j) {
+    if (!s_on[j]) continue;   // uniform
+    const int64_t rh = x.r * d.n_ret + hm.ih_heads[x.ih][j];
+    const float* row = scores + rh * l_pad;
+    const float M = s_M[j];
+    for (int n0 = ks.k_lo + 4 * (int)threadIdx.x; n0 < ks.k_hi; n0 += 4 * kThreads) {
+      const float4 v = ld_scores4(row + n0);
+      const float s4[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-    for (int i = 0; i < 4; ++i) v[i] = vn[i];
-    if (p + kWarps < x.p_hi) load_page(cv, x, p + kWarps, lane, vn);   // in flight while this page is worked on
-    const bool tail = (p + 1) * kPage > x.n_keys;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float s_lo[4], s_hi[4];
-      score16(qf, v[i], lane, s_lo, s_hi);
-      const LaneElems<NH4> el = lane_elems<NH4>(s_lo, s_hi, lane);
-#pragma unroll
-      for (int e = 0; e < LaneElems<NH4>::kN; ++e) {
-        const bool set_a = NH4 || e < 4;
-        if (!(set_a ? on_a : on_b)) continue;
-        if (tail && p * kPage + i * 16 + el.koff[e] >= x.n_keys) continue;
-        const float s = finish_score(el.raw[e], d.score_scale);
-        const float M = set_a ? M_a : M_b;
+      for (int e = 0; e < 4; ++e) {
+        if (n0 + e >= ks.k_hi) continue;
         float bin_f;
-        const int bin = l1_bin_f(M, s, bin_f);
-        add_mass(&hist[set_a ? slot_a : slot_b][bin][0], l1_mass_arg(M, s, bin_f));
+        const int bin = l1_bin_f(M, s4[e], bin_f);
+        add_mass(&hist[warp][bin][0], l1_mass_arg(M, s4[e], bin_f));
       }
     }
-  }
-  __syncthreads();
-  for (int i = threadIdx.x; i < x.nh * kBins; i += kThreads) {
-    const int j = i / kBins, bin = i % kBins;
-    const uint32_t sum = hist[j][bin][0], car = hist[j][bin][1];
-    if (sum | car)
-      atomicAdd(g_mass + (x.r * d.n_ret + hm.ih_heads[x.ih][j]) * kBins + bin, ((unsigned long long)car << 32) | sum);
+    __syncthreads();
+    if (threadIdx.x < kBins) {
+      unsigned long long tot = 0ull;
+      for (int w = 0; w < kWarps; ++w) {
+        tot += ((unsigned long long)hist[w][threadIdx.x][1] << 32) | hist[w][threadIdx.x][0];
+        hist[w][threadIdx.x][0] = 0u;
+        hist[w][threadIdx.x][1] = 0u;
+      }
+      if (tot) atomicAdd(g_mass + rh * kBins + threadIdx.x, tot);
+    }
+    __syncthreads();
   }
   if (!take_last_ticket(tickets + blockIdx.x, gridDim.y)) return;
 
@@ -346,46 +368,24 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
 // ---- pass 3 (repeated): 64-bin mass histogram of the next six key bits inside the bucket --------------------------
 // Only a small share of the scores falls into a head's bucket: a warp appends those hits to a queue in shared
 // memory and works them off 32 at a time, one hit per lane.
-constexpr int kQueueCapR = 160;   // >= 31 + 4 x 32 entries
-
 struct KeyParams {   // per head slot, shared memory
   uint32_t base_key;
   int32_t shift;
   float ref_s;
 };
 
-// (the count is passed by value: a reference would pin the caller's counter to local memory)
-__device__ __noinline__ void drain_row_hits(uint32_t* wq, int qcnt, int lane, const KeyParams* kp,
-                                            uint32_t (*hist)[kBins][3], float scale) {
-  __syncwarp();
-  for (int base = 0; base < qcnt; base += 32) {
-    const int i = base + lane;
-    if (i < qcnt) {
-      const int slot = (int)wq[2 * i];
-      const float s = finish_score(__uint_as_float(wq[2 * i + 1]), scale);
-      const uint32_t t = okey(s) - kp[slot].base_key;
-      uint32_t* acc = &hist[slot][t >> kp[slot].shift][0];
-      add_mass(acc, fmaf(s - kp[slot].ref_s, kLog2eH, 20.0f));
-      atomicAdd(acc + 2, 1u);
-    }
-  }
-  __syncwarp();
-}
-
-template <bool NH4>
 __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
-                                                           const Rows rows, const __nv_bfloat16* __restrict__ qt,
+                                                           const Rows rows, const float* __restrict__ scores,
+                                                           const int64_t l_pad,
                                                            SelState* __restrict__ state, unsigned long long* __restrict__ g_mass,
                                                            uint32_t* __restrict__ g_cnt, uint32_t* __restrict__ tickets,
                                                            int n_splits, int max_levels, int32_t* status) {
   __shared__ uint32_t hist[16][kBins][3];   // {sum, carries, count}
-  __shared__ uint32_t queue[kWarps][kQueueCapR * 2];
   __shared__ KeyParams kp[16];
-  __shared__ float s_lo_raw[16], s_hi_raw[16];
+  __shared__ uint32_t s_span[16];
   __shared__ int s_on[16];
   RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const float kInf = __int_as_float(0x7f800000);
   uint32_t n_ctas = gridDim.y;
   // The first level is split over the unit's CTAs.  The CTA that resolves it goes on alone with whatever is still
   // unresolved (rare: dense clusters of nearly equal scores), scanning the whole unit, up to max_levels in all.
@@ -393,22 +393,20 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
   for (int level = 0; level < max_levels; ++level) {
   if (threadIdx.x < 16) {
     int on = 0;
-    float lo = kInf, hi = -kInf;
+    uint32_t span = 0u;
     KeyParams k = {0u, 0, 0.f};
     if (threadIdx.x < x.nh) {
       const volatile SelState* st = state + (x.r * d.n_ret + hm.ih_heads[x.ih][threadIdx.x]);
       on = st->mode == kRefine && st->n_keys > 0;
       if (on) {
-        lo = st->raw_lo;
-        hi = st->raw_hi;
+        span = st->span;
         k.base_key = st->lo_key;
         k.shift = st->shift;
         k.ref_s = st->ref_s;
       }
     }
     s_on[threadIdx.x] = on;
-    s_lo_raw[threadIdx.x] = lo;
-    s_hi_raw[threadIdx.x] = hi;
+    s_span[threadIdx.x] = span;
     kp[threadIdx.x] = k;
   }
   for (int i = threadIdx.x; i < 16 * kBins * 3; i += kThreads) (&hist[0][0][0])[i] = 0u;
@@ -417,56 +415,28 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
   for (int j = 0; j < x.nh; ++j) any |= s_on[j];
   if (!any) return;   // the same decision in every CTA of the unit
 
-  const int slot_a = elem_slot<NH4>(lane, 0), slot_b = NH4 ? slot_a : elem_slot<NH4>(lane, 4);
-  const float lo_a = s_lo_raw[slot_a], hi_a = s_hi_raw[slot_a];
-  const float lo_b = NH4 ? kInf : s_lo_raw[slot_b], hi_b = NH4 ? -kInf : s_hi_raw[slot_b];
-  const QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
-  uint32_t* wq = queue[warp];
-  int qcnt = 0;
-  const uint32_t lt = (1u << lane) - 1u;
-  uint4 v[4], vn[4];
-  if (x.p_lo + warp < x.p_hi) load_page(cv, x, x.p_lo + warp, lane, vn);
-  for (int p = x.p_lo + warp; p < x.p_hi; p += kWarps) {
+  // hits are rare (the bucket holds a few per cent of the keys at most): each is added where it is found
+  const KeySpan ks = key_span(x);
+  for (int j = 0; j < x.nh; ++j) {
+    if (!s_on[j]) continue;   // uniform
+    const float* row = scores + (x.r * d.n_ret + hm.ih_heads[x.ih][j]) * l_pad;
+    const uint32_t base_key = kp[j].base_key, span = s_span[j];
+    const int shift = kp[j].shift;
+    const float ref_s = kp[j].ref_s;
+    for (int n0 = ks.k_lo + 4 * (int)threadIdx.x; n0 < ks.k_hi; n0 += 4 * kThreads) {
+      const float4 v = ld_scores4(row + n0);
+      const float s4[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-    for (int i = 0; i < 4; ++i) v[i] = vn[i];
-    if (p + kWarps < x.p_hi) load_page(cv, x, p + kWarps, lane, vn);   // in flight while this page is worked on
-    const bool tail = (p + 1) * kPage > x.n_keys;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float s_lo[4], s_hi[4];
-      score16(qf, v[i], lane, s_lo, s_hi);
-      const LaneElems<NH4> el = lane_elems<NH4>(s_lo, s_hi, lane);
-      bool hit[LaneElems<NH4>::kN];
-      bool any_hit = false;
-#pragma unroll
-      for (int e = 0; e < LaneElems<NH4>::kN; ++e) {
-        const bool set_a = NH4 || e < 4;
-        hit[e] = el.raw[e] >= (set_a ? lo_a : lo_b) && el.raw[e] <= (set_a ? hi_a : hi_b);
-        if (tail && p * kPage + i * 16 + el.koff[e] >= x.n_keys) hit[e] = false;
-        any_hit = any_hit || hit[e];
-      }
-      if (!__any_sync(0xffffffffu, any_hit)) continue;
-#pragma unroll
-      for (int e = 0; e < LaneElems<NH4>::kN; ++e) {
-        const uint32_t m = __ballot_sync(0xffffffffu, hit[e]);
-        if (m) {
-          if (hit[e]) {
-            const int pos = qcnt + __popc(m & lt);
-            wq[2 * pos] = (uint32_t)((NH4 || e < 4) ? slot_a : slot_b);
-            wq[2 * pos + 1] = __float_as_uint(el.raw[e]);
-          }
-          qcnt += __popc(m);
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t t = okey(s4[e]) - base_key;
+        if (n0 + e < ks.k_hi && t < span) {
+          uint32_t* acc = &hist[j][t >> shift][0];
+          add_mass(acc, fmaf(s4[e] - ref_s, kLog2eH, 20.0f));
+          atomicAdd(acc + 2, 1u);
         }
-        if ((e & 3) == 3 || e == LaneElems<NH4>::kN - 1)
-          if (qcnt >= 32) {
-            drain_row_hits(wq, qcnt, lane, kp, hist, d.score_scale);
-            qcnt = 0;
-          }
       }
     }
   }
-  if (qcnt > 0) drain_row_hits(wq, qcnt, lane, kp, hist, d.score_scale);
-  qcnt = 0;
   __syncthreads();
   for (int i = threadIdx.x; i < x.nh * kBins; i += kThreads) {
     const int j = i / kBins, bin = i % kBins;
@@ -565,315 +535,86 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
 }
 
 // ---- compaction -------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) sel_compact_kernel(
-    const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows,
-    const __nv_bfloat16* __restrict__ qt, SelState* __restrict__ state, uint2* __restrict__ cand,
-    int32_t* __restrict__ sel_idx, int64_t sel_stride, int n_splits, int32_t* status) {
-  __shared__ int stage[kWarps][kHeadsPerCta][kStage];
-  __shared__ uint2 cstage[kWarps][kHeadsPerCta][kCandStage];
-  __shared__ int stage_cnt[kWarps][kHeadsPerCta];
-  __shared__ int cstage_cnt[kWarps][kHeadsPerCta];
+// Keys above a head's bucket are counted and, when id lists are requested, emitted; keys inside it become candidates
+// for the exact finish.  A CTA takes up to four heads of the unit (blockIdx.z), one after the other; a warp reads 128
+// consecutive stored scores per step and ballots the hits into its two stages in shared memory, which are appended
+// to the row's list / candidate array with one counter update per flush.
+constexpr int kIdStage = 384;     // a step adds at most 128 entries: flushed when more than 256 are staged
+constexpr int kCandStageW = 256;  // flushed when more than 128 are staged
 
+__global__ void __launch_bounds__(kThreads) sel_compact_kernel(
+    const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows, const float* __restrict__ scores,
+    const int64_t l_pad, SelState* __restrict__ state, uint2* __restrict__ cand, int32_t* __restrict__ sel_idx,
+    int64_t sel_stride, int n_splits, int32_t* status) {
+  __shared__ int id_stage[kWarps][kIdStage];
+  __shared__ uint2 cand_stage[kWarps][kCandStageW];
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
   const int z = blockIdx.z;
   if (z * kHeadsPerCta >= x.nh || x.p_lo >= x.p_hi) return;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, c = lane & 3;
-  const int slot = lane_head_slot(lane, z);
-  const bool use_hi = (z >> 1) != 0;
-  const int j = (lane >> 2) & 3;
-  const int head = (slot >= 0 && slot < x.nh) ? hm.ih_heads[x.ih][slot] : -1;
-  SelState* st = head >= 0 ? state + (x.r * d.n_ret + head) : nullptr;
-  int mode = -1;
-  uint32_t lo_key = 0, hi_key = 0;
-  if (st) {
-    mode = st->mode;
-    lo_key = st->lo_key;
-    hi_key = st->hi_key;
-  }
-  if (lane < kHeadsPerCta) {
-    stage_cnt[warp][lane] = 0;
-    cstage_cnt[warp][lane] = 0;
-  }
-  __syncwarp();
-  const bool emit_ids = sel_idx != nullptr;
-  const QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
-  int n_above = 0;   // keys above the bucket seen by this lane
-
-  auto row_head = [&](int jj) -> int64_t {
-    const int slot2 = (z >> 1) * 8 + (z & 1) * 4 + jj;
-    return x.r * d.n_ret + hm.ih_heads[x.ih][slot2];
-  };
-  auto flush_ids = [&](int jj) {  // warp-uniform
-    const int n = stage_cnt[warp][jj];
-    if (n == 0) return;
-    const int64_t rh = row_head(jj);
-    int gbase = 0;
-    if (lane == 0) gbase = atomicAdd(&state[rh].emit_cnt, n);
-    gbase = __shfl_sync(0xffffffffu, gbase, 0);
-    for (int i = lane; i < n; i += 32)
-      if (gbase + i < sel_stride) sel_idx[rh * sel_stride + gbase + i] = stage[warp][jj][i];
-    if (gbase + n > sel_stride && lane == 0) set_status(status, RTP_ERR_CAPACITY);
-    __syncwarp();
-    if (lane == 0) stage_cnt[warp][jj] = 0;
-    __syncwarp();
-  };
-  auto flush_cands = [&](int jj) {  // warp-uniform
-    const int n = cstage_cnt[warp][jj];
-    if (n == 0) return;
-    const int64_t rh = row_head(jj);
-    int gbase = 0;
-    if (lane == 0) gbase = atomicAdd(&state[rh].cand_cnt, n);
-    gbase = __shfl_sync(0xffffffffu, gbase, 0);
-    for (int i = lane; i < n; i += 32)
-      if (gbase + i < kCandCap) cand[rh * kCandCap + gbase + i] = cstage[warp][jj][i];
-    __syncwarp();
-    if (lane == 0) cstage_cnt[warp][jj] = 0;
-    __syncwarp();
-  };
-  // Appends the entries flagged in `flags` (bit e = key n0 + e) of every head to a per-warp stage.
-  auto group_offsets = [&](int k, int& incl) {
-    incl = k;
-    int t = __shfl_up_sync(0xffffffffu, incl, 1, 4);
-    if (c >= 1) incl += t;
-    t = __shfl_up_sync(0xffffffffu, incl, 2, 4);
-    if (c >= 2) incl += t;
-  };
-
-  for (int p = x.p_lo + warp; p < x.p_hi; p += kWarps) {
-    const __nv_bfloat16* base = ikey_page_ptr(cv, x.seq, p, x.ih);
-    uint4 v[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) v[i] = ld_stream_v4(base + (i * 32 + lane) * 8);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float s_lo[4], s_hi[4];
-      score16(qf, v[i], lane, s_lo, s_hi);
-      const int n0 = p * kPage + i * 16 + 4 * c;
-      int flags = 0, cflags = 0;
-      uint32_t keys4[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) keys4[e] = okey(finish_score(use_hi ? s_hi[e] : s_lo[e], d.score_scale));
-      if (mode == kSelectAll) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if (n0 + e < x.n_keys) flags |= 1 << e;
-      } else if (mode == kCollect || mode == kTieScan) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (n0 + e >= x.n_keys) continue;
-          if (keys4[e] > hi_key)
-            flags |= 1 << e;
-          else if (keys4[e] >= lo_key && mode == kCollect)
-            cflags |= 1 << e;
-        }
-      }
-      // boundary candidates
-      {
-        const int k = __popc(cflags);
-        int incl;
-        group_offsets(k, incl);
-        if (head >= 0 && k) {
-          int w = cstage_cnt[warp][j] + incl - k;
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            if (cflags & (1 << e)) cstage[warp][j][w++] = make_uint2(keys4[e], (uint32_t)(n0 + e));
-        }
-        __syncwarp();
-        if (head >= 0 && c == 3 && incl) cstage_cnt[warp][j] += incl;
-        __syncwarp();
-#pragma unroll
-        for (int jj = 0; jj < kHeadsPerCta; ++jj)
-          if (cstage_cnt[warp][jj] > kCandStage - 16) flush_cands(jj);
-      }
-      n_above += __popc(flags);
-      if (!emit_ids) continue;
-      {
-        const int k = __popc(flags);
-        int incl;
-        group_offsets(k, incl);
-        if (head >= 0 && k) {
-          int w = stage_cnt[warp][j] + incl - k;
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            if (flags & (1 << e)) stage[warp][j][w++] = n0 + e;
-        }
-        __syncwarp();
-        if (head >= 0 && c == 3 && incl) stage_cnt[warp][j] += incl;
-        __syncwarp();
-#pragma unroll
-        for (int jj = 0; jj < kHeadsPerCta; ++jj)
-          if (stage_cnt[warp][jj] > kStage - 16) flush_ids(jj);
-      }
-    }
-  }
-#pragma unroll
-  for (int jj = 0; jj < kHeadsPerCta; ++jj) {
-    flush_cands(jj);
-    if (emit_ids) flush_ids(jj);
-  }
-  n_above += __shfl_xor_sync(0xffffffffu, n_above, 1);
-  n_above += __shfl_xor_sync(0xffffffffu, n_above, 2);
-  if (st && c == 0 && n_above && mode != kSelectAll) atomicAdd(&st->cnt_above, n_above);
-}
-
-// ---- compaction, at most four heads per index head ----------------------------------------------------------------
-// Every lane handles two scores of head slot (lane >> 2) & 3 (see lane_elems).  Keys above the bucket are counted and,
-// when id lists are requested, emitted; keys inside it become candidates for the exact finish.  Both kinds are rare
-// (a few per cent of the keys): a warp ballots them into per-head stages in shared memory.  The eight lanes of a
-// head keep the fill of its two stages in a register each (equal across those lanes).  The kernel runs for a few
-// microseconds per CTA, so its code is kept small: one 16-key group per loop iteration, flushes out of line.
-struct CompactStages {
-  int ids[kWarps][4][kStage];
-  uint2 cands[kWarps][4][kCandStage];
-};
-
-// Flushes the stages of all four heads of a warp (ids: which = 0, candidates: which = 1); cnt = this lane's head's fill.
-// (cnt is passed by value: a reference would pin the caller's counter to local memory)
-// heads4 = the retrieval-head indices of the four slots, one byte each.
-__device__ __noinline__ void flush_stage(CompactStages* sm, int which, int cnt, int warp, int lane, int64_t row_base,
-                                         uint32_t heads4, SelState* state, uint2* cand, int32_t* sel_idx,
-                                         int64_t sel_stride, int32_t* status) {
-  __syncwarp();
-#pragma unroll 1
-  for (int j = 0; j < 4; ++j) {
-    const int n = __shfl_sync(0xffffffffu, cnt, 4 * j);
-    if (n == 0) continue;
-    const int64_t rh = row_base + ((heads4 >> (8 * j)) & 0xffu);
-    int gbase = 0;
-    if (lane == 0) gbase = atomicAdd(which == 0 ? &state[rh].emit_cnt : &state[rh].cand_cnt, n);
-    gbase = __shfl_sync(0xffffffffu, gbase, 0);
-    for (int i = lane; i < n; i += 32) {
-      if (which == 0) {
-        if (gbase + i < sel_stride) sel_idx[rh * sel_stride + gbase + i] = sm->ids[warp][j][i];
-      } else {
-        if (gbase + i < kCandCap) cand[rh * kCandCap + gbase + i] = sm->cands[warp][j][i];
-      }
-    }
-    if (which == 0 && gbase + n > sel_stride && lane == 0) set_status(status, RTP_ERR_CAPACITY);
-  }
-  __syncwarp();
-}
-
-__global__ void __launch_bounds__(kThreads) sel_compact4_kernel(
-    const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows,
-    const __nv_bfloat16* __restrict__ qt, SelState* __restrict__ state, uint2* __restrict__ cand,
-    int32_t* __restrict__ sel_idx, int64_t sel_stride, int n_splits, int32_t* status) {
-  __shared__ CompactStages sm;
-  __shared__ int s_left[2][kWarps][4];   // [ids / candidates][warp][head]
-  __shared__ int s_base[2][4];
-  const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
-  if (x.p_lo >= x.p_hi) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int slot = (lane >> 2) & 3;
-  const float kInf = __int_as_float(0x7f800000);
-  const int64_t row_base = x.r * d.n_ret;
-  // (kernel parameters are only ever read by value: a pointer into them would force a copy of the struct to local memory)
-  const uint32_t heads4 = (uint32_t)hm.ih_heads[x.ih][0] | ((uint32_t)hm.ih_heads[x.ih][1] << 8) |
-                          ((uint32_t)hm.ih_heads[x.ih][2] << 16) | ((uint32_t)hm.ih_heads[x.ih][3] << 24);
-  SelState* st = slot < x.nh ? state + (row_base + ((heads4 >> (8 * slot)) & 0xffu)) : nullptr;
-  const int mode = st ? st->mode : -1;
-  float above = kInf, c_lo = kInf, c_hi = -kInf;   // emit raw > above; candidate raw in [c_lo, c_hi]
-  if (mode == kSelectAll) above = -kInf;
-  if (mode == kCollect || mode == kTieScan) above = st->raw_hi;
-  if (mode == kCollect) {
-    c_lo = st->raw_lo;
-    c_hi = st->raw_hi;
-  }
+  const KeySpan ks = key_span(x);
   const bool emit_ids = sel_idx != nullptr;
   const uint32_t lt = (1u << lane) - 1u;
-  const uint32_t mine = 0x000f000fu << (4 * slot);   // the lanes of this lane's head
-  int cnt_i = 0, cnt_c = 0;                          // fill of this head's stages (equal across its lanes)
-  int n_above = 0;
-  const QFrag qf = load_qfrag(qt + row_base * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
-
-  // flat loop over the 16-key groups of the warp's pages, the next two groups' keys in flight
-  const int n_it = x.p_lo + warp < x.p_hi ? ((x.p_hi - 1 - (x.p_lo + warp)) / kWarps + 1) * 4 : 0;
-  auto group_ptr = [&](int it) {
-    return ikey_page_ptr(cv, x.seq, x.p_lo + warp + (it >> 2) * kWarps, x.ih) + ((it & 3) * 32 + lane) * 8;
-  };
-  uint4 v1 = make_uint4(0u, 0u, 0u, 0u), v2 = v1;
-  if (n_it > 0) v1 = ld_stream_v4(group_ptr(0));
-  if (n_it > 1) v2 = ld_stream_v4(group_ptr(1));
+  const int nj = min(kHeadsPerCta, x.nh - z * kHeadsPerCta);
 #pragma unroll 1
-  for (int it = 0; it < n_it; ++it) {
-    const uint4 v = v1;
-    v1 = v2;
-    if (it + 2 < n_it) v2 = ld_stream_v4(group_ptr(it + 2));
-    const int n_grp = (x.p_lo + warp + (it >> 2) * kWarps) * kPage + (it & 3) * 16;
-    float s_lo[4], s_hi[4];
-    score16(qf, v, lane, s_lo, s_hi);
-    const LaneElems<true> el = lane_elems<true>(s_lo, s_hi, lane);
-    bool fa[2], fc[2];
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const bool ok = n_grp + el.koff[e] < x.n_keys;
-      fa[e] = ok && el.raw[e] > above;
-      fc[e] = ok && el.raw[e] >= c_lo && el.raw[e] <= c_hi;
-    }
-    n_above += (int)fa[0] + (int)fa[1];
-    if (!__any_sync(0xffffffffu, fc[0] || fc[1] || (emit_ids && (fa[0] || fa[1])))) continue;
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int n = n_grp + el.koff[e];
-      const uint32_t mc = __ballot_sync(0xffffffffu, fc[e]) & mine;
-      if (fc[e]) sm.cands[warp][slot][cnt_c + __popc(mc & lt)] = make_uint2(okey(finish_score(el.raw[e], d.score_scale)), (uint32_t)n);
-      cnt_c += __popc(mc);
-      if (emit_ids) {
-        const uint32_t ma = __ballot_sync(0xffffffffu, fa[e]) & mine;
-        if (fa[e]) sm.ids[warp][slot][cnt_i + __popc(ma & lt)] = n;
-        cnt_i += __popc(ma);
-      }
-    }
-    // one group of 16 keys adds at most 16 entries per head
-    if (__any_sync(0xffffffffu, cnt_c > kCandStage - 16)) {
-      flush_stage(&sm, 1, cnt_c, warp, lane, row_base, heads4, state, cand, sel_idx, sel_stride, status);
-      cnt_c = 0;
-    }
-    if (__any_sync(0xffffffffu, cnt_i > kStage - 16)) {
-      flush_stage(&sm, 0, cnt_i, warp, lane, row_base, heads4, state, cand, sel_idx, sel_stride, status);
+  for (int j = 0; j < nj; ++j) {
+    const int64_t rh = x.r * d.n_ret + hm.ih_heads[x.ih][z * kHeadsPerCta + j];
+    SelState* st = state + rh;
+    const int mode = st->mode;
+    const uint32_t lo_key = st->lo_key, hi_key = st->hi_key;
+    const bool all = mode == kSelectAll, bucket = mode == kCollect || mode == kTieScan, collect = mode == kCollect;
+    const float* row = scores + rh * l_pad;
+    int cnt_i = 0, cnt_c = 0, n_above = 0;   // fills are equal across the warp
+    auto flush_ids = [&]() {
+      int gbase = 0;
+      if (lane == 0) gbase = atomicAdd(&st->emit_cnt, cnt_i);
+      gbase = __shfl_sync(0xffffffffu, gbase, 0);
+      for (int i = lane; i < cnt_i; i += 32)
+        if (gbase + i < sel_stride) sel_idx[rh * sel_stride + gbase + i] = id_stage[warp][i];
+      if (gbase + cnt_i > sel_stride && lane == 0) set_status(status, RTP_ERR_CAPACITY);
       cnt_i = 0;
+      __syncwarp();
+    };
+    auto flush_cands = [&]() {
+      int gbase = 0;
+      if (lane == 0) gbase = atomicAdd(&st->cand_cnt, cnt_c);
+      gbase = __shfl_sync(0xffffffffu, gbase, 0);
+      for (int i = lane; i < cnt_c; i += 32)
+        if (gbase + i < kCandCap) cand[rh * kCandCap + gbase + i] = cand_stage[warp][i];
+      cnt_c = 0;
+      __syncwarp();
+    };
+    for (int nw = ks.k_lo + 128 * warp; nw < ks.k_hi; nw += 128 * kWarps) {
+      const int n0 = nw + 4 * lane;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (n0 < ks.k_hi) v = ld_scores4(row + n0);
+      const float s4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool ok = n0 + e < ks.k_hi;
+        const uint32_t key = okey(s4[e]);
+        const bool fa = ok && (all || (bucket && key > hi_key));
+        const bool fc = ok && collect && key >= lo_key && key <= hi_key;
+        n_above += (int)fa;
+        if (emit_ids) {
+          const uint32_t ma = __ballot_sync(0xffffffffu, fa);
+          if (fa) id_stage[warp][cnt_i + __popc(ma & lt)] = n0 + e;
+          cnt_i += __popc(ma);
+        }
+        const uint32_t mc = __ballot_sync(0xffffffffu, fc);
+        if (fc) cand_stage[warp][cnt_c + __popc(mc & lt)] = make_uint2(key, (uint32_t)(n0 + e));
+        cnt_c += __popc(mc);
+      }
+      __syncwarp();
+      if (cnt_i > kIdStage - 128) flush_ids();
+      if (cnt_c > kCandStageW - 128) flush_cands();
     }
+    if (cnt_i > 0) flush_ids();
+    if (cnt_c > 0) flush_cands();
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) n_above += __shfl_xor_sync(0xffffffffu, n_above, o);
+    if (lane == 0 && n_above && !all) atomicAdd(&st->cnt_above, n_above);
   }
-
-  // What is left in the stages is written with one counter update per CTA and head (thousands of warps updating the
-  // same few counters one by one would serialise in L2).
-  if ((lane & 19) == 0) {   // lanes 0, 4, 8, 12: one per head
-    s_left[0][warp][slot] = cnt_i;
-    s_left[1][warp][slot] = cnt_c;
-  }
-  __syncthreads();
-  if (threadIdx.x < 8) {
-    const int kind = threadIdx.x >> 2, j = threadIdx.x & 3;
-    int tot = 0;
-    for (int w = 0; w < kWarps; ++w) tot += s_left[kind][w][j];
-    int gbase = 0;
-    if (tot > 0) {
-      SelState* sj = state + (row_base + ((heads4 >> (8 * j)) & 0xffu));
-      gbase = atomicAdd(kind == 0 ? &sj->emit_cnt : &sj->cand_cnt, tot);
-      if (kind == 0 && gbase + tot > sel_stride) set_status(status, RTP_ERR_CAPACITY);
-    }
-    s_base[kind][j] = gbase;
-  }
-  __syncthreads();
-#pragma unroll 1
-  for (int j = 0; j < 4; ++j) {
-    const int ni = s_left[0][warp][j], nc = s_left[1][warp][j];
-    if (ni == 0 && nc == 0) continue;
-    const int64_t rh = row_base + ((heads4 >> (8 * j)) & 0xffu);
-    int off_i = s_base[0][j], off_c = s_base[1][j];
-    for (int w = 0; w < warp; ++w) {
-      off_i += s_left[0][w][j];
-      off_c += s_left[1][w][j];
-    }
-    for (int i = lane; i < ni; i += 32)
-      if (off_i + i < sel_stride) sel_idx[rh * sel_stride + off_i + i] = sm.ids[warp][j][i];
-    for (int i = lane; i < nc; i += 32)
-      if (off_c + i < kCandCap) cand[rh * kCandCap + off_c + i] = sm.cands[warp][j][i];
-  }
-  n_above += __shfl_xor_sync(0xffffffffu, n_above, 1);
-  n_above += __shfl_xor_sync(0xffffffffu, n_above, 2);
-  n_above += __shfl_xor_sync(0xffffffffu, n_above, 16);
-  if (st && lane < 16 && (lane & 3) == 0 && n_above && mode != kSelectAll) atomicAdd(&st->cnt_above, n_above);
 }
 
 // ---- finalize ---------------------------------------------------------------------------------------
@@ -882,9 +623,8 @@ constexpr int kFinWarps = kFinThreads / 32;
 constexpr int kNoPick = 0x7fffffff;
 
 __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
-    const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows,
-    const __nv_bfloat16* __restrict__ qt, SelState* __restrict__ state, const uint2* __restrict__ cand,
-    int32_t* __restrict__ sel_idx, int64_t sel_stride, int32_t* __restrict__ sel_count,
+    const Dims d, const float* __restrict__ scores, const int64_t l_pad, SelState* __restrict__ state,
+    const uint2* __restrict__ cand, int32_t* __restrict__ sel_idx, int64_t sel_stride, int32_t* __restrict__ sel_count,
     float* __restrict__ sel_mass, float* __restrict__ sel_thresh, int32_t* __restrict__ sel_tie_last,
     int32_t* status) {
   extern __shared__ __align__(16) unsigned char fin_smem[];
@@ -1094,13 +834,7 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
     const float e_t = __expf(okey_to_float(t_key) - M);
     int c = (int)ceilf((target - above) / e_t);
     c = max(1, min(c, st->bucket_cnt));
-    const int64_t r = rh / d.n_ret;
-    const int head = (int)(rh % d.n_ret);
-    const int ih = hm.q2ih[head];
-    const int slot = hm.slot_in_ih[head];
-    const int seq = rows.row_seq(r);
-    const QFrag qf = load_qfrag(qt + r * d.n_ret * kIndexDim, hm.ih_heads[ih], hm.ih_nheads[ih], lane);
-    unsigned char* flags = reinterpret_cast<unsigned char*>(keys);  // [kFinWarps * 64]
+    const float* row = scores + rh * l_pad;
     if (tid == 0) {
       s_emitted = 0;
       s_last = -1;
@@ -1109,29 +843,14 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
     const int n_pages = (n_keys + kPage - 1) >> kPageShift;
     for (int p0 = 0; p0 < n_pages; p0 += kFinWarps) {
       if (s_emitted >= c) break;  // uniform (see barrier at the end of the round)
-      const int p = p0 + warp;
-      if (p < n_pages) {
-        const __nv_bfloat16* pb = ikey_page_ptr(cv, seq, p, ih);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint4 v = ld_stream_v4(pb + (i * 32 + lane) * 8);
-          float s_lo[4], s_hi[4];
-          score16(qf, v, lane, s_lo, s_hi);
-          if ((lane >> 2) == (slot & 7)) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int n = p * kPage + i * 16 + 4 * (lane & 3) + e;
-              const uint32_t key = okey(finish_score((slot >> 3) ? s_hi[e] : s_lo[e], d.score_scale));
-              flags[warp * kPage + i * 16 + 4 * (lane & 3) + e] = (n < n_keys && key == t_key) ? 1 : 0;
-            }
-          }
-        }
-      } else {
-        for (int i = lane; i < kPage; i += 32) flags[warp * kPage + i] = 0;
-      }
-      __syncthreads();
       // ordered emission: thread t owns keys 2t, 2t+1 of this round
-      const int f0 = flags[2 * tid], f1 = flags[2 * tid + 1];
+      const int n_first = p0 * kPage + 2 * tid;
+      int f0 = 0, f1 = 0;
+      if (n_first < n_keys) {
+        const float2 sv = *reinterpret_cast<const float2*>(row + n_first);
+        f0 = okey(sv.x) == t_key;
+        f1 = n_first + 1 < n_keys && okey(sv.y) == t_key;
+      }
       int inc = f0 + f1;
       const int mine = inc;
 #pragma unroll
@@ -1147,7 +866,6 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
         tot += w_cnt[w];
       }
       int before = s_emitted + wbase + inc - mine;
-      const int n_first = p0 * kPage + 2 * tid;
       if (f0) {
         if (before < c) {
           if (ids && emit_base + before < sel_stride) ids[emit_base + before] = n_first;
@@ -1195,11 +913,12 @@ struct SelWorkspace {
   uint32_t* g_cnt;              // [row heads][64] merged bin counts
   uint32_t* tickets;            // [rows * index heads]
   uint2* cand;
+  float* scores;                // [row heads][l_pad] scores of the first pass
   size_t zero_off, zero_bytes;  // the part that must be zero before the first pass
   size_t bytes;
 };
 
-SelWorkspace carve(void* ws, int64_t n_rowheads, int64_t n_units) {
+SelWorkspace carve(void* ws, int64_t n_rowheads, int64_t n_units, int64_t l_pad) {
   SelWorkspace w;
   size_t off = 0;
   auto take = [&](size_t n) {
@@ -1212,12 +931,14 @@ SelWorkspace carve(void* ws, int64_t n_rowheads, int64_t n_units) {
   const size_t o_cnt = take(sizeof(uint32_t) * kBins * n_rowheads);
   const size_t o_tick = take(sizeof(uint32_t) * n_units);
   const size_t o_cand = take(sizeof(uint2) * kCandCap * n_rowheads);
+  const size_t o_scores = take(sizeof(float) * (size_t)l_pad * n_rowheads);
   char* b = reinterpret_cast<char*>(ws);
   w.state = reinterpret_cast<SelState*>(b + o_state);
   w.g_mass = reinterpret_cast<unsigned long long*>(b + o_mass);
   w.g_cnt = reinterpret_cast<uint32_t*>(b + o_cnt);
   w.tickets = reinterpret_cast<uint32_t*>(b + o_tick);
   w.cand = reinterpret_cast<uint2*>(b + o_cand);
+  w.scores = reinterpret_cast<float*>(b + o_scores);
   w.zero_off = o_mass;
   w.zero_bytes = o_cand - o_mass;
   w.bytes = off;
@@ -1226,23 +947,13 @@ SelWorkspace carve(void* ws, int64_t n_rowheads, int64_t n_units) {
 
 constexpr int kKeyLevels = 6;   // 6 bits each: a level-1 bucket spans fewer than 2^32 key values
 
-template <bool NH4>
-cudaError_t launch_passes(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
-                          const __nv_bfloat16* qt, const SelWorkspace& w, int n_splits, int32_t* status,
-                          cudaStream_t st) {
-  dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
-  sel_max_kernel<NH4><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, n_splits, status);
-  sel_l1_kernel<NH4><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.g_mass, w.tickets, n_splits, status);
-  sel_key_kernel<NH4><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.g_mass, w.g_cnt, w.tickets, n_splits,
-                                                 1 + kKeyLevels, status);
-  return cudaGetLastError();
-}
-
 }  // namespace
 
-size_t select_rows_workspace_bytes(const Dims& d, int64_t R) {
+int64_t padded_len(int64_t max_len) { return (max_len + kPage - 1) / kPage * kPage; }
+
+size_t select_rows_workspace_bytes(const Dims& d, int64_t R, int64_t max_len) {
   if (R <= 0 || d.n_ret <= 0) return 0;
-  return carve(nullptr, R * d.n_ret, R * d.n_ih).bytes;
+  return carve(nullptr, R * d.n_ret, R * d.n_ih, padded_len(max_len)).bytes;
 }
 
 cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
@@ -1251,7 +962,8 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
                                int32_t* status, void* ws, int sm_count, cudaStream_t st) {
   if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
   const int64_t nrh = rows.R * d.n_ret;
-  const SelWorkspace w = carve(ws, nrh, rows.R * d.n_ih);
+  const int64_t l_pad = padded_len(max_len);
+  const SelWorkspace w = carve(ws, nrh, rows.R * d.n_ih, l_pad);
   cudaError_t e = cudaSuccess;
   {
     const int64_t n_zero = (int64_t)(w.zero_bytes / 4);
@@ -1264,25 +976,28 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
   int max_nh = 0;
   for (int i = 0; i < d.n_ih; ++i) max_nh = hm.ih_nheads[i] > max_nh ? hm.ih_nheads[i] : max_nh;
   const int n_splits = select_splits(d, rows.R, max_len, sm_count);
-  e = max_nh <= 4 ? launch_passes<true>(cv, d, hm, rows, qt, w, n_splits, status, st)
-                  : launch_passes<false>(cv, d, hm, rows, qt, w, n_splits, status, st);
-  if (e != cudaSuccess) return e;
-  if (max_nh <= 4) {
-    dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
-    sel_compact4_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.cand, sel_idx, sel_stride, n_splits,
-                                                   status);
-  } else {
-    dim3 grid((unsigned)(rows.R * d.n_ih), n_splits, (max_nh + kHeadsPerCta - 1) / kHeadsPerCta);
-    sel_compact_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.cand, sel_idx, sel_stride, n_splits,
-                                                  status);
+  const dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
+  // one scan of the index keys (scores stored, row maxima), then three passes over the stored scores
+  if (max_nh <= 4)
+    sel_score_kernel<true><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status);
+  else
+    sel_score_kernel<false><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status);
+  sel_l1_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.tickets, n_splits, status);
+  sel_key_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.g_cnt, w.tickets,
+                                            n_splits, 1 + kKeyLevels, status);
+  {
+    const dim3 grid3((unsigned)(rows.R * d.n_ih), n_splits, (max_nh + kHeadsPerCta - 1) / kHeadsPerCta);
+    sel_compact_kernel<<<grid3, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.cand, sel_idx, sel_stride,
+                                                   n_splits, status);
   }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
   constexpr int kFinSmem = 2 * kCandCap * 8;
   static PerDeviceOnce fin_once;
   e = set_dyn_smem_once(sel_finalize_kernel, kFinSmem, fin_once);
   if (e != cudaSuccess) return e;
-  sel_finalize_kernel<<<(unsigned)nrh, kFinThreads, kFinSmem, st>>>(cv, d, hm, rows, qt, w.state, w.cand, sel_idx,
-                                                             sel_stride, sel_count, sel_mass, sel_thresh,
-                                                             sel_tie_last, status);
+  sel_finalize_kernel<<<(unsigned)nrh, kFinThreads, kFinSmem, st>>>(d, w.scores, l_pad, w.state, w.cand, sel_idx, sel_stride,
+                                                             sel_count, sel_mass, sel_thresh, sel_tie_last, status);
   return cudaGetLastError();
 }
 
