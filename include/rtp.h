@@ -242,13 +242,13 @@ rtp_status rtp_sparse_attn_decode(rtp_ctx* ctx, const rtp_params* params, const 
  * Same computation, arguments and results as rtp_sparse_attn_decode, for hosts that cannot provide
  * scratch memory at call time: e.g. a serving process whose device heap was handed over entirely to a
  * pool it does not own, a plugin that runs inside someone else's allocator-free region, or code that
- * runs where cudaMalloc is forbidden.  The split partials live in a fixed 1 MiB array that is part of
+ * runs where cudaMalloc is forbidden.  The split partials live in a fixed 512 KiB array that is part of
  * the library image (every GPU that loads the library holds it until the process exits); the call
  * allocates nothing and calls no allocating routine.
- *  - Limit: rows * n_ret_q_heads * n_splits * 520 bytes must fit in 1 MiB, where n_splits is the
- *    split count the library plans for the call (about 8 * SM count / (rows * heads), at most one
- *    split per 256 listed tokens; a decode batch of up to 64 sequences x 8 retrieval heads always
- *    fits).  Larger calls return RTP_ERR_CAPACITY before anything is launched
+ *  - Limit: rows * n_ret_q_heads * n_splits * 520 bytes must fit in 512 KiB, where n_splits is the
+ *    split count the library plans for the call (about 4 * SM count / (rows * heads), at most one
+ *    split per 512 listed tokens, nothing at all for a single split; on a 148-SM device a decode
+ *    batch of up to 63 sequences x 8 retrieval heads always fits).  Larger calls return RTP_ERR_CAPACITY before anything is launched
  *    and rtp_last_error says how many bytes were needed.
  *  - The first call on each device looks up the array's device address (once per device, with that
  *    device current); make that first call outside any CUDA stream capture.

@@ -265,7 +265,7 @@ def rtp_sparse_attn_decode(ctx, params, cache, q, row_seq, row_pos, sel_idx, sel
 def rtp_sparse_attn_decode_static(ctx, params, cache, q, row_seq, row_pos, sel_idx, sel_count, out, lse, status,
                                   stream=None):
     """rtp_sparse_attn_decode for callers that cannot hand over scratch memory: the split partials go to a
-    1 MiB array built into the library, so nothing is allocated.  Calls must not overlap on the GPU."""
+    512 KiB array built into the library, so nothing is allocated.  Calls must not overlap on the GPU."""
     ctx._check(ctx.lib.rtp_sparse_attn_decode_static(ctx.h, params.ref(), C.byref(cache), _ptr(q), _ptr(row_seq),
                                                      _ptr(row_pos), int(row_seq.shape[0]), _ptr(sel_idx),
                                                      int(sel_idx.shape[-1]), _ptr(sel_count), _ptr(out), _ptr(lse),

@@ -1,7 +1,13 @@
 // S5 / S7 (decode) / S8 / S9 (decode): attention of single query rows over a token set (Eq. 5):
-// a selection list, the sink + window pattern, or the full causal prefix.  Bandwidth-bound: every
-// K and V row is read once with 16-byte loads (a half-warp per 256-byte row), all query heads of a
-// KV group share the loaded rows, the set is split over CTAs and merged by log-sum-exp.
+// a selection list, the sink + window pattern, or the full causal prefix.  Bandwidth-bound, so the kernel is built
+// around keeping many K / V rows in flight with few instructions per row:
+//   - the set is split over CTAs (merged by log-sum-exp) and, inside a CTA, dealt to four warps in tiles of 16 tokens;
+//   - every warp owns a ring of three tiles in shared memory, filled with 16-byte cp.async copies (a half-warp per
+//     256-byte row) two tiles ahead of the one it works on; where a row lives (list entry -> block table -> offset) is
+//     resolved another two tiles ahead, so that none of these dependent loads is waited for;
+//   - Q K^T and P V of a tile are warp MMAs (m16n8k16, bf16 -> fp32): the G query heads of the KV group are rows of the
+//     A operand (the other rows are zero), the tile's K rows are read with ldmatrix, its V rows with ldmatrix.trans,
+//     from a layout whose 16-byte chunks are XOR-swizzled with the token number (no bank conflicts).
 #include <mutex>
 
 #include "rtp_device.cuh"
@@ -12,36 +18,54 @@ namespace {
 
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
-constexpr int kStreams = kWarps * 2;   // one online-softmax stream per half-warp
-constexpr int kUnroll = 4;             // tokens in flight per half-warp
-constexpr int kPartial = kHeadDim + 2; // acc[128], m, l
+constexpr int kTileTok = 16;                               // tokens per tile
+constexpr int kRing = 3;                                   // tiles per warp in shared memory
+constexpr int kTileBytes = kTileTok * kHeadDim * 2;        // K (or V) rows of a tile: 4 KB
+constexpr int kWarpRingBytes = kRing * 2 * kTileBytes;     // 24 KB
+constexpr int kRowsSmem = kWarps * kWarpRingBytes;         // 96 KB: two CTAs per SM
+constexpr int kPartial = kHeadDim + 2;                     // acc[128], m, l
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
-  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float2 x = __bfloat1622float2(p[i]);
-    f[2 * i] = x.x;
-    f[2 * i + 1] = x.y;
-  }
+__device__ __forceinline__ void cp16z(uint32_t dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
 }
+__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldsm4t(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+// d (rows g of the 16 x 8 result) += A B, where rows 8-15 of A are zero: only the two accumulators of row g are kept.
+__device__ __forceinline__ void mma_row8(float (&d)[2], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "{\n"
+      ".reg .f32 x2, x3;\n"
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,x2,x3}, {%2,%3,%4,%3}, {%5,%6}, {%0,%1,%7,%7};\n"
+      "}\n"
+      : "+f"(d[0]), "+f"(d[1])
+      : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1), "f"(0.f));
+}
+// byte offset of 16-byte chunk ch (0..15) of token t inside a tile
+__device__ __forceinline__ uint32_t tile_off(int t, int ch) { return (uint32_t)(t * 256 + (((ch & 8) | ((ch ^ t) & 7)) << 4)); }
 
 template <int G, int SET>
-__global__ void __launch_bounds__(kThreads, (G == 1) ? 6 : 1) attn_rows_kernel(
+__global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
     const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows, const int n_units,
     const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ sel_idx, const int64_t sel_stride,
     const int32_t* __restrict__ sel_count, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
     float* __restrict__ partial, const int n_splits, int32_t* status) {
-  __shared__ float red[kStreams][G][kPartial];
+  static_assert(G >= 1 && G <= 8, "the query heads of a KV group are rows 0..7 of the MMA");
+  extern __shared__ __align__(128) unsigned char smem_rows[];
 
   const int64_t r = blockIdx.x / n_units;
   const int u = blockIdx.x % n_units;
   const int split = blockIdx.y;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int l16 = lane & 15, hw = lane >> 4;
-  const int stream = warp * 2 + hw;
+  const int g = lane >> 2, c = lane & 3;
 
   int qh0, kvh;
   if (SET == kSetList) {
@@ -80,159 +104,198 @@ __global__ void __launch_bounds__(kThreads, (G == 1) ? 6 : 1) attn_rows_kernel(
   const int per = (n_set + n_splits - 1) / n_splits;
   const int t_lo = split * per;
   const int t_hi = min(n_set, t_lo + per);
+  const int n_tiles = t_hi > t_lo ? (t_hi - t_lo + kTileTok - 1) / kTileTok : 0;
+  const int n_mine = n_tiles > warp ? (n_tiles - warp + kWarps - 1) / kWarps : 0;   // tiles warp, warp + 4, ...
 
-  // queries of the group, pre-scaled so that logits are in log2 units
-  float qf[G][8];
-  {
-    const float sc = d.sm_scale * kLog2e;
+  // A fragments of the queries: row g = head g of the group (zero rows beyond G), 8 steps of 16 dims
+  uint32_t qa[8][2];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      const uint4 v = ld_nc_v4(q + ((int64_t)r * d.n_q + qh0 + g) * kHeadDim + l16 * 8);
-      unpack8(v, qf[g]);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) qf[g][i] *= sc;
+  for (int ks = 0; ks < 8; ++ks) {
+    qa[ks][0] = 0u;
+    qa[ks][1] = 0u;
+    if (g < G) {
+      const __nv_bfloat16* qp = q + ((int64_t)r * d.n_q + qh0 + g) * kHeadDim + 16 * ks + 2 * c;
+      qa[ks][0] = *reinterpret_cast<const uint32_t*>(qp);
+      qa[ks][1] = *reinterpret_cast<const uint32_t*>(qp + 8);
     }
   }
-  float m_run[G], l_run[G], acc[G][8];
+  const float sc = d.sm_scale * kLog2e;   // logits in log2 units
+  float o[16][2];                         // row g, dims 8 j + 2 c, + 1
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
-    m_run[g] = -INFINITY;
-    l_run[g] = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc[g][i] = 0.f;
-  }
-  const int64_t bt_base = (int64_t)seq * cv.max_pages;
+  for (int j = 0; j < 16; ++j) o[j][0] = o[j][1] = 0.f;
+  float m_run = -INFINITY, l_part = 0.f;
 
-  // Where the rows of a batch of tokens live (list entry -> block table -> offset) is resolved one batch ahead, so
-  // that these two dependent loads are in flight together with the K / V rows of the current batch.
-  int64_t off_n[kUnroll];
-  bool ok_n[kUnroll];
-  auto resolve = [&](int tb) {
-#pragma unroll
-    for (int x = 0; x < kUnroll; ++x) {
-      const int t = tb + hw + x * kStreams;
-      ok_n[x] = t < t_hi;
-      off_n[x] = 0;
-      if (ok_n[x]) {
-        int tok;
-        if (SET == kSetList) {
-          tok = __ldg(ids + t);
-          if (tok < 0 || tok >= n_keys) {
-            set_status(status, RTP_ERR_INVALID);
-            ok_n[x] = false;
-          }
-        } else if (SET == kSetLocal) {
-          tok = t < ns ? t : wlo + (t - ns);
-        } else {
-          tok = t;
-        }
-        if (ok_n[x]) {
-          const int phys = safe_phys(cv, bt_base + (tok >> kPageShift), status);
-          off_n[x] = (((int64_t)phys * cv.n_kv + kvh) * kPage + (tok & (kPage - 1))) * kHeadDim + l16 * 8;
-        }
+  const int64_t bt_base = (int64_t)seq * cv.max_pages;
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(smem_rows) + warp * kWarpRingBytes;
+  // token of entry (lane & 15) of this warp's i-th tile, or -1
+  auto load_tok = [&](int i) -> int {
+    const int t = t_lo + (warp + i * kWarps) * kTileTok + (lane & 15);
+    if (i >= n_mine || t >= t_hi) return -1;
+    if (SET == kSetList) {
+      const int tok = __ldg(ids + t);
+      if (tok < 0 || tok >= n_keys) {
+        set_status(status, RTP_ERR_INVALID);
+        return -1;
       }
+      return tok;
+    }
+    if (SET == kSetLocal) return t < ns ? t : wlo + (t - ns);
+    return t;
+  };
+  auto load_phys = [&](int tok) -> int { return tok >= 0 ? safe_phys(cv, bt_base + (tok >> kPageShift), status) : 0; };
+  // requests the K and V rows of a tile: token tt of the tile is copied by the half-warp (tt & 1) in step tt >> 1
+  auto issue = [&](int stage, int tok, int phys) {
+    const int64_t off = (((int64_t)phys * cv.n_kv + kvh) * kPage + (tok & (kPage - 1))) * kHeadDim;
+    const uint32_t sk = ring + stage * 2 * kTileBytes, sv = sk + kTileBytes;
+    const int ch = lane & 15;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int tt = 2 * i + (lane >> 4);
+      const int64_t o_t = __shfl_sync(0xffffffffu, off, tt);
+      const bool ok = __shfl_sync(0xffffffffu, tok, tt) >= 0;
+      const int64_t src = ok ? o_t + ch * 8 : 0;
+      cp16z(sk + tile_off(tt, ch), cv.k + src, ok);
+      cp16z(sv + tile_off(tt, ch), cv.v + src, ok);
     }
   };
-  // (only lists have the extra dependent load; the other sets resolve in place and keep their register count)
-  if (SET == kSetList) resolve(t_lo + warp * 2);
-  for (int tb = t_lo + warp * 2; tb < t_hi; tb += kStreams * kUnroll) {
-    if (SET != kSetList) resolve(tb);
-    uint4 kr[kUnroll], vr[kUnroll];
-    bool ok[kUnroll];
+  // prologue: two tiles requested; the addresses of the third resolved, the tokens of the fourth on their way
+  int tok_c[kRing];   // tokens of the tiles in the ring (for the validity mask)
+  {
+    const int t0 = load_tok(0), t1 = load_tok(1);
+    const int p0 = load_phys(t0), p1 = load_phys(t1);
+    issue(0, t0, p0);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    issue(1, t1, p1);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    tok_c[0] = t0;
+    tok_c[1] = t1;
+    tok_c[2] = -1;
+  }
+  int tok_a = load_tok(2);
+  int phys_a = load_phys(tok_a);
+  int tok_b = load_tok(3);
+
+#pragma unroll 1
+  for (int i0 = 0; i0 < n_mine; i0 += kRing) {
 #pragma unroll
-    for (int x = 0; x < kUnroll; ++x) {
-      ok[x] = ok_n[x];
-      kr[x] = make_uint4(0, 0, 0, 0);
-      vr[x] = make_uint4(0, 0, 0, 0);
-      if (ok[x]) {
-        kr[x] = ld_stream_v4(cv.k + off_n[x]);
-        vr[x] = ld_stream_v4(cv.v + off_n[x]);
+    for (int sgi = 0; sgi < kRing; ++sgi) {
+      const int i = i0 + sgi;
+      if (i < n_mine) {   // uniform in the warp
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+        __syncwarp();
+        // tile i + 2 goes where tile i - 1 was
+        const int next_stage = (sgi + 2) % kRing;
+        issue(next_stage, tok_a, phys_a);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        tok_c[next_stage] = tok_a;
+        tok_a = tok_b;
+        phys_a = load_phys(tok_a);      // used in the next step
+        tok_b = load_tok(i + 4);        // used in the step after that
+
+        const uint32_t sk = ring + sgi * 2 * kTileBytes, sv = sk + kTileBytes;
+        const uint32_t vmask = __ballot_sync(0xffffffffu, tok_c[sgi] >= 0) & 0xffffu;   // bit t = token t of the tile exists
+        // ---- S = Q K^T: two 8-token halves ----
+        float s[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+        {
+          const int mi = lane >> 3, rr = lane & 7;
+          const int tk = (mi >> 1) * 8 + rr;
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            uint32_t b[4];
+            ldsm4(sk + tile_off(tk, 2 * ks + (mi & 1)), b);
+            mma_row8(s[0], qa[ks][0], qa[ks][1], b[0], b[1]);
+            mma_row8(s[1], qa[ks][0], qa[ks][1], b[2], b[3]);
+          }
+        }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const bool ok = (vmask >> (8 * nt + 2 * c + e)) & 1u;
+            s[nt][e] = ok ? s[nt][e] * sc : -INFINITY;
+            mx = fmaxf(mx, s[nt][e]);
+          }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);
+        if (__any_sync(0xffffffffu, m_new > m_run)) {
+          const float corr = (m_run == -INFINITY) ? 0.f : fast_ex2(m_run - m_new);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            o[j][0] *= corr;
+            o[j][1] *= corr;
+          }
+          l_part *= corr;
+          m_run = m_new;
+        }
+        const float mb = (m_run == -INFINITY) ? 0.f : m_run;
+        const float p00 = fast_ex2(s[0][0] - mb), p01 = fast_ex2(s[0][1] - mb);
+        const float p10 = fast_ex2(s[1][0] - mb), p11 = fast_ex2(s[1][1] - mb);
+        l_part += (p00 + p01) + (p10 + p11);
+        uint32_t pa0, pa2;
+        {
+          const __nv_bfloat162 x = __floats2bfloat162_rn(p00, p01), y = __floats2bfloat162_rn(p10, p11);
+          pa0 = *reinterpret_cast<const uint32_t*>(&x);
+          pa2 = *reinterpret_cast<const uint32_t*>(&y);
+        }
+        // ---- O += P V: 16 slices of eight dims, two per ldmatrix ----
+        {
+          const int mi = lane >> 3, rr = lane & 7;
+          const int tk = (mi & 1) * 8 + rr;
+#pragma unroll
+          for (int j = 0; j < 16; j += 2) {
+            uint32_t b[4];
+            ldsm4t(sv + tile_off(tk, j + (mi >> 1)), b);
+            mma_row8(o[j], pa0, pa2, b[0], b[1]);
+            mma_row8(o[j + 1], pa0, pa2, b[2], b[3]);
+          }
+        }
       }
-    }
-    if (SET == kSetList) resolve(tb + kStreams * kUnroll);
-    float logit[kUnroll][G];
-#pragma unroll
-    for (int x = 0; x < kUnroll; ++x) {
-      float kf[8];
-      unpack8(kr[x], kf);
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float s = 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) s = fmaf(qf[g][i], kf[i], s);
-        s += __shfl_xor_sync(0xffffffffu, s, 8);
-        s += __shfl_xor_sync(0xffffffffu, s, 4);
-        s += __shfl_xor_sync(0xffffffffu, s, 2);
-        s += __shfl_xor_sync(0xffffffffu, s, 1);
-        logit[x][g] = ok[x] ? s : -INFINITY;
-      }
-    }
-    float pw[kUnroll][G];
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float mx = m_run[g];
-#pragma unroll
-      for (int x = 0; x < kUnroll; ++x) mx = fmaxf(mx, logit[x][g]);
-      if (mx == -INFINITY) {
-#pragma unroll
-        for (int x = 0; x < kUnroll; ++x) pw[x][g] = 0.f;
-        continue;
-      }
-      const float corr = fast_ex2(m_run[g] - mx);
-      float ls = l_run[g] * corr;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) acc[g][i] *= corr;
-#pragma unroll
-      for (int x = 0; x < kUnroll; ++x) {
-        pw[x][g] = fast_ex2(logit[x][g] - mx);
-        ls += pw[x][g];
-      }
-      l_run[g] = ls;
-      m_run[g] = mx;
-    }
-#pragma unroll
-    for (int x = 0; x < kUnroll; ++x) {
-      float vf[8];
-      unpack8(vr[x], vf);
-#pragma unroll
-      for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc[g][i] = fmaf(pw[x][g], vf[i], acc[g][i]);
     }
   }
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();   // the rings are free: they now hold the warps' partial results
 
-  // merge the eight streams of the CTA
+  float l_run = l_part;
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+  float* red = reinterpret_cast<float*>(smem_rows);   // [kWarps][G][kPartial]
+  if (g < G) {
+    float* rw = red + (warp * G + g) * kPartial;
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) red[stream][g][l16 * 8 + i] = acc[g][i];
-    if (l16 == 0) {
-      red[stream][g][kHeadDim] = m_run[g];
-      red[stream][g][kHeadDim + 1] = l_run[g];
+    for (int j = 0; j < 16; ++j) {
+      rw[8 * j + 2 * c] = o[j][0];
+      rw[8 * j + 2 * c + 1] = o[j][1];
+    }
+    if (c == 0) {
+      rw[kHeadDim] = m_run;
+      rw[kHeadDim + 1] = l_run;
     }
   }
   __syncthreads();
   const int dim = threadIdx.x;  // 128 threads = 128 dims
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
+  for (int gg = 0; gg < G; ++gg) {
     float mt = -INFINITY;
 #pragma unroll
-    for (int s = 0; s < kStreams; ++s) mt = fmaxf(mt, red[s][g][kHeadDim]);
+    for (int w = 0; w < kWarps; ++w) mt = fmaxf(mt, red[(w * G + gg) * kPartial + kHeadDim]);
     float lt = 0.f, a = 0.f;
     if (mt != -INFINITY) {
 #pragma unroll
-      for (int s = 0; s < kStreams; ++s) {
-        const float w = fast_ex2(red[s][g][kHeadDim] - mt);
-        lt += red[s][g][kHeadDim + 1] * w;
-        a += red[s][g][dim] * w;
+      for (int w = 0; w < kWarps; ++w) {
+        const float* rw = red + (w * G + gg) * kPartial;
+        const float wgt = fast_ex2(rw[kHeadDim] - mt);
+        lt += rw[kHeadDim + 1] * wgt;
+        a += rw[dim] * wgt;
       }
     }
-    const int64_t oh = (int64_t)r * d.n_q + qh0 + g;
+    const int64_t oh = (int64_t)r * d.n_q + qh0 + gg;
     if (n_splits == 1) {
       out[oh * kHeadDim + dim] = __float2bfloat16_rn(lt > 0.f ? a / lt : 0.f);
       if (lse && dim == 0) lse[oh] = lt > 0.f ? (mt + log2f(lt)) * kLn2 : -INFINITY;
     } else {
-      float* p = partial + (((int64_t)blockIdx.x * G + g) * n_splits + split) * kPartial;
+      float* p = partial + (((int64_t)blockIdx.x * G + gg) * n_splits + split) * kPartial;
       p[dim] = a;
       if (dim == 0) {
         p[kHeadDim] = mt;
@@ -272,8 +335,8 @@ __global__ void __launch_bounds__(kHeadDim) attn_merge_kernel(const Dims d, cons
 
 int plan_splits(int64_t units, int64_t max_set, int sm_count) {
   if (units <= 0) return 1;
-  int64_t want = (8LL * sm_count + units - 1) / units;
-  int64_t cap = (max_set + 255) / 256;  // at least 256 tokens per CTA
+  int64_t want = (4LL * sm_count + units - 1) / units;   // two rounds of two resident CTAs per SM
+  int64_t cap = (max_set + 511) / 512;                   // at least 512 tokens (eight tiles per warp) per CTA
   int64_t s = want < cap ? want : cap;
   if (s < 1) s = 1;
   if (s > 512) s = 512;
@@ -295,9 +358,12 @@ cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm,
                          const int32_t* sel_count, __nv_bfloat16* out, float* lse, float* partial, int n_splits,
                          int32_t* status, cudaStream_t st) {
   dim3 grid((unsigned)(rows.R * n_units), n_splits);
-  attn_rows_kernel<G, SET><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, n_units, q, sel_idx, sel_stride, sel_count,
-                                                      out, lse, partial, n_splits, status);
-  cudaError_t e = cudaGetLastError();
+  static PerDeviceOnce once;   // (one per instantiation)
+  cudaError_t e = set_dyn_smem_once(attn_rows_kernel<G, SET>, kRowsSmem, once);
+  if (e != cudaSuccess) return e;
+  attn_rows_kernel<G, SET><<<grid, kThreads, kRowsSmem, st>>>(cv, d, hm, rows, n_units, q, sel_idx, sel_stride,
+                                                              sel_count, out, lse, partial, n_splits, status);
+  e = cudaGetLastError();
   if (e != cudaSuccess || n_splits == 1) return e;
   attn_merge_kernel<SET><<<(unsigned)(rows.R * n_units * G), kHeadDim, 0, st>>>(d, hm, n_units, G, partial,
                                                                                 n_splits, out, lse);
@@ -346,7 +412,7 @@ cudaError_t launch_attn_rows(const CacheView& cv, const Dims& d, const HeadMaps&
 
 // ---- split partials in a static device array (entry point for callers that must not allocate) --------
 // kStaticScratchBytes of global memory are part of the library image on every GPU that loads it.
-constexpr size_t kStaticScratchBytes = 1u << 20;
+constexpr size_t kStaticScratchBytes = 512u << 10;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 namespace {

@@ -53,12 +53,12 @@ def test_static_scratch_rejects_oversized_calls():
     from tests import gpu_harness as gh
     wl = synth.config_5(L=4096, batch=2, top_p=0.9, frac=0.2)
     dw = gh.DeviceWorkload(wl)
-    R = 138                                                              # 138 rows x 8 heads x 2 splits x 520 B > 1 MiB
+    R = 70                                                               # 70 rows x 8 heads x 2 splits x 520 B > 512 KiB
     q = dw.q[:1].expand(R, -1, -1).contiguous()
     row_seq = torch.zeros(R, dtype=torch.int32, device="cuda")
     row_pos = torch.full((R,), 4095, dtype=torch.int32, device="cuda")
-    idx = torch.zeros((R, dw.n_ret, 512), dtype=torch.int32, device="cuda")
-    cnt = torch.full((R, dw.n_ret), 512, dtype=torch.int32, device="cuda")
+    idx = torch.zeros((R, dw.n_ret, 1024), dtype=torch.int32, device="cuda")
+    cnt = torch.full((R, dw.n_ret), 1024, dtype=torch.int32, device="cuda")
     out = torch.zeros((R, wl.heads.n_q_heads, 128), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(rb.RtpError) as e:
         rb.rtp_sparse_attn_decode_static(dw.ctx, dw.params, dw.cache, q, row_seq, row_pos, idx, cnt, out, None,
