@@ -210,6 +210,7 @@ __global__ void __launch_bounds__(kThreads) sel_score_kernel(const CacheView cv,
 
 // The later passes read the stored scores: the CTA's share of a row is keys [k_lo, k_hi), four consecutive keys per
 // thread and step (one 16-byte load).
+constexpr int kLoads = 4;   // 16-byte loads a thread keeps in flight in the passes over the stored scores
 struct KeySpan {
   int k_lo, k_hi;
 };
@@ -230,8 +231,9 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
                                                           const Rows rows, const float* __restrict__ scores,
                                                           const int64_t l_pad, SelState* __restrict__ state,
                                                           unsigned long long* __restrict__ g_mass,
-                                                          uint32_t* __restrict__ tickets, int n_splits, int32_t* status) {
-  __shared__ uint32_t hist[kWarps][kBins][2];   // one private histogram per warp, for the head being scanned
+                                                          uint32_t* __restrict__ tickets, int n_splits, const int list_cap,
+                                                          int32_t* status) {
+  __shared__ uint32_t hist[kHeadsPerCta][kWarps][kBins][2];   // one private histogram per warp and head of the chunk
   __shared__ float s_M[16];
   __shared__ int s_on[16];
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
@@ -247,38 +249,50 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
     s_on[threadIdx.x] = on;
     s_M[threadIdx.x] = M;
   }
-  for (int i = threadIdx.x; i < kWarps * kBins * 2; i += kThreads) (&hist[0][0][0])[i] = 0u;
+  for (int i = threadIdx.x; i < kHeadsPerCta * kWarps * kBins * 2; i += kThreads) (&hist[0][0][0][0])[i] = 0u;
   __syncthreads();
   int any = 0;
   for (int j = 0; j < x.nh; ++j) any |= s_on[j];
   if (!any) return;   // the same decision in every CTA of the unit
 
   const KeySpan ks = key_span(x);
-  for (int j = 0; j < x.nh; ++j) {
-    if (!s_on[j]) continue;   // uniform
-    const int64_t rh = x.r * d.n_ret + hm.ih_heads[x.ih][j];
-    const float* row = scores + rh * l_pad;
-    const float M = s_M[j];
-    for (int n0 = ks.k_lo + 4 * (int)threadIdx.x; n0 < ks.k_hi; n0 += 4 * kThreads) {
-      const float4 v = ld_scores4(row + n0);
-      const float s4[4] = {v.x, v.y, v.z, v.w};
+  for (int j0 = 0; j0 < x.nh; j0 += kHeadsPerCta) {   // four heads at a time: their loads are in flight together
+    const float* row[kHeadsPerCta];
+    float Mj[kHeadsPerCta];
+    bool on[kHeadsPerCta];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (n0 + e >= ks.k_hi) continue;
-        float bin_f;
-        const int bin = l1_bin_f(M, s4[e], bin_f);
-        add_mass(&hist[warp][bin][0], l1_mass_arg(M, s4[e], bin_f));
+    for (int jj = 0; jj < kHeadsPerCta; ++jj) {
+      on[jj] = j0 + jj < x.nh && s_on[j0 + jj];
+      row[jj] = scores + (x.r * d.n_ret + (on[jj] ? hm.ih_heads[x.ih][j0 + jj] : 0)) * l_pad;
+      Mj[jj] = on[jj] ? s_M[j0 + jj] : 0.f;
+    }
+    for (int n0 = ks.k_lo + 4 * (int)threadIdx.x; n0 < ks.k_hi; n0 += 4 * kThreads) {
+      float4 v[kHeadsPerCta];
+#pragma unroll
+      for (int jj = 0; jj < kHeadsPerCta; ++jj) v[jj] = on[jj] ? ld_scores4(row[jj] + n0) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int jj = 0; jj < kHeadsPerCta; ++jj) {
+        if (!on[jj]) continue;   // uniform
+        const float s4[4] = {v[jj].x, v[jj].y, v[jj].z, v[jj].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (n0 + e >= ks.k_hi) continue;
+          float bin_f;
+          const int bin = l1_bin_f(Mj[jj], s4[e], bin_f);
+          add_mass(&hist[jj][warp][bin][0], l1_mass_arg(Mj[jj], s4[e], bin_f));
+        }
       }
     }
     __syncthreads();
-    if (threadIdx.x < kBins) {
+    {
+      const int jj = threadIdx.x / kBins, bin = threadIdx.x % kBins;   // 256 threads = 4 heads x 64 bins
       unsigned long long tot = 0ull;
       for (int w = 0; w < kWarps; ++w) {
-        tot += ((unsigned long long)hist[w][threadIdx.x][1] << 32) | hist[w][threadIdx.x][0];
-        hist[w][threadIdx.x][0] = 0u;
-        hist[w][threadIdx.x][1] = 0u;
+        tot += ((unsigned long long)hist[jj][w][bin][1] << 32) | hist[jj][w][bin][0];
+        hist[jj][w][bin][0] = 0u;
+        hist[jj][w][bin][1] = 0u;
       }
-      if (tot) atomicAdd(g_mass + rh * kBins + threadIdx.x, tot);
+      if (tot) atomicAdd(g_mass + (x.r * d.n_ret + hm.ih_heads[x.ih][j0 + jj]) * kBins + bin, tot);
     }
     __syncthreads();
   }
@@ -358,7 +372,7 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
           st->raw_hi = rhi;
           st->ref_s = l1_bin_hi(M, found);
           st->e_ref = fast_ex2(-kLog2eH * (0.5f * (float)found - 0.25f));
-          if (q < 0.999f * kMinQ * (float)kCandCap) st->mode = kCollect;   // fewer than kCandCap keys in the bin
+          if (q < 0.999f * kMinQ * (float)list_cap) st->mode = kCollect;   // fewer than list_cap keys in the bin
         }
       }
     }
@@ -379,7 +393,7 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
                                                            const int64_t l_pad,
                                                            SelState* __restrict__ state, unsigned long long* __restrict__ g_mass,
                                                            uint32_t* __restrict__ g_cnt, uint32_t* __restrict__ tickets,
-                                                           int n_splits, int max_levels, int32_t* status) {
+                                                           int n_splits, int max_levels, const int list_cap, int32_t* status) {
   __shared__ uint32_t hist[16][kBins][3];   // {sum, carries, count}
   __shared__ KeyParams kp[16];
   __shared__ uint32_t s_span[16];
@@ -423,16 +437,25 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
     const uint32_t base_key = kp[j].base_key, span = s_span[j];
     const int shift = kp[j].shift;
     const float ref_s = kp[j].ref_s;
-    for (int n0 = ks.k_lo + 4 * (int)threadIdx.x; n0 < ks.k_hi; n0 += 4 * kThreads) {
-      const float4 v = ld_scores4(row + n0);
-      const float s4[4] = {v.x, v.y, v.z, v.w};
+    for (int nb = ks.k_lo + 4 * (int)threadIdx.x; nb < ks.k_hi; nb += kLoads * 4 * kThreads) {
+      float4 v[kLoads];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const uint32_t t = okey(s4[e]) - base_key;
-        if (n0 + e < ks.k_hi && t < span) {
-          uint32_t* acc = &hist[j][t >> shift][0];
-          add_mass(acc, fmaf(s4[e] - ref_s, kLog2eH, 20.0f));
-          atomicAdd(acc + 2, 1u);
+      for (int k = 0; k < kLoads; ++k) {
+        const int n0 = nb + k * 4 * kThreads;
+        v[k] = n0 < ks.k_hi ? ld_scores4(row + n0) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int k = 0; k < kLoads; ++k) {
+        const int n0 = nb + k * 4 * kThreads;
+        const float s4[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t t = okey(s4[e]) - base_key;
+          if (n0 + e < ks.k_hi && t < span) {
+            uint32_t* acc = &hist[j][t >> shift][0];
+            add_mass(acc, fmaf(s4[e] - ref_s, kLog2eH, 20.0f));
+            atomicAdd(acc + 2, 1u);
+          }
         }
       }
     }
@@ -518,10 +541,10 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
         st->raw_lo = rlo;
         st->raw_hi = rhi;
         st->shift = max(0, shift - 6);
-        if (cnt <= (uint32_t)kCandCap)
+        if (cnt <= (uint32_t)list_cap)
           st->mode = kCollect;
         else if (sub_span == 1u)
-          st->mode = kTieScan;         // more than kCandCap equal scores straddle the cut
+          st->mode = kTieScan;         // more than list_cap equal scores straddle the cut
       }
       __syncwarp();
     }
@@ -544,8 +567,8 @@ constexpr int kCandStageW = 256;  // flushed when more than 128 are staged
 
 __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
     const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows, const float* __restrict__ scores,
-    const int64_t l_pad, SelState* __restrict__ state, uint2* __restrict__ cand, int32_t* __restrict__ sel_idx,
-    int64_t sel_stride, int n_splits, int32_t* status) {
+    const int64_t l_pad, SelState* __restrict__ state, uint2* __restrict__ cand, const int list_cap,
+    int32_t* __restrict__ sel_idx, int64_t sel_stride, int n_splits, int32_t* status) {
   __shared__ int id_stage[kWarps][kIdStage];
   __shared__ uint2 cand_stage[kWarps][kCandStageW];
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
@@ -580,7 +603,7 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
       if (lane == 0) gbase = atomicAdd(&st->cand_cnt, cnt_c);
       gbase = __shfl_sync(0xffffffffu, gbase, 0);
       for (int i = lane; i < cnt_c; i += 32)
-        if (gbase + i < kCandCap) cand[rh * kCandCap + gbase + i] = cand_stage[warp][i];
+        if (gbase + i < list_cap) cand[rh * (int64_t)list_cap + gbase + i] = cand_stage[warp][i];
       cnt_c = 0;
       __syncwarp();
     };
@@ -618,13 +641,14 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
 }
 
 // ---- finalize ---------------------------------------------------------------------------------------
-constexpr int kFinThreads = 256;
+constexpr int kFinThreads = 1024;
 constexpr int kFinWarps = kFinThreads / 32;
 constexpr int kNoPick = 0x7fffffff;
 
 __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
     const Dims d, const float* __restrict__ scores, const int64_t l_pad, SelState* __restrict__ state,
-    const uint2* __restrict__ cand, int32_t* __restrict__ sel_idx, int64_t sel_stride, int32_t* __restrict__ sel_count,
+    const uint2* __restrict__ cand, const int list_cap, int32_t* __restrict__ sel_idx, int64_t sel_stride,
+    int32_t* __restrict__ sel_count,
     float* __restrict__ sel_mass, float* __restrict__ sel_thresh, int32_t* __restrict__ sel_tie_last,
     int32_t* status) {
   extern __shared__ __align__(16) unsigned char fin_smem[];
@@ -666,20 +690,31 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
   int base = st->cnt_above;
   int emit_base = ids ? st->emit_cnt : base;
 
+  bool tie = mode == kTieScan;
+  uint32_t tie_key = st->lo_key;
+  int tie_bucket = st->bucket_cnt;
+  int n_fin = 0;   // candidates left for the exact sort
   if (mode == kCollect) {
-    int n = min(st->cand_cnt, kCandCap);
-    for (int i = tid; i < n; i += kFinThreads) {
-      const uint2 cnd = cand[rh * kCandCap + i];
-      keys[i] = ((unsigned long long)(~cnd.x) << 32) | (unsigned long long)cnd.y;
+    // The candidates of the bucket: a list in global memory (up to list_cap entries).  A list that fits is copied to
+    // shared memory at once; a longer one is narrowed where it is until the chosen part fits.
+    const uint2* gl = cand + rh * (int64_t)list_cap;
+    const int n_src = min(st->cand_cnt, list_cap);
+    bool in_global = n_src > kCandCap;
+    int n = n_src;   // candidates inside [lo_key, lo_key + span)
+    if (!in_global) {
+      for (int i = tid; i < n; i += kFinThreads) {
+        const uint2 cnd = gl[i];
+        keys[i] = ((unsigned long long)(~cnd.x) << 32) | (unsigned long long)cnd.y;
+      }
     }
     __syncthreads();
     // Narrowing: while many candidates are left, one more 64-bin mass histogram over the next six key bits of the
-    // bucket, now on the candidate list in shared memory: candidates above the chosen bin are selected (and their
-    // ids emitted), those below are dropped, those inside go on.  The exact sort below then sees a short list.
+    // bucket on the candidate list: candidates above the chosen bin are selected (and their ids emitted), those below
+    // are dropped, those inside go on.  The exact sort below then sees a short list.
     {
       uint32_t lo_key = st->lo_key, span = st->span;
       const float ref_s = st->ref_s, sc = st->e_ref * 9.5367431640625e-07f;   // 2^-20
-      while (n > 256 && span > 1u) {
+      while ((n > 256 || in_global) && span > 1u) {
         const int bits = 32 - __clz(span - 1u);
         const int shift = max(0, bits - 6);
         for (int i = tid; i < kBins * 3; i += kFinThreads) (&fh[0][0])[i] = 0u;
@@ -688,11 +723,23 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
           s_sel = 0;
         }
         __syncthreads();
-        for (int i = tid; i < n; i += kFinThreads) {
-          const uint32_t key = ~(uint32_t)(keys[i] >> 32);
-          uint32_t* acc = &fh[(key - lo_key) >> shift][0];
-          add_mass(acc, fmaf(okey_to_float(key) - ref_s, kLog2eH, 20.0f));
-          atomicAdd(acc + 2, 1u);
+        if (in_global) {
+          for (int i = tid; i < n_src; i += kFinThreads) {
+            const uint32_t key = __ldcg(&gl[i].x);
+            const uint32_t t = key - lo_key;
+            if (t < span) {
+              uint32_t* acc = &fh[t >> shift][0];
+              add_mass(acc, fmaf(okey_to_float(key) - ref_s, kLog2eH, 20.0f));
+              atomicAdd(acc + 2, 1u);
+            }
+          }
+        } else {
+          for (int i = tid; i < n; i += kFinThreads) {
+            const uint32_t key = ~(uint32_t)(keys[i] >> 32);
+            uint32_t* acc = &fh[(key - lo_key) >> shift][0];
+            add_mass(acc, fmaf(okey_to_float(key) - ref_s, kLog2eH, 20.0f));
+            atomicAdd(acc + 2, 1u);
+          }
         }
         __syncthreads();
         if (warp == 0) {   // lane l looks at bins 63 - 2l, 62 - 2l (bin 63 is the top)
@@ -728,30 +775,60 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
         }
         __syncthreads();
         const int bin = s_bin;
-        for (int i = tid; i < n; i += kFinThreads) {
-          const unsigned long long k = keys[i];
-          const int b = (int)((~(uint32_t)(k >> 32) - lo_key) >> shift);
-          if (b > bin) {
-            const int pos = atomicAdd(&s_sel, 1);
-            if (ids && emit_base + pos < sel_stride) ids[emit_base + pos] = (int)(uint32_t)k;
-          } else if (b == bin) {
-            keys2[atomicAdd(&s_n2, 1)] = k;
+        const int cnt_bin = (int)fh[bin][2];
+        const bool to_smem = in_global && cnt_bin <= kCandCap;
+        if (in_global) {
+          for (int i = tid; i < n_src; i += kFinThreads) {
+            const uint2 cnd = __ldcg(&gl[i]);
+            const uint32_t t = cnd.x - lo_key;
+            if (t < span) {
+              const int b = (int)(t >> shift);
+              if (b > bin) {
+                const int pos = atomicAdd(&s_sel, 1);
+                if (ids && emit_base + pos < sel_stride) ids[emit_base + pos] = (int)cnd.y;
+              } else if (b == bin && to_smem) {
+                keys2[atomicAdd(&s_n2, 1)] = ((unsigned long long)(~cnd.x) << 32) | (unsigned long long)cnd.y;
+              }
+            }
+          }
+        } else {
+          for (int i = tid; i < n; i += kFinThreads) {
+            const unsigned long long k = keys[i];
+            const int b = (int)((~(uint32_t)(k >> 32) - lo_key) >> shift);
+            if (b > bin) {
+              const int pos = atomicAdd(&s_sel, 1);
+              if (ids && emit_base + pos < sel_stride) ids[emit_base + pos] = (int)(uint32_t)k;
+            } else if (b == bin) {
+              keys2[atomicAdd(&s_n2, 1)] = k;
+            }
           }
         }
         __syncthreads();
         above = s_above;
         base += s_sel;
         emit_base += s_sel;
-        n = s_n2;
+        n = cnt_bin;
         const uint32_t ofs = (uint32_t)bin << shift;
         lo_key += ofs;
         span = min(1u << shift, span - ofs);
-        unsigned long long* t = keys;
-        keys = keys2;
-        keys2 = t;
+        if (!in_global || to_smem) {
+          unsigned long long* t = keys;
+          keys = keys2;
+          keys2 = t;
+          in_global = false;
+        }
         __syncthreads();
       }
+      if (in_global) {   // one key value with more candidates than the sort takes: exact ties
+        tie = true;
+        tie_key = lo_key;
+        tie_bucket = n;
+      }
     }
+    n_fin = n;
+  }
+  if (mode == kCollect && !tie) {
+    const int n = n_fin;
     int np = 1;
     while (np < n) np <<= 1;
     for (int i = n + tid; i < np; i += kFinThreads) keys[i] = ~0ull;
@@ -827,13 +904,13 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
     return;
   }
 
-  if (mode == kTieScan) {
+  if (tie) {
     // More than kCandCap keys share the threshold score exactly: take the first c of them in
     // position order, c = the number of equal masses still needed.
-    const uint32_t t_key = st->lo_key;
+    const uint32_t t_key = tie_key;
     const float e_t = __expf(okey_to_float(t_key) - M);
     int c = (int)ceilf((target - above) / e_t);
-    c = max(1, min(c, st->bucket_cnt));
+    c = max(1, min(c, tie_bucket));
     const float* row = scores + rh * l_pad;
     if (tid == 0) {
       s_emitted = 0;
@@ -918,6 +995,9 @@ struct SelWorkspace {
   size_t bytes;
 };
 
+constexpr int kListCap = 65536;   // candidates per (row, head) kept in global memory (never more than the padded length)
+int list_capacity(int64_t l_pad) { return (int)(l_pad < kListCap ? l_pad : kListCap); }
+
 SelWorkspace carve(void* ws, int64_t n_rowheads, int64_t n_units, int64_t l_pad) {
   SelWorkspace w;
   size_t off = 0;
@@ -930,7 +1010,7 @@ SelWorkspace carve(void* ws, int64_t n_rowheads, int64_t n_units, int64_t l_pad)
   const size_t o_mass = take(sizeof(unsigned long long) * kBins * n_rowheads);
   const size_t o_cnt = take(sizeof(uint32_t) * kBins * n_rowheads);
   const size_t o_tick = take(sizeof(uint32_t) * n_units);
-  const size_t o_cand = take(sizeof(uint2) * kCandCap * n_rowheads);
+  const size_t o_cand = take(sizeof(uint2) * (size_t)list_capacity(l_pad) * n_rowheads);
   const size_t o_scores = take(sizeof(float) * (size_t)l_pad * n_rowheads);
   char* b = reinterpret_cast<char*>(ws);
   w.state = reinterpret_cast<SelState*>(b + o_state);
@@ -964,6 +1044,7 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
   const int64_t nrh = rows.R * d.n_ret;
   const int64_t l_pad = padded_len(max_len);
   const SelWorkspace w = carve(ws, nrh, rows.R * d.n_ih, l_pad);
+  const int list_cap = list_capacity(l_pad);
   cudaError_t e = cudaSuccess;
   {
     const int64_t n_zero = (int64_t)(w.zero_bytes / 4);
@@ -982,13 +1063,13 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
     sel_score_kernel<true><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status);
   else
     sel_score_kernel<false><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status);
-  sel_l1_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.tickets, n_splits, status);
+  sel_l1_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.tickets, n_splits, list_cap, status);
   sel_key_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.g_cnt, w.tickets,
-                                            n_splits, 1 + kKeyLevels, status);
+                                            n_splits, 1 + kKeyLevels, list_cap, status);
   {
     const dim3 grid3((unsigned)(rows.R * d.n_ih), n_splits, (max_nh + kHeadsPerCta - 1) / kHeadsPerCta);
-    sel_compact_kernel<<<grid3, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.cand, sel_idx, sel_stride,
-                                                   n_splits, status);
+    sel_compact_kernel<<<grid3, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.cand, list_cap, sel_idx,
+                                                   sel_stride, n_splits, status);
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -996,7 +1077,7 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
   static PerDeviceOnce fin_once;
   e = set_dyn_smem_once(sel_finalize_kernel, kFinSmem, fin_once);
   if (e != cudaSuccess) return e;
-  sel_finalize_kernel<<<(unsigned)nrh, kFinThreads, kFinSmem, st>>>(d, w.scores, l_pad, w.state, w.cand, sel_idx, sel_stride,
+  sel_finalize_kernel<<<(unsigned)nrh, kFinThreads, kFinSmem, st>>>(d, w.scores, l_pad, w.state, w.cand, list_cap, sel_idx, sel_stride,
                                                              sel_count, sel_mass, sel_thresh, sel_tie_last, status);
   return cudaGetLastError();
 }
