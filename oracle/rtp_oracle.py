@@ -20,6 +20,11 @@ What it follows
                          softmax mass reaches p.  Token level (Section 3 speaks
                          of token-level sparse computation; the 64-token blocks
                          of Section 3.4 are a kernel approximation).
+* ``block_lse`` / ``topp_select_blocks``
+                         Section 3.4, the block-wise form of Eq. 5: the keys are
+                         cut into blocks of 64, every block is reduced to a
+                         log-sum-exp pair (m_b, l_b), blocks are taken in order
+                         of decreasing m_b until their softmax mass reaches p.
 * ``attention_over_set`` Eq. 5, softmax(q.k/sqrt(d_h)) restricted to S, times V.
 * ``local_set``          Section 3.2 / Table 2: attention sinks plus a sliding
                          window on local heads.
@@ -30,14 +35,19 @@ Readings taken where the paper is silent (each also listed in the design notes):
 no extra scale inside the top-p softmax; ties broken towards the smaller token
 index; p = 1 keeps every causal key; the selection is never empty; sinks, the
 recent window and the query's own position are NOT forced into a retrieval
-head's set; a query at position m sees keys 0..m; the window is the last W
+head's set; the block-wise selection orders blocks by their maximum score m_b
+(the quantity the kernel of Section 3.4 indexes its histogram by), exactly
+rather than through 256 bins, with ties towards the smaller block index, and
+a block's mass is l_b exp(m_b - M) / Z; a query at position m sees keys 0..m; the window is the last W
 positions including m; query head h reads KV head h // G.
 
 Pins (tests/test_oracle_*.py): brute force over all subsets for tiny L, closed
 forms (equal scores, geometric scores, one dominant score, Gaussian scores),
 shift / permutation / monotonicity invariants, dense attention against
 torch's scaled_dot_product_attention, boolean-mask SDPA for the local pattern,
-and the matrix-product identity for the indexer.  The selection statistics the
+the matrix-product identity for the indexer; for the block-wise selection:
+equal blocks, one dominant block, block size 1 against the token-level rule,
+brute force over all block subsets in m_b order.  The selection statistics the
 paper prints (its Tables 1, 6, 7) depend on model activations that are not
 available: parity unpinned for those numbers; they only shape synthetic data.
 
@@ -148,6 +158,72 @@ def set_mass(s: np.ndarray, ids) -> float:
     """Softmax mass (over the whole row) carried by the tokens ``ids``."""
     _, _, P = softmax_mass(s)
     return float(np.sum(P[np.asarray(sorted(ids), dtype=np.int64)]))
+
+
+# ---------------------------------------------------------------- block-wise top-p (Section 3.4)
+def block_lse(s: np.ndarray, block: int = 64):
+    """Per-block log-sum-exp pairs of one row's scores (Section 3.4): block b holds keys
+    b*block .. min((b+1)*block, n) - 1; m_b is its largest score (as fp32) and
+    l_b = sum exp(s - m_b) over its keys (fp64)."""
+    s = np.asarray(s, dtype=np.float32)
+    n = s.shape[0]
+    if n == 0:
+        raise ValueError("empty row")
+    n_b = (n + block - 1) // block
+    m = np.empty(n_b, dtype=np.float32)
+    l = np.empty(n_b, dtype=np.float64)
+    for b in range(n_b):
+        blk = s[b * block: (b + 1) * block].astype(np.float64)
+        m[b] = np.float32(blk.max())
+        l[b] = np.sum(np.exp(blk - float(m[b])))
+    return m, l
+
+
+def topp_select_blocks(s: np.ndarray, p: float, block: int = 64):
+    """Block-wise Top-P of Section 3.4 on the fp32 scores of one query row.
+
+    Blocks are ordered by decreasing m_b (equal maxima: smaller block first); the
+    selection is the shortest prefix of that order whose mass, sum of
+    l_b exp(m_b - M) / Z, reaches p; p >= 1 keeps every block.  Returns
+    (selected block ids ascending, their number, mass of the selection, m_b of the
+    last block taken, order, cumulative mass along the order)."""
+    if not (p > 0.0):
+        raise ValueError("top_p must be in (0, 1]")
+    m, l = block_lse(s, block)
+    M = float(m.max())
+    w = l * np.exp(m.astype(np.float64) - M)
+    P = w / float(np.sum(w))
+    order = np.argsort(-m.astype(np.float64), kind="stable")
+    cum = np.cumsum(P[order])
+    n_b = m.shape[0]
+    if p >= 1.0:
+        k_star = n_b
+    else:
+        hit = np.nonzero(cum >= p)[0]
+        k_star = int(hit[0]) + 1 if hit.size else n_b
+    ids = np.sort(order[:k_star])
+    return ids, k_star, float(cum[k_star - 1]), float(m[order[k_star - 1]]), order, cum
+
+
+def classify_blocks_against_band(s: np.ndarray, p: float, block: int = 64, band: float = 1e-4):
+    """Mandatory / forbidden blocks for comparing a block selection made with fp32 mass
+    sums: a block whose cumulative mass before its own inclusion lies within ``band`` of p
+    may go either way."""
+    ids, k_star, mass, thr, order, cum = topp_select_blocks(s, p, block)
+    before = np.concatenate([[0.0], cum[:-1]])
+    mandatory = order[before < p - band]
+    forbidden = order[before >= p + band]
+    if p >= 1.0:
+        mandatory, forbidden = order, order[:0]
+    return set(mandatory.tolist()), set(forbidden.tolist())
+
+
+def block_token_set(block_ids, m: int, block: int = 64) -> np.ndarray:
+    """Token positions 0..m covered by the given blocks."""
+    n = np.arange(m + 1, dtype=np.int64)
+    keep = np.zeros((m + block) // block + 1, dtype=bool)
+    keep[np.asarray(sorted(block_ids), dtype=np.int64)] = True
+    return n[keep[n // block]]
 
 
 # ---------------------------------------------------------------- token sets
