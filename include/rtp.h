@@ -284,6 +284,40 @@ rtp_status rtp_sparse_attn_prefill(rtp_ctx* ctx, const rtp_params* params, const
                                    void* workspace, size_t workspace_bytes, int32_t* status,
                                    void* stream);
 
+
+/* ---- NEXT: block-wise top-p for prefill (Section 3.4) --------------------------------------------
+ * The paper's kernel selects whole blocks of 64 keys rather than single tokens: every block of a row's indexer
+ * scores is reduced to a log-sum-exp pair (m_b, l_b); blocks are taken in order of decreasing m_b (equal maxima:
+ * the smaller block first) until their softmax mass, sum of l_b exp(m_b - M) / Z, reaches top_p.  Here a block is
+ * one cache page, the order is exact (the paper deposits the pairs in a 256-bin histogram indexed by m_b; this
+ * library resolves the bin in which the mass is reached down to single blocks), and the result is a bit per page.
+ *
+ * rtp_topp_select_blocks: rows are the C positions q_start .. q_start + C - 1 of sequence seq_id (a prefill chunk;
+ * the chunk's index keys must have been appended).  q_pre: bf16 [C, n_q_heads, 128] device; w_q as in
+ * rtp_topp_select.
+ *   block_mask   uint32 [C, n_ret_q_heads, mask_words] device, written: bit (b & 31) of word b >> 5 of a row is set
+ *                iff block b (keys 64 b .. 64 b + 63, cut at the row's own position) is selected.  Words beyond the
+ *                row's last block are not written.  mask_words * 32 must cover ceil((q_start + C) / 64) blocks.
+ *   sel_count    int32 [C, n_ret_q_heads]: number of selected blocks; sel_mass (may be NULL): their softmax mass;
+ *   sel_thresh   (may be NULL): m_b of the last block taken (-inf when every block is taken);
+ *   sel_tie_last (may be NULL): index of that block.
+ *   workspace    device scratch of rtp_block_workspace_bytes(params, C, q_start + C) bytes.
+ * Errors as rtp_topp_select; RTP_ERR_CAPACITY when mask_words or the workspace is too small.
+ *
+ * rtp_sparse_attn_prefill_blocks: exact attention of the retrieval heads' rows of the chunk over the keys of their
+ * selected blocks (causal inside the row's last block); q: bf16 [C, n_q_heads, 128] post-RoPE; out / lse as
+ * rtp_sparse_attn_prefill (retrieval heads' slots only).  Like the token-level call it needs every index head to
+ * serve the whole query-head group of its KV head. */
+size_t rtp_block_workspace_bytes(const rtp_params* params, int64_t rows, int64_t max_seq_len);
+rtp_status rtp_topp_select_blocks(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q_pre,
+                                  const void* w_q, int32_t seq_id, int32_t q_start, int64_t C, uint32_t* block_mask,
+                                  int64_t mask_words, int32_t* sel_count, float* sel_mass, float* sel_thresh,
+                                  int32_t* sel_tie_last, int32_t* status, void* workspace, size_t workspace_bytes,
+                                  void* stream);
+rtp_status rtp_sparse_attn_prefill_blocks(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q,
+                                          int32_t seq_id, int32_t q_start, int64_t C, const uint32_t* block_mask,
+                                          int64_t mask_words, void* out, float* lse, int32_t* status, void* stream);
+
 /* ---- S7: local heads, attention sinks + sliding window (Section 3.2, Table 2) -
  * Row at position m attends to {n <= m : n < n_sink or n > m - window}.
  * Rows as in rtp_topp_select (row arrays = decode path with split-KV; NULL

@@ -23,6 +23,7 @@ EXPORTS = [
     "rtp_version", "rtp_create", "rtp_destroy", "rtp_last_error", "rtp_debug_wait_test", "rtp_workspace_bytes", "rtp_check_status",
     "rtp_kv_append", "rtp_index_keys", "rtp_index_queries", "rtp_index_score", "rtp_topp_select", "rtp_sparse_attn_decode", "rtp_sparse_attn_decode_static",
     "rtp_sparse_attn_prefill", "rtp_local_attn", "rtp_dense_attn_prefill", "rtp_dense_attn_decode",
+    "rtp_block_workspace_bytes", "rtp_topp_select_blocks", "rtp_sparse_attn_prefill_blocks",
 ]
 
 
@@ -96,6 +97,12 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.rtp_sparse_attn_prefill.restype = i32
     lib.rtp_sparse_attn_prefill.argtypes = [vp, PP, PC, vp, vp, vp, i32, i32, i64, vp, i64, vp, vp, vp, vp, vp, vp,
                                             sz, vp, vp]
+    lib.rtp_block_workspace_bytes.restype = sz
+    lib.rtp_block_workspace_bytes.argtypes = [PP, i64, i64]
+    lib.rtp_topp_select_blocks.restype = i32
+    lib.rtp_topp_select_blocks.argtypes = [vp, PP, PC, vp, vp, i32, i32, i64, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.rtp_sparse_attn_prefill_blocks.restype = i32
+    lib.rtp_sparse_attn_prefill_blocks.argtypes = [vp, PP, PC, vp, i32, i32, i64, vp, i64, vp, vp, vp, vp]
     lib.rtp_local_attn.restype = i32
     lib.rtp_local_attn.argtypes = [vp, PP, PC, vp, vp, vp, i32, i32, i64, vp, vp, vp, sz, vp, vp]
     lib.rtp_dense_attn_prefill.restype = i32
@@ -282,6 +289,29 @@ def rtp_sparse_attn_prefill(ctx, params, cache, q, q_pre, w_q, seq_id, q_start, 
                                                _ptr(lse), _ptr(workspace),
                                                int(workspace.numel() * workspace.element_size()), _ptr(status),
                                                _stream(stream)), "rtp_sparse_attn_prefill")
+
+
+def rtp_block_workspace_bytes(params: Params, rows: int, max_seq_len: int) -> int:
+    return int(load_library().rtp_block_workspace_bytes(params.ref(), rows, max_seq_len))
+
+
+def rtp_topp_select_blocks(ctx, params, cache, q_pre, w_q, seq_id, q_start, n_rows, block_mask, sel_count, sel_mass,
+                           sel_thresh, sel_tie_last, status, workspace, stream=None):
+    """block_mask: int32 / uint32 tensor [n_rows, n_ret, mask_words]."""
+    ctx._check(ctx.lib.rtp_topp_select_blocks(ctx.h, params.ref(), C.byref(cache), _ptr(q_pre), _ptr(w_q), int(seq_id),
+                                              int(q_start), int(n_rows), _ptr(block_mask), int(block_mask.shape[-1]),
+                                              _ptr(sel_count), _ptr(sel_mass), _ptr(sel_thresh), _ptr(sel_tie_last),
+                                              _ptr(status), _ptr(workspace),
+                                              int(workspace.numel() * workspace.element_size()), _stream(stream)),
+               "rtp_topp_select_blocks")
+
+
+def rtp_sparse_attn_prefill_blocks(ctx, params, cache, q, seq_id, q_start, n_rows, block_mask, out, lse, status,
+                                   stream=None):
+    ctx._check(ctx.lib.rtp_sparse_attn_prefill_blocks(ctx.h, params.ref(), C.byref(cache), _ptr(q), int(seq_id),
+                                                      int(q_start), int(n_rows), _ptr(block_mask),
+                                                      int(block_mask.shape[-1]), _ptr(out), _ptr(lse), _ptr(status),
+                                                      _stream(stream)), "rtp_sparse_attn_prefill_blocks")
 
 
 def rtp_local_attn(ctx, params, cache, q, row_seq, row_pos, seq_id, q_start, n_rows, out, lse, workspace, status,

@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const CacheView cv, const Dims d, const HeadMaps hm, const __nv_bfloat16* __restrict__ q,
     const __nv_bfloat16* __restrict__ qt, const float* __restrict__ sel_thresh, const int32_t* __restrict__ sel_tie_last,
     const int seq_id, const int q_start, const int C, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
-    int32_t* status, const int n_row_tiles) {
+    int32_t* status, const int n_row_tiles, const uint32_t* __restrict__ blk_mask, const int64_t mask_words) {
   constexpr int BMP = kBM / G;
   extern __shared__ __align__(1024) unsigned char smem[];
   const uint32_t sbase = s_u32(smem);
@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile = n_row_tiles - 1 - blockIdx.x;
-  const int kvh = (MODE == kPrefillSparse) ? hm.ih_kv[blockIdx.y] : hm.kv_list[blockIdx.y];
+  const int kvh = (MODE == kPrefillSparse || MODE == kPrefillBlocks) ? hm.ih_kv[blockIdx.y] : hm.kv_list[blockIdx.y];
   const int r0 = tile * BMP, m0 = q_start + r0;
   const int rows_here = min(BMP, C - r0);
   const int m_last = m0 + rows_here - 1;
@@ -268,7 +268,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     // float above up, so that raw > up <=> raw >= upn.  The per-row values live in shared memory (the region the
     // final merge reuses) and are re-read for every tile, like the projected-query fragments (from global
     // memory): nothing of the rule stays in registers across the softmax of a tile.
-    const int ih = (MODE == kPrefillSparse) ? blockIdx.y : 0;
+    const int ih = (MODE == kPrefillSparse || MODE == kPrefillBlocks) ? blockIdx.y : 0;
+    // block mode: the row's page bits (one word per 32 pages)
+    const uint32_t* mrow = (MODE == kPrefillBlocks && row_ok) ? blk_mask + ((int64_t)(r0 + po) * d.n_ret + hm.ih_heads[ih][hs]) * mask_words : nullptr;
     const int gq = lane >> 2, cq = lane & 3;
     float* thr_lo = xch;                                      // [128 rows]
     float* thr_upn = xch + 256;
@@ -416,6 +418,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
           my[c] = kk == 0 ? v0 : kk == 1 ? v1 : kk == 2 ? v2 : v3;
         }
       }
+      uint32_t page_bits = 3u;   // block mode: bit 0 / 1 = the tile's first / second page is selected by the row
+      if (MODE == kPrefillBlocks) {
+        const int pg = 2 * (n_base / kBNt);
+        page_bits = mrow ? (__ldg(mrow + (pg >> 5)) >> (pg & 31)) & 3u : 0u;
+      }
       mbar_wait(bar(kSFull0 + grp), n_mine & 1, abort_flag, status, d.wait_ns);
       tc_fence_after();
       float s[kBNt];
@@ -432,6 +439,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 #pragma unroll
         for (int i = 0; i < kBNt; ++i)
           if ((my[(i & 7) >> 1] >> (31 - (2 * (i >> 3) + (i & 1)))) & 1u) s[i] = -INFINITY;
+      }
+      if (MODE == kPrefillBlocks) {
+        if (!(page_bits & 1u)) {
+#pragma unroll
+          for (int i = 0; i < kPage; ++i) s[i] = -INFINITY;
+        }
+        if (!(page_bits & 2u)) {
+#pragma unroll
+          for (int i = kPage; i < kBNt; ++i) s[i] = -INFINITY;
+        }
       }
       bool need_mask = n_base + kBNt - 1 > pos;
       if (MODE == kPrefillLocal) need_mask = need_mask || (n_base <= pos - d.window);
@@ -577,7 +594,8 @@ template <int G, int MODE>
 cudaError_t launch_tc_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm, const __nv_bfloat16* q,
                             const __nv_bfloat16* qt, const float* sel_thresh, const int32_t* sel_tie_last,
                             int32_t seq_id, int32_t q_start, int64_t C, __nv_bfloat16* out, float* lse,
-                            int32_t* status, int n_units, cudaStream_t st) {
+                            int32_t* status, int n_units, cudaStream_t st, const uint32_t* blk_mask = nullptr,
+                            int64_t mask_words = 0) {
   static PerDeviceOnce once;
   if (cudaError_t e0 = set_dyn_smem_once(attn_prefill_tc_kernel<G, MODE>, kTcSmem, once)) return e0;
   CUtensorMap map_k, map_v;
@@ -590,7 +608,8 @@ cudaError_t launch_tc_typed(const CacheView& cv, const Dims& d, const HeadMaps& 
   const int n_row_tiles = (int)((C + BMP - 1) / BMP);
   dim3 grid(n_row_tiles, n_units);
   attn_prefill_tc_kernel<G, MODE><<<grid, kTcThreads, kTcSmem, st>>>(map_k, map_v, cv, d, hm, q, qt, sel_thresh, sel_tie_last,
-                                                                     seq_id, q_start, (int)C, out, lse, status, n_row_tiles);
+                                                                     seq_id, q_start, (int)C, out, lse, status, n_row_tiles, blk_mask,
+                                                                     mask_words);
   return cudaGetLastError();
 }
 
@@ -598,12 +617,12 @@ template <int MODE>
 cudaError_t launch_tc_mode(const CacheView& cv, const Dims& d, const HeadMaps& hm, const __nv_bfloat16* q,
                            const __nv_bfloat16* qt, const float* sel_thresh, const int32_t* sel_tie_last,
                            int32_t seq_id, int32_t q_start, int64_t C, __nv_bfloat16* out, float* lse, int32_t* status,
-                           int n_units, cudaStream_t st) {
+                           int n_units, cudaStream_t st, const uint32_t* blk_mask = nullptr, int64_t mask_words = 0) {
   switch (d.group) {
-    case 1: return launch_tc_typed<1, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st);
-    case 2: return launch_tc_typed<2, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st);
-    case 4: return launch_tc_typed<4, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st);
-    case 8: return launch_tc_typed<8, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st);
+    case 1: return launch_tc_typed<1, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st, blk_mask, mask_words);
+    case 2: return launch_tc_typed<2, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st, blk_mask, mask_words);
+    case 4: return launch_tc_typed<4, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st, blk_mask, mask_words);
+    case 8: return launch_tc_typed<8, MODE>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, n_units, st, blk_mask, mask_words);
     default: return cudaErrorNotSupported;
   }
 }
@@ -615,8 +634,13 @@ cudaError_t launch_tc_mode(const CacheView& cv, const Dims& d, const HeadMaps& h
 cudaError_t launch_attn_prefill_tc(const CacheView& cv, const Dims& d, const HeadMaps& hm, int mode,
                                    const __nv_bfloat16* q, const __nv_bfloat16* qt, const float* sel_thresh,
                                    const int32_t* sel_tie_last, int32_t seq_id, int32_t q_start, int64_t C,
-                                   __nv_bfloat16* out, float* lse, int32_t* status, cudaStream_t st) {
+                                   __nv_bfloat16* out, float* lse, int32_t* status, cudaStream_t st,
+                                   const uint32_t* blk_mask, int64_t mask_words) {
   if (C == 0) return cudaSuccess;
+  if (mode == kPrefillBlocks)
+    return d.n_ih == 0 ? cudaSuccess
+                       : launch_tc_mode<kPrefillBlocks>(cv, d, hm, q, nullptr, nullptr, nullptr, seq_id, q_start, C, out, lse,
+                                                        status, d.n_ih, st, blk_mask, mask_words);
   if (mode == kPrefillSparse)
     return d.n_ih == 0 ? cudaSuccess
                        : launch_tc_mode<kPrefillSparse>(cv, d, hm, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out,
@@ -635,19 +659,21 @@ cudaError_t launch_attn_prefill_tc(const CacheView& cv, const Dims& d, const Hea
 cudaError_t launch_attn_prefill(const CacheView& cv, const Dims& d, const HeadMaps& hm, int mode,
                                 const __nv_bfloat16* q, const __nv_bfloat16* qt, int32_t seq_id, int32_t q_start,
                                 int64_t C, const float* sel_thresh, const int32_t* sel_tie_last,
-                                __nv_bfloat16* out, float* lse, int32_t* status, int sm_count, cudaStream_t st) {
+                                __nv_bfloat16* out, float* lse, int32_t* status, int sm_count, cudaStream_t st,
+                                const uint32_t* blk_mask, int64_t mask_words) {
   (void)sm_count;
   if (C == 0) return cudaSuccess;
-  if (mode == kPrefillSparse) {
+  if (mode == kPrefillSparse || mode == kPrefillBlocks) {
     // one CTA column per index head; every query head of its KV head must be a retrieval head on it
     for (int j = 0; j < d.n_ih; ++j)
       if (hm.ih_nheads[j] != d.group) return cudaErrorNotSupported;
     for (int i = 0; i < d.n_ret; ++i)
       if (hm.ret_q_head[i] != hm.ih_kv[hm.q2ih[i]] * d.group + hm.slot_in_ih[i]) return cudaErrorNotSupported;
-    return launch_attn_prefill_tc(cv, d, hm, mode, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, st);
+    return launch_attn_prefill_tc(cv, d, hm, mode, q, qt, sel_thresh, sel_tie_last, seq_id, q_start, C, out, lse, status, st,
+                                  blk_mask, mask_words);
   }
   if (hm.n_kv_list == 0) return cudaSuccess;
-  return launch_attn_prefill_tc(cv, d, hm, mode, q, nullptr, nullptr, nullptr, seq_id, q_start, C, out, lse, status, st);
+  return launch_attn_prefill_tc(cv, d, hm, mode, q, nullptr, nullptr, nullptr, seq_id, q_start, C, out, lse, status, st, nullptr, 0);
 }
 
 }  // namespace rtp

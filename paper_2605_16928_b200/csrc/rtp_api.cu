@@ -407,6 +407,61 @@ rtp_status rtp_sparse_attn_prefill(rtp_ctx* ctx, const rtp_params* params, const
   return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_sparse_attn_prefill");
 }
 
+size_t rtp_block_workspace_bytes(const rtp_params* params, int64_t rows, int64_t max_seq_len) {
+  Dims d;
+  HeadMaps hm;
+  if (check_params(params, &d, &hm) || rows <= 0 || max_seq_len <= 0) return 0;
+  WsCarver w(nullptr);
+  w.take(qt_bytes(d, rows));
+  w.take(select_blocks_workspace_bytes(d, hm, rows, max_seq_len, current_sm_count(kFallbackSm)));
+  return w.off;
+}
+
+rtp_status rtp_topp_select_blocks(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q_pre,
+                                  const void* w_q, int32_t seq_id, int32_t q_start, int64_t C, uint32_t* block_mask,
+                                  int64_t mask_words, int32_t* sel_count, float* sel_mass, float* sel_thresh,
+                                  int32_t* sel_tie_last, int32_t* status, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+  RTP_COMMON_PROLOGUE(false, true)
+  Rows rows;
+  int64_t max_len = 0;
+  if (const char* m = check_rows(nullptr, nullptr, seq_id, q_start, C, cache, &rows, &max_len)) return fail(ctx, RTP_ERR_INVALID, m);
+  if (C == 0 || d.n_ret == 0) return RTP_OK;
+  if (!q_pre || !w_q || !workspace || !sel_count || !block_mask) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
+  if (!aligned16(q_pre) || !aligned16(w_q) || !aligned16(workspace)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
+  if (mask_words * 32 < ((int64_t)q_start + C + kPage - 1) / kPage) return fail(ctx, RTP_ERR_CAPACITY, "mask_words too small for the chunk's pages");
+  WsCarver w(workspace);
+  __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(w.take(qt_bytes(d, C)));
+  const size_t sel_off = w.off;
+  void* sel_ws = w.take(select_blocks_workspace_bytes(d, hm, C, (int64_t)q_start + C, ctx->sm_count));
+  if (w.off > workspace_bytes) return fail(ctx, RTP_ERR_CAPACITY, "workspace too small");
+  cudaError_t e = launch_index_queries(d, hm, reinterpret_cast<const __nv_bfloat16*>(q_pre),
+                                       reinterpret_cast<const __nv_bfloat16*>(w_q), C, qt, st);
+  if (e == cudaSuccess)
+    e = launch_select_blocks(cv, d, hm, rows, qt, block_mask, mask_words, sel_count, sel_mass, sel_thresh, sel_tie_last,
+                             status, sel_ws, workspace_bytes - sel_off, ctx->sm_count, st);
+  if (e == cudaErrorNotSupported) return fail(ctx, RTP_ERR_UNSUPPORTED, "not implemented in this build");
+  return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_topp_select_blocks");
+}
+
+rtp_status rtp_sparse_attn_prefill_blocks(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q,
+                                          int32_t seq_id, int32_t q_start, int64_t C, const uint32_t* block_mask,
+                                          int64_t mask_words, void* out, float* lse, int32_t* status, void* stream) {
+  RTP_COMMON_PROLOGUE(true, false)
+  Rows rows;
+  int64_t max_len = 0;
+  if (const char* m = check_rows(nullptr, nullptr, seq_id, q_start, C, cache, &rows, &max_len)) return fail(ctx, RTP_ERR_INVALID, m);
+  if (C == 0 || d.n_ret == 0) return RTP_OK;
+  if (!q || !out || !block_mask) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
+  if (!aligned16(q) || !aligned16(out)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
+  if (mask_words * 32 < ((int64_t)q_start + C + kPage - 1) / kPage) return fail(ctx, RTP_ERR_INVALID, "mask_words too small for the chunk's pages");
+  cudaError_t e = launch_attn_prefill(cv, d, hm, kPrefillBlocks, reinterpret_cast<const __nv_bfloat16*>(q), nullptr, seq_id,
+                                      q_start, C, nullptr, nullptr, reinterpret_cast<__nv_bfloat16*>(out), lse, status,
+                                      ctx->sm_count, st, block_mask, mask_words);
+  if (e == cudaErrorNotSupported) return fail(ctx, RTP_ERR_UNSUPPORTED, "not implemented in this build");
+  return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_sparse_attn_prefill_blocks");
+}
+
 rtp_status rtp_local_attn(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q,
                           const int32_t* row_seq, const int32_t* row_pos, int32_t seq_id, int32_t q_start, int64_t R,
                           void* out, float* lse, void* workspace, size_t workspace_bytes, int32_t* status,

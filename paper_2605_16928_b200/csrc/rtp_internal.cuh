@@ -170,15 +170,24 @@ cudaError_t launch_attn_rows_static(const CacheView& cv, const Dims& d, const He
                                     const int32_t* sel_count, __nv_bfloat16* out, float* lse, int64_t max_len,
                                     int32_t* status, int sm_count, size_t* needed_bytes, cudaStream_t st);
 
-enum PrefillMode { kPrefillDense = 0, kPrefillLocal = 1, kPrefillSparse = 2 };
+enum PrefillMode { kPrefillDense = 0, kPrefillLocal = 1, kPrefillSparse = 2, kPrefillBlocks = 3 };
 cudaError_t launch_attn_prefill(const CacheView& cv, const Dims& d, const HeadMaps& hm, int mode,
                                 const __nv_bfloat16* q, const __nv_bfloat16* qt, int32_t seq_id, int32_t q_start,
                                 int64_t C, const float* sel_thresh, const int32_t* sel_tie_last,
-                                __nv_bfloat16* out, float* lse, int32_t* status, int sm_count, cudaStream_t st);
+                                __nv_bfloat16* out, float* lse, int32_t* status, int sm_count, cudaStream_t st,
+                                const uint32_t* blk_mask = nullptr, int64_t mask_words = 0);
 
 cudaError_t launch_attn_prefill_tc(const CacheView& cv, const Dims& d, const HeadMaps& hm, int mode,
                                    const __nv_bfloat16* q, const __nv_bfloat16* qt, const float* sel_thresh,
                                    const int32_t* sel_tie_last, int32_t seq_id, int32_t q_start, int64_t C,
-                                   __nv_bfloat16* out, float* lse, int32_t* status, cudaStream_t st);
+                                   __nv_bfloat16* out, float* lse, int32_t* status, cudaStream_t st,
+                                   const uint32_t* blk_mask, int64_t mask_words);
+
+// Block-wise top-p of a prefill chunk (Section 3.4): one bit per (row, retrieval head, page).
+size_t select_blocks_workspace_bytes(const Dims& d, const HeadMaps& hm, int64_t R, int64_t max_len, int sm_count);
+cudaError_t launch_select_blocks(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                                 const __nv_bfloat16* qt, uint32_t* mask, int64_t mask_words, int32_t* sel_count,
+                                 float* sel_mass, float* sel_thresh, int32_t* sel_tie_last, int32_t* status, void* ws,
+                                 size_t ws_bytes, int sm_count, cudaStream_t st);
 
 }  // namespace rtp
