@@ -646,6 +646,29 @@ def main():
         line["paper_prefill_mode"] = {"what": "retrieval heads dense + local heads sink/window + index-key append",
                                       "ms_per_step": t_paper, "tokens_per_s": L / (t_paper * 1e-3),
                                       "speedup_vs_dense": t_dense / t_paper}
+        # the block-wise selection of Section 3.4 (whole pages instead of tokens) on the same workload
+        def step_blocks():
+            for (s, C) in chunks:
+                path.run_chunk_blocks(s, C, data.q[s:s + C], k_pre[s:s + C], out[s:s + C])
+
+        step_blocks()
+        torch.cuda.synchronize()
+        t_blocks = min(ev_time_ms(step_blocks, stream) for _ in range(2))
+        kb = {"select_blocks": 0.0, "attn_blocks": 0.0}
+        n_blk_sel = torch.zeros((), dtype=torch.float64, device=device)
+        n_blk_all = 0.0
+        for (s, C) in chunks:
+            q = data.q[s:s + C]
+            kb["select_blocks"] += ev_time_ms(lambda: rb.rtp_topp_select_blocks(path.ctx, path.params, path.cache, q, data.w_q, 0, s, C, path.blk_mask[:C], path.sel_cnt[:C], path.sel_mass[:C], path.sel_thr[:C], path.sel_tie[:C], path.status, path.blk_ws), stream)
+            kb["attn_blocks"] += ev_time_ms(lambda: rb.rtp_sparse_attn_prefill_blocks(path.ctx, path.params, path.cache, q, 0, s, C, path.blk_mask[:C], out[s:s + C], None, path.status), stream)
+            n_blk_sel += path.sel_cnt[:C].sum(dtype=torch.float64)
+            n_blk_all += float(((torch.arange(s, s + C, device=device) // 64 + 1).sum() * len(data.heads.ret_q_heads)).item())
+        line["block_topp_path"] = {"what": "index keys + block-wise top-p (one bit per row, head, page) + attention over the selected pages + local heads",
+                                   "ms_per_step": t_blocks, "tokens_per_s": L / (t_blocks * 1e-3),
+                                   "speedup_vs_dense": t_dense / t_blocks, "kernel_ms_per_step": kb,
+                                   "selected_block_fraction": float(n_blk_sel.item()) / n_blk_all,
+                                   "attn_tflops": fl_sparse / kb["attn_blocks"] / 1e9,
+                                   "status": path.status_code()}
         if not c4:   # the 1M run stops at the comparators: no CPU sample, no decode points
             # CPU oracle on a bounded sample of the same workload
             rows = np.linspace(L // 8, L - 1, 160).astype(np.int64)

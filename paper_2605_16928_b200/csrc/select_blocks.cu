@@ -52,6 +52,17 @@ __device__ __forceinline__ float lds_f(uint32_t a) {
   return v;
 }
 __device__ __forceinline__ void sts_f(uint32_t a, float v) { asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory"); }
+// The stored pairs of a row are streamed through a small ring in shared memory with 8-byte cp.async copies, so that
+// many pages are in flight per thread without holding them in registers.
+constexpr int kRingDepth = 12;   // pages in flight per warp: 12 x 256 bytes (the key stages and the query tile are idle)
+__device__ __forceinline__ void cp_async8(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ float2 lds_f2(uint32_t a) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a) : "memory");
+  return v;
+}
 __device__ __forceinline__ void tmem_wait16b(uint32_t (&r)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;"
                : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
@@ -270,6 +281,27 @@ __global__ void __launch_bounds__(kBSubs * kBThreads, 1) select_blocks_kernel(
       }
     }
 
+    // ---- the row's stored pairs, page after page (rows of a warp see at most one page more or less than each other) ----
+    const int nb_warp = __reduce_max_sync(0xffffffffu, nb_row);
+    const uint32_t ring = sbase + kBStageOff + (uint32_t)(warp * kRingDepth * 256 + lane * 8);
+    auto for_pairs = [&](auto&& fn) {
+#pragma unroll 1
+      for (int k = 0; k < kRingDepth; ++k) {
+        if (k < nb_warp) cp_async8(ring + (uint32_t)(k * 256), my_stats + (int64_t)k * kBRows);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      }
+      int slot = 0;
+#pragma unroll 1
+      for (int b = 0; b < nb_warp; ++b) {
+        asm volatile("cp.async.wait_group %0;" ::"n"(kRingDepth - 1) : "memory");
+        const float2 v = lds_f2(ring + (uint32_t)(slot * 256));
+        if (b + kRingDepth < nb_warp) cp_async8(ring + (uint32_t)(slot * 256), my_stats + (int64_t)(b + kRingDepth) * kBRows);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        slot = slot + 1 == kRingDepth ? 0 : slot + 1;
+        if (b < nb_row) fn(b, v);
+      }
+      asm volatile("cp.async.wait_all;" ::: "memory");
+    };
     // ================================ levels: the cut in (m_b descending, block ascending) order ================================
     if (row_ok) {
       const int64_t o = (int64_t)(r0 + po) * d.n_ret + rh_head;
@@ -304,47 +336,39 @@ __global__ void __launch_bounds__(kBSubs * kBThreads, 1) select_blocks_kernel(
         const bool tie_scan = !grid_level && span == 1u;
         float acc = mass_above;   // tie scan: mass up to and including the current block of the cut's key
         bool tie_found = false;
-#pragma unroll 1
-        for (int b0 = 0; b0 < nb_row; b0 += 4) {
-          float2 v[4];
-#pragma unroll
-          for (int k = 0; k < 4; ++k) v[k] = b0 + k < nb_row ? __ldcg(my_stats + (int64_t)(b0 + k) * kBRows) : make_float2(-INFINITY, 0.f);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            if (b0 + k >= nb_row) break;
-            const float ms = mass_of(v[k]);
-            if (grid_level) {
-              float t = fmaf(v[k].x, -4.0f, dd);
-              if (!(t < kMagicB)) {   // (t < magic: above the window, counted by an earlier window)
-                t = fminf(t, kMagicB + (float)kPoolBinB);
-                const uint32_t a = hist_col + (__float_as_uint(t) & 63u) * kStep;
-                sts_f(a, lds_f(a) + ms);
-              }
-            } else {
-              const uint32_t t = okey(v[k].x) - lo_key;
-              if (t < span) {
-                if (tie_scan) {
-                  if (!tie_found) {
-                    acc += ms;
-                    tie_idx = b0 + k;
-                    if (acc >= target) tie_found = true;
-                  }
-                } else {
-                  const uint32_t a = hist_col + (t >> shift) * kStep;
-                  sts_f(a, lds_f(a) + ms);
-#pragma unroll
-                  for (int q = 0; q < kCandB; ++q)
-                    if (cnt == q) {
-                      ck[q] = okey(v[k].x);
-                      cb[q] = b0 + k;
-                      cm[q] = ms;
-                    }
-                  ++cnt;
+        for_pairs([&](const int b, const float2 v) {
+          const float ms = mass_of(v);
+          if (grid_level) {
+            float t = fmaf(v.x, -4.0f, dd);
+            if (!(t < kMagicB)) {   // (t < magic: above the window, counted by an earlier window)
+              t = fminf(t, kMagicB + (float)kPoolBinB);
+              const uint32_t a = hist_col + (__float_as_uint(t) & 63u) * kStep;
+              sts_f(a, lds_f(a) + ms);
+            }
+          } else {
+            const uint32_t t = okey(v.x) - lo_key;
+            if (t < span) {
+              if (tie_scan) {
+                if (!tie_found) {
+                  acc += ms;
+                  tie_idx = b;
+                  if (acc >= target) tie_found = true;
                 }
+              } else {
+                const uint32_t a = hist_col + (t >> shift) * kStep;
+                sts_f(a, lds_f(a) + ms);
+#pragma unroll
+                for (int q = 0; q < kCandB; ++q)
+                  if (cnt == q) {
+                    ck[q] = okey(v.x);
+                    cb[q] = b;
+                    cm[q] = ms;
+                  }
+                ++cnt;
               }
             }
           }
-        }
+        });
         if (tie_scan) {
           thr_key = lo_key;
           sel_m = acc / Z;
@@ -433,25 +457,16 @@ __global__ void __launch_bounds__(kBSubs * kBThreads, 1) select_blocks_kernel(
       uint32_t* mrow = mask + o * mask_words;
       const bool all = d.top_p >= 1.0f || nb_row <= 1 || thr_key == 0u;
       uint32_t bits = 0u;
-#pragma unroll 1
-      for (int b0 = 0; b0 < nb_row; b0 += 4) {
-        float2 v[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) v[k] = b0 + k < nb_row ? __ldcg(my_stats + (int64_t)(b0 + k) * kBRows) : make_float2(-INFINITY, 0.f);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const int b = b0 + k;
-          if (b >= nb_row) break;
-          const uint32_t key = okey(v[k].x);
-          const bool sel = all || key > thr_key || (key == thr_key && b <= tie_idx);
-          count += (int)sel;
-          bits |= (sel ? 1u : 0u) << (b & 31);
-          if ((b & 31) == 31 || b == nb_row - 1) {
-            mrow[b >> 5] = bits;
-            bits = 0u;
-          }
+      for_pairs([&](const int b, const float2 v) {
+        const uint32_t key = okey(v.x);
+        const bool sel = all || key > thr_key || (key == thr_key && b <= tie_idx);
+        count += (int)sel;
+        bits |= (sel ? 1u : 0u) << (b & 31);
+        if ((b & 31) == 31 || b == nb_row - 1) {
+          mrow[b >> 5] = bits;
+          bits = 0u;
         }
-      }
+      });
       sel_count[o] = count;
       if (sel_mass) sel_mass[o] = n_keys == 0 ? 0.f : (all ? 1.0f : sel_m);
       if (sel_thresh) sel_thresh[o] = (all || n_keys == 0) ? -INFINITY : okey_to_float(thr_key);

@@ -54,6 +54,7 @@ class PrefillPath(_Base):
         self.tok_seq = torch.zeros(chunk, dtype=torch.int32, device=self.dev)
         self.pos_all = torch.arange(L, dtype=torch.int32, device=self.dev)
         self.launches_per_chunk = 6   # index_keys, 2 x query projection, select, sparse attention, local attention
+        self.blk_mask = None          # block-wise path (Section 3.4): allocated on first use
 
     def chunks(self):
         return [(s, min(self.chunk, self.L - s)) for s in range(0, self.L, self.chunk)]
@@ -67,6 +68,20 @@ class PrefillPath(_Base):
                            self.sel_mass, self.sel_thr, self.sel_tie, self.status, self.workspace)
         rb.rtp_sparse_attn_prefill(self.ctx, p, self.cache, q, q, d.w_q, 0, q_start, C, None, self.sel_cnt,
                                    self.sel_thr, self.sel_tie, out, lse, self.workspace, self.status)
+        rb.rtp_local_attn(self.ctx, p, self.cache, q, None, None, 0, q_start, C, out, lse, self.workspace, self.status)
+
+    def run_chunk_blocks(self, q_start: int, C: int, q, k_pre, out, lse=None):
+        """The same chunk with the block-wise selection of Section 3.4 on the retrieval heads: append index keys ->
+        one bit per (row, head, page) -> attention over the selected pages -> sink + window attention on local heads."""
+        d, p = self.data, self.params
+        if self.blk_mask is None:
+            words = (((self.L + 63) // 64 + 31) // 32 + 3) // 4 * 4
+            self.blk_mask = torch.zeros((self.chunk, self.n_ret, words), dtype=torch.int32, device=self.dev)
+            self.blk_ws = torch.empty(rb.rtp_block_workspace_bytes(p, self.chunk, self.L), dtype=torch.uint8, device=self.dev)
+        rb.rtp_index_keys(self.ctx, p, self.cache, k_pre, d.w_k, self.tok_seq[:C], self.pos_all[q_start:q_start + C])
+        rb.rtp_topp_select_blocks(self.ctx, p, self.cache, q, d.w_q, 0, q_start, C, self.blk_mask[:C], self.sel_cnt[:C],
+                                  self.sel_mass[:C], self.sel_thr[:C], self.sel_tie[:C], self.status, self.blk_ws)
+        rb.rtp_sparse_attn_prefill_blocks(self.ctx, p, self.cache, q, 0, q_start, C, self.blk_mask[:C], out, lse, self.status)
         rb.rtp_local_attn(self.ctx, p, self.cache, q, None, None, 0, q_start, C, out, lse, self.workspace, self.status)
 
     def run_chunk_dense(self, q_start: int, C: int, q, out, lse=None):

@@ -231,3 +231,50 @@ def test_decode_512k_batch4_sampled_rows():
 
 def test_decode_1m_batch16_sampled_rows():
     _decode_point(1048576, 16, 0.9, 0.01, 4096, [1, 14], e2e=False)
+
+
+def test_prefill_128k_blocks_sampled_rows():
+    """Block-wise top-p (Section 3.4) at the benchmark's size: the last chunk and one from the middle."""
+    from paper_2605_16928_b200 import pipeline, synth_device
+    L, chunk = 131072, 8192
+    data = synth_device.config_3_device(L=L)
+    path = pipeline.PrefillPath(data, chunk)
+    for s in range(0, L, 131072):
+        path.index_keys_range(0, s, min(L, s + 131072))
+    heads, g = data.heads, data.heads.group
+    rng = np.random.default_rng(11)
+    out = torch.zeros((chunk, 32, 128), dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros((chunk, 32), dtype=torch.float32, device="cuda")
+    kv = {}
+    for s0 in (6 * chunk, L - chunk):
+        path.run_chunk_blocks(s0, chunk, data.q[s0:s0 + chunk], data.k_pre_rows(0, s0, s0 + chunk), out, lse)
+        torch.cuda.synchronize()
+        assert path.status_code() == rb.RTP_OK
+        rows = sorted({s0, s0 + chunk - 1, *map(int, rng.integers(s0, s0 + chunk, 6))})
+        sc, _, qh = _gpu_scores(path, data, rows, L)
+        r_t = torch.tensor([m - s0 for m in rows], device="cuda")
+        mask = path.blk_mask[r_t].cpu().numpy()
+        cnt, mass = path.sel_cnt[r_t].cpu().numpy(), path.sel_mass[r_t].cpu().numpy()
+        thr, tie = path.sel_thr[r_t].cpu().numpy(), path.sel_tie[r_t].cpu().numpy()
+        o_h, l_h = out[r_t].float().cpu().numpy(), lse[r_t].cpu().numpy()
+        for k, m in enumerate(rows):
+            n_b = m // 64 + 1
+            for i, h in enumerate(heads.ret_q_heads):
+                s = sc[k, i, : m + 1]
+                w = mask[k, i].view(np.uint32)
+                got = {b for b in range(n_b) if (int(w[b >> 5]) >> (b & 31)) & 1}
+                assert len(got) == int(cnt[k, i])
+                mb, lb = orc.block_lse(s)
+                assert got == {b for b in range(n_b) if mb[b] > thr[k, i] or (mb[b] == thr[k, i] and b <= tie[k, i])}
+                mand, forb = orc.classify_blocks_against_band(s, data.top_p)
+                assert mand <= got and not (forb & got), f"row {m} head {i}"
+                wgt = lb * np.exp(mb.astype(np.float64) - float(mb.max()))
+                tm = float(wgt[sorted(got)].sum() / wgt.sum())
+                assert tm >= data.top_p and abs(tm - mass[k, i]) <= 1e-4
+                kh = h // g
+                if kh not in kv:
+                    kv[kh] = data.logical_kv(0, kh)
+                want, wlse = orc.attention_over_set(qh[k, h], kv[kh][0], kv[kh][1], orc.block_token_set(sorted(got), m),
+                                                    data.sm_scale)
+                assert np.abs(o_h[k, h] - want).max() <= 2e-2, f"row {m} head {h}"
+                assert abs(l_h[k, h] - wlse) <= 1e-3 * max(1.0, abs(wlse))
