@@ -271,8 +271,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
   const bool want_ids = sel_idx != nullptr;
   const float scale = d.score_scale;
   const int n_units = n_row_tiles * d.n_ih;
-  const int dbg = max_passes_in >> 8;            // TEMPORARY (timing probes)
-  const int max_passes = max_passes_in & 255;
+  const int max_passes = max_passes_in;
 
   if (tid == 0) {
     for (int i = 0; i < kSStages; ++i) mbar_init(bar(kFullK + i), 1);
@@ -399,7 +398,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
     if (kind == kPassNone || n_tiles == 0) break;
     // pages walked by the pass: all of them, except when only tie rows are left, which know where to look
     int t_lo = 0, t_hi = n_tiles;
-    if (kind == kPassLate && flags == (1 << kPhTie) && !(dbg & 8)) {
+    if (kind == kPassLate && flags == (1 << kPhTie)) {
       t_lo = max(0, min(pass_rng[2 * (pass & 1)], n_tiles - 1));
       t_hi = max(t_lo + 1, min(pass_rng[2 * (pass & 1) + 1], n_tiles));
     }
@@ -460,7 +459,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           const float s_max = finish_score(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)), scale);
           if (!(fabsf(s_max) < 262144.0f)) {
             // no finite score, or scores beyond the range of the fixed grid: every key is kept and the call reports it
-            { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 1); }
+            set_status(status, RTP_ERR_UNSUPPORTED);
             phase = kPhDone;
             tie_last = n_keys - 1;
             count = n_keys;
@@ -554,7 +553,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
           }
           if (found < 0) {
             // an empty window below the mass already counted: nothing is left to add
-            { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 2); }
+            set_status(status, RTP_ERR_UNSUPPORTED);
             phase = kPhDone;
             tie_last = n_keys - 1;
             count = n_keys;
@@ -712,7 +711,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
             }
           }
           if (__any_sync(0xffffffffu, qa > qfull)) {
-            if (dbg & 2) qa = qbase; else warp_flush(false, (n0 + 8) >> 3);
+            warp_flush(false, (n0 + 8) >> 3);
           }
         };
         auto proc_late = [&](const uint32_t(&r)[16], const int n0, const bool interior) {
@@ -782,7 +781,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
         if (collecting && ovf) phase = kPhKey;   // no room for the bucket's keys: one key level first
         __syncwarp();   // every thread has read its histogram column: it now receives the row's final candidates
         // ---- exact finish of the rows that collected ----
-        const bool fin = collecting && !ovf && !(dbg & 1);
+        const bool fin = collecting && !ovf;
         bool new_tie = false;
         uint32_t sub_base = base_key, sub_span = span;
         float sub_above = mass_above;
@@ -939,14 +938,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
             each = fast_ex2((okey_to_float(sub_base) - ref0) * kLog2eC);
             if (sub_span != 1u) set_status(status, RTP_ERR_UNSUPPORTED);   // (more levels than any key has bits)
           } else {
-            if (c_in <= 0) { set_status(status, RTP_ERR_UNSUPPORTED); atomicOr(pool_ctr + 30, 1u << 6);
-              if (atomicCAS(pool_ctr + 32, 0u, 1u) == 0u) {   // TEMPORARY
-                pool_ctr[33] = (uint32_t)pos; pool_ctr[34] = (uint32_t)cnt; pool_ctr[35] = (uint32_t)n_words; pool_ctr[36] = base_key;
-                pool_ctr[37] = span; pool_ctr[38] = sub_base; pool_ctr[39] = sub_span; pool_ctr[40] = blk_first; pool_ctr[41] = (uint32_t)c_up;
-                pool_ctr[42] = (uint32_t)pass; pool_ctr[43] = __float_as_uint(raw_lo); pool_ctr[44] = __float_as_uint(raw_hi);
-                pool_ctr[45] = __float_as_uint(mass_above); pool_ctr[46] = __float_as_uint(target); pool_ctr[47] = (uint32_t)above;
-                pool_ctr[48] = __float_as_uint(sub_above); pool_ctr[49] = __float_as_uint(ref_s); pool_ctr[50] = __float_as_uint(scale);
-              } }
+            if (c_in <= 0) set_status(status, RTP_ERR_UNSUPPORTED);   // a chosen bucket always holds a key
             uint32_t bound = 0u;
             bool first_step = true;
             for (int step = 0; step < kCandCapC; ++step) {
@@ -1042,7 +1034,7 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
               done += n_here;
               blk = __ldcg(b);
             }
-            if (lane == rr && g_hi >= 0 && !(dbg & 16)) {
+            if (lane == rr && g_hi >= 0) {
               tie_pos_lo = g_lo << 3;
               tie_pos_hi = g_hi >= (int)kMarkerMask ? 0x7fffffff : g_hi << 3;
               tie_run = ties_at_mark;
@@ -1097,7 +1089,6 @@ __global__ void __launch_bounds__(kSubs * kSThreads, 1) select_chunk_kernel(
     const int64_t o = (int64_t)(r0 + po) * d.n_ret + rh_head;
     if (phase != kPhDone) {
       set_status(status, RTP_ERR_TIMEOUT);
-      atomicAdd(pool_ctr + 8 + phase, 1u);   // (diagnostic: rows left in each phase when the passes ran out)
     }
     sel_count[o] = n_keys == 0 ? 0 : count;
     if (sel_mass) sel_mass[o] = sel_m;
@@ -1133,9 +1124,7 @@ cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm,
   const int n_row_tiles = (int)((rows.R + BMP - 1) / BMP);
   const int n_units = n_row_tiles * d.n_ih;
   dim3 grid(std::max(1, std::min(sm_count, (n_units + kSubs - 1) / kSubs)));
-  int mp = kMaxPasses;
-  if (const char* e_ = getenv("RTP_SEL_MAX_PASSES")) mp = atoi(e_);   // TEMPORARY (timing probe)
-  if (const char* e_ = getenv("RTP_SEL_DBG")) mp |= atoi(e_) << 8;    // TEMPORARY
+  const int mp = kMaxPasses;
   select_chunk_kernel<G><<<grid, kSubs * kSThreads, kSmemS, st>>>(map_ik, cv, d, hm, qt, rows.seq_id, rows.q_start, (int)rows.R,
                                                           sel_idx, sel_stride, sel_count, sel_mass, sel_thresh,
                                                           sel_tie_last, status, reinterpret_cast<uint32_t*>(ws) + 64, (uint32_t)n_blocks,
