@@ -140,6 +140,10 @@ def bench_prefill(args, rank, world, device):
     chunks = path.chunks()
 
     def step():
+        if args.path == "blocks":
+            for (s, C) in chunks:
+                path.run_chunk_blocks(s, C, data.q[s:s + C], k_pre[s:s + C], out[s:s + C])
+            return
         for (s, C) in chunks:
             path.run_chunk(s, C, data.q[s:s + C], k_pre[s:s + C], out[s:s + C])
 
@@ -323,7 +327,14 @@ def bench_c5_sweep(device, iters=10, batches=(1, 4, 16), contexts=(131072, 52428
                     del valid, bi, hi, ji, mask
                     sel_rows = float(cnt.sum().item())
                     alg = B * n_ih * 32.0 * L + 520.0 * sel_rows + B * len(heads.local_kv_heads) * 512.0 * min(L, 4 + 4096)
+                    # K and V bytes held: every head in full, against retrieval heads in full + sink page and a ring of
+                    # window / 64 + 2 pages for the local heads (the truncated cache layout of rtp_cache)
+                    pages = (L + 63) // 64
+                    kv_full = 2.0 * B * pages * heads.n_kv_heads * 16384
+                    kv_trunc = 2.0 * B * (pages * (heads.n_kv_heads - len(heads.local_kv_heads)) +
+                                          (1 + 4096 // 64 + 2) * len(heads.local_kv_heads)) * 16384
                     table.append({"batch": B, "context": L, "top_p": p, "target_fraction": frac,
+                                  "kv_bytes_full": kv_full, "kv_bytes_truncated_local_heads": kv_trunc,
                                   "selected_fraction": sel_rows / (B * n_ret * L),
                                   "union_fraction_per_kv_head": float(union.mean().item()) / L,
                                   "sparse_step_us": t, "dense_step_us": t_dense, "speedup_vs_dense": t_dense / t,
@@ -345,6 +356,9 @@ def main():
                     help="c3: 128K chunked prefill, 2 retrieval KV heads (default, the bench line); "
                          "c4: 1M prefill with planted needles, chunk 16K, 1 retrieval KV head (long run, no end-to-end "
                          "leg); c5: the long-context decode sweep as one table")
+    ap.add_argument("--path", default="tokens", choices=["tokens", "blocks"],
+                    help="selection used by the timed step: token-level top-p (default, the bench line) or the block-wise "
+                         "top-p of the paper's kernel section (reported as block_topp_path in the default run)")
     ap.add_argument("--seq-len", type=int, default=0)
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the dense baseline, decode points and CPU oracle")
@@ -363,7 +377,8 @@ def main():
                            "c3_chunked_prefill_128k" if L == 131072 else f"c3_chunked_prefill_{L}"),
               "seq_len": L, "chunk": chunk, "n_q_heads": 32, "n_kv_heads": 8, "retrieval_kv_heads": 1 if c4 else 2,
               "index_dim": 16, "top_p": 0.9, "n_sink": 4, "window": 8192, "page_size": 64,
-              "l2": "inputs_larger_than_l2", "parallelism": "replicas" if world > 1 else "single_gpu"}
+              "l2": "inputs_larger_than_l2", "parallelism": "replicas" if world > 1 else "single_gpu",
+              "selection": "token-level top-p" if args.path == "tokens" else "block-wise top-p (64-key pages)"}
 
     if args.impl == "reference":
         # The reference arm is the CPU oracle, as it stands, on a bounded sample of the same workload.
@@ -464,7 +479,7 @@ def main():
     ms_per_step = ms / args.steps
     value = replicas.whole_job_rate(world, L, ms_per_step)
     status = path.status_code()
-    sel_frac = float((path.sel_cnt.float() / (path.pos_all[L - len(path.sel_cnt):].float()[:, None] + 1)).mean().item())
+    sel_frac = None if args.path == "blocks" else float((path.sel_cnt.float() / (path.pos_all[L - len(path.sel_cnt):].float()[:, None] + 1)).mean().item())
 
     from paper_2605_16928_b200 import binding as rb
     Hq, Hkv, nih = path.Hq, data.heads.n_kv_heads, data.heads.n_index_heads
@@ -548,8 +563,8 @@ def main():
         e2e_ok = bool(torch.equal(h_out[s_chk:s_chk + C_chk].to(device), out[s_chk:s_chk + C_chk]))
         return ms_e2e, h2d, d2h, e2e_ok
 
-    if args.workload == "c4":
-        # 1M tokens: the pinned host copies of q and out alone are 17 GB; the end-to-end leg is run on c3 only
+    if args.workload == "c4" or args.path == "blocks":
+        # 1M tokens: the pinned host copies of q and out alone are 17 GB; the end-to-end leg is run on c3's default path only
         ms_e2e, h2d, d2h, e2e_ok = None, 0, 0, None
     else:
         ms_e2e, h2d, d2h, e2e_ok = run_e2e()

@@ -95,6 +95,26 @@ typedef struct rtp_cache {
   int32_t num_pages;
   int32_t batch;
   int32_t max_pages;
+  /* Optional: truncated cache for local heads (Sections 1 and 3.2: the full KV cache is kept for retrieval heads only).
+   * When k_local_pages is not NULL,
+   *   - k_pages / v_pages hold only the KV heads that are NOT in rtp_params.local_kv_heads, in increasing head order:
+   *     bf16 [num_pages, n_kv_heads - n_local_kv_heads, 64, 128];
+   *   - the local KV heads, in the order of rtp_params.local_kv_heads, live in
+   *     k_local_pages / v_local_pages: bf16 [n_local_pages, n_local_kv_heads, 64, 128] behind their own table
+   *     local_block_table: int32 [batch, sink_pages + ring_pages]: logical page p of a sequence is entry p for
+   *     p < sink_pages and entry sink_pages + (p - sink_pages) % ring_pages otherwise, so a sequence holds its first
+   *     sink_pages pages and its newest ring_pages pages.  sink_pages * 64 must cover n_sink; a call of rtp_local_attn
+   *     needs ring_pages * 64 >= window + (tokens appended beyond the oldest row of the call) + 64;
+   *   - rtp_kv_append writes every head to its pool (one call must not carry more than ring_pages * 64 tokens of a
+   *     sequence: tokens of one call are written in no particular order); rtp_local_attn reads the local pool; the sparse and dense calls
+   *     read the main pool (dense calls may then only name heads that live there).
+   * All zero / NULL: one pool with every KV head (the layout above). */
+  void* k_local_pages;
+  void* v_local_pages;
+  const int32_t* local_block_table;
+  int32_t n_local_pages;
+  int32_t sink_pages;
+  int32_t ring_pages;
 } rtp_cache;
 
 /* ---- utility ------------------------------------------------------------ */

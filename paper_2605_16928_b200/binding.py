@@ -51,6 +51,8 @@ class RtpCache(C.Structure):
         ("k_pages", C.c_void_p), ("v_pages", C.c_void_p), ("ikey_pages", C.c_void_p),
         ("block_table", C.c_void_p), ("seq_lens", C.c_void_p),
         ("num_pages", C.c_int32), ("batch", C.c_int32), ("max_pages", C.c_int32),
+        ("k_local_pages", C.c_void_p), ("v_local_pages", C.c_void_p), ("local_block_table", C.c_void_p),
+        ("n_local_pages", C.c_int32), ("sink_pages", C.c_int32), ("ring_pages", C.c_int32),
     ]
 
 
@@ -172,11 +174,19 @@ class Params:
         return C.byref(self.c)
 
 
-def make_cache(k_pages, v_pages, ikey_pages, block_table, seq_lens) -> RtpCache:
-    """Describes caller-owned paged caches (torch CUDA tensors) to the library."""
+def make_cache(k_pages, v_pages, ikey_pages, block_table, seq_lens, k_local_pages=None, v_local_pages=None,
+               local_block_table=None, sink_pages: int = 0) -> RtpCache:
+    """Describes caller-owned paged caches (torch CUDA tensors) to the library.  With ``k_local_pages`` the cache is
+    truncated for local heads: ``k_pages`` / ``v_pages`` hold the other KV heads only, the local heads live in the
+    local pool behind ``local_block_table`` [batch, sink_pages + ring_pages]."""
     num_pages = int((k_pages if k_pages is not None else ikey_pages).shape[0])
+    n_local, ring = 0, 0
+    if k_local_pages is not None:
+        n_local = int(k_local_pages.shape[0])
+        ring = int(local_block_table.shape[1]) - int(sink_pages)
     return RtpCache(_ptr(k_pages), _ptr(v_pages), _ptr(ikey_pages), _ptr(block_table), _ptr(seq_lens),
-                    num_pages, int(block_table.shape[0]), int(block_table.shape[1]))
+                    num_pages, int(block_table.shape[0]), int(block_table.shape[1]),
+                    _ptr(k_local_pages), _ptr(v_local_pages), _ptr(local_block_table), n_local, int(sink_pages), ring)
 
 
 class Context:

@@ -152,6 +152,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     const int64_t bt_base = (int64_t)seq_id * cv.max_pages;
     const int last_page = m_last >> kPageShift;
     const int rsub = lane >> 3, ch = lane & 7;     // 4 rows x 8 chunks per warp instruction
+    const int kslot = cv.kv_slot[kvh];              // the KV head's place inside a page of this pool
     const __nv_bfloat16* pages = which ? cv.v : cv.k;
     const CUtensorMap* map = which ? &map_v : &map_k;
     for (int it = 0; it < n_tiles; ++it) {
@@ -165,8 +166,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
           mbar_expect_tx(fb, 2 * kBlk);
 #pragma unroll
           for (int pg = 0; pg < 2; ++pg) {
-            const int phys = safe_phys(cv, bt_base + kt * 2 + pg, status);
-            const int y = (phys * cv.n_kv + kvh) * kPage;
+            const int phys = safe_phys(cv, bt_base + page_entry(cv, kt * 2 + pg), status);
+            const int y = (phys * cv.n_kv + kslot) * kPage;
             tma_load_2d(dst0 + pg * (kPage * 128), map, 0, y, fb);
             tma_load_2d(dst0 + kBlk + pg * (kPage * 128), map, 64, y, fb);
           }
@@ -178,8 +179,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
       for (int pg = 0; pg < 2; ++pg) {
         const int page = kt * 2 + pg;
         const bool page_ok = page <= last_page;
-        const int phys = page_ok ? safe_phys(cv, bt_base + page, status) : 0;
-        const __nv_bfloat16* src0 = pages + ((int64_t)phys * cv.n_kv + kvh) * (kPage * kHeadDim);
+        const int phys = page_ok ? safe_phys(cv, bt_base + page_entry(cv, page), status) : 0;
+        const __nv_bfloat16* src0 = pages + ((int64_t)phys * cv.n_kv + kslot) * (kPage * kHeadDim);
         const int n_ok = page_ok ? m_last - page * kPage + 1 : 0;   // keys of the page any row may attend
 #pragma unroll 4
         for (int r4 = 0; r4 < 16; ++r4) {

@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
   const int m_pos = rows.row_pos(r);
   int n_keys = m_pos + 1;
   {
-    const int sl = (seq >= 0 && seq < cv.batch) ? min(cv.seq_lens[seq], cv.max_pages * kPage) : 0;   // (never beyond the block table)
+    const int sl = (seq >= 0 && seq < cv.batch) ? min(cv.seq_lens[seq], cv.cap_tokens) : 0;   // (never beyond the block table)
     if (n_keys > sl) {
       if (threadIdx.x == 0) set_status(status, RTP_ERR_INVALID);
       n_keys = sl;
@@ -142,10 +142,11 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
     if (SET == kSetLocal) return t < ns ? t : wlo + (t - ns);
     return t;
   };
-  auto load_phys = [&](int tok) -> int { return tok >= 0 ? safe_phys(cv, bt_base + (tok >> kPageShift), status) : 0; };
+  const int kslot = cv.kv_slot[kvh];   // the KV head's place inside a page of this pool
+  auto load_phys = [&](int tok) -> int { return tok >= 0 ? safe_phys(cv, bt_base + page_entry(cv, tok >> kPageShift), status) : 0; };
   // requests the K and V rows of a tile: token tt of the tile is copied by the half-warp (tt & 1) in step tt >> 1
   auto issue = [&](int stage, int tok, int phys) {
-    const int64_t off = (((int64_t)phys * cv.n_kv + kvh) * kPage + (tok & (kPage - 1))) * kHeadDim;
+    const int64_t off = (((int64_t)phys * cv.n_kv + kslot) * kPage + (tok & (kPage - 1))) * kHeadDim;
     const uint32_t sk = ring + stage * 2 * kTileBytes, sv = sk + kTileBytes;
     const int ch = lane & 15;
 #pragma unroll

@@ -63,10 +63,11 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(
 }
 
 // ---- K/V append: one 16-byte chunk per thread, K and V -----------------------------------------
-__global__ void kv_append_kernel(CacheView cv, const __nv_bfloat16* __restrict__ k_new,
+// k_new / v_new hold all n_src_heads KV heads of every token; the view stores those with a slot in its pool.
+__global__ void kv_append_kernel(CacheView cv, const int n_src_heads, const __nv_bfloat16* __restrict__ k_new,
                                  const __nv_bfloat16* __restrict__ v_new, const int32_t* __restrict__ tok_seq,
                                  const int32_t* __restrict__ tok_pos, int64_t T, int32_t* status) {
-  const int64_t chunks_per_tok = (int64_t)cv.n_kv * 16;
+  const int64_t chunks_per_tok = (int64_t)n_src_heads * 16;
   const int64_t total = T * chunks_per_tok;
   __nv_bfloat16* kp = const_cast<__nv_bfloat16*>(cv.k);
   __nv_bfloat16* vp = const_cast<__nv_bfloat16*>(cv.v);
@@ -74,18 +75,20 @@ __global__ void kv_append_kernel(CacheView cv, const __nv_bfloat16* __restrict__
     const int64_t t = i / chunks_per_tok;
     const int rem = (int)(i % chunks_per_tok);
     const int head = rem >> 4, ch = rem & 15;
+    const int slot = cv.kv_slot[head];
+    if (slot == 0xff) continue;   // the head lives in the other pool
     const int seq = tok_seq[t], pos = tok_pos[t];
-    if (seq < 0 || seq >= cv.batch || pos < 0 || (pos >> kPageShift) >= cv.max_pages) {
+    if (seq < 0 || seq >= cv.batch || pos < 0 || pos >= cv.cap_tokens) {
       set_status(status, RTP_ERR_INVALID);
       continue;
     }
-    const int phys = cv.block_table[(int64_t)seq * cv.max_pages + (pos >> kPageShift)];
+    const int phys = cv.block_table[(int64_t)seq * cv.max_pages + page_entry(cv, pos >> kPageShift)];
     if (phys < 0 || phys >= cv.num_pages) {
       set_status(status, RTP_ERR_INVALID);
       continue;
     }
-    const int64_t src = (t * cv.n_kv + head) * kHeadDim + ch * 8;
-    const int64_t dst = (((int64_t)phys * cv.n_kv + head) * kPage + (pos & (kPage - 1))) * kHeadDim + ch * 8;
+    const int64_t src = (t * n_src_heads + head) * kHeadDim + ch * 8;
+    const int64_t dst = (((int64_t)phys * cv.n_kv + slot) * kPage + (pos & (kPage - 1))) * kHeadDim + ch * 8;
     *reinterpret_cast<uint4*>(kp + dst) = ld_stream_v4(k_new + src);
     *reinterpret_cast<uint4*>(vp + dst) = ld_stream_v4(v_new + src);
   }
@@ -215,15 +218,15 @@ int score_splits(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
 
 }  // namespace
 
-cudaError_t launch_kv_append(const CacheView& cv, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new,
+cudaError_t launch_kv_append(const CacheView& cv, int n_src_heads, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new,
                              const int32_t* tok_seq, const int32_t* tok_pos, int64_t T, int32_t* status,
                              cudaStream_t st) {
   if (T == 0) return cudaSuccess;
-  const int64_t total = T * cv.n_kv * 16;
+  const int64_t total = T * n_src_heads * 16;
   int64_t blocks = (total + 255) / 256;
   const int64_t cap = (int64_t)current_sm_count(148) * 16;   // a few waves of grid-stride blocks
   if (blocks > cap) blocks = cap;
-  kv_append_kernel<<<(unsigned)blocks, 256, 0, st>>>(cv, k_new, v_new, tok_seq, tok_pos, T, status);
+  kv_append_kernel<<<(unsigned)blocks, 256, 0, st>>>(cv, n_src_heads, k_new, v_new, tok_seq, tok_pos, T, status);
   return cudaGetLastError();
 }
 

@@ -90,6 +90,7 @@ const char* check_cache(const rtp_cache* c, const rtp_params* p, bool need_kv, b
   if (need_kv && (!c->k_pages || !c->v_pages)) return "k_pages / v_pages is NULL";
   if (need_ikey && !c->ikey_pages) return "ikey_pages is NULL";
   if (!aligned16(c->k_pages) || !aligned16(c->v_pages) || !aligned16(c->ikey_pages)) return "cache pages must be 16-byte aligned";
+  if (p->n_kv_heads > 32) return "more than 32 KV heads";
   cv->k = reinterpret_cast<const __nv_bfloat16*>(c->k_pages);
   cv->v = reinterpret_cast<const __nv_bfloat16*>(c->v_pages);
   cv->ikey = reinterpret_cast<__nv_bfloat16*>(c->ikey_pages);
@@ -100,7 +101,41 @@ const char* check_cache(const rtp_cache* c, const rtp_params* p, bool need_kv, b
   cv->max_pages = c->max_pages;
   cv->n_kv = p->n_kv_heads;
   cv->n_ih = p->n_index_heads;
+  cv->cap_tokens = (int32_t)std::min<int64_t>((int64_t)c->max_pages * kPage, 0x7fffffff);
+  cv->sink_pages = 0;
+  cv->ring_pages = 0;
+  for (int h = 0; h < 32; ++h) cv->kv_slot[h] = h < p->n_kv_heads ? (uint8_t)h : (uint8_t)0xff;
+  if (c->k_local_pages) {
+    // truncated layout: the main pool holds the KV heads that are not local, in increasing order
+    if (!c->v_local_pages || !c->local_block_table) return "v_local_pages / local_block_table is NULL";
+    if (!aligned16(c->k_local_pages) || !aligned16(c->v_local_pages)) return "local cache pages must be 16-byte aligned";
+    if (c->n_local_pages <= 0 || c->ring_pages <= 0 || c->sink_pages < 0) return "local cache sizes must be positive";
+    if ((int64_t)c->sink_pages * kPage < p->n_sink) return "sink_pages does not cover n_sink";
+    if (p->n_local_kv_heads <= 0) return "a local cache without local KV heads";
+    bool local[32] = {};
+    for (int i = 0; i < p->n_local_kv_heads; ++i) local[p->local_kv_heads[i]] = true;
+    int n_main = 0;
+    for (int h = 0; h < p->n_kv_heads; ++h) cv->kv_slot[h] = local[h] ? (uint8_t)0xff : (uint8_t)n_main++;
+    cv->n_kv = n_main;
+  }
   return nullptr;
+}
+
+// The local heads' pool of a truncated cache as a view of its own (the index-key cache is not reachable through it).
+CacheView local_view(const CacheView& main, const rtp_cache* c, const rtp_params* p) {
+  CacheView v = main;
+  v.k = reinterpret_cast<const __nv_bfloat16*>(c->k_local_pages);
+  v.v = reinterpret_cast<const __nv_bfloat16*>(c->v_local_pages);
+  v.ikey = nullptr;
+  v.block_table = c->local_block_table;
+  v.num_pages = c->n_local_pages;
+  v.max_pages = c->sink_pages + c->ring_pages;
+  v.n_kv = p->n_local_kv_heads;
+  v.sink_pages = c->sink_pages;
+  v.ring_pages = c->ring_pages;
+  for (int h = 0; h < 32; ++h) v.kv_slot[h] = 0xff;
+  for (int i = 0; i < p->n_local_kv_heads; ++i) v.kv_slot[p->local_kv_heads[i]] = (uint8_t)i;
+  return v;
 }
 
 const char* check_rows(const int32_t* row_seq, const int32_t* row_pos, int32_t seq_id, int32_t q_start, int64_t R,
@@ -243,10 +278,14 @@ rtp_status rtp_kv_append(rtp_ctx* ctx, const rtp_params* params, const rtp_cache
   if (T == 0) return RTP_OK;
   if (!k_new || !v_new || !tok_seq || !tok_pos) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
   if (!aligned16(k_new) || !aligned16(v_new)) return fail(ctx, RTP_ERR_INVALID, "k_new / v_new must be 16-byte aligned");
-  (void)d;
   (void)hm;
-  cudaError_t e = launch_kv_append(cv, reinterpret_cast<const __nv_bfloat16*>(k_new),
-                                   reinterpret_cast<const __nv_bfloat16*>(v_new), tok_seq, tok_pos, T, status, st);
+  cudaError_t e = cudaSuccess;
+  if (cv.n_kv > 0)
+    e = launch_kv_append(cv, d.n_kv, reinterpret_cast<const __nv_bfloat16*>(k_new),
+                         reinterpret_cast<const __nv_bfloat16*>(v_new), tok_seq, tok_pos, T, status, st);
+  if (e == cudaSuccess && cache->k_local_pages)
+    e = launch_kv_append(local_view(cv, cache, params), d.n_kv, reinterpret_cast<const __nv_bfloat16*>(k_new),
+                         reinterpret_cast<const __nv_bfloat16*>(v_new), tok_seq, tok_pos, T, status, st);
   return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_kv_append");
 }
 
@@ -475,6 +514,13 @@ rtp_status rtp_local_attn(rtp_ctx* ctx, const rtp_params* params, const rtp_cach
   if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
   hm.n_kv_list = params->n_local_kv_heads;
   for (int i = 0; i < hm.n_kv_list; ++i) hm.kv_list[i] = (uint8_t)params->local_kv_heads[i];
+  if (cache->k_local_pages) {
+    // truncated cache: the local heads' ring must still hold the window of the call's oldest row
+    const int64_t ahead = row_seq ? 0 : R;   // a chunk is appended before it is attended
+    if ((int64_t)cache->ring_pages * kPage < (int64_t)d.window + ahead + kPage)
+      return fail(ctx, RTP_ERR_CAPACITY, "ring_pages too small for the window (plus the chunk) of this call");
+    cv = local_view(cv, cache, params);
+  }
   cudaError_t e;
   if (row_seq) {
     if (d.group != 1 && d.group != 2 && d.group != 4 && d.group != 8)
@@ -514,6 +560,9 @@ rtp_status rtp_dense_attn_prefill(rtp_ctx* ctx, const rtp_params* params, const 
   int64_t max_len = 0;
   if (const char* m = check_rows(nullptr, nullptr, seq_id, q_start, C, cache, &rows, &max_len)) return fail(ctx, RTP_ERR_INVALID, m);
   if (const char* m = fill_kv_list(params, kv_heads, n_heads, &hm)) return fail(ctx, RTP_ERR_INVALID, m);
+  for (int i = 0; i < hm.n_kv_list; ++i)
+    if (cv.kv_slot[hm.kv_list[i]] == 0xff)
+      return fail(ctx, RTP_ERR_UNSUPPORTED, "the cache is truncated for local heads: a dense call may only name the other KV heads");
   if (C == 0 || hm.n_kv_list == 0) return RTP_OK;
   if (!q || !out) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
   if (!aligned16(q) || !aligned16(out)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
@@ -534,6 +583,9 @@ rtp_status rtp_dense_attn_decode(rtp_ctx* ctx, const rtp_params* params, const r
   if (!row_seq || !row_pos) return fail(ctx, RTP_ERR_INVALID, "row_seq / row_pos is NULL");
   if (const char* m = check_rows(row_seq, row_pos, 0, 0, R, cache, &rows, &max_len)) return fail(ctx, RTP_ERR_INVALID, m);
   if (const char* m = fill_kv_list(params, kv_heads, n_heads, &hm)) return fail(ctx, RTP_ERR_INVALID, m);
+  for (int i = 0; i < hm.n_kv_list; ++i)
+    if (cv.kv_slot[hm.kv_list[i]] == 0xff)
+      return fail(ctx, RTP_ERR_UNSUPPORTED, "the cache is truncated for local heads: a dense call may only name the other KV heads");
   if (R == 0 || hm.n_kv_list == 0) return RTP_OK;
   if (!q || !out) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
   if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");

@@ -163,6 +163,10 @@ __device__ __forceinline__ void raw_preimage_warp(float scale, uint32_t key_lo, 
 
 // Physical page of a block-table entry.  An entry outside [0, num_pages) (a corrupt table) is read as page 0, so that
 // no kernel leaves the caches; kernels that have a status word also record RTP_ERR_INVALID for it.
+// Block-table entry (within a sequence's row) of logical page `page` of this view's pool.
+__device__ __forceinline__ int page_entry(const CacheView& cv, int page) {
+  return (cv.ring_pages > 0 && page >= cv.sink_pages) ? cv.sink_pages + (page - cv.sink_pages) % cv.ring_pages : page;
+}
 __device__ __forceinline__ int safe_phys(const CacheView& cv, int64_t entry, int32_t* status = nullptr) {
   const int phys = __ldg(cv.block_table + entry);
   if ((unsigned)phys < (unsigned)cv.num_pages) return phys;

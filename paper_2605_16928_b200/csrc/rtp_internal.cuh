@@ -39,7 +39,13 @@ struct CacheView {
   const int32_t* block_table;
   const int32_t* seq_lens;
   int32_t num_pages, batch, max_pages;
-  int32_t n_kv, n_ih;
+  int32_t n_kv, n_ih;      // n_kv: KV heads per page of the pool k / v point to
+  // A view of one pool.  cap_tokens: logical capacity of a sequence (the main block table's pages), used wherever a
+  // length is clamped.  ring_pages > 0: block_table has sink_pages + ring_pages entries per sequence and logical
+  // page p >= sink_pages lives in entry sink_pages + (p - sink_pages) % ring_pages.  kv_slot[h]: position of KV head h
+  // inside a page of this pool (0xff: the head is not stored here).
+  int32_t cap_tokens, sink_pages, ring_pages;
+  uint8_t kv_slot[32];
 };
 
 struct Dims {
@@ -133,7 +139,7 @@ inline int current_sm_count(int fallback) {
 cudaError_t launch_index_keys(const CacheView& cv, const Dims& d, const __nv_bfloat16* k_pre,
                               const __nv_bfloat16* w_k, const int32_t* tok_seq, const int32_t* tok_pos,
                               int64_t T, cudaStream_t st);
-cudaError_t launch_kv_append(const CacheView& cv, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new,
+cudaError_t launch_kv_append(const CacheView& cv, int n_src_heads, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new,
                              const int32_t* tok_seq, const int32_t* tok_pos, int64_t T, int32_t* status,
                              cudaStream_t st);
 cudaError_t launch_index_queries(const Dims& d, const HeadMaps& hm, const __nv_bfloat16* q_pre,
