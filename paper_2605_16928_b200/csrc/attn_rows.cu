@@ -334,9 +334,12 @@ __global__ void __launch_bounds__(kHeadDim) attn_merge_kernel(const Dims d, cons
   if (lse && dim == 0) lse[oh] = lt > 0.f ? (mt + log2f(lt)) * kLn2 : -INFINITY;
 }
 
-int plan_splits(int64_t units, int64_t max_set, int sm_count) {
+// Split count of a call.  Long contiguous sets (dense, sink + window) get at most two full rounds of two resident
+// CTAs per SM, rounded down: a few CTAs beyond a full round would cost a round of their own (dense decode at
+// B = 4 / 512K: 1411 -> 1246 us).  List gathers are short and latency-bound, their count is rounded up.
+int plan_splits(int64_t units, int64_t max_set, int sm_count, bool round_up) {
   if (units <= 0) return 1;
-  int64_t want = (4LL * sm_count + units - 1) / units;   // two rounds of two resident CTAs per SM
+  int64_t want = (4LL * sm_count + (round_up ? units - 1 : 0)) / units;
   int64_t cap = (max_set + 511) / 512;                   // at least 512 tokens (eight tiles per warp) per CTA
   int64_t s = want < cap ? want : cap;
   if (s < 1) s = 1;
@@ -375,7 +378,7 @@ cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm,
 
 size_t attn_rows_workspace_bytes(const Dims& d, int64_t R, int n_units, int group, int sm_count, int64_t max_len) {
   if (R <= 0 || n_units <= 0) return 0;
-  const int n_splits = plan_splits(R * n_units, max_len, sm_count);
+  const int n_splits = plan_splits(R * n_units, max_len, sm_count, true);   // (the larger of the two roundings)
   return (size_t)R * n_units * group * n_splits * kPartial * sizeof(float);
 }
 
@@ -386,7 +389,7 @@ cudaError_t launch_attn_rows(const CacheView& cv, const Dims& d, const HeadMaps&
   const int n_units = set == kSetList ? d.n_ret : hm.n_kv_list;
   if (rows.R == 0 || n_units == 0) return cudaSuccess;
   const int G = set == kSetList ? 1 : d.group;
-  int n_splits = plan_splits(rows.R * n_units, max_set_len(d, set, sel_stride, max_len), sm_count);
+  int n_splits = plan_splits(rows.R * n_units, max_set_len(d, set, sel_stride, max_len), sm_count, set == kSetList);
   // never plan more splits than the workspace holds
   const size_t per_split = (size_t)rows.R * n_units * G * kPartial * sizeof(float);
   if (n_splits > 1 && (size_t)n_splits * per_split > ws_bytes) n_splits = (int)(ws_bytes / per_split);
@@ -432,7 +435,7 @@ cudaError_t launch_attn_rows_static(const CacheView& cv, const Dims& d, const He
                                     int32_t* status, int sm_count, size_t* needed_bytes, cudaStream_t st) {
   *needed_bytes = 0;
   if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
-  const int n_splits = plan_splits(rows.R * d.n_ret, max_set_len(d, kSetList, sel_stride, max_len), sm_count);
+  const int n_splits = plan_splits(rows.R * d.n_ret, max_set_len(d, kSetList, sel_stride, max_len), sm_count, true);
   const size_t need = n_splits > 1 ? (size_t)rows.R * d.n_ret * n_splits * kPartial * sizeof(float) : 0;
   *needed_bytes = need;
   if (need > kStaticScratchBytes) return cudaErrorMemoryAllocation;   // reported as RTP_ERR_CAPACITY by the caller
