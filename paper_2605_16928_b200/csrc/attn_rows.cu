@@ -58,6 +58,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
     const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ sel_idx, const int64_t sel_stride,
     const int32_t* __restrict__ sel_count, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
     float* __restrict__ partial, const int n_splits, int32_t* status) {
+  chain_wait();
   static_assert(G >= 1 && G <= 8, "the query heads of a KV group are rows 0..7 of the MMA");
   extern __shared__ __align__(128) unsigned char smem_rows[];
 
@@ -312,6 +313,7 @@ __global__ void __launch_bounds__(kHeadDim) attn_merge_kernel(const Dims d, cons
                                                               const int G, const float* __restrict__ partial,
                                                               const int n_splits, __nv_bfloat16* __restrict__ out,
                                                               float* __restrict__ lse) {
+  chain_wait();
   const int64_t unit = blockIdx.x / G;
   const int g = blockIdx.x % G;
   const int64_t r = unit / n_units;
@@ -365,11 +367,11 @@ cudaError_t launch_typed(const CacheView& cv, const Dims& d, const HeadMaps& hm,
   static PerDeviceOnce once;   // (one per instantiation)
   cudaError_t e = set_dyn_smem_once(attn_rows_kernel<G, SET>, kRowsSmem, once);
   if (e != cudaSuccess) return e;
-  attn_rows_kernel<G, SET><<<grid, kThreads, kRowsSmem, st>>>(cv, d, hm, rows, n_units, q, sel_idx, sel_stride,
+  (void)launch_chained(attn_rows_kernel<G, SET>, dim3(grid), dim3(kThreads), kRowsSmem, st, cv, d, hm, rows, n_units, q, sel_idx, sel_stride,
                                                               sel_count, out, lse, partial, n_splits, status);
   e = cudaGetLastError();
   if (e != cudaSuccess || n_splits == 1) return e;
-  attn_merge_kernel<SET><<<(unsigned)(rows.R * n_units * G), kHeadDim, 0, st>>>(d, hm, n_units, G, partial,
+  (void)launch_chained(attn_merge_kernel<SET>, dim3((unsigned)(rows.R * n_units * G)), dim3(kHeadDim), 0, st, d, hm, n_units, G, partial,
                                                                                 n_splits, out, lse);
   return cudaGetLastError();
 }

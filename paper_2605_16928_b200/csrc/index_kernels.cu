@@ -16,6 +16,7 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(
     CacheView cv, Dims d, HeadMaps hm, const __nv_bfloat16* __restrict__ src,
     const __nv_bfloat16* __restrict__ w, const int32_t* __restrict__ tok_seq,
     const int32_t* __restrict__ tok_pos, int64_t T, __nv_bfloat16* __restrict__ qt) {
+  chain_wait();
   __shared__ float ws[kHeadDim * kIndexDim];                      // 8 KB
   __shared__ __align__(16) __nv_bfloat16 xs[kProjTokens][kHeadDim];  // 4 KB
   const int head = blockIdx.y;
@@ -236,7 +237,7 @@ cudaError_t launch_index_keys(const CacheView& cv, const Dims& d, const __nv_bfl
   if (T == 0) return cudaSuccess;
   HeadMaps hm = {};
   dim3 grid((unsigned)((T + kProjTokens - 1) / kProjTokens), d.n_ih);
-  project_kernel<true><<<grid, kProjThreads, 0, st>>>(cv, d, hm, k_pre, w_k, tok_seq, tok_pos, T, nullptr);
+  (void)launch_chained(project_kernel<true>, dim3(grid), dim3(kProjThreads), 0, st, cv, d, hm, k_pre, w_k, tok_seq, tok_pos, T, nullptr);
   return cudaGetLastError();
 }
 
@@ -245,7 +246,7 @@ cudaError_t launch_index_queries(const Dims& d, const HeadMaps& hm, const __nv_b
   if (R == 0 || d.n_ret == 0) return cudaSuccess;
   CacheView cv = {};
   dim3 grid((unsigned)((R + kProjTokens - 1) / kProjTokens), d.n_ret);
-  project_kernel<false><<<grid, kProjThreads, 0, st>>>(cv, d, hm, q_pre, w_q, nullptr, nullptr, R, qt);
+  (void)launch_chained(project_kernel<false>, dim3(grid), dim3(kProjThreads), 0, st, cv, d, hm, q_pre, w_q, nullptr, nullptr, R, qt);
   return cudaGetLastError();
 }
 

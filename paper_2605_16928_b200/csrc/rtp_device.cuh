@@ -163,6 +163,12 @@ __device__ __forceinline__ void raw_preimage_warp(float scale, uint32_t key_lo, 
 
 // Physical page of a block-table entry.  An entry outside [0, num_pages) (a corrupt table) is read as page 0, so that
 // no kernel leaves the caches; kernels that have a status word also record RTP_ERR_INVALID for it.
+// Kernels of the decode chain are launched with programmatic stream serialization: a kernel may be set up and start
+// while its predecessor in the stream is still running, and waits here (first statement, before any exit) until that
+// predecessor has completed and its writes are visible.  Every kernel of the chain waits, so completion is transitive.
+// A no-op for a kernel launched the ordinary way.
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Block-table entry (within a sequence's row) of logical page `page` of this view's pool.
 __device__ __forceinline__ int page_entry(const CacheView& cv, int page) {
   return (cv.ring_pages > 0 && page >= cv.sink_pages) ? cv.sink_pages + (page - cv.sink_pages) % cv.ring_pages : page;

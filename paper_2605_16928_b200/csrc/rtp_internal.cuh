@@ -1,6 +1,8 @@
 // Internal declarations shared by the kernels and the C-ABI layer (sm_100a only).
 #pragma once
 
+#include <utility>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -114,6 +116,24 @@ inline cudaError_t set_dyn_smem_once(Kernel kernel, int bytes, PerDeviceOnce& on
   }
   once.bits[dev >> 6].fetch_or(bit, std::memory_order_release);
   return cudaSuccess;
+}
+
+// Launch of a kernel of the decode chain (see chain_wait in rtp_device.cuh): the kernel may overlap the tail and the
+// launch latency of the kernel before it in the stream.
+template <class... KArgs, class... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
 }
 
 // SM count of the current device (queried once per device; `fallback` when no device can be asked, e.g. when only

@@ -61,6 +61,7 @@ __device__ __forceinline__ void load_page(const CacheView& cv, const RowCtx& x, 
 
 __global__ void sel_init_kernel(const CacheView cv, const Dims d, const Rows rows, SelState* state,
                                 int64_t n_rowheads, uint32_t* zero_words, int64_t n_zero_words) {
+  chain_wait();
   const int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   // merged histograms, counts and tickets start at zero (this replaces a separate memset)
@@ -141,6 +142,7 @@ __global__ void __launch_bounds__(kThreads) sel_score_kernel(const CacheView cv,
                                                              const Rows rows, const __nv_bfloat16* __restrict__ qt,
                                                              SelState* __restrict__ state, float* __restrict__ scores,
                                                              const int64_t l_pad, int n_splits, int32_t* status) {
+  chain_wait();
   __shared__ float s_max[kWarps][16];
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, status);
   if (x.p_lo >= x.p_hi) return;
@@ -233,6 +235,7 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
                                                           unsigned long long* __restrict__ g_mass,
                                                           uint32_t* __restrict__ tickets, int n_splits, const int list_cap,
                                                           int32_t* status) {
+  chain_wait();
   __shared__ uint32_t hist[kHeadsPerCta][kWarps][kBins][2];   // one private histogram per warp and head of the chunk
   __shared__ float s_M[16];
   __shared__ int s_on[16];
@@ -394,6 +397,7 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
                                                            SelState* __restrict__ state, unsigned long long* __restrict__ g_mass,
                                                            uint32_t* __restrict__ g_cnt, uint32_t* __restrict__ tickets,
                                                            int n_splits, int max_levels, const int list_cap, int32_t* status) {
+  chain_wait();
   __shared__ uint32_t hist[16][kBins][3];   // {sum, carries, count}
   __shared__ KeyParams kp[16];
   __shared__ uint32_t s_span[16];
@@ -569,6 +573,7 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
     const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows, const float* __restrict__ scores,
     const int64_t l_pad, SelState* __restrict__ state, uint2* __restrict__ cand, const int list_cap,
     int32_t* __restrict__ sel_idx, int64_t sel_stride, int n_splits, int32_t* status) {
+  chain_wait();
   __shared__ int id_stage[kWarps][kIdStage];
   __shared__ uint2 cand_stage[kWarps][kCandStageW];
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
@@ -651,6 +656,7 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
     int32_t* __restrict__ sel_count,
     float* __restrict__ sel_mass, float* __restrict__ sel_thresh, int32_t* __restrict__ sel_tie_last,
     int32_t* status) {
+  chain_wait();
   extern __shared__ __align__(16) unsigned char fin_smem[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(fin_smem);       // [kCandCap] candidates
   unsigned long long* keys2 = keys + kCandCap;                                       // [kCandCap] the other buffer
@@ -1051,7 +1057,7 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
     const int64_t work = n_zero > nrh ? n_zero : nrh;
     const int64_t cap_blocks = (int64_t)sm_count * 8;
     const unsigned blocks = (unsigned)((work + 255) / 256 < cap_blocks ? (work + 255) / 256 : cap_blocks);
-    sel_init_kernel<<<blocks, 256, 0, st>>>(cv, d, rows, w.state, nrh,
+    (void)launch_chained(sel_init_kernel, dim3(blocks), dim3(256), 0, st, cv, d, rows, w.state, nrh,
                                             reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + w.zero_off), n_zero);
   }
   int max_nh = 0;
@@ -1060,15 +1066,15 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
   const dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
   // one scan of the index keys (scores stored, row maxima), then three passes over the stored scores
   if (max_nh <= 4)
-    sel_score_kernel<true><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status);
+    (void)launch_chained(sel_score_kernel<true>, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status);
   else
-    sel_score_kernel<false><<<grid, kThreads, 0, st>>>(cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status);
-  sel_l1_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.tickets, n_splits, list_cap, status);
-  sel_key_kernel<<<grid, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.g_cnt, w.tickets,
+    (void)launch_chained(sel_score_kernel<false>, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status);
+  (void)launch_chained(sel_l1_kernel, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.tickets, n_splits, list_cap, status);
+  (void)launch_chained(sel_key_kernel, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.g_cnt, w.tickets,
                                             n_splits, 1 + kKeyLevels, list_cap, status);
   {
     const dim3 grid3((unsigned)(rows.R * d.n_ih), n_splits, (max_nh + kHeadsPerCta - 1) / kHeadsPerCta);
-    sel_compact_kernel<<<grid3, kThreads, 0, st>>>(cv, d, hm, rows, w.scores, l_pad, w.state, w.cand, list_cap, sel_idx,
+    (void)launch_chained(sel_compact_kernel, dim3(grid3), dim3(kThreads), 0, st, cv, d, hm, rows, w.scores, l_pad, w.state, w.cand, list_cap, sel_idx,
                                                    sel_stride, n_splits, status);
   }
   e = cudaGetLastError();
@@ -1077,7 +1083,7 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
   static PerDeviceOnce fin_once;
   e = set_dyn_smem_once(sel_finalize_kernel, kFinSmem, fin_once);
   if (e != cudaSuccess) return e;
-  sel_finalize_kernel<<<(unsigned)nrh, kFinThreads, kFinSmem, st>>>(d, w.scores, l_pad, w.state, w.cand, list_cap, sel_idx, sel_stride,
+  (void)launch_chained(sel_finalize_kernel, dim3((unsigned)nrh), dim3(kFinThreads), kFinSmem, st, d, w.scores, l_pad, w.state, w.cand, list_cap, sel_idx, sel_stride,
                                                              sel_count, sel_mass, sel_thresh, sel_tie_last, status);
   return cudaGetLastError();
 }
