@@ -128,23 +128,30 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
 
   const int64_t bt_base = (int64_t)seq * cv.max_pages;
   const uint32_t ring = (uint32_t)__cvta_generic_to_shared(smem_rows) + warp * kWarpRingBytes;
-  // token of entry (lane & 15) of this warp's i-th tile, or -1
-  auto load_tok = [&](int i) -> int {
+  // Token of entry (lane & 15) of this warp's i-th tile, or -1, and the physical page it lives in.  The loads and the
+  // checks of what they return are separate steps: a value is looked at one tile later than it was requested, so that
+  // the warp never waits for these dependent loads.
+  auto raw_tok = [&](int i) -> int {
     const int t = t_lo + (warp + i * kWarps) * kTileTok + (lane & 15);
     if (i >= n_mine || t >= t_hi) return -1;
-    if (SET == kSetList) {
-      const int tok = __ldg(ids + t);
-      if (tok < 0 || tok >= n_keys) {
-        set_status(status, RTP_ERR_INVALID);
-        return -1;
-      }
-      return tok;
-    }
+    if (SET == kSetList) return __ldg(ids + t);
     if (SET == kSetLocal) return t < ns ? t : wlo + (t - ns);
     return t;
   };
+  auto check_tok = [&](int tok) -> int {
+    if (SET == kSetList && tok != -1 && (tok < 0 || tok >= n_keys)) {
+      set_status(status, RTP_ERR_INVALID);
+      return -1;
+    }
+    return tok;
+  };
   const int kslot = cv.kv_slot[kvh];   // the KV head's place inside a page of this pool
-  auto load_phys = [&](int tok) -> int { return tok >= 0 ? safe_phys(cv, bt_base + page_entry(cv, tok >> kPageShift), status) : 0; };
+  auto raw_phys = [&](int tok) -> int { return tok >= 0 ? __ldg(cv.block_table + bt_base + page_entry(cv, tok >> kPageShift)) : 0; };
+  auto check_phys = [&](int phys) -> int {
+    if ((unsigned)phys < (unsigned)cv.num_pages) return phys;
+    set_status(status, RTP_ERR_INVALID);
+    return 0;
+  };
   // requests the K and V rows of a tile: token tt of the tile is copied by the half-warp (tt & 1) in step tt >> 1
   auto issue = [&](int stage, int tok, int phys) {
     const int64_t off = (((int64_t)phys * cv.n_kv + kslot) * kPage + (tok & (kPage - 1))) * kHeadDim;
@@ -163,8 +170,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
   // prologue: two tiles requested; the addresses of the third resolved, the tokens of the fourth on their way
   int tok_c[kRing];   // tokens of the tiles in the ring (for the validity mask)
   {
-    const int t0 = load_tok(0), t1 = load_tok(1);
-    const int p0 = load_phys(t0), p1 = load_phys(t1);
+    const int t0 = check_tok(raw_tok(0)), t1 = check_tok(raw_tok(1));
+    const int p0 = check_phys(raw_phys(t0)), p1 = check_phys(raw_phys(t1));
     issue(0, t0, p0);
     asm volatile("cp.async.commit_group;" ::: "memory");
     issue(1, t1, p1);
@@ -173,9 +180,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
     tok_c[1] = t1;
     tok_c[2] = -1;
   }
-  int tok_a = load_tok(2);
-  int phys_a = load_phys(tok_a);
-  int tok_b = load_tok(3);
+  int tok_a = check_tok(raw_tok(2));
+  int phys_a = raw_phys(tok_a);   // (looked at when tile 2 is requested)
+  int tok_b = raw_tok(3);         // (looked at one step later)
 
 #pragma unroll 1
   for (int i0 = 0; i0 < n_mine; i0 += kRing) {
@@ -187,12 +194,12 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
         __syncwarp();
         // tile i + 2 goes where tile i - 1 was
         const int next_stage = (sgi + 2) % kRing;
-        issue(next_stage, tok_a, phys_a);
+        issue(next_stage, tok_a, check_phys(phys_a));
         asm volatile("cp.async.commit_group;" ::: "memory");
         tok_c[next_stage] = tok_a;
-        tok_a = tok_b;
-        phys_a = load_phys(tok_a);      // used in the next step
-        tok_b = load_tok(i + 4);        // used in the step after that
+        tok_a = check_tok(tok_b);       // (requested one step ago)
+        phys_a = raw_phys(tok_a);       // looked at in the next step
+        tok_b = raw_tok(i + 4);         // looked at in the next step, used in the one after
 
         const uint32_t sk = ring + sgi * 2 * kTileBytes, sv = sk + kTileBytes;
         const uint32_t vmask = __ballot_sync(0xffffffffu, tok_c[sgi] >= 0) & 0xffffu;   // bit t = token t of the tile exists
