@@ -53,6 +53,12 @@ __device__ __forceinline__ void add_mass(uint32_t* acc, float x) {
   const uint32_t old = atomicAdd(acc, q);
   if (old + q < old) atomicAdd(acc + 1, 1u);
 }
+// The same contribution at 2^17 (x is still the 2^20-scale logarithm), added with a reduction that returns nothing:
+// the thread does not wait for it.  The caller bounds the number of adds per bin so that the 32-bit sum cannot wrap.
+__device__ __forceinline__ void add_mass17(uint32_t* acc, float x) {
+  const uint32_t q = __float_as_uint(fast_ex2(x - 3.0f) + 8388608.0f) - 0x4b000000u;
+  asm volatile("red.shared.add.u32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(acc)), "r"(q) : "memory");
+}
 __device__ __forceinline__ float acc_mass(uint32_t sum, uint32_t carries) {   // in units of 2^-20
   return (float)carries * 4294967296.0f + (float)sum;
 }

@@ -236,7 +236,10 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
                                                           uint32_t* __restrict__ tickets, int n_splits, const int list_cap,
                                                           int32_t* status) {
   chain_wait();
-  __shared__ uint32_t hist[kHeadsPerCta][kWarps][kBins][2];   // one private histogram per warp and head of the chunk
+  // One private histogram per warp and head of the chunk, 2^17 fixed point, added to with reductions that return
+  // nothing (the thread does not wait for them): a warp sees at most 32768 keys per head between two merges
+  // (select_splits), so a 32-bit sum cannot wrap.
+  __shared__ uint32_t hist[kHeadsPerCta][kWarps][kBins];
   __shared__ float s_M[16];
   __shared__ int s_on[16];
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
@@ -252,7 +255,7 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
     s_on[threadIdx.x] = on;
     s_M[threadIdx.x] = M;
   }
-  for (int i = threadIdx.x; i < kHeadsPerCta * kWarps * kBins * 2; i += kThreads) (&hist[0][0][0][0])[i] = 0u;
+  for (int i = threadIdx.x; i < kHeadsPerCta * kWarps * kBins; i += kThreads) (&hist[0][0][0])[i] = 0u;
   __syncthreads();
   int any = 0;
   for (int j = 0; j < x.nh; ++j) any |= s_on[j];
@@ -282,7 +285,7 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
           if (n0 + e >= ks.k_hi) continue;
           float bin_f;
           const int bin = l1_bin_f(Mj[jj], s4[e], bin_f);
-          add_mass(&hist[jj][warp][bin][0], l1_mass_arg(Mj[jj], s4[e], bin_f));
+          add_mass17(&hist[jj][warp][bin], l1_mass_arg(Mj[jj], s4[e], bin_f));
         }
       }
     }
@@ -291,9 +294,8 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
       const int jj = threadIdx.x / kBins, bin = threadIdx.x % kBins;   // 256 threads = 4 heads x 64 bins
       unsigned long long tot = 0ull;
       for (int w = 0; w < kWarps; ++w) {
-        tot += ((unsigned long long)hist[jj][w][bin][1] << 32) | hist[jj][w][bin][0];
-        hist[jj][w][bin][0] = 0u;
-        hist[jj][w][bin][1] = 0u;
+        tot += (unsigned long long)hist[jj][w][bin] << 3;   // back to the 2^20 scale of the merged histogram
+        hist[jj][w][bin] = 0u;
       }
       if (tot) atomicAdd(g_mass + (x.r * d.n_ret + hm.ih_heads[x.ih][j0 + jj]) * kBins + bin, tot);
     }
@@ -985,6 +987,8 @@ int select_splits(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
   int64_t want = (4LL * sm_count + R * d.n_ih - 1) / (R * d.n_ih);
   int64_t cap = (pages + 31) / 32;  // at least 32 pages (2048 keys) per CTA
   int64_t s = want < cap ? want : cap;
+  const int64_t least = (pages + 4095) / 4096;   // at most 4096 pages per CTA = 32768 keys per warp (32-bit bin sums)
+  if (s < least) s = least;
   if (s < 1) s = 1;
   if (s > 4096) s = 4096;
   return (int)s;
