@@ -25,6 +25,12 @@ What it follows
                          cut into blocks of 64, every block is reduced to a
                          log-sum-exp pair (m_b, l_b), blocks are taken in order
                          of decreasing m_b until their softmax mass reaches p.
+* ``topk_select``        Section 4.1, the fixed-budget variant the paper compares
+                         with ("w/ top-k", k = 4096): the k largest scores.
+* ``forced_tokens`` / ``with_forced``
+                         an optional variant that is not in Eq. 5: the first
+                         n_sink and the newest n_recent keys joined to a
+                         selected set (off by default: the paper forces nothing).
 * ``attention_over_set`` Eq. 5, softmax(q.k/sqrt(d_h)) restricted to S, times V.
 * ``local_set``          Section 3.2 / Table 2: attention sinks plus a sliding
                          window on local heads.
@@ -47,7 +53,10 @@ shift / permutation / monotonicity invariants, dense attention against
 torch's scaled_dot_product_attention, boolean-mask SDPA for the local pattern,
 the matrix-product identity for the indexer; for the block-wise selection:
 equal blocks, one dominant block, block size 1 against the token-level rule,
-brute force over all block subsets in m_b order.  The selection statistics the
+brute force over all block subsets in m_b order; for the fixed-budget selector:
+numpy's argpartition on distinct scores, the count rule, the tie rule on equal
+scores, agreement with Top-P at the p that its own mass defines; for the forced
+positions: their number in closed form and the subset / union laws.  The selection statistics the
 paper prints (its Tables 1, 6, 7) depend on model activations that are not
 available: parity unpinned for those numbers; they only shape synthetic data.
 
@@ -158,6 +167,42 @@ def set_mass(s: np.ndarray, ids) -> float:
     """Softmax mass (over the whole row) carried by the tokens ``ids``."""
     _, _, P = softmax_mass(s)
     return float(np.sum(P[np.asarray(sorted(ids), dtype=np.int64)]))
+
+
+# ---------------------------------------------------------------- fixed-budget variant (Section 4.1)
+def topk_select(s: np.ndarray, k: int):
+    """The fixed-budget selector the paper compares against in Section 4.1 (k = 4096
+    there): the k keys with the largest scores, equal scores going to the smaller
+    position; every key when the row has no more than k.  Returns (ids ascending,
+    number taken, threshold score = the smallest score taken, largest position taken
+    among the keys that have the threshold score)."""
+    if k < 1:
+        raise ValueError("top_k must be >= 1")
+    s = np.asarray(s, dtype=np.float32)
+    n = s.shape[0]
+    if n == 0:
+        raise ValueError("empty row")
+    order = descending_order(s)
+    c = min(int(k), n)
+    taken = order[:c]
+    thr = float(s[taken[-1]])
+    tie_last = int(max(int(i) for i in taken if s[i] == s[taken[-1]]))
+    return np.sort(taken), c, thr, tie_last
+
+
+def forced_tokens(m: int, n_sink: int, n_recent: int) -> np.ndarray:
+    """Positions a variant may force into the set of query position m whatever their
+    scores: the first n_sink keys and the n_recent newest ones (m itself included),
+    restricted to the causal range [0, m]."""
+    n = m + 1
+    head = np.arange(0, min(max(n_sink, 0), n), dtype=np.int64)
+    tail = np.arange(max(0, n - max(n_recent, 0)), n, dtype=np.int64)
+    return np.union1d(head, tail)
+
+
+def with_forced(ids, m: int, n_sink: int, n_recent: int) -> np.ndarray:
+    """Union of a selected set with the forced positions (ascending)."""
+    return np.union1d(np.asarray(ids, dtype=np.int64), forced_tokens(m, n_sink, n_recent))
 
 
 # ---------------------------------------------------------------- block-wise top-p (Section 3.4)
