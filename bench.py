@@ -266,6 +266,12 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
         t_graph = timed(graph.replay)
     except Exception as exc:   # capture is an extra; the plain numbers above stand on their own
         t_graph = f"not captured: {type(exc).__name__}"
+    # the fixed-budget variant the paper compares with (Section 4.1, k = 4096), same data and step
+    path_k = pipeline.DecodePath(data, max(stride, 4096), top_k=4096)
+    path_k.build_index_cache()
+    t_topk = timed(lambda: path_k.step(data.q, k_pre_new))
+    topk_status = path_k.status_code()
+    del path_k
     cnt = path.sel_cnt.float()
     n_ih = data.heads.n_index_heads
     sel_rows = float(cnt.sum().item())
@@ -275,6 +281,7 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
            "selected_fraction_mean": float(cnt.mean().item()) / L,
            "sparse_step_us": t_sparse, "sparse_step_us_cuda_graph": t_graph, "dense_step_us": t_dense,
            "speedup_vs_dense": t_dense / t_sparse,
+           "fixed_budget_4096_step_us": t_topk, "fixed_budget_status": topk_status,
            "algorithmic_bytes": alg_bytes, "sparse_path_gbs": alg_bytes / t_sparse / 1e3,
            "dense_gbs": B * data.heads.n_kv_heads * 512.0 * L / t_dense / 1e3,
            "status": path.status_code()}

@@ -83,6 +83,20 @@ typedef struct rtp_params {
   const int32_t* q_head_to_index_head; /* HOST [n_ret_q_heads] */
   const int32_t* index_head_kv;        /* HOST [n_index_heads] KV head of each index head */
   const int32_t* local_kv_heads;       /* HOST [n_local_kv_heads] */
+  /* Selectable variants of the decode selection (row lists: rtp_topp_select with row arrays, rtp_sparse_attn_decode).
+   * All zero = Eq. 5 as the paper states it.
+   *   top_k > 0: the fixed-budget selector of Section 4.1 (k = 4096 there) instead of Top-P: the top_k keys with the
+   *     largest indexer scores, equal scores going to the smaller position; every key when the row has fewer.  top_p is
+   *     ignored; sel_mass then receives (keys taken) / (causal keys), not a softmax mass.
+   *   force_sink / force_recent > 0: the first force_sink keys and the newest force_recent keys of the row (its own
+   *     position included) are joined to the selected set whatever their scores.  They come after the regular entries
+   *     of a list, sel_count counts them, sel_mass includes their softmax mass; sel_thresh / sel_tie_last still describe
+   *     the regular rule alone.  force_sink + force_recent <= 65536.
+   * The chunk (prefill) forms of the selection and the block-wise calls return RTP_ERR_UNSUPPORTED when any of the
+   * three is set. */
+  int32_t top_k;
+  int32_t force_sink;
+  int32_t force_recent;
 } rtp_params;
 
 /* Paged caches.  The index-key cache shares the KV block table. */

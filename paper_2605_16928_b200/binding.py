@@ -43,6 +43,7 @@ class RtpParams(C.Structure):
         ("top_p", C.c_float), ("score_scale", C.c_float), ("sm_scale", C.c_float),
         ("ret_q_heads", C.POINTER(C.c_int32)), ("q_head_to_index_head", C.POINTER(C.c_int32)),
         ("index_head_kv", C.POINTER(C.c_int32)), ("local_kv_heads", C.POINTER(C.c_int32)),
+        ("top_k", C.c_int32), ("force_sink", C.c_int32), ("force_recent", C.c_int32),
     ]
 
 
@@ -144,7 +145,8 @@ class Params:
     def __init__(self, n_q_heads: int, n_kv_heads: int, ret_q_heads: Sequence[int],
                  q_head_to_index_head: Sequence[int], index_head_kv: Sequence[int],
                  local_kv_heads: Sequence[int], n_sink: int = 4, window: int = 8192, top_p: float = 0.9,
-                 score_scale: float = 1.0, sm_scale: float = 128 ** -0.5):
+                 score_scale: float = 1.0, sm_scale: float = 128 ** -0.5, top_k: int = 0, force_sink: int = 0,
+                 force_recent: int = 0):
         self._a = _i32_array(ret_q_heads)
         self._b = _i32_array(q_head_to_index_head)
         self._c = _i32_array(index_head_kv)
@@ -158,7 +160,8 @@ class Params:
         self.c = RtpParams(128, 16, 64, n_q_heads, n_kv_heads, len(index_head_kv), len(ret_q_heads),
                            len(local_kv_heads), n_sink, window, top_p, score_scale, sm_scale,
                            C.cast(self._a, C.POINTER(C.c_int32)), C.cast(self._b, C.POINTER(C.c_int32)),
-                           C.cast(self._c, C.POINTER(C.c_int32)), C.cast(self._d, C.POINTER(C.c_int32)))
+                           C.cast(self._c, C.POINTER(C.c_int32)), C.cast(self._d, C.POINTER(C.c_int32)),
+                           top_k, force_sink, force_recent)
 
     @classmethod
     def from_workload(cls, wl, **over) -> "Params":

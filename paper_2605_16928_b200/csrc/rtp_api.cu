@@ -28,6 +28,9 @@ rtp_status cuda_fail(rtp_ctx* ctx, cudaError_t e, const char* where) {
   return RTP_ERR_CUDA;
 }
 
+// Any of the selectable variants of the decode selection (fixed budget, forced positions) is on.
+bool variant_set(const Dims& d) { return d.top_k > 0 || d.force_sink > 0 || d.force_recent > 0; }
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Validates the parameter block and fills the device-side views.  Returns NULL on success, else a message.
@@ -48,6 +51,9 @@ const char* check_params(const rtp_params* p, Dims* d, HeadMaps* hm) {
   if (!(p->score_scale > 0.0f) || !(p->score_scale < 1e30f)) return "score_scale must be positive and finite";
   if (!(p->sm_scale > 0.0f) || !(p->sm_scale < 1e30f)) return "sm_scale must be positive and finite";
   if (p->n_sink < 0 || p->window < 1) return "n_sink must be >= 0 and window >= 1";
+  if (p->top_k < 0) return "top_k must be >= 0";
+  if (p->force_sink < 0 || p->force_recent < 0 || (int64_t)p->force_sink + p->force_recent > 65536)
+    return "force_sink and force_recent must be >= 0 and sum to at most 65536";
   d->n_q = p->n_q_heads;
   d->n_kv = p->n_kv_heads;
   d->n_ih = p->n_index_heads;
@@ -56,6 +62,9 @@ const char* check_params(const rtp_params* p, Dims* d, HeadMaps* hm) {
   d->n_sink = p->n_sink;
   d->window = p->window;
   d->top_p = p->top_p;
+  d->top_k = p->top_k;
+  d->force_sink = p->force_sink;
+  d->force_recent = p->force_recent;
   d->score_scale = p->score_scale;
   d->sm_scale = p->sm_scale;
   d->wait_ns = 2000000000ull;
@@ -347,6 +356,7 @@ rtp_status rtp_topp_select(rtp_ctx* ctx, const rtp_params* params, const rtp_cac
   WsCarver w(workspace);
   __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(w.take(qt_bytes(d, R)));
   const bool chunk = row_seq == nullptr;
+  if (chunk && variant_set(d)) return fail(ctx, RTP_ERR_UNSUPPORTED, "top_k / forced positions: row lists only");
   const size_t sel_off = w.off;
   void* sel_ws = w.take(chunk ? select_chunk_workspace_bytes(d, hm, R) : select_rows_workspace_bytes(d, R, max_len));
   if (w.off > workspace_bytes) return fail(ctx, RTP_ERR_CAPACITY, "workspace too small");
@@ -432,6 +442,7 @@ rtp_status rtp_sparse_attn_prefill(rtp_ctx* ctx, const rtp_params* params, const
   }
   if (!sel_thresh || !sel_tie_last || !q_pre || !w_q || !workspace)
     return fail(ctx, RTP_ERR_INVALID, "threshold mode needs sel_thresh, sel_tie_last, q_pre, w_q and a workspace");
+  if (variant_set(d)) return fail(ctx, RTP_ERR_UNSUPPORTED, "top_k / forced positions: row lists only");
   if (!aligned16(q_pre) || !aligned16(w_q)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
   WsCarver w(workspace);
   __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(w.take(qt_bytes(d, C)));
@@ -469,6 +480,7 @@ rtp_status rtp_topp_select_blocks(rtp_ctx* ctx, const rtp_params* params, const 
   if (!q_pre || !w_q || !workspace || !sel_count || !block_mask) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
   if (!aligned16(q_pre) || !aligned16(w_q) || !aligned16(workspace)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
   if (mask_words * 32 < ((int64_t)q_start + C + kPage - 1) / kPage) return fail(ctx, RTP_ERR_CAPACITY, "mask_words too small for the chunk's pages");
+  if (variant_set(d)) return fail(ctx, RTP_ERR_UNSUPPORTED, "top_k / forced positions: row lists only");
   WsCarver w(workspace);
   __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(w.take(qt_bytes(d, C)));
   const size_t sel_off = w.off;

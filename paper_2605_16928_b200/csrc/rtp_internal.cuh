@@ -54,6 +54,8 @@ struct Dims {
   int32_t n_q, n_kv, n_ih, n_ret, group;
   int32_t n_sink, window;
   float top_p, score_scale, sm_scale;
+  int32_t top_k;                       // > 0: the fixed-budget selector (Section 4.1) in the decode selection
+  int32_t force_sink, force_recent;    // positions joined to every selected set of the decode selection
   // bounded device-side waits give up after this many nanoseconds; wait_test != 0: the key loader of the prefill
   // attention kernel withholds the signal for its first tile (rtp_debug_wait_test)
   unsigned long long wait_ns;

@@ -74,7 +74,8 @@ __global__ void sel_init_kernel(const CacheView cv, const Dims d, const Rows row
     n_keys = max(0, min(n_keys, sl));
     SelState s = {};
     s.n_keys = n_keys;
-    s.mode = (d.top_p >= 1.0f || n_keys <= 1) ? kSelectAll : kRefine;
+    const bool every = d.top_k > 0 ? d.top_k >= n_keys : d.top_p >= 1.0f;
+    s.mode = (every || n_keys <= 1) ? kSelectAll : kRefine;
     s.hi_key = 0xffffffffu;
     state[i] = s;
   }
@@ -228,6 +229,8 @@ __device__ __forceinline__ float4 ld_scores4(const float* p) {
   return v;
 }
 
+constexpr float kCountScale = 9.5367431640625e-07f;   // 2^-20: a key of the fixed-budget selector adds 2^20 to its bin
+
 // ---- pass 2: level-1 mass histogram over M - s, resolved by the unit's last CTA ----------------------------------
 __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
                                                           const Rows rows, const float* __restrict__ scores,
@@ -237,8 +240,8 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
                                                           int32_t* status) {
   chain_wait();
   // One private histogram per warp and head of the chunk, 2^17 fixed point, added to with reductions that return
-  // nothing (the thread does not wait for them): a warp sees at most 32768 keys per head between two merges
-  // (select_splits), so a 32-bit sum cannot wrap.
+  // nothing (the thread does not wait for them): a warp sees at most 16384 keys per head between two merges
+  // (select_splits) and a key adds at most 2^17 (+ rounding), so a 32-bit sum cannot wrap.
   __shared__ uint32_t hist[kHeadsPerCta][kWarps][kBins];
   __shared__ float s_M[16];
   __shared__ int s_on[16];
@@ -262,6 +265,7 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
   if (!any) return;   // the same decision in every CTA of the unit
 
   const KeySpan ks = key_span(x);
+  const bool by_count = d.top_k > 0;   // fixed budget: every key weighs the same, the "mass" is a count
   for (int j0 = 0; j0 < x.nh; j0 += kHeadsPerCta) {   // four heads at a time: their loads are in flight together
     const float* row[kHeadsPerCta];
     float Mj[kHeadsPerCta];
@@ -285,7 +289,8 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
           if (n0 + e >= ks.k_hi) continue;
           float bin_f;
           const int bin = l1_bin_f(Mj[jj], s4[e], bin_f);
-          add_mass17(&hist[jj][warp][bin], l1_mass_arg(Mj[jj], s4[e], bin_f));
+          const float arg = l1_mass_arg(Mj[jj], s4[e], bin_f);
+          add_mass17(&hist[jj][warp][bin], by_count ? 20.0f : arg);
         }
       }
     }
@@ -314,7 +319,7 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
     gm[b0] = 0ull;
     gm[b1] = 0ull;
     const float q0 = __ull2float_rn(u0), q1 = __ull2float_rn(u1);
-    const float m0 = q0 * l1_bin_scale(b0), m1 = q1 * l1_bin_scale(b1);
+    const float m0 = q0 * (by_count ? kCountScale : l1_bin_scale(b0)), m1 = q1 * (by_count ? kCountScale : l1_bin_scale(b1));
     float inc = m0 + m1;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -322,7 +327,8 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
       if (lane >= o) inc += t;
     }
     const float Z = __shfl_sync(0xffffffffu, inc, 31);
-    const float target = d.top_p * Z * (1.0f + kMassMargin);
+    // (counts are small integers: their sums are exact and the target needs no margin)
+    const float target = by_count ? (float)d.top_k : d.top_p * Z * (1.0f + kMassMargin);
     const float run = inc - (m0 + m1);
     int found = 64, last = -1;
     if (u0) {
@@ -355,8 +361,12 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
       const float q = __shfl_sync(0xffffffffu, first ? q0 : q1, owner);
       uint32_t klo = 0u, khi = 0u;
       float rlo = 0.f, rhi = 0.f;
-      if (found != kBins - 1) {
+      // Top-P: a cut inside the pooled last bin (mass below 1e-13 per key) keeps every key.  The fixed budget counts
+      // keys, so its cut can fall there: the bucket is then every key from the bottom up to the pool's upper end.
+      const bool pooled = found == kBins - 1 && !by_count;
+      if (!pooled) {
         l1_bin_keys_warp(M, found, lane, klo, khi);
+        if (found == kBins - 1) klo = 0u;
         raw_preimage_warp(d.score_scale, klo, khi, lane, rlo, rhi);
       }
       if (lane == 0) {
@@ -364,8 +374,8 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
         st->Z = Z;
         st->target = target;
         st->mass_above = above;
-        if (found == kBins - 1) {
-          st->mode = kSelectAll;       // the cut falls into the pooled tail (mass below 1e-13 per key): take every key
+        if (pooled) {
+          st->mode = kSelectAll;       // the cut falls into the pooled tail: take every key
         } else {
           const uint32_t span = khi - klo + 1u;
           const int bits = span > 1u ? 32 - __clz(span - 1u) : 0;
@@ -376,7 +386,7 @@ __global__ void __launch_bounds__(kThreads) sel_l1_kernel(const CacheView cv, co
           st->raw_lo = rlo;
           st->raw_hi = rhi;
           st->ref_s = l1_bin_hi(M, found);
-          st->e_ref = fast_ex2(-kLog2eH * (0.5f * (float)found - 0.25f));
+          st->e_ref = by_count ? 1.0f : fast_ex2(-kLog2eH * (0.5f * (float)found - 0.25f));
           if (q < 0.999f * kMinQ * (float)list_cap) st->mode = kCollect;   // fewer than list_cap keys in the bin
         }
       }
@@ -443,6 +453,7 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
     const uint32_t base_key = kp[j].base_key, span = s_span[j];
     const int shift = kp[j].shift;
     const float ref_s = kp[j].ref_s;
+    const float lw = d.top_k > 0 ? 0.f : kLog2eH;   // fixed budget: every key adds 2^20
     for (int nb = ks.k_lo + 4 * (int)threadIdx.x; nb < ks.k_hi; nb += kLoads * 4 * kThreads) {
       float4 v[kLoads];
 #pragma unroll
@@ -459,7 +470,7 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
           const uint32_t t = okey(s4[e]) - base_key;
           if (n0 + e < ks.k_hi && t < span) {
             uint32_t* acc = &hist[j][t >> shift][0];
-            add_mass(acc, fmaf(s4[e] - ref_s, kLog2eH, 20.0f));
+            add_mass(acc, fmaf(s4[e] - ref_s, lw, 20.0f));
             atomicAdd(acc + 2, 1u);
           }
         }
@@ -694,6 +705,7 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
     return;
   }
   const float M = st->M, Z = st->Z, target = st->target;
+  const bool by_count = d.top_k > 0;
   float above = st->mass_above;
   int base = st->cnt_above;
   int emit_base = ids ? st->emit_cnt : base;
@@ -702,6 +714,41 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
   uint32_t tie_key = st->lo_key;
   int tie_bucket = st->bucket_cnt;
   int n_fin = 0;   // candidates left for the exact sort
+
+  // Forced positions (a selectable variant, off in the paper's method): the first force_sink and the newest
+  // force_recent keys of the row that the regular rule (score above the threshold, or equal to it and not beyond
+  // t_last) left out are appended behind the `count` regular entries.  Returns how many were added; their mass
+  // (relative to exp(M), or their number under the fixed budget) is added to mass_io.  Called by every thread.
+  auto add_forced = [&](uint32_t t_key, int t_last, int count, float& mass_io) -> int {
+    const int n_head = min(d.force_sink, n_keys), tail_lo = max(n_head, n_keys - d.force_recent);
+    const int nf = n_head + (n_keys - tail_lo);
+    if (nf <= 0) return 0;   // uniform
+    __syncthreads();
+    if (tid == 0) s_n2 = 0;
+    __syncthreads();
+    const float* row = scores + rh * l_pad;
+    float em = 0.f;
+    for (int i = tid; i < nf; i += kFinThreads) {
+      const int n = i < n_head ? i : tail_lo + (i - n_head);
+      const float sv = __ldcg(row + n);
+      const uint32_t key = okey(sv);
+      if (!(key > t_key || (key == t_key && n <= t_last))) {
+        const int pos = count + atomicAdd(&s_n2, 1);
+        if (ids && pos < sel_stride) ids[pos] = n;
+        em += by_count ? 1.0f : __expf(sv - M);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) em += __shfl_xor_sync(0xffffffffu, em, o);
+    if (lane == 0) w_sum[warp] = em;
+    __syncthreads();
+    float tot = 0.f;
+    for (int w = 0; w < kFinWarps; ++w) tot += w_sum[w];   // the same order in every thread and every run
+    mass_io += tot;
+    const int added = s_n2;
+    __syncthreads();
+    return added;
+  };
   if (mode == kCollect) {
     // The candidates of the bucket: a list in global memory (up to list_cap entries).  A list that fits is copied to
     // shared memory at once; a longer one is narrowed where it is until the chosen part fits.
@@ -722,6 +769,7 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
     {
       uint32_t lo_key = st->lo_key, span = st->span;
       const float ref_s = st->ref_s, sc = st->e_ref * 9.5367431640625e-07f;   // 2^-20
+      const float lw = by_count ? 0.f : kLog2eH;
       while ((n > 256 || in_global) && span > 1u) {
         const int bits = 32 - __clz(span - 1u);
         const int shift = max(0, bits - 6);
@@ -737,7 +785,7 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
             const uint32_t t = key - lo_key;
             if (t < span) {
               uint32_t* acc = &fh[t >> shift][0];
-              add_mass(acc, fmaf(okey_to_float(key) - ref_s, kLog2eH, 20.0f));
+              add_mass(acc, fmaf(okey_to_float(key) - ref_s, lw, 20.0f));
               atomicAdd(acc + 2, 1u);
             }
           }
@@ -745,7 +793,7 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
           for (int i = tid; i < n; i += kFinThreads) {
             const uint32_t key = ~(uint32_t)(keys[i] >> 32);
             uint32_t* acc = &fh[(key - lo_key) >> shift][0];
-            add_mass(acc, fmaf(okey_to_float(key) - ref_s, kLog2eH, 20.0f));
+            add_mass(acc, fmaf(okey_to_float(key) - ref_s, lw, 20.0f));
             atomicAdd(acc + 2, 1u);
           }
         }
@@ -867,7 +915,7 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
       if (s_pick != kNoPick) break;  // uniform: written before the barrier that ends each round
       const int i = r0 + tid;
       float e = 0.f;
-      if (i < n) e = __expf(okey_to_float(~(uint32_t)(keys[i] >> 32)) - M);
+      if (i < n) e = by_count ? 1.0f : __expf(okey_to_float(~(uint32_t)(keys[i] >> 32)) - M);
       float inc = e;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -902,12 +950,15 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
         if (pos < sel_stride) ids[pos] = (int)(uint32_t)keys[i];
       }
     }
+    const uint32_t thr_key = ~(uint32_t)(keys[pick] >> 32);
+    const int thr_last = (int)(uint32_t)keys[pick];
+    const int extra = add_forced(thr_key, thr_last, base + c, mass);
     if (tid == 0) {
-      sel_count[rh] = base + c;
+      sel_count[rh] = base + c + extra;
       if (sel_mass) sel_mass[rh] = mass / Z;
-      if (sel_thresh) sel_thresh[rh] = okey_to_float(~(uint32_t)(keys[pick] >> 32));
-      if (sel_tie_last) sel_tie_last[rh] = (int)(uint32_t)keys[pick];
-      if (ids && base + c > sel_stride) set_status(status, RTP_ERR_CAPACITY);
+      if (sel_thresh) sel_thresh[rh] = okey_to_float(thr_key);
+      if (sel_tie_last) sel_tie_last[rh] = thr_last;
+      if (ids && base + c + extra > sel_stride) set_status(status, RTP_ERR_CAPACITY);
     }
     return;
   }
@@ -916,7 +967,7 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
     // More than kCandCap keys share the threshold score exactly: take the first c of them in
     // position order, c = the number of equal masses still needed.
     const uint32_t t_key = tie_key;
-    const float e_t = __expf(okey_to_float(t_key) - M);
+    const float e_t = by_count ? 1.0f : __expf(okey_to_float(t_key) - M);
     int c = (int)ceilf((target - above) / e_t);
     c = max(1, min(c, tie_bucket));
     const float* row = scores + rh * l_pad;
@@ -966,12 +1017,15 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
       if (tid == 0) s_emitted += tot;
       __syncthreads();
     }
+    float mass = above + (float)c * e_t;
+    const int t_last = s_last;
+    const int extra = add_forced(t_key, t_last, base + c, mass);
     if (tid == 0) {
-      sel_count[rh] = base + c;
-      if (sel_mass) sel_mass[rh] = (above + (float)c * e_t) / Z;
+      sel_count[rh] = base + c + extra;
+      if (sel_mass) sel_mass[rh] = mass / Z;
       if (sel_thresh) sel_thresh[rh] = okey_to_float(t_key);
-      if (sel_tie_last) sel_tie_last[rh] = s_last;
-      if (ids && base + c > sel_stride) set_status(status, RTP_ERR_CAPACITY);
+      if (sel_tie_last) sel_tie_last[rh] = t_last;
+      if (ids && base + c + extra > sel_stride) set_status(status, RTP_ERR_CAPACITY);
     }
     return;
   }
@@ -987,7 +1041,7 @@ int select_splits(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
   int64_t want = (4LL * sm_count + R * d.n_ih - 1) / (R * d.n_ih);
   int64_t cap = (pages + 31) / 32;  // at least 32 pages (2048 keys) per CTA
   int64_t s = want < cap ? want : cap;
-  const int64_t least = (pages + 4095) / 4096;   // at most 4096 pages per CTA = 32768 keys per warp (32-bit bin sums)
+  const int64_t least = (pages + 2047) / 2048;   // at most 2048 pages per CTA = 16384 keys per warp (32-bit bin sums)
   if (s < least) s = least;
   if (s < 1) s = 1;
   if (s > 4096) s = 4096;

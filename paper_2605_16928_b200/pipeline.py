@@ -14,12 +14,12 @@ from . import binding as rb
 
 
 class _Base:
-    def __init__(self, data, max_rows: int, max_len: int):
+    def __init__(self, data, max_rows: int, max_len: int, **param_over):
         self.data = data
         dev = data.q.device
         self.dev = dev
         self.ctx = rb.Context()
-        self.params = rb.Params.from_workload(data)
+        self.params = rb.Params.from_workload(data, **param_over)
         nih = max(1, data.heads.n_index_heads)
         self.ikey_pages = torch.zeros((data.num_pages, nih, 64, 16), dtype=torch.bfloat16, device=dev)
         self.cache = rb.make_cache(data.k_pages, data.v_pages, self.ikey_pages, data.block_table, data.seq_lens)
@@ -91,10 +91,11 @@ class PrefillPath(_Base):
 class DecodePath(_Base):
     """One decode step for a batch: row b is the newest token of sequence b."""
 
-    def __init__(self, data, sel_stride: int):
+    def __init__(self, data, sel_stride: int, **param_over):
+        """param_over: rtp_params fields that replace the workload's (top_k, force_sink, force_recent, top_p ...)."""
         B = int(data.seq_lens.shape[0])
         L = int(data.seq_lens.max())
-        super().__init__(data, B, L)
+        super().__init__(data, B, L, **param_over)
         self.B, self.L = B, L
         self.sel_idx = torch.empty((B, self.n_ret, sel_stride), dtype=torch.int32, device=self.dev)
         self.sel_cnt = torch.empty((B, self.n_ret), dtype=torch.int32, device=self.dev)

@@ -231,6 +231,51 @@ def check_selection(dw: DeviceWorkload, sc: np.ndarray, sel: dict, rows=None, p:
     return stats
 
 
+def check_variant_selection(dw: DeviceWorkload, sc: np.ndarray, sel: dict, top_k: int = 0, force_sink: int = 0,
+                            force_recent: int = 0, rows=None, p: float | None = None):
+    """Row lists of the selectable variants (fixed budget, forced positions) against the oracle run on the GPU's own
+    scores.  Fixed budget: the regular part is unique, so the lists must be the oracle's sets exactly.  Top-P with forced
+    positions: the regular part obeys the band rule of ``check_selection``; the rest is exactly the forced positions
+    the regular part left out, and they come last."""
+    wl = dw.wl
+    p = wl.top_p if p is None else p
+    idx, cnt = sel["idx"].cpu().numpy(), sel["cnt"].cpu().numpy()
+    mass, thr, tie = sel["mass"].cpu().numpy(), sel["thr"].cpu().numpy(), sel["tie"].cpu().numpy()
+    rows = range(dw.R) if rows is None else rows
+    counts = []
+    for r in rows:
+        m = int(wl.row_pos[r])
+        for i in range(dw.n_ret):
+            s = sc[r, i, : m + 1]
+            c = int(cnt[r, i])
+            assert 1 <= c <= m + 1 and c <= idx.shape[-1]
+            lst = idx[r, i, :c]
+            assert len(set(lst.tolist())) == c, "duplicate ids"
+            assert np.all(idx[r, i, c:] == -1), "wrote past the count"
+            member = (s > thr[r, i]) | ((s == thr[r, i]) & (np.arange(m + 1) <= tie[r, i]))
+            regular = np.nonzero(member)[0]
+            if top_k > 0:
+                want_reg, k_taken, want_thr, want_tie = orc.topk_select(s, top_k)
+                assert np.array_equal(regular, want_reg), f"row {r} head {i}: regular part differs from the k largest"
+                if k_taken <= m:                       # (when every key is taken the threshold outputs are -inf / m)
+                    assert thr[r, i] == want_thr and tie[r, i] == want_tie
+            else:
+                mand, forb = orc.classify_against_band(s, p)
+                got = set(regular.tolist())
+                assert mand <= got and not (forb & got)
+                assert orc.set_mass(s, got) >= p or len(got) == m + 1
+            want = orc.with_forced(regular, m, force_sink, force_recent)
+            assert c == want.size, f"row {r} head {i}: count {c}, oracle {want.size}"
+            assert np.array_equal(np.sort(lst), want)
+            assert set(lst[: regular.size].tolist()) == set(regular.tolist()), "forced positions must come last"
+            if top_k > 0:
+                assert abs(mass[r, i] - c / (m + 1)) <= 1e-6
+            else:
+                assert abs(mass[r, i] - orc.set_mass(s, want)) <= 1e-4
+            counts.append((c, int(regular.size), m + 1))
+    return counts
+
+
 def check_sparse_attention(dw: DeviceWorkload, sel: dict, out: np.ndarray, lse: np.ndarray, rows=None, tol=2e-2):
     wl = dw.wl
     g = wl.heads.group

@@ -221,6 +221,56 @@ def _decode_point(L, B, top_p, frac, window, seqs, peaked_half=False, name="c5_d
             assert np.abs(out[k, kh * g + jj] - want).max() <= 2e-2
 
 
+def _decode_variant_point(L, B, frac, window, seqs, **variant):
+    """The selectable variants at full size: lists of sampled sequences equal the oracle's sets on the GPU's scores,
+    attention over them matches the oracle."""
+    from paper_2605_16928_b200 import pipeline, synth_device
+    data = synth_device.decode_device(L, B, 0.9, frac, window, name="c5_decode_sweep")
+    path = pipeline.DecodePath(data, sel_stride=int(min(L, max(16384, 4 * frac * L))), **variant)
+    path.build_index_cache()
+    k_new = torch.stack([data.k_pre_rows(b, L - 1, L)[0] for b in range(B)]).contiguous()
+    path.step(data.q, k_new)
+    torch.cuda.synchronize()
+    assert path.status_code() == rb.RTP_OK
+    heads, g = data.heads, data.heads.group
+    rs = torch.tensor(seqs, device="cuda")
+    sc = torch.full((len(seqs), path.n_ret, L), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(rb.rtp_workspace_bytes(path.params, len(seqs), L), dtype=torch.uint8, device="cuda")
+    rb.rtp_index_score(path.ctx, path.params, path.cache, data.q[rs].contiguous(), data.w_q,
+                       data.row_seq[rs].contiguous(), data.row_pos[rs].contiguous(), sc, None, None, ws, path.status)
+    torch.cuda.synchronize()
+    sc = sc.cpu().numpy()
+    idx, cnt = path.sel_idx[rs].cpu().numpy(), path.sel_cnt[rs].cpu().numpy()
+    out = path.out[rs].float().cpu().numpy()
+    qh = _np16(data.q[rs])
+    top_k, fs, fr = variant.get("top_k", 0), variant.get("force_sink", 0), variant.get("force_recent", 0)
+    for k, b in enumerate(seqs):
+        for i, h in enumerate(heads.ret_q_heads):
+            c = int(cnt[k, i])
+            lst = idx[k, i, :c]
+            if top_k:
+                regular = orc.topk_select(sc[k, i], top_k)[0]
+            else:
+                thr, tie = float(path.sel_thr[b, i]), int(path.sel_tie[b, i])
+                regular = np.nonzero((sc[k, i] > thr) | ((sc[k, i] == thr) & (np.arange(L) <= tie)))[0]
+                mand, forb = orc.classify_against_band(sc[k, i], data.top_p)
+                assert mand <= set(regular.tolist()) and not (forb & set(regular.tolist()))
+            want = orc.with_forced(regular, L - 1, fs, fr)
+            assert np.array_equal(np.sort(lst), want), f"seq {b} head {i}"
+            kk, vv = data.logical_kv(b, h // g)
+            ref, _ = orc.attention_over_set(qh[k, h], kk, vv, want, data.sm_scale)
+            assert np.abs(out[k, h] - ref).max() <= 2e-2, f"seq {b} head {h}"
+
+
+def test_decode_512k_batch4_fixed_budget_4096():
+    _decode_variant_point(524288, 4, 0.05, 4096, [1, 2], top_k=4096)
+
+
+def test_decode_128k_forced_positions():
+    _decode_variant_point(131072, 2, 0.05, 4096, [0, 1], force_sink=4, force_recent=256)
+    _decode_variant_point(131072, 2, 0.05, 4096, [1], top_k=4096, force_sink=4, force_recent=256)
+
+
 def test_decode_32k_batch8_sampled_rows():
     _decode_point(32768, 8, 0.95, 0.1, 2048, [0, 3, 4, 7], peaked_half=True, name="c2_decode_batched_gqa")
 
