@@ -29,6 +29,12 @@
  *   index_dim 16, page_size 64.
  *
  * Head conventions: query head h reads KV head h / (n_q_heads / n_kv_heads).
+ * The partition into retrieval and local heads is over QUERY heads (Section 3.2): a KV head may be listed in
+ * local_kv_heads while some query heads of its group are retrieval heads (a mixed group).  rtp_local_attn then
+ * writes only the group's query heads that are not retrieval heads, the decode calls and the list form of
+ * rtp_sparse_attn_prefill serve its retrieval heads; the threshold and block-wise forms of the prefill attention
+ * need index heads that cover whole groups (RTP_ERR_UNSUPPORTED otherwise), and such a KV head cannot live in the
+ * truncated pool of rtp_cache (RTP_ERR_INVALID).
  * Retrieval query heads are listed in rtp_params.ret_q_heads; entry i has its
  * own W_q[i] and its own selection, and scores against the index-key stream
  * q_head_to_index_head[i].  Index head j projects the pre-RoPE keys of KV head

@@ -546,6 +546,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
     asm volatile("bar.sync 1, 256;" ::: "memory");
     if (grp == 0) {
       __nv_bfloat16* dst = out + ((int64_t)(r0 + (row_ok ? po : 0)) * d.n_q + qh) * kHeadDim;
+      // (a local call computes a retrieval head that sits in a local group but leaves its slot to the sparse call)
+      const bool row_wr = row_ok && !(MODE == kPrefillLocal && hm.skips(qh));
 #pragma unroll
       for (int c4 = 0; c4 < 4; ++c4) {
         uint32_t r[32];
@@ -556,7 +558,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = 0u;
         }
-        if (row_ok) {
+        if (row_wr) {
 #pragma unroll
           for (int c8 = 0; c8 < 4; ++c8) {
             const float4 a = *reinterpret_cast<const float4*>(stage_row + c4 * 32 + c8 * 8);
@@ -573,7 +575,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_prefill_tc_kernel(
           }
         }
       }
-      if (row_ok && lse) lse[(int64_t)(r0 + po) * d.n_q + qh] = l_tot > 0.f ? (m_tot + log2f(l_tot)) * kLn2T : -INFINITY;
+      if (row_wr && lse) lse[(int64_t)(r0 + po) * d.n_q + qh] = l_tot > 0.f ? (m_tot + log2f(l_tot)) * kLn2T : -INFINITY;
     }
   }
 

@@ -300,6 +300,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
       }
     }
     const int64_t oh = (int64_t)r * d.n_q + qh0 + gg;
+    if (SET == kSetLocal && hm.skips(qh0 + gg)) continue;   // a retrieval head inside a local group: not this call's
     if (n_splits == 1) {
       out[oh * kHeadDim + dim] = __float2bfloat16_rn(lt > 0.f ? a / lt : 0.f);
       if (lse && dim == 0) lse[oh] = lt > 0.f ? (mt + log2f(lt)) * kLn2 : -INFINITY;
@@ -326,6 +327,7 @@ __global__ void __launch_bounds__(kHeadDim) attn_merge_kernel(const Dims d, cons
   const int64_t r = unit / n_units;
   const int u = unit % n_units;
   const int qh = (SET == kSetList) ? hm.ret_q_head[u] : hm.kv_list[u] * d.group + g;
+  if (SET == kSetLocal && hm.skips(qh)) return;
   const float* p = partial + ((unit * G + g) * (int64_t)n_splits) * kPartial;
   const int dim = threadIdx.x;
   float mt = -INFINITY;

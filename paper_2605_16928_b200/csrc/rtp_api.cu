@@ -123,6 +123,10 @@ const char* check_cache(const rtp_cache* c, const rtp_params* p, bool need_kv, b
     if (p->n_local_kv_heads <= 0) return "a local cache without local KV heads";
     bool local[32] = {};
     for (int i = 0; i < p->n_local_kv_heads; ++i) local[p->local_kv_heads[i]] = true;
+    // a mixed group (retrieval and local query heads on one KV head) needs that head's whole history
+    const int group = p->n_q_heads / p->n_kv_heads;
+    for (int i = 0; i < p->n_ret_q_heads; ++i)
+      if (local[p->ret_q_heads[i] / group]) return "a KV head with retrieval query heads cannot live in the truncated pool";
     int n_main = 0;
     for (int h = 0; h < p->n_kv_heads; ++h) cv->kv_slot[h] = local[h] ? (uint8_t)0xff : (uint8_t)n_main++;
     cv->n_kv = n_main;
@@ -526,6 +530,8 @@ rtp_status rtp_local_attn(rtp_ctx* ctx, const rtp_params* params, const rtp_cach
   if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
   hm.n_kv_list = params->n_local_kv_heads;
   for (int i = 0; i < hm.n_kv_list; ++i) hm.kv_list[i] = (uint8_t)params->local_kv_heads[i];
+  // a mixed group: its retrieval heads are written by the sparse call, not by this one
+  for (int i = 0; i < d.n_ret; ++i) hm.skip_q[hm.ret_q_head[i] >> 5] |= 1u << (hm.ret_q_head[i] & 31);
   if (cache->k_local_pages) {
     // truncated cache: the local heads' ring must still hold the window of the call's oldest row
     const int64_t ahead = row_seq ? 0 : R;   // a chunk is appended before it is attended

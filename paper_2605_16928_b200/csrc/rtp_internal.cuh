@@ -32,6 +32,10 @@ struct HeadMaps {
   uint8_t ih_heads[RTP_MAX_INDEX_HEADS][RTP_MAX_HEADS_PER_INDEX_HEAD];
   uint8_t kv_list[RTP_MAX_Q_HEADS];         // KV heads processed by a local / dense call
   int32_t n_kv_list;
+  // Query heads a local call computes but does not write: the retrieval heads inside a KV group that is otherwise
+  // local (a mixed group, Section 3.2: the head partition is over query heads).  Bit q of word q / 32.
+  uint32_t skip_q[RTP_MAX_Q_HEADS / 32];
+  __host__ __device__ bool skips(int qh) const { return (skip_q[qh >> 5] >> (qh & 31)) & 1u; }
 };
 
 struct CacheView {

@@ -11,7 +11,8 @@ Conventions
 * "Logical" K/V of one sequence are ``[L, Hkv, 128]``; the paged cache is
   ``[num_pages, Hkv, 64, 128]`` (K and V separately) plus an index-key cache
   ``[num_pages, n_index_heads, 64, 16]`` that shares the block table.
-* A *retrieval KV head* makes all its G query heads retrieval heads.  Each
+* A *retrieval KV head* makes all its G query heads retrieval heads (or, with
+  ``ret_per_group``, only the first few of them: a mixed group).  Each
   retrieval query head has its own ``W_q``; each index head (one per retrieval
   KV head) has one ``W_k``.  The generators tie ``W_q = W_k`` inside a group so
   that a planted key aligned with a query really gets a high projected score
@@ -65,19 +66,32 @@ class HeadMap:
     ret_kv_heads: list            # KV heads whose query heads are retrieval heads
     n_sink: int = 4
     window: int = 8192
+    # > 0: a mixed group: only the first ret_per_group query heads of a retrieval KV head are retrieval heads, the
+    # others of the group attend locally (the KV head is then also a local KV head)
+    ret_per_group: int = 0
 
     @property
     def group(self) -> int:
         return self.n_q_heads // self.n_kv_heads
 
     @property
+    def _rpg(self) -> int:
+        return self.ret_per_group if 0 < self.ret_per_group < self.group else self.group
+
+    @property
     def local_kv_heads(self) -> list:
-        return [h for h in range(self.n_kv_heads) if h not in self.ret_kv_heads]
+        mixed = self._rpg < self.group
+        return [h for h in range(self.n_kv_heads) if mixed or h not in self.ret_kv_heads]
 
     @property
     def ret_q_heads(self) -> list:
         g = self.group
-        return [kv * g + j for kv in self.ret_kv_heads for j in range(g)]
+        return [kv * g + j for kv in self.ret_kv_heads for j in range(self._rpg)]
+
+    @property
+    def local_q_heads(self) -> list:
+        ret = set(self.ret_q_heads)
+        return [kv * self.group + j for kv in self.local_kv_heads for j in range(self.group) if kv * self.group + j not in ret]
 
     @property
     def n_index_heads(self) -> int:
@@ -86,7 +100,7 @@ class HeadMap:
     @property
     def q_head_to_index_head(self) -> list:
         """For retrieval query head number i (position in ret_q_heads)."""
-        return [i // self.group for i in range(len(self.ret_q_heads))]
+        return [i // self._rpg for i in range(len(self.ret_q_heads))]
 
     @property
     def index_head_kv(self) -> list:
@@ -234,9 +248,9 @@ def config_1(L: int = 4096, n_needles: int = 8, seed: int = BASE_SEED + 1, top_p
 def config_2(L: int = 32768, batch: int = 8, n_q_heads: int = 32, n_kv_heads: int = 8,
              ret_kv_heads=(0, 1), window: int = 2048, top_p: float = 0.95,
              flat_sigma: float = 2.5, seed: int = BASE_SEED + 2,
-             needle_range=(16, 64)) -> Workload:
+             needle_range=(16, 64), ret_per_group: int = 0) -> Workload:
     rng = _rng(seed)
-    heads = HeadMap(n_q_heads, n_kv_heads, list(ret_kv_heads), n_sink=4, window=window)
+    heads = HeadMap(n_q_heads, n_kv_heads, list(ret_kv_heads), n_sink=4, window=window, ret_per_group=ret_per_group)
     g = heads.group
     scale = 0.125
     W = [_normal(rng, (HEAD_DIM, INDEX_DIM)) / np.sqrt(np.float32(HEAD_DIM)) for _ in heads.ret_kv_heads]
@@ -282,9 +296,9 @@ def config_2(L: int = 32768, batch: int = 8, n_q_heads: int = 32, n_kv_heads: in
 # --------------------------------------------------------------------------
 def config_3(L: int = 131072, n_q_heads: int = 32, n_kv_heads: int = 8, ret_kv_heads=(0, 1),
              window: int = 8192, top_p: float = 0.9, score_scale: float = 0.146,
-             seed: int = BASE_SEED + 3) -> Workload:
+             seed: int = BASE_SEED + 3, ret_per_group: int = 0) -> Workload:
     rng = _rng(seed)
-    heads = HeadMap(n_q_heads, n_kv_heads, list(ret_kv_heads), n_sink=4, window=window)
+    heads = HeadMap(n_q_heads, n_kv_heads, list(ret_kv_heads), n_sink=4, window=window, ret_per_group=ret_per_group)
     U = []
     for _ in range(n_kv_heads):
         a, _r = np.linalg.qr(rng.standard_normal((HEAD_DIM, INDEX_DIM)))

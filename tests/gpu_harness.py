@@ -303,6 +303,8 @@ def check_range_attention(dw: DeviceWorkload, out, lse, kv_heads, kind: str, row
         for kv in kv_heads:
             for j in range(g):
                 h = kv * g + j
+                if kind == "local" and h in wl.heads.ret_q_heads:
+                    continue                      # a retrieval head inside a mixed group: not the local call's
                 if kind == "local":
                     want, wlse = orc.local_row(wl.q[r, h], wl.k[b][:, kv], wl.v[b][:, kv], m, wl.heads.n_sink,
                                                wl.heads.window, wl.sm_scale)
@@ -429,6 +431,8 @@ def check_prefill_rows(pr: PrefillRun, q_start: int, out, lse, rows, kind: str, 
         for kv in kv_heads:
             for j in range(g):
                 h = kv * g + j
+                if kind == "local" and h in wl.heads.ret_q_heads:
+                    continue
                 if kind == "local":
                     want, wlse = orc.local_row(wl.q[m, h], wl.k[0][:, kv], wl.v[0][:, kv], m, wl.heads.n_sink,
                                                wl.heads.window, wl.sm_scale)

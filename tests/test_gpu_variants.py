@@ -139,3 +139,95 @@ def test_chunk_and_block_forms_reject_the_variants():
     with pytest.raises(rb.RtpError) as e:
         pr.select_chunk(256, 256)
     assert e.value.code == rb.RTP_ERR_UNSUPPORTED
+
+
+# ---- mixed groups: retrieval and local query heads on one KV head (Section 3.2: the partition is over query heads) ----
+def test_mixed_group_decode():
+    """KV heads 0 and 1: two of the four query heads are retrieval heads, the other two attend locally."""
+    gh = _harness()
+    wl = synth.config_2(L=3000, batch=4, window=512, ret_per_group=2)
+    assert wl.heads.ret_q_heads == [0, 1, 4, 5] and wl.heads.local_kv_heads == list(range(8))
+    dw = gh.DeviceWorkload(wl)
+    dw.index_all_keys()
+    qt = gh.check_queries(dw)
+    sc = gh.check_scores(dw, qt)
+    sel = dw.select()
+    gh.check_selection(dw, sc, sel)
+    # both calls write into ONE output: each must leave the other's heads alone
+    out = torch.full((dw.R, 32, 128), 7.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((dw.R, 32), 7.0, dtype=torch.float32, device="cuda")
+    rb.rtp_local_attn(dw.ctx, dw.params, dw.cache, dw.q, dw.row_seq, dw.row_pos, 0, 0, dw.R, out, lse, dw.workspace,
+                      dw.status)
+    torch.cuda.synchronize()
+    o = out.float().cpu().numpy()
+    assert np.all(o[:, wl.heads.ret_q_heads] == 7.0) and np.all(lse.cpu().numpy()[:, wl.heads.ret_q_heads] == 7.0)
+    rb.rtp_sparse_attn_decode(dw.ctx, dw.params, dw.cache, dw.q, dw.row_seq, dw.row_pos, sel["idx"], sel["cnt"], out,
+                              lse, dw.workspace, dw.status)
+    torch.cuda.synchronize()
+    o, l = out.float().cpu().numpy(), lse.cpu().numpy()
+    gh.check_sparse_attention(dw, sel, o, l)
+    gh.check_range_attention(dw, o, l, [0, 1, 5], "local")          # heads 2, 3, 6, 7 of the mixed groups and a plain one
+    assert dw.status_code() == rb.RTP_OK
+
+
+def test_mixed_group_decode_long_context_split_kv():
+    """Long enough for the local call to split the window over several CTAs (the merge kernel must skip too)."""
+    gh = _harness()
+    wl = synth.config_2(L=20000, batch=2, window=8192, ret_per_group=1)
+    dw = gh.DeviceWorkload(wl)
+    dw.index_all_keys()
+    out = torch.full((dw.R, 32, 128), 7.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((dw.R, 32), 7.0, dtype=torch.float32, device="cuda")
+    rb.rtp_local_attn(dw.ctx, dw.params, dw.cache, dw.q, dw.row_seq, dw.row_pos, 0, 0, dw.R, out, lse, dw.workspace,
+                      dw.status)
+    torch.cuda.synchronize()
+    o, l = out.float().cpu().numpy(), lse.cpu().numpy()
+    assert wl.heads.ret_q_heads == [0, 4]
+    assert np.all(o[:, [0, 4]] == 7.0) and np.all(l[:, [0, 4]] == 7.0)
+    gh.check_range_attention(dw, o, l, [0, 1], "local")
+    assert dw.status_code() == rb.RTP_OK
+
+
+def test_mixed_group_prefill_lists_and_local():
+    gh = _harness()
+    wl = synth.config_3(L=768, window=128, ret_per_group=2)
+    dw = gh.DeviceWorkload(wl)
+    dw.index_all_keys()
+    pr = gh.PrefillRun(dw)
+    sel = pr.select_chunk(256, 512, with_lists=True)
+    rows = [256, 500, 767]
+    gh.check_chunk_selection(pr, 256, sel, rows)
+    idx, cnt = sel["idx"].cpu().numpy(), sel["cnt"].cpu().numpy()
+    sets = {(m, i): idx[m - 256, i, : cnt[m - 256, i]] for m in rows for i in range(dw.n_ret)}
+    o, l = pr.sparse_prefill(256, 512, sel, use_lists=True)
+    gh.check_prefill_rows(pr, 256, o, l, rows, "sparse", None, sets)
+    o, l = pr.local_prefill(256, 512)
+    assert np.all(o[:, wl.heads.ret_q_heads] == 0)              # (the harness zero-fills the output)
+    gh.check_prefill_rows(pr, 256, o, l, rows, "local", [0, 1, 4])
+    # the threshold form needs index heads that cover whole groups
+    with pytest.raises(rb.RtpError) as e:
+        pr.sparse_prefill(256, 512, sel, use_lists=False)
+    assert e.value.code == rb.RTP_ERR_UNSUPPORTED
+    assert dw.status_code() == rb.RTP_OK
+
+
+def test_mixed_group_cannot_use_the_truncated_pool():
+    wl = synth.config_2(L=300, batch=1, window=64, ret_per_group=2)
+    params = rb.Params.from_workload(wl)
+    dev = "cuda"
+    z = lambda *shape: torch.zeros(shape, dtype=torch.bfloat16, device=dev)
+    bt = torch.zeros((1, 8), dtype=torch.int32, device=dev)
+    lbt = torch.zeros((1, 4), dtype=torch.int32, device=dev)
+    sl = torch.full((1,), 300, dtype=torch.int32, device=dev)
+    cache = rb.make_cache(z(9, 1, 64, 128), z(9, 1, 64, 128), z(9, 2, 64, 16), bt, sl, k_local_pages=z(5, 8, 64, 128),
+                          v_local_pages=z(5, 8, 64, 128), local_block_table=lbt, sink_pages=1)
+    q = z(1, 32, 128)
+    out = z(1, 32, 128)
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    rs = torch.zeros(1, dtype=torch.int32, device=dev)
+    rp = torch.full((1,), 299, dtype=torch.int32, device=dev)
+    with pytest.raises(rb.RtpError) as e:
+        rb.rtp_local_attn(rb.Context(), params, cache, q, rs, rp, 0, 0, 1, out,
+                          torch.zeros((1, 32), dtype=torch.float32, device=dev), ws, st)
+    assert e.value.code == rb.RTP_ERR_INVALID
