@@ -31,6 +31,10 @@ What it follows
                          an optional variant that is not in Eq. 5: the first
                          n_sink and the newest n_recent keys joined to a
                          selected set (off by default: the paper forces nothing).
+* ``e4m3_encode`` / ``e4m3_decode`` / ``index_project_e4m3`` / ``index_scores_e4m3``
+                         an option that is not in the paper: the index-key cache
+                         held as 8-bit floats (E4M3), Eq. 4 evaluated on the
+                         decoded keys.
 * ``attention_over_set`` Eq. 5, softmax(q.k/sqrt(d_h)) restricted to S, times V.
 * ``local_set``          Section 3.2 / Table 2: attention sinks plus a sliding
                          window on local heads.
@@ -56,7 +60,9 @@ equal blocks, one dominant block, block size 1 against the token-level rule,
 brute force over all block subsets in m_b order; for the fixed-budget selector:
 numpy's argpartition on distinct scores, the count rule, the tie rule on equal
 scores, agreement with Top-P at the p that its own mass defines; for the forced
-positions: their number in closed form and the subset / union laws.  The selection statistics the
+positions: their number in closed form and the subset / union laws; for the 8-bit
+keys: all codes and a dense sample of reals against torch's float8_e4m3fn
+conversion, round trip of every finite code, ties, saturation, monotonicity.  The selection statistics the
 paper prints (its Tables 1, 6, 7) depend on model activations that are not
 available: parity unpinned for those numbers; they only shape synthetic data.
 
@@ -106,6 +112,48 @@ def index_scores(qt_bf16: np.ndarray, kt_bf16: np.ndarray, score_scale: float = 
     """
     q = bf16_to_f64(qt_bf16)
     k = bf16_to_f64(kt_bf16)
+    return (float(score_scale) * (k @ q)).astype(np.float32)
+
+
+# ---------------------------------------------------------------- 8-bit index keys (an option, not in the paper)
+# The index-key cache may hold the projected keys as 8-bit floats, 16 bytes per token and index head: the format is
+# E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities; codes 0x7f / 0xff are NaN; largest
+# finite magnitude 448; subnormals m / 8 * 2^-6).
+def e4m3_decode(c: np.ndarray) -> np.ndarray:
+    """E4M3 codes (uint8) -> float64, exactly."""
+    c = np.asarray(c, dtype=np.uint8).astype(np.int64)
+    e, m = (c >> 3) & 15, c & 7
+    mag = np.where(e == 0, (m / 8.0) * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64)))
+    mag = np.where((c & 0x7F) == 0x7F, np.nan, mag)
+    return np.where((c >> 7) == 1, -mag, mag)
+
+
+def e4m3_encode(x: np.ndarray) -> np.ndarray:
+    """Finite reals -> E4M3 codes: the nearest representable value, a tie going to the code with an even mantissa,
+    magnitudes beyond 448 saturating at 448; the sign bit is the sign of x (so a small negative number gives -0)."""
+    x = np.asarray(x, dtype=np.float64)
+    grid = e4m3_decode(np.arange(0, 127, dtype=np.uint8))          # the 127 finite non-negative values, ascending
+    a = np.minimum(np.abs(x), 448.0)
+    hi = np.clip(np.searchsorted(grid, a, side="left"), 1, 126)     # grid[hi-1] <= a <= grid[hi] (or a == grid[0])
+    lo = hi - 1
+    d_lo, d_hi = a - grid[lo], grid[hi] - a
+    code = np.where(d_lo < d_hi, lo, np.where(d_hi < d_lo, hi, np.where(lo % 2 == 0, lo, hi)))
+    return (code | np.where(np.signbit(x), 0x80, 0)).astype(np.uint8)
+
+
+def index_project_e4m3(x_bf16: np.ndarray, w_bf16: np.ndarray) -> np.ndarray:
+    """The projection of ``index_project`` stored as E4M3 codes: the fp64 sum is rounded to fp32, then encoded."""
+    y = (bf16_to_f64(x_bf16) @ bf16_to_f64(w_bf16)).astype(np.float32)
+    return e4m3_encode(y)
+
+
+def index_scores_e4m3(qt_bf16: np.ndarray, k8: np.ndarray, score_scale: float = 1.0) -> np.ndarray:
+    """Scores of one query row against 8-bit index keys: the bf16 projected query is taken in fp16 (exact for
+    magnitudes in [2^-14, 65504], which is every value a projection produces in practice; smaller ones round to
+    multiples of 2^-24), the keys are decoded exactly; the 16-term sum and the temperature are applied in fp64 and
+    the result is rounded once, as for bf16 keys."""
+    q = bf16_to_f64(qt_bf16).astype(np.float16).astype(np.float64)
+    k = e4m3_decode(k8)
     return (float(score_scale) * (k @ q)).astype(np.float32)
 
 
