@@ -249,29 +249,49 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
             ts.append(ev_time_ms(fn, stream) * 1e3)
         return float(np.median(ts))
 
+    def graph_timed(pth):
+        """The same step replayed from a CUDA graph (the library calls captured once): no host launch cost."""
+        try:
+            graph = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream(device=device)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                pth.step(data.q, k_pre_new)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph):
+                pth.step(data.q, k_pre_new)
+            return timed(graph.replay)
+        except Exception as exc:   # capture is an extra; the plain numbers stand on their own
+            return f"not captured: {type(exc).__name__}"
+
     t_sparse = timed(lambda: path.step(data.q, k_pre_new))
     t_dense = timed(lambda: path.step_dense(data.q))
-    # the same sparse step replayed from a CUDA graph (the four library calls captured once): no host launch cost
-    t_graph = None
-    try:
-        graph = torch.cuda.CUDAGraph()
-        side = torch.cuda.Stream(device=device)
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            path.step(data.q, k_pre_new)
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-        with torch.cuda.graph(graph):
-            path.step(data.q, k_pre_new)
-        t_graph = timed(graph.replay)
-    except Exception as exc:   # capture is an extra; the plain numbers above stand on their own
-        t_graph = f"not captured: {type(exc).__name__}"
+    t_graph = graph_timed(path)
     # the fixed-budget variant the paper compares with (Section 4.1, k = 4096), same data and step
     path_k = pipeline.DecodePath(data, max(stride, 4096), top_k=4096)
     path_k.build_index_cache()
     t_topk = timed(lambda: path_k.step(data.q, k_pre_new))
+    t_topk_graph = graph_timed(path_k)
     topk_status = path_k.status_code()
     del path_k
+    # the 8-bit index-key cache (16 bytes per token and index head): same data, same step; how much of the bf16
+    # selection it reproduces is reported beside the time
+    path_8 = pipeline.DecodePath(data, stride, ikey_e4m3=True)
+    path_8.build_index_cache()
+    t_ikey8 = timed(lambda: path_8.step(data.q, k_pre_new))
+    t_ikey8_graph = graph_timed(path_8)
+    ikey8_status = path_8.status_code()
+    inter = total = 0
+    for b_ in range(min(B, 4)):
+        for i_ in range(path.n_ret):
+            s16 = path.sel_idx[b_, i_, : int(path.sel_cnt[b_, i_])]
+            s8 = path_8.sel_idx[b_, i_, : int(path_8.sel_cnt[b_, i_])]
+            inter += int(torch.isin(s8, s16).sum().item())
+            total += int(s16.numel())
+    ikey8_overlap = inter / max(1, total)
+    ikey8_count_ratio = float(path_8.sel_cnt.float().mean().item()) / max(1.0, float(path.sel_cnt.float().mean().item()))
+    del path_8
     cnt = path.sel_cnt.float()
     n_ih = data.heads.n_index_heads
     sel_rows = float(cnt.sum().item())
@@ -281,7 +301,10 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
            "selected_fraction_mean": float(cnt.mean().item()) / L,
            "sparse_step_us": t_sparse, "sparse_step_us_cuda_graph": t_graph, "dense_step_us": t_dense,
            "speedup_vs_dense": t_dense / t_sparse,
-           "fixed_budget_4096_step_us": t_topk, "fixed_budget_status": topk_status,
+           "fixed_budget_4096_step_us": t_topk, "fixed_budget_4096_step_us_cuda_graph": t_topk_graph,
+           "fixed_budget_status": topk_status,
+           "ikey_e4m3_step_us": t_ikey8, "ikey_e4m3_step_us_cuda_graph": t_ikey8_graph, "ikey_e4m3_status": ikey8_status,
+           "ikey_e4m3_share_of_bf16_set_kept": ikey8_overlap, "ikey_e4m3_count_ratio": ikey8_count_ratio,
            "algorithmic_bytes": alg_bytes, "sparse_path_gbs": alg_bytes / t_sparse / 1e3,
            "dense_gbs": B * data.heads.n_kv_heads * 512.0 * L / t_dense / 1e3,
            "status": path.status_code()}

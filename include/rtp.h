@@ -109,7 +109,7 @@ typedef struct rtp_params {
 typedef struct rtp_cache {
   void* k_pages;              /* DEVICE bf16 [num_pages, n_kv_heads, 64, 128] */
   void* v_pages;              /* DEVICE bf16 [num_pages, n_kv_heads, 64, 128] */
-  void* ikey_pages;           /* DEVICE bf16 [num_pages, n_index_heads, 64, 16] */
+  void* ikey_pages;           /* DEVICE bf16 [num_pages, n_index_heads, 64, 16]; see ikey_format */
   const int32_t* block_table; /* DEVICE int32 [batch, max_pages] physical page ids */
   const int32_t* seq_lens;    /* DEVICE int32 [batch] tokens present per sequence */
   int32_t num_pages;
@@ -135,7 +135,19 @@ typedef struct rtp_cache {
   int32_t n_local_pages;
   int32_t sink_pages;
   int32_t ring_pages;
+  /* Storage type of the index-key cache.  RTP_IKEY_BF16 (0): bf16, 32 bytes per token and index head.
+   * RTP_IKEY_E4M3 (1): 8-bit floats (1 sign, 4 exponent, 3 mantissa bits, bias 7, largest magnitude 448, no
+   * infinities), uint8 [num_pages, n_index_heads, 64, 16], 16 bytes per token and index head: half the bytes of the
+   * decode scan.  rtp_index_keys then stores the fp32 projection rounded to the nearest E4M3 value (ties to even,
+   * saturating); rtp_index_score and the row form of rtp_topp_select evaluate Eq. 4 on the decoded keys, with the
+   * projected queries taken in fp16 (RTP_ERR_UNSUPPORTED in the status word if one exceeds 65504 in magnitude).  The
+   * chunk form of rtp_topp_select, rtp_topp_select_blocks and the threshold form of rtp_sparse_attn_prefill need
+   * the bf16 cache (RTP_ERR_UNSUPPORTED): the paper's method selects in decode only. */
+  int32_t ikey_format;
 } rtp_cache;
+
+#define RTP_IKEY_BF16 0
+#define RTP_IKEY_E4M3 1
 
 /* ---- utility ------------------------------------------------------------ */
 

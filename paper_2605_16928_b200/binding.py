@@ -16,6 +16,7 @@ _PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG_DIR, "librtp.so")
 
 RTP_OK, RTP_ERR_INVALID, RTP_ERR_CAPACITY, RTP_ERR_UNSUPPORTED, RTP_ERR_CUDA, RTP_ERR_TIMEOUT = range(6)
+RTP_IKEY_BF16, RTP_IKEY_E4M3 = 0, 1
 _STATUS_NAMES = ["RTP_OK", "RTP_ERR_INVALID", "RTP_ERR_CAPACITY", "RTP_ERR_UNSUPPORTED", "RTP_ERR_CUDA",
                  "RTP_ERR_TIMEOUT"]
 
@@ -54,6 +55,7 @@ class RtpCache(C.Structure):
         ("num_pages", C.c_int32), ("batch", C.c_int32), ("max_pages", C.c_int32),
         ("k_local_pages", C.c_void_p), ("v_local_pages", C.c_void_p), ("local_block_table", C.c_void_p),
         ("n_local_pages", C.c_int32), ("sink_pages", C.c_int32), ("ring_pages", C.c_int32),
+        ("ikey_format", C.c_int32),
     ]
 
 
@@ -178,18 +180,21 @@ class Params:
 
 
 def make_cache(k_pages, v_pages, ikey_pages, block_table, seq_lens, k_local_pages=None, v_local_pages=None,
-               local_block_table=None, sink_pages: int = 0) -> RtpCache:
+               local_block_table=None, sink_pages: int = 0, ikey_format: Optional[int] = None) -> RtpCache:
     """Describes caller-owned paged caches (torch CUDA tensors) to the library.  With ``k_local_pages`` the cache is
     truncated for local heads: ``k_pages`` / ``v_pages`` hold the other KV heads only, the local heads live in the
     local pool behind ``local_block_table`` [batch, sink_pages + ring_pages]."""
     num_pages = int((k_pages if k_pages is not None else ikey_pages).shape[0])
+    if ikey_format is None:   # the tensor's element size says which: uint8 pages are E4M3 codes
+        ikey_format = RTP_IKEY_E4M3 if (ikey_pages is not None and ikey_pages.element_size() == 1) else RTP_IKEY_BF16
     n_local, ring = 0, 0
     if k_local_pages is not None:
         n_local = int(k_local_pages.shape[0])
         ring = int(local_block_table.shape[1]) - int(sink_pages)
     return RtpCache(_ptr(k_pages), _ptr(v_pages), _ptr(ikey_pages), _ptr(block_table), _ptr(seq_lens),
                     num_pages, int(block_table.shape[0]), int(block_table.shape[1]),
-                    _ptr(k_local_pages), _ptr(v_local_pages), _ptr(local_block_table), n_local, int(sink_pages), ring)
+                    _ptr(k_local_pages), _ptr(v_local_pages), _ptr(local_block_table), n_local, int(sink_pages), ring,
+                    int(ikey_format))
 
 
 class Context:

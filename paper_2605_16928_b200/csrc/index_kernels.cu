@@ -57,7 +57,11 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(
     if (seq < 0 || seq >= cv.batch || pos < 0 || (pos >> kPageShift) >= cv.max_pages) return;
     const int phys = cv.block_table[(int64_t)seq * cv.max_pages + (pos >> kPageShift)];
     if (phys < 0 || phys >= cv.num_pages) return;
-    cv.ikey[(((int64_t)phys * cv.n_ih + head) * kPage + (pos & (kPage - 1))) * kIndexDim + j] = o;
+    const int64_t at = (((int64_t)phys * cv.n_ih + head) * kPage + (pos & (kPage - 1))) * kIndexDim + j;
+    if (cv.ikey_fp8)   // the fp32 sum straight to E4M3: nearest, ties to even, saturating at 448
+      reinterpret_cast<uint8_t*>(cv.ikey)[at] = (uint8_t)__nv_cvt_float_to_fp8(acc, __NV_SATFINITE, __NV_E4M3);
+    else
+      cv.ikey[at] = o;
   } else {
     qt[(t * d.n_ret + head) * kIndexDim + j] = o;
   }
@@ -100,6 +104,7 @@ constexpr int kScoreWarps = 4;
 
 // grid = (R * n_ih, splits).  Each CTA scans a contiguous range of pages of one (row, index head)
 // for all retrieval heads attached to that index head.
+template <bool F8>
 __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(
     CacheView cv, Dims d, HeadMaps hm, Rows rows, const __nv_bfloat16* __restrict__ qt,
     float* __restrict__ scores, int64_t score_stride, float2* __restrict__ partial, int n_splits,
@@ -125,20 +130,28 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(
   const int p_lo = split * per;
   const int p_hi = min(n_pages, p_lo + per);
 
-  const QFrag qf = load_qfrag(qt + r * d.n_ret * kIndexDim, hm.ih_heads[ih], nh, lane);
+  QFrag qf = load_qfrag(qt + r * d.n_ret * kIndexDim, hm.ih_heads[ih], nh, lane);
+  if (F8 && !qfrag_to_f16(qf)) set_status(status, RTP_ERR_UNSUPPORTED);   // a projected query beyond fp16's range
   const int head_lo = g < nh ? hm.ih_heads[ih][g] : -1;
   const int head_hi = g + 8 < nh ? hm.ih_heads[ih][g + 8] : -1;
   float m_lo = -INFINITY, l_lo = 0.f, m_hi = -INFINITY, l_hi = 0.f;
 
   for (int p = p_lo + warp; p < p_hi; p += kScoreWarps) {
-    const __nv_bfloat16* base = ikey_page_ptr(cv, seq, p, ih);
     uint4 v[4];
+    uint2 v8[4];
+    if (F8) {
+      const uint8_t* base = ikey_page_ptr8(cv, seq, p, ih);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) v[i] = ld_stream_v4(base + (i * 32 + lane) * 8);
+      for (int i = 0; i < 4; ++i) v8[i] = ld_stream_v2(base + (i * 32 + lane) * 8);
+    } else {
+      const __nv_bfloat16* base = ikey_page_ptr(cv, seq, p, ih);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) v[i] = ld_stream_v4(base + (i * 32 + lane) * 8);
+    }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       float s_lo[4], s_hi[4];
-      score16(qf, v[i], lane, s_lo, s_hi);
+      if (F8) score16_f8(qf, v8[i], lane, s_lo, s_hi); else score16(qf, v[i], lane, s_lo, s_hi);
       const int n0 = p * kPage + i * 16 + 4 * c;
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -262,8 +275,12 @@ cudaError_t launch_index_score(const CacheView& cv, const Dims& d, const HeadMap
   if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
   const int n_splits = score_splits(d, rows.R, max_len, sm_count);
   dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
-  score_kernel<<<grid, kScoreWarps * 32, 0, st>>>(cv, d, hm, rows, qt, scores, score_stride,
-                                                  reinterpret_cast<float2*>(ws), n_splits, status);
+  if (cv.ikey_fp8)
+    score_kernel<true><<<grid, kScoreWarps * 32, 0, st>>>(cv, d, hm, rows, qt, scores, score_stride,
+                                                          reinterpret_cast<float2*>(ws), n_splits, status);
+  else
+    score_kernel<false><<<grid, kScoreWarps * 32, 0, st>>>(cv, d, hm, rows, qt, scores, score_stride,
+                                                           reinterpret_cast<float2*>(ws), n_splits, status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (row_max || row_sum) {

@@ -113,6 +113,8 @@ const char* check_cache(const rtp_cache* c, const rtp_params* p, bool need_kv, b
   cv->cap_tokens = (int32_t)std::min<int64_t>((int64_t)c->max_pages * kPage, 0x7fffffff);
   cv->sink_pages = 0;
   cv->ring_pages = 0;
+  if (c->ikey_format != RTP_IKEY_BF16 && c->ikey_format != RTP_IKEY_E4M3) return "unknown ikey_format";
+  cv->ikey_fp8 = c->ikey_format == RTP_IKEY_E4M3;
   for (int h = 0; h < 32; ++h) cv->kv_slot[h] = h < p->n_kv_heads ? (uint8_t)h : (uint8_t)0xff;
   if (c->k_local_pages) {
     // truncated layout: the main pool holds the KV heads that are not local, in increasing order
@@ -361,6 +363,7 @@ rtp_status rtp_topp_select(rtp_ctx* ctx, const rtp_params* params, const rtp_cac
   __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(w.take(qt_bytes(d, R)));
   const bool chunk = row_seq == nullptr;
   if (chunk && variant_set(d)) return fail(ctx, RTP_ERR_UNSUPPORTED, "top_k / forced positions: row lists only");
+  if (chunk && cv.ikey_fp8) return fail(ctx, RTP_ERR_UNSUPPORTED, "8-bit index keys: row form only");
   const size_t sel_off = w.off;
   void* sel_ws = w.take(chunk ? select_chunk_workspace_bytes(d, hm, R) : select_rows_workspace_bytes(d, R, max_len));
   if (w.off > workspace_bytes) return fail(ctx, RTP_ERR_CAPACITY, "workspace too small");
@@ -446,6 +449,7 @@ rtp_status rtp_sparse_attn_prefill(rtp_ctx* ctx, const rtp_params* params, const
   }
   if (!sel_thresh || !sel_tie_last || !q_pre || !w_q || !workspace)
     return fail(ctx, RTP_ERR_INVALID, "threshold mode needs sel_thresh, sel_tie_last, q_pre, w_q and a workspace");
+  if (cv.ikey_fp8) return fail(ctx, RTP_ERR_UNSUPPORTED, "8-bit index keys: list form only");
   if (variant_set(d)) return fail(ctx, RTP_ERR_UNSUPPORTED, "top_k / forced positions: row lists only");
   if (!aligned16(q_pre) || !aligned16(w_q)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
   WsCarver w(workspace);
@@ -484,6 +488,7 @@ rtp_status rtp_topp_select_blocks(rtp_ctx* ctx, const rtp_params* params, const 
   if (!q_pre || !w_q || !workspace || !sel_count || !block_mask) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
   if (!aligned16(q_pre) || !aligned16(w_q) || !aligned16(workspace)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
   if (mask_words * 32 < ((int64_t)q_start + C + kPage - 1) / kPage) return fail(ctx, RTP_ERR_CAPACITY, "mask_words too small for the chunk's pages");
+  if (cv.ikey_fp8) return fail(ctx, RTP_ERR_UNSUPPORTED, "8-bit index keys: row form of the selection only");
   if (variant_set(d)) return fail(ctx, RTP_ERR_UNSUPPORTED, "top_k / forced positions: row lists only");
   WsCarver w(workspace);
   __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(w.take(qt_bytes(d, C)));

@@ -27,6 +27,11 @@ __device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
                : "l"(p));
   return v;
 }
+__device__ __forceinline__ uint2 ld_stream_v2(const void* p) {
+  uint2 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+  return v;
+}
 __device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
   uint4 v;
   asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -97,6 +102,60 @@ __device__ __forceinline__ void score16(const QFrag& q, const uint4& v, int lane
   float t0[4], t1[4];
   mma_bf16_16816(t0, q.a0, q.a1, q.a2, q.a3, e0, e1, zero);
   mma_bf16_16816(t1, q.a0, q.a1, q.a2, q.a3, o0, o1, zero);
+  s_lo[0] = t0[0]; s_lo[1] = t1[0]; s_lo[2] = t0[1]; s_lo[3] = t1[1];
+  s_hi[0] = t0[2]; s_hi[1] = t1[2]; s_hi[2] = t0[3]; s_hi[3] = t1[3];
+}
+
+// ---- the same core on 8-bit (E4M3) index keys ----
+// A 16-key group is 256 contiguous bytes, one 8-byte load per lane (lane l holds bytes [8 l, 8 l + 8): eight
+// dimensions of key l / 2).  The codes are widened to fp16 (exact) and the MMA runs on fp16 operands; the projected
+// queries are converted bf16 -> fp16 once (exact for magnitudes in [2^-14, 65504]).  The output layout is score16()'s.
+__device__ __forceinline__ void mma_f16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1, const float (&c)[4]) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%10,%11,%12,%13};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
+}
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t b, bool& overflow) {
+  const float lo = __uint_as_float(b << 16), hi = __uint_as_float(b & 0xffff0000u);
+  overflow = overflow || !(fabsf(lo) <= 65504.0f) || !(fabsf(hi) <= 65504.0f);
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+// Returns false when a projected query does not fit fp16 (the caller reports RTP_ERR_UNSUPPORTED).
+__device__ __forceinline__ bool qfrag_to_f16(QFrag& f) {
+  bool overflow = false;
+  f.a0 = bf16x2_to_f16x2(f.a0, overflow);
+  f.a1 = bf16x2_to_f16x2(f.a1, overflow);
+  f.a2 = bf16x2_to_f16x2(f.a2, overflow);
+  f.a3 = bf16x2_to_f16x2(f.a3, overflow);
+  return !overflow;
+}
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes) {
+  uint32_t r;
+  asm("{ .reg .b16 t; cvt.u16.u32 t, %1; cvt.rn.f16x2.e4m3x2 %0, t; }" : "=r"(r) : "r"(two_codes));
+  return r;
+}
+__device__ __forceinline__ void score16_f8(const QFrag& q, const uint2& raw, int lane, float (&s_lo)[4],
+                                           float (&s_hi)[4]) {
+  uint4 v;   // the lane's eight dimensions as fp16, in the order score16() expects them
+  v.x = e4m3x2_to_f16x2(raw.x);
+  v.y = e4m3x2_to_f16x2(raw.x >> 16);
+  v.z = e4m3x2_to_f16x2(raw.y);
+  v.w = e4m3x2_to_f16x2(raw.y >> 16);
+  const bool u = (lane & 2) != 0;
+  const uint32_t send0 = u ? v.x : v.z;
+  const uint32_t send1 = u ? v.y : v.w;
+  const uint32_t r0 = __shfl_xor_sync(0xffffffffu, send0, 2);
+  const uint32_t r1 = __shfl_xor_sync(0xffffffffu, send1, 2);
+  const uint32_t e0 = u ? r0 : v.x, e1 = u ? r1 : v.y;
+  const uint32_t o0 = u ? v.z : r0, o1 = u ? v.w : r1;
+  const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+  float t0[4], t1[4];
+  mma_f16_16816(t0, q.a0, q.a1, q.a2, q.a3, e0, e1, zero);
+  mma_f16_16816(t1, q.a0, q.a1, q.a2, q.a3, o0, o1, zero);
   s_lo[0] = t0[0]; s_lo[1] = t1[0]; s_lo[2] = t0[1]; s_lo[3] = t1[1];
   s_hi[0] = t0[2]; s_hi[1] = t1[2]; s_hi[2] = t0[3]; s_hi[3] = t1[3];
 }
@@ -185,6 +244,12 @@ __device__ __forceinline__ const __nv_bfloat16* ikey_page_ptr(const CacheView& c
                                                                int ih) {
   const int phys = safe_phys(cv, (int64_t)seq * cv.max_pages + page);
   return cv.ikey + ((int64_t)phys * cv.n_ih + ih) * (kPage * kIndexDim);
+}
+
+// The same for an 8-bit index-key cache (1 KB per page and index head).
+__device__ __forceinline__ const uint8_t* ikey_page_ptr8(const CacheView& cv, int seq, int page, int ih) {
+  const int phys = safe_phys(cv, (int64_t)seq * cv.max_pages + page);
+  return reinterpret_cast<const uint8_t*>(cv.ikey) + ((int64_t)phys * cv.n_ih + ih) * (kPage * kIndexDim);
 }
 
 // 2^x on the special-function unit (about 2 ulp; inputs of -inf give 0).

@@ -4,6 +4,8 @@
 #include <utility>
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -52,6 +54,8 @@ struct CacheView {
   // inside a page of this pool (0xff: the head is not stored here).
   int32_t cap_tokens, sink_pages, ring_pages;
   uint8_t kv_slot[32];
+  // != 0: the index-key cache holds 8-bit floats (E4M3), 16 bytes per token and index head, instead of bf16
+  int32_t ikey_fp8;
 };
 
 struct Dims {

@@ -52,11 +52,23 @@ __device__ __forceinline__ RowCtx make_row_ctx(const CacheView& cv, const Dims& 
   return x;
 }
 
-// One 64-key page of index keys: 2 KB, four 16-byte loads per lane.
+// One 64-key page of index keys: 2 KB, four 16-byte loads per lane (bf16), or 1 KB, four 8-byte loads (E4M3: the
+// upper half of each uint4 stays unused).
+template <bool F8>
 __device__ __forceinline__ void load_page(const CacheView& cv, const RowCtx& x, int p, int lane, uint4 (&v)[4]) {
-  const __nv_bfloat16* base = ikey_page_ptr(cv, x.seq, p, x.ih);
+  if (F8) {
+    const uint8_t* base = ikey_page_ptr8(cv, x.seq, p, x.ih);
 #pragma unroll
-  for (int i = 0; i < 4; ++i) v[i] = ld_stream_v4(base + (i * 32 + lane) * 8);
+    for (int i = 0; i < 4; ++i) {
+      const uint2 t = ld_stream_v2(base + (i * 32 + lane) * 8);
+      v[i].x = t.x;
+      v[i].y = t.y;
+    }
+  } else {
+    const __nv_bfloat16* base = ikey_page_ptr(cv, x.seq, p, x.ih);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = ld_stream_v4(base + (i * 32 + lane) * 8);
+  }
 }
 
 __global__ void sel_init_kernel(const CacheView cv, const Dims d, const Rows rows, SelState* state,
@@ -138,7 +150,7 @@ __device__ __forceinline__ bool take_last_ticket(uint32_t* ticket, uint32_t n_ct
 
 // ---- pass 1: scores of the unit's keys, written once for the later passes, and the row maximum -----------------------
 // scores: float [rows * retrieval heads][l_pad]; entry n of a row holds finish_score(q~ . k~_n) for n < n_keys.
-template <bool NH4>
+template <bool NH4, bool F8>
 __global__ void __launch_bounds__(kThreads) sel_score_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
                                                              const Rows rows, const __nv_bfloat16* __restrict__ qt,
                                                              SelState* __restrict__ state, float* __restrict__ scores,
@@ -148,22 +160,23 @@ __global__ void __launch_bounds__(kThreads) sel_score_kernel(const CacheView cv,
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, status);
   if (x.p_lo >= x.p_hi) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
+  QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
+  if (F8 && !qfrag_to_f16(qf)) set_status(status, RTP_ERR_UNSUPPORTED);   // a projected query beyond fp16's range
   const int slot_a = elem_slot<NH4>(lane, 0), slot_b = NH4 ? slot_a : elem_slot<NH4>(lane, 4);
   float* row_a = slot_a < x.nh ? scores + (x.r * d.n_ret + hm.ih_heads[x.ih][slot_a]) * l_pad : nullptr;
   float* row_b = (!NH4 && slot_b < x.nh) ? scores + (x.r * d.n_ret + hm.ih_heads[x.ih][slot_b]) * l_pad : nullptr;
   float mx_a = -INFINITY, mx_b = -INFINITY;
   uint4 v[4], vn[4];
-  if (x.p_lo + warp < x.p_hi) load_page(cv, x, x.p_lo + warp, lane, vn);
+  if (x.p_lo + warp < x.p_hi) load_page<F8>(cv, x, x.p_lo + warp, lane, vn);
   for (int p = x.p_lo + warp; p < x.p_hi; p += kWarps) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) v[i] = vn[i];
-    if (p + kWarps < x.p_hi) load_page(cv, x, p + kWarps, lane, vn);   // in flight while this page is worked on
+    if (p + kWarps < x.p_hi) load_page<F8>(cv, x, p + kWarps, lane, vn);   // in flight while this page is worked on
     const bool tail = (p + 1) * kPage > x.n_keys;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       float s_lo[4], s_hi[4];
-      score16(qf, v[i], lane, s_lo, s_hi);
+      if (F8) score16_f8(qf, make_uint2(v[i].x, v[i].y), lane, s_lo, s_hi); else score16(qf, v[i], lane, s_lo, s_hi);
       const LaneElems<NH4> el = lane_elems<NH4>(s_lo, s_hi, lane);
       const int n0 = p * kPage + i * 16 + el.koff[0];
       // (a page lies inside l_pad whatever n_keys is: entries beyond the row's keys are written and never read)
@@ -1123,10 +1136,14 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
   const int n_splits = select_splits(d, rows.R, max_len, sm_count);
   const dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
   // one scan of the index keys (scores stored, row maxima), then three passes over the stored scores
-  if (max_nh <= 4)
-    (void)launch_chained(sel_score_kernel<true>, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status);
-  else
-    (void)launch_chained(sel_score_kernel<false>, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status);
+#define RTP_SCORE(NH4_, F8_) \
+  (void)launch_chained(sel_score_kernel<NH4_, F8_>, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, qt, w.state, w.scores, l_pad, n_splits, status)
+  if (max_nh <= 4) {
+    if (cv.ikey_fp8) RTP_SCORE(true, true); else RTP_SCORE(true, false);
+  } else {
+    if (cv.ikey_fp8) RTP_SCORE(false, true); else RTP_SCORE(false, false);
+  }
+#undef RTP_SCORE
   (void)launch_chained(sel_l1_kernel, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.tickets, n_splits, list_cap, status);
   (void)launch_chained(sel_key_kernel, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.g_cnt, w.tickets,
                                             n_splits, 1 + kKeyLevels, list_cap, status);

@@ -14,14 +14,16 @@ from . import binding as rb
 
 
 class _Base:
-    def __init__(self, data, max_rows: int, max_len: int, **param_over):
+    def __init__(self, data, max_rows: int, max_len: int, ikey_e4m3: bool = False, **param_over):
+        """ikey_e4m3: the index-key cache holds 8-bit floats (16 bytes per token and index head) instead of bf16."""
         self.data = data
         dev = data.q.device
         self.dev = dev
         self.ctx = rb.Context()
         self.params = rb.Params.from_workload(data, **param_over)
         nih = max(1, data.heads.n_index_heads)
-        self.ikey_pages = torch.zeros((data.num_pages, nih, 64, 16), dtype=torch.bfloat16, device=dev)
+        self.ikey_pages = torch.zeros((data.num_pages, nih, 64, 16),
+                                      dtype=torch.uint8 if ikey_e4m3 else torch.bfloat16, device=dev)
         self.cache = rb.make_cache(data.k_pages, data.v_pages, self.ikey_pages, data.block_table, data.seq_lens)
         ws = max(1 << 20, rb.rtp_workspace_bytes(self.params, max_rows, max_len))
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)

@@ -25,8 +25,9 @@ def dev_i32(a) -> torch.Tensor:
 
 
 class DeviceWorkload:
-    def __init__(self, wl: synth.Workload, sel_stride: int | None = None, **param_over):
+    def __init__(self, wl: synth.Workload, sel_stride: int | None = None, ikey_e4m3: bool = False, **param_over):
         self.wl = wl
+        self.f8 = ikey_e4m3
         self.ctx = rb.Context()
         self.params = rb.Params.from_workload(wl, **param_over)
         self.pc = synth.build_paged_cache(wl.k, wl.v, wl.seed)
@@ -34,7 +35,10 @@ class DeviceWorkload:
         self.v_pages = dev_bf16(self.pc.v_pages)
         nih = max(1, wl.heads.n_index_heads)
         # poison the index-key cache so that unwritten slots are noticed
-        self.ikey_pages = torch.full((self.pc.num_pages, nih, 64, 16), float("nan"), dtype=torch.bfloat16, device=DEV)
+        if ikey_e4m3:   # (0x7f is the NaN code of the 8-bit format)
+            self.ikey_pages = torch.full((self.pc.num_pages, nih, 64, 16), 0x7F, dtype=torch.uint8, device=DEV)
+        else:
+            self.ikey_pages = torch.full((self.pc.num_pages, nih, 64, 16), float("nan"), dtype=torch.bfloat16, device=DEV)
         self.block_table = dev_i32(self.pc.block_table)
         self.seq_lens = dev_i32(self.pc.seq_lens)
         self.cache = rb.make_cache(self.k_pages, self.v_pages, self.ikey_pages, self.block_table, self.seq_lens)
@@ -64,7 +68,7 @@ class DeviceWorkload:
                 tok_pos = torch.arange(lo, hi, dtype=torch.int32, device=DEV)
                 rb.rtp_index_keys(self.ctx, self.params, self.cache, kp, self.w_k, tok_seq, tok_pos)
         torch.cuda.synchronize()
-        self.ikey_host = host_u16(self.ikey_pages)
+        self.ikey_host = self.ikey_pages.cpu().numpy() if self.f8 else host_u16(self.ikey_pages)
 
     def ikeys_logical(self, seq: int) -> np.ndarray:
         return synth.gather_index_keys(self.ikey_host, self.pc.block_table, seq, int(self.wl.seq_lens[seq]))
@@ -150,6 +154,17 @@ def check_index_keys(dw: DeviceWorkload):
         got = dw.ikeys_logical(b)                                   # [L, nih, 16]
         kp = synth.k_pre_for_index_heads(wl, b)
         for j in range(wl.heads.n_index_heads):
+            if dw.f8:
+                # E4M3 codes: equal, or one step apart where the fp32 sum lies at a rounding boundary of the 8-bit grid
+                want = orc.index_project_e4m3(kp[:, j], wl.w_k[j])
+                g8, w8 = got[:, j].astype(np.int32), want.astype(np.int32)
+                order = lambda c: np.where(c & 0x80, -(c & 0x7F), c & 0x7F)
+                d = np.abs(order(g8) - order(w8))
+                assert d.max() <= 1, f"index key off by {d.max()} E4M3 steps"
+                assert not np.any((g8 & 0x7F) == 0x7F), "NaN code written"
+                total += d.size
+                equal += int((d == 0).sum())
+                continue
             want = orc.index_project(kp[:, j], wl.w_k[j])
             d = bf16_ulp_diff(got[:, j], want)
             # one bf16 step, except where cancellation leaves a result so small that the fp32
@@ -184,10 +199,14 @@ def check_scores(dw: DeviceWorkload, qt: np.ndarray, rows=None):
         kt = dw.ikeys_logical(b)
         for i in range(dw.n_ret):
             j = wl.heads.q_head_to_index_head[i]
-            want = orc.index_scores(qt[r, i], kt[: m + 1, j], wl.score_scale)
+            if dw.f8:
+                want = orc.index_scores_e4m3(qt[r, i], kt[: m + 1, j], wl.score_scale)
+                kn = np.linalg.norm(orc.e4m3_decode(kt[: m + 1, j]), axis=-1)
+            else:
+                want = orc.index_scores(qt[r, i], kt[: m + 1, j], wl.score_scale)
+                kn = np.linalg.norm(orc.bf16_to_f64(kt[: m + 1, j]), axis=-1)
             got = sc[r, i, : m + 1]
             qn = np.linalg.norm(orc.bf16_to_f64(qt[r, i]))
-            kn = np.linalg.norm(orc.bf16_to_f64(kt[: m + 1, j]), axis=-1)
             tol = 1e-3 * np.abs(want) + 1e-5 * wl.score_scale * qn * kn
             assert np.all(np.abs(got - want) <= tol), f"row {r} head {i}: max err {np.abs(got - want).max()}"
             assert np.all(np.isnan(sc[r, i, m + 1:])), "wrote past the causal range"

@@ -172,10 +172,10 @@ def test_prefill_1m_config4_sampled_rows():
             assert int(cnt_r[i]) <= 64, f"needle row {m} head {i} keeps {int(cnt_r[i])} keys"
 
 
-def _decode_point(L, B, top_p, frac, window, seqs, peaked_half=False, name="c5_decode_sweep", e2e=True):
+def _decode_point(L, B, top_p, frac, window, seqs, peaked_half=False, name="c5_decode_sweep", e2e=True, **path_kw):
     from paper_2605_16928_b200 import pipeline, synth_device
     data = synth_device.decode_device(L, B, top_p, frac, window, peaked_half=peaked_half, name=name)
-    path = pipeline.DecodePath(data, sel_stride=int(min(L, max(16384, 4 * frac * L))))
+    path = pipeline.DecodePath(data, sel_stride=int(min(L, max(16384, 4 * frac * L))), **path_kw)
     path.build_index_cache()
     k_new = torch.stack([data.k_pre_rows(b, L - 1, L)[0] for b in range(B)]).contiguous()
     path.step(data.q, k_new)
@@ -269,6 +269,11 @@ def test_decode_512k_batch4_fixed_budget_4096():
 def test_decode_128k_forced_positions():
     _decode_variant_point(131072, 2, 0.05, 4096, [0, 1], force_sink=4, force_recent=256)
     _decode_variant_point(131072, 2, 0.05, 4096, [1], top_k=4096, force_sink=4, force_recent=256)
+
+
+def test_decode_512k_batch4_8bit_index_keys():
+    """The 8-bit index-key cache at full size: sets against the oracle's Top-P on the scores of that cache."""
+    _decode_point(524288, 4, 0.9, 0.05, 4096, [0, 2], e2e=False, ikey_e4m3=True)
 
 
 def test_decode_32k_batch8_sampled_rows():
