@@ -230,6 +230,7 @@ def cpu_oracle_prefill(data, L, rows, budget_s=25.0):
 def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, iters=20):
     import torch
     from paper_2605_16928_b200 import synth_device, pipeline
+    from paper_2605_16928_b200 import binding as rb
     data = synth_device.decode_device(L, B, top_p, frac, window, device=device, peaked_half=peaked_half, name=name)
     stride = int(min(L, max(4096, 4 * frac * L)))
     path = pipeline.DecodePath(data, stride)
@@ -290,6 +291,19 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
             inter += int(torch.isin(s8, s16).sum().item())
             total += int(s16.numel())
     ikey8_overlap = inter / max(1, total)
+    # softmax mass, under the scores of the bf16 cache, of the sets chosen on the 8-bit cache (the target is top_p)
+    nb = min(B, 4)
+    sc16 = torch.empty((nb, path.n_ret, L), dtype=torch.float32, device=device)
+    rb.rtp_index_score(path.ctx, path.params, path.cache, data.q[:nb].contiguous(), data.w_q, data.row_seq[:nb].contiguous(),
+                       data.row_pos[:nb].contiguous(), sc16, None, None, path.workspace, path.status)
+    masses = []
+    for b_ in range(nb):
+        for i_ in range(path.n_ret):
+            row = sc16[b_, i_].double()
+            w = torch.exp(row - row.max())
+            ids8 = path_8.sel_idx[b_, i_, : int(path_8.sel_cnt[b_, i_])].long()
+            masses.append(float((w[ids8].sum() / w.sum()).item()))
+    del sc16
     ikey8_count_ratio = float(path_8.sel_cnt.float().mean().item()) / max(1.0, float(path.sel_cnt.float().mean().item()))
     del path_8
     cnt = path.sel_cnt.float()
@@ -305,6 +319,7 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
            "fixed_budget_status": topk_status,
            "ikey_e4m3_step_us": t_ikey8, "ikey_e4m3_step_us_cuda_graph": t_ikey8_graph, "ikey_e4m3_status": ikey8_status,
            "ikey_e4m3_share_of_bf16_set_kept": ikey8_overlap, "ikey_e4m3_count_ratio": ikey8_count_ratio,
+           "ikey_e4m3_mass_under_bf16_scores": {"mean": float(np.mean(masses)), "min": float(np.min(masses))},
            "algorithmic_bytes": alg_bytes, "sparse_path_gbs": alg_bytes / t_sparse / 1e3,
            "dense_gbs": B * data.heads.n_kv_heads * 512.0 * L / t_dense / 1e3,
            "status": path.status_code()}
