@@ -370,6 +370,31 @@ rtp_status rtp_sparse_attn_prefill_blocks(rtp_ctx* ctx, const rtp_params* params
                                           int32_t seq_id, int32_t q_start, int64_t C, const uint32_t* block_mask,
                                           int64_t mask_words, void* out, float* lse, int32_t* status, void* stream);
 
+/* The same block-wise rule for explicit rows (decode: the use Section 3.4 describes it for).
+ * rtp_topp_select_blocks_rows: rows as in rtp_topp_select with row arrays.  For every (row, retrieval head) the
+ *   selected blocks are written as LOGICAL page numbers (block b = keys 64 b .. 64 b + 63 of the row's sequence), in
+ *   order of decreasing block maximum: block_idx DEVICE int32 [R, n_ret_q_heads, block_stride] (may be NULL: counts
+ *   only), sel_count = number of blocks (a list longer than block_stride is cut and RTP_ERR_CAPACITY set in the status
+ *   word), sel_mass = softmax mass of the selected blocks, sel_thresh = m_b of the last block taken, sel_tie_last = its
+ *   block number (-inf / last block when every block is taken).  At most 16384 blocks per row (RTP_ERR_UNSUPPORTED
+ *   beyond; max_pages of the cache is what counts).  Workspace: rtp_block_workspace_bytes(params, R, max_seq_len).
+ *   Works on bf16 and 8-bit index keys.  The selectable variants of rtp_params (top_k, forced positions) are for token
+ *   lists: RTP_ERR_UNSUPPORTED here.
+ * rtp_sparse_attn_decode_blocks: exact attention of every retrieval query head over the keys of its listed pages
+ *   (the positions of the row's last page beyond the row's own are left out), split-KV with LSE merge as
+ *   rtp_sparse_attn_decode; block_count as written by the selection; a page number outside the row's causal pages sets
+ *   RTP_ERR_INVALID in the status word and is skipped.  Workspace: rtp_workspace_bytes(params, R, max_seq_len). */
+rtp_status rtp_topp_select_blocks_rows(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q_pre,
+                                       const void* w_q, const int32_t* row_seq, const int32_t* row_pos, int64_t R,
+                                       int32_t* block_idx, int64_t block_stride, int32_t* sel_count, float* sel_mass,
+                                       float* sel_thresh, int32_t* sel_tie_last, int32_t* status, void* workspace,
+                                       size_t workspace_bytes, void* stream);
+rtp_status rtp_sparse_attn_decode_blocks(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q,
+                                         const int32_t* row_seq, const int32_t* row_pos, int64_t R,
+                                         const int32_t* block_idx, int64_t block_stride, const int32_t* block_count,
+                                         void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                         int32_t* status, void* stream);
+
 /* ---- S7: local heads, attention sinks + sliding window (Section 3.2, Table 2) -
  * Row at position m attends to {n <= m : n < n_sink or n > m - window}.
  * Rows as in rtp_topp_select (row arrays = decode path with split-KV; NULL

@@ -25,6 +25,7 @@ EXPORTS = [
     "rtp_kv_append", "rtp_index_keys", "rtp_index_queries", "rtp_index_score", "rtp_topp_select", "rtp_sparse_attn_decode", "rtp_sparse_attn_decode_static",
     "rtp_sparse_attn_prefill", "rtp_local_attn", "rtp_dense_attn_prefill", "rtp_dense_attn_decode",
     "rtp_block_workspace_bytes", "rtp_topp_select_blocks", "rtp_sparse_attn_prefill_blocks",
+    "rtp_topp_select_blocks_rows", "rtp_sparse_attn_decode_blocks",
 ]
 
 
@@ -108,6 +109,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.rtp_topp_select_blocks.argtypes = [vp, PP, PC, vp, vp, i32, i32, i64, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.rtp_sparse_attn_prefill_blocks.restype = i32
     lib.rtp_sparse_attn_prefill_blocks.argtypes = [vp, PP, PC, vp, i32, i32, i64, vp, i64, vp, vp, vp, vp]
+    lib.rtp_topp_select_blocks_rows.restype = i32
+    lib.rtp_topp_select_blocks_rows.argtypes = [vp, PP, PC, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.rtp_sparse_attn_decode_blocks.restype = i32
+    lib.rtp_sparse_attn_decode_blocks.argtypes = [vp, PP, PC, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, sz, vp, vp]
     lib.rtp_local_attn.restype = i32
     lib.rtp_local_attn.argtypes = [vp, PP, PC, vp, vp, vp, i32, i32, i64, vp, vp, vp, sz, vp, vp]
     lib.rtp_dense_attn_prefill.restype = i32
@@ -322,6 +327,27 @@ def rtp_topp_select_blocks(ctx, params, cache, q_pre, w_q, seq_id, q_start, n_ro
                                               _ptr(status), _ptr(workspace),
                                               int(workspace.numel() * workspace.element_size()), _stream(stream)),
                "rtp_topp_select_blocks")
+
+
+def rtp_topp_select_blocks_rows(ctx, params, cache, q_pre, w_q, row_seq, row_pos, block_idx, sel_count, sel_mass,
+                                sel_thresh, sel_tie_last, status, workspace, stream=None):
+    """block_idx: int32 tensor [R, n_ret, block_stride] of logical page numbers (or None: counts only)."""
+    stride = int(block_idx.shape[-1]) if block_idx is not None else 0
+    ctx._check(ctx.lib.rtp_topp_select_blocks_rows(ctx.h, params.ref(), C.byref(cache), _ptr(q_pre), _ptr(w_q),
+                                                   _ptr(row_seq), _ptr(row_pos), int(row_seq.shape[0]),
+                                                   _ptr(block_idx), stride, _ptr(sel_count), _ptr(sel_mass),
+                                                   _ptr(sel_thresh), _ptr(sel_tie_last), _ptr(status), _ptr(workspace),
+                                                   int(workspace.numel() * workspace.element_size()), _stream(stream)),
+               "rtp_topp_select_blocks_rows")
+
+
+def rtp_sparse_attn_decode_blocks(ctx, params, cache, q, row_seq, row_pos, block_idx, block_count, out, lse, workspace,
+                                  status, stream=None):
+    ctx._check(ctx.lib.rtp_sparse_attn_decode_blocks(ctx.h, params.ref(), C.byref(cache), _ptr(q), _ptr(row_seq),
+                                                     _ptr(row_pos), int(row_seq.shape[0]), _ptr(block_idx),
+                                                     int(block_idx.shape[-1]), _ptr(block_count), _ptr(out), _ptr(lse),
+                                                     _ptr(workspace), int(workspace.numel() * workspace.element_size()),
+                                                     _ptr(status), _stream(stream)), "rtp_sparse_attn_decode_blocks")
 
 
 def rtp_sparse_attn_prefill_blocks(ctx, params, cache, q, seq_id, q_start, n_rows, block_mask, out, lse, status,

@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(os.path.dirname(PKG_DIR), "include")
 LIB_PATH = os.path.join(PKG_DIR, "librtp.so")
-SOURCES = ["rtp_api.cu", "index_kernels.cu", "select_rows.cu", "select_chunk.cu", "select_blocks.cu", "attn_rows.cu", "attn_prefill_tc.cu", "tensor_map.cu"]
+SOURCES = ["rtp_api.cu", "index_kernels.cu", "select_rows.cu", "select_chunk.cu", "select_blocks.cu", "select_rows_blocks.cu", "attn_rows.cu", "attn_prefill_tc.cu", "tensor_map.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

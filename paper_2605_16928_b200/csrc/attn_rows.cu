@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
   const int g = lane >> 2, c = lane & 3;
 
   int qh0, kvh;
-  if (SET == kSetList) {
+  if (SET == kSetList || SET == kSetPages) {
     qh0 = hm.ret_q_head[u];
     kvh = qh0 / d.group;
   } else {
@@ -90,10 +90,11 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
   // enumerate the set as t = 0 .. n_set-1
   int n_set, ns = 0, wlo = 0;
   const int32_t* ids = nullptr;
-  if (SET == kSetList) {
+  if (SET == kSetList || SET == kSetPages) {
     const int64_t rh = r * d.n_ret + u;
     n_set = min((int64_t)sel_count[rh], sel_stride);
     n_set = max(n_set, 0);
+    if (SET == kSetPages) n_set *= kPage;   // every listed page is 64 entries (the row's last page: fewer are causal)
     ids = sel_idx + rh * sel_stride;
   } else if (SET == kSetLocal) {
     ns = min(d.n_sink, n_keys);
@@ -135,6 +136,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
     const int t = t_lo + (warp + i * kWarps) * kTileTok + (lane & 15);
     if (i >= n_mine || t >= t_hi) return -1;
     if (SET == kSetList) return __ldg(ids + t);
+    if (SET == kSetPages) return __ldg(ids + (t >> kPageShift)) * kPage + (t & (kPage - 1));
     if (SET == kSetLocal) return t < ns ? t : wlo + (t - ns);
     return t;
   };
@@ -142,6 +144,14 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
     if (SET == kSetList && tok != -1 && (tok < 0 || tok >= n_keys)) {
       set_status(status, RTP_ERR_INVALID);
       return -1;
+    }
+    if (SET == kSetPages && tok != -1) {
+      // a listed page must hold a causal key; the positions of the row's last page beyond its own are left out quietly
+      if (tok < 0 || (tok >> kPageShift) > ((n_keys - 1) >> kPageShift) || n_keys == 0) {
+        set_status(status, RTP_ERR_INVALID);
+        return -1;
+      }
+      if (tok >= n_keys) return -1;
     }
     return tok;
   };
@@ -326,7 +336,7 @@ __global__ void __launch_bounds__(kHeadDim) attn_merge_kernel(const Dims d, cons
   const int g = blockIdx.x % G;
   const int64_t r = unit / n_units;
   const int u = unit % n_units;
-  const int qh = (SET == kSetList) ? hm.ret_q_head[u] : hm.kv_list[u] * d.group + g;
+  const int qh = (SET == kSetList || SET == kSetPages) ? hm.ret_q_head[u] : hm.kv_list[u] * d.group + g;
   if (SET == kSetLocal && hm.skips(qh)) return;
   const float* p = partial + ((unit * G + g) * (int64_t)n_splits) * kPartial;
   const int dim = threadIdx.x;
@@ -360,6 +370,7 @@ int plan_splits(int64_t units, int64_t max_set, int sm_count, bool round_up) {
 
 int64_t max_set_len(const Dims& d, int set, int64_t sel_stride, int64_t max_len) {
   if (set == kSetList) return sel_stride < max_len ? sel_stride : max_len;
+  if (set == kSetPages) return sel_stride * kPage < max_len ? sel_stride * kPage : (max_len + kPage - 1) / kPage * kPage;
   if (set == kSetLocal) {
     const int64_t w = (int64_t)d.n_sink + d.window;
     return w < max_len ? w : max_len;
@@ -397,9 +408,10 @@ cudaError_t launch_attn_rows(const CacheView& cv, const Dims& d, const HeadMaps&
                              const __nv_bfloat16* q, const int32_t* sel_idx, int64_t sel_stride,
                              const int32_t* sel_count, __nv_bfloat16* out, float* lse, void* ws, size_t ws_bytes,
                              int64_t max_len, int32_t* status, int sm_count, cudaStream_t st) {
-  const int n_units = set == kSetList ? d.n_ret : hm.n_kv_list;
+  const bool per_head = set == kSetList || set == kSetPages;   // one set per retrieval query head
+  const int n_units = per_head ? d.n_ret : hm.n_kv_list;
   if (rows.R == 0 || n_units == 0) return cudaSuccess;
-  const int G = set == kSetList ? 1 : d.group;
+  const int G = per_head ? 1 : d.group;
   int n_splits = plan_splits(rows.R * n_units, max_set_len(d, set, sel_stride, max_len), sm_count, set == kSetList);
   // never plan more splits than the workspace holds
   const size_t per_split = (size_t)rows.R * n_units * G * kPartial * sizeof(float);
@@ -410,6 +422,7 @@ cudaError_t launch_attn_rows(const CacheView& cv, const Dims& d, const HeadMaps&
   return launch_typed<GG, SS>(cv, d, hm, rows, n_units, q, sel_idx, sel_stride, sel_count, out, lse, partial, \
                               n_splits, status, st)
   if (set == kSetList) RTP_LAUNCH(1, kSetList);
+  if (set == kSetPages) RTP_LAUNCH(1, kSetPages);
   if (set == kSetLocal) {
     if (G == 1) RTP_LAUNCH(1, kSetLocal);
     if (G == 2) RTP_LAUNCH(2, kSetLocal);

@@ -472,7 +472,56 @@ size_t rtp_block_workspace_bytes(const rtp_params* params, int64_t rows, int64_t
   WsCarver w(nullptr);
   w.take(qt_bytes(d, rows));
   w.take(select_blocks_workspace_bytes(d, hm, rows, max_seq_len, current_sm_count(kFallbackSm)));
+  w.take(select_rows_blocks_workspace_bytes(d, rows, max_seq_len));   // (the row form; one buffer serves either)
   return w.off;
+}
+
+rtp_status rtp_topp_select_blocks_rows(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q_pre,
+                                       const void* w_q, const int32_t* row_seq, const int32_t* row_pos, int64_t R,
+                                       int32_t* block_idx, int64_t block_stride, int32_t* sel_count, float* sel_mass,
+                                       float* sel_thresh, int32_t* sel_tie_last, int32_t* status, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+  RTP_COMMON_PROLOGUE(false, true)
+  Rows rows;
+  int64_t max_len = 0;
+  if (!row_seq || !row_pos) return fail(ctx, RTP_ERR_INVALID, "row_seq / row_pos is NULL");
+  if (const char* m = check_rows(row_seq, row_pos, 0, 0, R, cache, &rows, &max_len)) return fail(ctx, RTP_ERR_INVALID, m);
+  if (R == 0 || d.n_ret == 0) return RTP_OK;
+  if (!q_pre || !w_q || !workspace || !sel_count) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
+  if (!aligned16(q_pre) || !aligned16(w_q) || !aligned16(workspace)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
+  if (block_idx && block_stride <= 0) return fail(ctx, RTP_ERR_INVALID, "block_stride must be positive");
+  if (variant_set(d)) return fail(ctx, RTP_ERR_UNSUPPORTED, "top_k / forced positions: token lists only");
+  WsCarver w(workspace);
+  __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(w.take(qt_bytes(d, R)));
+  void* sel_ws = w.take(select_rows_blocks_workspace_bytes(d, R, max_len));
+  if (w.off > workspace_bytes) return fail(ctx, RTP_ERR_CAPACITY, "workspace too small");
+  cudaError_t e = launch_index_queries(d, hm, reinterpret_cast<const __nv_bfloat16*>(q_pre),
+                                       reinterpret_cast<const __nv_bfloat16*>(w_q), R, qt, st);
+  if (e == cudaSuccess)
+    e = launch_select_rows_blocks(cv, d, hm, rows, qt, max_len, block_idx, block_stride, sel_count, sel_mass, sel_thresh,
+                                  sel_tie_last, status, sel_ws, ctx->sm_count, st);
+  if (e == cudaErrorNotSupported) return fail(ctx, RTP_ERR_UNSUPPORTED, "more than 16384 blocks per row");
+  return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_topp_select_blocks_rows");
+}
+
+rtp_status rtp_sparse_attn_decode_blocks(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q,
+                                         const int32_t* row_seq, const int32_t* row_pos, int64_t R,
+                                         const int32_t* block_idx, int64_t block_stride, const int32_t* block_count,
+                                         void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                         int32_t* status, void* stream) {
+  RTP_COMMON_PROLOGUE(true, false)
+  Rows rows;
+  int64_t max_len = 0;
+  if (!row_seq || !row_pos) return fail(ctx, RTP_ERR_INVALID, "row_seq / row_pos is NULL");
+  if (const char* m = check_rows(row_seq, row_pos, 0, 0, R, cache, &rows, &max_len)) return fail(ctx, RTP_ERR_INVALID, m);
+  if (R == 0 || d.n_ret == 0) return RTP_OK;
+  if (!q || !block_idx || !block_count || !out) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
+  if (block_stride <= 0) return fail(ctx, RTP_ERR_INVALID, "block_stride must be positive");
+  if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
+  cudaError_t e = launch_attn_rows(cv, d, hm, rows, kSetPages, reinterpret_cast<const __nv_bfloat16*>(q), block_idx,
+                                   block_stride, block_count, reinterpret_cast<__nv_bfloat16*>(out), lse, workspace,
+                                   workspace ? workspace_bytes : 0, max_len, status, ctx->sm_count, st);
+  return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_sparse_attn_decode_blocks");
 }
 
 rtp_status rtp_topp_select_blocks(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q_pre,

@@ -193,7 +193,8 @@ cudaError_t launch_select_chunk(const CacheView& cv, const Dims& d, const HeadMa
                                 int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
                                 int32_t* status, void* ws, size_t ws_bytes, int sm_count, cudaStream_t st);
 
-enum AttnSet { kSetList = 0, kSetLocal = 1, kSetDense = 2 };
+// kSetPages: like kSetList, but the list holds logical page numbers and every listed page is taken whole
+enum AttnSet { kSetList = 0, kSetLocal = 1, kSetDense = 2, kSetPages = 3 };
 size_t attn_rows_workspace_bytes(const Dims& d, int64_t R, int n_units, int group, int sm_count, int64_t max_len);
 cudaError_t launch_attn_rows(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows, int set,
                              const __nv_bfloat16* q, const int32_t* sel_idx, int64_t sel_stride,
@@ -221,6 +222,11 @@ cudaError_t launch_attn_prefill_tc(const CacheView& cv, const Dims& d, const Hea
 
 // Block-wise top-p of a prefill chunk (Section 3.4): one bit per (row, retrieval head, page).
 size_t select_blocks_workspace_bytes(const Dims& d, const HeadMaps& hm, int64_t R, int64_t max_len, int sm_count);
+size_t select_rows_blocks_workspace_bytes(const Dims& d, int64_t R, int64_t max_len);
+cudaError_t launch_select_rows_blocks(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                                      const __nv_bfloat16* qt, int64_t max_len, int32_t* blk_idx, int64_t blk_stride,
+                                      int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
+                                      int32_t* status, void* ws, int sm_count, cudaStream_t st);
 cudaError_t launch_select_blocks(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                                  const __nv_bfloat16* qt, uint32_t* mask, int64_t mask_words, int32_t* sel_count,
                                  float* sel_mass, float* sel_thresh, int32_t* sel_tie_last, int32_t* status, void* ws,

@@ -1,0 +1,295 @@
+// Block-wise top-p for explicit rows (the decode path), Section 3.4: the index keys of a row are cut into blocks of
+// one cache page (64 keys), every block is reduced to a log-sum-exp pair (m_b, l_b), blocks are taken in order of
+// decreasing m_b (equal maxima: smaller block first) until their softmax mass l_b exp(m_b - M) / Z reaches p.
+//
+//   blk_stats_kernel    one scan of the index keys: a warp scores a page for the unit's heads (MMA, see score16) and
+//                       reduces it to (m_b, l_b) per head; nothing else is stored (8 bytes per head and page).
+//   blk_select_kernel   one CTA per (row, head): the pairs are sorted by (m_b desc, block asc) in shared memory and the
+//                       shortest prefix that reaches the target mass is written out as a list of logical page numbers.
+//
+// The paper's kernel deposits l_b into a 256-bin histogram indexed by m_b and takes the threshold's bin whole; here the
+// order inside that bin is resolved exactly (a row has at most 16384 blocks, which a CTA sorts in a few microseconds),
+// so the selection is the one the block-wise rule defines, not a superset of it.
+#include "row_scan.cuh"
+
+namespace rtp {
+
+namespace {
+
+using namespace rowscan;
+
+constexpr float kLog2eB = 1.4426950408889634f;
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kMaxBlocksRow = 16384;   // blocks of a row the select kernel sorts in shared memory (1M keys)
+
+// ---- pass 1: (m_b, l_b) of every page of the unit's slice ---------------------------------------------------------
+// stats: float2 [rows * retrieval heads][nb_pad]; entry b = (largest finished score of block b, sum of exp(s - m_b)).
+template <bool NH4, bool F8>
+__global__ void __launch_bounds__(kThreads) blk_stats_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
+                                                             const Rows rows, const __nv_bfloat16* __restrict__ qt,
+                                                             float2* __restrict__ stats, const int64_t nb_pad,
+                                                             int n_splits, int32_t* status) {
+  chain_wait();
+  const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, status);
+  if (x.p_lo >= x.p_hi) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  QFrag qf = load_qfrag(qt + x.r * d.n_ret * kIndexDim, hm.ih_heads[x.ih], x.nh, lane);
+  if (F8 && !qfrag_to_f16(qf)) set_status(status, RTP_ERR_UNSUPPORTED);   // a projected query beyond fp16's range
+  const int slot_a = elem_slot<NH4>(lane, 0), slot_b = NH4 ? slot_a : elem_slot<NH4>(lane, 4);
+  float2* st_a = slot_a < x.nh ? stats + (x.r * d.n_ret + hm.ih_heads[x.ih][slot_a]) * nb_pad : nullptr;
+  float2* st_b = (!NH4 && slot_b < x.nh) ? stats + (x.r * d.n_ret + hm.ih_heads[x.ih][slot_b]) * nb_pad : nullptr;
+  // the lane of a head slot that writes the pair: NH4: (g < 4, c = 0); otherwise c = 0 (slots g and g + 8)
+  const bool writer = NH4 ? ((lane & 3) == 0 && lane < 16) : ((lane & 3) == 0);
+  constexpr int kN = LaneElems<NH4>::kN;
+  uint4 v[4], vn[4];
+  if (x.p_lo + warp < x.p_hi) load_page<F8>(cv, x, x.p_lo + warp, lane, vn);
+  for (int p = x.p_lo + warp; p < x.p_hi; p += kWarps) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = vn[i];
+    if (p + kWarps < x.p_hi) load_page<F8>(cv, x, p + kWarps, lane, vn);   // in flight while this page is worked on
+    const bool tail = (p + 1) * kPage > x.n_keys;
+    float fs[4][kN];
+    float ma = -INFINITY, mb = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float s_lo[4], s_hi[4];
+      if (F8) score16_f8(qf, make_uint2(v[i].x, v[i].y), lane, s_lo, s_hi); else score16(qf, v[i], lane, s_lo, s_hi);
+      const LaneElems<NH4> el = lane_elems<NH4>(s_lo, s_hi, lane);
+#pragma unroll
+      for (int e = 0; e < kN; ++e) {
+        const bool beyond = tail && p * kPage + i * 16 + el.koff[e] >= x.n_keys;
+        fs[i][e] = beyond ? -INFINITY : finish_score(el.raw[e], d.score_scale);
+        if (NH4 || e < 4) ma = fmaxf(ma, fs[i][e]); else mb = fmaxf(mb, fs[i][e]);
+      }
+    }
+    ma = fmaxf(ma, __shfl_xor_sync(0xffffffffu, ma, 1));
+    ma = fmaxf(ma, __shfl_xor_sync(0xffffffffu, ma, 2));
+    if (NH4) ma = fmaxf(ma, __shfl_xor_sync(0xffffffffu, ma, 16));
+    if (!NH4) {
+      mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, 1));
+      mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, 2));
+    }
+    // (a page of the slice holds at least one causal key, so ma and mb are finite for the slots in use)
+    float la = 0.f, lb = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+#pragma unroll
+      for (int e = 0; e < kN; ++e) {
+        if (NH4 || e < 4) la += fast_ex2((fs[i][e] - ma) * kLog2eB); else lb += fast_ex2((fs[i][e] - mb) * kLog2eB);
+      }
+    }
+    la += __shfl_xor_sync(0xffffffffu, la, 1);
+    la += __shfl_xor_sync(0xffffffffu, la, 2);
+    if (NH4) la += __shfl_xor_sync(0xffffffffu, la, 16);
+    if (!NH4) {
+      lb += __shfl_xor_sync(0xffffffffu, lb, 1);
+      lb += __shfl_xor_sync(0xffffffffu, lb, 2);
+    }
+    if (writer) {
+      if (st_a) st_a[p] = make_float2(ma, la);
+      if (st_b) st_b[p] = make_float2(mb, lb);
+    }
+  }
+}
+
+// ---- pass 2: order the blocks, take the shortest prefix with mass >= p ---------------------------------------------
+// Dynamic shared memory: np2 sort keys of 8 bytes ((~ordered key of m_b) << 32 | block: ascending order = larger m_b
+// first, then smaller block) followed by nb_pad floats (l_b by block number).
+__global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
+    const CacheView cv, const Dims d, const Rows rows, const float2* __restrict__ stats, const int64_t nb_pad,
+    const int np2, int32_t* __restrict__ blk_idx, const int64_t blk_stride, int32_t* __restrict__ sel_count,
+    float* __restrict__ sel_mass, float* __restrict__ sel_thresh, int32_t* __restrict__ sel_tie_last, int32_t* status) {
+  chain_wait();
+  extern __shared__ __align__(16) unsigned char blk_smem[];
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(blk_smem);
+  float* lw = reinterpret_cast<float*>(blk_smem + (size_t)np2 * 8);
+  __shared__ float w_sum[kSelWarps];
+  __shared__ uint32_t w_max[kSelWarps];
+  __shared__ int s_pick;
+  __shared__ float s_run, s_pick_mass;
+  const int64_t rh = blockIdx.x;
+  const int64_t r = rh / d.n_ret;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int seq = rows.row_seq(r);
+  int n_keys = rows.row_pos(r) + 1;
+  {
+    const int sl = (seq >= 0 && seq < cv.batch) ? min(cv.seq_lens[seq], cv.max_pages * kPage) : 0;
+    n_keys = max(0, min(n_keys, sl));
+  }
+  const int nb = (n_keys + kPage - 1) >> kPageShift;
+  int32_t* out_ids = blk_idx ? blk_idx + rh * blk_stride : nullptr;
+  if (nb == 0) {
+    if (tid == 0) {
+      sel_count[rh] = 0;
+      if (sel_mass) sel_mass[rh] = 0.f;
+      if (sel_thresh) sel_thresh[rh] = 0.f;
+      if (sel_tie_last) sel_tie_last[rh] = -1;
+    }
+    return;
+  }
+  const float2* st = stats + rh * nb_pad;
+  int np = 1;
+  while (np < nb) np <<= 1;
+  uint32_t kmax = 0u;
+  for (int i = tid; i < np; i += kSelThreads) {
+    if (i < nb) {
+      const float2 s = __ldcg(st + i);
+      const uint32_t k = okey(s.x);
+      kmax = max(kmax, k);
+      keys[i] = ((unsigned long long)(~k) << 32) | (unsigned long long)(uint32_t)i;
+      lw[i] = s.y;
+    } else {
+      keys[i] = ~0ull;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+  if (lane == 0) w_max[warp] = kmax;
+  if (tid == 0) {
+    s_pick = 0x7fffffff;
+    s_run = 0.f;
+    s_pick_mass = 0.f;
+  }
+  __syncthreads();
+  for (int w = 0; w < kSelWarps; ++w) kmax = max(kmax, w_max[w]);
+  const float M = okey_to_float(kmax);
+
+  // bitonic sort, ascending
+  for (int size = 2; size <= np; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = tid; i < (np >> 1); i += kSelThreads) {
+        const int lo = 2 * i - (i & (stride - 1));
+        const int hi = lo + stride;
+        const bool up = (lo & size) == 0;
+        const unsigned long long a = keys[lo], b = keys[hi];
+        if ((a > b) == up) {
+          keys[lo] = b;
+          keys[hi] = a;
+        }
+      }
+      __syncthreads();
+    }
+  }
+  auto weight = [&](int i) -> float {   // mass of the i-th block of the order, relative to exp(M)
+    const unsigned long long k = keys[i];
+    return lw[(uint32_t)k] * fast_ex2((okey_to_float(~(uint32_t)(k >> 32)) - M) * kLog2eB);
+  };
+  // Z: every thread sums its blocks in a fixed order, then a fixed tree: the same value in every run
+  float z = 0.f;
+  for (int i = tid; i < nb; i += kSelThreads) z += weight(i);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+  if (lane == 0) w_sum[warp] = z;
+  __syncthreads();
+  float Z = 0.f;
+  for (int w = 0; w < kSelWarps; ++w) Z += w_sum[w];
+  __syncthreads();
+
+  int c;
+  float mass;
+  if (d.top_p >= 1.0f || nb <= 1) {
+    c = nb;
+    mass = Z;
+  } else {
+    const float target = d.top_p * Z * (1.0f + kMassMargin);
+    for (int r0 = 0; r0 < nb; r0 += kSelThreads) {
+      if (s_pick != 0x7fffffff) break;   // uniform: written before the barrier that ends each round
+      const int i = r0 + tid;
+      const float e = i < nb ? weight(i) : 0.f;
+      float inc = e;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const float a = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += a;
+      }
+      if (lane == 31) w_sum[warp] = inc;
+      __syncthreads();
+      float wbase = 0.f, tot = 0.f;
+      for (int w = 0; w < kSelWarps; ++w) {
+        if (w < warp) wbase += w_sum[w];
+        tot += w_sum[w];
+      }
+      const float cum = s_run + wbase + inc;
+      if (i < nb && cum >= target) atomicMin(&s_pick, i);
+      __syncthreads();
+      if (i == s_pick) s_pick_mass = cum;
+      if (tid == 0) s_run += tot;
+      __syncthreads();
+    }
+    int pick = s_pick;
+    mass = s_pick_mass;
+    if (pick == 0x7fffffff) {   // rounding left the target just out of reach: every block
+      pick = nb - 1;
+      mass = s_run;
+    }
+    c = pick + 1;
+  }
+  if (out_ids) {
+    for (int i = tid; i < c; i += kSelThreads)
+      if (i < blk_stride) out_ids[i] = (int)(uint32_t)keys[i];
+  }
+  if (tid == 0) {
+    const unsigned long long last = keys[c - 1];
+    sel_count[rh] = c;
+    if (sel_mass) sel_mass[rh] = Z > 0.f ? mass / Z : 1.0f;
+    if (sel_thresh) sel_thresh[rh] = c == nb ? -INFINITY : okey_to_float(~(uint32_t)(last >> 32));
+    if (sel_tie_last) sel_tie_last[rh] = c == nb ? nb - 1 : (int)(uint32_t)last;
+    if (out_ids && c > blk_stride) set_status(status, RTP_ERR_CAPACITY);
+  }
+}
+
+int64_t blocks_padded(int64_t max_len) { return (((max_len + kPage - 1) / kPage) + 3) / 4 * 4; }
+
+int stats_splits(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
+  const int64_t pages = (max_len + kPage - 1) / kPage;
+  int64_t want = (4LL * sm_count + R * d.n_ih - 1) / (R * d.n_ih);
+  const int64_t cap = (pages + 31) / 32;   // at least 32 pages per CTA
+  int64_t s = want < cap ? want : cap;
+  if (s < 1) s = 1;
+  if (s > 4096) s = 4096;
+  return (int)s;
+}
+
+}  // namespace
+
+size_t select_rows_blocks_workspace_bytes(const Dims& d, int64_t R, int64_t max_len) {
+  if (R <= 0 || d.n_ret <= 0) return 0;
+  return (size_t)R * d.n_ret * blocks_padded(max_len) * sizeof(float2);
+}
+
+cudaError_t launch_select_rows_blocks(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                                      const __nv_bfloat16* qt, int64_t max_len, int32_t* blk_idx, int64_t blk_stride,
+                                      int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,
+                                      int32_t* status, void* ws, int sm_count, cudaStream_t st) {
+  if (rows.R == 0 || d.n_ret == 0) return cudaSuccess;
+  const int64_t nb_pad = blocks_padded(max_len);
+  const int64_t nb_max = (max_len + kPage - 1) / kPage;
+  if (nb_max > kMaxBlocksRow) return cudaErrorNotSupported;
+  float2* stats = reinterpret_cast<float2*>(ws);
+  int max_nh = 0;
+  for (int i = 0; i < d.n_ih; ++i) max_nh = hm.ih_nheads[i] > max_nh ? hm.ih_nheads[i] : max_nh;
+  const int n_splits = stats_splits(d, rows.R, max_len, sm_count);
+  const dim3 grid((unsigned)(rows.R * d.n_ih), n_splits);
+#define RTP_STATS(NH4_, F8_) \
+  (void)launch_chained(blk_stats_kernel<NH4_, F8_>, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, qt, stats, nb_pad, n_splits, status)
+  if (max_nh <= 4) {
+    if (cv.ikey_fp8) RTP_STATS(true, true); else RTP_STATS(true, false);
+  } else {
+    if (cv.ikey_fp8) RTP_STATS(false, true); else RTP_STATS(false, false);
+  }
+#undef RTP_STATS
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  int np2 = 1;
+  while (np2 < nb_max) np2 <<= 1;
+  const int smem = np2 * 8 + (int)nb_pad * 4;
+  static PerDeviceOnce once;
+  e = set_dyn_smem_once(blk_select_kernel, kMaxBlocksRow * 8 + kMaxBlocksRow * 4, once);
+  if (e != cudaSuccess) return e;
+  (void)launch_chained(blk_select_kernel, dim3((unsigned)(rows.R * d.n_ret)), dim3(kSelThreads), (size_t)smem, st, cv, d, rows,
+                       stats, nb_pad, np2, blk_idx, blk_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status);
+  return cudaGetLastError();
+}
+
+}  // namespace rtp
