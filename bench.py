@@ -271,6 +271,12 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
     t_graph = graph_timed(path)
     var = {}
     if variants:
+        # the block-wise selector of Section 3.4 on the same data: 64-key pages chosen by log-sum-exp mass
+        t_blk = timed(lambda: path.step_blocks(data.q, k_pre_new))
+        blk_frac = float(path.blk_cnt.float().mean().item()) / ((L + 63) // 64)
+        blk_status = path.status_code()
+        path.step(data.q, k_pre_new)   # (the token-level outputs are what the figures below describe)
+        torch.cuda.synchronize()
         # the fixed-budget variant the paper compares with (Section 4.1, k = 4096), same data and step
         path_k = pipeline.DecodePath(data, max(stride, 4096), top_k=4096)
         path_k.build_index_cache()
@@ -308,7 +314,8 @@ def bench_decode_point(device, name, L, B, top_p, frac, window, peaked_half, ite
         del sc16
         ikey8_count_ratio = float(path_8.sel_cnt.float().mean().item()) / max(1.0, float(path.sel_cnt.float().mean().item()))
         del path_8
-        var = {"fixed_budget_4096_step_us": t_topk, "fixed_budget_4096_step_us_cuda_graph": t_topk_graph,
+        var = {"block_topp_step_us": t_blk, "block_topp_selected_block_fraction": blk_frac, "block_topp_status": blk_status,
+               "fixed_budget_4096_step_us": t_topk, "fixed_budget_4096_step_us_cuda_graph": t_topk_graph,
                "fixed_budget_status": topk_status,
                "ikey_e4m3_step_us": t_ikey8, "ikey_e4m3_step_us_cuda_graph": t_ikey8_graph, "ikey_e4m3_status": ikey8_status,
                "ikey_e4m3_share_of_bf16_set_kept": ikey8_overlap, "ikey_e4m3_count_ratio": ikey8_count_ratio,

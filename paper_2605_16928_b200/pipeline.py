@@ -133,6 +133,29 @@ class DecodePath(_Base):
         if self.has_local:
             main.wait_stream(self.side)
 
+    def step_blocks(self, q, k_pre_new):
+        """The same decode step with the block-wise selector of Section 3.4: whole 64-key pages are selected by their
+        log-sum-exp mass and attended to.  Buffers are made on first use."""
+        d, p = self.data, self.params
+        if not hasattr(self, "blk_idx"):
+            n_b = (self.L + 63) // 64
+            self.blk_idx = torch.empty((self.B, self.n_ret, n_b), dtype=torch.int32, device=self.dev)
+            self.blk_cnt = torch.empty((self.B, self.n_ret), dtype=torch.int32, device=self.dev)
+            self.blk_ws = torch.empty(max(1 << 16, rb.rtp_block_workspace_bytes(p, self.B, self.L)), dtype=torch.uint8,
+                                      device=self.dev)
+        main = torch.cuda.current_stream()
+        if self.has_local:
+            self.side.wait_stream(main)
+            rb.rtp_local_attn(self.ctx, p, self.cache, q, d.row_seq, d.row_pos, 0, 0, self.B, self.out, self.lse,
+                              self.workspace_local, self.status, stream=self.side)
+        rb.rtp_index_keys(self.ctx, p, self.cache, k_pre_new, d.w_k, d.row_seq, d.row_pos)
+        rb.rtp_topp_select_blocks_rows(self.ctx, p, self.cache, q, d.w_q, d.row_seq, d.row_pos, self.blk_idx, self.blk_cnt,
+                                       self.sel_mass, self.sel_thr, self.sel_tie, self.status, self.blk_ws)
+        rb.rtp_sparse_attn_decode_blocks(self.ctx, p, self.cache, q, d.row_seq, d.row_pos, self.blk_idx, self.blk_cnt,
+                                         self.out, self.lse, self.workspace, self.status)
+        if self.has_local:
+            main.wait_stream(self.side)
+
     def step_dense(self, q):
         d = self.data
         rb.rtp_dense_attn_decode(self.ctx, self.params, self.cache, q, d.row_seq, d.row_pos, None, self.out, self.lse,

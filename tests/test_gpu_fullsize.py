@@ -276,6 +276,43 @@ def test_decode_512k_batch4_8bit_index_keys():
     _decode_point(524288, 4, 0.9, 0.05, 4096, [0, 2], e2e=False, ikey_e4m3=True)
 
 
+def test_decode_512k_batch4_block_selection():
+    """Block-wise decode at full size: page lists of sampled sequences against the oracle's block rule on the GPU's
+    scores, attention over the listed pages against the oracle."""
+    from paper_2605_16928_b200 import pipeline, synth_device
+    L, B, seqs = 524288, 4, [0, 3]
+    data = synth_device.decode_device(L, B, 0.9, 0.05, 4096, name="c5_decode_sweep")
+    path = pipeline.DecodePath(data, sel_stride=4096)
+    path.build_index_cache()
+    k_new = torch.stack([data.k_pre_rows(b, L - 1, L)[0] for b in range(B)]).contiguous()
+    path.step_blocks(data.q, k_new)
+    torch.cuda.synchronize()
+    assert path.status_code() == rb.RTP_OK
+    heads, g = data.heads, data.heads.group
+    rs = torch.tensor(seqs, device="cuda")
+    sc = torch.full((len(seqs), path.n_ret, L), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(rb.rtp_workspace_bytes(path.params, len(seqs), L), dtype=torch.uint8, device="cuda")
+    rb.rtp_index_score(path.ctx, path.params, path.cache, data.q[rs].contiguous(), data.w_q,
+                       data.row_seq[rs].contiguous(), data.row_pos[rs].contiguous(), sc, None, None, ws, path.status)
+    torch.cuda.synchronize()
+    sc = sc.cpu().numpy()
+    idx, cnt = path.blk_idx[rs].cpu().numpy(), path.blk_cnt[rs].cpu().numpy()
+    out = path.out[rs].float().cpu().numpy()
+    qh = _np16(data.q[rs])
+    n_b = L // 64
+    for k, b in enumerate(seqs):
+        for i, h in enumerate(heads.ret_q_heads):
+            c = int(cnt[k, i])
+            got = set(idx[k, i, :c].tolist())
+            assert len(got) == c and 1 <= c <= n_b
+            mand, forb = orc.classify_blocks_against_band(sc[k, i], data.top_p)
+            assert mand <= got and not (forb & got), f"seq {b} head {i}"
+            if i % 4 == 0:
+                kk, vv = data.logical_kv(b, h // g)
+                want, _ = orc.attention_over_set(qh[k, h], kk, vv, orc.block_token_set(sorted(got), L - 1), data.sm_scale)
+                assert np.abs(out[k, h] - want).max() <= 2e-2, f"seq {b} head {h}"
+
+
 def test_decode_32k_batch8_sampled_rows():
     _decode_point(32768, 8, 0.95, 0.1, 2048, [0, 3, 4, 7], peaked_half=True, name="c2_decode_batched_gqa")
 
