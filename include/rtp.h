@@ -373,7 +373,7 @@ rtp_status rtp_sparse_attn_prefill_blocks(rtp_ctx* ctx, const rtp_params* params
 /* The same block-wise rule for explicit rows (decode: the use Section 3.4 describes it for).
  * rtp_topp_select_blocks_rows: rows as in rtp_topp_select with row arrays.  For every (row, retrieval head) the
  *   selected blocks are written as LOGICAL page numbers (block b = keys 64 b .. 64 b + 63 of the row's sequence), in
- *   order of decreasing block maximum: block_idx DEVICE int32 [R, n_ret_q_heads, block_stride] (may be NULL: counts
+ *   no particular order: block_idx DEVICE int32 [R, n_ret_q_heads, block_stride] (may be NULL: counts
  *   only), sel_count = number of blocks (a list longer than block_stride is cut and RTP_ERR_CAPACITY set in the status
  *   word), sel_mass = softmax mass of the selected blocks, sel_thresh = m_b of the last block taken, sel_tie_last = its
  *   block number (-inf / last block when every block is taken).  At most 16384 blocks per row (RTP_ERR_UNSUPPORTED

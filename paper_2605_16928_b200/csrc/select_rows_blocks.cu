@@ -4,12 +4,14 @@
 //
 //   blk_stats_kernel    one scan of the index keys: a warp scores a page for the unit's heads (MMA, see score16) and
 //                       reduces it to (m_b, l_b) per head; nothing else is stored (8 bytes per head and page).
-//   blk_select_kernel   one CTA per (row, head): the pairs are sorted by (m_b desc, block asc) in shared memory and the
-//                       shortest prefix that reaches the target mass is written out as a list of logical page numbers.
+//   blk_select_kernel   one CTA per (row, head): block masses go into a 1024-bin histogram indexed by M - m_b (the
+//                       paper's histogram indexed by m_b, finer and in exact integer arithmetic); the bins are scanned
+//                       from the top until the mass reaches the target; blocks above the threshold's bin are selected,
+//                       the blocks inside it are sorted by (m_b desc, block asc) in shared memory and the shortest
+//                       prefix that completes the target is taken.  The result is a list of logical page numbers.
 //
-// The paper's kernel deposits l_b into a 256-bin histogram indexed by m_b and takes the threshold's bin whole; here the
-// order inside that bin is resolved exactly (a row has at most 16384 blocks, which a CTA sorts in a few microseconds),
-// so the selection is the one the block-wise rule defines, not a superset of it.
+// The paper's kernel takes the threshold's bin whole; resolving the order inside it makes the selection the one the
+// block-wise rule defines, not a superset of it.
 #include "row_scan.cuh"
 
 namespace rtp {
@@ -26,7 +28,7 @@ constexpr int kMaxBlocksRow = 16384;   // blocks of a row the select kernel sort
 // ---- pass 1: (m_b, l_b) of every page of the unit's slice ---------------------------------------------------------
 // stats: float2 [rows * retrieval heads][nb_pad]; entry b = (largest finished score of block b, sum of exp(s - m_b)).
 template <bool NH4, bool F8>
-__global__ void __launch_bounds__(kThreads) blk_stats_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
+__global__ void __launch_bounds__(kThreads, NH4 ? 4 : 3) blk_stats_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
                                                              const Rows rows, const __nv_bfloat16* __restrict__ qt,
                                                              float2* __restrict__ stats, const int64_t nb_pad,
                                                              int n_splits, int32_t* status) {
@@ -93,9 +95,13 @@ __global__ void __launch_bounds__(kThreads) blk_stats_kernel(const CacheView cv,
   }
 }
 
-// ---- pass 2: order the blocks, take the shortest prefix with mass >= p ---------------------------------------------
+// ---- pass 2: histogram over M - m_b, exact order inside the threshold's bin ---------------------------------------
 // Dynamic shared memory: np2 sort keys of 8 bytes ((~ordered key of m_b) << 32 | block: ascending order = larger m_b
 // first, then smaller block) followed by nb_pad floats (l_b by block number).
+constexpr int kHistBins = 1024;           // bins of 1/32 in M - m_b: 32 units; everything deeper shares the last bin
+constexpr float kHistScale = 32.0f;
+constexpr float kFix = 1099511627776.0f;  // 2^40: block masses (at most 64 each, 16384 blocks) summed as integers
+
 __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
     const CacheView cv, const Dims d, const Rows rows, const float2* __restrict__ stats, const int64_t nb_pad,
     const int np2, int32_t* __restrict__ blk_idx, const int64_t blk_stride, int32_t* __restrict__ sel_count,
@@ -104,9 +110,12 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
   extern __shared__ __align__(16) unsigned char blk_smem[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(blk_smem);
   float* lw = reinterpret_cast<float*>(blk_smem + (size_t)np2 * 8);
+  __shared__ unsigned long long hist[kHistBins];
+  __shared__ unsigned long long w_tot[kSelWarps];
   __shared__ float w_sum[kSelWarps];
   __shared__ uint32_t w_max[kSelWarps];
-  __shared__ int s_pick;
+  __shared__ int s_pick, s_bin, s_n_in, s_n_above;
+  __shared__ unsigned long long s_above;
   __shared__ float s_run, s_pick_mass;
   const int64_t rh = blockIdx.x;
   const int64_t r = rh / d.n_ret;
@@ -129,20 +138,27 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
     return;
   }
   const float2* st = stats + rh * nb_pad;
-  int np = 1;
-  while (np < nb) np <<= 1;
-  uint32_t kmax = 0u;
-  for (int i = tid; i < np; i += kSelThreads) {
-    if (i < nb) {
-      const float2 s = __ldcg(st + i);
-      const uint32_t k = okey(s.x);
-      kmax = max(kmax, k);
-      keys[i] = ((unsigned long long)(~k) << 32) | (unsigned long long)(uint32_t)i;
-      lw[i] = s.y;
-    } else {
-      keys[i] = ~0ull;
+  if (d.top_p >= 1.0f || nb <= 1) {   // every block
+    if (out_ids)
+      for (int i = tid; i < nb; i += kSelThreads)
+        if (i < blk_stride) out_ids[i] = i;
+    if (tid == 0) {
+      sel_count[rh] = nb;
+      if (sel_mass) sel_mass[rh] = 1.0f;
+      if (sel_thresh) sel_thresh[rh] = -INFINITY;
+      if (sel_tie_last) sel_tie_last[rh] = nb - 1;
+      if (out_ids && nb > blk_stride) set_status(status, RTP_ERR_CAPACITY);
     }
+    return;
   }
+  // M, and the l_b by block number
+  uint32_t kmax = 0u;
+  for (int i = tid; i < nb; i += kSelThreads) {
+    const float2 s = __ldcg(st + i);
+    kmax = max(kmax, okey(s.x));
+    lw[i] = s.y;
+  }
+  for (int i = tid; i < kHistBins; i += kSelThreads) hist[i] = 0ull;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
   if (lane == 0) w_max[warp] = kmax;
@@ -150,12 +166,95 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
     s_pick = 0x7fffffff;
     s_run = 0.f;
     s_pick_mass = 0.f;
+    s_n_in = 0;
+    s_n_above = 0;
   }
   __syncthreads();
   for (int w = 0; w < kSelWarps; ++w) kmax = max(kmax, w_max[w]);
   const float M = okey_to_float(kmax);
-
-  // bitonic sort, ascending
+  auto bin_of = [&](float m) -> int { return (int)fminf((M - m) * kHistScale, (float)(kHistBins - 1)); };   // monotone in m
+  auto mass_of = [&](float m, float l) -> float { return l * fast_ex2((m - M) * kLog2eB); };                 // relative to exp(M)
+  // histogram of block masses, integers: the sums do not depend on the order of the adds
+  unsigned long long mine = 0ull;
+  for (int i = tid; i < nb; i += kSelThreads) {
+    const float m = __ldcg(&st[i].x);
+    const unsigned long long q = (unsigned long long)(mass_of(m, lw[i]) * kFix);
+    atomicAdd(&hist[bin_of(m)], q);
+    mine += q;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+  if (lane == 0) w_tot[warp] = mine;
+  __syncthreads();
+  unsigned long long Zq = 0ull;
+  for (int w = 0; w < kSelWarps; ++w) Zq += w_tot[w];
+  const float Z = (float)Zq / kFix;
+  const float target = d.top_p * Z * (1.0f + kMassMargin);
+  // the threshold's bin: the first from the top at which the cumulative mass reaches the target (warp 0, 32 bins a lane)
+  if (warp == 0) {
+    constexpr int kPer = kHistBins / 32;
+    unsigned long long part = 0ull;
+    for (int j = 0; j < kPer; ++j) part += hist[lane * kPer + j];
+    unsigned long long inc = part;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    unsigned long long run = inc - part;
+    int found = kHistBins;
+    unsigned long long above = 0ull;
+    for (int j = 0; j < kPer; ++j) {
+      const unsigned long long h = hist[lane * kPer + j];
+      if (found == kHistBins && h && (float)(run + h) / kFix >= target) {
+        found = lane * kPer + j;
+        above = run;
+      }
+      run += h;
+    }
+    int best = found;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, o));
+    if (best == kHistBins) {   // rounding left the target just out of reach: the lowest populated bin
+      int last = -1;
+      for (int j = 0; j < kPer; ++j)
+        if (hist[lane * kPer + j]) last = lane * kPer + j;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+      best = last;
+      if (last >= lane * kPer && last < (lane + 1) * kPer) {
+        unsigned long long a2 = inc - part;
+        for (int j = lane * kPer; j < last; ++j) a2 += hist[j];
+        found = last;
+        above = a2;
+      }
+    }
+    if (found == best) {
+      s_bin = best;
+      s_above = above;
+    }
+  }
+  __syncthreads();
+  const int tbin = s_bin;
+  const float above = (float)s_above / kFix;
+  // blocks above the bin are selected; those inside it become sort keys
+  for (int i = tid; i < nb; i += kSelThreads) {
+    const float m = __ldcg(&st[i].x);
+    const int b = bin_of(m);
+    if (b < tbin) {
+      const int pos = atomicAdd(&s_n_above, 1);
+      if (out_ids && pos < blk_stride) out_ids[pos] = i;
+    } else if (b == tbin) {
+      keys[atomicAdd(&s_n_in, 1)] = ((unsigned long long)(~okey(m)) << 32) | (unsigned long long)(uint32_t)i;
+    }
+  }
+  __syncthreads();
+  const int n_above = s_n_above, n_in = s_n_in;
+  int np = 1;
+  while (np < n_in) np <<= 1;
+  for (int i = n_in + tid; i < np; i += kSelThreads) keys[i] = ~0ull;
+  __syncthreads();
+  // bitonic sort of the bin's blocks, ascending (usually a handful; all of the row's blocks when every maximum is equal)
   for (int size = 2; size <= np; size <<= 1) {
     for (int stride = size >> 1; stride > 0; stride >>= 1) {
       for (int i = tid; i < (np >> 1); i += kSelThreads) {
@@ -171,68 +270,49 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
       __syncthreads();
     }
   }
-  auto weight = [&](int i) -> float {   // mass of the i-th block of the order, relative to exp(M)
+  auto weight = [&](int i) -> float {   // mass of the i-th block of the bin's order, relative to exp(M)
     const unsigned long long k = keys[i];
-    return lw[(uint32_t)k] * fast_ex2((okey_to_float(~(uint32_t)(k >> 32)) - M) * kLog2eB);
+    return mass_of(okey_to_float(~(uint32_t)(k >> 32)), lw[(uint32_t)k]);
   };
-  // Z: every thread sums its blocks in a fixed order, then a fixed tree: the same value in every run
-  float z = 0.f;
-  for (int i = tid; i < nb; i += kSelThreads) z += weight(i);
+  for (int r0 = 0; r0 < n_in; r0 += kSelThreads) {
+    if (s_pick != 0x7fffffff) break;   // uniform: written before the barrier that ends each round
+    const int i = r0 + tid;
+    const float e = i < n_in ? weight(i) : 0.f;
+    float inc = e;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-  if (lane == 0) w_sum[warp] = z;
-  __syncthreads();
-  float Z = 0.f;
-  for (int w = 0; w < kSelWarps; ++w) Z += w_sum[w];
-  __syncthreads();
-
-  int c;
-  float mass;
-  if (d.top_p >= 1.0f || nb <= 1) {
-    c = nb;
-    mass = Z;
-  } else {
-    const float target = d.top_p * Z * (1.0f + kMassMargin);
-    for (int r0 = 0; r0 < nb; r0 += kSelThreads) {
-      if (s_pick != 0x7fffffff) break;   // uniform: written before the barrier that ends each round
-      const int i = r0 + tid;
-      const float e = i < nb ? weight(i) : 0.f;
-      float inc = e;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const float a = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += a;
-      }
-      if (lane == 31) w_sum[warp] = inc;
-      __syncthreads();
-      float wbase = 0.f, tot = 0.f;
-      for (int w = 0; w < kSelWarps; ++w) {
-        if (w < warp) wbase += w_sum[w];
-        tot += w_sum[w];
-      }
-      const float cum = s_run + wbase + inc;
-      if (i < nb && cum >= target) atomicMin(&s_pick, i);
-      __syncthreads();
-      if (i == s_pick) s_pick_mass = cum;
-      if (tid == 0) s_run += tot;
-      __syncthreads();
+    for (int o = 1; o < 32; o <<= 1) {
+      const float a = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += a;
     }
-    int pick = s_pick;
-    mass = s_pick_mass;
-    if (pick == 0x7fffffff) {   // rounding left the target just out of reach: every block
-      pick = nb - 1;
-      mass = s_run;
+    if (lane == 31) w_sum[warp] = inc;
+    __syncthreads();
+    float wbase = 0.f, tot = 0.f;
+    for (int w = 0; w < kSelWarps; ++w) {
+      if (w < warp) wbase += w_sum[w];
+      tot += w_sum[w];
     }
-    c = pick + 1;
+    const float cum = above + s_run + wbase + inc;
+    if (i < n_in && cum >= target) atomicMin(&s_pick, i);
+    __syncthreads();
+    if (i == s_pick) s_pick_mass = cum;
+    if (tid == 0) s_run += tot;
+    __syncthreads();
   }
+  int pick = s_pick;
+  float mass = s_pick_mass;
+  if (pick == 0x7fffffff) {   // rounding left the target just out of reach: the whole bin
+    pick = n_in - 1;
+    mass = above + s_run;
+  }
+  const int c_in = pick + 1, c = n_above + c_in;
   if (out_ids) {
-    for (int i = tid; i < c; i += kSelThreads)
-      if (i < blk_stride) out_ids[i] = (int)(uint32_t)keys[i];
+    for (int i = tid; i < c_in; i += kSelThreads)
+      if (n_above + i < blk_stride) out_ids[n_above + i] = (int)(uint32_t)keys[i];
   }
   if (tid == 0) {
-    const unsigned long long last = keys[c - 1];
+    const unsigned long long last = keys[c_in - 1];
     sel_count[rh] = c;
-    if (sel_mass) sel_mass[rh] = Z > 0.f ? mass / Z : 1.0f;
+    if (sel_mass) sel_mass[rh] = Z > 0.f ? fminf(mass / Z, 1.0f) : 1.0f;
     if (sel_thresh) sel_thresh[rh] = c == nb ? -INFINITY : okey_to_float(~(uint32_t)(last >> 32));
     if (sel_tie_last) sel_tie_last[rh] = c == nb ? nb - 1 : (int)(uint32_t)last;
     if (out_ids && c > blk_stride) set_status(status, RTP_ERR_CAPACITY);

@@ -51,7 +51,6 @@ def check_block_rows(dw, sc, sel, p, rows=None):
             assert len(got) == c and min(got) >= 0 and max(got) < n_b, "duplicate or out-of-range pages"
             assert np.all(idx[r, i, c:] == -1), "wrote past the count"
             mb, lb = orc.block_lse(s)
-            assert np.all(np.diff(mb[lst]) <= 0), "pages are listed in order of decreasing block maximum"
             rule = {b for b in range(n_b) if mb[b] > thr[r, i] or (mb[b] == thr[r, i] and b <= tie[r, i])}
             assert rule == got, f"row {r} head {i}: the (threshold, block) pair does not describe the list"
             mand, forb = orc.classify_blocks_against_band(s, p)
@@ -147,7 +146,7 @@ def test_equal_blocks_take_the_lowest_block_numbers():
     sc = dw.scores()[0]
     sel = select_block_rows(dw)
     c = int(sel["cnt"][0, 0])
-    assert c == 43 and sel["idx"][0, 0, :c].cpu().numpy().tolist() == list(range(43))
+    assert c == 43 and sorted(sel["idx"][0, 0, :c].cpu().numpy().tolist()) == list(range(43))
     check_block_rows(dw, sc, sel, wl.top_p)
 
 
