@@ -383,7 +383,11 @@ rtp_status rtp_sparse_attn_prefill_blocks(rtp_ctx* ctx, const rtp_params* params
  * rtp_sparse_attn_decode_blocks: exact attention of every retrieval query head over the keys of its listed pages
  *   (the positions of the row's last page beyond the row's own are left out), split-KV with LSE merge as
  *   rtp_sparse_attn_decode; block_count as written by the selection; a page number outside the row's causal pages sets
- *   RTP_ERR_INVALID in the status word and is skipped.  Workspace: rtp_workspace_bytes(params, R, max_seq_len). */
+ *   RTP_ERR_INVALID in the status word and is skipped.  With a workspace of rtp_workspace_bytes(params, R,
+ *   max_seq_len) the lists of the query heads that share a KV head are first merged into their union (Section 3.2:
+ *   what a KV head must supply is the union of its heads' sets) and the group is attended in one pass over it, every
+ *   head seeing only its own pages: pages that several heads selected are read once.  With a smaller (or no)
+ *   workspace every head gathers its own pages; the results are the same. */
 rtp_status rtp_topp_select_blocks_rows(rtp_ctx* ctx, const rtp_params* params, const rtp_cache* cache, const void* q_pre,
                                        const void* w_q, const int32_t* row_seq, const int32_t* row_pos, int64_t R,
                                        int32_t* block_idx, int64_t block_stride, int32_t* sel_count, float* sel_mass,

@@ -96,6 +96,10 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
     n_set = max(n_set, 0);
     if (SET == kSetPages) n_set *= kPage;   // every listed page is 64 entries (the row's last page: fewer are causal)
     ids = sel_idx + rh * sel_stride;
+  } else if (SET == kSetUnion) {
+    const int64_t ru = r * n_units + u;
+    n_set = max(min((int64_t)sel_count[ru], sel_stride), (int64_t)0) * kPage;
+    ids = sel_idx + ru * sel_stride;
   } else if (SET == kSetLocal) {
     ns = min(d.n_sink, n_keys);
     wlo = max(ns, n_keys - d.window);
@@ -103,7 +107,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
   } else {
     n_set = n_keys;
   }
-  const int per = (n_set + n_splits - 1) / n_splits;
+  // (a union list is cut at page boundaries: the head flags of a 16-token tile are then those of one entry)
+  const int per = SET == kSetUnion ? (((n_set >> kPageShift) + n_splits - 1) / n_splits) << kPageShift
+                                   : (n_set + n_splits - 1) / n_splits;
   const int t_lo = split * per;
   const int t_hi = min(n_set, t_lo + per);
   const int n_tiles = t_hi > t_lo ? (t_hi - t_lo + kTileTok - 1) / kTileTok : 0;
@@ -137,6 +143,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
     if (i >= n_mine || t >= t_hi) return -1;
     if (SET == kSetList) return __ldg(ids + t);
     if (SET == kSetPages) return __ldg(ids + (t >> kPageShift)) * kPage + (t & (kPage - 1));
+    if (SET == kSetUnion) return (__ldg(ids + (t >> kPageShift)) & 0xffffff) * kPage + (t & (kPage - 1));
     if (SET == kSetLocal) return t < ns ? t : wlo + (t - ns);
     return t;
   };
@@ -145,7 +152,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
       set_status(status, RTP_ERR_INVALID);
       return -1;
     }
-    if (SET == kSetPages && tok != -1) {
+    if ((SET == kSetPages || SET == kSetUnion) && tok != -1) {
       // a listed page must hold a causal key; the positions of the row's last page beyond its own are left out quietly
       if (tok < 0 || (tok >> kPageShift) > ((n_keys - 1) >> kPageShift) || n_keys == 0) {
         set_status(status, RTP_ERR_INVALID);
@@ -213,6 +220,13 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
 
         const uint32_t sk = ring + sgi * 2 * kTileBytes, sv = sk + kTileBytes;
         const uint32_t vmask = __ballot_sync(0xffffffffu, tok_c[sgi] >= 0) & 0xffffu;   // bit t = token t of the tile exists
+        // union lists: which query heads of the group selected the page of this tile (the entry was loaded when the
+        // tile was requested: it comes from the L1 cache)
+        bool head_on = true;
+        if (SET == kSetUnion) {
+          const int t_first = t_lo + (warp + i * kWarps) * kTileTok;
+          head_on = ((uint32_t)__ldg(ids + (t_first >> kPageShift)) >> (24 + g)) & 1u;
+        }
         // ---- S = Q K^T: two 8-token halves ----
         float s[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
         {
@@ -231,7 +245,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
         for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
-            const bool ok = (vmask >> (8 * nt + 2 * c + e)) & 1u;
+            const bool ok = ((vmask >> (8 * nt + 2 * c + e)) & 1u) && head_on;
             s[nt][e] = ok ? s[nt][e] * sc : -INFINITY;
             mx = fmaxf(mx, s[nt][e]);
           }
@@ -310,7 +324,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_rows_kernel(
       }
     }
     const int64_t oh = (int64_t)r * d.n_q + qh0 + gg;
-    if (SET == kSetLocal && hm.skips(qh0 + gg)) continue;   // a retrieval head inside a local group: not this call's
+    // (a retrieval head inside a local group is not a local call's; a local head inside a retrieval group not a union call's)
+    if ((SET == kSetLocal || SET == kSetUnion) && hm.skips(qh0 + gg)) continue;
     if (n_splits == 1) {
       out[oh * kHeadDim + dim] = __float2bfloat16_rn(lt > 0.f ? a / lt : 0.f);
       if (lse && dim == 0) lse[oh] = lt > 0.f ? (mt + log2f(lt)) * kLn2 : -INFINITY;
@@ -337,7 +352,7 @@ __global__ void __launch_bounds__(kHeadDim) attn_merge_kernel(const Dims d, cons
   const int64_t r = unit / n_units;
   const int u = unit % n_units;
   const int qh = (SET == kSetList || SET == kSetPages) ? hm.ret_q_head[u] : hm.kv_list[u] * d.group + g;
-  if (SET == kSetLocal && hm.skips(qh)) return;
+  if ((SET == kSetLocal || SET == kSetUnion) && hm.skips(qh)) return;
   const float* p = partial + ((unit * G + g) * (int64_t)n_splits) * kPartial;
   const int dim = threadIdx.x;
   float mt = -INFINITY;
@@ -370,7 +385,7 @@ int plan_splits(int64_t units, int64_t max_set, int sm_count, bool round_up) {
 
 int64_t max_set_len(const Dims& d, int set, int64_t sel_stride, int64_t max_len) {
   if (set == kSetList) return sel_stride < max_len ? sel_stride : max_len;
-  if (set == kSetPages) return sel_stride * kPage < max_len ? sel_stride * kPage : (max_len + kPage - 1) / kPage * kPage;
+  if (set == kSetPages || set == kSetUnion) return sel_stride * kPage < max_len ? sel_stride * kPage : (max_len + kPage - 1) / kPage * kPage;
   if (set == kSetLocal) {
     const int64_t w = (int64_t)d.n_sink + d.window;
     return w < max_len ? w : max_len;
@@ -423,6 +438,12 @@ cudaError_t launch_attn_rows(const CacheView& cv, const Dims& d, const HeadMaps&
                               n_splits, status, st)
   if (set == kSetList) RTP_LAUNCH(1, kSetList);
   if (set == kSetPages) RTP_LAUNCH(1, kSetPages);
+  if (set == kSetUnion) {
+    if (G == 1) RTP_LAUNCH(1, kSetUnion);
+    if (G == 2) RTP_LAUNCH(2, kSetUnion);
+    if (G == 4) RTP_LAUNCH(4, kSetUnion);
+    if (G == 8) RTP_LAUNCH(8, kSetUnion);
+  }
   if (set == kSetLocal) {
     if (G == 1) RTP_LAUNCH(1, kSetLocal);
     if (G == 2) RTP_LAUNCH(2, kSetLocal);

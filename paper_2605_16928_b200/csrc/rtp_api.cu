@@ -242,8 +242,9 @@ size_t rtp_workspace_bytes(const rtp_params* params, int64_t rows, int64_t max_s
   const size_t t1 = attn_rows_workspace_bytes(d, rows, d.n_ret, 1, 1024, max_seq_len);
   const size_t t2 = attn_rows_workspace_bytes(d, rows, d.n_kv, d.group, 1024, max_seq_len);
   if (rows <= 4096) {
+    const size_t t3 = t2 + ((block_union_bytes(d, rows, max_seq_len) + 255) & ~(size_t)255);   // block-wise decode
     m = m > t1 ? m : t1;
-    m = m > t2 ? m : t2;
+    m = m > t3 ? m : t3;
   }
   w.take(m);
   return w.off;
@@ -518,9 +519,37 @@ rtp_status rtp_sparse_attn_decode_blocks(rtp_ctx* ctx, const rtp_params* params,
   if (!q || !block_idx || !block_count || !out) return fail(ctx, RTP_ERR_INVALID, "NULL argument");
   if (block_stride <= 0) return fail(ctx, RTP_ERR_INVALID, "block_stride must be positive");
   if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return fail(ctx, RTP_ERR_INVALID, "misaligned pointer");
-  cudaError_t e = launch_attn_rows(cv, d, hm, rows, kSetPages, reinterpret_cast<const __nv_bfloat16*>(q), block_idx,
-                                   block_stride, block_count, reinterpret_cast<__nv_bfloat16*>(out), lse, workspace,
-                                   workspace ? workspace_bytes : 0, max_len, status, ctx->sm_count, st);
+  // With a workspace the pages of a KV head's query heads are merged into one flagged list per (row, KV head) and the
+  // whole group is attended in one pass over that union (Section 3.2: the memory a KV head needs is the union of its
+  // heads' sets): shared pages are read once.  Without one every head gathers its own pages.
+  cudaError_t e;
+  const size_t uni_bytes = block_union_bytes(d, R, max_len);
+  const bool grouped = workspace && workspace_bytes > uni_bytes && (d.group == 1 || d.group == 2 || d.group == 4 || d.group == 8);
+  if (grouped) {
+    bool is_ret[RTP_MAX_Q_HEADS] = {};
+    bool kv_used[32] = {};
+    for (int i = 0; i < d.n_ret; ++i) {
+      is_ret[hm.ret_q_head[i]] = true;
+      kv_used[hm.ret_q_head[i] / d.group] = true;
+    }
+    hm.n_kv_list = 0;
+    for (int kv = 0; kv < d.n_kv; ++kv)
+      if (kv_used[kv]) hm.kv_list[hm.n_kv_list++] = (uint8_t)kv;
+    for (int h = 0; h < d.n_q; ++h)   // the group's heads that are not retrieval heads are computed but not written
+      if (!is_ret[h]) hm.skip_q[h >> 5] |= 1u << (h & 31);
+    int32_t *uni_idx = nullptr, *uni_cnt = nullptr;
+    int64_t uni_stride = 0;
+    e = launch_block_union(cv, d, hm, rows, block_idx, block_stride, block_count, max_len, workspace, &uni_idx, &uni_stride,
+                           &uni_cnt, status, st);
+    if (e == cudaSuccess)
+      e = launch_attn_rows(cv, d, hm, rows, kSetUnion, reinterpret_cast<const __nv_bfloat16*>(q), uni_idx, uni_stride, uni_cnt,
+                           reinterpret_cast<__nv_bfloat16*>(out), lse, reinterpret_cast<char*>(workspace) + uni_bytes,
+                           workspace_bytes - uni_bytes, max_len, status, ctx->sm_count, st);
+  } else {
+    e = launch_attn_rows(cv, d, hm, rows, kSetPages, reinterpret_cast<const __nv_bfloat16*>(q), block_idx, block_stride,
+                         block_count, reinterpret_cast<__nv_bfloat16*>(out), lse, workspace,
+                         workspace ? workspace_bytes : 0, max_len, status, ctx->sm_count, st);
+  }
   return e == cudaSuccess ? RTP_OK : cuda_fail(ctx, e, "rtp_sparse_attn_decode_blocks");
 }
 

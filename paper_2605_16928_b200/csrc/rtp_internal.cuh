@@ -194,7 +194,10 @@ cudaError_t launch_select_chunk(const CacheView& cv, const Dims& d, const HeadMa
                                 int32_t* status, void* ws, size_t ws_bytes, int sm_count, cudaStream_t st);
 
 // kSetPages: like kSetList, but the list holds logical page numbers and every listed page is taken whole
-enum AttnSet { kSetList = 0, kSetLocal = 1, kSetDense = 2, kSetPages = 3 };
+// kSetUnion: one list per (row, KV head): the union of the pages its query heads selected, every entry a page number
+//            (low 24 bits) with one flag bit per query head of the group (bit 24 + g: head g selected the page); the
+//            whole group is attended in one pass over the union (GQA packing), a head sees only its own pages
+enum AttnSet { kSetList = 0, kSetLocal = 1, kSetDense = 2, kSetPages = 3, kSetUnion = 4 };
 size_t attn_rows_workspace_bytes(const Dims& d, int64_t R, int n_units, int group, int sm_count, int64_t max_len);
 cudaError_t launch_attn_rows(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows, int set,
                              const __nv_bfloat16* q, const int32_t* sel_idx, int64_t sel_stride,
@@ -223,6 +226,12 @@ cudaError_t launch_attn_prefill_tc(const CacheView& cv, const Dims& d, const Hea
 // Block-wise top-p of a prefill chunk (Section 3.4): one bit per (row, retrieval head, page).
 size_t select_blocks_workspace_bytes(const Dims& d, const HeadMaps& hm, int64_t R, int64_t max_len, int sm_count);
 size_t select_rows_blocks_workspace_bytes(const Dims& d, int64_t R, int64_t max_len);
+size_t block_union_bytes(const Dims& d, int64_t R, int64_t max_len);
+// Page lists per retrieval head -> one flagged list per (row, KV head of hm.kv_list); ws holds block_union_bytes.
+cudaError_t launch_block_union(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                               const int32_t* blk_idx, int64_t blk_stride, const int32_t* blk_cnt, int64_t max_len,
+                               void* ws, int32_t** uni_idx, int64_t* uni_stride, int32_t** uni_cnt, int32_t* status,
+                               cudaStream_t st);
 cudaError_t launch_select_rows_blocks(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
                                       const __nv_bfloat16* qt, int64_t max_len, int32_t* blk_idx, int64_t blk_stride,
                                       int32_t* sel_count, float* sel_mass, float* sel_thresh, int32_t* sel_tie_last,

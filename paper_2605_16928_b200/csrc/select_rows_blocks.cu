@@ -319,6 +319,90 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
   }
 }
 
+// ---- union of the page lists of a KV head's query heads -------------------------------------------------------------
+// One CTA per (row, KV head).  Every head's list is turned into a bit per page in shared memory; the union is written
+// in increasing page order, each entry = page | (flags << 24), flag bit g = query head g of the group selected the page.
+constexpr int kUniThreads = 256;
+
+__global__ void __launch_bounds__(kUniThreads) blk_union_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
+                                                                const Rows rows, const int32_t* __restrict__ blk_idx,
+                                                                const int64_t blk_stride,
+                                                                const int32_t* __restrict__ blk_cnt,
+                                                                int32_t* __restrict__ uni_idx, const int64_t uni_stride,
+                                                                int32_t* __restrict__ uni_cnt, const int nbw_max,
+                                                                int32_t* status) {
+  chain_wait();
+  extern __shared__ uint32_t uni_bits[];   // [group][nbw_max]
+  __shared__ int w_cnt[kUniThreads / 32];
+  __shared__ int s_base;
+  const int n_units = hm.n_kv_list;
+  const int64_t r = blockIdx.x / n_units;
+  const int u = blockIdx.x % n_units;
+  const int kvh = hm.kv_list[u];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int seq = rows.row_seq(r);
+  int n_keys = rows.row_pos(r) + 1;
+  {
+    const int sl = (seq >= 0 && seq < cv.batch) ? min(cv.seq_lens[seq], cv.max_pages * kPage) : 0;
+    n_keys = max(0, min(n_keys, sl));
+  }
+  const int nb = (n_keys + kPage - 1) >> kPageShift;
+  const int nbw = (nb + 31) >> 5;
+  for (int i = tid; i < d.group * nbw_max; i += kUniThreads) uni_bits[i] = 0u;
+  if (tid == 0) s_base = 0;
+  __syncthreads();
+  for (int i = 0; i < d.n_ret; ++i) {
+    const int qh = hm.ret_q_head[i];
+    if (qh / d.group != kvh) continue;   // uniform
+    const int g = qh % d.group;
+    const int64_t rh = r * d.n_ret + i;
+    const int cnt = max(0, (int)min((int64_t)blk_cnt[rh], blk_stride));
+    for (int j = tid; j < cnt; j += kUniThreads) {
+      const int page = __ldg(blk_idx + rh * blk_stride + j);
+      if ((unsigned)page >= (unsigned)nb) {
+        set_status(status, RTP_ERR_INVALID);   // a page outside the row's causal pages is left out
+        continue;
+      }
+      atomicOr(&uni_bits[g * nbw_max + (page >> 5)], 1u << (page & 31));
+    }
+  }
+  __syncthreads();
+  int32_t* out = uni_idx + (int64_t)blockIdx.x * uni_stride;
+  for (int w0 = 0; w0 < nbw; w0 += kUniThreads) {
+    const int w = w0 + tid;
+    uint32_t any = 0u;
+    if (w < nbw)
+      for (int g = 0; g < d.group; ++g) any |= uni_bits[g * nbw_max + w];
+    const int mine = __popc(any);
+    int inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    if (lane == 31) w_cnt[warp] = inc;
+    __syncthreads();
+    int wbase = 0, tot = 0;
+    for (int k = 0; k < kUniThreads / 32; ++k) {
+      if (k < warp) wbase += w_cnt[k];
+      tot += w_cnt[k];
+    }
+    int pos = s_base + wbase + inc - mine;
+    while (any) {
+      const int b = __ffs(any) - 1;
+      any &= any - 1u;
+      uint32_t flags = 0u;
+      for (int g = 0; g < d.group; ++g) flags |= ((uni_bits[g * nbw_max + w] >> b) & 1u) << g;
+      if (pos < uni_stride) out[pos] = (int32_t)((uint32_t)(w * 32 + b) | (flags << 24));
+      ++pos;
+    }
+    __syncthreads();
+    if (tid == 0) s_base += tot;
+    __syncthreads();
+  }
+  if (tid == 0) uni_cnt[blockIdx.x] = min((int64_t)s_base, uni_stride);
+}
+
 int64_t blocks_padded(int64_t max_len) { return (((max_len + kPage - 1) / kPage) + 3) / 4 * 4; }
 
 int stats_splits(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
@@ -336,6 +420,29 @@ int stats_splits(const Dims& d, int64_t R, int64_t max_len, int sm_count) {
 size_t select_rows_blocks_workspace_bytes(const Dims& d, int64_t R, int64_t max_len) {
   if (R <= 0 || d.n_ret <= 0) return 0;
   return (size_t)R * d.n_ret * blocks_padded(max_len) * sizeof(float2);
+}
+
+size_t block_union_bytes(const Dims& d, int64_t R, int64_t max_len) {
+  if (R <= 0) return 0;
+  return (size_t)R * d.n_kv * (blocks_padded(max_len) + 16) * sizeof(int32_t);
+}
+
+cudaError_t launch_block_union(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,
+                               const int32_t* blk_idx, int64_t blk_stride, const int32_t* blk_cnt, int64_t max_len,
+                               void* ws, int32_t** uni_idx, int64_t* uni_stride, int32_t** uni_cnt, int32_t* status,
+                               cudaStream_t st) {
+  const int64_t units = rows.R * hm.n_kv_list;
+  const int64_t stride = blocks_padded(max_len);
+  int32_t* idx = reinterpret_cast<int32_t*>(ws);
+  int32_t* cnt = idx + units * stride;
+  *uni_idx = idx;
+  *uni_stride = stride;
+  *uni_cnt = cnt;
+  if (units == 0) return cudaSuccess;
+  const int nbw_max = (int)((stride + 31) / 32);
+  (void)launch_chained(blk_union_kernel, dim3((unsigned)units), dim3(kUniThreads), (size_t)d.group * nbw_max * 4, st, cv, d, hm,
+                       rows, blk_idx, blk_stride, blk_cnt, idx, stride, cnt, nbw_max, status);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_select_rows_blocks(const CacheView& cv, const Dims& d, const HeadMaps& hm, const Rows& rows,

@@ -64,11 +64,13 @@ def check_block_rows(dw, sc, sel, p, rows=None):
     return sets
 
 
-def attend_blocks(dw, sel):
+def attend_blocks(dw, sel, per_head=False):
+    """per_head: a workspace too small for the union lists, so that every head gathers its own pages."""
     out = torch.zeros((dw.R, dw.wl.heads.n_q_heads, 128), dtype=torch.bfloat16, device="cuda")
     lse = torch.zeros((dw.R, dw.wl.heads.n_q_heads), dtype=torch.float32, device="cuda")
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda") if per_head else dw.workspace
     rb.rtp_sparse_attn_decode_blocks(dw.ctx, dw.params, dw.cache, dw.q, dw.row_seq, dw.row_pos, sel["idx"], sel["cnt"], out,
-                                     lse, dw.workspace, dw.status)
+                                     lse, ws, dw.status)
     torch.cuda.synchronize()
     return out.float().cpu().numpy(), lse.cpu().numpy()
 
@@ -91,7 +93,11 @@ def _run(wl, p=None, **kw):
     sc = dw.scores()[0]
     sel = select_block_rows(dw)
     sets = check_block_rows(dw, sc, sel, wl.top_p if p is None else p)
-    out, lse = attend_blocks(dw, sel)
+    out, lse = attend_blocks(dw, sel)                       # the group over the union of its heads' pages
+    check_block_attention(dw, sets, out, lse)
+    local = [h for h in range(wl.heads.n_q_heads) if h not in wl.heads.ret_q_heads]
+    assert np.all(out[:, local] == 0), "only retrieval heads are written"
+    out, lse = attend_blocks(dw, sel, per_head=True)        # every head over its own pages
     check_block_attention(dw, sets, out, lse)
     assert dw.status_code() == rb.RTP_OK
     return dw, sel, sets
@@ -120,6 +126,11 @@ def test_ragged_lengths(L):
 
 def test_group_of_eight_query_heads_per_kv_head():
     _run(synth.config_2(L=2600, batch=2, n_q_heads=16, n_kv_heads=2, ret_kv_heads=(0,), window=300))
+
+
+def test_mixed_group_block_decode():
+    """Two of the four query heads of a KV head are retrieval heads: the union pass computes the group and writes two."""
+    _run(synth.config_2(L=3000, batch=2, window=512, ret_per_group=2))
 
 
 def test_on_8bit_index_keys():
