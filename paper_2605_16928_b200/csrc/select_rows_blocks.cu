@@ -100,7 +100,9 @@ __global__ void __launch_bounds__(kThreads, NH4 ? 4 : 3) blk_stats_kernel(const 
 // first, then smaller block) followed by nb_pad floats (l_b by block number).
 constexpr int kHistBins = 1024;           // bins of 1/32 in M - m_b: 32 units; everything deeper shares the last bin
 constexpr float kHistScale = 32.0f;
-constexpr float kFix = 1099511627776.0f;  // 2^40: block masses (at most 64 each, 16384 blocks) summed as integers
+// Block masses (at most 64 each, relative to exp(M)) are summed as integers at 2^24, so that the sums do not depend on
+// the order of the adds: a bin is {sum mod 2^32, carries}, added to with native 32-bit shared-memory atomics.
+constexpr float kFix = 16777216.0f;
 
 __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
     const CacheView cv, const Dims d, const Rows rows, const float2* __restrict__ stats, const int64_t nb_pad,
@@ -110,7 +112,8 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
   extern __shared__ __align__(16) unsigned char blk_smem[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(blk_smem);
   float* lw = reinterpret_cast<float*>(blk_smem + (size_t)np2 * 8);
-  __shared__ unsigned long long hist[kHistBins];
+  __shared__ uint32_t hist2[kHistBins][2];
+  auto hist_at = [&](int b) -> unsigned long long { return ((unsigned long long)hist2[b][1] << 32) | hist2[b][0]; };
   __shared__ unsigned long long w_tot[kSelWarps];
   __shared__ float w_sum[kSelWarps];
   __shared__ uint32_t w_max[kSelWarps];
@@ -151,14 +154,28 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
     }
     return;
   }
-  // M, and the l_b by block number
+  // A thread keeps the pairs of its (at most 16) blocks in registers: all loads are in flight together.  M, and the
+  // l_b by block number for the ordered scan at the end.
+  constexpr int kMine = kMaxBlocksRow / kSelThreads;
+  float m_r[kMine], l_r[kMine];
   uint32_t kmax = 0u;
-  for (int i = tid; i < nb; i += kSelThreads) {
-    const float2 s = __ldcg(st + i);
-    kmax = max(kmax, okey(s.x));
-    lw[i] = s.y;
+#pragma unroll
+  for (int k = 0; k < kMine; ++k) {
+    const int i = tid + k * kSelThreads;
+    float2 s = make_float2(-INFINITY, 0.f);
+    if (i < nb) s = __ldcg(st + i);
+    m_r[k] = s.x;
+    l_r[k] = s.y;
   }
-  for (int i = tid; i < kHistBins; i += kSelThreads) hist[i] = 0ull;
+#pragma unroll
+  for (int k = 0; k < kMine; ++k) {
+    const int i = tid + k * kSelThreads;
+    if (i < nb) {
+      kmax = max(kmax, okey(m_r[k]));
+      lw[i] = l_r[k];
+    }
+  }
+  for (int i = tid; i < 2 * kHistBins; i += kSelThreads) (&hist2[0][0])[i] = 0u;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
   if (lane == 0) w_max[warp] = kmax;
@@ -176,10 +193,13 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
   auto mass_of = [&](float m, float l) -> float { return l * fast_ex2((m - M) * kLog2eB); };                 // relative to exp(M)
   // histogram of block masses, integers: the sums do not depend on the order of the adds
   unsigned long long mine = 0ull;
-  for (int i = tid; i < nb; i += kSelThreads) {
-    const float m = __ldcg(&st[i].x);
-    const unsigned long long q = (unsigned long long)(mass_of(m, lw[i]) * kFix);
-    atomicAdd(&hist[bin_of(m)], q);
+#pragma unroll
+  for (int k = 0; k < kMine; ++k) {
+    if (tid + k * kSelThreads >= nb) continue;
+    const uint32_t q = (uint32_t)(mass_of(m_r[k], l_r[k]) * kFix);   // (below 2^31)
+    uint32_t* acc = hist2[bin_of(m_r[k])];
+    const uint32_t old = atomicAdd(acc, q);
+    if (old + q < old) atomicAdd(acc + 1, 1u);
     mine += q;
   }
 #pragma unroll
@@ -194,7 +214,7 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
   if (warp == 0) {
     constexpr int kPer = kHistBins / 32;
     unsigned long long part = 0ull;
-    for (int j = 0; j < kPer; ++j) part += hist[lane * kPer + j];
+    for (int j = 0; j < kPer; ++j) part += hist_at(lane * kPer + j);
     unsigned long long inc = part;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -205,7 +225,7 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
     int found = kHistBins;
     unsigned long long above = 0ull;
     for (int j = 0; j < kPer; ++j) {
-      const unsigned long long h = hist[lane * kPer + j];
+      const unsigned long long h = hist_at(lane * kPer + j);
       if (found == kHistBins && h && (float)(run + h) / kFix >= target) {
         found = lane * kPer + j;
         above = run;
@@ -218,13 +238,13 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
     if (best == kHistBins) {   // rounding left the target just out of reach: the lowest populated bin
       int last = -1;
       for (int j = 0; j < kPer; ++j)
-        if (hist[lane * kPer + j]) last = lane * kPer + j;
+        if (hist_at(lane * kPer + j)) last = lane * kPer + j;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
       best = last;
       if (last >= lane * kPer && last < (lane + 1) * kPer) {
         unsigned long long a2 = inc - part;
-        for (int j = lane * kPer; j < last; ++j) a2 += hist[j];
+        for (int j = lane * kPer; j < last; ++j) a2 += hist_at(j);
         found = last;
         above = a2;
       }
@@ -238,8 +258,11 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
   const int tbin = s_bin;
   const float above = (float)s_above / kFix;
   // blocks above the bin are selected; those inside it become sort keys
-  for (int i = tid; i < nb; i += kSelThreads) {
-    const float m = __ldcg(&st[i].x);
+#pragma unroll
+  for (int k = 0; k < kMine; ++k) {
+    const int i = tid + k * kSelThreads;
+    if (i >= nb) continue;
+    const float m = m_r[k];
     const int b = bin_of(m);
     if (b < tbin) {
       const int pos = atomicAdd(&s_n_above, 1);
@@ -322,7 +345,8 @@ __global__ void __launch_bounds__(kSelThreads) blk_select_kernel(
 // ---- union of the page lists of a KV head's query heads -------------------------------------------------------------
 // One CTA per (row, KV head).  Every head's list is turned into a bit per page in shared memory; the union is written
 // in increasing page order, each entry = page | (flags << 24), flag bit g = query head g of the group selected the page.
-constexpr int kUniThreads = 256;
+constexpr int kUniThreads = 1024;
+constexpr int kUniLoads = 8;   // list entries a thread has in flight
 
 __global__ void __launch_bounds__(kUniThreads) blk_union_kernel(const CacheView cv, const Dims d, const HeadMaps hm,
                                                                 const Rows rows, const int32_t* __restrict__ blk_idx,
@@ -348,22 +372,43 @@ __global__ void __launch_bounds__(kUniThreads) blk_union_kernel(const CacheView 
   }
   const int nb = (n_keys + kPage - 1) >> kPageShift;
   const int nbw = (nb + 31) >> 5;
+  __shared__ int s_cnt[8];                 // list length of head g of the group (0: not a retrieval head)
+  __shared__ const int32_t* s_lst[8];
   for (int i = tid; i < d.group * nbw_max; i += kUniThreads) uni_bits[i] = 0u;
   if (tid == 0) s_base = 0;
+  if (tid < 8) s_cnt[tid] = 0;
   __syncthreads();
-  for (int i = 0; i < d.n_ret; ++i) {
-    const int qh = hm.ret_q_head[i];
-    if (qh / d.group != kvh) continue;   // uniform
-    const int g = qh % d.group;
-    const int64_t rh = r * d.n_ret + i;
-    const int cnt = max(0, (int)min((int64_t)blk_cnt[rh], blk_stride));
-    for (int j = tid; j < cnt; j += kUniThreads) {
-      const int page = __ldg(blk_idx + rh * blk_stride + j);
-      if ((unsigned)page >= (unsigned)nb) {
-        set_status(status, RTP_ERR_INVALID);   // a page outside the row's causal pages is left out
-        continue;
+  if (tid < d.n_ret) {
+    const int qh = hm.ret_q_head[tid];
+    if (qh / d.group == kvh) {
+      const int64_t rh = r * d.n_ret + tid;
+      s_cnt[qh % d.group] = max(0, (int)min((int64_t)__ldg(blk_cnt + rh), blk_stride));
+      s_lst[qh % d.group] = blk_idx + rh * blk_stride;
+    }
+  }
+  __syncthreads();
+  int max_cnt = 0;
+  for (int g = 0; g < d.group; ++g) max_cnt = max(max_cnt, s_cnt[g]);
+  for (int j0 = tid; j0 < max_cnt; j0 += kUniThreads * kUniLoads) {
+    for (int g = 0; g < d.group; ++g) {   // (the loads of a head are in flight together; heads follow each other closely)
+      const int cnt = s_cnt[g];
+      if (j0 - tid >= cnt) continue;      // uniform
+      const int32_t* lst = s_lst[g];
+      int page[kUniLoads];
+#pragma unroll
+      for (int k = 0; k < kUniLoads; ++k) {
+        const int j = j0 + k * kUniThreads;
+        page[k] = j < cnt ? __ldg(lst + j) : -1;
       }
-      atomicOr(&uni_bits[g * nbw_max + (page >> 5)], 1u << (page & 31));
+#pragma unroll
+      for (int k = 0; k < kUniLoads; ++k) {
+        if (j0 + k * kUniThreads >= cnt) continue;
+        if ((unsigned)page[k] >= (unsigned)nb) {
+          set_status(status, RTP_ERR_INVALID);   // a page outside the row's causal pages is left out
+          continue;
+        }
+        atomicOr(&uni_bits[g * nbw_max + (page[k] >> 5)], 1u << (page[k] & 31));
+      }
     }
   }
   __syncthreads();
