@@ -371,6 +371,10 @@ def bench_c5_sweep(device, iters=10, batches=(1, 4, 16), contexts=(131072, 52428
                 for frac in fracs:
                     data = synth_device.decode_retarget(base, p, frac)
                     path.data, path.params = data, rb.Params.from_workload(data)
+                    # the block-wise selector of Section 3.4 on the same point (64-key pages by log-sum-exp mass)
+                    t_blk = timed(lambda: path.step_blocks(data.q, k_new))
+                    blk_frac = float(path.blk_cnt.float().mean().item()) / ((L + 63) // 64)
+                    blk_mass = float(path.sel_mass.mean().item())
                     t = timed(lambda: path.step(data.q, k_new))
                     cnt = path.sel_cnt.long()
                     # memory sparsity: union of the lists of the query heads that share a KV head
@@ -393,6 +397,8 @@ def bench_c5_sweep(device, iters=10, batches=(1, 4, 16), contexts=(131072, 52428
                                   "selected_fraction": sel_rows / (B * n_ret * L),
                                   "union_fraction_per_kv_head": float(union.mean().item()) / L,
                                   "sparse_step_us": t, "dense_step_us": t_dense, "speedup_vs_dense": t_dense / t,
+                                  "block_topp_step_us": t_blk, "block_topp_selected_block_fraction": blk_frac,
+                                  "block_topp_selected_mass": blk_mass,
                                   "algorithmic_bytes": alg, "sparse_path_gbs": alg / t / 1e3,
                                   "dense_gbs": dense_bytes / t_dense / 1e3, "status": path.status_code()})
             del path, base
@@ -485,12 +491,13 @@ def main():
             table = bench_c5_sweep(device, iters=max(3, args.steps))
             clocks = sampler.stop()
             ref = next(r for r in table if (r["batch"], r["context"], r["top_p"], r["target_fraction"]) == (4, 524288, 0.9, 0.02))
-            hdr = f"{'B':>3} {'context':>8} {'p':>5} {'target':>7} {'selected':>9} {'union':>7} {'sparse us':>10} {'dense us':>10} {'x':>6} {'GB/s':>7}"
+            hdr = f"{'B':>3} {'context':>8} {'p':>5} {'target':>7} {'selected':>9} {'union':>7} {'sparse us':>10} {'dense us':>10} {'x':>6} {'GB/s':>7} {'block us':>9} {'blocks':>7}"
             print(hdr, file=sys.stderr)
             for r in table:
                 print(f"{r['batch']:>3} {r['context']:>8} {r['top_p']:>5} {r['target_fraction']:>7.3f} {r['selected_fraction']:>9.4f} "
                       f"{r['union_fraction_per_kv_head']:>7.4f} {r['sparse_step_us']:>10.1f} {r['dense_step_us']:>10.1f} "
-                      f"{r['speedup_vs_dense']:>6.2f} {r['sparse_path_gbs']:>7.0f}", file=sys.stderr)
+                      f"{r['speedup_vs_dense']:>6.2f} {r['sparse_path_gbs']:>7.0f} {r['block_topp_step_us']:>9.1f} "
+                      f"{r['block_topp_selected_block_fraction']:>7.4f}", file=sys.stderr)
             print(json.dumps({"metric": "decode_step_us", "value": ref["sparse_step_us"], "unit": "us", "n_gpus": 1,
                               "steps": max(3, args.steps), "warmup": 3, "ms_per_step": ref["sparse_step_us"] / 1e3,
                               "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
