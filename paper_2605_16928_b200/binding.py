@@ -21,7 +21,7 @@ _STATUS_NAMES = ["RTP_OK", "RTP_ERR_INVALID", "RTP_ERR_CAPACITY", "RTP_ERR_UNSUP
                  "RTP_ERR_TIMEOUT"]
 
 EXPORTS = [
-    "rtp_version", "rtp_create", "rtp_destroy", "rtp_last_error", "rtp_debug_wait_test", "rtp_workspace_bytes", "rtp_check_status",
+    "rtp_version", "rtp_create", "rtp_destroy", "rtp_last_error", "rtp_debug_wait_test", "rtp_debug_select_path", "rtp_workspace_bytes", "rtp_check_status",
     "rtp_kv_append", "rtp_index_keys", "rtp_index_queries", "rtp_index_score", "rtp_topp_select", "rtp_sparse_attn_decode", "rtp_sparse_attn_decode_static",
     "rtp_sparse_attn_prefill", "rtp_local_attn", "rtp_dense_attn_prefill", "rtp_dense_attn_decode",
     "rtp_block_workspace_bytes", "rtp_topp_select_blocks", "rtp_sparse_attn_prefill_blocks",
@@ -82,6 +82,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.rtp_last_error.argtypes = [vp]
     lib.rtp_debug_wait_test.restype = i32
     lib.rtp_debug_wait_test.argtypes = [vp, i64, i32]
+    lib.rtp_debug_select_path.restype = i32
+    lib.rtp_debug_select_path.argtypes = [vp, i32]
     lib.rtp_workspace_bytes.restype = sz
     lib.rtp_workspace_bytes.argtypes = [PP, i64, i64]
     lib.rtp_check_status.restype = i32
@@ -227,6 +229,11 @@ class Context:
     def _check(self, rc: int, where: str):
         if rc != RTP_OK:
             raise RtpError(rc, where, (self.lib.rtp_last_error(self.h) or b"").decode())
+
+
+def rtp_debug_select_path(ctx: Context, path: int):
+    """0: the decode selection picks its implementation by size; 1: always the general (multi-kernel) path."""
+    ctx._check(ctx.lib.rtp_debug_select_path(ctx.h, int(path)), "rtp_debug_select_path")
 
 
 def rtp_debug_wait_test(ctx: Context, wait_limit_ns: int, drop_first_key_signal: bool):

@@ -11,6 +11,7 @@ struct rtp_ctx {
   int cc_major, cc_minor;
   unsigned long long wait_ns = 2000000000ull;   // limit of the bounded device-side waits
   int wait_test = 0;                            // rtp_debug_wait_test
+  int select_path = 0;                          // rtp_debug_select_path
   std::string last_error;
 };
 
@@ -69,6 +70,7 @@ const char* check_params(const rtp_params* p, Dims* d, HeadMaps* hm) {
   d->sm_scale = p->sm_scale;
   d->wait_ns = 2000000000ull;
   d->wait_test = 0;
+  d->select_path = 0;
   std::memset(hm, 0, sizeof(*hm));
   for (int j = 0; j < p->n_index_heads; ++j) {
     const int kv = p->index_head_kv[j];
@@ -216,6 +218,12 @@ rtp_status rtp_create(rtp_ctx** out_ctx) {
 
 void rtp_destroy(rtp_ctx* ctx) { delete ctx; }
 
+rtp_status rtp_debug_select_path(rtp_ctx* ctx, int32_t path) {
+  if (!ctx || path < 0 || path > 1) return RTP_ERR_INVALID;
+  ctx->select_path = path;
+  return RTP_OK;
+}
+
 const char* rtp_last_error(const rtp_ctx* ctx) { return ctx ? ctx->last_error.c_str() : "no context"; }
 
 rtp_status rtp_debug_wait_test(rtp_ctx* ctx, int64_t wait_limit_ns, int32_t drop_first_key_signal) {
@@ -270,6 +278,7 @@ rtp_status rtp_check_status(rtp_ctx* ctx, const int32_t* status, void* stream) {
   if (const char* m_ = check_params(params, &d, &hm)) return fail(ctx, RTP_ERR_INVALID, m_); \
   d.wait_ns = ctx->wait_ns;                                                       \
   d.wait_test = ctx->wait_test;                                                   \
+  d.select_path = ctx->select_path;                                               \
   if (const char* m_ = check_cache(cache, params, need_kv, need_ikey, &cv)) return fail(ctx, RTP_ERR_INVALID, m_); \
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 

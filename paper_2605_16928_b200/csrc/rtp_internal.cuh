@@ -68,6 +68,7 @@ struct Dims {
   // attention kernel withholds the signal for its first tile (rtp_debug_wait_test)
   unsigned long long wait_ns;
   int32_t wait_test;
+  int32_t select_path;   // decode selection: 0 = one CTA per (row, head) where the context is short enough, 1 = always the general path
 };
 
 // Rows of a call: explicit arrays (decode) or a contiguous chunk of one sequence.

@@ -91,7 +91,9 @@ class DeviceWorkload:
         return sc.cpu().numpy(), mx.cpu().numpy(), sm.cpu().numpy()
 
     # ---- S4
-    def select(self, with_lists: bool = True, chunk: tuple | None = None):
+    def select(self, with_lists: bool = True, chunk: tuple | None = None, general_path: bool = False):
+        """general_path: force the multi-kernel decode selection where the one-CTA path for short contexts would run."""
+        rb.rtp_debug_select_path(self.ctx, 1 if general_path else 0)
         R, n_ret = self.R, self.n_ret
         idx = torch.full((R, n_ret, self.sel_stride), -1, dtype=torch.int32, device=DEV) if with_lists else None
         cnt = torch.full((R, n_ret), -7, dtype=torch.int32, device=DEV)
@@ -106,6 +108,7 @@ class DeviceWorkload:
             rb.rtp_topp_select(self.ctx, self.params, self.cache, self.q, self.w_q, None, None, seq_id, q_start, R,
                                idx, cnt, mass, thr, tie, self.status, self.workspace)
         torch.cuda.synchronize()
+        rb.rtp_debug_select_path(self.ctx, 0)
         self.sel = dict(idx=idx, cnt=cnt, mass=mass, thr=thr, tie=tie)
         return self.sel
 

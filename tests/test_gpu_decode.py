@@ -21,8 +21,15 @@ def _run_decode(wl, sel_stride=None, check_rows=None, dense_heads=(0,)):
     gh.check_index_keys(dw)
     qt = gh.check_queries(dw)
     sc = gh.check_scores(dw, qt, rows=check_rows)
+    # the decode selection has two implementations (one CTA per (row, head) for short contexts, several kernels over
+    # stored scores otherwise): both are checked, and they must agree exactly
+    sel_g = dw.select(general_path=True)
+    gh.check_selection(dw, sc, sel_g, rows=check_rows)
     sel = dw.select()
     stats = gh.check_selection(dw, sc, sel, rows=check_rows)
+    for k in ("cnt", "thr", "tie"):
+        assert torch.equal(sel[k], sel_g[k]), f"the two selection paths disagree on {k}"
+    assert torch.equal(torch.sort(sel["idx"], dim=-1).values, torch.sort(sel_g["idx"], dim=-1).values)
     out, lse = dw.sparse_decode()
     gh.check_sparse_attention(dw, sel, out, lse, rows=check_rows)
     if wl.heads.local_kv_heads:
@@ -145,6 +152,23 @@ def test_dense_cluster_of_near_equal_scores():
     dw, stats = _run_decode(wl, sel_stride=20000)
     c, k_star, n = stats[0]
     assert 8000 <= c <= 12100                                   # about 90 % of the cluster carries 90 % of the mass
+
+
+def test_dense_cluster_in_a_short_context():
+    """The same kind of cluster in a context short enough for the one-CTA selection: 8000 near-equal scores, twice the
+    candidates its finish takes, so its key levels and its tie rule are exercised (and compared with the general path)."""
+    wl = synth.config_1(L=12000, n_needles=4)
+    K = wl.k[0]
+    rng = np.random.default_rng(11)
+    base = K[int(wl.notes["needles"][0]), 0].copy()
+    for n in range(2000, 10000):
+        k = base.copy()
+        dims = rng.integers(0, 128, size=3)
+        k[dims] ^= np.uint16(1)
+        K[n, 0] = k
+    dw, stats = _run_decode(wl, sel_stride=12000)
+    c, k_star, n = stats[0]
+    assert 5000 <= c <= 8100
 
 
 def test_window_larger_than_context_equals_dense():

@@ -21,8 +21,11 @@ def _run(wl, sel_stride=None, rows=None, attention=True, **variant):
     dw.index_all_keys()
     qt = gh.check_queries(dw)
     sc = gh.check_scores(dw, qt, rows=rows)
+    sel_g = dw.select(general_path=True)
+    gh.check_variant_selection(dw, sc, sel_g, rows=rows, **variant)
     sel = dw.select()
     counts = gh.check_variant_selection(dw, sc, sel, rows=rows, **variant)
+    assert torch.equal(sel["cnt"], sel_g["cnt"]), "the two selection paths disagree"
     if attention:
         out, lse = dw.sparse_decode()
         gh.check_sparse_attention(dw, sel, out, lse, rows=rows)
