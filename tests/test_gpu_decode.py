@@ -171,6 +171,20 @@ def test_dense_cluster_in_a_short_context():
     assert 5000 <= c <= 8100
 
 
+@pytest.mark.parametrize("general", [False, True])
+def test_counts_only_selection_matches_the_lists(general):
+    gh = _harness()
+    wl = synth.config_2(L=3000, batch=4, window=512)
+    dw = gh.DeviceWorkload(wl)
+    dw.index_all_keys()
+    a = dw.select(general_path=general)
+    a = {k: (v.clone() if v is not None else None) for k, v in a.items()}
+    b = dw.select(with_lists=False, general_path=general)
+    for k in ("cnt", "mass", "thr", "tie"):
+        assert torch.equal(a[k], b[k]), k
+    assert dw.status_code() == rb.RTP_OK
+
+
 def test_window_larger_than_context_equals_dense():
     gh = _harness()
     wl = synth.config_2(L=900, batch=2, window=4096)
