@@ -173,10 +173,11 @@ const char* rtp_last_error(const rtp_ctx* ctx);
 rtp_status rtp_debug_wait_test(rtp_ctx* ctx, int64_t wait_limit_ns, int32_t drop_first_key_signal);
 
 /* Diagnostic hook for the decode selection (row form of rtp_topp_select).  It has two implementations with the same
- * results: for short contexts (block table of at most 16384 keys, where it is the faster one) and a call of at most
- * 2 x SM count (row, head) pairs, one CTA per pair runs the whole selection on chip; otherwise the general path of
- * several kernels over stored scores runs.  path = 1 forces the general path on this context, path = 0 restores the
- * choice above.  Returns RTP_ERR_INVALID for a NULL context or another value. */
+ * results.  For contexts whose block table holds at most 36864 keys and calls of at most 2 x SM count (row, head) pairs
+ * one CTA per pair keeps the row's scores in shared memory and runs the whole selection on them (up to 8192 keys it
+ * also scores the keys itself; above, one kernel scores for all of them first): it is the faster one there.  Otherwise
+ * the general path of several kernels over stored scores runs.  path = 1 forces the general path on this context,
+ * path = 0 restores the choice above.  Returns RTP_ERR_INVALID for a NULL context or another value. */
 rtp_status rtp_debug_select_path(rtp_ctx* ctx, int32_t path);
 
 /* Bytes of DEVICE workspace that any call below needs for `rows` query rows

@@ -995,14 +995,17 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
 // of its heads' CTAs (they mostly come from the L2 cache).  The arithmetic is that of the general path: the same bin
 // functions, the same resolves (l1_resolve_warp, key_resolve_warp) and the same finish (finalize_core).
 // Measured against the general path (B = 8, call time of the selection): 38 against 60 us at 2K keys, 40 against 62 at 4K,
-// 45 against 56 at 8K, 50 against 56 at 16K, 71 against 59 at 32K (the heads of an index head each score all of its keys,
-// and 1024 threads do what 256 CTAs share in the general path): used up to 16K keys.
-constexpr int kSmallMaxKeys = 16384;   // 64 KB of scores beside the two candidate buffers of the finish (64 KB)
+// 45 against 56 at 8K; with its own scan 50 against 56 at 16K and 71 against 59 at 32K (the heads of an index head each
+// score all of its keys); with the scan shared (SCAN = false) 43 against 56 at 16K and 54 against 59 at 32K.
+constexpr int kSmallMaxKeys = 8192;    // own scan: 32 KB of scores beside the two candidate buffers of the finish (64 KB)
+constexpr int kMidMaxKeys = 36864;     // with stored scores: 144 KB of them in shared memory
 
-template <bool NH4, bool F8>
+// SCAN = false: the scores were stored by sel_score_kernel (all SMs share the scan); the CTA copies its row into shared
+// memory instead of scoring it (used between 8K and 36K keys, where one CTA's own scan is the slower way).
+template <bool NH4, bool F8, bool SCAN>
 __global__ void __launch_bounds__(kFinThreads) sel_small_kernel(
     const CacheView cv, const Dims d, const HeadMaps hm, const Rows rows, const __nv_bfloat16* __restrict__ qt,
-    int32_t* __restrict__ sel_idx, int64_t sel_stride, int32_t* __restrict__ sel_count, float* __restrict__ sel_mass,
+    const float* __restrict__ stored, const int64_t l_pad, int32_t* __restrict__ sel_idx, int64_t sel_stride, int32_t* __restrict__ sel_count, float* __restrict__ sel_mass,
     float* __restrict__ sel_thresh, int32_t* __restrict__ sel_tie_last, int32_t* status) {
   chain_wait();
   extern __shared__ __align__(16) unsigned char fin_smem[];
@@ -1035,7 +1038,17 @@ __global__ void __launch_bounds__(kFinThreads) sel_small_kernel(
 
   // ---- the scan: a warp scores a page for the index head's heads (MMA) and keeps this head's scores ----
   float mx = -INFINITY;
-  {
+  if (!SCAN) {
+    const float* src = stored + rh * l_pad;
+    for (int n4 = 4 * tid; n4 < n_pages * kPage; n4 += 4 * kFinThreads) {
+      const float4 v = ld_scores4(src + n4);
+      *reinterpret_cast<float4*>(sc + n4) = v;
+      if (n4 < n_keys) mx = fmaxf(mx, v.x);
+      if (n4 + 1 < n_keys) mx = fmaxf(mx, v.y);
+      if (n4 + 2 < n_keys) mx = fmaxf(mx, v.z);
+      if (n4 + 3 < n_keys) mx = fmaxf(mx, v.w);
+    }
+  } else {
     RowCtx x;
     x.r = r; x.ih = ih; x.split = 0; x.seq = seq; x.n_keys = n_keys; x.p_lo = 0; x.p_hi = n_pages; x.nh = nh;
     QFrag qf = load_qfrag(qt + r * d.n_ret * kIndexDim, hm.ih_heads[ih], nh, lane);
@@ -1254,17 +1267,18 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
   const int64_t l_pad = padded_len(max_len);
   int max_nh = 0;
   for (int i = 0; i < d.n_ih; ++i) max_nh = hm.ih_nheads[i] > max_nh ? hm.ih_nheads[i] : max_nh;
-  if (d.select_path != 1 && l_pad <= kSmallMaxKeys && nrh <= 2LL * sm_count) {
+  const bool one_cta = d.select_path != 1 && nrh <= 2LL * sm_count;
+  if (one_cta && l_pad <= kSmallMaxKeys) {
     // short contexts: one CTA per (row, head) does everything on chip
     const int smem = 2 * kCandCap * 8 + (int)l_pad * 4;
     cudaError_t es = cudaSuccess;
 #define RTP_SMALL(NH4_, F8_)                                                                                              \
   {                                                                                                                       \
     static PerDeviceOnce once;                                                                                            \
-    es = set_dyn_smem_once(sel_small_kernel<NH4_, F8_>, 2 * kCandCap * 8 + kSmallMaxKeys * 4, once);                      \
+    es = set_dyn_smem_once(sel_small_kernel<NH4_, F8_, true>, 2 * kCandCap * 8 + kSmallMaxKeys * 4, once);                \
     if (es == cudaSuccess)                                                                                                \
-      (void)launch_chained(sel_small_kernel<NH4_, F8_>, dim3((unsigned)nrh), dim3(kFinThreads), (size_t)smem, st, cv, d, hm, rows, \
-                           qt, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status);               \
+      (void)launch_chained(sel_small_kernel<NH4_, F8_, true>, dim3((unsigned)nrh), dim3(kFinThreads), (size_t)smem, st, cv, d, hm, \
+                           rows, qt, nullptr, l_pad, sel_idx, sel_stride, sel_count, sel_mass, sel_thresh, sel_tie_last, status); \
   }
     if (max_nh <= 4) {
       if (cv.ikey_fp8) RTP_SMALL(true, true) else RTP_SMALL(true, false)
@@ -1277,7 +1291,8 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
   const SelWorkspace w = carve(ws, nrh, rows.R * d.n_ih, l_pad);
   const int list_cap = list_capacity(l_pad);
   cudaError_t e = cudaSuccess;
-  {
+  const bool mid = one_cta && l_pad <= kMidMaxKeys;   // (its last kernel keeps the selection state on chip: nothing to reset)
+  if (!mid) {
     const int64_t n_zero = (int64_t)(w.zero_bytes / 4);
     const int64_t work = n_zero > nrh ? n_zero : nrh;
     const int64_t cap_blocks = (int64_t)sm_count * 8;
@@ -1296,6 +1311,17 @@ cudaError_t launch_select_rows(const CacheView& cv, const Dims& d, const HeadMap
     if (cv.ikey_fp8) RTP_SCORE(false, true); else RTP_SCORE(false, false);
   }
 #undef RTP_SCORE
+  if (mid) {
+    // medium contexts: the scan above is shared by all SMs; one CTA per (row, head) takes its stored scores on chip and
+    // does the rest (the state written by the kernels above is not used)
+    static PerDeviceOnce once;
+    e = set_dyn_smem_once(sel_small_kernel<true, false, false>, 2 * kCandCap * 8 + kMidMaxKeys * 4, once);
+    if (e != cudaSuccess) return e;
+    (void)launch_chained(sel_small_kernel<true, false, false>, dim3((unsigned)nrh), dim3(kFinThreads),
+                         (size_t)(2 * kCandCap * 8 + (int)l_pad * 4), st, cv, d, hm, rows, qt, w.scores, l_pad, sel_idx, sel_stride,
+                         sel_count, sel_mass, sel_thresh, sel_tie_last, status);
+    return cudaGetLastError();
+  }
   (void)launch_chained(sel_l1_kernel, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.tickets, n_splits, list_cap, status);
   (void)launch_chained(sel_key_kernel, dim3(grid), dim3(kThreads), 0, st, cv, d, hm, rows, w.scores, l_pad, w.state, w.g_mass, w.g_cnt, w.tickets,
                                             n_splits, 1 + kKeyLevels, list_cap, status);
