@@ -522,6 +522,18 @@ __global__ void __launch_bounds__(kThreads) sel_key_kernel(const CacheView cv, c
 // for the exact finish.  A CTA takes up to four heads of the unit (blockIdx.z), one after the other; a warp reads 128
 // consecutive stored scores per step and ballots the hits into its two stages in shared memory, which are appended
 // to the row's list / candidate array with one counter update per flush.
+// The float f with  s >= f  <=>  okey(s) >= k  (or okey(s) > k with `above`) for every score s (finite or infinite, never
+// NaN, never -0).  Keys at or below that of -inf give -inf (every score qualifies), keys beyond that of +inf give NaN (none).
+__device__ __forceinline__ float key_floor(uint32_t k, bool above) {
+  if (above) {
+    if (k == 0xffffffffu) return __int_as_float(0x7fc00000);
+    ++k;
+  }
+  if (k <= okey(-INFINITY)) return -INFINITY;
+  if (k > okey(INFINITY)) return __int_as_float(0x7fc00000);
+  return okey_to_float(k);   // (for k = key of +0 this is +0, for the key of -0 it is -0: both compare as zero)
+}
+
 constexpr int kIdStage = 384;     // a step adds at most 128 entries: flushed when more than 256 are staged
 constexpr int kCandStageW = 256;  // flushed when more than 128 are staged
 
@@ -532,13 +544,13 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
   chain_wait();
   __shared__ int id_stage[kWarps][kIdStage];
   __shared__ uint2 cand_stage[kWarps][kCandStageW];
+  __shared__ int st_fill[kWarps][2];   // entries in the warp's two stages
   const RowCtx x = make_row_ctx(cv, d, hm, rows, n_splits, nullptr);
   const int z = blockIdx.z;
   if (z * kHeadsPerCta >= x.nh || x.p_lo >= x.p_hi) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const KeySpan ks = key_span(x);
   const bool emit_ids = sel_idx != nullptr;
-  const uint32_t lt = (1u << lane) - 1u;
   const int nj = min(kHeadsPerCta, x.nh - z * kHeadsPerCta);
 #pragma unroll 1
   for (int j = 0; j < nj; ++j) {
@@ -548,24 +560,36 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
     const uint32_t lo_key = st->lo_key, hi_key = st->hi_key;
     const bool all = mode == kSelectAll, bucket = mode == kCollect || mode == kTieScan, collect = mode == kCollect;
     const float* row = scores + rh * l_pad;
-    int cnt_i = 0, cnt_c = 0, n_above = 0;   // fills are equal across the warp
-    auto flush_ids = [&]() {
+    // s >= f_above <=> key(s) > hi_key ("above the bucket", or every key); s >= f_lo <=> key(s) >= lo_key
+    const float f_above = all ? -INFINITY : (bucket ? key_floor(hi_key, true) : __int_as_float(0x7fc00000));
+    const float f_lo = collect ? key_floor(lo_key, false) : __int_as_float(0x7fc00000);
+    // Hits are sparse (a few per cent of the keys): a lane that has some reserves room in its warp's stage with one
+    // shared-memory add (the order inside a stage does not matter); the fills live in shared memory.
+    int n_above = 0;
+    if (lane == 0) {
+      st_fill[warp][0] = 0;
+      st_fill[warp][1] = 0;
+    }
+    __syncwarp();
+    auto flush_ids = [&](int cnt_i) {
       int gbase = 0;
       if (lane == 0) gbase = atomicAdd(&st->emit_cnt, cnt_i);
       gbase = __shfl_sync(0xffffffffu, gbase, 0);
       for (int i = lane; i < cnt_i; i += 32)
         if (gbase + i < sel_stride) sel_idx[rh * sel_stride + gbase + i] = id_stage[warp][i];
       if (gbase + cnt_i > sel_stride && lane == 0) set_status(status, RTP_ERR_CAPACITY);
-      cnt_i = 0;
+      __syncwarp();
+      if (lane == 0) st_fill[warp][0] = 0;
       __syncwarp();
     };
-    auto flush_cands = [&]() {
+    auto flush_cands = [&](int cnt_c) {
       int gbase = 0;
       if (lane == 0) gbase = atomicAdd(&st->cand_cnt, cnt_c);
       gbase = __shfl_sync(0xffffffffu, gbase, 0);
       for (int i = lane; i < cnt_c; i += 32)
         if (gbase + i < list_cap) cand[rh * (int64_t)list_cap + gbase + i] = cand_stage[warp][i];
-      cnt_c = 0;
+      __syncwarp();
+      if (lane == 0) st_fill[warp][1] = 0;
       __syncwarp();
     };
     for (int nw = ks.k_lo + 128 * warp; nw < ks.k_hi; nw += 128 * kWarps) {
@@ -573,28 +597,37 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
       if (n0 < ks.k_hi) v = ld_scores4(row + n0);
       const float s4[4] = {v.x, v.y, v.z, v.w};
+      uint32_t a_bits = 0u, c_bits = 0u;
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
+        // float comparisons against the bucket's ends (key_floor): one instruction each instead of an ordered key
         const bool ok = n0 + e < ks.k_hi;
-        const uint32_t key = okey(s4[e]);
-        const bool fa = ok && (all || (bucket && key > hi_key));
-        const bool fc = ok && collect && key >= lo_key && key <= hi_key;
-        n_above += (int)fa;
-        if (emit_ids) {
-          const uint32_t ma = __ballot_sync(0xffffffffu, fa);
-          if (fa) id_stage[warp][cnt_i + __popc(ma & lt)] = n0 + e;
-          cnt_i += __popc(ma);
-        }
-        const uint32_t mc = __ballot_sync(0xffffffffu, fc);
-        if (fc) cand_stage[warp][cnt_c + __popc(mc & lt)] = make_uint2(key, (uint32_t)(n0 + e));
-        cnt_c += __popc(mc);
+        const bool fa = ok && s4[e] >= f_above;
+        const bool fc = ok && s4[e] >= f_lo && !(s4[e] >= f_above);
+        a_bits |= (uint32_t)fa << e;
+        c_bits |= (uint32_t)fc << e;
+      }
+      n_above += __popc(a_bits);
+      if (emit_ids && a_bits) {
+        int at = atomicAdd(&st_fill[warp][0], __popc(a_bits));
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if ((a_bits >> e) & 1u) id_stage[warp][at++] = n0 + e;
+      }
+      if (c_bits) {
+        int at = atomicAdd(&st_fill[warp][1], __popc(c_bits));
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if ((c_bits >> e) & 1u) cand_stage[warp][at++] = make_uint2(okey(s4[e]), (uint32_t)(n0 + e));
       }
       __syncwarp();
-      if (cnt_i > kIdStage - 128) flush_ids();
-      if (cnt_c > kCandStageW - 128) flush_cands();
+      const int cnt_i = st_fill[warp][0], cnt_c = st_fill[warp][1];
+      if (cnt_i > kIdStage - 128) flush_ids(cnt_i);
+      if (cnt_c > kCandStageW - 128) flush_cands(cnt_c);
     }
-    if (cnt_i > 0) flush_ids();
-    if (cnt_c > 0) flush_cands();
+    __syncwarp();
+    if (st_fill[warp][0] > 0) flush_ids(st_fill[warp][0]);
+    if (st_fill[warp][1] > 0) flush_cands(st_fill[warp][1]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) n_above += __shfl_xor_sync(0xffffffffu, n_above, o);
     if (lane == 0 && n_above && !all) atomicAdd(&st->cnt_above, n_above);
