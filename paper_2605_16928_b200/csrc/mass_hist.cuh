@@ -16,19 +16,28 @@ constexpr float kLog2eH = 1.4426950408889634f;
 // least kMinQ, which bounds the number of keys of a bin by its sum.
 constexpr float kMinQ = 634880.0f;        // (floor(e^-0.5 * 1024) - 1) * 1024
 
-// Level-1 bin of a score: the integer nearest to 2 (M - s), clamped to [0, 63]; bin b holds M - s in
-// [b/2 - 1/4, b/2 + 1/4] (the last bin pools everything below).  Adding 1.5 * 2^23 leaves that integer in the low
-// mantissa bits, so no float <-> int conversion instruction is needed; the same arithmetic serves the histogram
-// pass and the bisection that turns a bin into a key interval.
+// Level-1 bin of a score.  M is an INTEGER not below any score of the row (the row maximum rounded up), so the bins
+// lie on a grid that does not depend on M: with g(s) = the integer nearest to -2 s (ties to even), the bin is
+// 2 M + g(s), clamped to 63; bin b holds M - s in [b/2 - 1/4, b/2 + 1/4] and the last bin pools everything below.
+// Two histograms of the same row taken against different integers M, M' therefore differ by a shift of 2 (M' - M)
+// bins exactly, whatever the rounding of s: partial histograms can be taken before the row maximum is known.
+// Adding 1.5 * 2^23 leaves g(s) in the low mantissa bits, so no float <-> int conversion instruction is needed; the
+// same arithmetic serves the histogram pass and the search that turns a bin into a key interval.
 constexpr float kMagic = 12582912.0f;     // 1.5 * 2^23
-// (s <= M for every score of the row, so only the upper clamp is needed; the mask keeps the index in range whatever
-// the inputs.)
+constexpr float kL1MaxAbs = 262144.0f;    // |M| must stay below 2^18: then every step below is exact
+// g(s) (scores far below any supported M are clamped first: they fall into the pooled bin either way)
+__device__ __forceinline__ float l1_grid(float s) { return fmaf(fmaxf(s, -4.0f * kL1MaxAbs), -kL1Scale, kMagic) - kMagic; }
 __device__ __forceinline__ int l1_bin_f(float M, float s, float& bin_f) {
-  const float u = fminf(fmaf(s, -kL1Scale, kL1Scale * M), (float)(kBins - 1));
-  const float t = u + kMagic;
+  const float t = fminf(fmaf(kL1Scale, M, l1_grid(s)), (float)(kBins - 1)) + kMagic;
   bin_f = t - kMagic;
   return __float_as_int(t) & (kBins - 1);
 }
+// The integer reference of a row whose largest score is m (kept inside the range in which l1_bin_f is exact; a row
+// beyond it is refused when it is resolved).
+__device__ __forceinline__ float l1_anchor(float m) {
+  return fminf(fmaxf(ceilf(m), -2.0f * kL1MaxAbs), 2.0f * kL1MaxAbs) + 0.0f;
+}
+
 __device__ __forceinline__ int l1_bin(float M, float s) {
   float f;
   return l1_bin_f(M, s, f);

@@ -133,8 +133,9 @@ __global__ void __launch_bounds__(kThreads) sel_score_kernel(const CacheView cv,
   if (threadIdx.x < x.nh) {
     float m = -INFINITY;
     for (int w = 0; w < kWarps; ++w) m = fmaxf(m, s_max[w][threadIdx.x]);
-    // the maximum was taken on unscaled MMA outputs; scaling by a positive factor is monotone
-    if (m > -INFINITY) atomicMax(&state[x.r * d.n_ret + hm.ih_heads[x.ih][threadIdx.x]].max_key, okey(finish_score(m, d.score_scale)));
+    // the maximum was taken on unscaled MMA outputs; scaling by a positive factor is monotone.  What the later passes
+    // need is a reference not below any score, an integer (see l1_bin_f): the maximum rounded up
+    if (m > -INFINITY) atomicMax(&state[x.r * d.n_ret + hm.ih_heads[x.ih][threadIdx.x]].max_key, okey(l1_anchor(finish_score(m, d.score_scale))));
   }
 }
 
@@ -165,6 +166,13 @@ __device__ __forceinline__ void l1_resolve_warp(const Dims& d, const float M, co
                                                 const bool has0, const bool has1, const int lane, const int list_cap,
                                                 SelState* st, int32_t* status) {
   const bool by_count = d.top_k > 0;
+  if (!(fabsf(M) < kL1MaxAbs)) {   // scores beyond the supported range (or not finite): every key is kept
+    if (lane == 0) {
+      st->mode = kSelectAll;
+      set_status(status, RTP_ERR_UNSUPPORTED);
+    }
+    return;
+  }
   const int b0 = 2 * lane, b1 = 2 * lane + 1;
   const float m0 = q0 * (by_count ? kCountScale : l1_bin_scale(b0)), m1 = q1 * (by_count ? kCountScale : l1_bin_scale(b1));
   float inc = m0 + m1;
@@ -1132,7 +1140,7 @@ __global__ void __launch_bounds__(kFinThreads) sel_small_kernel(
   __syncthreads();
   uint32_t kmax = 0u;
   for (int w = 0; w < kFinWarps; ++w) kmax = max(kmax, w_key[w]);
-  const float M = okey_to_float(kmax);
+  const float M = l1_anchor(okey_to_float(kmax));   // the reference of the histograms: the maximum rounded up
 
   if (s_st.mode == kRefine) {   // (uniform)
     // ---- level 1: mass histogram over M - s, one private copy per warp (2^17 fixed point, no wait per add) ----
