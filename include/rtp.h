@@ -154,6 +154,10 @@ typedef struct rtp_cache {
 /* Library version, major*10000 + minor*100 + patch.  (No counterpart in the paper.) */
 int32_t rtp_version(void);
 
+/* Size in bytes of the two argument blocks as this library was compiled (what = 0: rtp_params, 1: rtp_cache; 0 for any
+ * other value).  A binding that lays the blocks out itself compares them with its own before the first call. */
+size_t rtp_struct_bytes(int32_t what);
+
 /* Creates a context for the current CUDA device.  Returns RTP_ERR_CUDA when no
  * usable sm_100 device is current.  (No counterpart in the paper.) */
 rtp_status rtp_create(rtp_ctx** out_ctx);

@@ -21,7 +21,7 @@ _STATUS_NAMES = ["RTP_OK", "RTP_ERR_INVALID", "RTP_ERR_CAPACITY", "RTP_ERR_UNSUP
                  "RTP_ERR_TIMEOUT"]
 
 EXPORTS = [
-    "rtp_version", "rtp_create", "rtp_destroy", "rtp_last_error", "rtp_debug_wait_test", "rtp_debug_select_path", "rtp_workspace_bytes", "rtp_check_status",
+    "rtp_version", "rtp_struct_bytes", "rtp_create", "rtp_destroy", "rtp_last_error", "rtp_debug_wait_test", "rtp_debug_select_path", "rtp_workspace_bytes", "rtp_check_status",
     "rtp_kv_append", "rtp_index_keys", "rtp_index_queries", "rtp_index_score", "rtp_topp_select", "rtp_sparse_attn_decode", "rtp_sparse_attn_decode_static",
     "rtp_sparse_attn_prefill", "rtp_local_attn", "rtp_dense_attn_prefill", "rtp_dense_attn_decode",
     "rtp_block_workspace_bytes", "rtp_topp_select_blocks", "rtp_sparse_attn_prefill_blocks",
@@ -74,6 +74,11 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     PP, PC = C.POINTER(RtpParams), C.POINTER(RtpCache)
     lib.rtp_version.restype = i32
     lib.rtp_version.argtypes = []
+    lib.rtp_struct_bytes.restype = sz
+    lib.rtp_struct_bytes.argtypes = [i32]
+    if lib.rtp_struct_bytes(0) != C.sizeof(RtpParams) or lib.rtp_struct_bytes(1) != C.sizeof(RtpCache):
+        raise RtpError(RTP_ERR_INVALID, "load_library",
+                       "the binding's argument blocks do not have the library's layout (rebuild the library)")
     lib.rtp_create.restype = i32
     lib.rtp_create.argtypes = [C.POINTER(vp)]
     lib.rtp_destroy.restype = None

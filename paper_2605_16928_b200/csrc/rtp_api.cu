@@ -197,6 +197,8 @@ extern "C" {
 
 int32_t rtp_version(void) { return 100; }
 
+size_t rtp_struct_bytes(int32_t what) { return what == 0 ? sizeof(rtp_params) : (what == 1 ? sizeof(rtp_cache) : 0); }
+
 rtp_status rtp_create(rtp_ctx** out_ctx) {
   if (!out_ctx) return RTP_ERR_INVALID;
   *out_ctx = nullptr;

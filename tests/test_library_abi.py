@@ -61,6 +61,12 @@ def test_workspace_bytes_and_param_validation(lib):
     assert rb.rtp_workspace_bytes(p, 8, 32768) == 0
 
 
+def test_argument_blocks_have_the_library_layout(lib):
+    assert lib.rtp_struct_bytes(0) == ctypes.sizeof(rb.RtpParams) > 0
+    assert lib.rtp_struct_bytes(1) == ctypes.sizeof(rb.RtpCache) > 0
+    assert lib.rtp_struct_bytes(2) == 0
+
+
 def test_calls_without_context_are_rejected(lib):
     p = _params()
     cache = rb.RtpCache()
