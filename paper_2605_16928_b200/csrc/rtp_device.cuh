@@ -207,18 +207,6 @@ __device__ __forceinline__ unsigned long long warp_search_first(uint32_t a, uint
   return a;
 }
 
-// raw_preimage() with the work spread over a warp (same result).
-__device__ __forceinline__ void raw_preimage_warp(float scale, uint32_t key_lo, uint32_t key_hi, int lane, float& raw_lo,
-                                                  float& raw_hi) {
-  const uint32_t kmin = okey(-3.4028234e38f), kmax = okey(3.4028234e38f);
-  const unsigned long long lo =
-      warp_search_first(kmin, kmax, lane, [&](uint32_t k) { return okey(finish_score(okey_to_float(k), scale)) >= key_lo; });
-  const unsigned long long above =
-      warp_search_first(kmin, kmax, lane, [&](uint32_t k) { return okey(finish_score(okey_to_float(k), scale)) > key_hi; });
-  // lo > kmax: no float reaches key_lo; above == kmin: every float maps above key_hi: the interval is empty either way
-  raw_lo = lo > kmax ? __int_as_float(0x7f800000) : okey_to_float((uint32_t)lo);
-  raw_hi = above == kmin ? -__int_as_float(0x7f800000) : okey_to_float((uint32_t)(above - 1ull));
-}
 
 // Physical page of a block-table entry.  An entry outside [0, num_pages) (a corrupt table) is read as page 0, so that
 // no kernel leaves the caches; kernels that have a status word also record RTP_ERR_INVALID for it.

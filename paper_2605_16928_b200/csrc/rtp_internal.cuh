@@ -93,7 +93,6 @@ struct SelState {
   float Z;               // sum exp(s - M)
   float target;          // mass to reach, relative to M (p * Z * (1 + margin))
   float mass_above;      // mass of keys above the bucket
-  float raw_lo, raw_hi;  // the bucket as an interval of unscaled MMA outputs
   float ref_s;           // key levels: masses are accumulated relative to exp(ref_s - M)
   float e_ref;           // exp(ref_s - M)
   int32_t cnt_above;     // number of keys above the bucket (counted by the compaction pass)

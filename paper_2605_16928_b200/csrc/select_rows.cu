@@ -214,14 +214,12 @@ __device__ __forceinline__ void l1_resolve_warp(const Dims& d, const float M, co
     const float above = __shfl_sync(0xffffffffu, first ? run : run + m0, owner);
     const float q = __shfl_sync(0xffffffffu, first ? q0 : q1, owner);
     uint32_t klo = 0u, khi = 0u;
-    float rlo = 0.f, rhi = 0.f;
     // Top-P: a cut inside the pooled last bin (mass below 1e-13 per key) keeps every key.  The fixed budget counts
     // keys, so its cut can fall there: the bucket is then every key from the bottom up to the pool's upper end.
     const bool pooled = found == kBins - 1 && !by_count;
     if (!pooled) {
       l1_bin_keys_warp(M, found, lane, klo, khi);
       if (found == kBins - 1) klo = 0u;
-      raw_preimage_warp(d.score_scale, klo, khi, lane, rlo, rhi);
     }
     if (lane == 0) {
       st->M = M;
@@ -237,8 +235,6 @@ __device__ __forceinline__ void l1_resolve_warp(const Dims& d, const float M, co
         st->hi_key = khi;
         st->span = span;
         st->shift = max(0, bits - 6);
-        st->raw_lo = rlo;
-        st->raw_hi = rhi;
         st->ref_s = l1_bin_hi(M, found);
         st->e_ref = by_count ? 1.0f : fast_ex2(-kLog2eH * (0.5f * (float)found - 0.25f));
         if (q < 0.999f * kMinQ * (float)list_cap) st->mode = kCollect;   // fewer than list_cap keys in the bin
@@ -386,17 +382,12 @@ __device__ __forceinline__ void key_resolve_warp(const Dims& d, const float q0, 
     const uint32_t ofs = (uint32_t)bin << shift;
     const uint32_t lo_key = st->lo_key + ofs;
     const uint32_t sub_span = min(1u << shift, st->span - ofs);
-    float rlo, rhi;
-    raw_preimage_warp(d.score_scale, lo_key, lo_key + (sub_span - 1u), lane, rlo, rhi);
-    __syncwarp();
     if (lane == 0) {
       st->mass_above = above;
       st->lo_key = lo_key;
       st->hi_key = lo_key + (sub_span - 1u);
       st->span = sub_span;
       st->bucket_cnt = (int)cnt;
-      st->raw_lo = rlo;
-      st->raw_hi = rhi;
       st->shift = max(0, shift - 6);
       if (cnt <= (uint32_t)list_cap)
         st->mode = kCollect;
@@ -873,7 +864,21 @@ __device__ void finalize_core(const Dims& d, const float* row, SelState* st, con
       s_pick_mass = 0.f;
     }
     __syncthreads();
-    // bitonic sort, ascending: larger score first, then smaller position
+    // ascending order = larger score first, then smaller position.  A short list (the usual case after the narrowing) is
+    // sorted by rank: every candidate counts the smaller ones (the keys are distinct: they hold the position) and goes to
+    // that place of the other buffer, with one barrier; a long one (many equal scores) by a bitonic network.
+    if (n <= 1024) {
+      if (tid < n) {
+        const unsigned long long k = keys[tid];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += keys[j] < k;
+        keys2[tid < n ? rank : 0] = k;
+      }
+      __syncthreads();
+      unsigned long long* t = keys;
+      keys = keys2;
+      keys2 = t;
+    } else
     for (int size = 2; size <= np; size <<= 1) {
       for (int stride = size >> 1; stride > 0; stride >>= 1) {
         for (int i = tid; i < (np >> 1); i += kFinThreads) {
