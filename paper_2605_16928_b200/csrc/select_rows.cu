@@ -1040,9 +1040,9 @@ __global__ void __launch_bounds__(kFinThreads) sel_finalize_kernel(
 // launch instead of six, no pass over global memory after the scan.  The index keys of an index head are read by each
 // of its heads' CTAs (they mostly come from the L2 cache).  The arithmetic is that of the general path: the same bin
 // functions, the same resolves (l1_resolve_warp, key_resolve_warp) and the same finish (finalize_core).
-// Measured against the general path (B = 8, call time of the selection): 38 against 60 us at 2K keys, 40 against 62 at 4K,
-// 45 against 56 at 8K; with its own scan 50 against 56 at 16K and 71 against 59 at 32K (the heads of an index head each
-// score all of its keys); with the scan shared (SCAN = false) 43 against 56 at 16K and 54 against 59 at 32K.
+// Measured against the general path (B = 8, call time of the selection): 33 against 58 us at 2K keys, 36 against 59 at 4K,
+// 41 against 54 at 8K; with its own scan 50 against 56 at 16K and 71 against 59 at 32K (the heads of an index head each
+// score all of its keys); with the scan shared (SCAN = false) 41 against 55 at 16K and 52 against 57 at 32K.
 constexpr int kSmallMaxKeys = 8192;    // own scan: 32 KB of scores beside the two candidate buffers of the finish (64 KB)
 constexpr int kMidMaxKeys = 36864;     // with stored scores: 144 KB of them in shared memory
 
