@@ -276,11 +276,11 @@ def test_decode_512k_batch4_8bit_index_keys():
     _decode_point(524288, 4, 0.9, 0.05, 4096, [0, 2], e2e=False, ikey_e4m3=True)
 
 
-def test_decode_512k_batch4_block_selection():
-    """Block-wise decode at full size: page lists of sampled sequences against the oracle's block rule on the GPU's
-    scores, attention over the listed pages against the oracle."""
+@pytest.mark.parametrize("L,B,seqs", [(524288, 4, [0, 3]), (1048576, 2, [1])])
+def test_decode_block_selection_full_size(L, B, seqs):
+    """Block-wise decode at full size (one million keys = 16384 blocks is the most a row may have): page lists of sampled
+    sequences against the oracle's block rule on the GPU's scores, attention over the listed pages against the oracle."""
     from paper_2605_16928_b200 import pipeline, synth_device
-    L, B, seqs = 524288, 4, [0, 3]
     data = synth_device.decode_device(L, B, 0.9, 0.05, 4096, name="c5_decode_sweep")
     path = pipeline.DecodePath(data, sel_stride=4096)
     path.build_index_cache()
