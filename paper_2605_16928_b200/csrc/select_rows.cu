@@ -637,6 +637,7 @@ __global__ void __launch_bounds__(kThreads) sel_compact_kernel(
 constexpr int kFinThreads = 1024;
 constexpr int kFinWarps = kFinThreads / 32;
 constexpr int kNoPick = 0x7fffffff;
+constexpr int kFinLoads = 8;   // entries of a candidate list in global memory that a thread has in flight
 
 // The finish of one (row, head), run by a CTA of kFinThreads threads: `row` = the row's scores (global memory, or
 // shared memory in the one-kernel path for short contexts), `st` = its selection state, `gl` = its candidate list in
@@ -750,13 +751,22 @@ __device__ void finalize_core(const Dims& d, const float* row, SelState* st, con
         }
         __syncthreads();
         if (in_global) {
-          for (int i = tid; i < n_src; i += kFinThreads) {
-            const uint32_t key = __ldcg(&gl[i].x);
-            const uint32_t t = key - lo_key;
-            if (t < span) {
-              uint32_t* acc = &fh[t >> shift][0];
-              add_mass(acc, fmaf(okey_to_float(key) - ref_s, lw, 20.0f));
-              atomicAdd(acc + 2, 1u);
+          // (the list entries of a thread are loaded several at a time: one round trip for kFinLoads of them)
+          for (int i0 = tid; i0 < n_src; i0 += kFinThreads * kFinLoads) {
+            uint32_t key[kFinLoads];
+#pragma unroll
+            for (int k = 0; k < kFinLoads; ++k) {
+              const int i = i0 + k * kFinThreads;
+              key[k] = i < n_src ? __ldcg(&gl[i].x) : 0u;
+            }
+#pragma unroll
+            for (int k = 0; k < kFinLoads; ++k) {
+              const uint32_t t = key[k] - lo_key;
+              if (i0 + k * kFinThreads < n_src && t < span) {
+                uint32_t* acc = &fh[t >> shift][0];
+                add_mass(acc, fmaf(okey_to_float(key[k]) - ref_s, lw, 20.0f));
+                atomicAdd(acc + 2, 1u);
+              }
             }
           }
         } else {
@@ -804,16 +814,24 @@ __device__ void finalize_core(const Dims& d, const float* row, SelState* st, con
         const int cnt_bin = (int)fh[bin][2];
         const bool to_smem = in_global && cnt_bin <= kCandCap;
         if (in_global) {
-          for (int i = tid; i < n_src; i += kFinThreads) {
-            const uint2 cnd = __ldcg(&gl[i]);
-            const uint32_t t = cnd.x - lo_key;
-            if (t < span) {
-              const int b = (int)(t >> shift);
-              if (b > bin) {
-                const int pos = atomicAdd(&s_sel, 1);
-                if (ids && emit_base + pos < sel_stride) ids[emit_base + pos] = (int)cnd.y;
-              } else if (b == bin && to_smem) {
-                keys2[atomicAdd(&s_n2, 1)] = ((unsigned long long)(~cnd.x) << 32) | (unsigned long long)cnd.y;
+          for (int i0 = tid; i0 < n_src; i0 += kFinThreads * kFinLoads) {
+            uint2 cnd[kFinLoads];
+#pragma unroll
+            for (int k = 0; k < kFinLoads; ++k) {
+              const int i = i0 + k * kFinThreads;
+              cnd[k] = i < n_src ? __ldcg(&gl[i]) : make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int k = 0; k < kFinLoads; ++k) {
+              const uint32_t t = cnd[k].x - lo_key;
+              if (i0 + k * kFinThreads < n_src && t < span) {
+                const int b = (int)(t >> shift);
+                if (b > bin) {
+                  const int pos = atomicAdd(&s_sel, 1);
+                  if (ids && emit_base + pos < sel_stride) ids[emit_base + pos] = (int)cnd[k].y;
+                } else if (b == bin && to_smem) {
+                  keys2[atomicAdd(&s_n2, 1)] = ((unsigned long long)(~cnd[k].x) << 32) | (unsigned long long)cnd[k].y;
+                }
               }
             }
           }
