@@ -73,3 +73,17 @@ def test_projection_is_the_encoded_fp32_projection():
     # against the bf16 projection: the same value before rounding, so the two caches agree to the coarser step
     yb = orc.bf16_to_f64(orc.index_project(x, w))
     assert np.all(np.abs(orc.e4m3_decode(got) - yb) <= np.maximum(np.abs(y) * (2.0 ** -4 + 2.0 ** -8), 2.0 ** -9))
+
+
+def test_scores_by_hand_on_a_tiny_case():
+    # one query, three keys, written out term by term with exact binary fractions
+    q = orc.f32_to_bf16(np.array([1.0, -0.5, 2.0, 0.25] + [0.0] * 12, dtype=np.float32))
+    keys = np.zeros((3, 16), dtype=np.float64)
+    keys[0, :4] = [1.0, 1.0, 1.0, 1.0]          # 1 - 0.5 + 2 + 0.25 = 2.75
+    keys[1, :4] = [448.0, 0.0, -448.0, 0.0]     # 448 - 896 = -448
+    keys[2, :4] = [2.0 ** -9, 0.0, 0.0, 2.0 ** -6]   # subnormal and smallest normal: 2^-9 + 2^-8
+    codes = orc.e4m3_encode(keys)
+    assert np.array_equal(orc.e4m3_decode(codes), keys)
+    got = orc.index_scores_e4m3(q, codes, 0.5)
+    assert got.dtype == np.float32
+    assert got.tolist() == [1.375, -224.0, 0.5 * (2.0 ** -9 + 2.0 ** -8)]
