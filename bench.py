@@ -515,9 +515,9 @@ def main():
 
     if args.decode_only:
         if rank == 0:
-            dec = [bench_decode_point(device, "c1_sized_decode_b1_4k", 4096, 1, 0.9, 0.05, 2048, False, iters=max(3, args.steps), variants=False),
-                   bench_decode_point(device, "c2_decode_batched_gqa", 32768, 8, 0.95, 0.1, 2048, True, iters=max(3, args.steps), variants=not args.no_variants),
-                   bench_decode_point(device, "c5_decode_b4_512k", 524288, 4, 0.9, 0.05, 4096, False, iters=max(3, args.steps), variants=not args.no_variants)]
+            dec = [bench_decode_point(device, "c2_decode_batched_gqa", 32768, 8, 0.95, 0.1, 2048, True, iters=max(3, args.steps), variants=not args.no_variants),
+                   bench_decode_point(device, "c5_decode_b4_512k", 524288, 4, 0.9, 0.05, 4096, False, iters=max(3, args.steps), variants=not args.no_variants),
+                   bench_decode_point(device, "c1_sized_decode_b1_4k", 4096, 1, 0.9, 0.05, 2048, False, iters=max(3, args.steps), variants=False)]
             print(json.dumps({"decode": dec}))
         return
 
@@ -760,9 +760,9 @@ def main():
             del path, data, out, k_pre
             torch.cuda.empty_cache()
             dec = []
-            dec.append(bench_decode_point(device, "c1_sized_decode_b1_4k", 4096, 1, 0.9, 0.05, 2048, False, variants=False))
             dec.append(bench_decode_point(device, "c2_decode_batched_gqa", 32768, 8, 0.95, 0.1, 2048, True))
             dec.append(bench_decode_point(device, "c5_decode_b4_512k", 524288, 4, 0.9, 0.05, 4096, False))
+            dec.append(bench_decode_point(device, "c1_sized_decode_b1_4k", 4096, 1, 0.9, 0.05, 2048, False, variants=False))
             line["decode"] = dec
     elif "cpu_baseline" not in line:
         line["cpu_baseline"] = None
